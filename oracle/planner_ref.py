@@ -1,0 +1,99 @@
+"""Reference work planner (plain Python integers).  TEST INFRASTRUCTURE.
+
+Independent restatement of the planning rule the CUDA library implements in C++; the
+two share no code and are compared bit for bit.  Only tests, the smoke check and the
+benchmark's CPU baseline leg may import this file.
+
+Where the rule comes from.  The paper removes rollout stragglers by splitting the
+rollout cluster into buckets ordered by capacity, each with its own parallel degree
+taken from {1, 2, 4, 8}, and by sending longer requests to higher degrees (Section 2.3
+"Rollout Optimizations"; Section 4.3: degree set, requests sorted by length, contiguous
+segments, objective = smallest maximum completion time; Section 5: buckets ordered by
+capacity, histogram bins aligned with bucket thresholds).  On one GPU the "workers" are
+the resident thread blocks and the "degree" of a sequence is the number of blocks that
+share its KV range, so:
+
+  * bucket k holds the sequences whose length lies in (C * 2^(k-1), C * 2^k]; bucket 0
+    is (0, C]; the degree of bucket k is 2^k, capped at S_max;
+  * C, the base length, is recomputed for every batch from the total work so that the
+    launch has about `items_per_slot` work items per resident block;
+  * items are issued longest first (the classic greedy rule for the min-max objective).
+
+The paper states no single-GPU rule; this reading is listed among the readings of the
+paper in the design notes.
+
+All arithmetic is integer.  cd(a, b) = ceil(a / b); au(a, b) = cd(a, b) * b;
+p2(x) = least power of two >= x.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+
+@dataclass(frozen=True)
+class PlanParams:
+    n_sm: int = 148
+    ctas_per_sm: int = 2
+    items_per_slot: int = 4
+    chunk_align: int = 256      # A: chunk lengths are multiples of this many tokens
+    min_chunk: int = 512        # C_min
+    max_splits: int = 64        # S_max
+
+
+def cd(a: int, b: int) -> int:
+    return -(-a // b)
+
+
+def au(a: int, b: int) -> int:
+    return cd(a, b) * b
+
+
+def p2(x: int) -> int:
+    r = 1
+    while r < x:
+        r *= 2
+    return r
+
+
+@dataclass
+class Plan:
+    chunk_target: int            # C
+    bucket: list                 # per sequence: log2(split degree), -1 for an empty sequence
+    num_splits: list             # n_b: non-empty chunks of sequence b
+    chunk_len: list              # chunk_b
+    item_offset: list            # exclusive prefix sum of n_b (batch order)
+    items: list                  # sorted work list of (b, j, kv_begin, kv_end)
+    combine: list                # sequences with n_b > 1, batch order
+    empty: list                  # sequences with L_b == 0, batch order
+
+
+def plan(seq_lens, num_kv_heads: int, params: PlanParams = PlanParams()) -> Plan:
+    lens = [int(x) for x in seq_lens]
+    if any(L < 0 for L in lens):
+        raise ValueError("negative sequence length")
+    W = params.n_sm * params.ctas_per_sm
+    T = sum(lens)
+    A = params.chunk_align
+    C = max(params.min_chunk, au(cd(num_kv_heads * T, W * params.items_per_slot), A))
+    bucket, nsplit, chunk = [], [], []
+    for L in lens:
+        if L == 0:
+            bucket.append(-1); nsplit.append(0); chunk.append(0)
+            continue
+        s = min(p2(cd(L, C)), params.max_splits)
+        c = au(cd(L, s), A)
+        bucket.append(s.bit_length() - 1)
+        chunk.append(c)
+        nsplit.append(cd(L, c))
+    offs, run = [], 0
+    for n in nsplit:
+        offs.append(run)
+        run += n
+    items = []
+    for b, L in enumerate(lens):
+        for j in range(nsplit[b]):
+            items.append((b, j, j * chunk[b], min(L, (j + 1) * chunk[b])))
+    items.sort(key=lambda it: (-(it[3] - it[2]), it[0], it[1]))
+    return Plan(C, bucket, nsplit, chunk, offs, items,
+                [b for b, n in enumerate(nsplit) if n > 1],
+                [b for b, L in enumerate(lens) if L == 0])

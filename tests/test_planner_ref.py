@@ -1,0 +1,101 @@
+"""Properties the planning rule must have, checked on the reference planner (plain integers).
+The bucket facts come from the paper: degrees are powers of two like {1,2,4,8} (Section 4.3),
+buckets are ordered by capacity and longer requests go to higher degrees (Sections 2.3, 4.3, 5),
+work is issued longest first for the min-max objective (Section 4.3)."""
+import itertools
+
+import numpy as np
+import pytest
+
+from oracle import planner_ref as P
+from paper_2606_03077_b200 import workloads as W
+
+
+def check_plan(lens, hkv, params):
+    pl = P.plan(lens, hkv, params)
+    A = params.chunk_align
+    assert pl.chunk_target % A == 0 and pl.chunk_target >= params.min_chunk
+    run = 0
+    for b, L in enumerate(lens):
+        assert pl.item_offset[b] == run
+        run += pl.num_splits[b]
+        if L == 0:
+            assert pl.num_splits[b] == 0 and pl.bucket[b] == -1 and pl.chunk_len[b] == 0
+            continue
+        s = 1 << pl.bucket[b]
+        assert 1 <= pl.num_splits[b] <= s <= params.max_splits
+        assert pl.chunk_len[b] % A == 0 and pl.chunk_len[b] % 16 == 0
+        # bucket bins: (C 2^(k-1), C 2^k], except that the top bucket is open-ended
+        C = pl.chunk_target
+        if s < params.max_splits:
+            assert L <= C * s
+        if s > 1:
+            assert L > C * (s // 2)
+        # chunks tile [0, L) exactly
+        mine = sorted((it for it in pl.items if it[0] == b), key=lambda it: it[1])
+        assert [it[1] for it in mine] == list(range(pl.num_splits[b]))
+        pos = 0
+        for (_, j, lo, hi) in mine:
+            assert lo == pos and hi > lo and lo == j * pl.chunk_len[b]
+            pos = hi
+        assert pos == L
+    assert len(pl.items) == run
+    sizes = [it[3] - it[2] for it in pl.items]
+    assert sizes == sorted(sizes, reverse=True)
+    keys = [(-(it[3] - it[2]), it[0], it[1]) for it in pl.items]
+    assert keys == sorted(keys)
+    assert pl.combine == [b for b in range(len(lens)) if pl.num_splits[b] > 1]
+    assert pl.empty == [b for b in range(len(lens)) if lens[b] == 0]
+    # longer never gets a smaller bucket
+    order = np.argsort(lens, kind="stable")
+    bk = [pl.bucket[i] for i in order]
+    assert bk == sorted(bk)
+    return pl
+
+
+def test_exhaustive_small_vectors():
+    prm = P.PlanParams(n_sm=2, ctas_per_sm=1, items_per_slot=2, chunk_align=16, min_chunk=16, max_splits=4)
+    n = 0
+    for B in (1, 2, 3):
+        for lens in itertools.product(range(0, 41, 3 if B == 3 else 1), repeat=B):
+            check_plan(list(lens), 1, prm)
+            n += 1
+    assert n > 1000
+
+
+def test_hand_worked_example():
+    # n_sm 2, 1 block each, 2 items per slot, A = 16, C_min = 16, S_max = 4, one KV head
+    # T = 100 + 16 + 40 = 156; C = max(16, au(cd(156, 4), 16)) = au(39, 16) = 48
+    # L=100: cd(100,48)=3 -> p2 = 4 splits; chunk = au(25,16) = 32; n = cd(100,32) = 4
+    # L=16 : 1 split, chunk 16; L=40: 1 split, chunk au(40,16)=48, n = 1
+    prm = P.PlanParams(n_sm=2, ctas_per_sm=1, items_per_slot=2, chunk_align=16, min_chunk=16, max_splits=4)
+    pl = P.plan([100, 16, 40], 1, prm)
+    assert pl.chunk_target == 48
+    assert pl.bucket == [2, 0, 0] and pl.num_splits == [4, 1, 1] and pl.chunk_len == [32, 16, 48]
+    assert pl.item_offset == [0, 4, 5]
+    assert pl.items == [(2, 0, 0, 40), (0, 0, 0, 32), (0, 1, 32, 64), (0, 2, 64, 96), (1, 0, 0, 16), (0, 3, 96, 100)]
+    assert pl.combine == [0] and pl.empty == []
+
+
+def test_random_vectors_default_params():
+    rng = np.random.default_rng(0)
+    for _ in range(200):
+        B = int(rng.integers(1, 300))
+        lens = np.clip(np.floor(rng.choice([64, 1024, 8192]) * np.exp(rng.normal(size=B))), 0, 40960).astype(int)
+        check_plan(list(lens), int(rng.choice([1, 2, 8])), P.PlanParams())
+
+
+@pytest.mark.parametrize("name,step,C,n_items", [
+    ("tiny", 0, 512, 4), ("lognormal_b64", 0, 768, 158), ("longtail_mix_b256", 0, 8192, 334),
+    ("straggler_b8", 0, 1792, 256), ("shift_b128", 0, 1536, 226), ("shift_b128", 1, 2560, 222),
+    ("shift_b128", 2, 5632, 239)])
+def test_workload_plans(name, step, C, n_items):
+    lay, _ = W.make_layout(name, step)
+    pl = check_plan([int(x) for x in lay.seq_lens], lay.workload.num_kv_heads, P.PlanParams())
+    assert pl.chunk_target == C and len(pl.items) == n_items
+
+
+def test_straggler_is_split_32_ways():
+    lay, _ = W.make_layout("straggler_b8")
+    pl = P.plan(lay.seq_lens, 8)
+    assert set(pl.bucket) == {5} and set(pl.chunk_len) == {1024} and set(pl.num_splits) == {32}
