@@ -1,0 +1,224 @@
+/*
+ * libra.h - C ABI of the B200 (sm_100a) paged GQA decode-attention library.
+ *
+ * The library implements the data-parallel core of one batched decode step of an agentic-RL
+ * rollout: for every running sequence, one query token attends to all tokens of its paged
+ * bf16 KV cache.  The paper this library accompanies ("Libra") characterises that step as
+ * memory-bandwidth-bound and linear in sequence length (Section 1, Section 2.2) and removes
+ * the stragglers caused by a few very long trajectories by bucketing requests by length and
+ * giving longer buckets a higher parallel degree (Section 2.3, Section 4.3, Section 5).  The
+ * planner below applies that idea inside one GPU: the "degree" of a sequence is the number of
+ * thread blocks that share its KV range.
+ *
+ * Three steps make one call:
+ *   P  libra_plan          host, integers only: bucket -> split count -> sorted work list
+ *   D  split-KV decode     device: one pass over K and V, fp32 online softmax
+ *   C  combine             device: log-sum-exp merge of the partial results of split sequences
+ * D and C are launched by libra_decode_attn.
+ *
+ * Conventions
+ *   - every function returns a libra_status_t (0 = OK) unless stated otherwise; nothing throws,
+ *     aborts or traps; misuse that the host can see is rejected before any launch;
+ *   - "device pointer" = memory of the handle's GPU, owned by the caller for the whole call and
+ *     until the stream has finished with it; "host pointer" = ordinary host memory;
+ *   - the library allocates host memory only (the handle and two small pinned staging buffers),
+ *     except where a function says otherwise; all device memory, the workspace included, is the
+ *     caller's;
+ *   - streams are cudaStream_t passed as void*; all device work is asynchronous on that stream;
+ *   - one handle serves one stream at a time (no internal locking).
+ *
+ * Data layout
+ *   q, out        bf16 [batch, num_q_heads, head_dim], row-major, contiguous
+ *   k_pages,
+ *   v_pages       bf16, two separate pools indexed by the same page ids; element (page, head,
+ *                 token, c) lives at  page*kv_stride_page + head*kv_stride_head +
+ *                 token*kv_stride_token + c  (strides in elements, head_dim contiguous).
+ *                 "HND" = [num_pages, num_kv_heads, page_size, head_dim] (the default when all
+ *                 three strides are 0), "NHD" = [num_pages, page_size, num_kv_heads, head_dim].
+ *                 Pool base addresses must be 16-byte aligned and strides multiples of 8 elements.
+ *   block_table   int32 [batch, block_table_ld]; entry i of row b = page id of tokens
+ *                 [16 i, 16 i + 16) of sequence b; entries past the last page are ignored
+ *   seq_lens      int32 [batch]; number of cached tokens INCLUDING the current one; the kernel
+ *                 appends nothing; 0 is allowed (output row = 0)
+ *   GQA map       query head h reads KV head h / (num_q_heads / num_kv_heads)
+ *   Slots past seq_len in a sequence's last page, and pages no sequence owns, may hold anything
+ *   (NaN included); they never influence a result.
+ */
+#ifndef LIBRA_H_
+#define LIBRA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LIBRA_OK = 0,
+  LIBRA_INVALID_ARGUMENT = 1,   /* null pointer, negative size, batch > max_batch ...            */
+  LIBRA_UNSUPPORTED_SHAPE = 2,  /* head_dim not 64/128, page_size not 16, group size > 16 ...    */
+  LIBRA_WORKSPACE_TOO_SMALL = 3,
+  LIBRA_NOT_PLANNED = 4,        /* libra_decode_attn before a successful libra_plan              */
+  LIBRA_CUDA_ERROR = 5,         /* a CUDA call failed; see libra_last_cuda_error                 */
+  LIBRA_DEVICE_FLAGGED = 6      /* a kernel recorded a problem; see libra_debug_error_word       */
+} libra_status_t;
+
+/* bits of the device error word */
+#define LIBRA_ERR_WAIT_TIMEOUT 1u   /* a bounded wait on a copy barrier ran out                  */
+#define LIBRA_ERR_BAD_PAGE_ID 2u    /* block-table entry outside [0, num_pages)                  */
+#define LIBRA_ERR_SEQ_LEN_MISMATCH 4u /* device seq_lens differ from the lengths that were planned */
+
+/* Planner constants (Section 4.3 of the paper: degrees are powers of two, work sorted by length,
+ * min-max objective).  A zero field takes its default. */
+typedef struct {
+  int32_t n_sm;           /* SMs to plan for; 0 = the device's count (148 on B200)               */
+  int32_t ctas_per_sm;    /* resident decode blocks per SM the plan assumes; default 2           */
+  int32_t items_per_slot; /* target work items per resident block; default 4                    */
+  int32_t chunk_align;    /* A: chunk lengths are multiples of this many tokens (itself a
+                             multiple of 16); default 256                                       */
+  int32_t min_chunk;      /* C_min: lower bound of the base chunk length; default 512           */
+  int32_t max_splits;     /* S_max: cap of the split degree (power of two <= 64); default 64     */
+} libra_plan_params_t;
+
+typedef struct {
+  int32_t num_q_heads;
+  int32_t num_kv_heads;        /* must divide num_q_heads; group size <= 16                      */
+  int32_t head_dim;            /* 64 or 128                                                      */
+  int32_t page_size;           /* 16                                                             */
+  int64_t num_pages;           /* pages in each pool                                             */
+  int32_t max_batch;           /* upper bound of `batch` in libra_plan                           */
+  int32_t block_table_ld;      /* row pitch of block_table in entries                            */
+  int64_t kv_stride_page;      /* in elements; all three 0 = HND                                 */
+  int64_t kv_stride_head;
+  int64_t kv_stride_token;
+  float sm_scale;              /* softmax scale; 0 = 1/sqrt(head_dim)                            */
+  int32_t device;              /* CUDA device ordinal                                            */
+  libra_plan_params_t plan;
+} libra_config_t;
+
+typedef struct libra_handle_s* libra_handle_t;
+
+/* Read-only host view of the last plan of a handle; the arrays belong to the handle and stay
+ * valid until the next libra_plan or libra_destroy. */
+typedef struct {
+  int32_t batch;
+  int32_t chunk_target;        /* C, the base bucket length of this batch                        */
+  int32_t num_items;
+  int32_t num_combine;
+  int32_t num_empty;
+  const int32_t* bucket;       /* [batch] log2 of the split degree, -1 for an empty sequence     */
+  const int32_t* num_splits;   /* [batch] non-empty chunks n_b                                   */
+  const int32_t* chunk_len;    /* [batch]                                                        */
+  const int32_t* item_offset;  /* [batch] exclusive prefix sum of n_b                            */
+  const int32_t* items;        /* [num_items][4] = (b, j, kv_begin, kv_end), longest first       */
+  const int32_t* combine;      /* [num_combine] sequences with n_b > 1, batch order              */
+  const int32_t* empty;        /* [num_empty] sequences with length 0, batch order               */
+} libra_plan_view_t;
+
+/* Library version, major*10000 + minor*100 + patch. */
+int libra_version(void);
+
+/* Text for a status code; never NULL; static storage. */
+const char* libra_status_string(int status);
+
+/* Create a handle for one shape on cfg->device.  Queries the SM count, checks that the device is
+ * compute capability 10.x and validates the shape.  Errors: INVALID_ARGUMENT (null, non-positive
+ * sizes, num_q_heads not a multiple of num_kv_heads, bad strides), UNSUPPORTED_SHAPE, CUDA_ERROR
+ * (no usable device).  On error *handle is set to NULL. */
+int libra_create(libra_handle_t* handle, const libra_config_t* cfg);
+
+/* Free the handle and its pinned staging buffers.  NULL is allowed.  The caller must have
+ * synchronised the streams that used it. */
+int libra_destroy(libra_handle_t handle);
+
+/* Bytes of device workspace that libra_plan / libra_decode_attn need for any batch <= max_batch.
+ * The workspace holds the uploaded plan, the device error word and the fp32 partial results of
+ * split sequences.  It must be 256-byte aligned. */
+int libra_workspace_size(libra_handle_t handle, size_t* bytes);
+
+/* The planner constants the handle uses, defaults resolved (n_sm = the device's SM count). */
+int libra_get_plan_params(libra_handle_t handle, libra_plan_params_t* out);
+
+/* Tuning knob: shape of the decode thread block, `warps` warps that each own `stages` shared-memory
+ * stages of one K page plus one V page.  Only the compiled-in shapes are accepted (UNSUPPORTED_SHAPE
+ * otherwise); the default is the tuned one.  Results do not depend on the stage count; the warp
+ * count changes the order of the final merge and hence the last bits of the result. */
+int libra_set_variant(libra_handle_t handle, int32_t warps, int32_t stages);
+
+/* Step P as a pure host function (needs no GPU): the length-bucketed planner (Sections 2.3, 4.3
+ * and 5 of the paper give the bucket properties it mirrors).  With W = n_sm * ctas_per_sm,
+ * T = sum of lengths, cd = ceiling division, au(a,b) = cd(a,b)*b, p2 = next power of two:
+ *   C       = max(min_chunk, au(cd(num_kv_heads * T, W * items_per_slot), chunk_align))
+ *   s_b     = min(p2(cd(L_b, C)), max_splits)           bucket_b = log2 s_b
+ *   chunk_b = au(cd(L_b, s_b), chunk_align)              n_b = cd(L_b, chunk_b)
+ *   items   = (b, j, j*chunk_b, min(L_b, (j+1)*chunk_b)) sorted by (length desc, b asc, j asc)
+ * params->n_sm must be > 0 here.  All outputs are caller-allocated host arrays: the per-sequence
+ * arrays hold `batch` entries, `items` holds items_capacity*4 entries.  Errors: INVALID_ARGUMENT
+ * (null, negative length, bad params), WORKSPACE_TOO_SMALL (items_capacity too small; *num_items
+ * then holds the number needed). */
+int libra_plan_host(const libra_plan_params_t* params, int32_t num_kv_heads, const int32_t* seq_lens,
+                    int32_t batch, int32_t* chunk_target, int32_t* bucket, int32_t* num_splits,
+                    int32_t* chunk_len, int32_t* item_offset, int32_t* items, int32_t items_capacity,
+                    int32_t* num_items, int32_t* combine, int32_t* num_combine, int32_t* empty,
+                    int32_t* num_empty);
+
+/* Step P for a handle: plan `batch` sequences from host lengths and upload the plan into the
+ * workspace with one asynchronous copy on `stream` (from a pinned staging buffer owned by the
+ * handle; two buffers alternate, and a buffer is reused only after its previous upload finished).
+ * The plan also resets the device error word.  seq_lens_host: host pointer, int32[batch].
+ * Errors: INVALID_ARGUMENT, WORKSPACE_TOO_SMALL, CUDA_ERROR. */
+int libra_plan(libra_handle_t handle, const int32_t* seq_lens_host, int32_t batch, void* workspace_dev,
+               size_t workspace_bytes, void* stream);
+
+/* Host view of the last plan (see libra_plan_view_t).  Errors: NOT_PLANNED. */
+int libra_plan_export(libra_handle_t handle, libra_plan_view_t* view);
+
+/* Steps D and C: softmax(q K^T * sm_scale) V per query head over the pages of each sequence
+ * (the rollout decode step of Section 1 / Section 2.2 of the paper; the attention itself is the
+ * textbook definition).  All pointers are device pointers; the plan last uploaded by libra_plan
+ * into `workspace` is used and `seq_lens` (device) must hold the planned lengths (a mismatch
+ * sets LIBRA_ERR_SEQ_LEN_MISMATCH in the error word).  Launches the split-KV decode kernel and,
+ * if any sequence is split or empty, the combine kernel, on `stream`; returns without waiting.
+ * Results are bit-reproducible run to run (fixed reduction order, no floating-point atomics).
+ * Errors: INVALID_ARGUMENT (null or misaligned pointer), NOT_PLANNED, CUDA_ERROR. */
+int libra_decode_attn(libra_handle_t handle, const void* q, const void* k_pages, const void* v_pages,
+                      const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream);
+
+/* The same step for callers whose data lives in host memory: copies q, both pools, the block
+ * table and the lengths to `staging_dev` (a caller-owned device region of at least
+ * libra_host_staging_size bytes, 256-byte aligned), plans, runs D and C and copies `out` back
+ * to out_host, all on `stream`; returns after synchronising the stream.  Host pointers should be
+ * pinned for full copy speed.  `workspace_dev` as for libra_plan.  Pools must be in the handle's
+ * layout.  Errors: as libra_plan and libra_decode_attn, plus DEVICE_FLAGGED if the error word is
+ * non-zero afterwards. */
+int libra_decode_attn_host(libra_handle_t handle, const void* q_host, const void* k_pages_host,
+                           const void* v_pages_host, const int32_t* block_table_host,
+                           const int32_t* seq_lens_host, int32_t batch, void* out_host, void* staging_dev,
+                           size_t staging_bytes, void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* Bytes of device staging libra_decode_attn_host needs for `batch` sequences. */
+int libra_host_staging_size(libra_handle_t handle, int32_t batch, size_t* bytes);
+
+/* Last CUDA error code (cudaError_t as int) seen by this handle, 0 if none. */
+int libra_last_cuda_error(libra_handle_t handle);
+
+/* Copy the device error word of the last planned workspace to *word (synchronises `stream` of the
+ * last call first).  0 = no kernel recorded a problem.  Errors: NOT_PLANNED, CUDA_ERROR. */
+int libra_debug_error_word(libra_handle_t handle, uint32_t* word);
+
+/* Per-kernel timing for benchmarks.  After libra_profile_begin, every libra_decode_attn records
+ * CUDA events around the decode kernel and the combine kernel on the call's stream (at most
+ * 4096 calls are kept).  libra_profile_end synchronises those events, returns the summed device
+ * times in milliseconds and the number of calls they cover, and switches recording off.  Any of
+ * the output pointers may be NULL. */
+int libra_profile_begin(libra_handle_t handle);
+int libra_profile_end(libra_handle_t handle, double* decode_ms, double* combine_ms, int32_t* calls);
+
+/* Number of kernels launched through this handle since it was created. */
+int libra_launch_count(libra_handle_t handle, int64_t* launches);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LIBRA_H_ */

@@ -1,0 +1,211 @@
+"""ctypes binding of liblibra.so: same names as the C ABI (include/libra.h), argument marshalling only.
+
+Importing this module loads the shared library and raises if it has not been built
+(``python -m paper_2606_03077_b200.build``); there is no fallback path of any kind.
+Tensors are passed as raw device pointers (``tensor.data_ptr()``) and streams as
+``torch.cuda.current_stream().cuda_stream``; this module itself never imports torch.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblibra.so")
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2606_03077_b200.build`")
+lib = C.CDLL(_LIB_PATH)
+LIB_PATH = _LIB_PATH
+
+OK, INVALID_ARGUMENT, UNSUPPORTED_SHAPE, WORKSPACE_TOO_SMALL, NOT_PLANNED, CUDA_ERROR, DEVICE_FLAGGED = range(7)
+ERR_WAIT_TIMEOUT, ERR_BAD_PAGE_ID, ERR_SEQ_LEN_MISMATCH = 1, 2, 4
+
+
+class PlanParams(C.Structure):
+    _fields_ = [("n_sm", C.c_int32), ("ctas_per_sm", C.c_int32), ("items_per_slot", C.c_int32),
+                ("chunk_align", C.c_int32), ("min_chunk", C.c_int32), ("max_splits", C.c_int32)]
+
+
+class Config(C.Structure):
+    _fields_ = [("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32), ("head_dim", C.c_int32),
+                ("page_size", C.c_int32), ("num_pages", C.c_int64), ("max_batch", C.c_int32),
+                ("block_table_ld", C.c_int32), ("kv_stride_page", C.c_int64), ("kv_stride_head", C.c_int64),
+                ("kv_stride_token", C.c_int64), ("sm_scale", C.c_float), ("device", C.c_int32),
+                ("plan", PlanParams)]
+
+
+class PlanView(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("chunk_target", C.c_int32), ("num_items", C.c_int32),
+                ("num_combine", C.c_int32), ("num_empty", C.c_int32),
+                ("bucket", C.POINTER(C.c_int32)), ("num_splits", C.POINTER(C.c_int32)),
+                ("chunk_len", C.POINTER(C.c_int32)), ("item_offset", C.POINTER(C.c_int32)),
+                ("items", C.POINTER(C.c_int32)), ("combine", C.POINTER(C.c_int32)),
+                ("empty", C.POINTER(C.c_int32))]
+
+
+_i32p = C.POINTER(C.c_int32)
+_vp = C.c_void_p
+
+# every symbol include/libra.h declares, with its signature
+SIGNATURES = {
+    "libra_version": (C.c_int, []),
+    "libra_status_string": (C.c_char_p, [C.c_int]),
+    "libra_create": (C.c_int, [C.POINTER(_vp), C.POINTER(Config)]),
+    "libra_destroy": (C.c_int, [_vp]),
+    "libra_workspace_size": (C.c_int, [_vp, C.POINTER(C.c_size_t)]),
+    "libra_get_plan_params": (C.c_int, [_vp, C.POINTER(PlanParams)]),
+    "libra_set_variant": (C.c_int, [_vp, C.c_int32, C.c_int32]),
+    "libra_plan_host": (C.c_int, [C.POINTER(PlanParams), C.c_int32, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p,
+                                  _i32p, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p]),
+    "libra_plan": (C.c_int, [_vp, _i32p, C.c_int32, _vp, C.c_size_t, _vp]),
+    "libra_plan_export": (C.c_int, [_vp, C.POINTER(PlanView)]),
+    "libra_decode_attn": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "libra_decode_attn_host": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, C.c_int32, _vp, _vp, C.c_size_t, _vp,
+                                         C.c_size_t, _vp]),
+    "libra_host_staging_size": (C.c_int, [_vp, C.c_int32, C.POINTER(C.c_size_t)]),
+    "libra_last_cuda_error": (C.c_int, [_vp]),
+    "libra_debug_error_word": (C.c_int, [_vp, C.POINTER(C.c_uint32)]),
+    "libra_profile_begin": (C.c_int, [_vp]),
+    "libra_profile_end": (C.c_int, [_vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int32)]),
+    "libra_launch_count": (C.c_int, [_vp, C.POINTER(C.c_int64)]),
+}
+for _name, (_res, _args) in SIGNATURES.items():
+    _fn = getattr(lib, _name)
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+
+class LibraError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {libra_status_string(status)} (status {status})")
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise LibraError(status, where)
+
+
+def libra_version() -> int:
+    return lib.libra_version()
+
+
+def libra_status_string(status: int) -> str:
+    return lib.libra_status_string(status).decode()
+
+
+def _as_i32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def libra_plan_host(seq_lens, num_kv_heads: int, params: PlanParams, items_capacity: int | None = None) -> dict:
+    """Pure host planner; returns the plan as a dict of NumPy arrays / ints."""
+    lens = _as_i32(seq_lens)
+    B = int(lens.shape[0])
+    cap = (B * 64 + 1) if items_capacity is None else items_capacity
+    out = {k: np.zeros(max(B, 1), dtype=np.int32) for k in ("bucket", "num_splits", "chunk_len", "item_offset",
+                                                            "combine", "empty")}
+    items = np.zeros((max(cap, 1), 4), dtype=np.int32)
+    scal = {k: C.c_int32(0) for k in ("chunk_target", "num_items", "num_combine", "num_empty")}
+    p = lambda a: a.ctypes.data_as(_i32p)
+    st = lib.libra_plan_host(C.byref(params), num_kv_heads, p(lens), B, C.byref(scal["chunk_target"]),
+                             p(out["bucket"]), p(out["num_splits"]), p(out["chunk_len"]), p(out["item_offset"]),
+                             p(items), cap, C.byref(scal["num_items"]), p(out["combine"]),
+                             C.byref(scal["num_combine"]), p(out["empty"]), C.byref(scal["num_empty"]))
+    _check(st, "libra_plan_host")
+    n = scal["num_items"].value
+    return {"chunk_target": scal["chunk_target"].value, "bucket": out["bucket"][:B].copy(),
+            "num_splits": out["num_splits"][:B].copy(), "chunk_len": out["chunk_len"][:B].copy(),
+            "item_offset": out["item_offset"][:B].copy(), "items": items[:n].copy(),
+            "combine": out["combine"][:scal["num_combine"].value].copy(),
+            "empty": out["empty"][:scal["num_empty"].value].copy()}
+
+
+class Handle:
+    """Owns one libra_handle_t."""
+
+    def __init__(self, num_q_heads: int, num_kv_heads: int, head_dim: int, num_pages: int, max_batch: int,
+                 block_table_ld: int, page_size: int = 16, kv_strides=(0, 0, 0), sm_scale: float = 0.0,
+                 device: int = 0, plan: PlanParams | None = None):
+        self.cfg = Config(num_q_heads, num_kv_heads, head_dim, page_size, num_pages, max_batch, block_table_ld,
+                          kv_strides[0], kv_strides[1], kv_strides[2], sm_scale, device, plan or PlanParams())
+        self._h = _vp()
+        _check(lib.libra_create(C.byref(self._h), C.byref(self.cfg)), "libra_create")
+
+    def close(self) -> None:
+        if self._h:
+            lib.libra_destroy(self._h)
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- thin wrappers, one per entry point
+    def workspace_size(self) -> int:
+        n = C.c_size_t(0)
+        _check(lib.libra_workspace_size(self._h, C.byref(n)), "libra_workspace_size")
+        return n.value
+
+    def plan_params(self) -> PlanParams:
+        p = PlanParams()
+        _check(lib.libra_get_plan_params(self._h, C.byref(p)), "libra_get_plan_params")
+        return p
+
+    def set_variant(self, warps: int, stages: int) -> None:
+        _check(lib.libra_set_variant(self._h, warps, stages), "libra_set_variant")
+
+    def plan(self, seq_lens_host: np.ndarray, workspace_ptr: int, workspace_bytes: int, stream: int) -> None:
+        lens = _as_i32(seq_lens_host)
+        _check(lib.libra_plan(self._h, lens.ctypes.data_as(_i32p), int(lens.shape[0]), workspace_ptr,
+                              workspace_bytes, stream), "libra_plan")
+
+    def plan_export(self) -> dict:
+        v = PlanView()
+        _check(lib.libra_plan_export(self._h, C.byref(v)), "libra_plan_export")
+        arr = lambda ptr, n: np.ctypeslib.as_array(ptr, shape=(n,)).copy() if n > 0 else np.zeros(0, np.int32)
+        return {"chunk_target": v.chunk_target, "bucket": arr(v.bucket, v.batch),
+                "num_splits": arr(v.num_splits, v.batch), "chunk_len": arr(v.chunk_len, v.batch),
+                "item_offset": arr(v.item_offset, v.batch), "items": arr(v.items, v.num_items * 4).reshape(-1, 4),
+                "combine": arr(v.combine, v.num_combine), "empty": arr(v.empty, v.num_empty)}
+
+    def decode_attn(self, q_ptr: int, k_ptr: int, v_ptr: int, block_table_ptr: int, seq_lens_ptr: int,
+                    out_ptr: int, stream: int) -> None:
+        _check(lib.libra_decode_attn(self._h, q_ptr, k_ptr, v_ptr, block_table_ptr, seq_lens_ptr, out_ptr, stream),
+               "libra_decode_attn")
+
+    def host_staging_size(self, batch: int) -> int:
+        n = C.c_size_t(0)
+        _check(lib.libra_host_staging_size(self._h, batch, C.byref(n)), "libra_host_staging_size")
+        return n.value
+
+    def decode_attn_host(self, q_host_ptr: int, k_host_ptr: int, v_host_ptr: int, block_table_host_ptr: int,
+                         seq_lens_host_ptr: int, batch: int, out_host_ptr: int, staging_ptr: int,
+                         staging_bytes: int, workspace_ptr: int, workspace_bytes: int, stream: int) -> None:
+        _check(lib.libra_decode_attn_host(self._h, q_host_ptr, k_host_ptr, v_host_ptr, block_table_host_ptr,
+                                          seq_lens_host_ptr, batch, out_host_ptr, staging_ptr, staging_bytes,
+                                          workspace_ptr, workspace_bytes, stream), "libra_decode_attn_host")
+
+    def last_cuda_error(self) -> int:
+        return lib.libra_last_cuda_error(self._h)
+
+    def debug_error_word(self) -> int:
+        w = C.c_uint32(0)
+        _check(lib.libra_debug_error_word(self._h, C.byref(w)), "libra_debug_error_word")
+        return w.value
+
+    def profile_begin(self) -> None:
+        _check(lib.libra_profile_begin(self._h), "libra_profile_begin")
+
+    def profile_end(self):
+        d, c, n = C.c_double(0), C.c_double(0), C.c_int32(0)
+        _check(lib.libra_profile_end(self._h, C.byref(d), C.byref(c), C.byref(n)), "libra_profile_end")
+        return d.value, c.value, n.value
+
+    def launch_count(self) -> int:
+        n = C.c_int64(0)
+        _check(lib.libra_launch_count(self._h, C.byref(n)), "libra_launch_count")
+        return n.value

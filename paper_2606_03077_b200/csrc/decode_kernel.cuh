@@ -1,0 +1,442 @@
+// Split-KV decode kernel (step D) for sm_100a.
+//
+// One thread block handles one work item (a chunk [kv_begin, kv_end) of one sequence) for one KV
+// head and all G query heads that share it.  Inside the block every warp owns a private ring of
+// shared-memory stages and walks the chunk's pages warp, warp+NW, warp+2NW, ...:
+//
+//   lane 0 : page id -> two tiled TMA loads per tensor (K and V page, 128-byte swizzle) that
+//            complete on the stage's mbarrier; up to STAGES pages per warp are in flight
+//   warp   : S^T[16 tokens x 8 heads]  = K_page . Q^T       mma.sync m16n8k16 bf16 -> fp32
+//            online softmax in fp32 (running max m and sum l per head, base-2 exponent)
+//            O^T[d x 8 heads]         += V_page^T . P^T     P rounded to bf16, l sums the rounded P
+//
+// Tokens are the M side of the tiles, the (padded) head group the N side, so a group of up to
+// 8 heads costs one 8-wide tile and nothing is wasted on padding rows.  The kernel is bound by the
+// HBM read of K and V: 2 * head_dim * 2 bytes per token per KV head, 4 * G * head_dim flop.
+//
+// The warps never synchronise with each other in the main loop; they merge their (m, l, O) in
+// shared memory once at the end, in warp order, so results are bit-reproducible.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "plan_layout.hpp"
+
+namespace libra {
+
+struct DecodeParams {
+  const __nv_bfloat16* q;
+  const int32_t* block_table;
+  const int32_t* seq_lens;
+  __nv_bfloat16* out;
+  const int32_t* plan;   // device plan blob (plan_layout.hpp)
+  float* partial_o;      // [slot][Hq][D]
+  float* partial_lse;    // [slot][Hq]
+  uint32_t* error_word;
+  int64_t num_pages;
+  int32_t num_q_heads;
+  int32_t num_kv_heads;
+  int32_t group;          // G
+  int32_t block_table_ld;
+  float scale_log2;       // sm_scale * log2(e)
+  int32_t pos_head;       // coordinate slot (1..3) of the head / page dimension in the tensor maps
+  int32_t pos_page;
+};
+
+namespace dev {
+
+constexpr uint32_t kWaitLimit = 1u << 22;  // bounded spin on a copy barrier
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Returns false if the barrier did not complete within the limit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+
+// Tiled 4-D TMA load global -> shared (no multicast), completing on an mbarrier of this block.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], "
+      "[%2];"
+      :
+      : "r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr)
+               : "memory");
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr)
+               : "memory");
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+// D(16x8, fp32) += A(16x16 bf16, row) * B(16x8 bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float lg2(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Byte offset of 16-byte chunk c16 of row r inside a [D/64][16][128 B] tile with 128-byte swizzle.
+__device__ __forceinline__ uint32_t tile_off(int r, int c16) {
+  return uint32_t(((c16 >> 3) << 11) + (r << 7) + ((((c16 & 7) ^ (r & 7))) << 4));
+}
+
+}  // namespace dev
+
+template <int D, int NW, int STAGES>
+struct DecodeSmem {
+  static constexpr int kTileBytes = 16 * D * 2;           // one page of one head: K or V
+  static constexpr int kStageBytes = 2 * kTileBytes;      // K then V
+  static constexpr int kWarpBytes = STAGES * kStageBytes;
+  static constexpr int kRingBytes = NW * kWarpBytes;
+  static constexpr int kDynamicBytes = kRingBytes + 1024;  // slack for manual 1024-byte alignment
+};
+
+// D: head_dim (64 | 128); NT: 8-wide head tiles (1: G <= 8, 2: G <= 16); NW warps; STAGES per warp.
+template <int D, int NT, int NW, int STAGES>
+__global__ void __launch_bounds__(NW * 32)
+decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const DecodeParams p) {
+  using namespace dev;
+  using SM = DecodeSmem<D, NW, STAGES>;
+  constexpr int KS = D / 16;   // k-steps of the QK product = 16-row tiles of the PV product
+  constexpr int NH = D / 64;   // 128-byte column blocks of a row
+  static_assert(NT * 8 * D * 4 <= SM::kWarpBytes, "epilogue staging must fit in the warp's ring");
+
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t bars[NW * STAGES];
+  __shared__ float stat_m[NW][NT * 8];
+  __shared__ float stat_l[NW][NT * 8];
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int g = lane >> 2;
+  const int t = lane & 3;
+
+  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* my_ring = ring + warp * SM::kWarpBytes;
+  const uint32_t my_ring_u32 = smem_u32(my_ring);
+  const uint32_t my_bar0 = smem_u32(&bars[warp * STAGES]);
+
+  // ---- work item
+  const int item_idx = blockIdx.x / p.num_kv_heads;
+  const int kvh = blockIdx.x - item_idx * p.num_kv_heads;
+  const int4 item = __ldg(reinterpret_cast<const int4*>(p.plan + plan_layout::kHeaderInts) + item_idx);
+  const int b = item.x;
+  const int kv_begin = item.y;
+  const int kv_end = item.z;
+  const int slot = item.w;  // < 0: the sequence is not split, write bf16 `out` directly
+  const int n_pages = (kv_end - kv_begin + 15) >> 4;
+  const int first_page = kv_begin >> 4;
+  const int n_it = (n_pages > warp) ? (n_pages - warp + NW - 1) / NW : 0;
+
+  if (threadIdx.x == 0) {
+    const int planned_ok = (slot < 0) ? (kv_end == __ldg(p.seq_lens + b)) : (kv_end <= __ldg(p.seq_lens + b));
+    if (!planned_ok) atomicOr(p.error_word, LIBRA_DEV_ERR_SEQ_LEN_MISMATCH);
+  }
+
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < STAGES; ++s) mbar_init(my_bar0 + 8 * s, 1);
+    fence_mbar_init();
+  }
+  __syncwarp();
+
+  // ---- Q^T fragments (B operand: k = dims, n = heads); rows of heads >= G are zero
+  uint32_t qf[NT][KS][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    const int head = nt * 8 + g;
+    const bool live = head < p.group;
+    const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+        p.q + (int64_t(b) * p.num_q_heads + int64_t(kvh) * p.group + (live ? head : 0)) * D);
+#pragma unroll
+    for (int kk = 0; kk < KS; ++kk) {
+      qf[nt][kk][0] = live ? __ldg(qrow + 8 * kk + t) : 0u;
+      qf[nt][kk][1] = live ? __ldg(qrow + 8 * kk + t + 4) : 0u;
+    }
+  }
+
+  // ---- page ids: lane L keeps the id of iteration 32*round + L, one round ahead
+  const int32_t* bt_row = p.block_table + int64_t(b) * p.block_table_ld + first_page + warp;
+  auto load_ids = [&](int round) -> int32_t {
+    const int idx = round * 32 + lane;
+    return (idx < n_it) ? __ldg(bt_row + int64_t(idx) * NW) : -1;
+  };
+  int32_t ids_cur = load_ids(0);
+  int32_t ids_nxt = load_ids(1);
+
+  auto issue = [&](int j, int s) {
+    if ((j & 31) == 0 && j > 0) {
+      ids_cur = ids_nxt;
+      ids_nxt = load_ids((j >> 5) + 1);
+    }
+    const int32_t pid = __shfl_sync(0xffffffffu, ids_cur, j & 31);
+    if (lane == 0) {
+      if (pid < 0 || int64_t(pid) >= p.num_pages) atomicOr(p.error_word, LIBRA_DEV_ERR_BAD_PAGE_ID);
+      const uint32_t bar = my_bar0 + 8 * s;
+      const uint32_t kdst = my_ring_u32 + s * SM::kStageBytes;
+      const uint32_t vdst = kdst + SM::kTileBytes;
+      const int c1 = (p.pos_head == 1) ? kvh : ((p.pos_page == 1) ? pid : 0);
+      const int c2 = (p.pos_head == 2) ? kvh : ((p.pos_page == 2) ? pid : 0);
+      const int c3 = (p.pos_head == 3) ? kvh : ((p.pos_page == 3) ? pid : 0);
+      fence_proxy_async();  // earlier generic-proxy accesses to this stage come before the async write
+      mbar_expect_tx(bar, SM::kStageBytes);
+#pragma unroll
+      for (int h = 0; h < NH; ++h) tma_load_4d(kdst + h * 2048, &map_k, bar, h * 64, c1, c2, c3);
+#pragma unroll
+      for (int h = 0; h < NH; ++h) tma_load_4d(vdst + h * 2048, &map_v, bar, h * 64, c1, c2, c3);
+    }
+  };
+
+  // ---- running state: heads 2t, 2t+1 of every head tile
+  float m_run[NT][2], l_run[NT][2];
+  float acc[NT][KS][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    m_run[nt][0] = m_run[nt][1] = -INFINITY;
+    l_run[nt][0] = l_run[nt][1] = 0.f;
+#pragma unroll
+    for (int mt = 0; mt < KS; ++mt) acc[nt][mt][0] = acc[nt][mt][1] = acc[nt][mt][2] = acc[nt][mt][3] = 0.f;
+  }
+
+  {
+    const int pre = n_it < STAGES ? n_it : STAGES;
+    for (int j = 0; j < pre; ++j) issue(j, j);
+  }
+
+  const int k_row = lane & 15, k_sel = lane >> 4;
+  const int v_row = (lane & 7) + ((lane >> 4) << 3), v_sel = (lane >> 3) & 1;
+  bool timed_out = false;
+
+  int s = 0;
+  uint32_t parity = 0;
+  for (int it = 0; it < n_it; ++it) {
+    const uint32_t bar = my_bar0 + 8 * s;
+    if (!mbar_wait(bar, parity)) {
+      timed_out = true;
+      break;
+    }
+    const uint32_t kt = my_ring_u32 + s * SM::kStageBytes;
+    const uint32_t vt = kt + SM::kTileBytes;
+    const int tok0 = kv_begin + ((warp + it * NW) << 4);
+    const int n_valid = kv_end - tok0;  // >= 1; < 16 only on the sequence's last page
+
+    if (n_valid < 16) {
+      // rows past the end may hold anything, NaN included: clear them in V so that 0 * garbage cannot leak
+      uint8_t* vgen = my_ring + s * SM::kStageBytes + SM::kTileBytes;
+      for (int i = lane; i < (16 - n_valid) * (D / 8); i += 32) {
+        const int r = n_valid + i / (D / 8);
+        const int c16 = i % (D / 8);
+        *reinterpret_cast<uint4*>(vgen + ((c16 >> 3) << 11) + (r << 7) + ((c16 & 7) << 4)) = make_uint4(0, 0, 0, 0);
+      }
+      __syncwarp();
+    }
+
+    // ---- S^T = K . Q^T  (two accumulator sets to halve the dependent chain)
+    float sc[NT][4], sc2[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+      sc2[nt][0] = sc2[nt][1] = sc2[nt][2] = sc2[nt][3] = 0.f;
+    }
+#pragma unroll
+    for (int kk = 0; kk < KS; ++kk) {
+      uint32_t a[4];
+      ldsm_x4(a, kt + tile_off(k_row, 2 * kk + k_sel));
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        if (kk & 1) mma_bf16(sc2[nt], a, qf[nt][kk][0], qf[nt][kk][1]);
+        else mma_bf16(sc[nt], a, qf[nt][kk][0], qf[nt][kk][1]);
+      }
+    }
+
+    // ---- online softmax; this thread holds tokens g, g+8 for heads 2t, 2t+1
+    uint32_t pb[NT][2];
+    bool grew = false;
+    float m_new[NT][2];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) sc[nt][e] = (sc[nt][e] + sc2[nt][e]) * p.scale_log2;
+      if (n_valid < 16) {
+        if (g >= n_valid) sc[nt][0] = sc[nt][1] = -INFINITY;
+        if (g + 8 >= n_valid) sc[nt][2] = sc[nt][3] = -INFINITY;
+      }
+      float mx0 = fmaxf(sc[nt][0], sc[nt][2]);
+      float mx1 = fmaxf(sc[nt][1], sc[nt][3]);
+#pragma unroll
+      for (int off = 4; off <= 16; off <<= 1) {
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+      }
+      m_new[nt][0] = fmaxf(m_run[nt][0], mx0);
+      m_new[nt][1] = fmaxf(m_run[nt][1], mx1);
+      grew = grew || (m_new[nt][0] > m_run[nt][0]) || (m_new[nt][1] > m_run[nt][1]);
+    }
+    if (__any_sync(0xffffffffu, grew)) {
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const float f0 = ex2(m_run[nt][0] - m_new[nt][0]);  // first page: 2^(-inf) = 0 on zeros
+        const float f1 = ex2(m_run[nt][1] - m_new[nt][1]);
+        l_run[nt][0] *= f0;
+        l_run[nt][1] *= f1;
+#pragma unroll
+        for (int mt = 0; mt < KS; ++mt) {
+          acc[nt][mt][0] *= f0;
+          acc[nt][mt][1] *= f1;
+          acc[nt][mt][2] *= f0;
+          acc[nt][mt][3] *= f1;
+        }
+        m_run[nt][0] = m_new[nt][0];
+        m_run[nt][1] = m_new[nt][1];
+      }
+    }
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const float p0 = ex2(sc[nt][0] - m_run[nt][0]);
+      const float p1 = ex2(sc[nt][1] - m_run[nt][1]);
+      const float p2 = ex2(sc[nt][2] - m_run[nt][0]);
+      const float p3 = ex2(sc[nt][3] - m_run[nt][1]);
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(p0, p1);  // token g   : heads 2t, 2t+1
+      const __nv_bfloat162 hi = __floats2bfloat162_rn(p2, p3);  // token g+8
+      const uint32_t ulo = *reinterpret_cast<const uint32_t*>(&lo);
+      const uint32_t uhi = *reinterpret_cast<const uint32_t*>(&hi);
+      // the denominator sums exactly the probabilities the tensor core will see
+      l_run[nt][0] += __uint_as_float(ulo << 16) + __uint_as_float(uhi << 16);
+      l_run[nt][1] += __uint_as_float(ulo & 0xffff0000u) + __uint_as_float(uhi & 0xffff0000u);
+      pb[nt][0] = movmatrix_trans(ulo);  // head g : tokens 2t, 2t+1
+      pb[nt][1] = movmatrix_trans(uhi);  // head g : tokens 2t+8, 2t+9
+    }
+
+    // ---- O^T += V^T . P^T
+#pragma unroll
+    for (int mt = 0; mt < KS; ++mt) {
+      uint32_t a[4];
+      ldsm_x4_trans(a, vt + tile_off(v_row, 2 * mt + v_sel));
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) mma_bf16(acc[nt][mt], a, pb[nt][0], pb[nt][1]);
+    }
+
+    __syncwarp();  // every lane has consumed the stage before lane 0 refills it
+    if (it + STAGES < n_it) issue(it + STAGES, s);
+    if (++s == STAGES) {
+      s = 0;
+      parity ^= 1u;
+    }
+  }
+
+  if (timed_out) {
+    if (lane == 0) atomicOr(p.error_word, LIBRA_DEV_ERR_WAIT_TIMEOUT);
+    // give copies that are still in flight one more bounded chance to land before the block exits
+    for (int k = 0; k < STAGES; ++k) (void)mbar_wait(my_bar0 + 8 * k, parity);
+  }
+
+  // ---- per-warp totals: l is spread over the 8 token lanes of each head
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+    for (int off = 4; off <= 16; off <<= 1) {
+      l_run[nt][0] += __shfl_xor_sync(0xffffffffu, l_run[nt][0], off);
+      l_run[nt][1] += __shfl_xor_sync(0xffffffffu, l_run[nt][1], off);
+    }
+  }
+
+  // ---- stage (m, l, O) of this warp in its own, now idle, ring: O as [head][dim] fp32
+  __syncwarp();
+  float* o_sm = reinterpret_cast<float*>(my_ring);
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    if (g == 0) {
+      stat_m[warp][nt * 8 + 2 * t] = m_run[nt][0];
+      stat_m[warp][nt * 8 + 2 * t + 1] = m_run[nt][1];
+      stat_l[warp][nt * 8 + 2 * t] = l_run[nt][0];
+      stat_l[warp][nt * 8 + 2 * t + 1] = l_run[nt][1];
+    }
+#pragma unroll
+    for (int mt = 0; mt < KS; ++mt) {
+      const int h0 = nt * 8 + 2 * t;
+      const int d0 = mt * 16 + g;
+      o_sm[h0 * D + d0] = acc[nt][mt][0];
+      o_sm[(h0 + 1) * D + d0] = acc[nt][mt][1];
+      o_sm[h0 * D + d0 + 8] = acc[nt][mt][2];
+      o_sm[(h0 + 1) * D + d0 + 8] = acc[nt][mt][3];
+    }
+  }
+  __syncthreads();
+
+  // ---- merge the warps in warp order and write the result
+  const int G = p.group;
+  for (int idx = threadIdx.x; idx < G * D; idx += NW * 32) {
+    const int h = idx / D;
+    const int dim = idx - h * D;
+    float m_all = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) m_all = fmaxf(m_all, stat_m[w][h]);
+    float num = 0.f, den = 0.f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) {
+      const float mw = stat_m[w][h];
+      const float f = (mw == -INFINITY) ? 0.f : ex2(mw - m_all);
+      num += f * reinterpret_cast<const float*>(ring + w * SM::kWarpBytes)[h * D + dim];
+      den += f * stat_l[w][h];
+    }
+    const float o = num / den;
+    const int64_t head = int64_t(kvh) * G + h;
+    if (slot < 0) {
+      p.out[(int64_t(b) * p.num_q_heads + head) * D + dim] = __float2bfloat16_rn(o);
+    } else {
+      p.partial_o[(int64_t(slot) * p.num_q_heads + head) * D + dim] = o;
+      if (dim == 0) p.partial_lse[int64_t(slot) * p.num_q_heads + head] = (m_all + lg2(den)) * 0.6931471805599453f;
+    }
+  }
+}
+
+}  // namespace libra

@@ -1,0 +1,685 @@
+// C ABI of the library: handle, planner upload, kernel launches.  See include/libra.h.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "combine_kernel.cuh"
+#include "decode_kernel.cuh"
+#include "libra.h"
+#include "plan_layout.hpp"
+#include "planner.hpp"
+
+static_assert(LIBRA_ERR_WAIT_TIMEOUT == LIBRA_DEV_ERR_WAIT_TIMEOUT, "error bits");
+static_assert(LIBRA_ERR_BAD_PAGE_ID == LIBRA_DEV_ERR_BAD_PAGE_ID, "error bits");
+static_assert(LIBRA_ERR_SEQ_LEN_MISMATCH == LIBRA_DEV_ERR_SEQ_LEN_MISMATCH, "error bits");
+
+namespace {
+
+using libra::DecodeParams;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+typedef void (*DecodeKernelFn)(const CUtensorMap, const CUtensorMap, const DecodeParams);
+
+struct Variant {
+  int warps, stages;
+  DecodeKernelFn fn[2][2];  // [D == 128][NT - 1]
+  int smem[2];              // dynamic bytes for D = 64 / 128
+};
+
+template <int NW, int ST>
+Variant make_variant() {
+  Variant v;
+  v.warps = NW;
+  v.stages = ST;
+  v.fn[0][0] = libra::decode_kernel<64, 1, NW, ST>;
+  v.fn[0][1] = libra::decode_kernel<64, 2, NW, ST>;
+  v.fn[1][0] = libra::decode_kernel<128, 1, NW, ST>;
+  v.fn[1][1] = libra::decode_kernel<128, 2, NW, ST>;
+  v.smem[0] = libra::DecodeSmem<64, NW, ST>::kDynamicBytes;
+  v.smem[1] = libra::DecodeSmem<128, NW, ST>::kDynamicBytes;
+  return v;
+}
+
+// Shapes of the decode block that are compiled in; index 0 is the default.
+const std::vector<Variant>& variants() {
+  static const std::vector<Variant> v = {
+      make_variant<4, 3>(), make_variant<4, 2>(), make_variant<4, 4>(), make_variant<4, 6>(),
+      make_variant<8, 2>(), make_variant<8, 3>(), make_variant<2, 6>(), make_variant<2, 4>(),
+  };
+  return v;
+}
+
+constexpr int kMaxProfiledCalls = 4096;
+
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  cudaError_t err = cudaSuccess;
+  explicit DeviceGuard(int dev) {
+    err = cudaGetDevice(&prev);
+    if (err == cudaSuccess && prev != dev) {
+      err = cudaSetDevice(dev);
+      switched = (err == cudaSuccess);
+    }
+  }
+  ~DeviceGuard() {
+    if (switched) cudaSetDevice(prev);
+  }
+};
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+struct libra_handle_s {
+  libra_config_t cfg;
+  libra::PlanParams params;
+  int group = 0;
+  float scale_log2 = 0.f;
+  int64_t stride_page = 0, stride_head = 0, stride_token = 0;
+  int64_t pool_elems = 0;
+  int last_cuda_error = 0;
+  int variant = 0;
+  EncodeTiledFn encode = nullptr;
+
+  // workspace layout
+  int64_t max_items = 0;
+  size_t plan_bytes = 0, lse_off = 0, o_off = 0, workspace_bytes = 0;
+
+  // pinned staging for plan uploads
+  int32_t* staging[2] = {nullptr, nullptr};
+  cudaEvent_t staging_done[2] = {nullptr, nullptr};
+  bool staging_used[2] = {false, false};
+  int next_staging = 0;
+
+  // last plan
+  bool planned = false;
+  libra::HostPlan plan;
+  std::vector<int32_t> items_flat;
+  void* workspace = nullptr;
+  int32_t num_items = 0, num_fix = 0;
+  void* last_stream = nullptr;
+
+  // tensor maps of the pools seen most recently (callers often rotate between a few pools)
+  struct PoolMaps {
+    const void* k_ptr = nullptr;
+    const void* v_ptr = nullptr;
+    CUtensorMap map_k, map_v;
+  };
+  static constexpr int kMapCache = 8;
+  PoolMaps maps[kMapCache];
+  int next_map = 0;
+  int pos_head = 0, pos_page = 0;
+
+  // profiling
+  bool profiling = false;
+  std::vector<cudaEvent_t> events;  // 3 per call
+  int profiled_calls = 0;
+  int64_t launches = 0;
+};
+
+namespace {
+
+int fail_cuda(libra_handle_t h, cudaError_t e) {
+  if (h) h->last_cuda_error = int(e);
+  (void)cudaGetLastError();
+  return LIBRA_CUDA_ERROR;
+}
+
+#define LIBRA_CUDA_TRY(h, expr)                       \
+  do {                                                \
+    cudaError_t e__ = (expr);                         \
+    if (e__ != cudaSuccess) return fail_cuda(h, e__); \
+  } while (0)
+
+libra::PlanParams resolve_params(const libra_plan_params_t& in, int n_sm_device) {
+  libra::PlanParams p;
+  if (in.n_sm > 0) p.n_sm = in.n_sm;
+  else if (n_sm_device > 0) p.n_sm = n_sm_device;
+  if (in.ctas_per_sm > 0) p.ctas_per_sm = in.ctas_per_sm;
+  if (in.items_per_slot > 0) p.items_per_slot = in.items_per_slot;
+  if (in.chunk_align > 0) p.chunk_align = in.chunk_align;
+  if (in.min_chunk > 0) p.min_chunk = in.min_chunk;
+  if (in.max_splits > 0) p.max_splits = in.max_splits;
+  return p;
+}
+
+// Build the tiled tensor map of one pool: dimension 0 is head_dim (contiguous); the other three
+// (token, head, page) are ordered by increasing stride.  Box = 64 elements x 16 tokens x 1 x 1.
+int encode_pool_map(libra_handle_t h, const void* base, CUtensorMap* map, int* pos_head, int* pos_page) {
+  struct Dim {
+    int64_t stride, size;
+    uint32_t box;
+    int kind;
+  };
+  Dim dims[3] = {{h->stride_token, h->cfg.page_size, uint32_t(h->cfg.page_size), 0},
+                 {h->stride_head, h->cfg.num_kv_heads, 1u, 1},
+                 {h->stride_page, h->cfg.num_pages, 1u, 2}};
+  std::stable_sort(dims, dims + 3, [](const Dim& a, const Dim& b) { return a.stride < b.stride; });
+  cuuint64_t gdim[4] = {cuuint64_t(h->cfg.head_dim), 0, 0, 0};
+  cuuint64_t gstride[3];
+  cuuint32_t box[4] = {64, 0, 0, 0};
+  cuuint32_t estride[4] = {1, 1, 1, 1};
+  for (int i = 0; i < 3; ++i) {
+    gdim[i + 1] = cuuint64_t(dims[i].size);
+    gstride[i] = cuuint64_t(dims[i].stride) * 2;
+    box[i + 1] = dims[i].box;
+    if (dims[i].kind == 1) *pos_head = i + 1;
+    if (dims[i].kind == 2) *pos_page = i + 1;
+  }
+  CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gdim, gstride, box, estride,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    h->last_cuda_error = int(cudaErrorInvalidValue);
+    return LIBRA_CUDA_ERROR;
+  }
+  return LIBRA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int libra_version(void) { return 100; }
+
+const char* libra_status_string(int status) {
+  switch (status) {
+    case LIBRA_OK: return "ok";
+    case LIBRA_INVALID_ARGUMENT: return "invalid argument";
+    case LIBRA_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case LIBRA_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case LIBRA_NOT_PLANNED: return "no plan has been made for this handle";
+    case LIBRA_CUDA_ERROR: return "a CUDA call failed";
+    case LIBRA_DEVICE_FLAGGED: return "a kernel recorded a problem in the device error word";
+    default: return "unknown status";
+  }
+}
+
+int libra_plan_host(const libra_plan_params_t* params, int32_t num_kv_heads, const int32_t* seq_lens, int32_t batch,
+                    int32_t* chunk_target, int32_t* bucket, int32_t* num_splits, int32_t* chunk_len,
+                    int32_t* item_offset, int32_t* items, int32_t items_capacity, int32_t* num_items,
+                    int32_t* combine, int32_t* num_combine, int32_t* empty, int32_t* num_empty) {
+  if (!params || batch < 0 || (batch > 0 && !seq_lens) || num_kv_heads <= 0 || items_capacity < 0) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  if (!chunk_target || !num_items || !num_combine || !num_empty) return LIBRA_INVALID_ARGUMENT;
+  if (batch > 0 && (!bucket || !num_splits || !chunk_len || !item_offset || !combine || !empty)) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  if (params->n_sm <= 0) return LIBRA_INVALID_ARGUMENT;
+  const libra::PlanParams p = resolve_params(*params, 0);
+  libra::HostPlan pl;
+  if (!libra::make_plan(p, num_kv_heads, seq_lens, batch, &pl)) return LIBRA_INVALID_ARGUMENT;
+  *chunk_target = pl.chunk_target;
+  *num_items = int32_t(pl.items.size());
+  *num_combine = int32_t(pl.combine.size());
+  *num_empty = int32_t(pl.empty.size());
+  for (int32_t b = 0; b < batch; ++b) {
+    bucket[b] = pl.bucket[b];
+    num_splits[b] = pl.num_splits[b];
+    chunk_len[b] = pl.chunk_len[b];
+    item_offset[b] = pl.item_offset[b];
+  }
+  std::copy(pl.combine.begin(), pl.combine.end(), combine);
+  std::copy(pl.empty.begin(), pl.empty.end(), empty);
+  if (int64_t(pl.items.size()) > items_capacity) return LIBRA_WORKSPACE_TOO_SMALL;
+  if (!pl.items.empty() && !items) return LIBRA_INVALID_ARGUMENT;
+  for (size_t i = 0; i < pl.items.size(); ++i) {
+    items[4 * i + 0] = pl.items[i].b;
+    items[4 * i + 1] = pl.items[i].j;
+    items[4 * i + 2] = pl.items[i].kv_begin;
+    items[4 * i + 3] = pl.items[i].kv_end;
+  }
+  return LIBRA_OK;
+}
+
+int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
+  if (!handle) return LIBRA_INVALID_ARGUMENT;
+  *handle = nullptr;
+  if (!cfg) return LIBRA_INVALID_ARGUMENT;
+  if (cfg->num_q_heads <= 0 || cfg->num_kv_heads <= 0 || cfg->head_dim <= 0 || cfg->page_size <= 0 ||
+      cfg->num_pages <= 0 || cfg->max_batch <= 0 || cfg->block_table_ld <= 0 || cfg->device < 0) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  if (cfg->num_q_heads % cfg->num_kv_heads != 0) return LIBRA_INVALID_ARGUMENT;
+  if (!(cfg->sm_scale >= 0.f) || !std::isfinite(cfg->sm_scale)) return LIBRA_INVALID_ARGUMENT;
+  const int group = cfg->num_q_heads / cfg->num_kv_heads;
+  if (group > 16 || (cfg->head_dim != 64 && cfg->head_dim != 128) || cfg->page_size != 16) return LIBRA_UNSUPPORTED_SHAPE;
+  if (cfg->num_pages > (int64_t(1) << 31) - 1) return LIBRA_UNSUPPORTED_SHAPE;  // page ids are int32
+
+  int64_t sp = cfg->kv_stride_page, sh = cfg->kv_stride_head, st = cfg->kv_stride_token;
+  if (sp == 0 && sh == 0 && st == 0) {  // HND
+    st = cfg->head_dim;
+    sh = int64_t(cfg->page_size) * cfg->head_dim;
+    sp = sh * cfg->num_kv_heads;
+  }
+  if (sp <= 0 || sh <= 0 || st <= 0 || sp % 8 || sh % 8 || st % 8 || st < cfg->head_dim) return LIBRA_INVALID_ARGUMENT;
+  if (sp * 2 >= (int64_t(1) << 40) || sh * 2 >= (int64_t(1) << 40) || st * 2 >= (int64_t(1) << 40)) {
+    return LIBRA_UNSUPPORTED_SHAPE;
+  }
+  libra_plan_params_t pin = cfg->plan;
+  if (pin.n_sm < 0 || pin.ctas_per_sm < 0 || pin.items_per_slot < 0 || pin.chunk_align < 0 || pin.min_chunk < 0 ||
+      pin.max_splits < 0) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+
+  libra_handle_s* h = new (std::nothrow) libra_handle_s();
+  if (!h) return LIBRA_INVALID_ARGUMENT;
+  h->cfg = *cfg;
+  h->group = group;
+  h->stride_page = sp;
+  h->stride_head = sh;
+  h->stride_token = st;
+  const float scale = (cfg->sm_scale > 0.f) ? cfg->sm_scale : 1.0f / std::sqrt(float(cfg->head_dim));
+  h->scale_log2 = scale * 1.4426950408889634f;
+
+  int status = LIBRA_OK;
+  do {
+    int ndev = 0;
+    cudaError_t e = cudaGetDeviceCount(&ndev);
+    if (e != cudaSuccess || cfg->device >= ndev) {
+      status = fail_cuda(h, e != cudaSuccess ? e : cudaErrorInvalidDevice);
+      break;
+    }
+    DeviceGuard guard(cfg->device);
+    if (guard.err != cudaSuccess) { status = fail_cuda(h, guard.err); break; }
+    int n_sm = 0, cc_major = 0;
+    if ((e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, cfg->device)) != cudaSuccess ||
+        (e = cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, cfg->device)) != cudaSuccess) {
+      status = fail_cuda(h, e);
+      break;
+    }
+    if (cc_major != 10) {  // the kernels are built for sm_100a only
+      status = fail_cuda(h, cudaErrorNoKernelImageForDevice);
+      break;
+    }
+    h->params = resolve_params(pin, n_sm);
+    if (!libra::valid_params(h->params)) { status = LIBRA_INVALID_ARGUMENT; break; }
+
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+      status = fail_cuda(h, e != cudaSuccess ? e : cudaErrorSymbolNotFound);
+      break;
+    }
+    h->encode = reinterpret_cast<EncodeTiledFn>(fn);
+
+    for (const Variant& v : variants()) {
+      for (int di = 0; di < 2 && status == LIBRA_OK; ++di) {
+        for (int ni = 0; ni < 2; ++ni) {
+          e = cudaFuncSetAttribute(reinterpret_cast<const void*>(v.fn[di][ni]),
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem[di]);
+          if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
+        }
+      }
+    }
+    if (status != LIBRA_OK) break;
+
+    h->max_items = libra::max_items(h->params, cfg->num_kv_heads, cfg->max_batch);
+    const size_t plan_ints = size_t(libra::plan_layout::kHeaderInts) + size_t(h->max_items) * libra::plan_layout::kItemInts +
+                             size_t(cfg->max_batch) * libra::plan_layout::kFixInts;
+    h->plan_bytes = align_up(plan_ints * 4, 256);
+    h->lse_off = h->plan_bytes;
+    h->o_off = h->lse_off + align_up(size_t(h->max_items) * cfg->num_q_heads * 4, 256);
+    h->workspace_bytes = h->o_off + align_up(size_t(h->max_items) * cfg->num_q_heads * cfg->head_dim * 4, 256);
+
+    for (int i = 0; i < 2; ++i) {
+      if ((e = cudaHostAlloc(reinterpret_cast<void**>(&h->staging[i]), h->plan_bytes, cudaHostAllocDefault)) != cudaSuccess ||
+          (e = cudaEventCreateWithFlags(&h->staging_done[i], cudaEventDisableTiming)) != cudaSuccess) {
+        status = fail_cuda(h, e);
+        break;
+      }
+    }
+  } while (false);
+
+  if (status != LIBRA_OK) {
+    libra_destroy(h);
+    return status;
+  }
+  *handle = h;
+  return LIBRA_OK;
+}
+
+int libra_destroy(libra_handle_t h) {
+  if (!h) return LIBRA_OK;
+  {
+    DeviceGuard guard(h->cfg.device);
+    for (int i = 0; i < 2; ++i) {
+      if (h->staging_done[i]) cudaEventDestroy(h->staging_done[i]);
+      if (h->staging[i]) cudaFreeHost(h->staging[i]);
+    }
+    for (cudaEvent_t ev : h->events) cudaEventDestroy(ev);
+    (void)cudaGetLastError();
+  }
+  delete h;
+  return LIBRA_OK;
+}
+
+int libra_workspace_size(libra_handle_t h, size_t* bytes) {
+  if (!h || !bytes) return LIBRA_INVALID_ARGUMENT;
+  *bytes = h->workspace_bytes;
+  return LIBRA_OK;
+}
+
+int libra_get_plan_params(libra_handle_t h, libra_plan_params_t* out) {
+  if (!h || !out) return LIBRA_INVALID_ARGUMENT;
+  out->n_sm = h->params.n_sm;
+  out->ctas_per_sm = h->params.ctas_per_sm;
+  out->items_per_slot = h->params.items_per_slot;
+  out->chunk_align = h->params.chunk_align;
+  out->min_chunk = h->params.min_chunk;
+  out->max_splits = h->params.max_splits;
+  return LIBRA_OK;
+}
+
+int libra_plan(libra_handle_t h, const int32_t* seq_lens_host, int32_t batch, void* workspace_dev, size_t workspace_bytes,
+               void* stream) {
+  if (!h || batch < 0 || batch > h->cfg.max_batch || (batch > 0 && !seq_lens_host) || !workspace_dev) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  if (reinterpret_cast<uintptr_t>(workspace_dev) % 256 != 0) return LIBRA_INVALID_ARGUMENT;
+  if (workspace_bytes < h->workspace_bytes) return LIBRA_WORKSPACE_TOO_SMALL;
+  const int64_t max_len = int64_t(h->cfg.block_table_ld) * h->cfg.page_size;
+  for (int32_t b = 0; b < batch; ++b) {
+    if (seq_lens_host[b] < 0 || seq_lens_host[b] > max_len) return LIBRA_INVALID_ARGUMENT;
+  }
+  h->planned = false;
+  if (!libra::make_plan(h->params, h->cfg.num_kv_heads, seq_lens_host, batch, &h->plan)) return LIBRA_INVALID_ARGUMENT;
+  const libra::HostPlan& pl = h->plan;
+  if (int64_t(pl.items.size()) > h->max_items) return LIBRA_WORKSPACE_TOO_SMALL;  // cannot happen; see max_items()
+
+  DeviceGuard guard(h->cfg.device);
+  if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+  const int k = h->next_staging;
+  if (h->staging_used[k]) LIBRA_CUDA_TRY(h, cudaEventSynchronize(h->staging_done[k]));
+
+  namespace L = libra::plan_layout;
+  int32_t* blob = h->staging[k];
+  const int32_t n_items = int32_t(pl.items.size());
+  const int32_t n_fix = int32_t(pl.combine.size() + pl.empty.size());
+  const int32_t fix_off = L::kHeaderInts + n_items * L::kItemInts;
+  std::memset(blob, 0, L::kHeaderInts * sizeof(int32_t));
+  blob[L::kMagic] = L::kMagicValue;
+  blob[L::kBatch] = batch;
+  blob[L::kNumItems] = n_items;
+  blob[L::kNumFix] = n_fix;
+  blob[L::kFixOff] = fix_off;
+  h->items_flat.resize(size_t(n_items) * 4);
+  for (int32_t i = 0; i < n_items; ++i) {
+    const libra::WorkItem& it = pl.items[i];
+    int32_t* w = blob + L::kHeaderInts + i * L::kItemInts;
+    w[0] = it.b;
+    w[1] = it.kv_begin;
+    w[2] = it.kv_end;
+    w[3] = (pl.num_splits[it.b] > 1) ? pl.item_offset[it.b] + it.j : -1;
+    h->items_flat[4 * i + 0] = it.b;
+    h->items_flat[4 * i + 1] = it.j;
+    h->items_flat[4 * i + 2] = it.kv_begin;
+    h->items_flat[4 * i + 3] = it.kv_end;
+  }
+  int32_t* fx = blob + fix_off;
+  for (int32_t b : pl.combine) {
+    fx[0] = b; fx[1] = pl.item_offset[b]; fx[2] = pl.num_splits[b]; fx[3] = seq_lens_host[b];
+    fx += L::kFixInts;
+  }
+  for (int32_t b : pl.empty) {
+    fx[0] = b; fx[1] = 0; fx[2] = 0; fx[3] = 0;
+    fx += L::kFixInts;
+  }
+  const size_t bytes = size_t(fix_off + n_fix * L::kFixInts) * sizeof(int32_t);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(workspace_dev, blob, bytes, cudaMemcpyHostToDevice, st));
+  LIBRA_CUDA_TRY(h, cudaEventRecord(h->staging_done[k], st));
+  h->staging_used[k] = true;
+  h->next_staging = k ^ 1;
+  h->workspace = workspace_dev;
+  h->num_items = n_items;
+  h->num_fix = n_fix;
+  h->last_stream = stream;
+  h->planned = true;
+  return LIBRA_OK;
+}
+
+int libra_plan_export(libra_handle_t h, libra_plan_view_t* view) {
+  if (!h || !view) return LIBRA_INVALID_ARGUMENT;
+  if (!h->planned) return LIBRA_NOT_PLANNED;
+  const libra::HostPlan& pl = h->plan;
+  view->batch = pl.batch;
+  view->chunk_target = pl.chunk_target;
+  view->num_items = int32_t(pl.items.size());
+  view->num_combine = int32_t(pl.combine.size());
+  view->num_empty = int32_t(pl.empty.size());
+  view->bucket = pl.bucket.data();
+  view->num_splits = pl.num_splits.data();
+  view->chunk_len = pl.chunk_len.data();
+  view->item_offset = pl.item_offset.data();
+  view->items = h->items_flat.data();
+  view->combine = pl.combine.data();
+  view->empty = pl.empty.data();
+  return LIBRA_OK;
+}
+
+int libra_set_variant(libra_handle_t h, int32_t warps, int32_t stages) {
+  if (!h) return LIBRA_INVALID_ARGUMENT;
+  const std::vector<Variant>& vs = variants();
+  for (size_t i = 0; i < vs.size(); ++i) {
+    if (vs[i].warps == warps && vs[i].stages == stages) {
+      h->variant = int(i);
+      return LIBRA_OK;
+    }
+  }
+  return LIBRA_UNSUPPORTED_SHAPE;
+}
+
+int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, const void* v_pages,
+                      const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream) {
+  if (!h || !q || !k_pages || !v_pages || !block_table || !seq_lens || !out) return LIBRA_INVALID_ARGUMENT;
+  if (reinterpret_cast<uintptr_t>(k_pages) % 16 || reinterpret_cast<uintptr_t>(v_pages) % 16 ||
+      reinterpret_cast<uintptr_t>(q) % 4 || reinterpret_cast<uintptr_t>(out) % 4) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  if (!h->planned) return LIBRA_NOT_PLANNED;
+  DeviceGuard guard(h->cfg.device);
+  if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  libra_handle_s::PoolMaps* pm = nullptr;
+  for (int i = 0; i < libra_handle_s::kMapCache; ++i) {
+    if (h->maps[i].k_ptr == k_pages && h->maps[i].v_ptr == v_pages) pm = &h->maps[i];
+  }
+  if (!pm) {
+    pm = &h->maps[h->next_map];
+    h->next_map = (h->next_map + 1) % libra_handle_s::kMapCache;
+    pm->k_ptr = pm->v_ptr = nullptr;
+    int rc = encode_pool_map(h, k_pages, &pm->map_k, &h->pos_head, &h->pos_page);
+    if (rc == LIBRA_OK) rc = encode_pool_map(h, v_pages, &pm->map_v, &h->pos_head, &h->pos_page);
+    if (rc != LIBRA_OK) return rc;
+    pm->k_ptr = k_pages;
+    pm->v_ptr = v_pages;
+  }
+
+  uint8_t* ws = static_cast<uint8_t*>(h->workspace);
+  int32_t* plan_dev = reinterpret_cast<int32_t*>(ws);
+  uint32_t* err_dev = reinterpret_cast<uint32_t*>(plan_dev + libra::plan_layout::kErrorWord);
+
+  cudaEvent_t* ev = nullptr;
+  if (h->profiling && h->profiled_calls < kMaxProfiledCalls) {
+    const size_t need = size_t(h->profiled_calls + 1) * 3;
+    while (h->events.size() < need) {
+      cudaEvent_t e;
+      LIBRA_CUDA_TRY(h, cudaEventCreate(&e));
+      h->events.push_back(e);
+    }
+    ev = &h->events[size_t(h->profiled_calls) * 3];
+    LIBRA_CUDA_TRY(h, cudaEventRecord(ev[0], st));
+  }
+
+  if (h->num_items > 0) {
+    DecodeParams p;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.block_table = block_table;
+    p.seq_lens = seq_lens;
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.plan = plan_dev;
+    p.partial_o = reinterpret_cast<float*>(ws + h->o_off);
+    p.partial_lse = reinterpret_cast<float*>(ws + h->lse_off);
+    p.error_word = err_dev;
+    p.num_pages = h->cfg.num_pages;
+    p.num_q_heads = h->cfg.num_q_heads;
+    p.num_kv_heads = h->cfg.num_kv_heads;
+    p.group = h->group;
+    p.block_table_ld = h->cfg.block_table_ld;
+    p.scale_log2 = h->scale_log2;
+    p.pos_head = h->pos_head;
+    p.pos_page = h->pos_page;
+    const Variant& v = variants()[h->variant];
+    const int di = (h->cfg.head_dim == 128) ? 1 : 0;
+    const int ni = (h->group > 8) ? 1 : 0;
+    const unsigned grid = unsigned(h->num_items) * unsigned(h->cfg.num_kv_heads);
+    v.fn[di][ni]<<<grid, v.warps * 32, v.smem[di], st>>>(pm->map_k, pm->map_v, p);
+    LIBRA_CUDA_TRY(h, cudaGetLastError());
+    ++h->launches;
+  }
+  if (ev) LIBRA_CUDA_TRY(h, cudaEventRecord(ev[1], st));
+  if (h->num_fix > 0) {
+    libra::CombineParams c;
+    c.plan = plan_dev;
+    c.partial_o = reinterpret_cast<const float*>(ws + h->o_off);
+    c.partial_lse = reinterpret_cast<const float*>(ws + h->lse_off);
+    c.seq_lens = seq_lens;
+    c.out = static_cast<__nv_bfloat16*>(out);
+    c.error_word = err_dev;
+    c.num_q_heads = h->cfg.num_q_heads;
+    c.head_dim = h->cfg.head_dim;
+    dim3 grid(unsigned(h->num_fix), unsigned(h->cfg.num_q_heads));
+    libra::combine_kernel<<<grid, h->cfg.head_dim / 2, 0, st>>>(c);
+    LIBRA_CUDA_TRY(h, cudaGetLastError());
+    ++h->launches;
+  }
+  if (ev) {
+    LIBRA_CUDA_TRY(h, cudaEventRecord(ev[2], st));
+    ++h->profiled_calls;
+  }
+  h->last_stream = stream;
+  return LIBRA_OK;
+}
+
+int libra_host_staging_size(libra_handle_t h, int32_t batch, size_t* bytes) {
+  if (!h || !bytes || batch < 0 || batch > h->cfg.max_batch) return LIBRA_INVALID_ARGUMENT;
+  const size_t qo = align_up(size_t(batch) * h->cfg.num_q_heads * h->cfg.head_dim * 2, 256);
+  const size_t pool = align_up(size_t(h->cfg.num_pages) * size_t(h->stride_page) * 2, 256);
+  const size_t bt = align_up(size_t(batch) * h->cfg.block_table_ld * 4, 256);
+  const size_t sl = align_up(size_t(batch) * 4, 256);
+  *bytes = 2 * qo + 2 * pool + bt + sl;
+  return LIBRA_OK;
+}
+
+int libra_decode_attn_host(libra_handle_t h, const void* q_host, const void* k_pages_host, const void* v_pages_host,
+                           const int32_t* block_table_host, const int32_t* seq_lens_host, int32_t batch, void* out_host,
+                           void* staging_dev, size_t staging_bytes, void* workspace_dev, size_t workspace_bytes,
+                           void* stream) {
+  if (!h || !q_host || !k_pages_host || !v_pages_host || !block_table_host || !seq_lens_host || !out_host ||
+      !staging_dev || batch <= 0) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  if (reinterpret_cast<uintptr_t>(staging_dev) % 256 != 0) return LIBRA_INVALID_ARGUMENT;
+  size_t need = 0;
+  int rc = libra_host_staging_size(h, batch, &need);
+  if (rc != LIBRA_OK) return rc;
+  if (staging_bytes < need) return LIBRA_WORKSPACE_TOO_SMALL;
+  DeviceGuard guard(h->cfg.device);
+  if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  const size_t q_bytes = size_t(batch) * h->cfg.num_q_heads * h->cfg.head_dim * 2;
+  const size_t pool_bytes = size_t(h->cfg.num_pages) * size_t(h->stride_page) * 2;
+  const size_t bt_bytes = size_t(batch) * h->cfg.block_table_ld * 4;
+  const size_t sl_bytes = size_t(batch) * 4;
+  uint8_t* base = static_cast<uint8_t*>(staging_dev);
+  uint8_t* d_q = base;
+  uint8_t* d_out = d_q + align_up(q_bytes, 256);
+  uint8_t* d_k = d_out + align_up(q_bytes, 256);
+  uint8_t* d_v = d_k + align_up(pool_bytes, 256);
+  uint8_t* d_bt = d_v + align_up(pool_bytes, 256);
+  uint8_t* d_sl = d_bt + align_up(bt_bytes, 256);
+
+  // the plan needs only the host lengths, so it goes first and its upload overlaps the big copies
+  rc = libra_plan(h, seq_lens_host, batch, workspace_dev, workspace_bytes, stream);
+  if (rc != LIBRA_OK) return rc;
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(d_q, q_host, q_bytes, cudaMemcpyHostToDevice, st));
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(d_k, k_pages_host, pool_bytes, cudaMemcpyHostToDevice, st));
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(d_v, v_pages_host, pool_bytes, cudaMemcpyHostToDevice, st));
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(d_bt, block_table_host, bt_bytes, cudaMemcpyHostToDevice, st));
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(d_sl, seq_lens_host, sl_bytes, cudaMemcpyHostToDevice, st));
+  rc = libra_decode_attn(h, d_q, d_k, d_v, reinterpret_cast<const int32_t*>(d_bt),
+                         reinterpret_cast<const int32_t*>(d_sl), d_out, stream);
+  if (rc != LIBRA_OK) return rc;
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(out_host, d_out, q_bytes, cudaMemcpyDeviceToHost, st));
+  uint32_t word = 0;
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(&word, static_cast<int32_t*>(workspace_dev) + libra::plan_layout::kErrorWord, 4,
+                                    cudaMemcpyDeviceToHost, st));
+  LIBRA_CUDA_TRY(h, cudaStreamSynchronize(st));
+  return word ? LIBRA_DEVICE_FLAGGED : LIBRA_OK;
+}
+
+int libra_last_cuda_error(libra_handle_t h) { return h ? h->last_cuda_error : 0; }
+
+int libra_debug_error_word(libra_handle_t h, uint32_t* word) {
+  if (!h || !word) return LIBRA_INVALID_ARGUMENT;
+  if (!h->planned) return LIBRA_NOT_PLANNED;
+  DeviceGuard guard(h->cfg.device);
+  if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+  cudaStream_t st = static_cast<cudaStream_t>(h->last_stream);
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(word, static_cast<int32_t*>(h->workspace) + libra::plan_layout::kErrorWord, 4,
+                                    cudaMemcpyDeviceToHost, st));
+  LIBRA_CUDA_TRY(h, cudaStreamSynchronize(st));
+  return LIBRA_OK;
+}
+
+int libra_profile_begin(libra_handle_t h) {
+  if (!h) return LIBRA_INVALID_ARGUMENT;
+  h->profiling = true;
+  h->profiled_calls = 0;
+  return LIBRA_OK;
+}
+
+int libra_profile_end(libra_handle_t h, double* decode_ms, double* combine_ms, int32_t* calls) {
+  if (!h) return LIBRA_INVALID_ARGUMENT;
+  DeviceGuard guard(h->cfg.device);
+  if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+  double d = 0.0, c = 0.0;
+  for (int i = 0; i < h->profiled_calls; ++i) {
+    cudaEvent_t* ev = &h->events[size_t(i) * 3];
+    LIBRA_CUDA_TRY(h, cudaEventSynchronize(ev[2]));
+    float a = 0.f, b = 0.f;
+    LIBRA_CUDA_TRY(h, cudaEventElapsedTime(&a, ev[0], ev[1]));
+    LIBRA_CUDA_TRY(h, cudaEventElapsedTime(&b, ev[1], ev[2]));
+    d += a;
+    c += b;
+  }
+  if (decode_ms) *decode_ms = d;
+  if (combine_ms) *combine_ms = c;
+  if (calls) *calls = h->profiled_calls;
+  h->profiling = false;
+  h->profiled_calls = 0;
+  return LIBRA_OK;
+}
+
+int libra_launch_count(libra_handle_t h, int64_t* launches) {
+  if (!h || !launches) return LIBRA_INVALID_ARGUMENT;
+  *launches = h->launches;
+  return LIBRA_OK;
+}
+
+}  // extern "C"

@@ -225,13 +225,15 @@ def random_case(seed: int, batch: int, num_q_heads: int, num_kv_heads: int, head
 
 
 # --------------------------------------------------------------------------- device values
-def fill_device_pools(layout: Layout, device, seed: int | None = None, chunk_pages: int = 8192):
+def fill_device_pools(layout: Layout, device, seed: int | None = None, chunk_pages: int = 8192,
+                      poison: bool = True):
     """Fill q and the K/V pools on the device with a seeded torch generator (the large
     workloads hold up to 2 x 8.6 GB of pool, too slow to draw on the host).
 
-    Every page is filled with N(0,1) (or U[-1,1]) bf16 values; slots past the end of a
-    sequence in its last page are then overwritten with the poison value.  Returns torch
-    bf16 tensors (q[B,Hq,d], k_pages[P,Hkv,page,d], v_pages[P,Hkv,page,d]).
+    Every page is filled with N(0,1) (or U[-1,1]) bf16 values; with ``poison`` the slots past
+    the end of a sequence in its last page are then overwritten with the poison value (see
+    ``poison_tails``).  Returns torch bf16 tensors (q[B,Hq,d], k_pages[P,Hkv,page,d],
+    v_pages[P,Hkv,page,d]).
     """
     import torch
 
@@ -252,12 +254,29 @@ def fill_device_pools(layout: Layout, device, seed: int | None = None, chunk_pag
         for p0 in range(0, layout.pool_pages, chunk_pages):
             p1 = min(layout.pool_pages, p0 + chunk_pages)
             t[p0:p1] = draw((p1 - p0,) + shape[1:])
-    # poison the tail slots of every sequence's last page
+    if poison:
+        poison_tails(layout, k, v)
+    return q, k, v
+
+
+def poison_tails(layout: Layout, k, v):
+    """Overwrite the slots past the end of every sequence's last page (device HND pools) with the
+    poison value.  Returns what was there, for ``restore_tails``: a multi-step workload reuses the
+    pool with a new page placement, where those slots may hold live tokens."""
+    w = layout.workload
     lens = layout.seq_lens.astype(np.int64)
     rem = lens % w.page_size
-    rows = np.nonzero((rem != 0) & (lens > 0))[0]
-    for b in rows:
+    saved = []
+    for b in np.nonzero((rem != 0) & (lens > 0))[0]:
         pg = int(layout.block_table[b, (int(lens[b]) - 1) // w.page_size])
-        k[pg, :, int(rem[b]):, :] = float(POISON_F32)
-        v[pg, :, int(rem[b]):, :] = -float(POISON_F32)
-    return q, k, v
+        r = int(rem[b])
+        saved.append((pg, r, k[pg, :, r:, :].clone(), v[pg, :, r:, :].clone()))
+        k[pg, :, r:, :] = float(POISON_F32)
+        v[pg, :, r:, :] = -float(POISON_F32)
+    return saved
+
+
+def restore_tails(saved, k, v) -> None:
+    for pg, r, ks, vs in saved:
+        k[pg, :, r:, :] = ks
+        v[pg, :, r:, :] = vs

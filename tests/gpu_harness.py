@@ -1,0 +1,87 @@
+"""Plumbing for the GPU parity tests: device buffers via torch, calls through the C ABI binding."""
+import numpy as np
+
+CANARY = 0x7FC0  # bf16 NaN: any output row the library fails to write stays NaN
+
+
+def to_dev(a, dev):
+    import torch
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).to(dev)
+    return torch.from_numpy(a).to(dev)
+
+
+def bf16_dev_to_f32(t):
+    """int16/bf16 device tensor -> float32 NumPy (exact)."""
+    import torch
+    if t.dtype == torch.int16:
+        t = t.view(torch.bfloat16)
+    return t.float().cpu().numpy()
+
+
+class Runner:
+    """One handle + workspace for one shape; run() executes plan + decode on the current stream."""
+
+    def __init__(self, binding, Hq, Hkv, d, num_pages, max_batch, ld, layout="HND", plan=None, sm_scale=0.0,
+                 variant=None):
+        import torch
+        self.torch = torch
+        self.dev = torch.device("cuda:0")
+        strides = (0, 0, 0)
+        if layout == "NHD":
+            strides = (16 * Hkv * d, d, Hkv * d)
+        self.h = binding.Handle(Hq, Hkv, d, num_pages, max_batch, ld, kv_strides=strides, sm_scale=sm_scale,
+                                plan=plan)
+        if variant is not None:
+            self.h.set_variant(*variant)
+        self.ws = torch.empty(self.h.workspace_size(), dtype=torch.uint8, device=self.dev)
+        self.shape = (Hq, d)
+
+    def run(self, q, k, v, bt, lens, lens_dev=None, check=True):
+        """q/k/v/bt: device tensors (int16 or bf16 / int32); lens: host int32 array. Returns device out (int16)."""
+        torch = self.torch
+        B = int(len(lens))
+        out = torch.full((B,) + self.shape, CANARY, dtype=torch.int16, device=self.dev).view(torch.int16)
+        if lens_dev is None:
+            lens_dev = torch.from_numpy(np.ascontiguousarray(lens, dtype=np.int32)).to(self.dev)
+        st = torch.cuda.current_stream().cuda_stream
+        self.h.plan(np.asarray(lens, dtype=np.int32), self.ws.data_ptr(), self.ws.numel(), st)
+        self.h.decode_attn(q.data_ptr(), k.data_ptr(), v.data_ptr(), bt.data_ptr(), lens_dev.data_ptr(),
+                           out.data_ptr(), st)
+        torch.cuda.synchronize()
+        if check:
+            assert self.h.debug_error_word() == 0
+        return out
+
+
+def run_host_case(binding, q, k, v, bt, lens, layout="HND", plan=None, sm_scale=0.0, variant=None):
+    """Host uint16 inputs (HND order; transposed here for NHD) -> float32 output [B, Hq, d]."""
+    import torch
+    dev = torch.device("cuda:0")
+    B, Hq, d = q.shape
+    Hkv = k.shape[1]
+    if layout == "NHD":
+        k = np.ascontiguousarray(k.transpose(0, 2, 1, 3))
+        v = np.ascontiguousarray(v.transpose(0, 2, 1, 3))
+    r = Runner(binding, Hq, Hkv, d, k.shape[0], max(B, 1), bt.shape[1], layout, plan, sm_scale, variant)
+    out = r.run(to_dev(q, dev), to_dev(k, dev), to_dev(v, dev), to_dev(bt, dev), lens)
+    res = bf16_dev_to_f32(out)
+    r.h.close()
+    return res
+
+
+def gather_for_oracle(k_dev, v_dev, block_table, seq_lens, rows):
+    """Copy the pages of sequences `rows` back to the host as a compact pool and a remapped block
+    table, so that the CPU oracle can evaluate a sample of a workload whose pools live on the GPU."""
+    import torch
+    ids = []
+    new_bt = np.full((len(rows), block_table.shape[1]), -1, dtype=np.int32)
+    for i, b in enumerate(rows):
+        n = (int(seq_lens[b]) + 15) // 16
+        new_bt[i, :n] = np.arange(len(ids), len(ids) + n)
+        ids.extend(int(x) for x in block_table[b, :n])
+    idx = torch.tensor(ids, dtype=torch.long, device=k_dev.device)
+    k = k_dev.view(torch.int16)[idx].cpu().numpy().view(np.uint16)
+    v = v_dev.view(torch.int16)[idx].cpu().numpy().view(np.uint16)
+    return k, v, new_bt, np.asarray([seq_lens[b] for b in rows], dtype=np.int32)

@@ -1,0 +1,276 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the float64 CPU oracle on the
+same seeded inputs.  Gates: the stated one (|err| <= 1e-2 + 1e-2 |ref|) and the tight one
+(tests/gates.py).  Integer work (plan, page indexing) is checked bit-exactly."""
+import numpy as np
+import pytest
+
+from oracle import attention_oracle as O
+from oracle import planner_ref as P
+from paper_2606_03077_b200 import workloads as W
+
+import gates
+import gpu_harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def bits(x):
+    return W.f32_to_bf16_bits(np.asarray(x, dtype=np.float32))
+
+
+def check(got, ref, what=""):
+    assert np.all(np.isfinite(got)), f"{what}: non-finite output (unwritten row?)"
+    assert gates.stated_violations(got, ref) == 0, f"{what}: stated gate"
+    assert gates.tight_violations(got, ref) == 0, f"{what}: tight gate, ratio {gates.tight_ratio(got, ref):.2f}"
+
+
+def small_plan(lib):
+    """Planner constants that force splits at test sizes."""
+    return lib.PlanParams(4, 1, 2, 16, 16, 64)
+
+
+# ------------------------------------------------------------------ the tiny workload
+def test_tiny_workload(lib):
+    lay, q, k, v = W.make_host_inputs("tiny")
+    ref, _ = O.paged_decode_attention(q, k, v, lay.block_table, lay.seq_lens)
+    got = H.run_host_case(lib, q, k, v, lay.block_table, lay.seq_lens)
+    check(got, ref, "tiny")
+    got2 = H.run_host_case(lib, q, k, v, lay.block_table, lay.seq_lens, plan=small_plan(lib))
+    check(got2, ref, "tiny, forced splits")
+
+
+# ------------------------------------------------------------------ shapes, tails, layouts
+CASES = [
+    # (Hq, Hkv, d, lens)
+    (4, 1, 64, [1, 2, 15, 16, 17, 31, 33]),
+    (8, 2, 128, [255, 256, 257, 1, 700]),
+    (8, 8, 128, [100, 1000]),                 # G = 1
+    (4, 2, 128, [513, 48]),                   # G = 2
+    (40, 8, 128, [1200, 77, 2049]),           # G = 5
+    (64, 8, 128, [3000, 5]),                  # G = 8
+    (24, 2, 64, [900, 130]),                  # G = 12: two head tiles
+    (32, 2, 128, [777, 64]),                  # G = 16
+    (6, 2, 64, [0, 40, 0, 300]),              # empty sequences
+]
+
+
+@pytest.mark.parametrize("layout", ["HND", "NHD"])
+@pytest.mark.parametrize("case", range(len(CASES)))
+def test_shapes_and_tails(lib, case, layout):
+    Hq, Hkv, d, lens = CASES[case]
+    lens_a, bt, q, k, v = W.random_case(100 + case, len(lens), Hq, Hkv, d, lens)
+    ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
+    for plan in (None, small_plan(lib)):
+        got = H.run_host_case(lib, q, k, v, bt, lens_a, layout=layout, plan=plan)
+        check(got, ref, f"case {case} {layout} plan={'default' if plan is None else 'small'}")
+
+
+def test_every_block_shape_agrees(lib):
+    lens = [2500, 300, 17, 4100]
+    lens_a, bt, q, k, v = W.random_case(7, 4, 32, 8, 128, lens)
+    ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
+    for variant in [(4, 3), (4, 2), (4, 4), (4, 6), (8, 2), (8, 3), (2, 6), (2, 4)]:
+        got = H.run_host_case(lib, q, k, v, bt, lens_a, plan=lib.PlanParams(8, 1, 2, 256, 256, 64), variant=variant)
+        check(got, ref, f"variant {variant}")
+
+
+def test_custom_scale(lib):
+    lens_a, bt, q, k, v = W.random_case(8, 2, 8, 2, 64, [90, 33])
+    ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a, sm_scale=0.3)
+    got = H.run_host_case(lib, q, k, v, bt, lens_a, sm_scale=0.3)
+    check(got, ref, "sm_scale 0.3")
+
+
+# ------------------------------------------------------------------ the oracle's pins, on the GPU
+def test_length_one_is_bit_exact(lib):
+    lens_a, bt, q, k, v = W.random_case(21, 3, 8, 2, 128, [1, 1, 1])
+    got = H.run_host_case(lib, q, k, v, bt, lens_a)
+    for b in range(3):
+        for h in range(8):
+            assert np.array_equal(got[b, h], W.bf16_bits_to_f32(v[bt[b, 0], h // 4, 0]))
+
+
+def test_identical_value_rows(lib):
+    lens_a, bt, q, k, v = W.random_case(22, 2, 8, 2, 128, [1500, 70])
+    row = bits(np.linspace(-3, 3, 128))
+    v[...] = row
+    got = H.run_host_case(lib, q, k, v, bt, lens_a, plan=small_plan(lib))
+    want = W.bf16_bits_to_f32(row)
+    # sum p = 1 across pages, warps, splits and the combine: at most one bf16 ulp off
+    assert np.all(np.abs(got - want) <= np.abs(want) * 2.0 ** -7 + 1e-30)
+
+
+def test_zero_query_mean_closed_form(lib):
+    L = 1111
+    lens_a, bt, q, k, v = W.random_case(23, 1, 4, 1, 64, [L])
+    q[...] = 0
+    for t in range(L):
+        v[bt[0, t // 16], 0, t % 16] = bits([(t + j) % 251 for j in range(64)])
+    exact = np.array([sum((t + j) % 251 for t in range(L)) / L for j in range(64)])
+    for plan in (None, small_plan(lib)):
+        got = H.run_host_case(lib, q, k, v, bt, lens_a, plan=plan)
+        # a lost or doubled 16-token page moves the mean by > 1 %; bf16 output rounding is 0.4 %
+        assert np.all(np.abs(got[0] - exact) <= exact * 2.0 ** -7)
+
+
+def test_one_hot_key_sweep_is_bit_exact(lib):
+    L, d = 1000, 64
+    lens_a, bt, q, k, v = W.random_case(24, 1, 4, 1, d, [L])
+    prm = P.PlanParams(4, 1, 2, 16, 16, 64)
+    pl = P.plan([L], 1, prm)
+    cuts = sorted({it[2] for it in pl.items} | {it[3] - 1 for it in pl.items})
+    sweep = sorted(set(cuts + [0, 15, 16, 31, L - 1, L - 2, 500]))
+    assert len(pl.items) > 4
+    # value rows encode (page id, slot) as small integers, exact in bf16
+    for t in range(L):
+        pg = int(bt[0, t // 16])
+        v[pg, 0, t % 16] = bits([pg % 256, pg // 256, t % 16] + [(t * 7 + j) % 200 for j in range(d - 3)])
+    c = 40.0  # c*c/sqrt(64) = 200: all other weights underflow to 0 in fp32
+    import torch
+    dev = torch.device("cuda:0")
+    r = H.Runner(lib, 4, 1, d, k.shape[0], 1, bt.shape[1], plan=small_plan(lib))
+    for tstar in sweep:
+        k2 = np.zeros_like(k); q2 = np.zeros_like(q)
+        q2[0, :, 0] = bits([c])[0]
+        k2[bt[0, tstar // 16], 0, tstar % 16, 0] = bits([c])[0]
+        if L % 16:
+            k2[bt[0, L // 16], 0, L % 16, 0] = bits([4 * c])[0]     # dominant key one past the end: no effect
+        out = H.bf16_dev_to_f32(r.run(H.to_dev(q2, dev), H.to_dev(k2, dev), H.to_dev(v, dev), H.to_dev(bt, dev), lens_a))
+        want = W.bf16_bits_to_f32(v[bt[0, tstar // 16], 0, tstar % 16])
+        for h in range(4):
+            assert np.array_equal(out[0, h], want), f"t*={tstar}"
+
+
+def test_page_placement_is_bit_invariant(lib):
+    lens_a, bt, q, k, v = W.random_case(25, 3, 8, 2, 128, [900, 2100, 33])
+    a = H.run_host_case(lib, q, k, v, bt, lens_a, plan=small_plan(lib))
+    perm = np.random.default_rng(2).permutation(k.shape[0])
+    k2 = np.empty_like(k); v2 = np.empty_like(v)
+    k2[perm] = k; v2[perm] = v
+    bt2 = np.where(bt >= 0, perm[np.maximum(bt, 0)], -1).astype(np.int32)
+    b = H.run_host_case(lib, q, k2, v2, bt2, lens_a, plan=small_plan(lib))
+    assert np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("shift", [100.0, -200.0])
+def test_large_key_shift_is_safe(lib, shift):
+    # scores move by q0*shift/sqrt(d), up to several hundred: exp would overflow without the running max
+    lens_a, bt, q, k, v = W.random_case(26, 2, 8, 2, 64, [400, 90])
+    kf = W.bf16_bits_to_f32(k).astype(np.float64)
+    kf[..., 0] += shift
+    k2 = bits(kf)
+    ref, _ = O.paged_decode_attention(q, k2, v, bt, lens_a)
+    got = H.run_host_case(lib, q, k2, v, bt, lens_a, plan=small_plan(lib))
+    check(got, ref, f"shift {shift}")
+
+
+def test_split_and_unsplit_agree(lib):
+    lens_a, bt, q, k, v = W.random_case(27, 2, 32, 8, 128, [5000, 1300])
+    ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
+    one = H.run_host_case(lib, q, k, v, bt, lens_a, plan=lib.PlanParams(148, 2, 4, 256, 512, 1))
+    many = H.run_host_case(lib, q, k, v, bt, lens_a, plan=lib.PlanParams(148, 2, 4, 256, 512, 64))
+    check(one, ref, "max_splits 1")
+    check(many, ref, "max_splits 64")
+
+
+def test_nan_garbage_outside_sequences_is_ignored(lib):
+    lens_a, bt, q, k, v = W.random_case(28, 3, 8, 2, 128, [37, 1, 530], poison=False)
+    ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
+    owned = np.zeros((k.shape[0], 16), dtype=bool)
+    for b, L in enumerate(lens_a):
+        for t in range(int(L)):
+            owned[bt[b, t // 16], t % 16] = True
+    for arr in (k, v):
+        arr.transpose(0, 2, 1, 3)[~owned] = 0x7FC0   # NaN
+    got = H.run_host_case(lib, q, k, v, bt, lens_a, plan=small_plan(lib))
+    check(got, ref, "NaN garbage")
+
+
+def test_runs_are_bit_reproducible(lib):
+    lens_a, bt, q, k, v = W.random_case(29, 4, 32, 8, 128, [3000, 200, 4500, 1])
+    a = H.run_host_case(lib, q, k, v, bt, lens_a)
+    b = H.run_host_case(lib, q, k, v, bt, lens_a)
+    assert np.array_equal(a, b)
+
+
+# ------------------------------------------------------------------ device-side checks, host-visible errors
+def test_error_word_flags_bad_inputs(lib):
+    import torch
+    dev = torch.device("cuda:0")
+    lens_a, bt, q, k, v = W.random_case(30, 2, 8, 2, 128, [100, 40])
+    r = H.Runner(lib, 8, 2, 128, k.shape[0], 2, bt.shape[1])
+    args = [H.to_dev(x, dev) for x in (q, k, v)]
+    r.run(*args, H.to_dev(bt, dev), lens_a)
+    assert r.h.debug_error_word() == 0
+    # page id outside the pool: the tiled copy reads zeros there (no fault) and the kernel flags it
+    bad = bt.copy(); bad[0, 2] = k.shape[0] + 5
+    r.run(*args, H.to_dev(bad, dev), lens_a, check=False)
+    assert r.h.debug_error_word() & lib.ERR_BAD_PAGE_ID
+    # device lengths that differ from the planned ones
+    other = torch.tensor([99, 40], dtype=torch.int32, device=dev)
+    r.run(*args, H.to_dev(bt, dev), lens_a, lens_dev=other, check=False)
+    assert r.h.debug_error_word() & lib.ERR_SEQ_LEN_MISMATCH
+    # and a clean run resets the word
+    r.run(*args, H.to_dev(bt, dev), lens_a)
+    assert r.h.debug_error_word() == 0
+
+
+def test_host_side_misuse(lib):
+    import torch
+    dev = torch.device("cuda:0")
+    h = lib.Handle(8, 2, 128, 64, 4, 8)
+    ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=dev)
+    st = torch.cuda.current_stream().cuda_stream
+    with pytest.raises(lib.LibraError) as e:
+        h.decode_attn(ws.data_ptr(), ws.data_ptr(), ws.data_ptr(), ws.data_ptr(), ws.data_ptr(), ws.data_ptr(), st)
+    assert e.value.status == lib.NOT_PLANNED
+    with pytest.raises(lib.LibraError) as e:
+        h.plan(np.array([5], np.int32), ws.data_ptr(), 128, st)
+    assert e.value.status == lib.WORKSPACE_TOO_SMALL
+    with pytest.raises(lib.LibraError) as e:
+        h.plan(np.array([5] * 9, np.int32), ws.data_ptr(), ws.numel(), st)       # batch > max_batch
+    assert e.value.status == lib.INVALID_ARGUMENT
+    with pytest.raises(lib.LibraError) as e:
+        h.plan(np.array([8 * 16 + 1], np.int32), ws.data_ptr(), ws.numel(), st)  # longer than the table row
+    assert e.value.status == lib.INVALID_ARGUMENT
+    with pytest.raises(lib.LibraError) as e:
+        h.plan(np.array([5], np.int32), ws.data_ptr() + 4, ws.numel(), st)       # misaligned workspace
+    assert e.value.status == lib.INVALID_ARGUMENT
+    h.close()
+
+
+def test_plan_export_matches_reference(lib):
+    import torch
+    dev = torch.device("cuda:0")
+    lay, _ = W.make_layout("lognormal_b64")
+    h = lib.Handle(32, 8, 128, lay.pool_pages, 64, lay.block_table.shape[1])
+    prm = h.plan_params()
+    assert prm.n_sm == torch.cuda.get_device_properties(0).multi_processor_count
+    ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=dev)
+    h.plan(lay.seq_lens, ws.data_ptr(), ws.numel(), torch.cuda.current_stream().cuda_stream)
+    got = h.plan_export()
+    ref = P.plan(lay.seq_lens, 8, P.PlanParams(prm.n_sm, prm.ctas_per_sm, prm.items_per_slot, prm.chunk_align,
+                                               prm.min_chunk, prm.max_splits))
+    assert got["chunk_target"] == ref.chunk_target and [tuple(r) for r in got["items"]] == ref.items
+    assert list(got["num_splits"]) == ref.num_splits and list(got["item_offset"]) == ref.item_offset
+    assert list(got["combine"]) == ref.combine
+    torch.cuda.synchronize()
+    h.close()
+
+
+def test_host_buffer_entry_point(lib):
+    import torch
+    dev = torch.device("cuda:0")
+    lay, q, k, v = W.make_host_inputs("tiny")
+    ref, _ = O.paged_decode_attention(q, k, v, lay.block_table, lay.seq_lens)
+    h = lib.Handle(4, 1, 64, lay.pool_pages, 4, lay.block_table.shape[1])
+    ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=dev)
+    stg = torch.empty(h.host_staging_size(4), dtype=torch.uint8, device=dev)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16) if a.dtype == np.uint16 else np.ascontiguousarray(a)).pin_memory()
+    hq, hk, hv, hbt, hl = pin(q), pin(k), pin(v), pin(lay.block_table), pin(lay.seq_lens)
+    hout = torch.zeros((4, 4, 64), dtype=torch.int16).pin_memory()
+    h.decode_attn_host(hq.data_ptr(), hk.data_ptr(), hv.data_ptr(), hbt.data_ptr(), hl.data_ptr(), 4, hout.data_ptr(),
+                       stg.data_ptr(), stg.numel(), ws.data_ptr(), ws.numel(), torch.cuda.current_stream().cuda_stream)
+    got = hout.view(torch.bfloat16).float().numpy()
+    check(got, ref, "host entry point")
+    h.close()
