@@ -138,7 +138,7 @@ def aggregate_over_ranks(elapsed_ms: float, units: float, world: int, device=Non
 class Replica:
     """One workload resident on one GPU: pools (several copies), handle, workspace."""
 
-    def __init__(self, name: str, dev, copies: int | None = None):
+    def __init__(self, name: str, dev, copies: int | None = None, plan=None, variant=None, fused=None):
         import torch
 
         from paper_2606_03077_b200 import binding, workloads as W
@@ -166,7 +166,11 @@ class Replica:
             self.lens_dev.append(torch.from_numpy(lay.seq_lens.copy()).to(dev))
         self.out = torch.zeros((self.w.batch, self.w.num_q_heads, self.w.head_dim), dtype=torch.bfloat16, device=dev)
         self.h = binding.Handle(self.w.num_q_heads, self.w.num_kv_heads, self.w.head_dim, lay0.pool_pages,
-                                self.w.batch, self.ld, device=dev.index or 0)
+                                self.w.batch, self.ld, device=dev.index or 0, plan=plan)
+        if variant is not None:
+            self.h.set_variant(*variant)
+        if fused is not None:
+            self.h.set_combine_mode(fused)
         self.ws = torch.empty(self.h.workspace_size(), dtype=torch.uint8, device=dev)
         self.kv_bytes_per_step = float(np.mean([l.kv_bytes for l in self.layouts]))
         self.i = 0

@@ -140,11 +140,21 @@ int libra_workspace_size(libra_handle_t handle, size_t* bytes);
 /* The planner constants the handle uses, defaults resolved (n_sm = the device's SM count). */
 int libra_get_plan_params(libra_handle_t handle, libra_plan_params_t* out);
 
-/* Tuning knob: shape of the decode thread block, `warps` warps that each own `stages` shared-memory
- * stages of one K page plus one V page.  Only the compiled-in shapes are accepted (UNSUPPORTED_SHAPE
- * otherwise); the default is the tuned one.  Results do not depend on the stage count; the warp
- * count changes the order of the final merge and hence the last bits of the result. */
-int libra_set_variant(libra_handle_t handle, int32_t warps, int32_t stages);
+/* Tuning knob: schedule and shape of the decode kernel.  persistent = 0: one thread block per work
+ * unit; persistent = 1: n_sm * ctas_per_sm resident blocks that deal the longest-first unit list
+ * among themselves and keep their copies in flight across unit boundaries.  A block has `warps`
+ * warps that each own `stages` shared-memory stages of one K page plus one V page.  Only the
+ * compiled-in combinations that fit in shared memory for the handle's shape are accepted
+ * (UNSUPPORTED_SHAPE otherwise); the default is the tuned one.  Results do not depend on the
+ * schedule or the stage count; the warp count changes the order of the per-unit merge and hence
+ * the last bits of the result.  With the persistent schedule step C always runs as its own kernel. */
+int libra_set_variant(libra_handle_t handle, int32_t persistent, int32_t warps, int32_t stages);
+
+/* Where step C runs.  fused = 1: inside the decode kernel, by the block that publishes the
+ * last partial result of a split sequence (one launch per call).  fused = 0 (default): as a separate combine
+ * kernel after the decode kernel (two launches).  Both orders of evaluation are the same, so the two
+ * modes give bit-identical results. */
+int libra_set_combine_mode(libra_handle_t handle, int32_t fused);
 
 /* Step P as a pure host function (needs no GPU): the length-bucketed planner (Sections 2.3, 4.3
  * and 5 of the paper give the bucket properties it mirrors).  With W = n_sm * ctas_per_sm,
@@ -178,9 +188,13 @@ int libra_plan_export(libra_handle_t handle, libra_plan_view_t* view);
  * (the rollout decode step of Section 1 / Section 2.2 of the paper; the attention itself is the
  * textbook definition).  All pointers are device pointers; the plan last uploaded by libra_plan
  * into `workspace` is used and `seq_lens` (device) must hold the planned lengths (a mismatch
- * sets LIBRA_ERR_SEQ_LEN_MISMATCH in the error word).  Launches the split-KV decode kernel and,
- * if any sequence is split or empty, the combine kernel, on `stream`; returns without waiting.
+ * sets LIBRA_ERR_SEQ_LEN_MISMATCH in the error word).  Launches the split-KV decode kernel (and, in
+ * the two-launch combine mode, the combine kernel if any sequence is split or empty) on `stream`;
+ * returns without waiting.
  * Results are bit-reproducible run to run (fixed reduction order, no floating-point atomics).
+ * The workspace also holds per-sequence arrival counters that the kernels leave at zero; a call that
+ * is aborted (device reset, failed launch) may leave them dirty: plan into a different workspace, or
+ * clear the workspace and create a new handle, after such a failure.
  * Errors: INVALID_ARGUMENT (null or misaligned pointer), NOT_PLANNED, CUDA_ERROR. */
 int libra_decode_attn(libra_handle_t handle, const void* q, const void* k_pages, const void* v_pages,
                       const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream);

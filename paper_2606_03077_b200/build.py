@@ -65,4 +65,4 @@ def build_library(force: bool = False, verbose: bool = True, extra_flags=()) -> 
 
 
 if __name__ == "__main__":
-    build_library(force="--force" in sys.argv, extra_flags=[a for a in sys.argv[1:] if a.startswith("-X")])
+    build_library(force="--force" in sys.argv, extra_flags=[a for a in sys.argv[1:] if a.startswith(("-X", "-D"))])

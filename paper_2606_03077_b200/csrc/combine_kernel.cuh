@@ -4,6 +4,9 @@
 //   M = max_i LSE_i ;  w_i = exp(LSE_i - M) ;  out = sum_i w_i O_i / sum_i w_i   -> bf16
 // Partials are summed in chunk order, so the result does not depend on scheduling.  An entry with
 // n == 0 is an empty sequence: its output row is zero.
+//
+// One warp per (sequence, head): lane i keeps w_i and w_{i+32}; every lane owns D/32 output
+// columns and walks the n partial rows with eight independent loads in flight.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -22,36 +25,72 @@ struct CombineParams {
   __nv_bfloat16* out;        // [B][Hq][D]
   uint32_t* error_word;
   int32_t num_q_heads;
-  int32_t head_dim;
 };
 
-// grid = (fix-up entries, query heads), block = head_dim / 2 threads, two output dims per thread
-__global__ void combine_kernel(const CombineParams p) {
+constexpr int kCombineWarps = 4;
+
+// grid = (fix-up entries, ceil(Hq / kCombineWarps)), block = kCombineWarps warps
+template <int D>
+__global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const CombineParams p) {
+  constexpr int V = D / 32;  // columns per lane: 4 (float4) or 2 (float2)
+  const int lane = threadIdx.x & 31;
+  const int h = blockIdx.y * kCombineWarps + (threadIdx.x >> 5);
+  const int Hq = p.num_q_heads;
+  if (h >= Hq) return;
   const int32_t* fix = p.plan + __ldg(p.plan + plan_layout::kFixOff) + blockIdx.x * plan_layout::kFixInts;
   const int b = __ldg(fix + 0);
   const int first = __ldg(fix + 1);
-  const int n = __ldg(fix + 2);
-  const int h = blockIdx.y;
-  const int Hq = p.num_q_heads;
-  const int D = p.head_dim;
-  if (threadIdx.x == 0 && h == 0 && __ldg(fix + 3) != __ldg(p.seq_lens + b)) {
+  const int n = __ldg(fix + 2);  // <= 64
+  if (lane == 0 && h == 0 && __ldg(fix + 3) != __ldg(p.seq_lens + b)) {
     atomicOr(p.error_word, LIBRA_DEV_ERR_SEQ_LEN_MISMATCH);
   }
-  float m = -INFINITY;
-  for (int i = 0; i < n; ++i) m = fmaxf(m, __ldg(p.partial_lse + int64_t(first + i) * Hq + h));
-  float2 num = make_float2(0.f, 0.f);
+  const float* lse = p.partial_lse + int64_t(first) * Hq + h;
+  const float l0 = (lane < n) ? __ldg(lse + int64_t(lane) * Hq) : -INFINITY;
+  const float l1 = (lane + 32 < n) ? __ldg(lse + int64_t(lane + 32) * Hq) : -INFINITY;
+  float m = fmaxf(l0, l1);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+  const float w0 = (lane < n) ? __expf(l0 - m) : 0.f;
+  const float w1 = (lane + 32 < n) ? __expf(l1 - m) : 0.f;
+
+  float num[V];
+#pragma unroll
+  for (int v = 0; v < V; ++v) num[v] = 0.f;
   float den = 0.f;
-  for (int i = 0; i < n; ++i) {
-    const int64_t row = int64_t(first + i) * Hq + h;
-    const float w = __expf(__ldg(p.partial_lse + row) - m);
-    const float2 o = __ldg(reinterpret_cast<const float2*>(p.partial_o + row * D) + threadIdx.x);
-    num.x += w * o.x;
-    num.y += w * o.y;
-    den += w;
+  const float* po = p.partial_o + (int64_t(first) * Hq + h) * D + lane * V;
+  const int64_t stride = int64_t(Hq) * D;
+  for (int i0 = 0; i0 < n; i0 += 8) {
+    float o[8][V];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      if (i0 + k < n) {
+        if constexpr (V == 4) {
+          const float4 x = __ldg(reinterpret_cast<const float4*>(po + (i0 + k) * stride));
+          o[k][0] = x.x; o[k][1] = x.y; o[k][2] = x.z; o[k][3] = x.w;
+        } else {
+          const float2 x = __ldg(reinterpret_cast<const float2*>(po + (i0 + k) * stride));
+          o[k][0] = x.x; o[k][1] = x.y;
+        }
+      } else {
+#pragma unroll
+        for (int v = 0; v < V; ++v) o[k][v] = 0.f;
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int i = i0 + k;
+      const float w = __shfl_sync(0xffffffffu, (i < 32) ? w0 : w1, i & 31);  // 0 past n
+      den += w;
+#pragma unroll
+      for (int v = 0; v < V; ++v) num[v] += w * o[k][v];
+    }
   }
   const float inv = (n > 0) ? 1.f / den : 0.f;
-  __nv_bfloat162 r = __floats2bfloat162_rn(num.x * inv, num.y * inv);
-  reinterpret_cast<__nv_bfloat162*>(p.out + (int64_t(b) * Hq + h) * D)[threadIdx.x] = r;
+  __nv_bfloat16* dst = p.out + (int64_t(b) * Hq + h) * D + lane * V;
+#pragma unroll
+  for (int v = 0; v < V; v += 2) {
+    *reinterpret_cast<__nv_bfloat162*>(dst + v) = __floats2bfloat162_rn(num[v] * inv, num[v + 1] * inv);
+  }
 }
 
 }  // namespace libra

@@ -1,8 +1,8 @@
-// Split-KV decode kernel (step D) for sm_100a.
+// Split-KV decode kernels (step D) for sm_100a.
 //
-// One thread block handles one work item (a chunk [kv_begin, kv_end) of one sequence) for one KV
-// head and all G query heads that share it.  Inside the block every warp owns a private ring of
-// shared-memory stages and walks the chunk's pages warp, warp+NW, warp+2NW, ...:
+// A work unit is one work item of the plan (a chunk [kv_begin, kv_end) of one sequence) for one KV
+// head and all G query heads that share it.  Inside a thread block every warp owns a private ring
+// of shared-memory stages and takes the unit's pages warp, warp+NW, warp+2NW, ...:
 //
 //   lane 0 : page id -> two tiled TMA loads per tensor (K and V page, 128-byte swizzle) that
 //            complete on the stage's mbarrier; up to STAGES pages per warp are in flight
@@ -11,11 +11,22 @@
 //            O^T[d x 8 heads]         += V_page^T . P^T     P rounded to bf16, l sums the rounded P
 //
 // Tokens are the M side of the tiles, the (padded) head group the N side, so a group of up to
-// 8 heads costs one 8-wide tile and nothing is wasted on padding rows.  The kernel is bound by the
-// HBM read of K and V: 2 * head_dim * 2 bytes per token per KV head, 4 * G * head_dim flop.
+// 8 heads costs one 8-wide tile and nothing is wasted on padding rows.  The kernels are bound by
+// the HBM read of K and V: 2 * head_dim * 2 bytes per token per KV head, 4 * G * head_dim flop.
 //
-// The warps never synchronise with each other in the main loop; they merge their (m, l, O) in
-// shared memory once at the end, in warp order, so results are bit-reproducible.
+// The warps never synchronise with each other while they stream pages; they merge their (m, l, O)
+// in shared memory once per unit, in warp order, so results are bit-reproducible.
+//
+// Two schedules:
+//   decode_kernel             one thread block per unit, units in plan order (longest first)
+//   decode_persistent_kernel  one resident block per slot; block c takes units c, 2W-1-c, 2W+c, ...
+//                             of the longest-first list (W blocks, serpentine deal) and every warp
+//                             keeps its copy ring full ACROSS unit boundaries, so the loads of the
+//                             next unit are in flight while the current unit is merged and written
+//
+// Step C can run inside decode_kernel: every block of a split sequence bumps a per-(sequence, KV
+// head) counter after publishing its partial result, and the block that arrives last merges all
+// partials in chunk order (the same arithmetic, in the same order, as the stand-alone combine kernel).
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -36,6 +47,7 @@ struct DecodeParams {
   float* partial_o;      // [slot][Hq][D]
   float* partial_lse;    // [slot][Hq]
   uint32_t* error_word;
+  int32_t* counters;      // [batch][Hkv] arrival counters of split sequences (zero between launches)
   int64_t num_pages;
   int32_t num_q_heads;
   int32_t num_kv_heads;
@@ -44,6 +56,12 @@ struct DecodeParams {
   float scale_log2;       // sm_scale * log2(e)
   int32_t pos_head;       // coordinate slot (1..3) of the head / page dimension in the tensor maps
   int32_t pos_page;
+  int32_t num_units;      // work items x KV heads
+  int32_t num_empty;      // empty sequences whose output row this launch zeroes
+  int32_t fused_combine;  // 1: the last block of a split sequence merges its partials (step C) itself
+#ifdef LIBRA_TRACE
+  unsigned long long* trace;  // timeline experiment only: 6 words per block, right after the workspace
+#endif
 };
 
 namespace dev {
@@ -124,9 +142,252 @@ __device__ __forceinline__ float lg2(float x) {
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ void named_barrier(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 // Byte offset of 16-byte chunk c16 of row r inside a [D/64][16][128 B] tile with 128-byte swizzle.
 __device__ __forceinline__ uint32_t tile_off(int r, int c16) {
   return uint32_t(((c16 >> 3) << 11) + (r << 7) + ((((c16 & 7) ^ (r & 7))) << 4));
+}
+
+// One decoded work unit as a warp sees it.
+struct Unit {
+  int b, kvh, kv_begin, kv_end, slot, chunk_j, n_chunks;
+  int n_it;       // pages of the unit this warp takes
+  int first_page; // index of the unit's first page in the sequence's block-table row
+};
+
+template <int NW>
+__device__ __forceinline__ Unit decode_unit(const int4 item, int kvh, int warp) {
+  Unit u;
+  u.b = item.x & (plan_layout::kMaxBatch - 1);
+  u.chunk_j = (item.x >> plan_layout::kChunkShift) & 63;
+  u.n_chunks = item.x >> plan_layout::kCountShift;
+  u.kv_begin = item.y;
+  u.kv_end = item.z;
+  u.slot = item.w;  // < 0: the sequence is not split, write bf16 `out` directly
+  u.kvh = kvh;
+  const int n_pages = (u.kv_end - u.kv_begin + 15) >> 4;
+  u.first_page = u.kv_begin >> 4;
+  u.n_it = (n_pages > warp) ? (n_pages - warp + NW - 1) / NW : 0;
+  return u;
+}
+
+// Q^T fragments (B operand: k = dims, n = heads); rows of heads >= G are zero.
+template <int D, int NT>
+__device__ __forceinline__ void load_q_frags(uint32_t (&qf)[NT][D / 16][2], const DecodeParams& p, int b, int kvh,
+                                             int lane) {
+  const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    const int head = nt * 8 + g;
+    const bool live = head < p.group;
+    const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+        p.q + (int64_t(b) * p.num_q_heads + int64_t(kvh) * p.group + (live ? head : 0)) * D);
+#pragma unroll
+    for (int kk = 0; kk < D / 16; ++kk) {
+      qf[nt][kk][0] = live ? __ldg(qrow + 8 * kk + t) : 0u;
+      qf[nt][kk][1] = live ? __ldg(qrow + 8 * kk + t + 4) : 0u;
+    }
+  }
+}
+
+// Running softmax state of one warp: heads 2t, 2t+1 of every head tile.
+template <int D, int NT>
+struct WarpAcc {
+  float m[NT][2], l[NT][2];
+  float acc[NT][D / 16][4];
+  __device__ __forceinline__ void reset() {
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      m[nt][0] = m[nt][1] = -INFINITY;
+      l[nt][0] = l[nt][1] = 0.f;
+#pragma unroll
+      for (int mt = 0; mt < D / 16; ++mt) acc[nt][mt][0] = acc[nt][mt][1] = acc[nt][mt][2] = acc[nt][mt][3] = 0.f;
+    }
+  }
+};
+
+// One page (16 tokens) of one KV head: scores, online softmax update, PV accumulation.
+// kt / vt: shared-memory addresses of the K and V tiles; v_gen: generic pointer to the V tile.
+template <int D, int NT>
+__device__ __forceinline__ void process_page(WarpAcc<D, NT>& st, const uint32_t (&qf)[NT][D / 16][2], uint32_t kt,
+                                             uint32_t vt, uint8_t* v_gen, int n_valid, float scale_log2, int lane) {
+  constexpr int KS = D / 16;
+  const int g = lane >> 2;
+  const int k_row = lane & 15, k_sel = lane >> 4;
+  const int v_row = (lane & 7) + ((lane >> 4) << 3), v_sel = (lane >> 3) & 1;
+
+  if (n_valid < 16) {
+    // rows past the end may hold anything, NaN included: clear them in V so that 0 * garbage cannot leak
+    for (int i = lane; i < (16 - n_valid) * (D / 8); i += 32) {
+      const int r = n_valid + i / (D / 8);
+      const int c16 = i % (D / 8);
+      *reinterpret_cast<uint4*>(v_gen + ((c16 >> 3) << 11) + (r << 7) + ((c16 & 7) << 4)) = make_uint4(0, 0, 0, 0);
+    }
+    fence_proxy_async();  // these generic writes come before the next TMA write into this stage
+    __syncwarp();
+  }
+
+  // ---- S^T = K . Q^T  (two accumulator sets to halve the dependent chain)
+  float sc[NT][4], sc2[NT][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+    sc2[nt][0] = sc2[nt][1] = sc2[nt][2] = sc2[nt][3] = 0.f;
+  }
+#pragma unroll
+  for (int kk = 0; kk < KS; ++kk) {
+    uint32_t a[4];
+    ldsm_x4(a, kt + tile_off(k_row, 2 * kk + k_sel));
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      if (kk & 1) mma_bf16(sc2[nt], a, qf[nt][kk][0], qf[nt][kk][1]);
+      else mma_bf16(sc[nt], a, qf[nt][kk][0], qf[nt][kk][1]);
+    }
+  }
+
+  // ---- online softmax; this thread holds tokens g, g+8 for heads 2t, 2t+1
+  uint32_t pb[NT][2];
+  bool grew = false;
+  float m_new[NT][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) sc[nt][e] = (sc[nt][e] + sc2[nt][e]) * scale_log2;
+    if (n_valid < 16) {
+      if (g >= n_valid) sc[nt][0] = sc[nt][1] = -INFINITY;
+      if (g + 8 >= n_valid) sc[nt][2] = sc[nt][3] = -INFINITY;
+    }
+    float mx0 = fmaxf(sc[nt][0], sc[nt][2]);
+    float mx1 = fmaxf(sc[nt][1], sc[nt][3]);
+#pragma unroll
+    for (int off = 4; off <= 16; off <<= 1) {
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+    }
+    m_new[nt][0] = fmaxf(st.m[nt][0], mx0);
+    m_new[nt][1] = fmaxf(st.m[nt][1], mx1);
+    grew = grew || (m_new[nt][0] > st.m[nt][0]) || (m_new[nt][1] > st.m[nt][1]);
+  }
+  if (__any_sync(0xffffffffu, grew)) {
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const float f0 = ex2(st.m[nt][0] - m_new[nt][0]);  // first page: 2^(-inf) = 0 on zeros
+      const float f1 = ex2(st.m[nt][1] - m_new[nt][1]);
+      st.l[nt][0] *= f0;
+      st.l[nt][1] *= f1;
+#pragma unroll
+      for (int mt = 0; mt < KS; ++mt) {
+        st.acc[nt][mt][0] *= f0;
+        st.acc[nt][mt][1] *= f1;
+        st.acc[nt][mt][2] *= f0;
+        st.acc[nt][mt][3] *= f1;
+      }
+      st.m[nt][0] = m_new[nt][0];
+      st.m[nt][1] = m_new[nt][1];
+    }
+  }
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    const float p0 = ex2(sc[nt][0] - st.m[nt][0]);
+    const float p1 = ex2(sc[nt][1] - st.m[nt][1]);
+    const float p2 = ex2(sc[nt][2] - st.m[nt][0]);
+    const float p3 = ex2(sc[nt][3] - st.m[nt][1]);
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(p0, p1);  // token g   : heads 2t, 2t+1
+    const __nv_bfloat162 hi = __floats2bfloat162_rn(p2, p3);  // token g+8
+    const uint32_t ulo = *reinterpret_cast<const uint32_t*>(&lo);
+    const uint32_t uhi = *reinterpret_cast<const uint32_t*>(&hi);
+    // the denominator sums exactly the probabilities the tensor core will see
+    st.l[nt][0] += __uint_as_float(ulo << 16) + __uint_as_float(uhi << 16);
+    st.l[nt][1] += __uint_as_float(ulo & 0xffff0000u) + __uint_as_float(uhi & 0xffff0000u);
+    pb[nt][0] = movmatrix_trans(ulo);  // head g : tokens 2t, 2t+1
+    pb[nt][1] = movmatrix_trans(uhi);  // head g : tokens 2t+8, 2t+9
+  }
+
+  // ---- O^T += V^T . P^T
+#pragma unroll
+  for (int mt = 0; mt < KS; ++mt) {
+    uint32_t a[4];
+    ldsm_x4_trans(a, vt + tile_off(v_row, 2 * mt + v_sel));
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) mma_bf16(st.acc[nt][mt], a, pb[nt][0], pb[nt][1]);
+  }
+}
+
+// A warp's unit result -> shared memory: stats m, l per head and O as [head][dim] fp32.
+template <int D, int NT>
+__device__ __forceinline__ void stage_warp_result(WarpAcc<D, NT>& st, float* o_sm, float* m_sm, float* l_sm, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+    for (int off = 4; off <= 16; off <<= 1) {  // l is spread over the 8 token lanes of each head
+      st.l[nt][0] += __shfl_xor_sync(0xffffffffu, st.l[nt][0], off);
+      st.l[nt][1] += __shfl_xor_sync(0xffffffffu, st.l[nt][1], off);
+    }
+    if (g == 0) {
+      m_sm[nt * 8 + 2 * t] = st.m[nt][0];
+      m_sm[nt * 8 + 2 * t + 1] = st.m[nt][1];
+      l_sm[nt * 8 + 2 * t] = st.l[nt][0];
+      l_sm[nt * 8 + 2 * t + 1] = st.l[nt][1];
+    }
+#pragma unroll
+    for (int mt = 0; mt < D / 16; ++mt) {
+      const int h0 = nt * 8 + 2 * t;
+      const int d0 = mt * 16 + g;
+      o_sm[h0 * D + d0] = st.acc[nt][mt][0];
+      o_sm[(h0 + 1) * D + d0] = st.acc[nt][mt][1];
+      o_sm[h0 * D + d0 + 8] = st.acc[nt][mt][2];
+      o_sm[(h0 + 1) * D + d0 + 8] = st.acc[nt][mt][3];
+    }
+  }
+}
+
+// Merge the NW staged warp results in warp order and write the unit's result: bf16 `out` if the
+// sequence is not split, else fp32 partial O (normalised) and its natural-log LSE.
+// o_sm: [NW][o_stride floats], m_sm / l_sm: [NW][NT*8].
+template <int D, int NT, int NW>
+__device__ __forceinline__ void merge_and_write(const DecodeParams& p, const Unit& u, const float* o_sm, int o_stride,
+                                                const float* m_sm, const float* l_sm, int tid, int nthreads) {
+  const int G = p.group;
+  for (int idx = tid; idx < G * D; idx += nthreads) {
+    const int h = idx / D;
+    const int dim = idx - h * D;
+    float m_all = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) m_all = fmaxf(m_all, m_sm[w * NT * 8 + h]);
+    float num = 0.f, den = 0.f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) {
+      const float mw = m_sm[w * NT * 8 + h];
+      const float f = (mw == -INFINITY) ? 0.f : ex2(mw - m_all);
+      num += f * o_sm[w * o_stride + h * D + dim];
+      den += f * l_sm[w * NT * 8 + h];
+    }
+    const float o = num / den;
+    const int64_t head = int64_t(u.kvh) * G + h;
+    if (u.slot < 0) {
+      p.out[(int64_t(u.b) * p.num_q_heads + head) * D + dim] = __float2bfloat16_rn(o);
+    } else {
+      p.partial_o[(int64_t(u.slot) * p.num_q_heads + head) * D + dim] = o;
+      if (dim == 0) p.partial_lse[int64_t(u.slot) * p.num_q_heads + head] = (m_all + lg2(den)) * 0.6931471805599453f;
+    }
+  }
+}
+
+__device__ __forceinline__ void check_planned_length(const DecodeParams& p, const Unit& u, int len_dev) {
+  const bool ok = (u.chunk_j == u.n_chunks - 1) ? (u.kv_end == len_dev) : (u.kv_end < len_dev);
+  if (!ok) atomicOr(p.error_word, LIBRA_DEV_ERR_SEQ_LEN_MISMATCH);
+}
+
+// Output rows of empty sequences are zero; entry e of the plan's empty list.
+template <int D>
+__device__ __forceinline__ void zero_empty_row(const DecodeParams& p, int e, int tid, int nthreads) {
+  const int32_t* fix = p.plan + __ldg(p.plan + plan_layout::kFixOff) +
+                       (__ldg(p.plan + plan_layout::kNumCombine) + e) * plan_layout::kFixInts;
+  const int64_t row = int64_t(__ldg(fix)) * p.num_q_heads * D;
+  for (int i = tid; i < p.num_q_heads * D; i += nthreads) p.out[row + i] = __float2bfloat16_rn(0.f);
 }
 
 }  // namespace dev
@@ -140,13 +401,14 @@ struct DecodeSmem {
   static constexpr int kDynamicBytes = kRingBytes + 1024;  // slack for manual 1024-byte alignment
 };
 
+// ------------------------------------------------------------------------------------------------
+// One thread block per unit.
 // D: head_dim (64 | 128); NT: 8-wide head tiles (1: G <= 8, 2: G <= 16); NW warps; STAGES per warp.
 template <int D, int NT, int NW, int STAGES>
 __global__ void __launch_bounds__(NW * 32)
 decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const DecodeParams p) {
   using namespace dev;
   using SM = DecodeSmem<D, NW, STAGES>;
-  constexpr int KS = D / 16;   // k-steps of the QK product = 16-row tiles of the PV product
   constexpr int NH = D / 64;   // 128-byte column blocks of a row
   static_assert(NT * 8 * D * 4 <= SM::kWarpBytes, "epilogue staging must fit in the warp's ring");
 
@@ -154,33 +416,31 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   __shared__ uint64_t bars[NW * STAGES];
   __shared__ float stat_m[NW][NT * 8];
   __shared__ float stat_l[NW][NT * 8];
+  __shared__ int s_last;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int g = lane >> 2;
-  const int t = lane & 3;
 
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* my_ring = ring + warp * SM::kWarpBytes;
   const uint32_t my_ring_u32 = smem_u32(my_ring);
   const uint32_t my_bar0 = smem_u32(&bars[warp * STAGES]);
 
-  // ---- work item
+  if (int(blockIdx.x) >= p.num_units) {
+    zero_empty_row<D>(p, int(blockIdx.x) - p.num_units, threadIdx.x, NW * 32);
+    return;
+  }
+
+#ifdef LIBRA_TRACE
+  unsigned long long tr0 = 0, tr1 = 0, tr2 = 0;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr0));
+#endif
+  // ---- work unit
   const int item_idx = blockIdx.x / p.num_kv_heads;
   const int kvh = blockIdx.x - item_idx * p.num_kv_heads;
-  const int4 item = __ldg(reinterpret_cast<const int4*>(p.plan + plan_layout::kHeaderInts) + item_idx);
-  const int b = item.x;
-  const int kv_begin = item.y;
-  const int kv_end = item.z;
-  const int slot = item.w;  // < 0: the sequence is not split, write bf16 `out` directly
-  const int n_pages = (kv_end - kv_begin + 15) >> 4;
-  const int first_page = kv_begin >> 4;
-  const int n_it = (n_pages > warp) ? (n_pages - warp + NW - 1) / NW : 0;
-
-  if (threadIdx.x == 0) {
-    const int planned_ok = (slot < 0) ? (kv_end == __ldg(p.seq_lens + b)) : (kv_end <= __ldg(p.seq_lens + b));
-    if (!planned_ok) atomicOr(p.error_word, LIBRA_DEV_ERR_SEQ_LEN_MISMATCH);
-  }
+  const Unit u = decode_unit<NW>(__ldg(reinterpret_cast<const int4*>(p.plan + plan_layout::kHeaderInts) + item_idx), kvh, warp);
+  const int n_it = u.n_it;
+  if (threadIdx.x == 0) check_planned_length(p, u, __ldg(p.seq_lens + u.b));
 
   if (lane == 0) {
 #pragma unroll
@@ -189,23 +449,11 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   }
   __syncwarp();
 
-  // ---- Q^T fragments (B operand: k = dims, n = heads); rows of heads >= G are zero
-  uint32_t qf[NT][KS][2];
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
-    const int head = nt * 8 + g;
-    const bool live = head < p.group;
-    const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
-        p.q + (int64_t(b) * p.num_q_heads + int64_t(kvh) * p.group + (live ? head : 0)) * D);
-#pragma unroll
-    for (int kk = 0; kk < KS; ++kk) {
-      qf[nt][kk][0] = live ? __ldg(qrow + 8 * kk + t) : 0u;
-      qf[nt][kk][1] = live ? __ldg(qrow + 8 * kk + t + 4) : 0u;
-    }
-  }
+  uint32_t qf[NT][D / 16][2];
+  load_q_frags<D, NT>(qf, p, u.b, kvh, lane);
 
   // ---- page ids: lane L keeps the id of iteration 32*round + L, one round ahead
-  const int32_t* bt_row = p.block_table + int64_t(b) * p.block_table_ld + first_page + warp;
+  const int32_t* bt_row = p.block_table + int64_t(u.b) * p.block_table_ld + u.first_page + warp;
   auto load_ids = [&](int round) -> int32_t {
     const int idx = round * 32 + lane;
     return (idx < n_it) ? __ldg(bt_row + int64_t(idx) * NW) : -1;
@@ -236,26 +484,15 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     }
   };
 
-  // ---- running state: heads 2t, 2t+1 of every head tile
-  float m_run[NT][2], l_run[NT][2];
-  float acc[NT][KS][4];
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
-    m_run[nt][0] = m_run[nt][1] = -INFINITY;
-    l_run[nt][0] = l_run[nt][1] = 0.f;
-#pragma unroll
-    for (int mt = 0; mt < KS; ++mt) acc[nt][mt][0] = acc[nt][mt][1] = acc[nt][mt][2] = acc[nt][mt][3] = 0.f;
-  }
+  WarpAcc<D, NT> st;
+  st.reset();
 
   {
     const int pre = n_it < STAGES ? n_it : STAGES;
     for (int j = 0; j < pre; ++j) issue(j, j);
   }
 
-  const int k_row = lane & 15, k_sel = lane >> 4;
-  const int v_row = (lane & 7) + ((lane >> 4) << 3), v_sel = (lane >> 3) & 1;
   bool timed_out = false;
-
   int s = 0;
   uint32_t parity = 0;
   for (int it = 0; it < n_it; ++it) {
@@ -264,107 +501,13 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
       timed_out = true;
       break;
     }
+#ifdef LIBRA_TRACE
+    if (it == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr1));
+#endif
     const uint32_t kt = my_ring_u32 + s * SM::kStageBytes;
-    const uint32_t vt = kt + SM::kTileBytes;
-    const int tok0 = kv_begin + ((warp + it * NW) << 4);
-    const int n_valid = kv_end - tok0;  // >= 1; < 16 only on the sequence's last page
-
-    if (n_valid < 16) {
-      // rows past the end may hold anything, NaN included: clear them in V so that 0 * garbage cannot leak
-      uint8_t* vgen = my_ring + s * SM::kStageBytes + SM::kTileBytes;
-      for (int i = lane; i < (16 - n_valid) * (D / 8); i += 32) {
-        const int r = n_valid + i / (D / 8);
-        const int c16 = i % (D / 8);
-        *reinterpret_cast<uint4*>(vgen + ((c16 >> 3) << 11) + (r << 7) + ((c16 & 7) << 4)) = make_uint4(0, 0, 0, 0);
-      }
-      __syncwarp();
-    }
-
-    // ---- S^T = K . Q^T  (two accumulator sets to halve the dependent chain)
-    float sc[NT][4], sc2[NT][4];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
-      sc2[nt][0] = sc2[nt][1] = sc2[nt][2] = sc2[nt][3] = 0.f;
-    }
-#pragma unroll
-    for (int kk = 0; kk < KS; ++kk) {
-      uint32_t a[4];
-      ldsm_x4(a, kt + tile_off(k_row, 2 * kk + k_sel));
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        if (kk & 1) mma_bf16(sc2[nt], a, qf[nt][kk][0], qf[nt][kk][1]);
-        else mma_bf16(sc[nt], a, qf[nt][kk][0], qf[nt][kk][1]);
-      }
-    }
-
-    // ---- online softmax; this thread holds tokens g, g+8 for heads 2t, 2t+1
-    uint32_t pb[NT][2];
-    bool grew = false;
-    float m_new[NT][2];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-#pragma unroll
-      for (int e = 0; e < 4; ++e) sc[nt][e] = (sc[nt][e] + sc2[nt][e]) * p.scale_log2;
-      if (n_valid < 16) {
-        if (g >= n_valid) sc[nt][0] = sc[nt][1] = -INFINITY;
-        if (g + 8 >= n_valid) sc[nt][2] = sc[nt][3] = -INFINITY;
-      }
-      float mx0 = fmaxf(sc[nt][0], sc[nt][2]);
-      float mx1 = fmaxf(sc[nt][1], sc[nt][3]);
-#pragma unroll
-      for (int off = 4; off <= 16; off <<= 1) {
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
-      }
-      m_new[nt][0] = fmaxf(m_run[nt][0], mx0);
-      m_new[nt][1] = fmaxf(m_run[nt][1], mx1);
-      grew = grew || (m_new[nt][0] > m_run[nt][0]) || (m_new[nt][1] > m_run[nt][1]);
-    }
-    if (__any_sync(0xffffffffu, grew)) {
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        const float f0 = ex2(m_run[nt][0] - m_new[nt][0]);  // first page: 2^(-inf) = 0 on zeros
-        const float f1 = ex2(m_run[nt][1] - m_new[nt][1]);
-        l_run[nt][0] *= f0;
-        l_run[nt][1] *= f1;
-#pragma unroll
-        for (int mt = 0; mt < KS; ++mt) {
-          acc[nt][mt][0] *= f0;
-          acc[nt][mt][1] *= f1;
-          acc[nt][mt][2] *= f0;
-          acc[nt][mt][3] *= f1;
-        }
-        m_run[nt][0] = m_new[nt][0];
-        m_run[nt][1] = m_new[nt][1];
-      }
-    }
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      const float p0 = ex2(sc[nt][0] - m_run[nt][0]);
-      const float p1 = ex2(sc[nt][1] - m_run[nt][1]);
-      const float p2 = ex2(sc[nt][2] - m_run[nt][0]);
-      const float p3 = ex2(sc[nt][3] - m_run[nt][1]);
-      const __nv_bfloat162 lo = __floats2bfloat162_rn(p0, p1);  // token g   : heads 2t, 2t+1
-      const __nv_bfloat162 hi = __floats2bfloat162_rn(p2, p3);  // token g+8
-      const uint32_t ulo = *reinterpret_cast<const uint32_t*>(&lo);
-      const uint32_t uhi = *reinterpret_cast<const uint32_t*>(&hi);
-      // the denominator sums exactly the probabilities the tensor core will see
-      l_run[nt][0] += __uint_as_float(ulo << 16) + __uint_as_float(uhi << 16);
-      l_run[nt][1] += __uint_as_float(ulo & 0xffff0000u) + __uint_as_float(uhi & 0xffff0000u);
-      pb[nt][0] = movmatrix_trans(ulo);  // head g : tokens 2t, 2t+1
-      pb[nt][1] = movmatrix_trans(uhi);  // head g : tokens 2t+8, 2t+9
-    }
-
-    // ---- O^T += V^T . P^T
-#pragma unroll
-    for (int mt = 0; mt < KS; ++mt) {
-      uint32_t a[4];
-      ldsm_x4_trans(a, vt + tile_off(v_row, 2 * mt + v_sel));
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) mma_bf16(acc[nt][mt], a, pb[nt][0], pb[nt][1]);
-    }
-
+    const int tok0 = u.kv_begin + ((warp + it * NW) << 4);
+    process_page<D, NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes, u.kv_end - tok0,
+                        p.scale_log2, lane);
     __syncwarp();  // every lane has consumed the stage before lane 0 refills it
     if (it + STAGES < n_it) issue(it + STAGES, s);
     if (++s == STAGES) {
@@ -379,64 +522,281 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     for (int k = 0; k < STAGES; ++k) (void)mbar_wait(my_bar0 + 8 * k, parity);
   }
 
-  // ---- per-warp totals: l is spread over the 8 token lanes of each head
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
-#pragma unroll
-    for (int off = 4; off <= 16; off <<= 1) {
-      l_run[nt][0] += __shfl_xor_sync(0xffffffffu, l_run[nt][0], off);
-      l_run[nt][1] += __shfl_xor_sync(0xffffffffu, l_run[nt][1], off);
-    }
-  }
-
-  // ---- stage (m, l, O) of this warp in its own, now idle, ring: O as [head][dim] fp32
+#ifdef LIBRA_TRACE
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr2));
+#endif
+  // ---- stage (m, l, O) of this warp in its own, now idle, ring; merge the warps; write
   __syncwarp();
-  float* o_sm = reinterpret_cast<float*>(my_ring);
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
-    if (g == 0) {
-      stat_m[warp][nt * 8 + 2 * t] = m_run[nt][0];
-      stat_m[warp][nt * 8 + 2 * t + 1] = m_run[nt][1];
-      stat_l[warp][nt * 8 + 2 * t] = l_run[nt][0];
-      stat_l[warp][nt * 8 + 2 * t + 1] = l_run[nt][1];
-    }
-#pragma unroll
-    for (int mt = 0; mt < KS; ++mt) {
-      const int h0 = nt * 8 + 2 * t;
-      const int d0 = mt * 16 + g;
-      o_sm[h0 * D + d0] = acc[nt][mt][0];
-      o_sm[(h0 + 1) * D + d0] = acc[nt][mt][1];
-      o_sm[h0 * D + d0 + 8] = acc[nt][mt][2];
-      o_sm[(h0 + 1) * D + d0 + 8] = acc[nt][mt][3];
-    }
+  stage_warp_result<D, NT>(st, reinterpret_cast<float*>(my_ring), stat_m[warp], stat_l[warp], lane);
+  __syncthreads();
+  merge_and_write<D, NT, NW>(p, u, reinterpret_cast<const float*>(ring), SM::kWarpBytes / 4, &stat_m[0][0], &stat_l[0][0],
+                             threadIdx.x, NW * 32);
+
+#ifdef LIBRA_TRACE
+  if (threadIdx.x == 0) {
+    unsigned long long tr3;
+    unsigned smid;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr3));
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    unsigned long long* t = p.trace + 6ull * blockIdx.x;
+    t[0] = tr0; t[1] = tr1; t[2] = tr2; t[3] = tr3; t[4] = smid; t[5] = (unsigned long long)(u.kv_end - u.kv_begin);
+  }
+#endif
+  // ---- step C inside this kernel: the block that publishes the last partial of (b, kvh) merges them
+  if (u.slot < 0 || !p.fused_combine) return;
+  const int G = p.group;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int32_t* cnt = p.counters + int64_t(u.b) * p.num_kv_heads + kvh;
+    const int arrived = atomicAdd(cnt, 1);
+    s_last = (arrived == u.n_chunks - 1);
+    if (s_last) *cnt = 0;  // leave the counter clean for the next launch
   }
   __syncthreads();
-
-  // ---- merge the warps in warp order and write the result
-  const int G = p.group;
+  if (!s_last) return;
+  __threadfence();
+  const int first_slot = u.slot - u.chunk_j;
+  float* w_sm = reinterpret_cast<float*>(ring);   // [n_chunks][G] weights, then [G] 1/denominator
+  float* inv_sm = w_sm + u.n_chunks * G;
+  for (int h = threadIdx.x; h < G; h += NW * 32) {
+    const float* lse = p.partial_lse + int64_t(first_slot) * p.num_q_heads + int64_t(kvh) * G + h;
+    float mx = -INFINITY;
+    for (int i = 0; i < u.n_chunks; ++i) mx = fmaxf(mx, __ldcg(lse + int64_t(i) * p.num_q_heads));
+    float den = 0.f;
+    for (int i = 0; i < u.n_chunks; ++i) {
+      const float w = __expf(__ldcg(lse + int64_t(i) * p.num_q_heads) - mx);
+      w_sm[i * G + h] = w;
+      den += w;
+    }
+    inv_sm[h] = 1.f / den;
+  }
+  __syncthreads();
   for (int idx = threadIdx.x; idx < G * D; idx += NW * 32) {
     const int h = idx / D;
     const int dim = idx - h * D;
-    float m_all = -INFINITY;
-#pragma unroll
-    for (int w = 0; w < NW; ++w) m_all = fmaxf(m_all, stat_m[w][h]);
-    float num = 0.f, den = 0.f;
-#pragma unroll
-    for (int w = 0; w < NW; ++w) {
-      const float mw = stat_m[w][h];
-      const float f = (mw == -INFINITY) ? 0.f : ex2(mw - m_all);
-      num += f * reinterpret_cast<const float*>(ring + w * SM::kWarpBytes)[h * D + dim];
-      den += f * stat_l[w][h];
-    }
-    const float o = num / den;
-    const int64_t head = int64_t(kvh) * G + h;
-    if (slot < 0) {
-      p.out[(int64_t(b) * p.num_q_heads + head) * D + dim] = __float2bfloat16_rn(o);
-    } else {
-      p.partial_o[(int64_t(slot) * p.num_q_heads + head) * D + dim] = o;
-      if (dim == 0) p.partial_lse[int64_t(slot) * p.num_q_heads + head] = (m_all + lg2(den)) * 0.6931471805599453f;
-    }
+    const float* po = p.partial_o + (int64_t(first_slot) * p.num_q_heads + int64_t(kvh) * G + h) * D + dim;
+    float num = 0.f;
+#pragma unroll 4
+    for (int i = 0; i < u.n_chunks; ++i) num += w_sm[i * G + h] * __ldcg(po + int64_t(i) * p.num_q_heads * D);
+    p.out[(int64_t(u.b) * p.num_q_heads + int64_t(kvh) * G + h) * D + dim] = __float2bfloat16_rn(num * inv_sm[h]);
   }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Persistent schedule: gridDim.x resident blocks; block c takes units c, 2W-1-c, 2W+c, 4W-1-c, ...
+// of the longest-first list.  Every warp runs two cursors over its page stream: the issue cursor
+// keeps STAGES copies in flight and may run into the next unit (never further), the consume cursor
+// follows; the unit's descriptor, first page ids and query fragments of the next unit are loaded
+// while the current unit is still being consumed.  Shared memory: the copy rings plus one merge
+// area of NW x (NT*8 heads x D) floats.
+template <int D, int NT, int NW, int STAGES>
+struct PersistentSmem {
+  using Ring = DecodeSmem<D, NW, STAGES>;
+  static constexpr int kMergeWarpFloats = NT * 8 * D;
+  static constexpr int kMergeBytes = NW * kMergeWarpFloats * 4;
+  static constexpr int kDynamicBytes = Ring::kRingBytes + kMergeBytes + 1024;
+};
+
+template <int D, int NT, int NW, int STAGES>
+__global__ void __launch_bounds__(NW * 32)
+decode_persistent_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                         const DecodeParams p) {
+  using namespace dev;
+  using SM = DecodeSmem<D, NW, STAGES>;
+  using PS = PersistentSmem<D, NT, NW, STAGES>;
+  constexpr int NH = D / 64;
+
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t bars[NW * STAGES];
+  __shared__ float stat_m[NW][NT * 8];
+  __shared__ float stat_l[NW][NT * 8];
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int W = gridDim.x;
+  const int c = blockIdx.x;
+
+  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* my_ring = ring + warp * SM::kWarpBytes;
+  const uint32_t my_ring_u32 = smem_u32(my_ring);
+  const uint32_t my_bar0 = smem_u32(&bars[warp * STAGES]);
+  float* merge_sm = reinterpret_cast<float*>(ring + SM::kRingBytes);
+
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < STAGES; ++s) mbar_init(my_bar0 + 8 * s, 1);
+    fence_mbar_init();
+  }
+  __syncwarp();
+
+  // unit index of this block's k-th unit (serpentine deal), -1 past the end
+  auto unit_index = [&](int k) -> int {
+    const int u = k * W + ((k & 1) ? (W - 1 - c) : c);
+    return (u < p.num_units) ? u : -1;
+  };
+  const int4* items = reinterpret_cast<const int4*>(p.plan + plan_layout::kHeaderInts);
+  auto load_item = [&](int k) -> int4 {
+    const int u = unit_index(k);
+    return (u >= 0) ? __ldg(items + u / p.num_kv_heads) : make_int4(0, 0, 0, -1);
+  };
+  auto make_unit = [&](int k, const int4 raw) -> Unit {
+    const int u = unit_index(k);
+    Unit r = decode_unit<NW>(raw, (u >= 0) ? (u % p.num_kv_heads) : 0, warp);
+    if (u < 0) r.n_it = 0;
+    return r;
+  };
+  auto load_ids = [&](const Unit& u, int round) -> int32_t {
+    const int idx = round * 32 + lane;
+    return (idx < u.n_it)
+               ? __ldg(p.block_table + int64_t(u.b) * p.block_table_ld + u.first_page + warp + int64_t(idx) * NW)
+               : -1;
+  };
+
+  // ---- issue cursor
+  int i_k = 0;                         // ordinal of the unit being issued
+  bool i_live = unit_index(0) >= 0;    // false once the issue cursor has run past the block's last unit
+  Unit i_u = make_unit(0, load_item(0));
+  int i_j = 0;                         // next iteration of i_u to issue
+  int4 raw1 = load_item(1), raw2 = load_item(2);
+  int32_t ids_cur = load_ids(i_u, 0), ids_nxt = load_ids(i_u, 1);
+  int32_t ids_next_unit = load_ids(make_unit(1, raw1), 0);
+  uint32_t issued = 0, consumed = 0;
+
+  // ---- consume cursor
+  int c_k = 0;
+  Unit c_u = i_u;
+  Unit pend_u = i_u;                   // the unit the issue cursor moved into last
+  int c_len = (threadIdx.x == 0 && i_live) ? __ldg(p.seq_lens + c_u.b) : 0;  // device length, checked against the plan
+  int pend_len = 0;
+  uint32_t qf[NT][D / 16][2], qf_next[NT][D / 16][2];
+  if (i_live) load_q_frags<D, NT>(qf, p, c_u.b, c_u.kvh, lane);
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int kk = 0; kk < D / 16; ++kk) qf_next[nt][kk][0] = qf_next[nt][kk][1] = 0u;
+
+  // Move the issue cursor into the next unit; allowed only while it is at most one unit ahead.
+  auto advance_issue = [&]() {
+    ++i_k;
+    i_live = unit_index(i_k) >= 0;
+    i_u = make_unit(i_k, raw1);
+    raw1 = raw2;
+    raw2 = load_item(i_k + 2);
+    i_j = 0;
+    ids_cur = ids_next_unit;
+    ids_nxt = load_ids(i_u, 1);
+    ids_next_unit = load_ids(make_unit(i_k + 1, raw1), 0);
+    pend_u = i_u;
+    pend_len = (threadIdx.x == 0 && i_live) ? __ldg(p.seq_lens + i_u.b) : 0;
+    if (i_live) load_q_frags<D, NT>(qf_next, p, i_u.b, i_u.kvh, lane);
+  };
+
+  // Issue copies until STAGES are in flight, the stream ends, or the cursor would run two units ahead.
+  auto fill = [&]() {
+    while (issued - consumed < uint32_t(STAGES) && i_live) {
+      if (i_j >= i_u.n_it) {
+        if (i_k > c_k) break;   // already one unit ahead
+        advance_issue();
+        continue;
+      }
+      if ((i_j & 31) == 0 && i_j > 0) {
+        ids_cur = ids_nxt;
+        ids_nxt = load_ids(i_u, (i_j >> 5) + 1);
+      }
+      const int32_t pid = __shfl_sync(0xffffffffu, ids_cur, i_j & 31);
+      if (lane == 0) {
+        if (pid < 0 || int64_t(pid) >= p.num_pages) atomicOr(p.error_word, LIBRA_DEV_ERR_BAD_PAGE_ID);
+        const uint32_t s = issued % STAGES;
+        const uint32_t bar = my_bar0 + 8 * s;
+        const uint32_t kdst = my_ring_u32 + s * SM::kStageBytes;
+        const uint32_t vdst = kdst + SM::kTileBytes;
+        const int kvh = i_u.kvh;
+        const int c1 = (p.pos_head == 1) ? kvh : ((p.pos_page == 1) ? pid : 0);
+        const int c2 = (p.pos_head == 2) ? kvh : ((p.pos_page == 2) ? pid : 0);
+        const int c3 = (p.pos_head == 3) ? kvh : ((p.pos_page == 3) ? pid : 0);
+        fence_proxy_async();
+        mbar_expect_tx(bar, SM::kStageBytes);
+#pragma unroll
+        for (int h = 0; h < NH; ++h) tma_load_4d(kdst + h * 2048, &map_k, bar, h * 64, c1, c2, c3);
+#pragma unroll
+        for (int h = 0; h < NH; ++h) tma_load_4d(vdst + h * 2048, &map_v, bar, h * 64, c1, c2, c3);
+      }
+      ++issued;
+      ++i_j;
+    }
+  };
+
+  WarpAcc<D, NT> st;
+  bool dead = false;  // a copy barrier timed out: stop touching the ring, keep the block-wide barriers
+
+  for (; unit_index(c_k) >= 0; ++c_k) {
+    if (c_k > 0) {
+      // the issue cursor is in unit c_k already unless this warp had nothing left to issue
+      while (i_k < c_k) advance_issue();
+      c_u = pend_u;
+      c_len = pend_len;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          qf[nt][kk][0] = qf_next[nt][kk][0];
+          qf[nt][kk][1] = qf_next[nt][kk][1];
+        }
+    }
+    if (threadIdx.x == 0) check_planned_length(p, c_u, c_len);
+    st.reset();
+#ifdef LIBRA_TRACE
+    unsigned long long tr0 = 0, tr1 = 0, tr2 = 0;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr0));
+#endif
+    if (!dead) fill();
+
+    for (int it = 0; it < c_u.n_it && !dead; ++it) {
+      const uint32_t s = consumed % STAGES;
+      const uint32_t parity = (consumed / STAGES) & 1u;
+      if (!mbar_wait(my_bar0 + 8 * s, parity)) {
+        dead = true;
+        if (lane == 0) atomicOr(p.error_word, LIBRA_DEV_ERR_WAIT_TIMEOUT);
+        break;
+      }
+#ifdef LIBRA_TRACE
+      if (it == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr1));
+#endif
+      const uint32_t kt = my_ring_u32 + s * SM::kStageBytes;
+      const int tok0 = c_u.kv_begin + ((warp + it * NW) << 4);
+      process_page<D, NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes,
+                          c_u.kv_end - tok0, p.scale_log2, lane);
+      __syncwarp();  // every lane has consumed the stage before lane 0 refills it
+      ++consumed;
+      fill();
+    }
+
+#ifdef LIBRA_TRACE
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr2));
+#endif
+    // ---- unit epilogue: stage, merge in warp order, write; the next unit's copies stay in flight
+    stage_warp_result<D, NT>(st, merge_sm + warp * PS::kMergeWarpFloats, stat_m[warp], stat_l[warp], lane);
+    __syncthreads();
+    merge_and_write<D, NT, NW>(p, c_u, merge_sm, PS::kMergeWarpFloats, &stat_m[0][0], &stat_l[0][0], threadIdx.x, NW * 32);
+    __syncthreads();  // the merge area is free again
+#ifdef LIBRA_TRACE
+    if (threadIdx.x == 0) {
+      unsigned long long tr3;
+      unsigned smid;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr3));
+      asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+      unsigned long long* t = p.trace + 6ull * unit_index(c_k);
+      t[0] = tr0; t[1] = tr1; t[2] = tr2; t[3] = tr3; t[4] = smid; t[5] = (unsigned long long)(c_u.kv_end - c_u.kv_begin);
+    }
+#endif
+  }
+
+  if (dead) {
+    // bounded last chance for copies still in flight to land before the block exits
+    for (uint32_t k = consumed; k < issued; ++k) (void)mbar_wait(my_bar0 + 8 * (k % STAGES), (k / STAGES) & 1u);
+  }
+  for (int e = c; e < p.num_empty; e += W) zero_empty_row<D>(p, e, threadIdx.x, NW * 32);
 }
 
 }  // namespace libra

@@ -30,30 +30,56 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 typedef void (*DecodeKernelFn)(const CUtensorMap, const CUtensorMap, const DecodeParams);
 
 struct Variant {
-  int warps, stages;
-  DecodeKernelFn fn[2][2];  // [D == 128][NT - 1]
-  int smem[2];              // dynamic bytes for D = 64 / 128
+  int persistent, warps, stages;
+  DecodeKernelFn fn[2][2];  // [D == 128][NT - 1]; null where the shape does not fit in shared memory
+  int smem[2][2];           // dynamic bytes
 };
+
+constexpr int kMaxSmem = 227 * 1024 - 2048;  // per block, leaving room for the static part
 
 template <int NW, int ST>
 Variant make_variant() {
   Variant v;
+  v.persistent = 0;
   v.warps = NW;
   v.stages = ST;
   v.fn[0][0] = libra::decode_kernel<64, 1, NW, ST>;
   v.fn[0][1] = libra::decode_kernel<64, 2, NW, ST>;
   v.fn[1][0] = libra::decode_kernel<128, 1, NW, ST>;
   v.fn[1][1] = libra::decode_kernel<128, 2, NW, ST>;
-  v.smem[0] = libra::DecodeSmem<64, NW, ST>::kDynamicBytes;
-  v.smem[1] = libra::DecodeSmem<128, NW, ST>::kDynamicBytes;
+  v.smem[0][0] = v.smem[0][1] = libra::DecodeSmem<64, NW, ST>::kDynamicBytes;
+  v.smem[1][0] = v.smem[1][1] = libra::DecodeSmem<128, NW, ST>::kDynamicBytes;
   return v;
 }
 
-// Shapes of the decode block that are compiled in; index 0 is the default.
+template <int NW, int ST>
+Variant make_persistent_variant() {
+  Variant v;
+  v.persistent = 1;
+  v.warps = NW;
+  v.stages = ST;
+  v.fn[0][0] = libra::decode_persistent_kernel<64, 1, NW, ST>;
+  v.fn[0][1] = libra::decode_persistent_kernel<64, 2, NW, ST>;
+  v.fn[1][0] = libra::decode_persistent_kernel<128, 1, NW, ST>;
+  v.fn[1][1] = libra::decode_persistent_kernel<128, 2, NW, ST>;
+  v.smem[0][0] = libra::PersistentSmem<64, 1, NW, ST>::kDynamicBytes;
+  v.smem[0][1] = libra::PersistentSmem<64, 2, NW, ST>::kDynamicBytes;
+  v.smem[1][0] = libra::PersistentSmem<128, 1, NW, ST>::kDynamicBytes;
+  v.smem[1][1] = libra::PersistentSmem<128, 2, NW, ST>::kDynamicBytes;
+  for (int d = 0; d < 2; ++d)
+    for (int n = 0; n < 2; ++n)
+      if (v.smem[d][n] > kMaxSmem) v.fn[d][n] = nullptr;
+  return v;
+}
+
+// Schedules and block shapes that are compiled in; index 0 is the default.
 const std::vector<Variant>& variants() {
   static const std::vector<Variant> v = {
       make_variant<4, 3>(), make_variant<4, 2>(), make_variant<4, 4>(), make_variant<4, 6>(),
       make_variant<8, 2>(), make_variant<8, 3>(), make_variant<2, 6>(), make_variant<2, 4>(),
+      make_persistent_variant<8, 3>(), make_persistent_variant<8, 2>(), make_persistent_variant<4, 3>(),
+      make_persistent_variant<4, 2>(), make_persistent_variant<4, 4>(), make_persistent_variant<4, 6>(),
+      make_persistent_variant<2, 6>(), make_persistent_variant<2, 4>(),
   };
   return v;
 }
@@ -93,7 +119,9 @@ struct libra_handle_s {
 
   // workspace layout
   int64_t max_items = 0;
-  size_t plan_bytes = 0, lse_off = 0, o_off = 0, workspace_bytes = 0;
+  size_t plan_bytes = 0, cnt_off = 0, cnt_bytes = 0, lse_off = 0, o_off = 0, workspace_bytes = 0;
+  void* clean_workspace = nullptr;  // workspace whose arrival counters are known to be zero
+  bool fused_combine = false;
 
   // pinned staging for plan uploads
   int32_t* staging[2] = {nullptr, nullptr};
@@ -256,6 +284,7 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
   const int group = cfg->num_q_heads / cfg->num_kv_heads;
   if (group > 16 || (cfg->head_dim != 64 && cfg->head_dim != 128) || cfg->page_size != 16) return LIBRA_UNSUPPORTED_SHAPE;
   if (cfg->num_pages > (int64_t(1) << 31) - 1) return LIBRA_UNSUPPORTED_SHAPE;  // page ids are int32
+  if (cfg->max_batch > libra::plan_layout::kMaxBatch) return LIBRA_UNSUPPORTED_SHAPE;
 
   int64_t sp = cfg->kv_stride_page, sh = cfg->kv_stride_head, st = cfg->kv_stride_token;
   if (sp == 0 && sh == 0 && st == 0) {  // HND
@@ -318,8 +347,9 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
     for (const Variant& v : variants()) {
       for (int di = 0; di < 2 && status == LIBRA_OK; ++di) {
         for (int ni = 0; ni < 2; ++ni) {
+          if (!v.fn[di][ni]) continue;
           e = cudaFuncSetAttribute(reinterpret_cast<const void*>(v.fn[di][ni]),
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem[di]);
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem[di][ni]);
           if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
         }
       }
@@ -330,7 +360,9 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
     const size_t plan_ints = size_t(libra::plan_layout::kHeaderInts) + size_t(h->max_items) * libra::plan_layout::kItemInts +
                              size_t(cfg->max_batch) * libra::plan_layout::kFixInts;
     h->plan_bytes = align_up(plan_ints * 4, 256);
-    h->lse_off = h->plan_bytes;
+    h->cnt_off = h->plan_bytes;
+    h->cnt_bytes = align_up(size_t(cfg->max_batch) * cfg->num_kv_heads * 4, 256);
+    h->lse_off = h->cnt_off + h->cnt_bytes;
     h->o_off = h->lse_off + align_up(size_t(h->max_items) * cfg->num_q_heads * 4, 256);
     h->workspace_bytes = h->o_off + align_up(size_t(h->max_items) * cfg->num_q_heads * cfg->head_dim * 4, 256);
 
@@ -415,11 +447,12 @@ int libra_plan(libra_handle_t h, const int32_t* seq_lens_host, int32_t batch, vo
   blob[L::kNumItems] = n_items;
   blob[L::kNumFix] = n_fix;
   blob[L::kFixOff] = fix_off;
+  blob[L::kNumCombine] = int32_t(pl.combine.size());
   h->items_flat.resize(size_t(n_items) * 4);
   for (int32_t i = 0; i < n_items; ++i) {
     const libra::WorkItem& it = pl.items[i];
     int32_t* w = blob + L::kHeaderInts + i * L::kItemInts;
-    w[0] = it.b;
+    w[0] = it.b | (it.j << L::kChunkShift) | (pl.num_splits[it.b] << L::kCountShift);
     w[1] = it.kv_begin;
     w[2] = it.kv_end;
     w[3] = (pl.num_splits[it.b] > 1) ? pl.item_offset[it.b] + it.j : -1;
@@ -439,6 +472,11 @@ int libra_plan(libra_handle_t h, const int32_t* seq_lens_host, int32_t batch, vo
   }
   const size_t bytes = size_t(fix_off + n_fix * L::kFixInts) * sizeof(int32_t);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (h->clean_workspace != workspace_dev) {  // the kernels leave the counters at zero; a new workspace starts there
+    h->clean_workspace = nullptr;
+    LIBRA_CUDA_TRY(h, cudaMemsetAsync(static_cast<uint8_t*>(workspace_dev) + h->cnt_off, 0, h->cnt_bytes, st));
+    h->clean_workspace = workspace_dev;
+  }
   LIBRA_CUDA_TRY(h, cudaMemcpyAsync(workspace_dev, blob, bytes, cudaMemcpyHostToDevice, st));
   LIBRA_CUDA_TRY(h, cudaEventRecord(h->staging_done[k], st));
   h->staging_used[k] = true;
@@ -470,11 +508,19 @@ int libra_plan_export(libra_handle_t h, libra_plan_view_t* view) {
   return LIBRA_OK;
 }
 
-int libra_set_variant(libra_handle_t h, int32_t warps, int32_t stages) {
+int libra_set_combine_mode(libra_handle_t h, int32_t fused) {
+  if (!h || (fused != 0 && fused != 1)) return LIBRA_INVALID_ARGUMENT;
+  h->fused_combine = (fused == 1);
+  return LIBRA_OK;
+}
+
+int libra_set_variant(libra_handle_t h, int32_t persistent, int32_t warps, int32_t stages) {
   if (!h) return LIBRA_INVALID_ARGUMENT;
   const std::vector<Variant>& vs = variants();
+  const int di = (h->cfg.head_dim == 128) ? 1 : 0;
+  const int ni = (h->group > 8) ? 1 : 0;
   for (size_t i = 0; i < vs.size(); ++i) {
-    if (vs[i].warps == warps && vs[i].stages == stages) {
+    if (vs[i].persistent == persistent && vs[i].warps == warps && vs[i].stages == stages && vs[i].fn[di][ni]) {
       h->variant = int(i);
       return LIBRA_OK;
     }
@@ -525,7 +571,16 @@ int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, cons
     LIBRA_CUDA_TRY(h, cudaEventRecord(ev[0], st));
   }
 
-  if (h->num_items > 0) {
+  const Variant& v = variants()[h->variant];
+  const int di = (h->cfg.head_dim == 128) ? 1 : 0;
+  const int ni = (h->group > 8) ? 1 : 0;
+  const bool persistent = v.persistent != 0;
+  const bool fused = !persistent && h->fused_combine;
+  const bool decode_zeroes_empty_rows = persistent || fused;
+  const int32_t n_empty = int32_t(h->plan.empty.size());
+  const int32_t n_combine = int32_t(h->plan.combine.size());
+  const int32_t n_units = h->num_items * h->cfg.num_kv_heads;
+  if (n_units > 0 || (decode_zeroes_empty_rows && n_empty > 0)) {
     DecodeParams p;
     p.q = static_cast<const __nv_bfloat16*>(q);
     p.block_table = block_table;
@@ -535,6 +590,7 @@ int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, cons
     p.partial_o = reinterpret_cast<float*>(ws + h->o_off);
     p.partial_lse = reinterpret_cast<float*>(ws + h->lse_off);
     p.error_word = err_dev;
+    p.counters = reinterpret_cast<int32_t*>(ws + h->cnt_off);
     p.num_pages = h->cfg.num_pages;
     p.num_q_heads = h->cfg.num_q_heads;
     p.num_kv_heads = h->cfg.num_kv_heads;
@@ -543,16 +599,26 @@ int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, cons
     p.scale_log2 = h->scale_log2;
     p.pos_head = h->pos_head;
     p.pos_page = h->pos_page;
-    const Variant& v = variants()[h->variant];
-    const int di = (h->cfg.head_dim == 128) ? 1 : 0;
-    const int ni = (h->group > 8) ? 1 : 0;
-    const unsigned grid = unsigned(h->num_items) * unsigned(h->cfg.num_kv_heads);
-    v.fn[di][ni]<<<grid, v.warps * 32, v.smem[di], st>>>(pm->map_k, pm->map_v, p);
+    p.num_units = n_units;
+    p.num_empty = decode_zeroes_empty_rows ? n_empty : 0;
+    p.fused_combine = fused ? 1 : 0;
+#ifdef LIBRA_TRACE
+    p.trace = reinterpret_cast<unsigned long long*>(ws + h->workspace_bytes);
+#endif
+    unsigned grid;
+    if (persistent) {
+      const int slots = h->params.n_sm * h->params.ctas_per_sm;
+      grid = unsigned(std::max(1, std::min(n_units, slots)));
+    } else {
+      grid = unsigned(n_units) + unsigned(p.num_empty);
+    }
+    v.fn[di][ni]<<<grid, v.warps * 32, v.smem[di][ni], st>>>(pm->map_k, pm->map_v, p);
     LIBRA_CUDA_TRY(h, cudaGetLastError());
     ++h->launches;
   }
   if (ev) LIBRA_CUDA_TRY(h, cudaEventRecord(ev[1], st));
-  if (h->num_fix > 0) {
+  const int32_t n_entries = decode_zeroes_empty_rows ? n_combine : h->num_fix;  // merges come first in the list
+  if (!fused && n_entries > 0) {
     libra::CombineParams c;
     c.plan = plan_dev;
     c.partial_o = reinterpret_cast<const float*>(ws + h->o_off);
@@ -561,9 +627,9 @@ int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, cons
     c.out = static_cast<__nv_bfloat16*>(out);
     c.error_word = err_dev;
     c.num_q_heads = h->cfg.num_q_heads;
-    c.head_dim = h->cfg.head_dim;
-    dim3 grid(unsigned(h->num_fix), unsigned(h->cfg.num_q_heads));
-    libra::combine_kernel<<<grid, h->cfg.head_dim / 2, 0, st>>>(c);
+    dim3 grid(unsigned(n_entries), unsigned((h->cfg.num_q_heads + libra::kCombineWarps - 1) / libra::kCombineWarps));
+    if (h->cfg.head_dim == 128) libra::combine_kernel<128><<<grid, libra::kCombineWarps * 32, 0, st>>>(c);
+    else libra::combine_kernel<64><<<grid, libra::kCombineWarps * 32, 0, st>>>(c);
     LIBRA_CUDA_TRY(h, cudaGetLastError());
     ++h->launches;
   }

@@ -24,7 +24,7 @@ class Runner:
     """One handle + workspace for one shape; run() executes plan + decode on the current stream."""
 
     def __init__(self, binding, Hq, Hkv, d, num_pages, max_batch, ld, layout="HND", plan=None, sm_scale=0.0,
-                 variant=None):
+                 variant=None, fused=None):
         import torch
         self.torch = torch
         self.dev = torch.device("cuda:0")
@@ -35,6 +35,8 @@ class Runner:
                                 plan=plan)
         if variant is not None:
             self.h.set_variant(*variant)
+        if fused is not None:
+            self.h.set_combine_mode(fused)
         self.ws = torch.empty(self.h.workspace_size(), dtype=torch.uint8, device=self.dev)
         self.shape = (Hq, d)
 
@@ -55,7 +57,7 @@ class Runner:
         return out
 
 
-def run_host_case(binding, q, k, v, bt, lens, layout="HND", plan=None, sm_scale=0.0, variant=None):
+def run_host_case(binding, q, k, v, bt, lens, layout="HND", plan=None, sm_scale=0.0, variant=None, fused=None):
     """Host uint16 inputs (HND order; transposed here for NHD) -> float32 output [B, Hq, d]."""
     import torch
     dev = torch.device("cuda:0")
@@ -64,7 +66,7 @@ def run_host_case(binding, q, k, v, bt, lens, layout="HND", plan=None, sm_scale=
     if layout == "NHD":
         k = np.ascontiguousarray(k.transpose(0, 2, 1, 3))
         v = np.ascontiguousarray(v.transpose(0, 2, 1, 3))
-    r = Runner(binding, Hq, Hkv, d, k.shape[0], max(B, 1), bt.shape[1], layout, plan, sm_scale, variant)
+    r = Runner(binding, Hq, Hkv, d, k.shape[0], max(B, 1), bt.shape[1], layout, plan, sm_scale, variant, fused)
     out = r.run(to_dev(q, dev), to_dev(k, dev), to_dev(v, dev), to_dev(bt, dev), lens)
     res = bf16_dev_to_f32(out)
     r.h.close()

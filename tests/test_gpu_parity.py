@@ -63,15 +63,20 @@ def test_shapes_and_tails(lib, case, layout):
     for plan in (None, small_plan(lib)):
         got = H.run_host_case(lib, q, k, v, bt, lens_a, layout=layout, plan=plan)
         check(got, ref, f"case {case} {layout} plan={'default' if plan is None else 'small'}")
+    # step C as its own kernel gives the same bits as step C inside the decode kernel
+    two = H.run_host_case(lib, q, k, v, bt, lens_a, layout=layout, plan=small_plan(lib), fused=False)
+    assert np.array_equal(two, got)
 
 
 def test_every_block_shape_agrees(lib):
     lens = [2500, 300, 17, 4100]
     lens_a, bt, q, k, v = W.random_case(7, 4, 32, 8, 128, lens)
     ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
-    for variant in [(4, 3), (4, 2), (4, 4), (4, 6), (8, 2), (8, 3), (2, 6), (2, 4)]:
-        got = H.run_host_case(lib, q, k, v, bt, lens_a, plan=lib.PlanParams(8, 1, 2, 256, 256, 64), variant=variant)
-        check(got, ref, f"variant {variant}")
+    for sched in (0, 1):
+        for shape in [(4, 3), (4, 2), (4, 4), (4, 6), (8, 2), (8, 3), (2, 6), (2, 4)]:
+            variant = (sched,) + shape
+            got = H.run_host_case(lib, q, k, v, bt, lens_a, plan=lib.PlanParams(8, 1, 2, 256, 256, 64), variant=variant)
+            check(got, ref, f"variant {variant}")
 
 
 def test_custom_scale(lib):
@@ -187,10 +192,19 @@ def test_nan_garbage_outside_sequences_is_ignored(lib):
 
 
 def test_runs_are_bit_reproducible(lib):
+    import torch
+    dev = torch.device("cuda:0")
     lens_a, bt, q, k, v = W.random_case(29, 4, 32, 8, 128, [3000, 200, 4500, 1])
     a = H.run_host_case(lib, q, k, v, bt, lens_a)
     b = H.run_host_case(lib, q, k, v, bt, lens_a)
     assert np.array_equal(a, b)
+    # many launches on one handle: the arrival counters of the in-kernel combine reset themselves
+    r = H.Runner(lib, 32, 8, 128, k.shape[0], 4, bt.shape[1], plan=lib.PlanParams(8, 1, 2, 256, 256, 64))
+    args = [H.to_dev(x, dev) for x in (q, k, v, bt)]
+    first = H.bf16_dev_to_f32(r.run(*args, lens_a))
+    for _ in range(20):
+        assert np.array_equal(H.bf16_dev_to_f32(r.run(*args, lens_a)), first)
+    r.h.close()
 
 
 # ------------------------------------------------------------------ device-side checks, host-visible errors
