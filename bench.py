@@ -44,8 +44,8 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES_ASSUMED = 126 * 1024 * 1024
 # DRAM bytes (read + write) of one decode-kernel launch on MAIN_WORKLOAD from an ncu capture, see
-# profiles/; None until a capture has been taken.
-NCU_DECODE_TRAFFIC_BYTES = None
+# profiles/decode_kernel_lognormal_b64.md (370.61 MB read + 4.20 MB written).
+NCU_DECODE_TRAFFIC_BYTES = 374.8e6
 
 
 # ----------------------------------------------------------------------------- clocks

@@ -74,7 +74,7 @@ typedef enum {
 typedef struct {
   int32_t n_sm;           /* SMs to plan for; 0 = the device's count (148 on B200)               */
   int32_t ctas_per_sm;    /* resident decode blocks per SM the plan assumes; default 2           */
-  int32_t items_per_slot; /* target work items per resident block; default 4                    */
+  int32_t items_per_slot; /* target work units per resident block; default 1                    */
   int32_t chunk_align;    /* A: chunk lengths are multiples of this many tokens (itself a
                              multiple of 16); default 256                                       */
   int32_t min_chunk;      /* C_min: lower bound of the base chunk length; default 512           */
@@ -133,8 +133,8 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg);
 int libra_destroy(libra_handle_t handle);
 
 /* Bytes of device workspace that libra_plan / libra_decode_attn need for any batch <= max_batch.
- * The workspace holds the uploaded plan, the device error word and the fp32 partial results of
- * split sequences.  It must be 256-byte aligned. */
+ * The workspace holds the device error word, arrival counters, the fp32 partial results of split
+ * sequences and room for a plan too large for the kernel parameters.  It must be 256-byte aligned. */
 int libra_workspace_size(libra_handle_t handle, size_t* bytes);
 
 /* The planner constants the handle uses, defaults resolved (n_sm = the device's SM count). */
@@ -173,10 +173,13 @@ int libra_plan_host(const libra_plan_params_t* params, int32_t num_kv_heads, con
                     int32_t* num_items, int32_t* combine, int32_t* num_combine, int32_t* empty,
                     int32_t* num_empty);
 
-/* Step P for a handle: plan `batch` sequences from host lengths and upload the plan into the
- * workspace with one asynchronous copy on `stream` (from a pinned staging buffer owned by the
- * handle; two buffers alternate, and a buffer is reused only after its previous upload finished).
- * The plan also resets the device error word.  seq_lens_host: host pointer, int32[batch].
+/* Step P for a handle: plan `batch` sequences from host lengths.  The plan is kept in the handle
+ * and travels to the GPU inside the kernel parameters of every later libra_decode_attn, so in the
+ * usual case nothing is copied here.  Only a plan of more than 768 work items (or more than 256 split
+ * sequences) is uploaded into the workspace, with one asynchronous copy on `stream` from a pinned
+ * staging buffer owned by the handle (two buffers alternate; one is reused only after its previous
+ * upload finished).  The first plan into a given workspace also clears the workspace's control
+ * words and arrival counters on `stream`.  seq_lens_host: host pointer, int32[batch].
  * Errors: INVALID_ARGUMENT, WORKSPACE_TOO_SMALL, CUDA_ERROR. */
 int libra_plan(libra_handle_t handle, const int32_t* seq_lens_host, int32_t batch, void* workspace_dev,
                size_t workspace_bytes, void* stream);
@@ -189,7 +192,7 @@ int libra_plan_export(libra_handle_t handle, libra_plan_view_t* view);
  * textbook definition).  All pointers are device pointers; the plan last uploaded by libra_plan
  * into `workspace` is used and `seq_lens` (device) must hold the planned lengths (a mismatch
  * sets LIBRA_ERR_SEQ_LEN_MISMATCH in the error word).  Launches the split-KV decode kernel (and, in
- * the two-launch combine mode, the combine kernel if any sequence is split or empty) on `stream`;
+ * the two-launch combine mode, the combine kernel if any sequence is split) on `stream`;
  * returns without waiting.
  * Results are bit-reproducible run to run (fixed reduction order, no floating-point atomics).
  * The workspace also holds per-sequence arrival counters that the kernels leave at zero; a call that
@@ -218,7 +221,8 @@ int libra_host_staging_size(libra_handle_t handle, int32_t batch, size_t* bytes)
 int libra_last_cuda_error(libra_handle_t handle);
 
 /* Copy the device error word of the last planned workspace to *word (synchronises `stream` of the
- * last call first).  0 = no kernel recorded a problem.  Errors: NOT_PLANNED, CUDA_ERROR. */
+ * last call first).  0 = no kernel recorded a problem.  The word accumulates over launches; reading
+ * a non-zero word clears it.  Errors: NOT_PLANNED, CUDA_ERROR. */
 int libra_debug_error_word(libra_handle_t handle, uint32_t* word);
 
 /* Per-kernel timing for benchmarks.  After libra_profile_begin, every libra_decode_attn records

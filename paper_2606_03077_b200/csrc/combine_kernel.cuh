@@ -2,8 +2,7 @@
 //
 // For sequence b, head h with n partials (O_i normalised, LSE_i natural log):
 //   M = max_i LSE_i ;  w_i = exp(LSE_i - M) ;  out = sum_i w_i O_i / sum_i w_i   -> bf16
-// Partials are summed in chunk order, so the result does not depend on scheduling.  An entry with
-// n == 0 is an empty sequence: its output row is zero.
+// Partials are summed in chunk order, so the result does not depend on scheduling.
 //
 // One warp per (sequence, head): lane i keeps w_i and w_{i+32}; every lane owns D/32 output
 // columns and walks the n partial rows with eight independent loads in flight.
@@ -18,7 +17,7 @@
 namespace libra {
 
 struct CombineParams {
-  const int32_t* plan;
+  const int4* entries;       // merges {b, first_slot, n, planned_len} in device memory, or null: in `pf`
   const float* partial_o;    // [slot][Hq][D]
   const float* partial_lse;  // [slot][Hq]
   const int32_t* seq_lens;
@@ -31,22 +30,26 @@ constexpr int kCombineWarps = 4;
 
 // grid = (fix-up entries, ceil(Hq / kCombineWarps)), block = kCombineWarps warps
 template <int D>
-__global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const CombineParams p) {
+__global__ void __launch_bounds__(kCombineWarps * 32)
+combine_kernel(const __grid_constant__ CombineParams p, const __grid_constant__ ParamFix pf) {
   constexpr int V = D / 32;  // columns per lane: 4 (float4) or 2 (float2)
   const int lane = threadIdx.x & 31;
   const int h = blockIdx.y * kCombineWarps + (threadIdx.x >> 5);
   const int Hq = p.num_q_heads;
   if (h >= Hq) return;
-  const int32_t* fix = p.plan + __ldg(p.plan + plan_layout::kFixOff) + blockIdx.x * plan_layout::kFixInts;
-  const int b = __ldg(fix + 0);
-  const int first = __ldg(fix + 1);
-  const int n = __ldg(fix + 2);  // <= 64
-  if (lane == 0 && h == 0 && __ldg(fix + 3) != __ldg(p.seq_lens + b)) {
+  const int4 fix = (p.entries ? p.entries : pf.e)[blockIdx.x];  // plain load: may address parameter space
+  const int b = fix.x;
+  const int first = fix.y;
+  const int n = fix.z;  // <= 64
+  // launched as a programmatic dependent of the decode kernel: wait until that grid has finished
+  // and its partial results are visible
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (lane == 0 && h == 0 && fix.w != __ldg(p.seq_lens + b)) {
     atomicOr(p.error_word, LIBRA_DEV_ERR_SEQ_LEN_MISMATCH);
   }
   const float* lse = p.partial_lse + int64_t(first) * Hq + h;
-  const float l0 = (lane < n) ? __ldg(lse + int64_t(lane) * Hq) : -INFINITY;
-  const float l1 = (lane + 32 < n) ? __ldg(lse + int64_t(lane + 32) * Hq) : -INFINITY;
+  const float l0 = (lane < n) ? __ldcg(lse + int64_t(lane) * Hq) : -INFINITY;
+  const float l1 = (lane + 32 < n) ? __ldcg(lse + int64_t(lane + 32) * Hq) : -INFINITY;
   float m = fmaxf(l0, l1);
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
@@ -65,10 +68,10 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const Combi
     for (int k = 0; k < 8; ++k) {
       if (i0 + k < n) {
         if constexpr (V == 4) {
-          const float4 x = __ldg(reinterpret_cast<const float4*>(po + (i0 + k) * stride));
+          const float4 x = __ldcg(reinterpret_cast<const float4*>(po + (i0 + k) * stride));
           o[k][0] = x.x; o[k][1] = x.y; o[k][2] = x.z; o[k][3] = x.w;
         } else {
-          const float2 x = __ldg(reinterpret_cast<const float2*>(po + (i0 + k) * stride));
+          const float2 x = __ldcg(reinterpret_cast<const float2*>(po + (i0 + k) * stride));
           o[k][0] = x.x; o[k][1] = x.y;
         }
       } else {

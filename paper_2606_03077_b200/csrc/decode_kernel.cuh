@@ -43,7 +43,7 @@ struct DecodeParams {
   const int32_t* block_table;
   const int32_t* seq_lens;
   __nv_bfloat16* out;
-  const int32_t* plan;   // device plan blob (plan_layout.hpp)
+  const int4* entries;   // work items then empty-sequence entries in device memory, or null: in `pp`
   float* partial_o;      // [slot][Hq][D]
   float* partial_lse;    // [slot][Hq]
   uint32_t* error_word;
@@ -56,6 +56,7 @@ struct DecodeParams {
   float scale_log2;       // sm_scale * log2(e)
   int32_t pos_head;       // coordinate slot (1..3) of the head / page dimension in the tensor maps
   int32_t pos_page;
+  int32_t num_items;
   int32_t num_units;      // work items x KV heads
   int32_t num_empty;      // empty sequences whose output row this launch zeroes
   int32_t fused_combine;  // 1: the last block of a split sequence merges its partials (step C) itself
@@ -381,14 +382,15 @@ __device__ __forceinline__ void check_planned_length(const DecodeParams& p, cons
   if (!ok) atomicOr(p.error_word, LIBRA_DEV_ERR_SEQ_LEN_MISMATCH);
 }
 
-// Output rows of empty sequences are zero; entry e of the plan's empty list.
+// Output rows of empty sequences are zero; entry e of the plan's empty list (stored after the items).
 template <int D>
-__device__ __forceinline__ void zero_empty_row(const DecodeParams& p, int e, int tid, int nthreads) {
-  const int32_t* fix = p.plan + __ldg(p.plan + plan_layout::kFixOff) +
-                       (__ldg(p.plan + plan_layout::kNumCombine) + e) * plan_layout::kFixInts;
-  const int64_t row = int64_t(__ldg(fix)) * p.num_q_heads * D;
+__device__ __forceinline__ void zero_empty_row(const DecodeParams& p, const int4* entries, int e, int tid, int nthreads) {
+  const int64_t row = int64_t(entries[p.num_items + e].x) * p.num_q_heads * D;
   for (int i = tid; i < p.num_q_heads * D; i += nthreads) p.out[row + i] = __float2bfloat16_rn(0.f);
 }
+
+// Lets a dependent launch (the combine kernel) be scheduled early; it still waits for this grid to finish.
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 }  // namespace dev
 
@@ -406,7 +408,8 @@ struct DecodeSmem {
 // D: head_dim (64 | 128); NT: 8-wide head tiles (1: G <= 8, 2: G <= 16); NW warps; STAGES per warp.
 template <int D, int NT, int NW, int STAGES>
 __global__ void __launch_bounds__(NW * 32)
-decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const DecodeParams p) {
+decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+              const __grid_constant__ DecodeParams p, const __grid_constant__ ParamPlan pp) {
   using namespace dev;
   using SM = DecodeSmem<D, NW, STAGES>;
   constexpr int NH = D / 64;   // 128-byte column blocks of a row
@@ -426,8 +429,12 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   const uint32_t my_ring_u32 = smem_u32(my_ring);
   const uint32_t my_bar0 = smem_u32(&bars[warp * STAGES]);
 
+  launch_dependents();
+  // the plan lives in the kernel parameters unless it was too large for them (plain loads: the
+  // pointer may address parameter space)
+  const int4* entries = p.entries ? p.entries : pp.e;
   if (int(blockIdx.x) >= p.num_units) {
-    zero_empty_row<D>(p, int(blockIdx.x) - p.num_units, threadIdx.x, NW * 32);
+    zero_empty_row<D>(p, entries, int(blockIdx.x) - p.num_units, threadIdx.x, NW * 32);
     return;
   }
 
@@ -438,7 +445,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   // ---- work unit
   const int item_idx = blockIdx.x / p.num_kv_heads;
   const int kvh = blockIdx.x - item_idx * p.num_kv_heads;
-  const Unit u = decode_unit<NW>(__ldg(reinterpret_cast<const int4*>(p.plan + plan_layout::kHeaderInts) + item_idx), kvh, warp);
+  const Unit u = decode_unit<NW>(entries[item_idx], kvh, warp);
   const int n_it = u.n_it;
   if (threadIdx.x == 0) check_planned_length(p, u, __ldg(p.seq_lens + u.b));
 
@@ -601,7 +608,7 @@ struct PersistentSmem {
 template <int D, int NT, int NW, int STAGES>
 __global__ void __launch_bounds__(NW * 32)
 decode_persistent_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                         const DecodeParams p) {
+                         const __grid_constant__ DecodeParams p, const __grid_constant__ ParamPlan pp) {
   using namespace dev;
   using SM = DecodeSmem<D, NW, STAGES>;
   using PS = PersistentSmem<D, NT, NW, STAGES>;
@@ -612,6 +619,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
   __shared__ float stat_m[NW][NT * 8];
   __shared__ float stat_l[NW][NT * 8];
 
+  launch_dependents();
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int W = gridDim.x;
@@ -635,10 +643,10 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
     const int u = k * W + ((k & 1) ? (W - 1 - c) : c);
     return (u < p.num_units) ? u : -1;
   };
-  const int4* items = reinterpret_cast<const int4*>(p.plan + plan_layout::kHeaderInts);
+  const int4* items = p.entries ? p.entries : pp.e;  // plain loads: may address parameter space
   auto load_item = [&](int k) -> int4 {
     const int u = unit_index(k);
-    return (u >= 0) ? __ldg(items + u / p.num_kv_heads) : make_int4(0, 0, 0, -1);
+    return (u >= 0) ? items[u / p.num_kv_heads] : make_int4(0, 0, 0, -1);
   };
   auto make_unit = [&](int k, const int4 raw) -> Unit {
     const int u = unit_index(k);
@@ -796,7 +804,7 @@ decode_persistent_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
     // bounded last chance for copies still in flight to land before the block exits
     for (uint32_t k = consumed; k < issued; ++k) (void)mbar_wait(my_bar0 + 8 * (k % STAGES), (k / STAGES) & 1u);
   }
-  for (int e = c; e < p.num_empty; e += W) zero_empty_row<D>(p, e, threadIdx.x, NW * 32);
+  for (int e = c; e < p.num_empty; e += W) zero_empty_row<D>(p, items, e, threadIdx.x, NW * 32);
 }
 
 }  // namespace libra

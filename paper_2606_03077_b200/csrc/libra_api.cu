@@ -27,7 +27,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-typedef void (*DecodeKernelFn)(const CUtensorMap, const CUtensorMap, const DecodeParams);
+typedef void (*DecodeKernelFn)(const CUtensorMap, const CUtensorMap, const DecodeParams, const libra::ParamPlan);
 
 struct Variant {
   int persistent, warps, stages;
@@ -117,13 +117,14 @@ struct libra_handle_s {
   int variant = 0;
   EncodeTiledFn encode = nullptr;
 
-  // workspace layout
+  // workspace layout: control words | arrival counters | partial LSE | partial O | oversized plans
   int64_t max_items = 0;
-  size_t plan_bytes = 0, cnt_off = 0, cnt_bytes = 0, lse_off = 0, o_off = 0, workspace_bytes = 0;
-  void* clean_workspace = nullptr;  // workspace whose arrival counters are known to be zero
+  size_t cnt_off = 0, cnt_bytes = 0, lse_off = 0, o_off = 0, plan_off = 0, plan_bytes = 0, workspace_bytes = 0;
+  void* clean_workspace = nullptr;  // workspace whose control words and counters are known to be zero
   bool fused_combine = false;
+  bool pdl_combine = true;
 
-  // pinned staging for plan uploads
+  // pinned staging for uploads of plans too large for the kernel parameters
   int32_t* staging[2] = {nullptr, nullptr};
   cudaEvent_t staging_done[2] = {nullptr, nullptr};
   bool staging_used[2] = {false, false};
@@ -134,8 +135,11 @@ struct libra_handle_s {
   libra::HostPlan plan;
   std::vector<int32_t> items_flat;
   void* workspace = nullptr;
-  int32_t num_items = 0, num_fix = 0;
+  int32_t num_items = 0;
   void* last_stream = nullptr;
+  bool plan_in_params = true;   // the usual case: the plan travels with every launch
+  libra::ParamPlan pp;          // work items, then one entry per empty sequence
+  libra::ParamFix pf;           // merges for the combine kernel
 
   // tensor maps of the pools seen most recently (callers often rotate between a few pools)
   struct PoolMaps {
@@ -357,14 +361,13 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
     if (status != LIBRA_OK) break;
 
     h->max_items = libra::max_items(h->params, cfg->num_kv_heads, cfg->max_batch);
-    const size_t plan_ints = size_t(libra::plan_layout::kHeaderInts) + size_t(h->max_items) * libra::plan_layout::kItemInts +
-                             size_t(cfg->max_batch) * libra::plan_layout::kFixInts;
-    h->plan_bytes = align_up(plan_ints * 4, 256);
-    h->cnt_off = h->plan_bytes;
+    h->cnt_off = 256;  // the first 256 bytes hold the control words (the device error word)
     h->cnt_bytes = align_up(size_t(cfg->max_batch) * cfg->num_kv_heads * 4, 256);
     h->lse_off = h->cnt_off + h->cnt_bytes;
     h->o_off = h->lse_off + align_up(size_t(h->max_items) * cfg->num_q_heads * 4, 256);
-    h->workspace_bytes = h->o_off + align_up(size_t(h->max_items) * cfg->num_q_heads * cfg->head_dim * 4, 256);
+    h->plan_off = h->o_off + align_up(size_t(h->max_items) * cfg->num_q_heads * cfg->head_dim * 4, 256);
+    h->plan_bytes = align_up((size_t(h->max_items) + 2 * size_t(cfg->max_batch)) * sizeof(int4), 256);
+    h->workspace_bytes = h->plan_off + h->plan_bytes;
 
     for (int i = 0; i < 2; ++i) {
       if ((e = cudaHostAlloc(reinterpret_cast<void**>(&h->staging[i]), h->plan_bytes, cudaHostAllocDefault)) != cudaSuccess ||
@@ -433,57 +436,54 @@ int libra_plan(libra_handle_t h, const int32_t* seq_lens_host, int32_t batch, vo
 
   DeviceGuard guard(h->cfg.device);
   if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
-  const int k = h->next_staging;
-  if (h->staging_used[k]) LIBRA_CUDA_TRY(h, cudaEventSynchronize(h->staging_done[k]));
-
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
   namespace L = libra::plan_layout;
-  int32_t* blob = h->staging[k];
   const int32_t n_items = int32_t(pl.items.size());
-  const int32_t n_fix = int32_t(pl.combine.size() + pl.empty.size());
-  const int32_t fix_off = L::kHeaderInts + n_items * L::kItemInts;
-  std::memset(blob, 0, L::kHeaderInts * sizeof(int32_t));
-  blob[L::kMagic] = L::kMagicValue;
-  blob[L::kBatch] = batch;
-  blob[L::kNumItems] = n_items;
-  blob[L::kNumFix] = n_fix;
-  blob[L::kFixOff] = fix_off;
-  blob[L::kNumCombine] = int32_t(pl.combine.size());
+  const int32_t n_empty = int32_t(pl.empty.size());
+  const int32_t n_combine = int32_t(pl.combine.size());
+  h->plan_in_params = (n_items + n_empty <= L::kParamEntries) && (n_combine <= L::kParamFixEntries);
+
+  // entries: work items (longest first), then one entry per empty sequence; merges separately
+  int4* entries = h->pp.e;
+  int4* fixes = h->pf.e;
+  int k = 0;
+  if (!h->plan_in_params) {
+    k = h->next_staging;
+    if (h->staging_used[k]) LIBRA_CUDA_TRY(h, cudaEventSynchronize(h->staging_done[k]));
+    entries = reinterpret_cast<int4*>(h->staging[k]);
+    fixes = entries + n_items + n_empty;
+  }
   h->items_flat.resize(size_t(n_items) * 4);
   for (int32_t i = 0; i < n_items; ++i) {
     const libra::WorkItem& it = pl.items[i];
-    int32_t* w = blob + L::kHeaderInts + i * L::kItemInts;
-    w[0] = it.b | (it.j << L::kChunkShift) | (pl.num_splits[it.b] << L::kCountShift);
-    w[1] = it.kv_begin;
-    w[2] = it.kv_end;
-    w[3] = (pl.num_splits[it.b] > 1) ? pl.item_offset[it.b] + it.j : -1;
+    entries[i] = make_int4(it.b | (it.j << L::kChunkShift) | (pl.num_splits[it.b] << L::kCountShift), it.kv_begin,
+                           it.kv_end, (pl.num_splits[it.b] > 1) ? pl.item_offset[it.b] + it.j : -1);
     h->items_flat[4 * i + 0] = it.b;
     h->items_flat[4 * i + 1] = it.j;
     h->items_flat[4 * i + 2] = it.kv_begin;
     h->items_flat[4 * i + 3] = it.kv_end;
   }
-  int32_t* fx = blob + fix_off;
-  for (int32_t b : pl.combine) {
-    fx[0] = b; fx[1] = pl.item_offset[b]; fx[2] = pl.num_splits[b]; fx[3] = seq_lens_host[b];
-    fx += L::kFixInts;
+  for (int32_t e = 0; e < n_empty; ++e) entries[n_items + e] = make_int4(pl.empty[e], 0, 0, 0);
+  for (int32_t c = 0; c < n_combine; ++c) {
+    const int32_t b = pl.combine[c];
+    fixes[c] = make_int4(b, pl.item_offset[b], pl.num_splits[b], seq_lens_host[b]);
   }
-  for (int32_t b : pl.empty) {
-    fx[0] = b; fx[1] = 0; fx[2] = 0; fx[3] = 0;
-    fx += L::kFixInts;
-  }
-  const size_t bytes = size_t(fix_off + n_fix * L::kFixInts) * sizeof(int32_t);
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (h->clean_workspace != workspace_dev) {  // the kernels leave the counters at zero; a new workspace starts there
+
+  if (h->clean_workspace != workspace_dev) {  // control words and counters start at zero; the kernels keep the counters so
     h->clean_workspace = nullptr;
-    LIBRA_CUDA_TRY(h, cudaMemsetAsync(static_cast<uint8_t*>(workspace_dev) + h->cnt_off, 0, h->cnt_bytes, st));
+    LIBRA_CUDA_TRY(h, cudaMemsetAsync(workspace_dev, 0, h->cnt_off + h->cnt_bytes, st));
     h->clean_workspace = workspace_dev;
   }
-  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(workspace_dev, blob, bytes, cudaMemcpyHostToDevice, st));
-  LIBRA_CUDA_TRY(h, cudaEventRecord(h->staging_done[k], st));
-  h->staging_used[k] = true;
-  h->next_staging = k ^ 1;
+  if (!h->plan_in_params) {
+    const size_t bytes = size_t(n_items + n_empty + n_combine) * sizeof(int4);
+    LIBRA_CUDA_TRY(h, cudaMemcpyAsync(static_cast<uint8_t*>(workspace_dev) + h->plan_off, entries, bytes,
+                                      cudaMemcpyHostToDevice, st));
+    LIBRA_CUDA_TRY(h, cudaEventRecord(h->staging_done[k], st));
+    h->staging_used[k] = true;
+    h->next_staging = k ^ 1;
+  }
   h->workspace = workspace_dev;
   h->num_items = n_items;
-  h->num_fix = n_fix;
   h->last_stream = stream;
   h->planned = true;
   return LIBRA_OK;
@@ -556,8 +556,8 @@ int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, cons
   }
 
   uint8_t* ws = static_cast<uint8_t*>(h->workspace);
-  int32_t* plan_dev = reinterpret_cast<int32_t*>(ws);
-  uint32_t* err_dev = reinterpret_cast<uint32_t*>(plan_dev + libra::plan_layout::kErrorWord);
+  uint32_t* err_dev = reinterpret_cast<uint32_t*>(ws);
+  const int4* entries_dev = h->plan_in_params ? nullptr : reinterpret_cast<const int4*>(ws + h->plan_off);
 
   cudaEvent_t* ev = nullptr;
   if (h->profiling && h->profiled_calls < kMaxProfiledCalls) {
@@ -576,17 +576,16 @@ int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, cons
   const int ni = (h->group > 8) ? 1 : 0;
   const bool persistent = v.persistent != 0;
   const bool fused = !persistent && h->fused_combine;
-  const bool decode_zeroes_empty_rows = persistent || fused;
   const int32_t n_empty = int32_t(h->plan.empty.size());
   const int32_t n_combine = int32_t(h->plan.combine.size());
   const int32_t n_units = h->num_items * h->cfg.num_kv_heads;
-  if (n_units > 0 || (decode_zeroes_empty_rows && n_empty > 0)) {
+  if (n_units > 0 || n_empty > 0) {
     DecodeParams p;
     p.q = static_cast<const __nv_bfloat16*>(q);
     p.block_table = block_table;
     p.seq_lens = seq_lens;
     p.out = static_cast<__nv_bfloat16*>(out);
-    p.plan = plan_dev;
+    p.entries = entries_dev;
     p.partial_o = reinterpret_cast<float*>(ws + h->o_off);
     p.partial_lse = reinterpret_cast<float*>(ws + h->lse_off);
     p.error_word = err_dev;
@@ -599,8 +598,9 @@ int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, cons
     p.scale_log2 = h->scale_log2;
     p.pos_head = h->pos_head;
     p.pos_page = h->pos_page;
+    p.num_items = h->num_items;
     p.num_units = n_units;
-    p.num_empty = decode_zeroes_empty_rows ? n_empty : 0;
+    p.num_empty = n_empty;
     p.fused_combine = fused ? 1 : 0;
 #ifdef LIBRA_TRACE
     p.trace = reinterpret_cast<unsigned long long*>(ws + h->workspace_bytes);
@@ -610,27 +610,36 @@ int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, cons
       const int slots = h->params.n_sm * h->params.ctas_per_sm;
       grid = unsigned(std::max(1, std::min(n_units, slots)));
     } else {
-      grid = unsigned(n_units) + unsigned(p.num_empty);
+      grid = unsigned(n_units) + unsigned(n_empty);
     }
-    v.fn[di][ni]<<<grid, v.warps * 32, v.smem[di][ni], st>>>(pm->map_k, pm->map_v, p);
+    v.fn[di][ni]<<<grid, v.warps * 32, v.smem[di][ni], st>>>(pm->map_k, pm->map_v, p, h->pp);
     LIBRA_CUDA_TRY(h, cudaGetLastError());
     ++h->launches;
   }
   if (ev) LIBRA_CUDA_TRY(h, cudaEventRecord(ev[1], st));
-  const int32_t n_entries = decode_zeroes_empty_rows ? n_combine : h->num_fix;  // merges come first in the list
-  if (!fused && n_entries > 0) {
+  if (!fused && n_combine > 0) {
     libra::CombineParams c;
-    c.plan = plan_dev;
+    c.entries = h->plan_in_params ? nullptr : entries_dev + h->num_items + n_empty;
     c.partial_o = reinterpret_cast<const float*>(ws + h->o_off);
     c.partial_lse = reinterpret_cast<const float*>(ws + h->lse_off);
     c.seq_lens = seq_lens;
     c.out = static_cast<__nv_bfloat16*>(out);
     c.error_word = err_dev;
     c.num_q_heads = h->cfg.num_q_heads;
-    dim3 grid(unsigned(n_entries), unsigned((h->cfg.num_q_heads + libra::kCombineWarps - 1) / libra::kCombineWarps));
-    if (h->cfg.head_dim == 128) libra::combine_kernel<128><<<grid, libra::kCombineWarps * 32, 0, st>>>(c);
-    else libra::combine_kernel<64><<<grid, libra::kCombineWarps * 32, 0, st>>>(c);
-    LIBRA_CUDA_TRY(h, cudaGetLastError());
+    // a programmatic dependent of the decode kernel: it may be scheduled while that kernel drains and
+    // waits inside (griddepcontrol.wait) for it to finish
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(unsigned(n_combine), unsigned((h->cfg.num_q_heads + libra::kCombineWarps - 1) / libra::kCombineWarps));
+    lc.blockDim = dim3(libra::kCombineWarps * 32);
+    lc.dynamicSmemBytes = 0;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = (ev || !h->pdl_combine) ? 0 : 1;  // with events around it, it is an ordinary launch
+    if (h->cfg.head_dim == 128) LIBRA_CUDA_TRY(h, cudaLaunchKernelEx(&lc, libra::combine_kernel<128>, c, h->pf));
+    else LIBRA_CUDA_TRY(h, cudaLaunchKernelEx(&lc, libra::combine_kernel<64>, c, h->pf));
     ++h->launches;
   }
   if (ev) {
@@ -693,9 +702,9 @@ int libra_decode_attn_host(libra_handle_t h, const void* q_host, const void* k_p
   if (rc != LIBRA_OK) return rc;
   LIBRA_CUDA_TRY(h, cudaMemcpyAsync(out_host, d_out, q_bytes, cudaMemcpyDeviceToHost, st));
   uint32_t word = 0;
-  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(&word, static_cast<int32_t*>(workspace_dev) + libra::plan_layout::kErrorWord, 4,
-                                    cudaMemcpyDeviceToHost, st));
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(&word, workspace_dev, 4, cudaMemcpyDeviceToHost, st));
   LIBRA_CUDA_TRY(h, cudaStreamSynchronize(st));
+  if (word) LIBRA_CUDA_TRY(h, cudaMemsetAsync(workspace_dev, 0, 4, st));
   return word ? LIBRA_DEVICE_FLAGGED : LIBRA_OK;
 }
 
@@ -707,9 +716,9 @@ int libra_debug_error_word(libra_handle_t h, uint32_t* word) {
   DeviceGuard guard(h->cfg.device);
   if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
   cudaStream_t st = static_cast<cudaStream_t>(h->last_stream);
-  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(word, static_cast<int32_t*>(h->workspace) + libra::plan_layout::kErrorWord, 4,
-                                    cudaMemcpyDeviceToHost, st));
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(word, h->workspace, 4, cudaMemcpyDeviceToHost, st));
   LIBRA_CUDA_TRY(h, cudaStreamSynchronize(st));
+  if (*word) LIBRA_CUDA_TRY(h, cudaMemsetAsync(h->workspace, 0, 4, st));  // reading a set word clears it
   return LIBRA_OK;
 }
 
