@@ -217,6 +217,40 @@ int libra_decode_attn_host(libra_handle_t handle, const void* q_host, const void
 /* Bytes of device staging libra_decode_attn_host needs for `batch` sequences. */
 int libra_host_staging_size(libra_handle_t handle, int32_t batch, size_t* bytes);
 
+/* Size of the scratch region built into the library for libra_decode_attn_static: 8 MiB of device
+ * memory that every GPU holds from the moment it loads the library until the process exits. */
+#define LIBRA_STATIC_SCRATCH_BYTES (8u << 20)
+
+/* One whole step (P, D, C) without a caller-provided workspace and without any allocation.
+ * (The paper has no counterpart to this entry point; it exists for integration reasons only.)
+ *
+ * Who needs it: code that runs where device memory cannot be obtained any more -- an inference
+ * server that hands all free HBM to its KV-cache pool at start-up and runs with its allocator
+ * closed, a plug-in called from inside someone else's step loop where a cudaMalloc would
+ * synchronise the whole device and stall every stream, or a component that is simply not allowed to
+ * own device memory.  Such a caller still passes its inputs and its output buffer (device pointers,
+ * exactly as for libra_decode_attn, plus the host lengths that libra_plan takes); the workspace is
+ * a fixed LIBRA_STATIC_SCRATCH_BYTES region inside the library image instead.
+ *
+ * The call plans `batch` sequences, clears the part of the region that must start at zero (control
+ * words, arrival counters) on `stream`, and launches the same kernels as libra_decode_attn.  It calls
+ * no cudaMalloc / cudaFree / cudaHostAlloc and no other allocating CUDA routine.
+ *
+ * Limits and rules:
+ *  - the handle's shape must need no more than LIBRA_STATIC_SCRATCH_BYTES of workspace
+ *    (libra_workspace_size); otherwise WORKSPACE_TOO_SMALL is returned and nothing is launched;
+ *  - the first call on a device looks up the region's device address (once per device, kept for the
+ *    life of the process); make that first call outside of any stream capture;
+ *  - all handles and all calls on one device share the one region, which keeps the previous call's
+ *    contents: two calls whose kernels can overlap on the GPU (different streams, no ordering)
+ *    race on it and corrupt each other's results; issue them on one stream or order them with events;
+ *  - a device error word left by the previous call is cleared by the next call: read it
+ *    (libra_debug_error_word) in between if it matters.
+ * Errors: as libra_plan and libra_decode_attn. */
+int libra_decode_attn_static(libra_handle_t handle, const int32_t* seq_lens_host, int32_t batch, const void* q,
+                             const void* k_pages, const void* v_pages, const int32_t* block_table,
+                             const int32_t* seq_lens, void* out, void* stream);
+
 /* Last CUDA error code (cudaError_t as int) seen by this handle, 0 if none. */
 int libra_last_cuda_error(libra_handle_t handle);
 

@@ -18,6 +18,7 @@ if not os.path.exists(_LIB_PATH):
 lib = C.CDLL(_LIB_PATH)
 LIB_PATH = _LIB_PATH
 
+STATIC_SCRATCH_BYTES = 8 << 20
 OK, INVALID_ARGUMENT, UNSUPPORTED_SHAPE, WORKSPACE_TOO_SMALL, NOT_PLANNED, CUDA_ERROR, DEVICE_FLAGGED = range(7)
 ERR_WAIT_TIMEOUT, ERR_BAD_PAGE_ID, ERR_SEQ_LEN_MISMATCH = 1, 2, 4
 
@@ -64,6 +65,7 @@ SIGNATURES = {
     "libra_decode_attn": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_decode_attn_host": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, C.c_int32, _vp, _vp, C.c_size_t, _vp,
                                          C.c_size_t, _vp]),
+    "libra_decode_attn_static": (C.c_int, [_vp, _i32p, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_host_staging_size": (C.c_int, [_vp, C.c_int32, C.POINTER(C.c_size_t)]),
     "libra_last_cuda_error": (C.c_int, [_vp]),
     "libra_debug_error_word": (C.c_int, [_vp, C.POINTER(C.c_uint32)]),
@@ -180,6 +182,15 @@ class Handle:
                     out_ptr: int, stream: int) -> None:
         _check(lib.libra_decode_attn(self._h, q_ptr, k_ptr, v_ptr, block_table_ptr, seq_lens_ptr, out_ptr, stream),
                "libra_decode_attn")
+
+    def decode_attn_static(self, seq_lens_host: np.ndarray, q_ptr: int, k_ptr: int, v_ptr: int,
+                           block_table_ptr: int, seq_lens_ptr: int, out_ptr: int, stream: int) -> None:
+        """Plan + decode + combine on the scratch region built into the library: no workspace argument
+        and no allocation.  Calls on one device share that region, so they must not overlap on the GPU."""
+        lens = _as_i32(seq_lens_host)
+        _check(lib.libra_decode_attn_static(self._h, lens.ctypes.data_as(_i32p), int(lens.shape[0]), q_ptr, k_ptr,
+                                            v_ptr, block_table_ptr, seq_lens_ptr, out_ptr, stream),
+               "libra_decode_attn_static")
 
     def host_staging_size(self, batch: int) -> int:
         n = C.c_size_t(0)

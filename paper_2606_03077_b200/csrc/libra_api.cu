@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <mutex>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -216,6 +217,31 @@ int encode_pool_map(libra_handle_t h, const void* base, CUtensorMap* map, int* p
     return LIBRA_CUDA_ERROR;
   }
   return LIBRA_OK;
+}
+
+// ---- built-in scratch for libra_decode_attn_static --------------------------------------------
+// A fixed region of device memory that is part of the loaded library image on every GPU, used as the
+// workspace by callers that cannot provide one.  In host code `g_static_scratch` is only a handle
+// for the symbol, not a device address: the address each device gives it is looked up once per
+// device with cudaGetSymbolAddress and that pointer is what the kernels receive.
+static __device__ __align__(256) unsigned char g_static_scratch[LIBRA_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_ptr[kMaxDevices] = {};
+
+// Device address of the built-in scratch on `device`, which must be the current device.
+cudaError_t static_scratch_address(int device, void** ptr) {
+  if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_ptr[device]) {
+    void* p = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_scratch_ptr[device] = p;
+  }
+  *ptr = g_scratch_ptr[device];
+  return cudaSuccess;
 }
 
 }  // namespace
@@ -706,6 +732,26 @@ int libra_decode_attn_host(libra_handle_t h, const void* q_host, const void* k_p
   LIBRA_CUDA_TRY(h, cudaStreamSynchronize(st));
   if (word) LIBRA_CUDA_TRY(h, cudaMemsetAsync(workspace_dev, 0, 4, st));
   return word ? LIBRA_DEVICE_FLAGGED : LIBRA_OK;
+}
+
+int libra_decode_attn_static(libra_handle_t h, const int32_t* seq_lens_host, int32_t batch, const void* q,
+                             const void* k_pages, const void* v_pages, const int32_t* block_table,
+                             const int32_t* seq_lens, void* out, void* stream) {
+  if (!h) return LIBRA_INVALID_ARGUMENT;
+  if (h->workspace_bytes > size_t(LIBRA_STATIC_SCRATCH_BYTES)) return LIBRA_WORKSPACE_TOO_SMALL;
+  void* scratch = nullptr;
+  {
+    DeviceGuard guard(h->cfg.device);  // the symbol's address is per device: look it up with that device current
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    const cudaError_t e = static_scratch_address(h->cfg.device, &scratch);
+    if (e != cudaSuccess) return fail_cuda(h, e);
+  }
+  // the region keeps whatever the previous call (of any handle) left: have the plan step clear the
+  // control words and arrival counters again, on `stream`, before the kernels run
+  h->clean_workspace = nullptr;
+  int rc = libra_plan(h, seq_lens_host, batch, scratch, size_t(LIBRA_STATIC_SCRATCH_BYTES), stream);
+  if (rc != LIBRA_OK) return rc;
+  return libra_decode_attn(h, q, k_pages, v_pages, block_table, seq_lens, out, stream);
 }
 
 int libra_last_cuda_error(libra_handle_t h) { return h ? h->last_cuda_error : 0; }
