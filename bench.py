@@ -352,7 +352,11 @@ def run_libra(args):
     dev = torch.device("cuda", local_rank)
     barrier = (lambda: torch.distributed.barrier()) if world > 1 else None
 
-    rep = Replica(args.workload, dev)
+    from paper_2606_03077_b200 import binding as _b
+
+    variant = tuple(int(x) for x in args.variant.split(",")) if args.variant else None
+    plan = _b.PlanParams(0, args.ctas_per_sm, args.items_per_slot, 0, 0, 0) if (args.ctas_per_sm or args.items_per_slot) else None
+    rep = Replica(args.workload, dev, plan=plan, variant=variant)
     sampler = ClockSampler(local_rank)
     sampler.start()
     elapsed_ms, launches = rep.timed(args.steps, args.warmup, barrier)
@@ -451,6 +455,9 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
+    ap.add_argument("--variant", default="", help="warps,stages of the decode block (default: the library's)")
+    ap.add_argument("--ctas-per-sm", type=int, default=0, help="planner constant (0 = default)")
+    ap.add_argument("--items-per-slot", type=int, default=0, help="planner constant (0 = default)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":

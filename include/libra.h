@@ -140,15 +140,11 @@ int libra_workspace_size(libra_handle_t handle, size_t* bytes);
 /* The planner constants the handle uses, defaults resolved (n_sm = the device's SM count). */
 int libra_get_plan_params(libra_handle_t handle, libra_plan_params_t* out);
 
-/* Tuning knob: schedule and shape of the decode kernel.  persistent = 0: one thread block per work
- * unit; persistent = 1: n_sm * ctas_per_sm resident blocks that deal the longest-first unit list
- * among themselves and keep their copies in flight across unit boundaries.  A block has `warps`
- * warps that each own `stages` shared-memory stages of one K page plus one V page.  Only the
- * compiled-in combinations that fit in shared memory for the handle's shape are accepted
- * (UNSUPPORTED_SHAPE otherwise); the default is the tuned one.  Results do not depend on the
- * schedule or the stage count; the warp count changes the order of the per-unit merge and hence
- * the last bits of the result.  With the persistent schedule step C always runs as its own kernel. */
-int libra_set_variant(libra_handle_t handle, int32_t persistent, int32_t warps, int32_t stages);
+/* Tuning knob: shape of the decode thread block: `warps` warps that each own `stages` shared-memory
+ * stages of one K page plus one V page.  Only the compiled-in shapes are accepted (UNSUPPORTED_SHAPE
+ * otherwise); the default is the tuned one.  Results do not depend on the stage count; the warp
+ * count changes the order of the per-unit merge and hence the last bits of the result. */
+int libra_set_variant(libra_handle_t handle, int32_t warps, int32_t stages);
 
 /* Where step C runs.  fused = 1: inside the decode kernel, by the block that publishes the
  * last partial result of a split sequence (one launch per call).  fused = 0 (default): as a separate combine

@@ -56,7 +56,7 @@ SIGNATURES = {
     "libra_destroy": (C.c_int, [_vp]),
     "libra_workspace_size": (C.c_int, [_vp, C.POINTER(C.c_size_t)]),
     "libra_get_plan_params": (C.c_int, [_vp, C.POINTER(PlanParams)]),
-    "libra_set_variant": (C.c_int, [_vp, C.c_int32, C.c_int32, C.c_int32]),
+    "libra_set_variant": (C.c_int, [_vp, C.c_int32, C.c_int32]),
     "libra_set_combine_mode": (C.c_int, [_vp, C.c_int32]),
     "libra_plan_host": (C.c_int, [C.POINTER(PlanParams), C.c_int32, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p,
                                   _i32p, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p]),
@@ -158,8 +158,8 @@ class Handle:
         _check(lib.libra_get_plan_params(self._h, C.byref(p)), "libra_get_plan_params")
         return p
 
-    def set_variant(self, persistent: int, warps: int, stages: int) -> None:
-        _check(lib.libra_set_variant(self._h, int(persistent), warps, stages), "libra_set_variant")
+    def set_variant(self, warps: int, stages: int) -> None:
+        _check(lib.libra_set_variant(self._h, warps, stages), "libra_set_variant")
 
     def set_combine_mode(self, fused: bool) -> None:
         _check(lib.libra_set_combine_mode(self._h, 1 if fused else 0), "libra_set_combine_mode")

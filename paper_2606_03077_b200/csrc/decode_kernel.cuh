@@ -1,4 +1,4 @@
-// Split-KV decode kernels (step D) for sm_100a.
+// Split-KV decode kernel (step D) for sm_100a.
 //
 // A work unit is one work item of the plan (a chunk [kv_begin, kv_end) of one sequence) for one KV
 // head and all G query heads that share it.  Inside a thread block every warp owns a private ring
@@ -11,18 +11,11 @@
 //            O^T[d x 8 heads]         += V_page^T . P^T     P rounded to bf16, l sums the rounded P
 //
 // Tokens are the M side of the tiles, the (padded) head group the N side, so a group of up to
-// 8 heads costs one 8-wide tile and nothing is wasted on padding rows.  The kernels are bound by
+// 8 heads costs one 8-wide tile and nothing is wasted on padding rows.  The kernel is bound by
 // the HBM read of K and V: 2 * head_dim * 2 bytes per token per KV head, 4 * G * head_dim flop.
 //
 // The warps never synchronise with each other while they stream pages; they merge their (m, l, O)
 // in shared memory once per unit, in warp order, so results are bit-reproducible.
-//
-// Two schedules:
-//   decode_kernel             one thread block per unit, units in plan order (longest first)
-//   decode_persistent_kernel  one resident block per slot; block c takes units c, 2W-1-c, 2W+c, ...
-//                             of the longest-first list (W blocks, serpentine deal) and every warp
-//                             keeps its copy ring full ACROSS unit boundaries, so the loads of the
-//                             next unit are in flight while the current unit is merged and written
 //
 // Step C can run inside decode_kernel: every block of a split sequence bumps a per-(sequence, KV
 // head) counter after publishing its partial result, and the block that arrives last merges all
@@ -60,9 +53,6 @@ struct DecodeParams {
   int32_t num_units;      // work items x KV heads
   int32_t num_empty;      // empty sequences whose output row this launch zeroes
   int32_t fused_combine;  // 1: the last block of a split sequence merges its partials (step C) itself
-#ifdef LIBRA_TRACE
-  unsigned long long* trace;  // timeline experiment only: 6 words per block, right after the workspace
-#endif
 };
 
 namespace dev {
@@ -142,9 +132,6 @@ __device__ __forceinline__ float lg2(float x) {
   float y;
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
-}
-__device__ __forceinline__ void named_barrier(int id, int threads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 // Byte offset of 16-byte chunk c16 of row r inside a [D/64][16][128 B] tile with 128-byte swizzle.
 __device__ __forceinline__ uint32_t tile_off(int r, int c16) {
@@ -438,10 +425,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     return;
   }
 
-#ifdef LIBRA_TRACE
-  unsigned long long tr0 = 0, tr1 = 0, tr2 = 0;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr0));
-#endif
   // ---- work unit
   const int item_idx = blockIdx.x / p.num_kv_heads;
   const int kvh = blockIdx.x - item_idx * p.num_kv_heads;
@@ -508,9 +491,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
       timed_out = true;
       break;
     }
-#ifdef LIBRA_TRACE
-    if (it == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr1));
-#endif
     const uint32_t kt = my_ring_u32 + s * SM::kStageBytes;
     const int tok0 = u.kv_begin + ((warp + it * NW) << 4);
     process_page<D, NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes, u.kv_end - tok0,
@@ -529,9 +509,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     for (int k = 0; k < STAGES; ++k) (void)mbar_wait(my_bar0 + 8 * k, parity);
   }
 
-#ifdef LIBRA_TRACE
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr2));
-#endif
   // ---- stage (m, l, O) of this warp in its own, now idle, ring; merge the warps; write
   __syncwarp();
   stage_warp_result<D, NT>(st, reinterpret_cast<float*>(my_ring), stat_m[warp], stat_l[warp], lane);
@@ -539,16 +516,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   merge_and_write<D, NT, NW>(p, u, reinterpret_cast<const float*>(ring), SM::kWarpBytes / 4, &stat_m[0][0], &stat_l[0][0],
                              threadIdx.x, NW * 32);
 
-#ifdef LIBRA_TRACE
-  if (threadIdx.x == 0) {
-    unsigned long long tr3;
-    unsigned smid;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr3));
-    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-    unsigned long long* t = p.trace + 6ull * blockIdx.x;
-    t[0] = tr0; t[1] = tr1; t[2] = tr2; t[3] = tr3; t[4] = smid; t[5] = (unsigned long long)(u.kv_end - u.kv_begin);
-  }
-#endif
   // ---- step C inside this kernel: the block that publishes the last partial of (b, kvh) merges them
   if (u.slot < 0 || !p.fused_combine) return;
   const int G = p.group;
@@ -588,223 +555,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     for (int i = 0; i < u.n_chunks; ++i) num += w_sm[i * G + h] * __ldcg(po + int64_t(i) * p.num_q_heads * D);
     p.out[(int64_t(u.b) * p.num_q_heads + int64_t(kvh) * G + h) * D + dim] = __float2bfloat16_rn(num * inv_sm[h]);
   }
-}
-
-// ------------------------------------------------------------------------------------------------
-// Persistent schedule: gridDim.x resident blocks; block c takes units c, 2W-1-c, 2W+c, 4W-1-c, ...
-// of the longest-first list.  Every warp runs two cursors over its page stream: the issue cursor
-// keeps STAGES copies in flight and may run into the next unit (never further), the consume cursor
-// follows; the unit's descriptor, first page ids and query fragments of the next unit are loaded
-// while the current unit is still being consumed.  Shared memory: the copy rings plus one merge
-// area of NW x (NT*8 heads x D) floats.
-template <int D, int NT, int NW, int STAGES>
-struct PersistentSmem {
-  using Ring = DecodeSmem<D, NW, STAGES>;
-  static constexpr int kMergeWarpFloats = NT * 8 * D;
-  static constexpr int kMergeBytes = NW * kMergeWarpFloats * 4;
-  static constexpr int kDynamicBytes = Ring::kRingBytes + kMergeBytes + 1024;
-};
-
-template <int D, int NT, int NW, int STAGES>
-__global__ void __launch_bounds__(NW * 32)
-decode_persistent_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                         const __grid_constant__ DecodeParams p, const __grid_constant__ ParamPlan pp) {
-  using namespace dev;
-  using SM = DecodeSmem<D, NW, STAGES>;
-  using PS = PersistentSmem<D, NT, NW, STAGES>;
-  constexpr int NH = D / 64;
-
-  extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t bars[NW * STAGES];
-  __shared__ float stat_m[NW][NT * 8];
-  __shared__ float stat_l[NW][NT * 8];
-
-  launch_dependents();
-  const int warp = threadIdx.x >> 5;
-  const int lane = threadIdx.x & 31;
-  const int W = gridDim.x;
-  const int c = blockIdx.x;
-
-  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* my_ring = ring + warp * SM::kWarpBytes;
-  const uint32_t my_ring_u32 = smem_u32(my_ring);
-  const uint32_t my_bar0 = smem_u32(&bars[warp * STAGES]);
-  float* merge_sm = reinterpret_cast<float*>(ring + SM::kRingBytes);
-
-  if (lane == 0) {
-#pragma unroll
-    for (int s = 0; s < STAGES; ++s) mbar_init(my_bar0 + 8 * s, 1);
-    fence_mbar_init();
-  }
-  __syncwarp();
-
-  // unit index of this block's k-th unit (serpentine deal), -1 past the end
-  auto unit_index = [&](int k) -> int {
-    const int u = k * W + ((k & 1) ? (W - 1 - c) : c);
-    return (u < p.num_units) ? u : -1;
-  };
-  const int4* items = p.entries ? p.entries : pp.e;  // plain loads: may address parameter space
-  auto load_item = [&](int k) -> int4 {
-    const int u = unit_index(k);
-    return (u >= 0) ? items[u / p.num_kv_heads] : make_int4(0, 0, 0, -1);
-  };
-  auto make_unit = [&](int k, const int4 raw) -> Unit {
-    const int u = unit_index(k);
-    Unit r = decode_unit<NW>(raw, (u >= 0) ? (u % p.num_kv_heads) : 0, warp);
-    if (u < 0) r.n_it = 0;
-    return r;
-  };
-  auto load_ids = [&](const Unit& u, int round) -> int32_t {
-    const int idx = round * 32 + lane;
-    return (idx < u.n_it)
-               ? __ldg(p.block_table + int64_t(u.b) * p.block_table_ld + u.first_page + warp + int64_t(idx) * NW)
-               : -1;
-  };
-
-  // ---- issue cursor
-  int i_k = 0;                         // ordinal of the unit being issued
-  bool i_live = unit_index(0) >= 0;    // false once the issue cursor has run past the block's last unit
-  Unit i_u = make_unit(0, load_item(0));
-  int i_j = 0;                         // next iteration of i_u to issue
-  int4 raw1 = load_item(1), raw2 = load_item(2);
-  int32_t ids_cur = load_ids(i_u, 0), ids_nxt = load_ids(i_u, 1);
-  int32_t ids_next_unit = load_ids(make_unit(1, raw1), 0);
-  uint32_t issued = 0, consumed = 0;
-
-  // ---- consume cursor
-  int c_k = 0;
-  Unit c_u = i_u;
-  Unit pend_u = i_u;                   // the unit the issue cursor moved into last
-  int c_len = (threadIdx.x == 0 && i_live) ? __ldg(p.seq_lens + c_u.b) : 0;  // device length, checked against the plan
-  int pend_len = 0;
-  uint32_t qf[NT][D / 16][2], qf_next[NT][D / 16][2];
-  if (i_live) load_q_frags<D, NT>(qf, p, c_u.b, c_u.kvh, lane);
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-    for (int kk = 0; kk < D / 16; ++kk) qf_next[nt][kk][0] = qf_next[nt][kk][1] = 0u;
-
-  // Move the issue cursor into the next unit; allowed only while it is at most one unit ahead.
-  auto advance_issue = [&]() {
-    ++i_k;
-    i_live = unit_index(i_k) >= 0;
-    i_u = make_unit(i_k, raw1);
-    raw1 = raw2;
-    raw2 = load_item(i_k + 2);
-    i_j = 0;
-    ids_cur = ids_next_unit;
-    ids_nxt = load_ids(i_u, 1);
-    ids_next_unit = load_ids(make_unit(i_k + 1, raw1), 0);
-    pend_u = i_u;
-    pend_len = (threadIdx.x == 0 && i_live) ? __ldg(p.seq_lens + i_u.b) : 0;
-    if (i_live) load_q_frags<D, NT>(qf_next, p, i_u.b, i_u.kvh, lane);
-  };
-
-  // Issue copies until STAGES are in flight, the stream ends, or the cursor would run two units ahead.
-  auto fill = [&]() {
-    while (issued - consumed < uint32_t(STAGES) && i_live) {
-      if (i_j >= i_u.n_it) {
-        if (i_k > c_k) break;   // already one unit ahead
-        advance_issue();
-        continue;
-      }
-      if ((i_j & 31) == 0 && i_j > 0) {
-        ids_cur = ids_nxt;
-        ids_nxt = load_ids(i_u, (i_j >> 5) + 1);
-      }
-      const int32_t pid = __shfl_sync(0xffffffffu, ids_cur, i_j & 31);
-      if (lane == 0) {
-        if (pid < 0 || int64_t(pid) >= p.num_pages) atomicOr(p.error_word, LIBRA_DEV_ERR_BAD_PAGE_ID);
-        const uint32_t s = issued % STAGES;
-        const uint32_t bar = my_bar0 + 8 * s;
-        const uint32_t kdst = my_ring_u32 + s * SM::kStageBytes;
-        const uint32_t vdst = kdst + SM::kTileBytes;
-        const int kvh = i_u.kvh;
-        const int c1 = (p.pos_head == 1) ? kvh : ((p.pos_page == 1) ? pid : 0);
-        const int c2 = (p.pos_head == 2) ? kvh : ((p.pos_page == 2) ? pid : 0);
-        const int c3 = (p.pos_head == 3) ? kvh : ((p.pos_page == 3) ? pid : 0);
-        fence_proxy_async();
-        mbar_expect_tx(bar, SM::kStageBytes);
-#pragma unroll
-        for (int h = 0; h < NH; ++h) tma_load_4d(kdst + h * 2048, &map_k, bar, h * 64, c1, c2, c3);
-#pragma unroll
-        for (int h = 0; h < NH; ++h) tma_load_4d(vdst + h * 2048, &map_v, bar, h * 64, c1, c2, c3);
-      }
-      ++issued;
-      ++i_j;
-    }
-  };
-
-  WarpAcc<D, NT> st;
-  bool dead = false;  // a copy barrier timed out: stop touching the ring, keep the block-wide barriers
-
-  for (; unit_index(c_k) >= 0; ++c_k) {
-    if (c_k > 0) {
-      // the issue cursor is in unit c_k already unless this warp had nothing left to issue
-      while (i_k < c_k) advance_issue();
-      c_u = pend_u;
-      c_len = pend_len;
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          qf[nt][kk][0] = qf_next[nt][kk][0];
-          qf[nt][kk][1] = qf_next[nt][kk][1];
-        }
-    }
-    if (threadIdx.x == 0) check_planned_length(p, c_u, c_len);
-    st.reset();
-#ifdef LIBRA_TRACE
-    unsigned long long tr0 = 0, tr1 = 0, tr2 = 0;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr0));
-#endif
-    if (!dead) fill();
-
-    for (int it = 0; it < c_u.n_it && !dead; ++it) {
-      const uint32_t s = consumed % STAGES;
-      const uint32_t parity = (consumed / STAGES) & 1u;
-      if (!mbar_wait(my_bar0 + 8 * s, parity)) {
-        dead = true;
-        if (lane == 0) atomicOr(p.error_word, LIBRA_DEV_ERR_WAIT_TIMEOUT);
-        break;
-      }
-#ifdef LIBRA_TRACE
-      if (it == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr1));
-#endif
-      const uint32_t kt = my_ring_u32 + s * SM::kStageBytes;
-      const int tok0 = c_u.kv_begin + ((warp + it * NW) << 4);
-      process_page<D, NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes,
-                          c_u.kv_end - tok0, p.scale_log2, lane);
-      __syncwarp();  // every lane has consumed the stage before lane 0 refills it
-      ++consumed;
-      fill();
-    }
-
-#ifdef LIBRA_TRACE
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr2));
-#endif
-    // ---- unit epilogue: stage, merge in warp order, write; the next unit's copies stay in flight
-    stage_warp_result<D, NT>(st, merge_sm + warp * PS::kMergeWarpFloats, stat_m[warp], stat_l[warp], lane);
-    __syncthreads();
-    merge_and_write<D, NT, NW>(p, c_u, merge_sm, PS::kMergeWarpFloats, &stat_m[0][0], &stat_l[0][0], threadIdx.x, NW * 32);
-    __syncthreads();  // the merge area is free again
-#ifdef LIBRA_TRACE
-    if (threadIdx.x == 0) {
-      unsigned long long tr3;
-      unsigned smid;
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr3));
-      asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-      unsigned long long* t = p.trace + 6ull * unit_index(c_k);
-      t[0] = tr0; t[1] = tr1; t[2] = tr2; t[3] = tr3; t[4] = smid; t[5] = (unsigned long long)(c_u.kv_end - c_u.kv_begin);
-    }
-#endif
-  }
-
-  if (dead) {
-    // bounded last chance for copies still in flight to land before the block exits
-    for (uint32_t k = consumed; k < issued; ++k) (void)mbar_wait(my_bar0 + 8 * (k % STAGES), (k / STAGES) & 1u);
-  }
-  for (int e = c; e < p.num_empty; e += W) zero_empty_row<D>(p, items, e, threadIdx.x, NW * 32);
 }
 
 }  // namespace libra

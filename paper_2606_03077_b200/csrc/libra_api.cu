@@ -31,17 +31,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 typedef void (*DecodeKernelFn)(const CUtensorMap, const CUtensorMap, const DecodeParams, const libra::ParamPlan);
 
 struct Variant {
-  int persistent, warps, stages;
-  DecodeKernelFn fn[2][2];  // [D == 128][NT - 1]; null where the shape does not fit in shared memory
+  int warps, stages;
+  DecodeKernelFn fn[2][2];  // [D == 128][NT - 1]
   int smem[2][2];           // dynamic bytes
 };
 
-constexpr int kMaxSmem = 227 * 1024 - 2048;  // per block, leaving room for the static part
 
 template <int NW, int ST>
 Variant make_variant() {
   Variant v;
-  v.persistent = 0;
   v.warps = NW;
   v.stages = ST;
   v.fn[0][0] = libra::decode_kernel<64, 1, NW, ST>;
@@ -53,34 +51,11 @@ Variant make_variant() {
   return v;
 }
 
-template <int NW, int ST>
-Variant make_persistent_variant() {
-  Variant v;
-  v.persistent = 1;
-  v.warps = NW;
-  v.stages = ST;
-  v.fn[0][0] = libra::decode_persistent_kernel<64, 1, NW, ST>;
-  v.fn[0][1] = libra::decode_persistent_kernel<64, 2, NW, ST>;
-  v.fn[1][0] = libra::decode_persistent_kernel<128, 1, NW, ST>;
-  v.fn[1][1] = libra::decode_persistent_kernel<128, 2, NW, ST>;
-  v.smem[0][0] = libra::PersistentSmem<64, 1, NW, ST>::kDynamicBytes;
-  v.smem[0][1] = libra::PersistentSmem<64, 2, NW, ST>::kDynamicBytes;
-  v.smem[1][0] = libra::PersistentSmem<128, 1, NW, ST>::kDynamicBytes;
-  v.smem[1][1] = libra::PersistentSmem<128, 2, NW, ST>::kDynamicBytes;
-  for (int d = 0; d < 2; ++d)
-    for (int n = 0; n < 2; ++n)
-      if (v.smem[d][n] > kMaxSmem) v.fn[d][n] = nullptr;
-  return v;
-}
-
-// Schedules and block shapes that are compiled in; index 0 is the default.
+// Block shapes that are compiled in; index 0 is the default.
 const std::vector<Variant>& variants() {
   static const std::vector<Variant> v = {
       make_variant<4, 3>(), make_variant<4, 2>(), make_variant<4, 4>(), make_variant<4, 6>(),
       make_variant<8, 2>(), make_variant<8, 3>(), make_variant<2, 6>(), make_variant<2, 4>(),
-      make_persistent_variant<8, 3>(), make_persistent_variant<8, 2>(), make_persistent_variant<4, 3>(),
-      make_persistent_variant<4, 2>(), make_persistent_variant<4, 4>(), make_persistent_variant<4, 6>(),
-      make_persistent_variant<2, 6>(), make_persistent_variant<2, 4>(),
   };
   return v;
 }
@@ -540,13 +515,13 @@ int libra_set_combine_mode(libra_handle_t h, int32_t fused) {
   return LIBRA_OK;
 }
 
-int libra_set_variant(libra_handle_t h, int32_t persistent, int32_t warps, int32_t stages) {
+int libra_set_variant(libra_handle_t h, int32_t warps, int32_t stages) {
   if (!h) return LIBRA_INVALID_ARGUMENT;
   const std::vector<Variant>& vs = variants();
   const int di = (h->cfg.head_dim == 128) ? 1 : 0;
   const int ni = (h->group > 8) ? 1 : 0;
   for (size_t i = 0; i < vs.size(); ++i) {
-    if (vs[i].persistent == persistent && vs[i].warps == warps && vs[i].stages == stages && vs[i].fn[di][ni]) {
+    if (vs[i].warps == warps && vs[i].stages == stages && vs[i].fn[di][ni]) {
       h->variant = int(i);
       return LIBRA_OK;
     }
@@ -600,8 +575,7 @@ int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, cons
   const Variant& v = variants()[h->variant];
   const int di = (h->cfg.head_dim == 128) ? 1 : 0;
   const int ni = (h->group > 8) ? 1 : 0;
-  const bool persistent = v.persistent != 0;
-  const bool fused = !persistent && h->fused_combine;
+  const bool fused = h->fused_combine;
   const int32_t n_empty = int32_t(h->plan.empty.size());
   const int32_t n_combine = int32_t(h->plan.combine.size());
   const int32_t n_units = h->num_items * h->cfg.num_kv_heads;
@@ -628,16 +602,7 @@ int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, cons
     p.num_units = n_units;
     p.num_empty = n_empty;
     p.fused_combine = fused ? 1 : 0;
-#ifdef LIBRA_TRACE
-    p.trace = reinterpret_cast<unsigned long long*>(ws + h->workspace_bytes);
-#endif
-    unsigned grid;
-    if (persistent) {
-      const int slots = h->params.n_sm * h->params.ctas_per_sm;
-      grid = unsigned(std::max(1, std::min(n_units, slots)));
-    } else {
-      grid = unsigned(n_units) + unsigned(n_empty);
-    }
+    const unsigned grid = unsigned(n_units) + unsigned(n_empty);
     v.fn[di][ni]<<<grid, v.warps * 32, v.smem[di][ni], st>>>(pm->map_k, pm->map_v, p, h->pp);
     LIBRA_CUDA_TRY(h, cudaGetLastError());
     ++h->launches;

@@ -72,11 +72,9 @@ def test_every_block_shape_agrees(lib):
     lens = [2500, 300, 17, 4100]
     lens_a, bt, q, k, v = W.random_case(7, 4, 32, 8, 128, lens)
     ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
-    for sched in (0, 1):
-        for shape in [(4, 3), (4, 2), (4, 4), (4, 6), (8, 2), (8, 3), (2, 6), (2, 4)]:
-            variant = (sched,) + shape
-            got = H.run_host_case(lib, q, k, v, bt, lens_a, plan=lib.PlanParams(8, 1, 2, 256, 256, 64), variant=variant)
-            check(got, ref, f"variant {variant}")
+    for variant in [(4, 3), (4, 2), (4, 4), (4, 6), (8, 2), (8, 3), (2, 6), (2, 4)]:
+        got = H.run_host_case(lib, q, k, v, bt, lens_a, plan=lib.PlanParams(8, 1, 2, 256, 256, 64), variant=variant)
+        check(got, ref, f"variant {variant}")
 
 
 def test_plan_too_large_for_kernel_parameters(lib):
@@ -85,7 +83,7 @@ def test_plan_too_large_for_kernel_parameters(lib):
     lens_a, bt, q, k, v = W.random_case(9, 20, 4, 1, 64, lens)
     ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
     prm = lib.PlanParams(148, 2, 4, 16, 16, 64)
-    for variant in [(0, 4, 3), (1, 8, 3)]:
+    for variant in [(4, 3), (8, 3)]:
         got = H.run_host_case(lib, q, k, v, bt, lens_a, plan=prm, variant=variant)
         check(got, ref, f"uploaded plan, variant {variant}")
     import torch
