@@ -19,8 +19,7 @@ share its KV range, so:
     launch has about `items_per_slot` work items per resident block;
   * items are issued longest first (the classic greedy rule for the min-max objective).
 
-The paper states no single-GPU rule; this reading is listed among the readings of the
-paper in the design notes.
+The paper states no single-GPU rule; this is the reading this library takes.
 
 All arithmetic is integer.  cd(a, b) = ceil(a / b); au(a, b) = cd(a, b) * b;
 p2(x) = least power of two >= x.

@@ -65,7 +65,7 @@ class Workload:
 
 
 WORKLOADS = {
-    # index in BASELINE configs: 0
+    # the five workloads, in the order the benchmark lists them: 0
     "tiny": Workload("tiny", 4, 4, 1, 64, "uniform", "fixed", pool_pages=64,
                      params={"lens": [1, 7, 64, 300]}),
     # 1

@@ -95,6 +95,15 @@ def test_plan_too_large_for_kernel_parameters(lib):
     h.close()
 
 
+def test_longest_supported_sequence(lib):
+    # the paper's rollout length cap is 40,960 tokens (2,560 pages); split 64 ways and unsplit
+    lens_a, bt, q, k, v = W.random_case(10, 2, 8, 2, 128, [40960, 40959])
+    ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
+    for plan in (lib.PlanParams(148, 2, 64, 256, 512, 64), lib.PlanParams(148, 2, 1, 256, 512, 1)):
+        got = H.run_host_case(lib, q, k, v, bt, lens_a, plan=plan)
+        check(got, ref, "40960 tokens")
+
+
 def test_custom_scale(lib):
     lens_a, bt, q, k, v = W.random_case(8, 2, 8, 2, 64, [90, 33])
     ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a, sm_scale=0.3)

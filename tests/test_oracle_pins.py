@@ -84,7 +84,7 @@ def test_identical_keys_give_mean():
 def test_one_hot_key_selects_its_value_row(tstar):
     L, d = 37, 16
     lens, bt, q, k, v = W.random_case(9, 1, 2, 1, d, (L,))
-    c = 32.0  # c*c/sqrt(d) = 256 >= 150: every other weight underflows to exactly 0 in float64? no: e^-256 > 0
+    c = 32.0  # score gap c*c/sqrt(d) = 256: every other weight is e^-256, far below float64 resolution
     k[...] = 0
     q[...] = 0
     q[0, :, 0] = bits([c])[0]
@@ -251,3 +251,23 @@ def test_gates_catch_mutations():
     # bf16 rounding of a correct result passes both gates
     assert gates.tight_violations(O.round_to_bf16(ref), ref) == 0
     assert gates.stated_violations(O.round_to_bf16(ref), ref) == 0
+
+
+def test_tiny_workload_matches_stored_oracle_values():
+    """Regression pin: the stored values were written by tests/golden/make_tiny_golden.py from this
+    oracle; a change of its arithmetic shows up here and has to be justified."""
+    import os
+    lay, q, k, v = W.make_host_inputs("tiny")
+    out, lse = O.paged_decode_attention(q, k, v, lay.block_table, lay.seq_lens)
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "tiny_expected.txt")
+    n = 0
+    for line in open(path):
+        if line.startswith("#"):
+            continue
+        f = line.split()
+        b, h = int(f[0]), int(f[1])
+        want = [float(x) for x in f[2:]]
+        got = [lse[b, h]] + [out[b, h, j] for j in (0, 21, 42, 63)]
+        assert np.allclose(got, want, rtol=1e-13, atol=1e-15)
+        n += 1
+    assert n == 16
