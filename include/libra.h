@@ -198,6 +198,19 @@ int libra_plan_export(libra_handle_t handle, libra_plan_view_t* view);
 int libra_decode_attn(libra_handle_t handle, const void* q, const void* k_pages, const void* v_pages,
                       const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream);
 
+/* The same step with the KV append fused in (the step before attention inside one decode step of
+ * the rollout, Section 1 / Section 2.2 of the paper: the cache grows by one token per step).  k_new and
+ * v_new are device pointers to the current token's key and value rows, bf16 [batch, num_kv_heads,
+ * head_dim], 16-byte aligned; seq_lens still COUNTS that token.  For every sequence with L_b >= 1 the
+ * rows are written into slot (L_b - 1) % 16 of page block_table[b][(L_b - 1) / 16] of both pools (the
+ * pools are therefore not const) and the attention result is exactly what libra_decode_attn returns on
+ * the updated pools.  The block that owns the sequence's last page does both: it patches the staged copy
+ * of that page in shared memory and stores the rows to the pools, so no ordering between the store and
+ * the page reads is needed.  Errors: as libra_decode_attn. */
+int libra_decode_attn_append(libra_handle_t handle, const void* q, const void* k_new, const void* v_new,
+                             void* k_pages, void* v_pages, const int32_t* block_table, const int32_t* seq_lens,
+                             void* out, void* stream);
+
 /* The same step for callers whose data lives in host memory: copies q, both pools, the block
  * table and the lengths to `staging_dev` (a caller-owned device region of at least
  * libra_host_staging_size bytes, 256-byte aligned), plans, runs D and C and copies `out` back

@@ -63,6 +63,7 @@ SIGNATURES = {
     "libra_plan": (C.c_int, [_vp, _i32p, C.c_int32, _vp, C.c_size_t, _vp]),
     "libra_plan_export": (C.c_int, [_vp, C.POINTER(PlanView)]),
     "libra_decode_attn": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "libra_decode_attn_append": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_decode_attn_host": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, C.c_int32, _vp, _vp, C.c_size_t, _vp,
                                          C.c_size_t, _vp]),
     "libra_decode_attn_static": (C.c_int, [_vp, _i32p, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -182,6 +183,11 @@ class Handle:
                     out_ptr: int, stream: int) -> None:
         _check(lib.libra_decode_attn(self._h, q_ptr, k_ptr, v_ptr, block_table_ptr, seq_lens_ptr, out_ptr, stream),
                "libra_decode_attn")
+
+    def decode_attn_append(self, q_ptr: int, k_new_ptr: int, v_new_ptr: int, k_ptr: int, v_ptr: int,
+                           block_table_ptr: int, seq_lens_ptr: int, out_ptr: int, stream: int) -> None:
+        _check(lib.libra_decode_attn_append(self._h, q_ptr, k_new_ptr, v_new_ptr, k_ptr, v_ptr, block_table_ptr,
+                                            seq_lens_ptr, out_ptr, stream), "libra_decode_attn_append")
 
     def decode_attn_static(self, seq_lens_host: np.ndarray, q_ptr: int, k_ptr: int, v_ptr: int,
                            block_table_ptr: int, seq_lens_ptr: int, out_ptr: int, stream: int) -> None:

@@ -53,6 +53,13 @@ struct DecodeParams {
   int32_t num_units;      // work items x KV heads
   int32_t num_empty;      // empty sequences whose output row this launch zeroes
   int32_t fused_combine;  // 1: the last block of a split sequence merges its partials (step C) itself
+  // KV append fused into the step (null k_new = off): the current token's K and V rows, bf16 [B, Hkv, D],
+  // are written into slot (L_b - 1) % 16 of the sequence's last page, in the pools and in the staged tile
+  const __nv_bfloat16* k_new;
+  const __nv_bfloat16* v_new;
+  __nv_bfloat16* k_pool;
+  __nv_bfloat16* v_pool;
+  int64_t stride_page, stride_head, stride_token;  // pool strides in elements
 };
 
 namespace dev {
@@ -493,6 +500,27 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     }
     const uint32_t kt = my_ring_u32 + s * SM::kStageBytes;
     const int tok0 = u.kv_begin + ((warp + it * NW) << 4);
+    if (p.k_new != nullptr && u.chunk_j == u.n_chunks - 1 && u.kv_end - tok0 <= 16) {
+      // this page holds the sequence's newest token: its K and V rows come from k_new / v_new.  The copy
+      // that just landed predates them, so patch the staged tiles (swizzled row) and write the pools.
+      const int r = (u.kv_end - 1) & 15;
+      const int which = lane / (D / 8);   // 0: K, 1: V
+      const int c16 = lane % (D / 8);
+      if (which < 2) {
+        const int64_t page = __ldg(p.block_table + int64_t(u.b) * p.block_table_ld + ((u.kv_end - 1) >> 4));
+        const __nv_bfloat16* src = (which ? p.v_new : p.k_new) + (int64_t(u.b) * p.num_kv_heads + kvh) * D + c16 * 8;
+        const uint4 row = __ldg(reinterpret_cast<const uint4*>(src));
+        uint8_t* tile = my_ring + s * SM::kStageBytes + which * SM::kTileBytes;
+        *reinterpret_cast<uint4*>(tile + tile_off(r, c16)) = row;
+        if (page >= 0 && page < p.num_pages) {
+          __nv_bfloat16* dst = (which ? p.v_pool : p.k_pool) + page * p.stride_page + int64_t(kvh) * p.stride_head +
+                               int64_t(r) * p.stride_token + c16 * 8;
+          *reinterpret_cast<uint4*>(dst) = row;
+        }
+      }
+      fence_proxy_async();  // these generic writes come before the next TMA write into this stage
+      __syncwarp();
+    }
     process_page<D, NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes, u.kv_end - tok0,
                         p.scale_log2, lane);
     __syncwarp();  // every lane has consumed the stage before lane 0 refills it

@@ -529,9 +529,16 @@ int libra_set_variant(libra_handle_t h, int32_t warps, int32_t stages) {
   return LIBRA_UNSUPPORTED_SHAPE;
 }
 
-int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, const void* v_pages,
-                      const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream) {
+}  // extern "C"
+
+namespace {
+
+// Steps D and C; k_new / v_new non-null = append the current token's K and V rows on the way.
+int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* v_new, const void* k_pages,
+                const void* v_pages, const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream) {
   if (!h || !q || !k_pages || !v_pages || !block_table || !seq_lens || !out) return LIBRA_INVALID_ARGUMENT;
+  if ((k_new == nullptr) != (v_new == nullptr)) return LIBRA_INVALID_ARGUMENT;
+  if (reinterpret_cast<uintptr_t>(k_new) % 16 || reinterpret_cast<uintptr_t>(v_new) % 16) return LIBRA_INVALID_ARGUMENT;
   if (reinterpret_cast<uintptr_t>(k_pages) % 16 || reinterpret_cast<uintptr_t>(v_pages) % 16 ||
       reinterpret_cast<uintptr_t>(q) % 4 || reinterpret_cast<uintptr_t>(out) % 4) {
     return LIBRA_INVALID_ARGUMENT;
@@ -602,6 +609,13 @@ int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, cons
     p.num_units = n_units;
     p.num_empty = n_empty;
     p.fused_combine = fused ? 1 : 0;
+    p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+    p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+    p.k_pool = static_cast<__nv_bfloat16*>(const_cast<void*>(k_pages));
+    p.v_pool = static_cast<__nv_bfloat16*>(const_cast<void*>(v_pages));
+    p.stride_page = h->stride_page;
+    p.stride_head = h->stride_head;
+    p.stride_token = h->stride_token;
     const unsigned grid = unsigned(n_units) + unsigned(n_empty);
     v.fn[di][ni]<<<grid, v.warps * 32, v.smem[di][ni], st>>>(pm->map_k, pm->map_v, p, h->pp);
     LIBRA_CUDA_TRY(h, cudaGetLastError());
@@ -639,6 +653,22 @@ int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, cons
   }
   h->last_stream = stream;
   return LIBRA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int libra_decode_attn(libra_handle_t h, const void* q, const void* k_pages, const void* v_pages,
+                      const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream) {
+  return decode_impl(h, q, nullptr, nullptr, k_pages, v_pages, block_table, seq_lens, out, stream);
+}
+
+int libra_decode_attn_append(libra_handle_t h, const void* q, const void* k_new, const void* v_new, void* k_pages,
+                             void* v_pages, const int32_t* block_table, const int32_t* seq_lens, void* out,
+                             void* stream) {
+  if (!k_new || !v_new) return LIBRA_INVALID_ARGUMENT;
+  return decode_impl(h, q, k_new, v_new, k_pages, v_pages, block_table, seq_lens, out, stream);
 }
 
 int libra_host_staging_size(libra_handle_t h, int32_t batch, size_t* bytes) {
