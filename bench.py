@@ -184,6 +184,49 @@ class Replica:
         self.h.decode_attn(self.q.data_ptr(), k.data_ptr(), v.data_ptr(), self.bts[s].data_ptr(),
                            self.lens_dev[s].data_ptr(), self.out.data_ptr(), stream)
 
+    def step_device(self, stream: int) -> None:
+        """The same step planned on the GPU (libra_plan_device): the host never reads the lengths."""
+        s = self.i % len(self.layouts)
+        k, v = self.pools[self.i % len(self.pools)]
+        self.i += 1
+        self.h.plan_device(self.lens_dev[s].data_ptr(), self.w.batch, self.ws.data_ptr(), self.ws.numel(), stream)
+        self.h.decode_attn(self.q.data_ptr(), k.data_ptr(), v.data_ptr(), self.bts[s].data_ptr(),
+                           self.lens_dev[s].data_ptr(), self.out.data_ptr(), stream)
+
+    def timed_device_plan(self, steps: int, warmup: int, graph: bool):
+        """ms per step with the device-side planner, issued eagerly or replayed from one CUDA graph that
+        holds one step per layout x pool copy."""
+        torch = self.torch
+        side = torch.cuda.Stream()
+        per_replay = len(self.layouts) * len(self.pools)
+        with torch.cuda.stream(side):
+            for _ in range(max(warmup, per_replay)):
+                self.step_device(side.cuda_stream)
+        torch.cuda.synchronize()
+        g = None
+        if graph:
+            self.i = 0
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for _ in range(per_replay):
+                    self.step_device(side.cuda_stream)
+            g.replay()
+            torch.cuda.synchronize()
+        reps = max(1, steps // per_replay)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(side):
+            e0.record()
+            for _ in range(reps):
+                if graph:
+                    g.replay()
+                else:
+                    for _ in range(per_replay):
+                        self.step_device(side.cuda_stream)
+            e1.record()
+        torch.cuda.synchronize()
+        assert self.h.debug_error_word() == 0, "device error word set"
+        return e0.elapsed_time(e1) / (reps * per_replay)
+
     def timed(self, steps: int, warmup: int, barrier=None):
         torch = self.torch
         st = torch.cuda.current_stream().cuda_stream
@@ -432,6 +475,13 @@ def run_libra(args):
                             "frac_of_nominal_8TBs": r.kv_bytes_per_step / (per * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
                             "frac_of_measured_copy": r.kv_bytes_per_step / (per * 1e-3) / 1e9 / peak,
                             "kv_bytes_per_step": r.kv_bytes_per_step, "pool_copies": len(r.pools)}
+            if name == "shift_b128":  # the re-planned-every-step workload: also with the device-side planner
+                eager = r.timed_device_plan(n, 6, graph=False)
+                graph = r.timed_device_plan(n, 6, graph=True)
+                others[name]["device_plan"] = {
+                    "ms_per_step_eager": eager, "ms_per_step_cuda_graph": graph,
+                    "kv_gbs_cuda_graph": r.kv_bytes_per_step / (graph * 1e-3) / 1e9,
+                    "note": "libra_plan_device + decode + combine; the graph holds one step per layout and is replayed"}
             r.close()
             del r
             torch.cuda.empty_cache()

@@ -68,6 +68,8 @@ typedef enum {
 #define LIBRA_ERR_WAIT_TIMEOUT 1u   /* a bounded wait on a copy barrier ran out                  */
 #define LIBRA_ERR_BAD_PAGE_ID 2u    /* block-table entry outside [0, num_pages)                  */
 #define LIBRA_ERR_SEQ_LEN_MISMATCH 4u /* device seq_lens differ from the lengths that were planned */
+#define LIBRA_ERR_PLAN_OVERFLOW 8u  /* device-side planner: too many sequences or work items, or a length
+                                       longer than a block-table row can describe; nothing was computed */
 
 /* Planner constants (Section 4.3 of the paper: degrees are powers of two, work sorted by length,
  * min-max objective).  A zero field takes its default. */
@@ -180,7 +182,22 @@ int libra_plan_host(const libra_plan_params_t* params, int32_t num_kv_heads, con
 int libra_plan(libra_handle_t handle, const int32_t* seq_lens_host, int32_t batch, void* workspace_dev,
                size_t workspace_bytes, void* stream);
 
-/* Host view of the last plan (see libra_plan_view_t).  Errors: NOT_PLANNED. */
+/* Step P on the GPU: the same planning rule as libra_plan, evaluated by one thread block from the
+ * DEVICE copy of the lengths (int32[batch]; negative values count as 0), enqueued on `stream`.  The
+ * host never reads the lengths, so plan + libra_decode_attn can be enqueued back to back - or recorded
+ * once and replayed - while the lengths change underneath (the paper re-plans as lengths drift:
+ * Section 2.2, Section 4.3).  The plan is written into the workspace; later libra_decode_attn calls
+ * launch grids sized for the worst case and the kernels read the real counts from the workspace.
+ * Limits: batch <= 4096 (UNSUPPORTED_SHAPE otherwise); at most 4096 work items and no length beyond
+ * block_table_ld * 16, else the plan is empty and LIBRA_ERR_PLAN_OVERFLOW is set in the device error
+ * word (checked on the device, since the host does not see the lengths).  The result equals
+ * libra_plan's bit for bit (libra_plan_export reads it back).
+ * Errors: INVALID_ARGUMENT, WORKSPACE_TOO_SMALL, UNSUPPORTED_SHAPE, CUDA_ERROR. */
+int libra_plan_device(libra_handle_t handle, const int32_t* seq_lens_dev, int32_t batch, void* workspace_dev,
+                      size_t workspace_bytes, void* stream);
+
+/* Host view of the last plan (see libra_plan_view_t); after libra_plan_device this copies the plan
+ * back from the workspace and synchronises that call's stream.  Errors: NOT_PLANNED, CUDA_ERROR. */
 int libra_plan_export(libra_handle_t handle, libra_plan_view_t* view);
 
 /* Steps D and C: softmax(q K^T * sm_scale) V per query head over the pages of each sequence

@@ -20,7 +20,7 @@ LIB_PATH = _LIB_PATH
 
 STATIC_SCRATCH_BYTES = 8 << 20
 OK, INVALID_ARGUMENT, UNSUPPORTED_SHAPE, WORKSPACE_TOO_SMALL, NOT_PLANNED, CUDA_ERROR, DEVICE_FLAGGED = range(7)
-ERR_WAIT_TIMEOUT, ERR_BAD_PAGE_ID, ERR_SEQ_LEN_MISMATCH = 1, 2, 4
+ERR_WAIT_TIMEOUT, ERR_BAD_PAGE_ID, ERR_SEQ_LEN_MISMATCH, ERR_PLAN_OVERFLOW = 1, 2, 4, 8
 
 
 class PlanParams(C.Structure):
@@ -61,6 +61,7 @@ SIGNATURES = {
     "libra_plan_host": (C.c_int, [C.POINTER(PlanParams), C.c_int32, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p,
                                   _i32p, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p]),
     "libra_plan": (C.c_int, [_vp, _i32p, C.c_int32, _vp, C.c_size_t, _vp]),
+    "libra_plan_device": (C.c_int, [_vp, _vp, C.c_int32, _vp, C.c_size_t, _vp]),
     "libra_plan_export": (C.c_int, [_vp, C.POINTER(PlanView)]),
     "libra_decode_attn": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_decode_attn_append": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -169,6 +170,11 @@ class Handle:
         lens = _as_i32(seq_lens_host)
         _check(lib.libra_plan(self._h, lens.ctypes.data_as(_i32p), int(lens.shape[0]), workspace_ptr,
                               workspace_bytes, stream), "libra_plan")
+
+    def plan_device(self, seq_lens_dev_ptr: int, batch: int, workspace_ptr: int, workspace_bytes: int,
+                    stream: int) -> None:
+        _check(lib.libra_plan_device(self._h, seq_lens_dev_ptr, batch, workspace_ptr, workspace_bytes, stream),
+               "libra_plan_device")
 
     def plan_export(self) -> dict:
         v = PlanView()

@@ -18,6 +18,7 @@ namespace libra {
 
 struct CombineParams {
   const int4* entries;       // merges {b, first_slot, n, planned_len} in device memory, or null: in `pf`
+  const int32_t* dev_counts; // device-side plan: the number of merges is read from here (null = host plan)
   const float* partial_o;    // [slot][Hq][D]
   const float* partial_lse;  // [slot][Hq]
   const int32_t* seq_lens;
@@ -37,6 +38,7 @@ combine_kernel(const __grid_constant__ CombineParams p, const __grid_constant__ 
   const int h = blockIdx.y * kCombineWarps + (threadIdx.x >> 5);
   const int Hq = p.num_q_heads;
   if (h >= Hq) return;
+  if (p.dev_counts && int(blockIdx.x) >= p.dev_counts[plan_layout::kCntCombine]) return;  // grid is an upper bound
   const int4 fix = (p.entries ? p.entries : pf.e)[blockIdx.x];  // plain load: may address parameter space
   const int b = fix.x;
   const int first = fix.y;

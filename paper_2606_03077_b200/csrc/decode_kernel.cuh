@@ -37,6 +37,7 @@ struct DecodeParams {
   const int32_t* seq_lens;
   __nv_bfloat16* out;
   const int4* entries;   // work items then empty-sequence entries in device memory, or null: in `pp`
+  const int32_t* dev_counts;  // device-side plan: the counts below are read from here (null = host plan)
   float* partial_o;      // [slot][Hq][D]
   float* partial_lse;    // [slot][Hq]
   uint32_t* error_word;
@@ -378,8 +379,9 @@ __device__ __forceinline__ void check_planned_length(const DecodeParams& p, cons
 
 // Output rows of empty sequences are zero; entry e of the plan's empty list (stored after the items).
 template <int D>
-__device__ __forceinline__ void zero_empty_row(const DecodeParams& p, const int4* entries, int e, int tid, int nthreads) {
-  const int64_t row = int64_t(entries[p.num_items + e].x) * p.num_q_heads * D;
+__device__ __forceinline__ void zero_empty_row(const DecodeParams& p, const int4* entries, int num_items, int e, int tid,
+                                               int nthreads) {
+  const int64_t row = int64_t(entries[num_items + e].x) * p.num_q_heads * D;
   for (int i = tid; i < p.num_q_heads * D; i += nthreads) p.out[row + i] = __float2bfloat16_rn(0.f);
 }
 
@@ -427,8 +429,16 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   // the plan lives in the kernel parameters unless it was too large for them (plain loads: the
   // pointer may address parameter space)
   const int4* entries = p.entries ? p.entries : pp.e;
-  if (int(blockIdx.x) >= p.num_units) {
-    zero_empty_row<D>(p, entries, int(blockIdx.x) - p.num_units, threadIdx.x, NW * 32);
+  int num_items = p.num_items, num_units = p.num_units, num_empty = p.num_empty;
+  if (p.dev_counts) {  // planned on the device: the grid is an upper bound, the real counts are here
+    num_items = p.dev_counts[plan_layout::kCntItems];
+    num_empty = p.dev_counts[plan_layout::kCntEmpty];
+    num_units = num_items * p.num_kv_heads;
+  }
+  if (int(blockIdx.x) >= num_units) {
+    if (int(blockIdx.x) - num_units < num_empty) {
+      zero_empty_row<D>(p, entries, num_items, int(blockIdx.x) - num_units, threadIdx.x, NW * 32);
+    }
     return;
   }
 

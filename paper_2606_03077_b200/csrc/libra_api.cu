@@ -13,12 +13,14 @@
 #include "combine_kernel.cuh"
 #include "decode_kernel.cuh"
 #include "libra.h"
+#include "plan_kernel.cuh"
 #include "plan_layout.hpp"
 #include "planner.hpp"
 
 static_assert(LIBRA_ERR_WAIT_TIMEOUT == LIBRA_DEV_ERR_WAIT_TIMEOUT, "error bits");
 static_assert(LIBRA_ERR_BAD_PAGE_ID == LIBRA_DEV_ERR_BAD_PAGE_ID, "error bits");
 static_assert(LIBRA_ERR_SEQ_LEN_MISMATCH == LIBRA_DEV_ERR_SEQ_LEN_MISMATCH, "error bits");
+static_assert(LIBRA_ERR_PLAN_OVERFLOW == LIBRA_DEV_ERR_PLAN_OVERFLOW, "error bits");
 
 namespace {
 
@@ -113,6 +115,10 @@ struct libra_handle_s {
   void* workspace = nullptr;
   int32_t num_items = 0;
   void* last_stream = nullptr;
+  bool device_planned = false;  // the last plan was made by the device-side planner: counts live in the workspace
+  int32_t planned_batch = 0;
+  size_t dev_counts_off = 0, dev_per_seq_off = 0, dev_entries_off = 0, dev_fixes_off = 0;
+  std::vector<int32_t> export_scratch;
   bool plan_in_params = true;   // the usual case: the plan travels with every launch
   libra::ParamPlan pp;          // work items, then one entry per empty sequence
   libra::ParamFix pf;           // merges for the combine kernel
@@ -360,6 +366,9 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
       }
     }
     if (status != LIBRA_OK) break;
+    e = cudaFuncSetAttribute(reinterpret_cast<const void*>(libra::plan_kernel), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             int(libra::plan_kernel_smem_bytes()));
+    if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
 
     h->max_items = libra::max_items(h->params, cfg->num_kv_heads, cfg->max_batch);
     h->cnt_off = 256;  // the first 256 bytes hold the control words (the device error word)
@@ -367,7 +376,12 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
     h->lse_off = h->cnt_off + h->cnt_bytes;
     h->o_off = h->lse_off + align_up(size_t(h->max_items) * cfg->num_q_heads * 4, 256);
     h->plan_off = h->o_off + align_up(size_t(h->max_items) * cfg->num_q_heads * cfg->head_dim * 4, 256);
-    h->plan_bytes = align_up((size_t(h->max_items) + 2 * size_t(cfg->max_batch)) * sizeof(int4), 256);
+    // plan region: counts | per-sequence arrays (device planner) | entries (items + empties) | merges
+    h->dev_counts_off = h->plan_off;
+    h->dev_per_seq_off = h->dev_counts_off + 256;
+    h->dev_entries_off = h->dev_per_seq_off + align_up(size_t(4) * cfg->max_batch * sizeof(int32_t), 256);
+    h->dev_fixes_off = h->dev_entries_off + align_up((size_t(h->max_items) + size_t(cfg->max_batch)) * sizeof(int4), 256);
+    h->plan_bytes = h->dev_fixes_off + align_up(size_t(cfg->max_batch) * sizeof(int4), 256) - h->plan_off;
     h->workspace_bytes = h->plan_off + h->plan_bytes;
 
     for (int i = 0; i < 2; ++i) {
@@ -477,7 +491,7 @@ int libra_plan(libra_handle_t h, const int32_t* seq_lens_host, int32_t batch, vo
   }
   if (!h->plan_in_params) {
     const size_t bytes = size_t(n_items + n_empty + n_combine) * sizeof(int4);
-    LIBRA_CUDA_TRY(h, cudaMemcpyAsync(static_cast<uint8_t*>(workspace_dev) + h->plan_off, entries, bytes,
+    LIBRA_CUDA_TRY(h, cudaMemcpyAsync(static_cast<uint8_t*>(workspace_dev) + h->dev_entries_off, entries, bytes,
                                       cudaMemcpyHostToDevice, st));
     LIBRA_CUDA_TRY(h, cudaEventRecord(h->staging_done[k], st));
     h->staging_used[k] = true;
@@ -487,12 +501,99 @@ int libra_plan(libra_handle_t h, const int32_t* seq_lens_host, int32_t batch, vo
   h->num_items = n_items;
   h->last_stream = stream;
   h->planned = true;
+  h->device_planned = false;
+  h->planned_batch = batch;
+  return LIBRA_OK;
+}
+
+int libra_plan_device(libra_handle_t h, const int32_t* seq_lens_dev, int32_t batch, void* workspace_dev,
+                      size_t workspace_bytes, void* stream) {
+  if (!h || batch < 0 || batch > h->cfg.max_batch || !seq_lens_dev || !workspace_dev) return LIBRA_INVALID_ARGUMENT;
+  if (reinterpret_cast<uintptr_t>(workspace_dev) % 256 != 0) return LIBRA_INVALID_ARGUMENT;
+  if (workspace_bytes < h->workspace_bytes) return LIBRA_WORKSPACE_TOO_SMALL;
+  if (batch > libra::kDevPlanMax) return LIBRA_UNSUPPORTED_SHAPE;
+  DeviceGuard guard(h->cfg.device);
+  if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace_dev);
+  if (h->clean_workspace != workspace_dev) {
+    h->clean_workspace = nullptr;
+    LIBRA_CUDA_TRY(h, cudaMemsetAsync(workspace_dev, 0, h->cnt_off + h->cnt_bytes, st));
+    h->clean_workspace = workspace_dev;
+  }
+  libra::PlanKernelParams p;
+  p.seq_lens = seq_lens_dev;
+  p.batch = batch;
+  p.heads = h->cfg.num_kv_heads;
+  p.slots = int64_t(h->params.n_sm) * h->params.ctas_per_sm * h->params.items_per_slot;
+  p.chunk_align = h->params.chunk_align;
+  p.min_chunk = h->params.min_chunk;
+  p.max_splits = h->params.max_splits;
+  p.max_items = int32_t(std::min<int64_t>(h->max_items, libra::kDevPlanMax));
+  p.max_len = int32_t(std::min<int64_t>(int64_t(h->cfg.block_table_ld) * h->cfg.page_size, 0x7fffffff));
+  p.counts = reinterpret_cast<int32_t*>(ws + h->dev_counts_off);
+  p.per_seq = reinterpret_cast<int32_t*>(ws + h->dev_per_seq_off);
+  p.entries = reinterpret_cast<int4*>(ws + h->dev_entries_off);
+  p.fixes = reinterpret_cast<int4*>(ws + h->dev_fixes_off);
+  p.error_word = reinterpret_cast<uint32_t*>(ws);
+  libra::plan_kernel<<<1, libra::kDevPlanThreads, libra::plan_kernel_smem_bytes(), st>>>(p);
+  LIBRA_CUDA_TRY(h, cudaGetLastError());
+  ++h->launches;
+  h->workspace = workspace_dev;
+  h->last_stream = stream;
+  h->planned = true;
+  h->device_planned = true;
+  h->plan_in_params = false;
+  h->planned_batch = batch;
   return LIBRA_OK;
 }
 
 int libra_plan_export(libra_handle_t h, libra_plan_view_t* view) {
   if (!h || !view) return LIBRA_INVALID_ARGUMENT;
   if (!h->planned) return LIBRA_NOT_PLANNED;
+  if (h->device_planned) {  // bring the device plan back (synchronises the stream of the plan call)
+    DeviceGuard guard(h->cfg.device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(h->last_stream);
+    const uint8_t* ws = static_cast<const uint8_t*>(h->workspace);
+    int32_t counts[libra::plan_layout::kCountInts];
+    LIBRA_CUDA_TRY(h, cudaMemcpyAsync(counts, ws + h->dev_counts_off, sizeof(counts), cudaMemcpyDeviceToHost, st));
+    LIBRA_CUDA_TRY(h, cudaStreamSynchronize(st));
+    namespace L = libra::plan_layout;
+    const int32_t B = h->planned_batch, n_items = counts[L::kCntItems], n_cmb = counts[L::kCntCombine],
+                  n_empty = counts[L::kCntEmpty];
+    std::vector<int32_t> per_seq(size_t(4) * std::max(B, 1));
+    std::vector<int4> entries(size_t(std::max(n_items + n_empty, 1)));
+    std::vector<int4> fixes(size_t(std::max(n_cmb, 1)));
+    LIBRA_CUDA_TRY(h, cudaMemcpyAsync(per_seq.data(), ws + h->dev_per_seq_off, size_t(4) * B * 4, cudaMemcpyDeviceToHost, st));
+    LIBRA_CUDA_TRY(h, cudaMemcpyAsync(entries.data(), ws + h->dev_entries_off, size_t(n_items + n_empty) * 16,
+                                      cudaMemcpyDeviceToHost, st));
+    LIBRA_CUDA_TRY(h, cudaMemcpyAsync(fixes.data(), ws + h->dev_fixes_off, size_t(n_cmb) * 16, cudaMemcpyDeviceToHost, st));
+    LIBRA_CUDA_TRY(h, cudaStreamSynchronize(st));
+    libra::HostPlan& pl = h->plan;
+    pl.batch = B;
+    pl.chunk_target = counts[L::kCntChunkTarget];
+    pl.bucket.assign(per_seq.begin(), per_seq.begin() + B);
+    pl.num_splits.assign(per_seq.begin() + B, per_seq.begin() + 2 * B);
+    pl.chunk_len.assign(per_seq.begin() + 2 * B, per_seq.begin() + 3 * B);
+    pl.item_offset.assign(per_seq.begin() + 3 * B, per_seq.begin() + 4 * B);
+    pl.items.resize(size_t(n_items));
+    h->items_flat.resize(size_t(n_items) * 4);
+    for (int32_t i = 0; i < n_items; ++i) {
+      const int4 e = entries[size_t(i)];
+      const int32_t b = e.x & (L::kMaxBatch - 1), j = (e.x >> L::kChunkShift) & 63;
+      pl.items[size_t(i)] = libra::WorkItem{b, j, e.y, e.z};
+      h->items_flat[4 * size_t(i) + 0] = b;
+      h->items_flat[4 * size_t(i) + 1] = j;
+      h->items_flat[4 * size_t(i) + 2] = e.y;
+      h->items_flat[4 * size_t(i) + 3] = e.z;
+    }
+    pl.combine.resize(size_t(n_cmb));
+    for (int32_t c = 0; c < n_cmb; ++c) pl.combine[size_t(c)] = fixes[size_t(c)].x;
+    pl.empty.resize(size_t(n_empty));
+    for (int32_t e = 0; e < n_empty; ++e) pl.empty[size_t(e)] = entries[size_t(n_items + e)].x;
+    h->num_items = n_items;
+  }
   const libra::HostPlan& pl = h->plan;
   view->batch = pl.batch;
   view->chunk_target = pl.chunk_target;
@@ -565,7 +666,8 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
 
   uint8_t* ws = static_cast<uint8_t*>(h->workspace);
   uint32_t* err_dev = reinterpret_cast<uint32_t*>(ws);
-  const int4* entries_dev = h->plan_in_params ? nullptr : reinterpret_cast<const int4*>(ws + h->plan_off);
+  const int4* entries_dev = h->plan_in_params ? nullptr : reinterpret_cast<const int4*>(ws + h->dev_entries_off);
+  const int32_t* dev_counts = h->device_planned ? reinterpret_cast<const int32_t*>(ws + h->dev_counts_off) : nullptr;
 
   cudaEvent_t* ev = nullptr;
   if (h->profiling && h->profiled_calls < kMaxProfiledCalls) {
@@ -583,9 +685,12 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
   const int di = (h->cfg.head_dim == 128) ? 1 : 0;
   const int ni = (h->group > 8) ? 1 : 0;
   const bool fused = h->fused_combine;
-  const int32_t n_empty = int32_t(h->plan.empty.size());
-  const int32_t n_combine = int32_t(h->plan.combine.size());
-  const int32_t n_units = h->num_items * h->cfg.num_kv_heads;
+  // host plan: exact counts; device plan: upper bounds for the grids, the kernels read the counts themselves
+  const int32_t n_empty = h->device_planned ? h->planned_batch : int32_t(h->plan.empty.size());
+  const int32_t n_combine = h->device_planned ? h->planned_batch : int32_t(h->plan.combine.size());
+  const int32_t n_items_bound =
+      h->device_planned ? int32_t(std::min<int64_t>(h->max_items, libra::kDevPlanMax)) : h->num_items;
+  const int32_t n_units = n_items_bound * h->cfg.num_kv_heads;
   if (n_units > 0 || n_empty > 0) {
     DecodeParams p;
     p.q = static_cast<const __nv_bfloat16*>(q);
@@ -593,6 +698,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     p.seq_lens = seq_lens;
     p.out = static_cast<__nv_bfloat16*>(out);
     p.entries = entries_dev;
+    p.dev_counts = dev_counts;
     p.partial_o = reinterpret_cast<float*>(ws + h->o_off);
     p.partial_lse = reinterpret_cast<float*>(ws + h->lse_off);
     p.error_word = err_dev;
@@ -624,7 +730,10 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
   if (ev) LIBRA_CUDA_TRY(h, cudaEventRecord(ev[1], st));
   if (!fused && n_combine > 0) {
     libra::CombineParams c;
-    c.entries = h->plan_in_params ? nullptr : entries_dev + h->num_items + n_empty;
+    c.entries = h->plan_in_params ? nullptr
+                                  : (h->device_planned ? reinterpret_cast<const int4*>(ws + h->dev_fixes_off)
+                                                       : entries_dev + h->num_items + n_empty);
+    c.dev_counts = dev_counts;
     c.partial_o = reinterpret_cast<const float*>(ws + h->o_off);
     c.partial_lse = reinterpret_cast<const float*>(ws + h->lse_off);
     c.seq_lens = seq_lens;

@@ -1,0 +1,234 @@
+// Device-side planner (step P on the GPU): the same length-bucketed rule as planner.cpp, computed by
+// one thread block from the device copy of the sequence lengths, so that a whole decode step (plan,
+// decode, combine) can be enqueued - or captured in a CUDA graph - without the host ever seeing the
+// lengths.  The paper re-plans as the length distribution drifts (Section 4.3: the planner is re-run
+// every K iterations; Section 2.2: lengths grow during training); here that means every step.
+//
+//   C       = max(min_chunk, au(cd(heads * T, slots), chunk_align))          T = sum of lengths
+//   s_b     = min(p2(cd(L_b, C)), max_splits)      chunk_b = au(cd(L_b, s_b), chunk_align)
+//   n_b     = cd(L_b, chunk_b)                     items sorted by (length desc, b asc, j asc)
+//
+// Integer arithmetic only; the result must equal the host planner's bit for bit.  Limits: batch and
+// work items <= kDevPlanMax each (one block, four elements per thread); beyond that, or when a length
+// exceeds what a block-table row can describe, the kernel writes an empty plan and sets
+// LIBRA_DEV_ERR_PLAN_OVERFLOW.  Negative lengths count as empty sequences.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "plan_layout.hpp"
+
+namespace libra {
+
+constexpr int kDevPlanThreads = 1024;
+constexpr int kDevPlanPerThread = 4;
+constexpr int kDevPlanMax = kDevPlanThreads * kDevPlanPerThread;
+
+struct PlanKernelParams {
+  const int32_t* seq_lens;   // device, [batch]
+  int32_t batch;
+  int32_t heads;             // work units per item (KV heads)
+  int64_t slots;             // n_sm * ctas_per_sm * items_per_slot
+  int32_t chunk_align, min_chunk, max_splits;
+  int32_t max_items;         // capacity of `entries` for work items
+  int32_t max_len;           // longest sequence the block table can describe
+  int32_t* counts;           // [plan_layout::kCountInts]: num_items, num_combine, num_empty, chunk_target, overflow
+  int32_t* per_seq;          // [4][batch]: bucket, num_splits, chunk_len, item_offset
+  int4* entries;             // work items, then one entry per empty sequence
+  int4* fixes;               // merges for the combine kernel
+  uint32_t* error_word;
+};
+
+namespace dev {
+
+// Exclusive scan of `n` ints in shared memory (n <= kDevPlanMax), in place; returns the total.
+// `warp_tot` is scratch for 32 ints.  All threads of the block call it.
+__device__ __forceinline__ int block_exclusive_scan(int* data, int n, int* warp_tot) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int v[kDevPlanPerThread];
+  int sum = 0;
+#pragma unroll
+  for (int k = 0; k < kDevPlanPerThread; ++k) {
+    const int i = tid * kDevPlanPerThread + k;
+    v[k] = (i < n) ? data[i] : 0;
+    sum += v[k];
+  }
+  int incl = sum;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += t;
+  }
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = warp_tot[lane];
+    int wi = w;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, wi, off);
+      if (lane >= off) wi += t;
+    }
+    warp_tot[lane] = wi - w;  // exclusive prefix of the warp totals
+    if (lane == 31) warp_tot[32] = wi;
+  }
+  __syncthreads();
+  int run = warp_tot[warp] + incl - sum;
+#pragma unroll
+  for (int k = 0; k < kDevPlanPerThread; ++k) {
+    const int i = tid * kDevPlanPerThread + k;
+    if (i < n) data[i] = run;
+    run += v[k];
+  }
+  const int total = warp_tot[32];
+  __syncthreads();
+  return total;
+}
+
+}  // namespace dev
+
+// grid = 1 block of kDevPlanThreads threads; dynamic shared memory = plan_kernel_smem_bytes()
+constexpr size_t plan_kernel_smem_bytes() { return size_t(7) * kDevPlanMax * sizeof(int); }
+
+__global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelParams p) {
+  extern __shared__ int sm[];
+  int* nsplit = sm;                      // [batch]
+  int* chunk = sm + kDevPlanMax;         // [batch]
+  int* offs = sm + 2 * kDevPlanMax;      // [batch] exclusive scan of nsplit
+  int* aux = sm + 3 * kDevPlanMax;       // [batch] flags / their scans
+  int* it_len = sm + 4 * kDevPlanMax;    // [items]
+  int* it_b = sm + 5 * kDevPlanMax;      // [items]
+  int* it_j = sm + 6 * kDevPlanMax;      // [items]
+  __shared__ int warp_tot[33];
+  __shared__ long long s_total;
+
+  const int tid = threadIdx.x;
+  const int B = p.batch;
+  namespace L = plan_layout;
+
+  bool overflow = B > kDevPlanMax;
+  if (overflow) {
+    if (tid == 0) {
+      p.counts[L::kCntItems] = 0; p.counts[L::kCntCombine] = 0; p.counts[L::kCntEmpty] = 0;
+      p.counts[L::kCntChunkTarget] = 0; p.counts[L::kCntOverflow] = 1;
+      atomicOr(p.error_word, LIBRA_DEV_ERR_PLAN_OVERFLOW);
+    }
+    return;
+  }
+
+  // ---- T = sum of lengths
+  if (tid == 0) s_total = 0;
+  __syncthreads();
+  long long part = 0;
+  int too_long = 0;
+  for (int b = tid; b < B; b += kDevPlanThreads) {
+    part += max(p.seq_lens[b], 0);
+    too_long |= (p.seq_lens[b] > p.max_len) ? 1 : 0;
+  }
+  if (__syncthreads_or(too_long)) {  // a length the block table cannot hold: refuse the whole batch
+    if (tid == 0) {
+      p.counts[L::kCntItems] = 0; p.counts[L::kCntCombine] = 0; p.counts[L::kCntEmpty] = 0;
+      p.counts[L::kCntChunkTarget] = 0; p.counts[L::kCntOverflow] = 1;
+      atomicOr(p.error_word, LIBRA_DEV_ERR_PLAN_OVERFLOW);
+    }
+    return;
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+  if ((tid & 31) == 0 && part) atomicAdd(reinterpret_cast<unsigned long long*>(&s_total), (unsigned long long)part);
+  __syncthreads();
+  const long long T = s_total;
+  const long long A = p.chunk_align;
+  long long base = (p.heads * T + p.slots - 1) / p.slots;
+  base = (base + A - 1) / A * A;
+  if (base < p.min_chunk) base = p.min_chunk;
+
+  // ---- per sequence: degree, chunk length, chunk count
+  for (int b = tid; b < B; b += kDevPlanThreads) {
+    const long long len = max(p.seq_lens[b], 0);
+    int bucket = -1, n = 0, c = 0;
+    if (len > 0) {
+      long long deg = 1;
+      const long long want = (len + base - 1) / base;
+      while (deg < want) deg <<= 1;
+      if (deg > p.max_splits) deg = p.max_splits;
+      const long long ch = ((len + deg - 1) / deg + A - 1) / A * A;
+      n = int((len + ch - 1) / ch);
+      c = int(ch);
+      bucket = 0;
+      while ((1ll << bucket) < deg) ++bucket;
+    }
+    nsplit[b] = n;
+    chunk[b] = c;
+    offs[b] = n;
+    p.per_seq[b] = bucket;
+    p.per_seq[B + b] = n;
+    p.per_seq[2 * B + b] = c;
+  }
+  __syncthreads();
+  const int n_items = dev::block_exclusive_scan(offs, B, warp_tot);
+  for (int b = tid; b < B; b += kDevPlanThreads) p.per_seq[3 * B + b] = offs[b];
+
+  overflow = n_items > kDevPlanMax || n_items > p.max_items;
+  if (overflow) {
+    if (tid == 0) {
+      p.counts[L::kCntItems] = 0; p.counts[L::kCntCombine] = 0; p.counts[L::kCntEmpty] = 0;
+      p.counts[L::kCntChunkTarget] = int(base); p.counts[L::kCntOverflow] = 1;
+      atomicOr(p.error_word, LIBRA_DEV_ERR_PLAN_OVERFLOW);
+    }
+    return;
+  }
+
+  // ---- merges (n_b > 1) and empty sequences, each in batch order
+  for (int b = tid; b < B; b += kDevPlanThreads) aux[b] = nsplit[b] > 1 ? 1 : 0;
+  __syncthreads();
+  const int n_combine = dev::block_exclusive_scan(aux, B, warp_tot);
+  for (int b = tid; b < B; b += kDevPlanThreads) {
+    if (nsplit[b] > 1) p.fixes[aux[b]] = make_int4(b, offs[b], nsplit[b], p.seq_lens[b]);
+  }
+  __syncthreads();
+  for (int b = tid; b < B; b += kDevPlanThreads) aux[b] = (nsplit[b] == 0) ? 1 : 0;
+  __syncthreads();
+  const int n_empty = dev::block_exclusive_scan(aux, B, warp_tot);
+  for (int b = tid; b < B; b += kDevPlanThreads) {
+    if (nsplit[b] == 0) p.entries[n_items + aux[b]] = make_int4(b, 0, 0, 0);
+  }
+
+  // ---- items in (b, j) order
+  for (int b = tid; b < B; b += kDevPlanThreads) {
+    const int len = p.seq_lens[b];
+    for (int j = 0; j < nsplit[b]; ++j) {
+      const int i = offs[b] + j;
+      const int lo = j * chunk[b];
+      const int hi = min(len, lo + chunk[b]);
+      it_len[i] = hi - lo;
+      it_b[i] = b;
+      it_j[i] = j;
+    }
+  }
+  __syncthreads();
+
+  // ---- longest first, ties in (b, j) order: the rank of item i is the number of items before it
+  for (int i = tid; i < n_items; i += kDevPlanThreads) {
+    const int len = it_len[i];
+    int rank = 0;
+    for (int k = 0; k < n_items; ++k) {
+      const int lk = it_len[k];
+      rank += (lk > len || (lk == len && k < i)) ? 1 : 0;
+    }
+    const int b = it_b[i], j = it_j[i];
+    const int lo = j * chunk[b];
+    p.entries[rank] = make_int4(b | (j << L::kChunkShift) | (nsplit[b] << L::kCountShift), lo, lo + len,
+                                (nsplit[b] > 1) ? offs[b] + j : -1);
+  }
+  if (tid == 0) {
+    p.counts[L::kCntItems] = n_items;
+    p.counts[L::kCntCombine] = n_combine;
+    p.counts[L::kCntEmpty] = n_empty;
+    p.counts[L::kCntChunkTarget] = int(base);
+    p.counts[L::kCntOverflow] = 0;
+  }
+}
+
+}  // namespace libra

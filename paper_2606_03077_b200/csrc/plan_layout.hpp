@@ -8,7 +8,8 @@
 //
 // Plans of up to kParamEntries entries (and kParamFixEntries merges) do not go through device memory
 // at all: they are passed to the kernels by value as a kernel parameter, which saves the upload and
-// its place in the stream.  Larger plans are uploaded into the workspace in the same format.
+// its place in the stream.  Larger plans are uploaded into the workspace in the same format, and the
+// device-side planner writes its plan there too, preceded by kCountInts counts that the kernels read.
 #pragma once
 #include <cstdint>
 
@@ -22,6 +23,13 @@ constexpr int kCountShift = 24;
 constexpr int kMaxBatch = 1 << kChunkShift;
 constexpr int kParamEntries = 768;  // 12 KB of the 32 KB kernel-parameter space
 constexpr int kParamFixEntries = 256;
+// counts written by the device-side planner (int32 words at the start of the workspace's plan region)
+constexpr int kCountInts = 8;
+constexpr int kCntItems = 0;
+constexpr int kCntCombine = 1;
+constexpr int kCntEmpty = 2;
+constexpr int kCntChunkTarget = 3;
+constexpr int kCntOverflow = 4;
 }  // namespace plan_layout
 
 struct ParamPlan {
@@ -35,3 +43,4 @@ struct ParamFix {  // merges for the stand-alone combine kernel: {b, first_slot,
 #define LIBRA_DEV_ERR_WAIT_TIMEOUT 1u
 #define LIBRA_DEV_ERR_BAD_PAGE_ID 2u
 #define LIBRA_DEV_ERR_SEQ_LEN_MISMATCH 4u
+#define LIBRA_DEV_ERR_PLAN_OVERFLOW 8u

@@ -1,0 +1,173 @@
+"""The device-side planner (libra_plan_device): bit-exact against the reference planner, the decode
+step on a device-made plan against the step on a host-made plan, the overflow checks, and a whole step
+recorded once in a CUDA graph and replayed over changing lengths."""
+import numpy as np
+import pytest
+
+from oracle import attention_oracle as O
+from oracle import planner_ref as P
+from paper_2606_03077_b200 import workloads as W
+
+import gates
+import gpu_harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def ref_params(h):
+    p = h.plan_params()
+    return P.PlanParams(p.n_sm, p.ctas_per_sm, p.items_per_slot, p.chunk_align, p.min_chunk, p.max_splits)
+
+
+def assert_same_plan(got, ref):
+    assert got["chunk_target"] == ref.chunk_target
+    assert list(got["bucket"]) == ref.bucket
+    assert list(got["num_splits"]) == ref.num_splits
+    assert list(got["chunk_len"]) == ref.chunk_len
+    assert list(got["item_offset"]) == ref.item_offset
+    assert [tuple(r) for r in got["items"]] == ref.items
+    assert list(got["combine"]) == ref.combine
+    assert list(got["empty"]) == ref.empty
+
+
+def device_plan(lib, lens, hkv, plan=None, ld=None, max_batch=None):
+    import torch
+    lens = np.asarray(lens, dtype=np.int32)
+    B = len(lens)
+    ld = ld or max(1, int((lens.max() + 15) // 16) if B else 1)
+    h = lib.Handle(hkv * 4, hkv, 128, 16, max_batch or max(B, 1), ld, plan=plan)
+    ws = torch.zeros(h.workspace_size(), dtype=torch.uint8, device="cuda:0")
+    dl = torch.from_numpy(lens.copy()).to("cuda:0")
+    h.plan_device(dl.data_ptr(), B, ws.data_ptr(), ws.numel(), torch.cuda.current_stream().cuda_stream)
+    return h, ws, dl
+
+
+@pytest.mark.parametrize("name", W.WORKLOAD_ORDER)
+def test_workload_plans_bit_exact(lib, name):
+    w = W.WORKLOADS[name]
+    for step in range(w.steps):
+        lay, _ = W.make_layout(name, step)
+        for plan in (None, lib.PlanParams(0, 2, 4, 256, 512, 64)):
+            h, ws, dl = device_plan(lib, lay.seq_lens, w.num_kv_heads, plan)
+            assert_same_plan(h.plan_export(), P.plan(lay.seq_lens, w.num_kv_heads, ref_params(h)))
+            assert h.debug_error_word() == 0
+            h.close()
+
+
+def test_random_and_edge_vectors_bit_exact(lib):
+    rng = np.random.default_rng(11)
+    cases = [np.zeros(5, np.int32), np.array([1], np.int32), np.array([40960] * 64, np.int32),
+             np.array([16, 17, 255, 256, 257, 511, 512, 513, 0, 0, 4096], np.int32),
+             np.array([1024] * 7 + [2048] * 3, np.int32)]
+    for _ in range(40):
+        B = int(rng.integers(1, 600))
+        cases.append(np.clip(np.floor(rng.choice([16, 300, 2000, 12000]) * np.exp(rng.normal(size=B) * rng.uniform(0.2, 1.5))),
+                             0, 40960).astype(np.int32))
+    for i, lens in enumerate(cases):
+        hkv = int(rng.choice([1, 2, 8]))
+        plan = lib.PlanParams(int(rng.choice([4, 148])), int(rng.integers(1, 4)), int(rng.integers(1, 6)),
+                              int(rng.choice([16, 64, 256])), int(rng.choice([16, 512])), int(rng.choice([1, 8, 64])))
+        h, ws, dl = device_plan(lib, lens, hkv, plan)
+        ref = P.plan(lens, hkv, ref_params(h))
+        if len(ref.items) > 4096:
+            assert h.debug_error_word() & lib.ERR_PLAN_OVERFLOW
+        else:
+            assert_same_plan(h.plan_export(), ref)
+            assert h.debug_error_word() == 0
+        h.close()
+
+
+def test_overflow_is_flagged_and_nothing_runs(lib):
+    import torch
+    # a length longer than a block-table row can describe
+    h, ws, dl = device_plan(lib, [100, 5000], 2, ld=8)
+    assert h.debug_error_word() & lib.ERR_PLAN_OVERFLOW
+    assert len(h.plan_export()["items"]) == 0
+    h.close()
+    # more than 4096 work items
+    h, ws, dl = device_plan(lib, [40960] * 100, 1, plan=lib.PlanParams(148, 2, 64, 16, 16, 64))
+    assert h.debug_error_word() & lib.ERR_PLAN_OVERFLOW
+    h.close()
+    # more sequences than one block plans
+    h = lib.Handle(8, 2, 128, 16, 5000, 4)
+    ws = torch.zeros(h.workspace_size(), dtype=torch.uint8, device="cuda:0")
+    dl = torch.zeros(5000, dtype=torch.int32, device="cuda:0")
+    with pytest.raises(lib.LibraError) as e:
+        h.plan_device(dl.data_ptr(), 5000, ws.data_ptr(), ws.numel(), torch.cuda.current_stream().cuda_stream)
+    assert e.value.status == lib.UNSUPPORTED_SHAPE
+    h.close()
+
+
+def test_step_on_device_plan_equals_step_on_host_plan(lib):
+    import torch
+    dev = torch.device("cuda:0")
+    lens = [5000, 1300, 0, 37, 2049, 1]
+    Hq, Hkv, d = 32, 8, 128
+    lens_a, bt, q, k, v = W.random_case(51, len(lens), Hq, Hkv, d, lens)
+    ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
+    for plan in (None, lib.PlanParams(0, 2, 8, 256, 256, 64)):
+        r = H.Runner(lib, Hq, Hkv, d, k.shape[0], len(lens), bt.shape[1], plan=plan)
+        dq, dk, dv, dbt = (H.to_dev(x, dev) for x in (q, k, v, bt))
+        host = H.bf16_dev_to_f32(r.run(dq, dk, dv, dbt, lens_a))
+        dl = torch.from_numpy(lens_a.copy()).to(dev)
+        out = torch.full((len(lens), Hq, d), H.CANARY, dtype=torch.int16, device=dev)
+        st = torch.cuda.current_stream().cuda_stream
+        r.h.plan_device(dl.data_ptr(), len(lens), r.ws.data_ptr(), r.ws.numel(), st)
+        r.h.decode_attn(dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dbt.data_ptr(), dl.data_ptr(), out.data_ptr(), st)
+        torch.cuda.synchronize()
+        assert r.h.debug_error_word() == 0
+        got = H.bf16_dev_to_f32(out)
+        assert np.array_equal(got, host)
+        assert gates.tight_violations(got, ref) == 0 and gates.stated_violations(got, ref) == 0
+        r.h.close()
+
+
+def test_recorded_step_replays_over_changing_lengths(lib):
+    """plan + decode + combine recorded once in a CUDA graph; every replay plans the lengths that are in
+    device memory at that moment."""
+    import torch
+    dev = torch.device("cuda:0")
+    Hq, Hkv, d, B = 16, 4, 128, 6
+    steps = [[3000, 40, 1, 700, 2049, 16], [17, 4096, 900, 0, 333, 2500], [1, 1, 1, 1, 1, 1]]
+    ld = 4096 // 16
+    pool = sum((max(L, 1) + 15) // 16 for L in steps[0]) + 400
+    rng = np.random.default_rng(3)
+    k = W.f32_to_bf16_bits(rng.standard_normal((pool, Hkv, 16, d), dtype=np.float32))
+    v = W.f32_to_bf16_bits(rng.standard_normal((pool, Hkv, 16, d), dtype=np.float32))
+    q = W.f32_to_bf16_bits(rng.standard_normal((B, Hq, d), dtype=np.float32))
+    h = lib.Handle(Hq, Hkv, d, pool, B, ld, plan=lib.PlanParams(0, 2, 8, 256, 256, 64))
+    ws = torch.zeros(h.workspace_size(), dtype=torch.uint8, device=dev)
+    dq, dk, dv = (H.to_dev(x, dev) for x in (q, k, v))
+    dbt = torch.full((B, ld), -1, dtype=torch.int32, device=dev)
+    dl = torch.zeros(B, dtype=torch.int32, device=dev)
+    out = torch.zeros((B, Hq, d), dtype=torch.int16, device=dev)
+
+    def tables(lens):
+        bt, _ = W.draw_block_table(np.asarray(lens, np.int32), pool, np.random.default_rng(sum(lens)), ld=ld)
+        return bt
+
+    side = torch.cuda.Stream()
+    bt0 = tables(steps[0])
+    dbt.copy_(torch.from_numpy(bt0)); dl.copy_(torch.tensor(steps[0], dtype=torch.int32))
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):   # one eager step first: sets up the workspace outside the recording
+        h.plan_device(dl.data_ptr(), B, ws.data_ptr(), ws.numel(), side.cuda_stream)
+        h.decode_attn(dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dbt.data_ptr(), dl.data_ptr(), out.data_ptr(), side.cuda_stream)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        h.plan_device(dl.data_ptr(), B, ws.data_ptr(), ws.numel(), side.cuda_stream)
+        h.decode_attn(dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dbt.data_ptr(), dl.data_ptr(), out.data_ptr(), side.cuda_stream)
+    for lens in steps + [steps[0]]:
+        bt = tables(lens)
+        dbt.copy_(torch.from_numpy(bt)); dl.copy_(torch.tensor(lens, dtype=torch.int32))
+        out.fill_(H.CANARY)
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        got = H.bf16_dev_to_f32(out)
+        ref, _ = O.paged_decode_attention(q, k, v, bt, np.asarray(lens, np.int32))
+        assert np.all(np.isfinite(got))
+        assert gates.tight_violations(got, ref) == 0 and gates.stated_violations(got, ref) == 0, lens
+    assert h.debug_error_word() == 0
+    h.close()
