@@ -44,8 +44,8 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES_ASSUMED = 126 * 1024 * 1024
 # DRAM bytes (read + write) of one decode-kernel launch on MAIN_WORKLOAD from an ncu capture, see
-# profiles/decode_kernel_lognormal_b64.md (370.61 MB read + 4.20 MB written).
-NCU_DECODE_TRAFFIC_BYTES = 374.8e6
+# profiles/decode_kernel_lognormal_b64.md (370.62 MB read + 4.10 MB written).
+NCU_DECODE_TRAFFIC_BYTES = 374.7e6
 
 
 # ----------------------------------------------------------------------------- clocks
@@ -412,12 +412,19 @@ def run_libra(args):
     value = units_all / (t_max * 1e-3) / 1e9
 
     peak, peak_src = measured_hbm_peak()
-    achieved = rep.kv_bytes_per_step / (dec_ms * 1e-3) / 1e9
+    # average launch duration of the decode kernel: when a step is that one launch, the timed region itself
+    # (events around K back-to-back launches) gives it; otherwise the per-kernel event pairs do, each of
+    # which adds ~3 us to what it brackets
+    one_launch_per_step = launches == args.steps
+    kernel_ms = (elapsed_ms / args.steps) if one_launch_per_step else dec_ms
+    achieved = rep.kv_bytes_per_step / (kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_src, "traffic": NCU_DECODE_TRAFFIC_BYTES,
-                "algorithmic_bytes_per_launch": rep.kv_bytes_per_step, "decode_kernel_us": dec_ms * 1e3,
-                "combine_kernel_us": cmb_ms * 1e3, "launches_timed": n_prof,
-                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
+                "algorithmic_bytes_per_launch": rep.kv_bytes_per_step, "kernel_us": kernel_ms * 1e3,
+                "timing": ("CUDA events around the timed region, one decode launch per step" if one_launch_per_step
+                           else "CUDA event pair around every decode launch"),
+                "decode_kernel_us_with_event_pairs": dec_ms * 1e3, "after_decode_us_with_event_pairs": cmb_ms * 1e3,
+                "launches_timed": n_prof, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -427,7 +434,7 @@ def run_libra(args):
                        "kv_bytes_per_step": rep.kv_bytes_per_step, "parallelism": f"replicas x{world}",
                        "l2": f"rotating {len(rep.pools)} copies of the KV pools "
                              f"({len(rep.pools) * rep.layouts[0].kv_bytes / 1e9:.2f} GB live KV vs 126 MB L2)",
-                       "step": "libra_plan + decode kernel + combine kernel"},
+                       "step": "libra_plan + decode kernel (step C runs inside it)"},
             "steps_per_s": 1e3 / ms_per_step * world,
             "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
             "frac_of_measured_copy": value / world / peak,

@@ -75,7 +75,7 @@ typedef enum {
  * min-max objective).  A zero field takes its default. */
 typedef struct {
   int32_t n_sm;           /* SMs to plan for; 0 = the device's count (148 on B200)               */
-  int32_t ctas_per_sm;    /* resident decode blocks per SM the plan assumes; default 2           */
+  int32_t ctas_per_sm;    /* resident decode blocks per SM the plan assumes; default 1           */
   int32_t items_per_slot; /* target work units per resident block; default 1                    */
   int32_t chunk_align;    /* A: chunk lengths are multiples of this many tokens (itself a
                              multiple of 16); default 256                                       */
@@ -148,11 +148,11 @@ int libra_get_plan_params(libra_handle_t handle, libra_plan_params_t* out);
  * count changes the order of the per-unit merge and hence the last bits of the result. */
 int libra_set_variant(libra_handle_t handle, int32_t warps, int32_t stages);
 
-/* Where step C runs.  fused = 1: inside the decode kernel, by the block that publishes the
- * last partial result of a split sequence (one launch per call).  fused = 0 (default): as a separate combine
- * kernel after the decode kernel (two launches).  Both orders of evaluation are the same, so the two
- * modes give bit-identical results. */
-int libra_set_combine_mode(libra_handle_t handle, int32_t fused);
+/* Where step C runs.  mode 1 (default): inside the decode kernel, by the block that publishes the last
+ * partial result of a split sequence (one launch per step).  mode 0: as a separate combine kernel after
+ * the decode kernel (two launches; the second is a programmatic dependent of the first).  The merge code
+ * and its order of evaluation are the same, so both modes give bit-identical results. */
+int libra_set_combine_mode(libra_handle_t handle, int32_t mode);
 
 /* Step P as a pure host function (needs no GPU): the length-bucketed planner (Sections 2.3, 4.3
  * and 5 of the paper give the bucket properties it mirrors).  With W = n_sm * ctas_per_sm,

@@ -32,7 +32,7 @@ from dataclasses import dataclass
 @dataclass(frozen=True)
 class PlanParams:
     n_sm: int = 148
-    ctas_per_sm: int = 2
+    ctas_per_sm: int = 1
     items_per_slot: int = 1
     chunk_align: int = 256      # A: chunk lengths are multiples of this many tokens
     min_chunk: int = 512        # C_min

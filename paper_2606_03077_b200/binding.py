@@ -163,8 +163,9 @@ class Handle:
     def set_variant(self, warps: int, stages: int) -> None:
         _check(lib.libra_set_variant(self._h, warps, stages), "libra_set_variant")
 
-    def set_combine_mode(self, fused: bool) -> None:
-        _check(lib.libra_set_combine_mode(self._h, 1 if fused else 0), "libra_set_combine_mode")
+    def set_combine_mode(self, mode: int) -> None:
+        """0: separate combine kernel, 1: inside the decode kernel (default)."""
+        _check(lib.libra_set_combine_mode(self._h, int(mode)), "libra_set_combine_mode")
 
     def plan(self, seq_lens_host: np.ndarray, workspace_ptr: int, workspace_bytes: int, stream: int) -> None:
         lens = _as_i32(seq_lens_host)

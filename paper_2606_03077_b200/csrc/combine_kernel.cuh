@@ -4,7 +4,7 @@
 //   M = max_i LSE_i ;  w_i = exp(LSE_i - M) ;  out = sum_i w_i O_i / sum_i w_i   -> bf16
 // Partials are summed in chunk order, so the result does not depend on scheduling.
 //
-// One warp per (sequence, head): lane i keeps w_i and w_{i+32}; every lane owns D/32 output
+// One warp per (sequence, head) row: lane i keeps w_i and w_{i+32}; every lane owns D/32 output
 // columns and walks the n partial rows with eight independent loads in flight.
 #pragma once
 #include <cuda_bf16.h>
@@ -29,27 +29,14 @@ struct CombineParams {
 
 constexpr int kCombineWarps = 4;
 
-// grid = (fix-up entries, ceil(Hq / kCombineWarps)), block = kCombineWarps warps
+// One warp merges the n (<= 64) partial results of one (sequence, head) row and writes the bf16 row.
+// Shared by the combine kernel and by the decode kernel's in-kernel merge, so both give the same bits.
+// Loads bypass L1 (the partials were written by other SMs, possibly during this very launch).
 template <int D>
-__global__ void __launch_bounds__(kCombineWarps * 32)
-combine_kernel(const __grid_constant__ CombineParams p, const __grid_constant__ ParamFix pf) {
+__device__ __forceinline__ void combine_row(const float* partial_o, const float* partial_lse, __nv_bfloat16* out, int b,
+                                            int first, int n, int Hq, int h, int lane) {
   constexpr int V = D / 32;  // columns per lane: 4 (float4) or 2 (float2)
-  const int lane = threadIdx.x & 31;
-  const int h = blockIdx.y * kCombineWarps + (threadIdx.x >> 5);
-  const int Hq = p.num_q_heads;
-  if (h >= Hq) return;
-  if (p.dev_counts && int(blockIdx.x) >= p.dev_counts[plan_layout::kCntCombine]) return;  // grid is an upper bound
-  const int4 fix = (p.entries ? p.entries : pf.e)[blockIdx.x];  // plain load: may address parameter space
-  const int b = fix.x;
-  const int first = fix.y;
-  const int n = fix.z;  // <= 64
-  // launched as a programmatic dependent of the decode kernel: wait until that grid has finished
-  // and its partial results are visible
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (lane == 0 && h == 0 && fix.w != __ldg(p.seq_lens + b)) {
-    atomicOr(p.error_word, LIBRA_DEV_ERR_SEQ_LEN_MISMATCH);
-  }
-  const float* lse = p.partial_lse + int64_t(first) * Hq + h;
+  const float* lse = partial_lse + int64_t(first) * Hq + h;
   const float l0 = (lane < n) ? __ldcg(lse + int64_t(lane) * Hq) : -INFINITY;
   const float l1 = (lane + 32 < n) ? __ldcg(lse + int64_t(lane + 32) * Hq) : -INFINITY;
   float m = fmaxf(l0, l1);
@@ -62,7 +49,7 @@ combine_kernel(const __grid_constant__ CombineParams p, const __grid_constant__ 
 #pragma unroll
   for (int v = 0; v < V; ++v) num[v] = 0.f;
   float den = 0.f;
-  const float* po = p.partial_o + (int64_t(first) * Hq + h) * D + lane * V;
+  const float* po = partial_o + (int64_t(first) * Hq + h) * D + lane * V;
   const int64_t stride = int64_t(Hq) * D;
   for (int i0 = 0; i0 < n; i0 += 8) {
     float o[8][V];
@@ -91,11 +78,30 @@ combine_kernel(const __grid_constant__ CombineParams p, const __grid_constant__ 
     }
   }
   const float inv = (n > 0) ? 1.f / den : 0.f;
-  __nv_bfloat16* dst = p.out + (int64_t(b) * Hq + h) * D + lane * V;
+  __nv_bfloat16* dst = out + (int64_t(b) * Hq + h) * D + lane * V;
 #pragma unroll
   for (int v = 0; v < V; v += 2) {
     *reinterpret_cast<__nv_bfloat162*>(dst + v) = __floats2bfloat162_rn(num[v] * inv, num[v + 1] * inv);
   }
+}
+
+// grid = (fix-up entries, ceil(Hq / kCombineWarps)), block = kCombineWarps warps
+template <int D>
+__global__ void __launch_bounds__(kCombineWarps * 32)
+combine_kernel(const __grid_constant__ CombineParams p, const __grid_constant__ ParamFix pf) {
+  const int lane = threadIdx.x & 31;
+  const int h = blockIdx.y * kCombineWarps + (threadIdx.x >> 5);
+  const int Hq = p.num_q_heads;
+  if (h >= Hq) return;
+  if (p.dev_counts && int(blockIdx.x) >= p.dev_counts[plan_layout::kCntCombine]) return;  // grid is an upper bound
+  const int4 fix = (p.entries ? p.entries : pf.e)[blockIdx.x];  // plain load: may address parameter space
+  // launched as a programmatic dependent of the decode kernel: wait until that grid has finished
+  // and its partial results are visible
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (lane == 0 && h == 0 && fix.w != __ldg(p.seq_lens + fix.x)) {
+    atomicOr(p.error_word, LIBRA_DEV_ERR_SEQ_LEN_MISMATCH);
+  }
+  combine_row<D>(p.partial_o, p.partial_lse, p.out, fix.x, fix.y, fix.z, Hq, h, lane);
 }
 
 }  // namespace libra

@@ -27,6 +27,7 @@
 
 #include <cstdint>
 
+#include "combine_kernel.cuh"
 #include "plan_layout.hpp"
 
 namespace libra {
@@ -568,30 +569,9 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  const int first_slot = u.slot - u.chunk_j;
-  float* w_sm = reinterpret_cast<float*>(ring);   // [n_chunks][G] weights, then [G] 1/denominator
-  float* inv_sm = w_sm + u.n_chunks * G;
-  for (int h = threadIdx.x; h < G; h += NW * 32) {
-    const float* lse = p.partial_lse + int64_t(first_slot) * p.num_q_heads + int64_t(kvh) * G + h;
-    float mx = -INFINITY;
-    for (int i = 0; i < u.n_chunks; ++i) mx = fmaxf(mx, __ldcg(lse + int64_t(i) * p.num_q_heads));
-    float den = 0.f;
-    for (int i = 0; i < u.n_chunks; ++i) {
-      const float w = __expf(__ldcg(lse + int64_t(i) * p.num_q_heads) - mx);
-      w_sm[i * G + h] = w;
-      den += w;
-    }
-    inv_sm[h] = 1.f / den;
-  }
-  __syncthreads();
-  for (int idx = threadIdx.x; idx < G * D; idx += NW * 32) {
-    const int h = idx / D;
-    const int dim = idx - h * D;
-    const float* po = p.partial_o + (int64_t(first_slot) * p.num_q_heads + int64_t(kvh) * G + h) * D + dim;
-    float num = 0.f;
-#pragma unroll 4
-    for (int i = 0; i < u.n_chunks; ++i) num += w_sm[i * G + h] * __ldcg(po + int64_t(i) * p.num_q_heads * D);
-    p.out[(int64_t(u.b) * p.num_q_heads + int64_t(kvh) * G + h) * D + dim] = __float2bfloat16_rn(num * inv_sm[h]);
+  // one warp per query head of this KV head, exactly as the combine kernel would do it
+  for (int h = warp; h < G; h += NW) {
+    combine_row<D>(p.partial_o, p.partial_lse, p.out, u.b, u.slot - u.chunk_j, u.n_chunks, p.num_q_heads, kvh * G + h, lane);
   }
 }
 

@@ -10,7 +10,6 @@
 #include <new>
 #include <vector>
 
-#include "combine_kernel.cuh"
 #include "decode_kernel.cuh"
 #include "libra.h"
 #include "plan_kernel.cuh"
@@ -56,8 +55,8 @@ Variant make_variant() {
 // Block shapes that are compiled in; index 0 is the default.
 const std::vector<Variant>& variants() {
   static const std::vector<Variant> v = {
-      make_variant<4, 3>(), make_variant<4, 2>(), make_variant<4, 4>(), make_variant<4, 6>(),
-      make_variant<8, 2>(), make_variant<8, 3>(), make_variant<2, 6>(), make_variant<2, 4>(),
+      make_variant<8, 3>(), make_variant<8, 2>(), make_variant<4, 3>(), make_variant<4, 2>(),
+      make_variant<4, 4>(), make_variant<4, 6>(), make_variant<2, 6>(), make_variant<2, 4>(),
   };
   return v;
 }
@@ -99,7 +98,7 @@ struct libra_handle_s {
   int64_t max_items = 0;
   size_t cnt_off = 0, cnt_bytes = 0, lse_off = 0, o_off = 0, plan_off = 0, plan_bytes = 0, workspace_bytes = 0;
   void* clean_workspace = nullptr;  // workspace whose control words and counters are known to be zero
-  bool fused_combine = false;
+  int combine_mode = 1;     // 0: separate kernel, 1: inside the decode kernel
   bool pdl_combine = true;
 
   // pinned staging for uploads of plans too large for the kernel parameters
@@ -610,9 +609,9 @@ int libra_plan_export(libra_handle_t h, libra_plan_view_t* view) {
   return LIBRA_OK;
 }
 
-int libra_set_combine_mode(libra_handle_t h, int32_t fused) {
-  if (!h || (fused != 0 && fused != 1)) return LIBRA_INVALID_ARGUMENT;
-  h->fused_combine = (fused == 1);
+int libra_set_combine_mode(libra_handle_t h, int32_t mode) {
+  if (!h || mode < 0 || mode > 1) return LIBRA_INVALID_ARGUMENT;
+  h->combine_mode = mode;
   return LIBRA_OK;
 }
 
@@ -684,7 +683,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
   const Variant& v = variants()[h->variant];
   const int di = (h->cfg.head_dim == 128) ? 1 : 0;
   const int ni = (h->group > 8) ? 1 : 0;
-  const bool fused = h->fused_combine;
+  const bool fused = h->combine_mode == 1;
   // host plan: exact counts; device plan: upper bounds for the grids, the kernels read the counts themselves
   const int32_t n_empty = h->device_planned ? h->planned_batch : int32_t(h->plan.empty.size());
   const int32_t n_combine = h->device_planned ? h->planned_batch : int32_t(h->plan.combine.size());

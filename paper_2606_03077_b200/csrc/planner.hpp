@@ -13,7 +13,7 @@ namespace libra {
 
 struct PlanParams {
   int32_t n_sm = 148;
-  int32_t ctas_per_sm = 2;
+  int32_t ctas_per_sm = 1;
   int32_t items_per_slot = 1;
   int32_t chunk_align = 256;
   int32_t min_chunk = 512;

@@ -64,8 +64,9 @@ def test_shapes_and_tails(lib, case, layout):
         got = H.run_host_case(lib, q, k, v, bt, lens_a, layout=layout, plan=plan)
         check(got, ref, f"case {case} {layout} plan={'default' if plan is None else 'small'}")
     # step C as its own kernel gives the same bits as step C inside the decode kernel
-    two = H.run_host_case(lib, q, k, v, bt, lens_a, layout=layout, plan=small_plan(lib), fused=False)
-    assert np.array_equal(two, got)
+    two = H.run_host_case(lib, q, k, v, bt, lens_a, layout=layout, plan=small_plan(lib), fused=0)
+    one = H.run_host_case(lib, q, k, v, bt, lens_a, layout=layout, plan=small_plan(lib), fused=1)
+    assert np.array_equal(two, got) and np.array_equal(one, got)
 
 
 def test_every_block_shape_agrees(lib):

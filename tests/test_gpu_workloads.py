@@ -47,9 +47,10 @@ def test_workload_parity(lib, name, n_sample):
         assert gates.tight_violations(got, ref) == 0, gates.tight_ratio(got, ref)
         # property that holds for every sequence: |out| <= max |v| over the pool (a convex combination)
         assert np.max(np.abs(out)) <= 6.5
-        r.h.set_combine_mode(False)   # the two-launch form of step C: same bits
-        out2 = H.bf16_dev_to_f32(r.run(q, k, v, H.to_dev(bt, dev), lay.seq_lens))
-        r.h.set_combine_mode(True)
-        assert np.array_equal(out, out2)
+        for mode in (0, 1):           # step C as its own kernel / inside the decode kernel: same bits
+            r.h.set_combine_mode(mode)
+            out2 = H.bf16_dev_to_f32(r.run(q, k, v, H.to_dev(bt, dev), lay.seq_lens))
+            assert np.array_equal(out, out2)
+        r.h.set_combine_mode(1)
         W.restore_tails(saved, k, v)
     r.h.close()

@@ -91,12 +91,12 @@ def test_random_vectors_default_params():
     ("shift_b128", 2, 5632, 239)])
 def test_workload_plans(name, step, C, n_items):
     lay, _ = W.make_layout(name, step)
-    pl = check_plan([int(x) for x in lay.seq_lens], lay.workload.num_kv_heads, P.PlanParams(items_per_slot=4))
+    pl = check_plan([int(x) for x in lay.seq_lens], lay.workload.num_kv_heads, P.PlanParams(ctas_per_sm=2, items_per_slot=4))
     assert pl.chunk_target == C and len(pl.items) == n_items
     check_plan([int(x) for x in lay.seq_lens], lay.workload.num_kv_heads, P.PlanParams())
 
 
 def test_straggler_is_split_32_ways():
     lay, _ = W.make_layout("straggler_b8")
-    pl = P.plan(lay.seq_lens, 8, P.PlanParams(items_per_slot=4))
+    pl = P.plan(lay.seq_lens, 8, P.PlanParams(ctas_per_sm=2, items_per_slot=4))
     assert set(pl.bucket) == {5} and set(pl.chunk_len) == {1024} and set(pl.num_splits) == {32}

@@ -23,7 +23,7 @@ def test_static_scratch_entry_point_matches_workspace_path(lib):
     Hq, Hkv, d = 32, 8, 128
     lens_a, bt, q, k, v = W.random_case(41, len(lens), Hq, Hkv, d, lens)
     plan = lib.PlanParams(0, 2, 4, 256, 512, 64)     # several split sequences: partial results go through the scratch
-    r = H.Runner(lib, Hq, Hkv, d, k.shape[0], len(lens), bt.shape[1], plan=plan)
+    r = H.Runner(lib, Hq, Hkv, d, k.shape[0], len(lens), bt.shape[1], plan=plan, fused=0)   # decode + combine kernels
     assert r.h.workspace_size() <= lib.STATIC_SCRATCH_BYTES
     dq, dk, dv, dbt = (H.to_dev(x, dev) for x in (q, k, v, bt))
     want = H.bf16_dev_to_f32(r.run(dq, dk, dv, dbt, lens_a))
