@@ -148,6 +148,13 @@ int libra_get_plan_params(libra_handle_t handle, libra_plan_params_t* out);
  * count changes the order of the per-unit merge and hence the last bits of the result. */
 int libra_set_variant(libra_handle_t handle, int32_t warps, int32_t stages);
 
+/* Programmatic dependent launch, on by default: the decode kernel is launched so that its blocks may
+ * become resident while the kernel before it in the stream drains (and the separate combine kernel
+ * likewise after the decode kernel); inside, they wait for that kernel to finish before they read any
+ * input, so ordering and results are exactly those of ordinary launches - only the launch latency
+ * and block start-up overlap the predecessor's tail.  on = 0 makes every launch an ordinary one. */
+int libra_set_dependent_launch(libra_handle_t handle, int32_t on);
+
 /* Where step C runs.  mode 1 (default): inside the decode kernel, by the block that publishes the last
  * partial result of a split sequence (one launch per step).  mode 0: as a separate combine kernel after
  * the decode kernel (two launches; the second is a programmatic dependent of the first).  The merge code

@@ -57,6 +57,7 @@ SIGNATURES = {
     "libra_workspace_size": (C.c_int, [_vp, C.POINTER(C.c_size_t)]),
     "libra_get_plan_params": (C.c_int, [_vp, C.POINTER(PlanParams)]),
     "libra_set_variant": (C.c_int, [_vp, C.c_int32, C.c_int32]),
+    "libra_set_dependent_launch": (C.c_int, [_vp, C.c_int32]),
     "libra_set_combine_mode": (C.c_int, [_vp, C.c_int32]),
     "libra_plan_host": (C.c_int, [C.POINTER(PlanParams), C.c_int32, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p,
                                   _i32p, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p]),
@@ -162,6 +163,9 @@ class Handle:
 
     def set_variant(self, warps: int, stages: int) -> None:
         _check(lib.libra_set_variant(self._h, warps, stages), "libra_set_variant")
+
+    def set_dependent_launch(self, on: bool) -> None:
+        _check(lib.libra_set_dependent_launch(self._h, 1 if on else 0), "libra_set_dependent_launch")
 
     def set_combine_mode(self, mode: int) -> None:
         """0: separate combine kernel, 1: inside the decode kernel (default)."""

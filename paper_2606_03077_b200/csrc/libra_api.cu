@@ -99,7 +99,7 @@ struct libra_handle_s {
   size_t cnt_off = 0, cnt_bytes = 0, lse_off = 0, o_off = 0, plan_off = 0, plan_bytes = 0, workspace_bytes = 0;
   void* clean_workspace = nullptr;  // workspace whose control words and counters are known to be zero
   int combine_mode = 1;     // 0: separate kernel, 1: inside the decode kernel
-  bool pdl_combine = true;
+  bool pdl = true;          // programmatic dependent launches (decode after its predecessor, combine after decode)
 
   // pinned staging for uploads of plans too large for the kernel parameters
   int32_t* staging[2] = {nullptr, nullptr};
@@ -615,6 +615,12 @@ int libra_set_combine_mode(libra_handle_t h, int32_t mode) {
   return LIBRA_OK;
 }
 
+int libra_set_dependent_launch(libra_handle_t h, int32_t on) {
+  if (!h || (on != 0 && on != 1)) return LIBRA_INVALID_ARGUMENT;
+  h->pdl = (on == 1);
+  return LIBRA_OK;
+}
+
 int libra_set_variant(libra_handle_t h, int32_t warps, int32_t stages) {
   if (!h) return LIBRA_INVALID_ARGUMENT;
   const std::vector<Variant>& vs = variants();
@@ -722,8 +728,19 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     p.stride_head = h->stride_head;
     p.stride_token = h->stride_token;
     const unsigned grid = unsigned(n_units) + unsigned(n_empty);
-    v.fn[di][ni]<<<grid, v.warps * 32, v.smem[di][ni], st>>>(pm->map_k, pm->map_v, p, h->pp);
-    LIBRA_CUDA_TRY(h, cudaGetLastError());
+    // launched as a programmatic dependent of whatever precedes it in the stream: its blocks may become
+    // resident while that kernel drains; inside, they wait for it to finish before reading any input
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(grid);
+    lc.blockDim = dim3(unsigned(v.warps * 32));
+    lc.dynamicSmemBytes = size_t(v.smem[di][ni]);
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = h->pdl ? 1 : 0;
+    LIBRA_CUDA_TRY(h, cudaLaunchKernelEx(&lc, v.fn[di][ni], pm->map_k, pm->map_v, p, h->pp));
     ++h->launches;
   }
   if (ev) LIBRA_CUDA_TRY(h, cudaEventRecord(ev[1], st));
@@ -750,7 +767,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
-    lc.numAttrs = (ev || !h->pdl_combine) ? 0 : 1;  // with events around it, it is an ordinary launch
+    lc.numAttrs = (ev || !h->pdl) ? 0 : 1;  // with events around it, it is an ordinary launch
     if (h->cfg.head_dim == 128) LIBRA_CUDA_TRY(h, cudaLaunchKernelEx(&lc, libra::combine_kernel<128>, c, h->pf));
     else LIBRA_CUDA_TRY(h, cudaLaunchKernelEx(&lc, libra::combine_kernel<64>, c, h->pf));
     ++h->launches;
