@@ -292,6 +292,12 @@ int libra_last_cuda_error(libra_handle_t handle);
  * a non-zero word clears it.  Errors: NOT_PLANNED, CUDA_ERROR. */
 int libra_debug_error_word(libra_handle_t handle, uint32_t* word);
 
+/* Self-test of the kernels' bounded waits: enqueues a one-warp kernel that waits, with a limit of a few
+ * milliseconds, on a copy barrier that nothing completes.  It must return (no hang, no trap) and leave
+ * LIBRA_ERR_WAIT_TIMEOUT in the device error word of the last planned workspace, which is how a real
+ * timeout inside the decode kernel would surface.  Errors: NOT_PLANNED, CUDA_ERROR. */
+int libra_debug_wait_selftest(libra_handle_t handle, void* stream);
+
 /* Per-kernel timing for benchmarks.  After libra_profile_begin, every libra_decode_attn records
  * CUDA events around the decode kernel and the combine kernel on the call's stream (at most
  * 4096 calls are kept).  libra_profile_end synchronises those events, returns the summed device

@@ -72,6 +72,7 @@ SIGNATURES = {
     "libra_host_staging_size": (C.c_int, [_vp, C.c_int32, C.POINTER(C.c_size_t)]),
     "libra_last_cuda_error": (C.c_int, [_vp]),
     "libra_debug_error_word": (C.c_int, [_vp, C.POINTER(C.c_uint32)]),
+    "libra_debug_wait_selftest": (C.c_int, [_vp, _vp]),
     "libra_profile_begin": (C.c_int, [_vp]),
     "libra_profile_end": (C.c_int, [_vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int32)]),
     "libra_launch_count": (C.c_int, [_vp, C.POINTER(C.c_int64)]),
@@ -228,6 +229,9 @@ class Handle:
         w = C.c_uint32(0)
         _check(lib.libra_debug_error_word(self._h, C.byref(w)), "libra_debug_error_word")
         return w.value
+
+    def debug_wait_selftest(self, stream: int) -> None:
+        _check(lib.libra_debug_wait_selftest(self._h, stream), "libra_debug_wait_selftest")
 
     def profile_begin(self) -> None:
         _check(lib.libra_profile_begin(self._h), "libra_profile_begin")

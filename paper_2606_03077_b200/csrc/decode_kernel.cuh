@@ -66,7 +66,8 @@ struct DecodeParams {
 
 namespace dev {
 
-constexpr uint32_t kWaitLimit = 1u << 22;  // bounded spin on a copy barrier
+constexpr uint32_t kWaitLimit = 1u << 20;  // tries of a bounded wait on a copy barrier (each suspends <= ~2 us)
+constexpr uint32_t kWaitHintNs = 2000;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
@@ -80,16 +81,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(kWaitHintNs)
       : "memory");
   return ok != 0;
 }
-// Returns false if the barrier did not complete within the limit.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+// Returns false if the barrier did not complete within `limit` tries.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit = kWaitLimit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
   }
   return false;
@@ -394,6 +395,19 @@ __device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontr
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 }  // namespace dev
+
+// Self-test of the bounded wait: one warp waits on a barrier that nothing ever completes, with a small
+// limit, and must come back with LIBRA_DEV_ERR_WAIT_TIMEOUT recorded instead of hanging.
+__global__ void wait_timeout_selftest_kernel(uint32_t* error_word, uint32_t tries) {
+  __shared__ uint64_t bar;
+  const uint32_t b = dev::smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    dev::mbar_init(b, 1);
+    dev::fence_mbar_init();
+  }
+  __syncwarp();
+  if (!dev::mbar_wait(b, 0, tries) && threadIdx.x == 0) atomicOr(error_word, LIBRA_DEV_ERR_WAIT_TIMEOUT);
+}
 
 template <int D, int NW, int STAGES>
 struct DecodeSmem {

@@ -888,6 +888,18 @@ int libra_debug_error_word(libra_handle_t h, uint32_t* word) {
   return LIBRA_OK;
 }
 
+int libra_debug_wait_selftest(libra_handle_t h, void* stream) {
+  if (!h) return LIBRA_INVALID_ARGUMENT;
+  if (!h->planned) return LIBRA_NOT_PLANNED;
+  DeviceGuard guard(h->cfg.device);
+  if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+  libra::wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(
+      reinterpret_cast<uint32_t*>(h->workspace), 1024u);
+  LIBRA_CUDA_TRY(h, cudaGetLastError());
+  h->last_stream = stream;
+  return LIBRA_OK;
+}
+
 int libra_profile_begin(libra_handle_t h) {
   if (!h) return LIBRA_INVALID_ARGUMENT;
   h->profiling = true;

@@ -255,6 +255,23 @@ def test_error_word_flags_bad_inputs(lib):
     assert r.h.debug_error_word() == 0
 
 
+def test_bounded_wait_times_out_cleanly(lib):
+    """A wait that can never be satisfied ends by itself, is reported in the error word, and the context
+    stays usable: the next step computes correct results."""
+    import torch
+    dev = torch.device("cuda:0")
+    lens_a, bt, q, k, v = W.random_case(31, 2, 8, 2, 128, [100, 40])
+    ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
+    r = H.Runner(lib, 8, 2, 128, k.shape[0], 2, bt.shape[1])
+    args = [H.to_dev(x, dev) for x in (q, k, v, bt)]
+    r.run(*args, lens_a)
+    r.h.debug_wait_selftest(torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert r.h.debug_error_word() == lib.ERR_WAIT_TIMEOUT
+    check(H.bf16_dev_to_f32(r.run(*args, lens_a)), ref, "after a timed-out wait")
+    r.h.close()
+
+
 def test_host_side_misuse(lib):
     import torch
     dev = torch.device("cuda:0")
