@@ -297,6 +297,55 @@ def e2e_measure(rep: Replica, steps: int):
     return ms, int(h2d), int(d2h), bool(same)
 
 
+def kv_migration_measure(rep: Replica, reps: int = 10):
+    """libra_kv_gather / libra_kv_scatter on the sequences of 16K tokens and more (the ones the paper's
+    scheduler would move to a larger bucket): bytes moved = read + write of K and V."""
+    torch = rep.torch
+    lay = rep.layouts[0]
+    rows = np.nonzero(lay.seq_lens >= 16384)[0]
+    if len(rows) == 0:
+        return None
+    lens = lay.seq_lens[rows]
+    offs = np.concatenate([[0], np.cumsum(lens.astype(np.int64))])
+    total = int(offs[-1])
+    w = rep.w
+    dbt = rep.bts[0][torch.from_numpy(rows).to(rep.dev)].contiguous()
+    dl = torch.from_numpy(lens.copy()).to(rep.dev)
+    doffs = torch.from_numpy(offs[:-1].copy()).to(rep.dev)
+    err = torch.zeros(1, dtype=torch.int32, device=rep.dev)
+    kd = torch.empty((total, w.num_kv_heads, w.head_dim), dtype=torch.bfloat16, device=rep.dev)
+    vd = torch.empty_like(kd)
+    k, v = rep.pools[0]
+    st = torch.cuda.current_stream().cuda_stream
+    args = (dbt.data_ptr(), dl.data_ptr(), doffs.data_ptr(), len(rows), int(lens.max()), 0, w.num_kv_heads)
+    res = {}
+    for what in ("gather", "scatter"):
+        def one():
+            if what == "gather":
+                rep.h.kv_gather(k.data_ptr(), v.data_ptr(), *args, kd.data_ptr(), vd.data_ptr(), err.data_ptr(), st)
+            else:
+                rep.h.kv_scatter(kd.data_ptr(), vd.data_ptr(), *args, k.data_ptr(), v.data_ptr(), err.data_ptr(), st)
+        for _ in range(3):
+            one()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            one()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        moved = 2 * 2 * total * w.num_kv_heads * w.head_dim * 2    # K and V, read and write
+        res[what] = {"ms": ms, "copy_gbs": moved / (ms * 1e-3) / 1e9}
+    assert int(err.item()) == 0
+    peak, _ = measured_hbm_peak()
+    return {"sequences": int(len(rows)), "tokens": total, "kv_bytes": 2 * total * w.num_kv_heads * w.head_dim * 2,
+            "gather": res["gather"], "scatter": res["scatter"],
+            "gather_frac_of_measured_copy": res["gather"]["copy_gbs"] / peak,
+            "scatter_frac_of_measured_copy": res["scatter"]["copy_gbs"] / peak,
+            "note": "dense buffer in device memory; read + write bytes over time, against the measured copy rate"}
+
+
 def oracle_baseline(name: str, k_dev=None, v_dev=None, q_dev=None, budget_s: float = 20.0):
     """Times the float64 oracle, as it stands, on the host cores on a bounded sample of the workload:
     whole sequences in batch order until about `budget_s` seconds of CPU work are spent."""
@@ -482,6 +531,8 @@ def run_libra(args):
                             "frac_of_nominal_8TBs": r.kv_bytes_per_step / (per * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
                             "frac_of_measured_copy": r.kv_bytes_per_step / (per * 1e-3) / 1e9 / peak,
                             "kv_bytes_per_step": r.kv_bytes_per_step, "pool_copies": len(r.pools)}
+            if name == "longtail_mix_b256":  # migrating the long tail: gather its KV to a dense buffer and scatter it back
+                others[name]["kv_migration"] = kv_migration_measure(r)
             if name == "shift_b128":  # the re-planned-every-step workload: also with the device-side planner
                 eager = r.timed_device_plan(n, 6, graph=False)
                 graph = r.timed_device_plan(n, 6, graph=True)

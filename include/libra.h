@@ -292,6 +292,34 @@ int libra_last_cuda_error(libra_handle_t handle);
  * a non-zero word clears it.  Errors: NOT_PLANNED, CUDA_ERROR. */
 int libra_debug_error_word(libra_handle_t handle, uint32_t* word);
 
+/* KV migration, data movement (Section 5.3 of the paper: a paused request's KV cache is offloaded,
+ * resharded along the attention-head dimension to the target bucket's tensor-parallel degree - a source
+ * partition split into TP_tgt/TP_src shards, or TP_src/TP_tgt partitions concatenated - and reloaded).
+ * The reshard is folded into the copies: both calls take a head range.
+ *
+ * libra_kv_gather copies, for each of `batch` sequences, tokens [0, seq_lens[b]) of KV heads
+ * [head_begin, head_begin + head_count) from the handle's paged pools into dense buffers:
+ *     k_dense[((token_offsets[b] + t) * head_count + (h - head_begin)) * head_dim + c]
+ * libra_kv_scatter is the inverse: it writes the dense rows into the pages that `block_table` names, at
+ * heads [head_begin, head_begin + head_count) of the handle's pools (slots past seq_lens[b] are left
+ * untouched).  Splitting heads = several gathers with disjoint head ranges; concatenating = several
+ * scatters into one pool at different head offsets.
+ *
+ * block_table, seq_lens (int32) and token_offsets (int64[batch], in tokens) are device pointers;
+ * max_seq_len is an upper bound of the lengths (it sizes the grid; <= block_table_ld * 16); the dense
+ * buffers are 16-byte-aligned device memory or pinned host memory mapped into the device's address
+ * space; error_word_dev points to a 32-bit device word that receives LIBRA_ERR_BAD_PAGE_ID if a page
+ * id is outside the pool (that page is skipped).  The handle supplies the pool geometry only; no plan
+ * and no workspace are needed.  Asynchronous on `stream`.  Errors: INVALID_ARGUMENT, CUDA_ERROR. */
+int libra_kv_gather(libra_handle_t handle, const void* k_pages, const void* v_pages, const int32_t* block_table,
+                    const int32_t* seq_lens, const int64_t* token_offsets, int32_t batch, int32_t max_seq_len,
+                    int32_t head_begin, int32_t head_count, void* k_dense, void* v_dense, void* error_word_dev,
+                    void* stream);
+int libra_kv_scatter(libra_handle_t handle, const void* k_dense, const void* v_dense, const int32_t* block_table,
+                     const int32_t* seq_lens, const int64_t* token_offsets, int32_t batch, int32_t max_seq_len,
+                     int32_t head_begin, int32_t head_count, void* k_pages, void* v_pages, void* error_word_dev,
+                     void* stream);
+
 /* Self-test of the kernels' bounded waits: enqueues a one-warp kernel that waits, with a limit of a few
  * milliseconds, on a copy barrier that nothing completes.  It must return (no hang, no trap) and leave
  * LIBRA_ERR_WAIT_TIMEOUT in the device error word of the last planned workspace, which is how a real

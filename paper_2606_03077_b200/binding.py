@@ -72,6 +72,10 @@ SIGNATURES = {
     "libra_host_staging_size": (C.c_int, [_vp, C.c_int32, C.POINTER(C.c_size_t)]),
     "libra_last_cuda_error": (C.c_int, [_vp]),
     "libra_debug_error_word": (C.c_int, [_vp, C.POINTER(C.c_uint32)]),
+    "libra_kv_gather": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _vp, _vp,
+                                  _vp, _vp]),
+    "libra_kv_scatter": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _vp, _vp,
+                                   _vp, _vp]),
     "libra_debug_wait_selftest": (C.c_int, [_vp, _vp]),
     "libra_profile_begin": (C.c_int, [_vp]),
     "libra_profile_end": (C.c_int, [_vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int32)]),
@@ -229,6 +233,20 @@ class Handle:
         w = C.c_uint32(0)
         _check(lib.libra_debug_error_word(self._h, C.byref(w)), "libra_debug_error_word")
         return w.value
+
+    def kv_gather(self, k_ptr: int, v_ptr: int, block_table_ptr: int, seq_lens_ptr: int, token_offsets_ptr: int,
+                  batch: int, max_seq_len: int, head_begin: int, head_count: int, k_dense_ptr: int, v_dense_ptr: int,
+                  error_word_ptr: int, stream: int) -> None:
+        _check(lib.libra_kv_gather(self._h, k_ptr, v_ptr, block_table_ptr, seq_lens_ptr, token_offsets_ptr, batch,
+                                   max_seq_len, head_begin, head_count, k_dense_ptr, v_dense_ptr, error_word_ptr,
+                                   stream), "libra_kv_gather")
+
+    def kv_scatter(self, k_dense_ptr: int, v_dense_ptr: int, block_table_ptr: int, seq_lens_ptr: int,
+                   token_offsets_ptr: int, batch: int, max_seq_len: int, head_begin: int, head_count: int, k_ptr: int,
+                   v_ptr: int, error_word_ptr: int, stream: int) -> None:
+        _check(lib.libra_kv_scatter(self._h, k_dense_ptr, v_dense_ptr, block_table_ptr, seq_lens_ptr,
+                                    token_offsets_ptr, batch, max_seq_len, head_begin, head_count, k_ptr, v_ptr,
+                                    error_word_ptr, stream), "libra_kv_scatter")
 
     def debug_wait_selftest(self, stream: int) -> None:
         _check(lib.libra_debug_wait_selftest(self._h, stream), "libra_debug_wait_selftest")

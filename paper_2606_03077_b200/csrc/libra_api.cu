@@ -11,6 +11,7 @@
 #include <vector>
 
 #include "decode_kernel.cuh"
+#include "kv_move_kernel.cuh"
 #include "libra.h"
 #include "plan_kernel.cuh"
 #include "plan_layout.hpp"
@@ -886,6 +887,81 @@ int libra_debug_error_word(libra_handle_t h, uint32_t* word) {
   LIBRA_CUDA_TRY(h, cudaStreamSynchronize(st));
   if (*word) LIBRA_CUDA_TRY(h, cudaMemsetAsync(h->workspace, 0, 4, st));  // reading a set word clears it
   return LIBRA_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+int kv_move_impl(libra_handle_t h, bool gather, void* k_pages, void* v_pages, void* k_dense, void* v_dense,
+                 const int32_t* block_table, const int32_t* seq_lens, const int64_t* token_offsets, int32_t batch,
+                 int32_t max_seq_len, int32_t head_begin, int32_t head_count, void* error_word_dev, void* stream) {
+  if (!h || !k_pages || !v_pages || !k_dense || !v_dense || !block_table || !seq_lens || !token_offsets ||
+      !error_word_dev) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  if (batch < 0 || max_seq_len < 0 || head_begin < 0 || head_count <= 0 ||
+      head_begin + head_count > h->cfg.num_kv_heads) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  if (int64_t(max_seq_len) > int64_t(h->cfg.block_table_ld) * h->cfg.page_size) return LIBRA_INVALID_ARGUMENT;
+  if (reinterpret_cast<uintptr_t>(k_pages) % 16 || reinterpret_cast<uintptr_t>(v_pages) % 16 ||
+      reinterpret_cast<uintptr_t>(k_dense) % 16 || reinterpret_cast<uintptr_t>(v_dense) % 16 ||
+      reinterpret_cast<uintptr_t>(error_word_dev) % 4) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  if (batch == 0 || max_seq_len == 0) return LIBRA_OK;
+  DeviceGuard guard(h->cfg.device);
+  if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+  libra::KvMoveParams p;
+  p.k_pool = static_cast<__nv_bfloat16*>(k_pages);
+  p.v_pool = static_cast<__nv_bfloat16*>(v_pages);
+  p.k_dense = static_cast<__nv_bfloat16*>(k_dense);
+  p.v_dense = static_cast<__nv_bfloat16*>(v_dense);
+  p.block_table = block_table;
+  p.seq_lens = seq_lens;
+  p.token_offsets = token_offsets;
+  p.stride_page = h->stride_page;
+  p.stride_head = h->stride_head;
+  p.stride_token = h->stride_token;
+  p.num_pages = h->cfg.num_pages;
+  p.block_table_ld = h->cfg.block_table_ld;
+  p.head_begin = head_begin;
+  p.head_count = head_count;
+  p.error_word = static_cast<uint32_t*>(error_word_dev);
+  const int pages = (max_seq_len + h->cfg.page_size - 1) / h->cfg.page_size;
+  dim3 grid(unsigned((pages + libra::kMovePagesPerBlock - 1) / libra::kMovePagesPerBlock), unsigned(batch));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (h->cfg.head_dim == 128) {
+    if (gather) libra::kv_move_kernel<128, true><<<grid, libra::kMoveThreads, 0, st>>>(p);
+    else libra::kv_move_kernel<128, false><<<grid, libra::kMoveThreads, 0, st>>>(p);
+  } else {
+    if (gather) libra::kv_move_kernel<64, true><<<grid, libra::kMoveThreads, 0, st>>>(p);
+    else libra::kv_move_kernel<64, false><<<grid, libra::kMoveThreads, 0, st>>>(p);
+  }
+  LIBRA_CUDA_TRY(h, cudaGetLastError());
+  ++h->launches;
+  return LIBRA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int libra_kv_gather(libra_handle_t h, const void* k_pages, const void* v_pages, const int32_t* block_table,
+                    const int32_t* seq_lens, const int64_t* token_offsets, int32_t batch, int32_t max_seq_len,
+                    int32_t head_begin, int32_t head_count, void* k_dense, void* v_dense, void* error_word_dev,
+                    void* stream) {
+  return kv_move_impl(h, true, const_cast<void*>(k_pages), const_cast<void*>(v_pages), k_dense, v_dense, block_table,
+                      seq_lens, token_offsets, batch, max_seq_len, head_begin, head_count, error_word_dev, stream);
+}
+
+int libra_kv_scatter(libra_handle_t h, const void* k_dense, const void* v_dense, const int32_t* block_table,
+                     const int32_t* seq_lens, const int64_t* token_offsets, int32_t batch, int32_t max_seq_len,
+                     int32_t head_begin, int32_t head_count, void* k_pages, void* v_pages, void* error_word_dev,
+                     void* stream) {
+  return kv_move_impl(h, false, k_pages, v_pages, const_cast<void*>(k_dense), const_cast<void*>(v_dense), block_table,
+                      seq_lens, token_offsets, batch, max_seq_len, head_begin, head_count, error_word_dev, stream);
 }
 
 int libra_debug_wait_selftest(libra_handle_t h, void* stream) {
