@@ -297,6 +297,43 @@ def e2e_measure(rep: Replica, steps: int):
     return ms, int(h2d), int(d2h), bool(same)
 
 
+def e2e_resident_kv_measure(rep: Replica, steps: int):
+    """One decode step as a serving engine issues it: the KV cache stays in HBM; the step's own inputs (q,
+    block table, lengths) start in pinned host memory and the output ends there; every step is
+    synchronised (latency, not pipelined throughput)."""
+    torch = rep.torch
+    k, v = rep.pools[0]
+    hq = rep.q.cpu().pin_memory()
+    hbt = rep.bts[0].cpu().pin_memory()
+    hl = rep.lens_dev[0].cpu().pin_memory()
+    hout = torch.zeros(rep.out.shape, dtype=torch.bfloat16).pin_memory()
+    dq, dbt, dl = torch.empty_like(rep.q), torch.empty_like(rep.bts[0]), torch.empty_like(rep.lens_dev[0])
+    lens_host = rep.layouts[0].seq_lens
+    stream = torch.cuda.current_stream()
+    st = stream.cuda_stream
+
+    def one():
+        dq.copy_(hq, non_blocking=True)
+        dbt.copy_(hbt, non_blocking=True)
+        dl.copy_(hl, non_blocking=True)
+        rep.h.plan(lens_host, rep.ws.data_ptr(), rep.ws.numel(), st)
+        rep.h.decode_attn(dq.data_ptr(), k.data_ptr(), v.data_ptr(), dbt.data_ptr(), dl.data_ptr(), rep.out.data_ptr(), st)
+        hout.copy_(rep.out, non_blocking=True)
+        stream.synchronize()
+
+    for _ in range(5):
+        one()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one()
+    ms = (time.perf_counter() - t0) / steps * 1e3
+    return {"value": rep.layouts[0].kv_bytes / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms, "steps": steps,
+            "h2d_bytes_per_step": int(hq.numel() * 2 + hbt.numel() * 4 + hl.numel() * 4),
+            "d2h_bytes_per_step": int(hout.numel() * 2),
+            "note": "KV pools resident in HBM (as in any serving engine); q, block table and lengths copied from pinned "
+                    "host memory and the output copied back every step; host-synchronised per step, wall clock"}
+
+
 def kv_migration_measure(rep: Replica, reps: int = 10):
     """libra_kv_gather / libra_kv_scatter on the sequences of 16K tokens and more (the ones the paper's
     scheduler would move to a larger bucket): bytes moved = read + write of K and V."""
@@ -498,6 +535,7 @@ def run_libra(args):
                            "matches_resident_run": same,
                            "note": "libra_decode_attn_host: q, both KV pools, block table, lengths copied from pinned "
                                    "host memory every step, output copied back"}
+            line["e2e_resident_kv"] = e2e_resident_kv_measure(rep, 200)
         if not args.no_cpu:
             cb = oracle_baseline(args.workload, k0, v0, rep.q, budget_s=args.cpu_budget)
             line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}

@@ -320,6 +320,54 @@ int libra_kv_scatter(libra_handle_t handle, const void* k_dense, const void* v_d
                      int32_t head_begin, int32_t head_count, void* k_pages, void* v_pages, void* error_word_dev,
                      void* stream);
 
+/* ---- the paper's rollout-side schedulers, host code only (no GPU) ------------------------------------ */
+
+/* RolloutDP of the Global Resource Planner (Section 4.3, Algorithm 1): split `n_gpus` GPUs into inference
+ * instances with tensor-parallel degrees from `tp_set` and give each a contiguous segment of the requests
+ * sorted by length, minimising the largest instance time:
+ *     dp[g][i] = min over tp in tp_set, tp <= g, 0 <= x <= i of max(dp[g - tp][i - x], Cost(tp, i-x+1, i))
+ * with dp[0][0] = 0 and every GPU used ("exactly g GPUs").  Cost of an instance of degree tp_set[t] on a
+ * segment: cost_coef[4t+0] * sum(L) + cost_coef[4t+1] * sum(L^2) + cost_coef[4t+2] * count +
+ * cost_coef[4t+3], and 0 for an empty segment (the polynomial form of the paper's cost evaluator,
+ * Section 4.6, with caller-supplied coefficients).  `lengths` may be in any order (sorted inside).
+ * Outputs: *makespan (+inf if no partition uses exactly n_gpus GPUs) and the optimal partition recovered
+ * by backtracking, instances in sorted-request order: degree, index of the first request in the sorted
+ * list, number of requests.  Errors: INVALID_ARGUMENT, WORKSPACE_TOO_SMALL (inst_capacity too small;
+ * *n_instances holds the number needed). */
+int libra_rollout_dp(int32_t n_gpus, const int32_t* lengths, int32_t n_requests, const int32_t* tp_set, int32_t n_tp,
+                     const double* cost_coef, double* makespan, int32_t* inst_tp, int32_t* inst_first,
+                     int32_t* inst_count, int32_t inst_capacity, int32_t* n_instances);
+
+/* Causality-aware prefix tree (Section 5): a node is (prompt id, sequence of tool-return states); every
+ * node keeps a histogram of the remaining trajectory length seen from that point, with bins aligned to
+ * the buckets' length thresholds: bin k holds lengths <= bin_upper[k] (increasing), the last bin
+ * everything above; n_thresholds + 1 bins in all. */
+typedef struct libra_trie_s* libra_trie_t;
+int libra_trie_create(libra_trie_t* trie, const int32_t* bin_upper, int32_t n_thresholds);
+int libra_trie_destroy(libra_trie_t trie);
+
+/* Phase 3 / profile phase: insert one finished trajectory.  states[k] is the label of the k-th tool return
+ * (tool type x payload size class x success/failure, encoded by the caller); residual_lengths[0] is the
+ * trajectory's remaining length at the start and residual_lengths[k+1] the remaining length after the
+ * k-th tool return (n_states + 1 values).  Child nodes are created as needed. */
+int libra_trie_insert(libra_trie_t trie, int64_t prompt_id, const int32_t* states, int32_t n_states,
+                      const int32_t* residual_lengths);
+
+/* Phase 2 look-up: walk down from the prompt's root along `states`; at an unseen state stay at the parent
+ * (back-off).  hist[n_thresholds + 1] receives the node's empirical distribution (all zero for an unknown
+ * prompt), *depth_reached how many states were matched (-1: unknown prompt), *samples the node's count.
+ * depth_reached and samples may be NULL. */
+int libra_trie_lookup(libra_trie_t trie, int64_t prompt_id, const int32_t* states, int32_t n_states, double* hist,
+                      int32_t* depth_reached, int64_t* samples);
+
+/* Phase 2 routing: B* = argmin_B ( sum_k p_k * decode_cost[B][k] + migration_cost[B] ), p from the
+ * look-up above, decode_cost [n_buckets][n_thresholds + 1] row-major, migration_cost[B] the cost of
+ * moving from the current bucket to B (0 for the current one).  Ties go to the lower bucket index.
+ * best_cost may be NULL. */
+int libra_trie_route(libra_trie_t trie, int64_t prompt_id, const int32_t* states, int32_t n_states,
+                     int32_t n_buckets, const double* decode_cost, const double* migration_cost,
+                     int32_t* best_bucket, double* best_cost);
+
 /* Self-test of the kernels' bounded waits: enqueues a one-warp kernel that waits, with a limit of a few
  * milliseconds, on a copy barrier that nothing completes.  It must return (no hang, no trap) and leave
  * LIBRA_ERR_WAIT_TIMEOUT in the device error word of the last planned workspace, which is how a real

@@ -76,6 +76,15 @@ SIGNATURES = {
                                   _vp, _vp]),
     "libra_kv_scatter": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _vp, _vp,
                                    _vp, _vp]),
+    "libra_rollout_dp": (C.c_int, [C.c_int32, _i32p, C.c_int32, _i32p, C.c_int32, C.POINTER(C.c_double),
+                                   C.POINTER(C.c_double), _i32p, _i32p, _i32p, C.c_int32, _i32p]),
+    "libra_trie_create": (C.c_int, [C.POINTER(_vp), _i32p, C.c_int32]),
+    "libra_trie_destroy": (C.c_int, [_vp]),
+    "libra_trie_insert": (C.c_int, [_vp, C.c_int64, _i32p, C.c_int32, _i32p]),
+    "libra_trie_lookup": (C.c_int, [_vp, C.c_int64, _i32p, C.c_int32, C.POINTER(C.c_double), _i32p,
+                                    C.POINTER(C.c_int64)]),
+    "libra_trie_route": (C.c_int, [_vp, C.c_int64, _i32p, C.c_int32, C.c_int32, C.POINTER(C.c_double),
+                                   C.POINTER(C.c_double), _i32p, C.POINTER(C.c_double)]),
     "libra_debug_wait_selftest": (C.c_int, [_vp, _vp]),
     "libra_profile_begin": (C.c_int, [_vp]),
     "libra_profile_end": (C.c_int, [_vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int32)]),
@@ -131,6 +140,66 @@ def libra_plan_host(seq_lens, num_kv_heads: int, params: PlanParams, items_capac
             "item_offset": out["item_offset"][:B].copy(), "items": items[:n].copy(),
             "combine": out["combine"][:scal["num_combine"].value].copy(),
             "empty": out["empty"][:scal["num_empty"].value].copy()}
+
+
+def libra_rollout_dp(n_gpus: int, lengths, tp_set, cost_coef):
+    """RolloutDP: returns (makespan, [(tp, first_sorted_index, count), ...])."""
+    lens = _as_i32(lengths)
+    tps = _as_i32(tp_set)
+    coef = np.ascontiguousarray(cost_coef, dtype=np.float64).reshape(len(tps), 4)
+    cap = max(1, n_gpus)
+    itp, ifirst, icount = (np.zeros(cap, np.int32) for _ in range(3))
+    mk, n = C.c_double(0), C.c_int32(0)
+    p = lambda a: a.ctypes.data_as(_i32p)
+    st = lib.libra_rollout_dp(n_gpus, p(lens), len(lens), p(tps), len(tps), coef.ctypes.data_as(C.POINTER(C.c_double)),
+                              C.byref(mk), p(itp), p(ifirst), p(icount), cap, C.byref(n))
+    _check(st, "libra_rollout_dp")
+    return mk.value, [(int(itp[k]), int(ifirst[k]), int(icount[k])) for k in range(n.value)]
+
+
+class Trie:
+    """Owns one libra_trie_t (the causality-aware prefix tree)."""
+
+    def __init__(self, bin_upper):
+        self.bins = _as_i32(bin_upper)
+        self._t = _vp()
+        _check(lib.libra_trie_create(C.byref(self._t), self.bins.ctypes.data_as(_i32p), len(self.bins)), "libra_trie_create")
+
+    def close(self):
+        if self._t:
+            lib.libra_trie_destroy(self._t)
+            self._t = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def insert(self, prompt_id: int, states, residual_lengths) -> None:
+        s, r = _as_i32(states), _as_i32(residual_lengths)
+        assert len(r) == len(s) + 1
+        _check(lib.libra_trie_insert(self._t, prompt_id, s.ctypes.data_as(_i32p), len(s), r.ctypes.data_as(_i32p)),
+               "libra_trie_insert")
+
+    def lookup(self, prompt_id: int, states):
+        s = _as_i32(states)
+        hist = np.zeros(len(self.bins) + 1, np.float64)
+        depth, n = C.c_int32(0), C.c_int64(0)
+        _check(lib.libra_trie_lookup(self._t, prompt_id, s.ctypes.data_as(_i32p), len(s),
+                                     hist.ctypes.data_as(C.POINTER(C.c_double)), C.byref(depth), C.byref(n)),
+               "libra_trie_lookup")
+        return hist, depth.value, n.value
+
+    def route(self, prompt_id: int, states, decode_cost, migration_cost):
+        s = _as_i32(states)
+        dc = np.ascontiguousarray(decode_cost, dtype=np.float64)
+        mc = np.ascontiguousarray(migration_cost, dtype=np.float64)
+        best, cost = C.c_int32(0), C.c_double(0)
+        _check(lib.libra_trie_route(self._t, prompt_id, s.ctypes.data_as(_i32p), len(s), len(mc),
+                                    dc.ctypes.data_as(C.POINTER(C.c_double)), mc.ctypes.data_as(C.POINTER(C.c_double)),
+                                    C.byref(best), C.byref(cost)), "libra_trie_route")
+        return best.value, cost.value
 
 
 class Handle:
