@@ -37,7 +37,7 @@
  *                 three strides are 0), "NHD" = [num_pages, page_size, num_kv_heads, head_dim].
  *                 Pool base addresses must be 16-byte aligned and strides multiples of 8 elements.
  *   block_table   int32 [batch, block_table_ld]; entry i of row b = page id of tokens
- *                 [16 i, 16 i + 16) of sequence b; entries past the last page are ignored
+ *                 [P i, P i + P) of sequence b (P = page_size); entries past the last page are ignored
  *   seq_lens      int32 [batch]; number of cached tokens INCLUDING the current one; the kernel
  *                 appends nothing; 0 is allowed (output row = 0)
  *   GQA map       query head h reads KV head h / (num_q_heads / num_kv_heads)
@@ -57,7 +57,7 @@ extern "C" {
 typedef enum {
   LIBRA_OK = 0,
   LIBRA_INVALID_ARGUMENT = 1,   /* null pointer, negative size, batch > max_batch ...            */
-  LIBRA_UNSUPPORTED_SHAPE = 2,  /* head_dim not 64/128, page_size not 16, group size > 16 ...    */
+  LIBRA_UNSUPPORTED_SHAPE = 2,  /* head_dim not 64/128, page_size not 16/32/64, group size > 16  */
   LIBRA_WORKSPACE_TOO_SMALL = 3,
   LIBRA_NOT_PLANNED = 4,        /* libra_decode_attn before a successful libra_plan              */
   LIBRA_CUDA_ERROR = 5,         /* a CUDA call failed; see libra_last_cuda_error                 */
@@ -87,7 +87,7 @@ typedef struct {
   int32_t num_q_heads;
   int32_t num_kv_heads;        /* must divide num_q_heads; group size <= 16                      */
   int32_t head_dim;            /* 64 or 128                                                      */
-  int32_t page_size;           /* 16                                                             */
+  int32_t page_size;           /* 16, 32 or 64 tokens per page                                   */
   int64_t num_pages;           /* pages in each pool                                             */
   int32_t max_batch;           /* upper bound of `batch` in libra_plan                           */
   int32_t block_table_ld;      /* row pitch of block_table in entries                            */
@@ -196,7 +196,7 @@ int libra_plan(libra_handle_t handle, const int32_t* seq_lens_host, int32_t batc
  * Section 2.2, Section 4.3).  The plan is written into the workspace; later libra_decode_attn calls
  * launch grids sized for the worst case and the kernels read the real counts from the workspace.
  * Limits: batch <= 4096 (UNSUPPORTED_SHAPE otherwise); at most 4096 work items and no length beyond
- * block_table_ld * 16, else the plan is empty and LIBRA_ERR_PLAN_OVERFLOW is set in the device error
+ * block_table_ld * page_size, else the plan is empty and LIBRA_ERR_PLAN_OVERFLOW is set in the device error
  * word (checked on the device, since the host does not see the lengths).  The result equals
  * libra_plan's bit for bit (libra_plan_export reads it back).
  * Errors: INVALID_ARGUMENT, WORKSPACE_TOO_SMALL, UNSUPPORTED_SHAPE, CUDA_ERROR. */
@@ -226,7 +226,7 @@ int libra_decode_attn(libra_handle_t handle, const void* q, const void* k_pages,
  * the rollout, Section 1 / Section 2.2 of the paper: the cache grows by one token per step).  k_new and
  * v_new are device pointers to the current token's key and value rows, bf16 [batch, num_kv_heads,
  * head_dim], 16-byte aligned; seq_lens still COUNTS that token.  For every sequence with L_b >= 1 the
- * rows are written into slot (L_b - 1) % 16 of page block_table[b][(L_b - 1) / 16] of both pools (the
+ * rows are written into slot (L_b - 1) % P of page block_table[b][(L_b - 1) / P] of both pools (the
  * pools are therefore not const) and the attention result is exactly what libra_decode_attn returns on
  * the updated pools.  The block that owns the sequence's last page does both: it patches the staged copy
  * of that page in shared memory and stores the rows to the pools, so no ordering between the store and
@@ -306,7 +306,7 @@ int libra_debug_error_word(libra_handle_t handle, uint32_t* word);
  * scatters into one pool at different head offsets.
  *
  * block_table, seq_lens (int32) and token_offsets (int64[batch], in tokens) are device pointers;
- * max_seq_len is an upper bound of the lengths (it sizes the grid; <= block_table_ld * 16); the dense
+ * max_seq_len is an upper bound of the lengths (it sizes the grid; <= block_table_ld * page_size); the dense
  * buffers are 16-byte-aligned device memory or pinned host memory mapped into the device's address
  * space; error_word_dev points to a 32-bit device word that receives LIBRA_ERR_BAD_PAGE_ID if a page
  * id is outside the pool (that page is skipped).  The handle supplies the pool geometry only; no plan

@@ -15,9 +15,10 @@ import numpy as np
 def gather(pages: np.ndarray, block_table: np.ndarray, seq_lens, head_begin: int, head_count: int) -> np.ndarray:
     """Dense shard [total_tokens, head_count, d]: sequences one after the other, tokens in order."""
     rows = []
+    P = pages.shape[2]
     for b, L in enumerate(seq_lens):
         for t in range(int(L)):
-            rows.append(pages[block_table[b, t // 16], head_begin:head_begin + head_count, t % 16, :])
+            rows.append(pages[block_table[b, t // P], head_begin:head_begin + head_count, t % P, :])
     if not rows:
         return np.zeros((0, head_count, pages.shape[3]), dtype=pages.dtype)
     return np.stack(rows)
@@ -26,10 +27,11 @@ def gather(pages: np.ndarray, block_table: np.ndarray, seq_lens, head_begin: int
 def scatter(dense: np.ndarray, pages: np.ndarray, block_table: np.ndarray, seq_lens, head_begin: int) -> None:
     """Inverse of gather, in place: dense rows go to the pages `block_table` names, at head offset head_begin."""
     n = dense.shape[1]
+    P = pages.shape[2]
     row = 0
     for b, L in enumerate(seq_lens):
         for t in range(int(L)):
-            pages[block_table[b, t // 16], head_begin:head_begin + n, t % 16, :] = dense[row]
+            pages[block_table[b, t // P], head_begin:head_begin + n, t % P, :] = dense[row]
             row += 1
 
 

@@ -1,8 +1,9 @@
 // Split-KV decode kernel (step D) for sm_100a.
 //
 // A work unit is one work item of the plan (a chunk [kv_begin, kv_end) of one sequence) for one KV
-// head and all G query heads that share it.  Inside a thread block every warp owns a private ring
-// of shared-memory stages and takes the unit's pages warp, warp+NW, warp+2NW, ...:
+// head and all G query heads that share it.  The kernel works in tiles of 16 tokens: a page of 16, 32
+// or 64 tokens is 1, 2 or 4 tiles ("page" below means such a tile).  Inside a thread block every warp
+// owns a private ring of shared-memory stages and takes the unit's tiles warp, warp+NW, warp+2NW, ...:
 //
 //   lane 0 : page id -> two tiled TMA loads per tensor (K and V page, 128-byte swizzle) that
 //            complete on the stage's mbarrier; up to STAGES pages per warp are in flight
@@ -49,8 +50,10 @@ struct DecodeParams {
   int32_t group;          // G
   int32_t block_table_ld;
   float scale_log2;       // sm_scale * log2(e)
-  int32_t pos_head;       // coordinate slot (1..3) of the head / page dimension in the tensor maps
+  int32_t pos_head;       // coordinate slot (1..3) of the head / page / token dimension in the tensor maps
   int32_t pos_page;
+  int32_t pos_token;
+  int32_t tile_shift;     // log2(page_size / 16): a page holds 1, 2 or 4 tiles of 16 tokens
   int32_t num_items;
   int32_t num_units;      // work items x KV heads
   int32_t num_empty;      // empty sequences whose output row this launch zeroes
@@ -477,10 +480,11 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   const int n_it = u.n_it;
 
   // ---- page ids first (the copies wait for them): lane L keeps the id of iteration 32*round + L, one round ahead
-  const int32_t* bt_row = p.block_table + int64_t(u.b) * p.block_table_ld + u.first_page + warp;
+  const int32_t* bt_row = p.block_table + int64_t(u.b) * p.block_table_ld;
+  const int first_tile = u.first_page + warp;   // tile index within the sequence of this warp's iteration 0
   auto load_ids = [&](int round) -> int32_t {
     const int idx = round * 32 + lane;
-    return (idx < n_it) ? __ldg(bt_row + int64_t(idx) * NW) : -1;
+    return (idx < n_it) ? __ldg(bt_row + ((first_tile + idx * NW) >> p.tile_shift)) : -1;
   };
   int32_t ids_cur = load_ids(0);
   int32_t ids_nxt = load_ids(1);
@@ -500,9 +504,10 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
       const uint32_t bar = my_bar0 + 8 * s;
       const uint32_t kdst = my_ring_u32 + s * SM::kStageBytes;
       const uint32_t vdst = kdst + SM::kTileBytes;
-      const int c1 = (p.pos_head == 1) ? kvh : ((p.pos_page == 1) ? pid : 0);
-      const int c2 = (p.pos_head == 2) ? kvh : ((p.pos_page == 2) ? pid : 0);
-      const int c3 = (p.pos_head == 3) ? kvh : ((p.pos_page == 3) ? pid : 0);
+      const int tok = ((first_tile + j * NW) & ((1 << p.tile_shift) - 1)) << 4;   // first token of the tile in its page
+      const int c1 = (p.pos_head == 1) ? kvh : ((p.pos_page == 1) ? pid : tok);
+      const int c2 = (p.pos_head == 2) ? kvh : ((p.pos_page == 2) ? pid : tok);
+      const int c3 = (p.pos_head == 3) ? kvh : ((p.pos_page == 3) ? pid : tok);
       fence_proxy_async();  // earlier generic-proxy accesses to this stage come before the async write
       mbar_expect_tx(bar, SM::kStageBytes);
 #pragma unroll
@@ -539,14 +544,16 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
       const int which = lane / (D / 8);   // 0: K, 1: V
       const int c16 = lane % (D / 8);
       if (which < 2) {
-        const int64_t page = __ldg(p.block_table + int64_t(u.b) * p.block_table_ld + ((u.kv_end - 1) >> 4));
+        const int last = u.kv_end - 1;                       // the newest token
+        const int64_t page = __ldg(p.block_table + int64_t(u.b) * p.block_table_ld + (last >> (4 + p.tile_shift)));
+        const int slot = last & ((16 << p.tile_shift) - 1);  // its slot in that page
         const __nv_bfloat16* src = (which ? p.v_new : p.k_new) + (int64_t(u.b) * p.num_kv_heads + kvh) * D + c16 * 8;
         const uint4 row = __ldg(reinterpret_cast<const uint4*>(src));
         uint8_t* tile = my_ring + s * SM::kStageBytes + which * SM::kTileBytes;
         *reinterpret_cast<uint4*>(tile + tile_off(r, c16)) = row;
         if (page >= 0 && page < p.num_pages) {
           __nv_bfloat16* dst = (which ? p.v_pool : p.k_pool) + page * p.stride_page + int64_t(kvh) * p.stride_head +
-                               int64_t(r) * p.stride_token + c16 * 8;
+                               int64_t(slot) * p.stride_token + c16 * 8;
           *reinterpret_cast<uint4*>(dst) = row;
         }
       }

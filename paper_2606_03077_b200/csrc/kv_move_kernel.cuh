@@ -34,6 +34,7 @@ struct KvMoveParams {
   int64_t num_pages;
   int32_t block_table_ld;
   int32_t head_begin, head_count;
+  int32_t page_size;            // tokens per page (16, 32 or 64)
   uint32_t* error_word;
 };
 
@@ -41,19 +42,20 @@ constexpr int kMovePagesPerBlock = 4;
 constexpr int kMoveThreads = 256;
 
 // grid = (ceil(max pages per sequence / kMovePagesPerBlock), batch); block = kMoveThreads.
-// One 16-byte vector per thread per step; a (page, head) tile is 16 tokens x D elements.
+// One 16-byte vector per thread per step; a (page, head) tile is page_size tokens x D elements.
 template <int D, bool kGather>
 __global__ void __launch_bounds__(kMoveThreads) kv_move_kernel(const KvMoveParams p) {
   constexpr int VEC = 8;                    // bf16 per 16-byte vector
   constexpr int VPR = D / VEC;              // vectors per token row of one head
   const int b = blockIdx.y;
   const int len = __ldg(p.seq_lens + b);
-  const int n_pages = (len + 15) >> 4;
+  const int P = p.page_size;
+  const int n_pages = (len + P - 1) / P;
   const int page0 = blockIdx.x * kMovePagesPerBlock;
   if (page0 >= n_pages) return;
   const int page1 = min(n_pages, page0 + kMovePagesPerBlock);
   const int64_t row0 = __ldg(p.token_offsets + b);
-  const int vec_per_page = 16 * p.head_count * VPR;   // token-major inside the page: (token, head, vec)
+  const int vec_per_page = P * p.head_count * VPR;    // token-major inside the page: (token, head, vec)
 
   for (int pg = page0; pg < page1; ++pg) {
     const int64_t pid = __ldg(p.block_table + int64_t(b) * p.block_table_ld + pg);
@@ -61,7 +63,7 @@ __global__ void __launch_bounds__(kMoveThreads) kv_move_kernel(const KvMoveParam
       if (threadIdx.x == 0) atomicOr(p.error_word, LIBRA_DEV_ERR_BAD_PAGE_ID);
       continue;
     }
-    const int valid = min(16, len - pg * 16);
+    const int valid = min(P, len - pg * P);
     for (int i = threadIdx.x; i < vec_per_page; i += kMoveThreads) {
       const int vec = i % VPR;
       const int head = (i / VPR) % p.head_count;
@@ -69,7 +71,7 @@ __global__ void __launch_bounds__(kMoveThreads) kv_move_kernel(const KvMoveParam
       if (tok >= valid) continue;
       const int64_t pool_off = pid * p.stride_page + int64_t(p.head_begin + head) * p.stride_head +
                                int64_t(tok) * p.stride_token + vec * VEC;
-      const int64_t dense_off = ((row0 + int64_t(pg) * 16 + tok) * p.head_count + head) * D + vec * VEC;
+      const int64_t dense_off = ((row0 + int64_t(pg) * P + tok) * p.head_count + head) * D + vec * VEC;
       if (kGather) {
         *reinterpret_cast<uint4*>(p.k_dense + dense_off) = __ldg(reinterpret_cast<const uint4*>(p.k_pool + pool_off));
         *reinterpret_cast<uint4*>(p.v_dense + dense_off) = __ldg(reinterpret_cast<const uint4*>(p.v_pool + pool_off));

@@ -132,7 +132,7 @@ struct libra_handle_s {
   static constexpr int kMapCache = 8;
   PoolMaps maps[kMapCache];
   int next_map = 0;
-  int pos_head = 0, pos_page = 0;
+  int pos_head = 0, pos_page = 0, pos_token = 0;
 
   // profiling
   bool profiling = false;
@@ -168,14 +168,15 @@ libra::PlanParams resolve_params(const libra_plan_params_t& in, int n_sm_device)
 }
 
 // Build the tiled tensor map of one pool: dimension 0 is head_dim (contiguous); the other three
-// (token, head, page) are ordered by increasing stride.  Box = 64 elements x 16 tokens x 1 x 1.
-int encode_pool_map(libra_handle_t h, const void* base, CUtensorMap* map, int* pos_head, int* pos_page) {
+// (token, head, page) are ordered by increasing stride.  Box = 64 elements x 16 tokens x 1 x 1 (a page of
+// 32 or 64 tokens is read as 2 or 4 such boxes at token offsets 0, 16, ...).
+int encode_pool_map(libra_handle_t h, const void* base, CUtensorMap* map, int* pos_head, int* pos_page, int* pos_token) {
   struct Dim {
     int64_t stride, size;
     uint32_t box;
     int kind;
   };
-  Dim dims[3] = {{h->stride_token, h->cfg.page_size, uint32_t(h->cfg.page_size), 0},
+  Dim dims[3] = {{h->stride_token, h->cfg.page_size, 16u, 0},
                  {h->stride_head, h->cfg.num_kv_heads, 1u, 1},
                  {h->stride_page, h->cfg.num_pages, 1u, 2}};
   std::stable_sort(dims, dims + 3, [](const Dim& a, const Dim& b) { return a.stride < b.stride; });
@@ -187,6 +188,7 @@ int encode_pool_map(libra_handle_t h, const void* base, CUtensorMap* map, int* p
     gdim[i + 1] = cuuint64_t(dims[i].size);
     gstride[i] = cuuint64_t(dims[i].stride) * 2;
     box[i + 1] = dims[i].box;
+    if (dims[i].kind == 0) *pos_token = i + 1;
     if (dims[i].kind == 1) *pos_head = i + 1;
     if (dims[i].kind == 2) *pos_page = i + 1;
   }
@@ -293,7 +295,8 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
   if (cfg->num_q_heads % cfg->num_kv_heads != 0) return LIBRA_INVALID_ARGUMENT;
   if (!(cfg->sm_scale >= 0.f) || !std::isfinite(cfg->sm_scale)) return LIBRA_INVALID_ARGUMENT;
   const int group = cfg->num_q_heads / cfg->num_kv_heads;
-  if (group > 16 || (cfg->head_dim != 64 && cfg->head_dim != 128) || cfg->page_size != 16) return LIBRA_UNSUPPORTED_SHAPE;
+  if (group > 16 || (cfg->head_dim != 64 && cfg->head_dim != 128)) return LIBRA_UNSUPPORTED_SHAPE;
+  if (cfg->page_size != 16 && cfg->page_size != 32 && cfg->page_size != 64) return LIBRA_UNSUPPORTED_SHAPE;
   if (cfg->num_pages > (int64_t(1) << 31) - 1) return LIBRA_UNSUPPORTED_SHAPE;  // page ids are int32
   if (cfg->max_batch > libra::plan_layout::kMaxBatch) return LIBRA_UNSUPPORTED_SHAPE;
 
@@ -344,7 +347,10 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
       break;
     }
     h->params = resolve_params(pin, n_sm);
-    if (!libra::valid_params(h->params)) { status = LIBRA_INVALID_ARGUMENT; break; }
+    if (!libra::valid_params(h->params) || h->params.chunk_align % cfg->page_size != 0) {
+      status = LIBRA_INVALID_ARGUMENT;  // chunks must start on page boundaries
+      break;
+    }
 
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -663,8 +669,8 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     pm = &h->maps[h->next_map];
     h->next_map = (h->next_map + 1) % libra_handle_s::kMapCache;
     pm->k_ptr = pm->v_ptr = nullptr;
-    int rc = encode_pool_map(h, k_pages, &pm->map_k, &h->pos_head, &h->pos_page);
-    if (rc == LIBRA_OK) rc = encode_pool_map(h, v_pages, &pm->map_v, &h->pos_head, &h->pos_page);
+    int rc = encode_pool_map(h, k_pages, &pm->map_k, &h->pos_head, &h->pos_page, &h->pos_token);
+    if (rc == LIBRA_OK) rc = encode_pool_map(h, v_pages, &pm->map_v, &h->pos_head, &h->pos_page, &h->pos_token);
     if (rc != LIBRA_OK) return rc;
     pm->k_ptr = k_pages;
     pm->v_ptr = v_pages;
@@ -717,6 +723,8 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     p.scale_log2 = h->scale_log2;
     p.pos_head = h->pos_head;
     p.pos_page = h->pos_page;
+    p.pos_token = h->pos_token;
+    p.tile_shift = (h->cfg.page_size == 16) ? 0 : (h->cfg.page_size == 32 ? 1 : 2);
     p.num_items = h->num_items;
     p.num_units = n_units;
     p.num_empty = n_empty;
@@ -928,6 +936,7 @@ int kv_move_impl(libra_handle_t h, bool gather, void* k_pages, void* v_pages, vo
   p.block_table_ld = h->cfg.block_table_ld;
   p.head_begin = head_begin;
   p.head_count = head_count;
+  p.page_size = h->cfg.page_size;
   p.error_word = static_cast<uint32_t*>(error_word_dev);
   const int pages = (max_seq_len + h->cfg.page_size - 1) / h->cfg.page_size;
   dim3 grid(unsigned((pages + libra::kMovePagesPerBlock - 1) / libra::kMovePagesPerBlock), unsigned(batch));

@@ -24,15 +24,15 @@ class Runner:
     """One handle + workspace for one shape; run() executes plan + decode on the current stream."""
 
     def __init__(self, binding, Hq, Hkv, d, num_pages, max_batch, ld, layout="HND", plan=None, sm_scale=0.0,
-                 variant=None, fused=None):
+                 variant=None, fused=None, page_size=16):
         import torch
         self.torch = torch
         self.dev = torch.device("cuda:0")
         strides = (0, 0, 0)
         if layout == "NHD":
-            strides = (16 * Hkv * d, d, Hkv * d)
-        self.h = binding.Handle(Hq, Hkv, d, num_pages, max_batch, ld, kv_strides=strides, sm_scale=sm_scale,
-                                plan=plan)
+            strides = (page_size * Hkv * d, d, Hkv * d)
+        self.h = binding.Handle(Hq, Hkv, d, num_pages, max_batch, ld, page_size=page_size, kv_strides=strides,
+                                sm_scale=sm_scale, plan=plan)
         if variant is not None:
             self.h.set_variant(*variant)
         if fused is not None:
@@ -58,6 +58,7 @@ class Runner:
 
 
 def run_host_case(binding, q, k, v, bt, lens, layout="HND", plan=None, sm_scale=0.0, variant=None, fused=None):
+    page_size = k.shape[2]
     """Host uint16 inputs (HND order; transposed here for NHD) -> float32 output [B, Hq, d]."""
     import torch
     dev = torch.device("cuda:0")
@@ -66,7 +67,7 @@ def run_host_case(binding, q, k, v, bt, lens, layout="HND", plan=None, sm_scale=
     if layout == "NHD":
         k = np.ascontiguousarray(k.transpose(0, 2, 1, 3))
         v = np.ascontiguousarray(v.transpose(0, 2, 1, 3))
-    r = Runner(binding, Hq, Hkv, d, k.shape[0], max(B, 1), bt.shape[1], layout, plan, sm_scale, variant, fused)
+    r = Runner(binding, Hq, Hkv, d, k.shape[0], max(B, 1), bt.shape[1], layout, plan, sm_scale, variant, fused, page_size)
     out = r.run(to_dev(q, dev), to_dev(k, dev), to_dev(v, dev), to_dev(bt, dev), lens)
     res = bf16_dev_to_f32(out)
     r.h.close()

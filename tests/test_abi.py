@@ -37,7 +37,7 @@ def test_create_rejects_bad_shapes_before_touching_cuda(lib):
         (dict(num_q_heads=30, num_kv_heads=8, head_dim=128), lib.INVALID_ARGUMENT),
         (dict(num_q_heads=32, num_kv_heads=8, head_dim=96), lib.UNSUPPORTED_SHAPE),
         (dict(num_q_heads=32, num_kv_heads=1, head_dim=128), lib.UNSUPPORTED_SHAPE),   # group 32 > 16
-        (dict(num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=32), lib.UNSUPPORTED_SHAPE),
+        (dict(num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=48), lib.UNSUPPORTED_SHAPE),
         (dict(num_q_heads=32, num_kv_heads=8, head_dim=128, kv_strides=(16384, 2048, 100)), lib.INVALID_ARGUMENT),
         (dict(num_q_heads=32, num_kv_heads=8, head_dim=128, sm_scale=-1.0), lib.INVALID_ARGUMENT),
         (dict(num_q_heads=0, num_kv_heads=8, head_dim=128), lib.INVALID_ARGUMENT),

@@ -16,42 +16,45 @@ pytestmark = pytest.mark.gpu
 
 def reference_append(k, v, bt, lens, k_new, v_new):
     k2, v2 = k.copy(), v.copy()
+    P = k.shape[2]
     for b, L in enumerate(lens):
         L = int(L)
         if L == 0:
             continue
-        page, slot = bt[b, (L - 1) // 16], (L - 1) % 16
+        page, slot = bt[b, (L - 1) // P], (L - 1) % P
         k2[page, :, slot, :] = k_new[b]
         v2[page, :, slot, :] = v_new[b]
     return k2, v2
 
 
 @pytest.mark.parametrize("layout", ["HND", "NHD"])
-@pytest.mark.parametrize("Hq,Hkv,d,lens", [
-    (8, 2, 128, [1, 16, 17, 32, 33, 700]),
-    (32, 8, 128, [5000, 1300, 0, 2049]),
-    (4, 1, 64, [300, 64, 7, 1]),
-    (40, 8, 128, [48, 1025]),
+@pytest.mark.parametrize("Hq,Hkv,d,lens,P", [
+    (8, 2, 128, [1, 16, 17, 32, 33, 700], 16),
+    (32, 8, 128, [5000, 1300, 0, 2049], 16),
+    (4, 1, 64, [300, 64, 7, 1], 16),
+    (40, 8, 128, [48, 1025], 16),
+    (8, 2, 128, [1, 17, 32, 33, 64, 65, 700], 64),
+    (8, 2, 128, [31, 32, 33, 1000], 32),
 ])
-def test_append_matches_definition(lib, Hq, Hkv, d, lens, layout):
+def test_append_matches_definition(lib, Hq, Hkv, d, lens, P, layout):
     import torch
     dev = torch.device("cuda:0")
     B = len(lens)
-    lens_a, bt, q, k, v = W.random_case(77, B, Hq, Hkv, d, lens)   # the new token's slot holds poison, as any unowned slot
+    lens_a, bt, q, k, v = W.random_case(77, B, Hq, Hkv, d, lens, page_size=P)   # the new token's slot holds poison
     for b, L in enumerate(lens):                                   # make sure of it even though the slot is "owned"
         if L:
-            k[bt[b, (L - 1) // 16], :, (L - 1) % 16, :] = W.f32_to_bf16_bits(np.array([W.POISON_F32]))[0]
-            v[bt[b, (L - 1) // 16], :, (L - 1) % 16, :] = W.f32_to_bf16_bits(np.array([-W.POISON_F32]))[0]
+            k[bt[b, (L - 1) // P], :, (L - 1) % P, :] = W.f32_to_bf16_bits(np.array([W.POISON_F32]))[0]
+            v[bt[b, (L - 1) // P], :, (L - 1) % P, :] = W.f32_to_bf16_bits(np.array([-W.POISON_F32]))[0]
     rng = np.random.default_rng(5)
     k_new = W.f32_to_bf16_bits(rng.standard_normal((B, Hkv, d), dtype=np.float32))
     v_new = W.f32_to_bf16_bits(rng.standard_normal((B, Hkv, d), dtype=np.float32))
     k_ref, v_ref = reference_append(k, v, bt, lens_a, k_new, v_new)
     ref, _ = O.paged_decode_attention(q, k_ref, v_ref, bt, lens_a)
 
-    for plan in (None, lib.PlanParams(4, 1, 2, 16, 16, 64)):
+    for plan in (None, lib.PlanParams(4, 1, 2, 64, 64, 64)):
         kd = k if layout == "HND" else np.ascontiguousarray(k.transpose(0, 2, 1, 3))
         vd = v if layout == "HND" else np.ascontiguousarray(v.transpose(0, 2, 1, 3))
-        r = H.Runner(lib, Hq, Hkv, d, k.shape[0], B, bt.shape[1], layout, plan)
+        r = H.Runner(lib, Hq, Hkv, d, k.shape[0], B, bt.shape[1], layout, plan, page_size=P)
         dq, dk, dv, dbt, dkn, dvn = (H.to_dev(x, dev) for x in (q, kd, vd, bt, k_new, v_new))
         dl = torch.from_numpy(lens_a.copy()).to(dev)
         out = torch.full((B, Hq, d), H.CANARY, dtype=torch.int16, device=dev)

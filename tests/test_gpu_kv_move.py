@@ -18,20 +18,21 @@ def dev_i64(a, dev):
 
 
 @pytest.mark.parametrize("layout", ["HND", "NHD"])
-@pytest.mark.parametrize("Hkv,d,lens,h0,hn", [
-    (8, 128, [1, 16, 17, 700, 0, 2049], 0, 8),
-    (8, 128, [333, 64], 2, 4),
-    (4, 64, [40, 5, 1000], 3, 1),
+@pytest.mark.parametrize("Hkv,d,lens,h0,hn,P", [
+    (8, 128, [1, 16, 17, 700, 0, 2049], 0, 8, 16),
+    (8, 128, [333, 64], 2, 4, 16),
+    (4, 64, [40, 5, 1000], 3, 1, 16),
+    (4, 128, [1, 33, 64, 65, 700], 1, 2, 64),
 ])
-def test_gather_and_scatter_are_exact(lib, Hkv, d, lens, h0, hn, layout):
+def test_gather_and_scatter_are_exact(lib, Hkv, d, lens, h0, hn, P, layout):
     import torch
     dev = torch.device("cuda:0")
     B = len(lens)
-    lens_a, bt, q, k, v = W.random_case(91, B, Hkv, Hkv, d, lens, poison=False)
+    lens_a, bt, q, k, v = W.random_case(91, B, Hkv, Hkv, d, lens, poison=False, page_size=P)
     kd = k if layout == "HND" else np.ascontiguousarray(k.transpose(0, 2, 1, 3))
     vd = v if layout == "HND" else np.ascontiguousarray(v.transpose(0, 2, 1, 3))
-    strides = (0, 0, 0) if layout == "HND" else (16 * Hkv * d, d, Hkv * d)
-    h = lib.Handle(Hkv, Hkv, d, k.shape[0], B, bt.shape[1], kv_strides=strides)
+    strides = (0, 0, 0) if layout == "HND" else (P * Hkv * d, d, Hkv * d)
+    h = lib.Handle(Hkv, Hkv, d, k.shape[0], B, bt.shape[1], page_size=P, kv_strides=strides)
     offs = np.concatenate([[0], np.cumsum(lens_a.astype(np.int64))])
     total = int(offs[-1])
     dk, dv, dbt = (H.to_dev(x, dev) for x in (kd, vd, bt))
@@ -50,10 +51,10 @@ def test_gather_and_scatter_are_exact(lib, Hkv, d, lens, h0, hn, layout):
 
     # scatter the shard into a fresh pool under a new placement, at head offset 0 of a pool with hn heads
     rng = np.random.default_rng(4)
-    bt2, pool2 = W.draw_block_table(lens_a, int(W.pages_needed(lens_a).sum()) + 5, rng, ld=bt.shape[1])
-    strides2 = (0, 0, 0) if layout == "HND" else (16 * hn * d, d, hn * d)
-    h2 = lib.Handle(hn, hn, d, pool2, B, bt.shape[1], kv_strides=strides2)
-    shape2 = (pool2, hn, 16, d) if layout == "HND" else (pool2, 16, hn, d)
+    bt2, pool2 = W.draw_block_table(lens_a, int(W.pages_needed(lens_a, P).sum()) + 5, rng, page_size=P, ld=bt.shape[1])
+    strides2 = (0, 0, 0) if layout == "HND" else (P * hn * d, d, hn * d)
+    h2 = lib.Handle(hn, hn, d, pool2, B, bt.shape[1], page_size=P, kv_strides=strides2)
+    shape2 = (pool2, hn, P, d) if layout == "HND" else (pool2, P, hn, d)
     k2 = torch.full(shape2, -1, dtype=torch.int16, device=dev)
     v2 = torch.full(shape2, -1, dtype=torch.int16, device=dev)
     dbt2 = H.to_dev(bt2, dev)
@@ -61,8 +62,8 @@ def test_gather_and_scatter_are_exact(lib, Hkv, d, lens, h0, hn, layout):
                   B, int(lens_a.max()), 0, hn, k2.data_ptr(), v2.data_ptr(), err.data_ptr(), st)
     torch.cuda.synchronize()
     assert int(err.item()) == 0
-    want_k = np.full((pool2, hn, 16, d), 0xFFFF, np.uint16)
-    want_v = np.full((pool2, hn, 16, d), 0xFFFF, np.uint16)
+    want_k = np.full((pool2, hn, P, d), 0xFFFF, np.uint16)
+    want_v = np.full((pool2, hn, P, d), 0xFFFF, np.uint16)
     M.scatter(M.gather(k, bt, lens_a, h0, hn), want_k, bt2, lens_a, 0)
     M.scatter(M.gather(v, bt, lens_a, h0, hn), want_v, bt2, lens_a, 0)
     got_k = k2.cpu().numpy().view(np.uint16)

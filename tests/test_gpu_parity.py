@@ -69,6 +69,20 @@ def test_shapes_and_tails(lib, case, layout):
     assert np.array_equal(two, got) and np.array_equal(one, got)
 
 
+@pytest.mark.parametrize("layout", ["HND", "NHD"])
+@pytest.mark.parametrize("page_size", [32, 64])
+def test_larger_pages(lib, page_size, layout):
+    # a page of 32 or 64 tokens is read as 2 or 4 tiles of 16; lengths around page and tile boundaries
+    lens = [1, 16, 17, page_size - 1, page_size, page_size + 1, 700, 2049, 0]
+    lens_a, bt, q, k, v = W.random_case(60 + page_size, len(lens), 8, 2, 128, lens, page_size=page_size)
+    ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
+    for plan in (None, lib.PlanParams(4, 1, 2, 64, 64, 64)):
+        got = H.run_host_case(lib, q, k, v, bt, lens_a, layout=layout, plan=plan)
+        check(got, ref, f"page {page_size} {layout}")
+    with pytest.raises(lib.LibraError):     # chunks must start on page boundaries
+        lib.Handle(8, 2, 128, 64, 4, 8, page_size=page_size, plan=lib.PlanParams(4, 1, 2, 16, 16, 64))
+
+
 def test_every_block_shape_agrees(lib):
     lens = [2500, 300, 17, 4100]
     lens_a, bt, q, k, v = W.random_case(7, 4, 32, 8, 128, lens)
