@@ -536,6 +536,8 @@ def run_libra(args):
                            "note": "libra_decode_attn_host: q, both KV pools, block table, lengths copied from pinned "
                                    "host memory every step, output copied back"}
             line["e2e_resident_kv"] = e2e_resident_kv_measure(rep, 200)
+        if args.workload in ("longtail_mix_b256", "straggler_b8"):
+            line["kv_migration"] = kv_migration_measure(rep)
         if not args.no_cpu:
             cb = oracle_baseline(args.workload, k0, v0, rep.q, budget_s=args.cpu_budget)
             line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
@@ -569,7 +571,7 @@ def run_libra(args):
                             "frac_of_nominal_8TBs": r.kv_bytes_per_step / (per * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
                             "frac_of_measured_copy": r.kv_bytes_per_step / (per * 1e-3) / 1e9 / peak,
                             "kv_bytes_per_step": r.kv_bytes_per_step, "pool_copies": len(r.pools)}
-            if name == "longtail_mix_b256":  # migrating the long tail: gather its KV to a dense buffer and scatter it back
+            if name in ("longtail_mix_b256", "straggler_b8"):  # migrating the long sequences: gather to a dense buffer, scatter back
                 others[name]["kv_migration"] = kv_migration_measure(r)
             if name == "shift_b128":  # the re-planned-every-step workload: also with the device-side planner
                 eager = r.timed_device_plan(n, 6, graph=False)

@@ -112,6 +112,11 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// Pull a tensor map (a kernel parameter) into the descriptor cache ahead of its first use.
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
@@ -448,6 +453,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   const uint32_t my_bar0 = smem_u32(&bars[warp * STAGES]);
 
   if (lane == 0) {
+    prefetch_tensormap(&map_k);
+    prefetch_tensormap(&map_v);
 #pragma unroll
     for (int s = 0; s < STAGES; ++s) mbar_init(my_bar0 + 8 * s, 1);
     fence_mbar_init();
