@@ -248,6 +248,37 @@ class Replica:
         assert self.h.debug_error_word() == 0, "device error word set"
         return e0.elapsed_time(e1), self.h.launch_count() - n0
 
+    def step_gather_read(self, stream: int) -> None:
+        """The step with the attention math removed: same plan, page walk and copies (a read ceiling)."""
+        s = self.i % len(self.layouts)
+        k, v = self.pools[self.i % len(self.pools)]
+        self.i += 1
+        self.h.plan(self.layouts[s].seq_lens, self.ws.data_ptr(), self.ws.numel(), stream)
+        self.h.debug_gather_read(self.q.data_ptr(), k.data_ptr(), v.data_ptr(), self.bts[s].data_ptr(),
+                                 self.lens_dev[s].data_ptr(), self.scratch_out().data_ptr(), stream)
+
+    def scratch_out(self):
+        if not hasattr(self, "_scratch_out"):
+            self._scratch_out = self.torch.zeros_like(self.out)
+        return self._scratch_out
+
+    def repeats(self, fn, reps: int, calls_each: int):
+        """(median, best) ms per call over `reps` event-timed batches of `calls_each` back-to-back calls."""
+        torch = self.torch
+        st = torch.cuda.current_stream().cuda_stream
+        times = []
+        for r in range(reps + 3):  # three untimed batches first
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(calls_each):
+                fn(st)
+            e1.record()
+            torch.cuda.synchronize()
+            if r >= 3:
+                times.append(e0.elapsed_time(e1) / calls_each)
+        return float(np.median(times)), float(min(times))
+
     def kernel_times(self, steps: int):
         """Same steps with CUDA events around each kernel (recorded by the library on its stream)."""
         torch = self.torch
@@ -262,6 +293,33 @@ class Replica:
 
     def close(self):
         self.h.close()
+
+
+def ceilings_measure(rep: Replica, reps: int = 20):
+    """What the step's read rate is set against: the step itself, the same step with the attention math removed
+    (same plan, page walk and tiled copies), and a plain streaming read of a contiguous 4 GiB buffer; each as
+    (median, best) over `reps` batches."""
+    torch = rep.torch
+    ms_guess = rep.kv_bytes_per_step / 6.4e12 * 1e3   # batches of ~1.5 ms, whole cycles of a multi-step workload
+    per_batch = len(rep.layouts) * max(1, int(round(1.5 / (ms_guess * len(rep.layouts)))))
+    step_med, step_best = rep.repeats(rep.step, reps, per_batch)
+    gat_med, gat_best = rep.repeats(rep.step_gather_read, reps, per_batch)
+    assert rep.h.debug_error_word() == 0, "device error word set"
+    nbytes = 4 << 30
+    buf = torch.zeros(nbytes, dtype=torch.uint8, device=rep.dev)
+    rd_med, rd_best = rep.repeats(lambda st: rep.h.debug_stream_read(buf.data_ptr(), nbytes, st), reps, 2)
+    del buf
+    gbs = lambda b, ms: b / (ms * 1e-3) / 1e9
+    kv = rep.kv_bytes_per_step
+    return {"reps": reps, "calls_per_rep": per_batch,
+            "step_us_median": step_med * 1e3, "step_us_best": step_best * 1e3,
+            "step_gbs_median": gbs(kv, step_med), "step_gbs_best": gbs(kv, step_best),
+            "page_gather_read_gbs_median": gbs(kv, gat_med), "page_gather_read_gbs_best": gbs(kv, gat_best),
+            "contiguous_read_gbs_median": gbs(nbytes, rd_med), "contiguous_read_gbs_best": gbs(nbytes, rd_best),
+            "step_frac_of_page_gather_read": gat_med / step_med,
+            "step_frac_of_contiguous_read": gbs(kv, step_med) / gbs(nbytes, rd_med),
+            "note": "page_gather_read = libra_debug_gather_read (the decode kernel's plan, grid, block-table walk and "
+                    "tiled copies, no math); contiguous_read = libra_debug_stream_read over 4 GiB"}
 
 
 def e2e_measure(rep: Replica, steps: int):
@@ -536,6 +594,7 @@ def run_libra(args):
                            "note": "libra_decode_attn_host: q, both KV pools, block table, lengths copied from pinned "
                                    "host memory every step, output copied back"}
             line["e2e_resident_kv"] = e2e_resident_kv_measure(rep, 200)
+        line["ceilings"] = ceilings_measure(rep)
         if args.workload in ("longtail_mix_b256", "straggler_b8"):
             line["kv_migration"] = kv_migration_measure(rep)
         if not args.no_cpu:
@@ -571,6 +630,7 @@ def run_libra(args):
                             "frac_of_nominal_8TBs": r.kv_bytes_per_step / (per * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
                             "frac_of_measured_copy": r.kv_bytes_per_step / (per * 1e-3) / 1e9 / peak,
                             "kv_bytes_per_step": r.kv_bytes_per_step, "pool_copies": len(r.pools)}
+            others[name]["ceilings"] = ceilings_measure(r, reps=10)
             if name in ("longtail_mix_b256", "straggler_b8"):  # migrating the long sequences: gather to a dense buffer, scatter back
                 others[name]["kv_migration"] = kv_migration_measure(r)
             if name == "shift_b128":  # the re-planned-every-step workload: also with the device-side planner

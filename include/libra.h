@@ -374,6 +374,20 @@ int libra_trie_route(libra_trie_t trie, int64_t prompt_id, const int32_t* states
  * timeout inside the decode kernel would surface.  Errors: NOT_PLANNED, CUDA_ERROR. */
 int libra_debug_wait_selftest(libra_handle_t handle, void* stream);
 
+/* Two read ceilings to set the decode kernel's rate against (the step is bound by one pass over K and V,
+ * Section 2.1); both only read, neither computes attention.
+ * libra_debug_stream_read: one kernel that streams `bytes` (>= 16; the tail past a multiple of 16 is not
+ *   read) of the contiguous device buffer `buf_dev` (16-byte aligned) with plain vector loads.
+ * libra_debug_gather_read: the decode kernel's measurement build - same arguments, plan, grid, block-table
+ *   walk and tiled page copies as libra_decode_attn with the default block shape, but a staged page is only
+ *   touched, not computed on.  `out` and the partial buffers receive meaningless values; the device error
+ *   word is updated as usual.
+ * Both are asynchronous on `stream` and need a plan (the stream read only for its workspace).
+ * Errors: INVALID_ARGUMENT, NOT_PLANNED, CUDA_ERROR. */
+int libra_debug_stream_read(libra_handle_t handle, const void* buf_dev, size_t bytes, void* stream);
+int libra_debug_gather_read(libra_handle_t handle, const void* q, const void* k_pages, const void* v_pages,
+                            const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream);
+
 /* Per-kernel timing for benchmarks.  After libra_profile_begin, every libra_decode_attn records
  * CUDA events around the decode kernel and the combine kernel on the call's stream (at most
  * 4096 calls are kept).  libra_profile_end synchronises those events, returns the summed device

@@ -58,6 +58,8 @@ SIGNATURES = {
     "libra_get_plan_params": (C.c_int, [_vp, C.POINTER(PlanParams)]),
     "libra_set_variant": (C.c_int, [_vp, C.c_int32, C.c_int32]),
     "libra_set_dependent_launch": (C.c_int, [_vp, C.c_int32]),
+    "libra_debug_stream_read": (C.c_int, [_vp, _vp, C.c_size_t, _vp]),
+    "libra_debug_gather_read": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_set_combine_mode": (C.c_int, [_vp, C.c_int32]),
     "libra_plan_host": (C.c_int, [C.POINTER(PlanParams), C.c_int32, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p,
                                   _i32p, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p]),
@@ -268,6 +270,14 @@ class Handle:
                     out_ptr: int, stream: int) -> None:
         _check(lib.libra_decode_attn(self._h, q_ptr, k_ptr, v_ptr, block_table_ptr, seq_lens_ptr, out_ptr, stream),
                "libra_decode_attn")
+
+    def debug_stream_read(self, buf_ptr: int, nbytes: int, stream: int) -> None:
+        _check(lib.libra_debug_stream_read(self._h, buf_ptr, nbytes, stream), "libra_debug_stream_read")
+
+    def debug_gather_read(self, q_ptr: int, k_ptr: int, v_ptr: int, block_table_ptr: int, seq_lens_ptr: int,
+                          out_ptr: int, stream: int) -> None:
+        _check(lib.libra_debug_gather_read(self._h, q_ptr, k_ptr, v_ptr, block_table_ptr, seq_lens_ptr, out_ptr, stream),
+               "libra_debug_gather_read")
 
     def decode_attn_append(self, q_ptr: int, k_new_ptr: int, v_new_ptr: int, k_ptr: int, v_ptr: int,
                            block_table_ptr: int, seq_lens_ptr: int, out_ptr: int, stream: int) -> None:

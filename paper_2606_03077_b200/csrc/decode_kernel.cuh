@@ -429,7 +429,9 @@ struct DecodeSmem {
 // ------------------------------------------------------------------------------------------------
 // One thread block per unit.
 // D: head_dim (64 | 128); NT: 8-wide head tiles (1: G <= 8, 2: G <= 16); NW warps; STAGES per warp.
-template <int D, int NT, int NW, int STAGES>
+// kLoadsOnly: measurement build of the same kernel - same plan, page walk and copies, but each staged page
+// is only touched (one shared-memory word per lane) instead of computed on; `out` gets meaningless values.
+template <int D, int NT, int NW, int STAGES, bool kLoadsOnly = false>
 __global__ void __launch_bounds__(NW * 32)
 decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
               const __grid_constant__ DecodeParams p, const __grid_constant__ ParamPlan pp) {
@@ -544,6 +546,11 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     }
     const uint32_t kt = my_ring_u32 + s * SM::kStageBytes;
     const int tok0 = u.kv_begin + ((warp + it * NW) << 4);
+    if constexpr (kLoadsOnly) {
+      const uint32_t* words = reinterpret_cast<const uint32_t*>(my_ring + s * SM::kStageBytes);
+      st.l[0][0] += float((words[lane * 16] ^ words[SM::kTileBytes / 4 + lane * 16]) & 0xffu);
+      st.m[0][0] = 0.f;
+    } else {
     if (p.k_new != nullptr && u.chunk_j == u.n_chunks - 1 && u.kv_end - tok0 <= 16) {
       // this page holds the sequence's newest token: its K and V rows come from k_new / v_new.  The copy
       // that just landed predates them, so patch the staged tiles (swizzled row) and write the pools.
@@ -569,6 +576,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     }
     process_page<D, NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes, u.kv_end - tok0,
                         p.scale_log2, lane);
+    }
     __syncwarp();  // every lane has consumed the stage before lane 0 refills it
     if (it + STAGES < n_it) issue(it + STAGES, s);
     if (++s == STAGES) {

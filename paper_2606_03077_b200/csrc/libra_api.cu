@@ -16,6 +16,7 @@
 #include "plan_kernel.cuh"
 #include "plan_layout.hpp"
 #include "planner.hpp"
+#include "read_kernel.cuh"
 
 static_assert(LIBRA_ERR_WAIT_TIMEOUT == LIBRA_DEV_ERR_WAIT_TIMEOUT, "error bits");
 static_assert(LIBRA_ERR_BAD_PAGE_ID == LIBRA_DEV_ERR_BAD_PAGE_ID, "error bits");
@@ -61,6 +62,13 @@ const std::vector<Variant>& variants() {
   };
   return v;
 }
+
+// Measurement build of the default block shape (copies only, no math); [D == 128]
+constexpr int kLoadsOnlyWarps = 8, kLoadsOnlyStages = 3;
+const DecodeKernelFn kLoadsOnlyFn[2] = {libra::decode_kernel<64, 1, kLoadsOnlyWarps, kLoadsOnlyStages, true>,
+                                        libra::decode_kernel<128, 1, kLoadsOnlyWarps, kLoadsOnlyStages, true>};
+const int kLoadsOnlySmem[2] = {libra::DecodeSmem<64, kLoadsOnlyWarps, kLoadsOnlyStages>::kDynamicBytes,
+                               libra::DecodeSmem<128, kLoadsOnlyWarps, kLoadsOnlyStages>::kDynamicBytes};
 
 constexpr int kMaxProfiledCalls = 4096;
 
@@ -372,6 +380,12 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
       }
     }
     if (status != LIBRA_OK) break;
+    for (int di = 0; di < 2; ++di) {
+      e = cudaFuncSetAttribute(reinterpret_cast<const void*>(kLoadsOnlyFn[di]), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               kLoadsOnlySmem[di]);
+      if (e != cudaSuccess) break;
+    }
+    if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
     e = cudaFuncSetAttribute(reinterpret_cast<const void*>(libra::plan_kernel), cudaFuncAttributeMaxDynamicSharedMemorySize,
                              int(libra::plan_kernel_smem_bytes()));
     if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
@@ -648,7 +662,8 @@ namespace {
 
 // Steps D and C; k_new / v_new non-null = append the current token's K and V rows on the way.
 int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* v_new, const void* k_pages,
-                const void* v_pages, const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream) {
+                const void* v_pages, const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream,
+                bool loads_only = false) {
   if (!h || !q || !k_pages || !v_pages || !block_table || !seq_lens || !out) return LIBRA_INVALID_ARGUMENT;
   if ((k_new == nullptr) != (v_new == nullptr)) return LIBRA_INVALID_ARGUMENT;
   if (reinterpret_cast<uintptr_t>(k_new) % 16 || reinterpret_cast<uintptr_t>(v_new) % 16) return LIBRA_INVALID_ARGUMENT;
@@ -696,7 +711,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
   const Variant& v = variants()[h->variant];
   const int di = (h->cfg.head_dim == 128) ? 1 : 0;
   const int ni = (h->group > 8) ? 1 : 0;
-  const bool fused = h->combine_mode == 1;
+  const bool fused = h->combine_mode == 1 || loads_only;
   // host plan: exact counts; device plan: upper bounds for the grids, the kernels read the counts themselves
   const int32_t n_empty = h->device_planned ? h->planned_batch : int32_t(h->plan.empty.size());
   const int32_t n_combine = h->device_planned ? h->planned_batch : int32_t(h->plan.combine.size());
@@ -741,15 +756,15 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     // resident while that kernel drains; inside, they wait for it to finish before reading any input
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(grid);
-    lc.blockDim = dim3(unsigned(v.warps * 32));
-    lc.dynamicSmemBytes = size_t(v.smem[di][ni]);
+    lc.blockDim = dim3(unsigned((loads_only ? kLoadsOnlyWarps : v.warps) * 32));
+    lc.dynamicSmemBytes = size_t(loads_only ? kLoadsOnlySmem[di] : v.smem[di][ni]);
     lc.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = h->pdl ? 1 : 0;
-    LIBRA_CUDA_TRY(h, cudaLaunchKernelEx(&lc, v.fn[di][ni], pm->map_k, pm->map_v, p, h->pp));
+    LIBRA_CUDA_TRY(h, cudaLaunchKernelEx(&lc, loads_only ? kLoadsOnlyFn[di] : v.fn[di][ni], pm->map_k, pm->map_v, p, h->pp));
     ++h->launches;
   }
   if (ev) LIBRA_CUDA_TRY(h, cudaEventRecord(ev[1], st));
@@ -981,6 +996,25 @@ int libra_debug_wait_selftest(libra_handle_t h, void* stream) {
   libra::wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(
       reinterpret_cast<uint32_t*>(h->workspace), 1024u);
   LIBRA_CUDA_TRY(h, cudaGetLastError());
+  h->last_stream = stream;
+  return LIBRA_OK;
+}
+
+int libra_debug_gather_read(libra_handle_t h, const void* q, const void* k_pages, const void* v_pages,
+                            const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream) {
+  return decode_impl(h, q, nullptr, nullptr, k_pages, v_pages, block_table, seq_lens, out, stream, true);
+}
+
+int libra_debug_stream_read(libra_handle_t h, const void* buf_dev, size_t bytes, void* stream) {
+  if (!h || !buf_dev || bytes < 16 || reinterpret_cast<uintptr_t>(buf_dev) % 16 != 0) return LIBRA_INVALID_ARGUMENT;
+  if (!h->planned) return LIBRA_NOT_PLANNED;
+  DeviceGuard guard(h->cfg.device);
+  if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+  uint32_t* sink = reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(h->workspace) + 128);  // an unused control word
+  libra::stream_read_kernel<<<unsigned(h->params.n_sm * libra::kReadBlocksPerSm), libra::kReadThreads, 0,
+                              static_cast<cudaStream_t>(stream)>>>(static_cast<const uint4*>(buf_dev), bytes / 16, sink);
+  LIBRA_CUDA_TRY(h, cudaGetLastError());
+  ++h->launches;
   h->last_stream = stream;
   return LIBRA_OK;
 }
