@@ -30,7 +30,10 @@ that row; zero query gives the mean of V (closed-form rational with integer V); 
 dominant one-hot key returns exactly its value row; page placement does not matter;
 shifting every key by u shifts every score by q.u*scale and nothing else; a dense,
 loop-only brute force agrees on tiny inputs; chunked evaluation plus merge equals the
-direct formula; an analytic two-token case.
+direct formula; an analytic two-token case.  The several-query-token form is pinned by
+its reduction to the single-token function row by row, by the loop-only brute force, by
+one-hot keys planted on either side of each query token's causal limit, and by the
+zero-query running mean in closed form.
 """
 from __future__ import annotations
 
@@ -99,6 +102,49 @@ def paged_decode_attention(q, k_pages, v_pages, block_table, seq_lens, layout: s
         z = e.sum(axis=2, keepdims=True)
         out[b] = np.matmul(e / z, V).reshape(Hq, d)
         lse[b] = (m + np.log(z)).reshape(Hq)
+    return out, lse
+
+
+def paged_multi_token_attention(q, k_pages, v_pages, block_table, seq_lens, layout: str = "HND",
+                                sm_scale: float | None = None):
+    """Several query tokens per sequence: the last Tq tokens of every sequence are new in this step
+    (a tool return or a few drafted tokens appended at once; Section 2.2 describes how tool returns
+    extend a trajectory mid-rollout).  Their K and V rows are already in the cache and seq_lens
+    counts them.  Query token i (i = 0 .. Tq-1) sits at position L - Tq + i and, being causal,
+    attends to cached tokens 0 .. L - Tq + i:
+
+        n_i = L - Tq + 1 + i
+        out[b, i, h] = sum_{t < n_i} softmax(s_0 .. s_{n_i - 1})_t * V_b[t],   s_t = (q[b, i, h] . K_b[t]) * sm_scale
+
+    A query token with n_i <= 0 (a sequence shorter than Tq) has out = 0, lse = -inf.
+    q: uint16[B, Tq, Hq, d].  Returns (out float64[B, Tq, Hq, d], lse float64[B, Tq, Hq]).
+    Tq = 1 is the single-token definition above.
+    """
+    q = np.asarray(q)
+    B, Tq, Hq, d = q.shape
+    Hkv = k_pages.shape[1] if layout == "HND" else k_pages.shape[2]
+    assert Hq % Hkv == 0
+    G = Hq // Hkv
+    scale = 1.0 / math.sqrt(d) if sm_scale is None else float(sm_scale)
+    out = np.zeros((B, Tq, Hq, d), dtype=np.float64)
+    lse = np.full((B, Tq, Hq), -np.inf, dtype=np.float64)
+    for b in range(B):
+        L = int(seq_lens[b])
+        if L == 0:
+            continue
+        K = gather_sequence(k_pages, block_table[b], L, layout)      # [Hkv, L, d]
+        V = gather_sequence(v_pages, block_table[b], L, layout)
+        for i in range(Tq):
+            n = L - Tq + 1 + i
+            if n <= 0:
+                continue
+            qi = bf16_bits_to_f64(q[b, i]).reshape(Hkv, G, d)
+            s = np.matmul(qi, K[:, :n].transpose(0, 2, 1)) * scale   # [Hkv, G, n]
+            m = s.max(axis=2, keepdims=True)
+            e = np.exp(s - m)
+            z = e.sum(axis=2, keepdims=True)
+            out[b, i] = np.matmul(e / z, V[:, :n]).reshape(Hq, d)
+            lse[b, i] = (m + np.log(z)).reshape(Hq)
     return out, lse
 
 
