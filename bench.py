@@ -322,6 +322,45 @@ def ceilings_measure(rep: Replica, reps: int = 20):
                     "tiled copies, no math); contiguous_read = libra_debug_stream_read over 4 GiB"}
 
 
+def multi_token_measure(rep: Replica, q_len: int, steps: int = 200):
+    """The step with q_len query tokens per sequence (libra_decode_attn_multi) on the same pools, block tables
+    and lengths: one pass over K and V serves all q_len tokens."""
+    torch, w = rep.torch, rep.w
+    if q_len * (w.num_q_heads // w.num_kv_heads) > 16:
+        return None
+    h = rep.binding.Handle(w.num_q_heads, w.num_kv_heads, w.head_dim, rep.layouts[0].pool_pages, w.batch, rep.ld,
+                           device=rep.dev.index or 0)
+    h.set_max_query_tokens(q_len)
+    ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=rep.dev)
+    gen = torch.Generator(device=rep.dev).manual_seed(7)
+    q = torch.randn((w.batch, q_len, w.num_q_heads, w.head_dim), generator=gen, device=rep.dev).to(torch.bfloat16)
+    out = torch.zeros_like(q)
+    st = torch.cuda.current_stream().cuda_stream
+
+    def step(i):
+        s = i % len(rep.layouts)
+        k, v = rep.pools[i % len(rep.pools)]
+        h.plan(rep.layouts[s].seq_lens, ws.data_ptr(), ws.numel(), st)
+        h.decode_attn_multi(q.data_ptr(), q_len, k.data_ptr(), v.data_ptr(), rep.bts[s].data_ptr(),
+                            rep.lens_dev[s].data_ptr(), out.data_ptr(), st)
+
+    steps = max(len(rep.layouts), steps // len(rep.layouts) * len(rep.layouts))
+    for i in range(10):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    assert h.debug_error_word() == 0, "device error word set"
+    h.close()
+    ms = e0.elapsed_time(e1) / steps
+    return {"q_len": q_len, "ms_per_step": ms, "kv_gbs": rep.kv_bytes_per_step / (ms * 1e-3) / 1e9,
+            "query_tokens_per_s": w.batch * q_len / (ms * 1e-3), "steps": steps}
+
+
 def e2e_measure(rep: Replica, steps: int):
     """The step through libra_decode_attn_host with every input in pinned host memory."""
     torch = rep.torch
@@ -595,6 +634,7 @@ def run_libra(args):
                                    "host memory every step, output copied back"}
             line["e2e_resident_kv"] = e2e_resident_kv_measure(rep, 200)
         line["ceilings"] = ceilings_measure(rep)
+        line["multi_token"] = [m for m in (multi_token_measure(rep, t) for t in (2, 4)) if m]
         if args.workload in ("longtail_mix_b256", "straggler_b8"):
             line["kv_migration"] = kv_migration_measure(rep)
         if not args.no_cpu:
@@ -631,6 +671,7 @@ def run_libra(args):
                             "frac_of_measured_copy": r.kv_bytes_per_step / (per * 1e-3) / 1e9 / peak,
                             "kv_bytes_per_step": r.kv_bytes_per_step, "pool_copies": len(r.pools)}
             others[name]["ceilings"] = ceilings_measure(r, reps=10)
+            others[name]["multi_token"] = [m for m in (multi_token_measure(r, t, 60) for t in (2, 3, 4)) if m]
             if name in ("longtail_mix_b256", "straggler_b8"):  # migrating the long sequences: gather to a dense buffer, scatter back
                 others[name]["kv_migration"] = kv_migration_measure(r)
             if name == "shift_b128":  # the re-planned-every-step workload: also with the device-side planner

@@ -142,6 +142,12 @@ int libra_workspace_size(libra_handle_t handle, size_t* bytes);
 /* The planner constants the handle uses, defaults resolved (n_sm = the device's SM count). */
 int libra_get_plan_params(libra_handle_t handle, libra_plan_params_t* out);
 
+/* Several query tokens per sequence (default 1).  Lays the workspace out for up to `max_q_len` query tokens
+ * per sequence in libra_decode_attn_multi: the partial buffers grow by that factor, so ask
+ * libra_workspace_size again afterwards; the current plan is dropped.  A KV head's score tile has at most
+ * 16 columns: max_q_len * (num_q_heads / num_kv_heads) <= 16, else UNSUPPORTED_SHAPE. */
+int libra_set_max_query_tokens(libra_handle_t handle, int32_t max_q_len);
+
 /* Tuning knob: shape of the decode thread block: `warps` warps that each own `stages` shared-memory
  * stages of one K page plus one V page.  Only the compiled-in shapes are accepted (UNSUPPORTED_SHAPE
  * otherwise); the default is the tuned one.  Results do not depend on the stage count; the warp
@@ -221,6 +227,19 @@ int libra_plan_export(libra_handle_t handle, libra_plan_view_t* view);
  * Errors: INVALID_ARGUMENT (null or misaligned pointer), NOT_PLANNED, CUDA_ERROR. */
 int libra_decode_attn(libra_handle_t handle, const void* q, const void* k_pages, const void* v_pages,
                       const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream);
+
+/* The step for several query tokens per sequence: the last q_len tokens of every sequence are new in this
+ * step (a tool return absorbed at once - Section 2.2: tool returns extend a trajectory mid-rollout - or a few
+ * drafted tokens); their K and V rows are already in the cache and seq_lens counts them.  q and out are bf16
+ * [batch, q_len, num_q_heads, head_dim].  Query token i attends causally to cached tokens
+ * 0 .. L_b - q_len + i:  out[b, i, h] = softmax over those tokens of (q[b, i, h] . K_b[t]) * sm_scale, times V.
+ * A query token with nothing to attend to (L_b - q_len + i < 0) gets a zero row.  The plan is the one
+ * libra_plan made from seq_lens (it depends on the lengths only); all query tokens of a KV head's group share
+ * one pass over K and V.  1 <= q_len <= the value given to libra_set_max_query_tokens; q_len = 1 is
+ * libra_decode_attn.  Errors: as libra_decode_attn, INVALID_ARGUMENT for q_len out of range. */
+int libra_decode_attn_multi(libra_handle_t handle, const void* q, int32_t q_len, const void* k_pages,
+                            const void* v_pages, const int32_t* block_table, const int32_t* seq_lens, void* out,
+                            void* stream);
 
 /* The same step with the KV append fused in (the step before attention inside one decode step of
  * the rollout, Section 1 / Section 2.2 of the paper: the cache grows by one token per step).  k_new and

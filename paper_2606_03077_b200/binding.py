@@ -58,6 +58,8 @@ SIGNATURES = {
     "libra_get_plan_params": (C.c_int, [_vp, C.POINTER(PlanParams)]),
     "libra_set_variant": (C.c_int, [_vp, C.c_int32, C.c_int32]),
     "libra_set_dependent_launch": (C.c_int, [_vp, C.c_int32]),
+    "libra_set_max_query_tokens": (C.c_int, [_vp, C.c_int32]),
+    "libra_decode_attn_multi": (C.c_int, [_vp, _vp, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_debug_stream_read": (C.c_int, [_vp, _vp, C.c_size_t, _vp]),
     "libra_debug_gather_read": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_set_combine_mode": (C.c_int, [_vp, C.c_int32]),
@@ -278,6 +280,14 @@ class Handle:
                           out_ptr: int, stream: int) -> None:
         _check(lib.libra_debug_gather_read(self._h, q_ptr, k_ptr, v_ptr, block_table_ptr, seq_lens_ptr, out_ptr, stream),
                "libra_debug_gather_read")
+
+    def set_max_query_tokens(self, max_q_len: int) -> None:
+        _check(lib.libra_set_max_query_tokens(self._h, max_q_len), "libra_set_max_query_tokens")
+
+    def decode_attn_multi(self, q_ptr: int, q_len: int, k_ptr: int, v_ptr: int, block_table_ptr: int,
+                          seq_lens_ptr: int, out_ptr: int, stream: int) -> None:
+        _check(lib.libra_decode_attn_multi(self._h, q_ptr, q_len, k_ptr, v_ptr, block_table_ptr, seq_lens_ptr,
+                                           out_ptr, stream), "libra_decode_attn_multi")
 
     def decode_attn_append(self, q_ptr: int, k_new_ptr: int, v_new_ptr: int, k_ptr: int, v_ptr: int,
                            block_table_ptr: int, seq_lens_ptr: int, out_ptr: int, stream: int) -> None:

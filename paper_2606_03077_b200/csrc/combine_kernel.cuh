@@ -42,6 +42,7 @@ __device__ __forceinline__ void combine_row(const float* partial_o, const float*
   float m = fmaxf(l0, l1);
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+  if (m == -INFINITY) m = 0.f;  // no partial holds anything (a query token that sees no cached token): all weights 0
   const float w0 = (lane < n) ? __expf(l0 - m) : 0.f;
   const float w1 = (lane + 32 < n) ? __expf(l1 - m) : 0.f;
 
@@ -77,7 +78,7 @@ __device__ __forceinline__ void combine_row(const float* partial_o, const float*
       for (int v = 0; v < V; ++v) num[v] += w * o[k][v];
     }
   }
-  const float inv = (n > 0) ? 1.f / den : 0.f;
+  const float inv = (den > 0.f) ? 1.f / den : 0.f;
   __nv_bfloat16* dst = out + (int64_t(b) * Hq + h) * D + lane * V;
 #pragma unroll
   for (int v = 0; v < V; v += 2) {

@@ -45,9 +45,12 @@ struct DecodeParams {
   uint32_t* error_word;
   int32_t* counters;      // [batch][Hkv] arrival counters of split sequences (zero between launches)
   int64_t num_pages;
-  int32_t num_q_heads;
+  int32_t num_q_heads;    // rows of q / out per sequence: query tokens x query heads
   int32_t num_kv_heads;
   int32_t group;          // G
+  int32_t q_len;          // Tq: query tokens per sequence (the last Tq tokens of the cache are theirs); usually 1
+  int32_t hq;             // query heads of the model (num_q_heads = q_len * hq)
+  int32_t cols;           // q_len * G: rows of q that share one KV head = columns of a unit's score tile
   int32_t block_table_ld;
   float scale_log2;       // sm_scale * log2(e)
   int32_t pos_head;       // coordinate slot (1..3) of the head / page / token dimension in the tensor maps
@@ -179,7 +182,14 @@ __device__ __forceinline__ Unit decode_unit(const int4 item, int kvh, int warp) 
   return u;
 }
 
-// Q^T fragments (B operand: k = dims, n = heads); rows of heads >= G are zero.
+// Column c of a unit (KV head kvh) is query token c / G, head kvh * G + c % G of that token; q and out are
+// [B, q_len, hq, d], so the row within a sequence is:
+__device__ __forceinline__ int col_row(const DecodeParams& p, int kvh, int c) {
+  const int i = c / p.group;
+  return i * p.hq + kvh * p.group + (c - i * p.group);
+}
+
+// Q^T fragments (B operand: k = dims, n = columns); columns >= cols are zero.
 template <int D, int NT>
 __device__ __forceinline__ void load_q_frags(uint32_t (&qf)[NT][D / 16][2], const DecodeParams& p, int b, int kvh,
                                              int lane) {
@@ -187,9 +197,9 @@ __device__ __forceinline__ void load_q_frags(uint32_t (&qf)[NT][D / 16][2], cons
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
     const int head = nt * 8 + g;
-    const bool live = head < p.group;
+    const bool live = head < p.cols;
     const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
-        p.q + (int64_t(b) * p.num_q_heads + int64_t(kvh) * p.group + (live ? head : 0)) * D);
+        p.q + (int64_t(b) * p.num_q_heads + col_row(p, kvh, live ? head : 0)) * D);
 #pragma unroll
     for (int kk = 0; kk < D / 16; ++kk) {
       qf[nt][kk][0] = live ? __ldg(qrow + 8 * kk + t) : 0u;
@@ -198,7 +208,12 @@ __device__ __forceinline__ void load_q_frags(uint32_t (&qf)[NT][D / 16][2], cons
   }
 }
 
-// Running softmax state of one warp: heads 2t, 2t+1 of every head tile.
+// The running maximum starts at a huge negative finite value, not -inf: a column all of whose tokens so far were
+// masked (score -inf) then keeps m finite, so m_old - m_new = 0 and score - m = -inf give the factors 1 and 0
+// that leave its zeros alone, with no special case.  Real scores are nowhere near it.
+constexpr float kNegBig = -1.0e30f;
+
+// Running softmax state of one warp: columns 2t, 2t+1 of every 8-wide tile.
 template <int D, int NT>
 struct WarpAcc {
   float m[NT][2], l[NT][2];
@@ -206,7 +221,7 @@ struct WarpAcc {
   __device__ __forceinline__ void reset() {
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-      m[nt][0] = m[nt][1] = -INFINITY;
+      m[nt][0] = m[nt][1] = kNegBig;
       l[nt][0] = l[nt][1] = 0.f;
 #pragma unroll
       for (int mt = 0; mt < D / 16; ++mt) acc[nt][mt][0] = acc[nt][mt][1] = acc[nt][mt][2] = acc[nt][mt][3] = 0.f;
@@ -216,9 +231,13 @@ struct WarpAcc {
 
 // One page (16 tokens) of one KV head: scores, online softmax update, PV accumulation.
 // kt / vt: shared-memory addresses of the K and V tiles; v_gen: generic pointer to the V tile.
+// n_valid: tokens of the tile inside the unit's chunk.  n_common: tokens of the tile that EVERY column sees
+// (< n_valid only where several query tokens end at different positions); when it is < 16 the columns are
+// masked one by one: column (nt, e) of this thread sees the first len_rel - cut[nt][e] tokens of the tile.
 template <int D, int NT>
 __device__ __forceinline__ void process_page(WarpAcc<D, NT>& st, const uint32_t (&qf)[NT][D / 16][2], uint32_t kt,
-                                             uint32_t vt, uint8_t* v_gen, int n_valid, float scale_log2, int lane) {
+                                             uint32_t vt, uint8_t* v_gen, int n_valid, float scale_log2, int lane,
+                                             int n_common, int len_rel, const int (&cut)[NT][2]) {
   constexpr int KS = D / 16;
   const int g = lane >> 2;
   const int k_row = lane & 15, k_sel = lane >> 4;
@@ -261,9 +280,12 @@ __device__ __forceinline__ void process_page(WarpAcc<D, NT>& st, const uint32_t 
   for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) sc[nt][e] = (sc[nt][e] + sc2[nt][e]) * scale_log2;
-    if (n_valid < 16) {
-      if (g >= n_valid) sc[nt][0] = sc[nt][1] = -INFINITY;
-      if (g + 8 >= n_valid) sc[nt][2] = sc[nt][3] = -INFINITY;
+    if (n_common < 16) {
+      const int nv0 = min(n_valid, len_rel - cut[nt][0]), nv1 = min(n_valid, len_rel - cut[nt][1]);
+      if (g >= nv0) sc[nt][0] = -INFINITY;
+      if (g >= nv1) sc[nt][1] = -INFINITY;
+      if (g + 8 >= nv0) sc[nt][2] = -INFINITY;
+      if (g + 8 >= nv1) sc[nt][3] = -INFINITY;
     }
     float mx0 = fmaxf(sc[nt][0], sc[nt][2]);
     float mx1 = fmaxf(sc[nt][1], sc[nt][3]);
@@ -279,7 +301,7 @@ __device__ __forceinline__ void process_page(WarpAcc<D, NT>& st, const uint32_t 
   if (__any_sync(0xffffffffu, grew)) {
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-      const float f0 = ex2(st.m[nt][0] - m_new[nt][0]);  // first page: 2^(-inf) = 0 on zeros
+      const float f0 = ex2(st.m[nt][0] - m_new[nt][0]);  // first page: 2^(-huge) = 0 on zeros
       const float f1 = ex2(st.m[nt][1] - m_new[nt][1]);
       st.l[nt][0] *= f0;
       st.l[nt][1] *= f1;
@@ -351,33 +373,35 @@ __device__ __forceinline__ void stage_warp_result(WarpAcc<D, NT>& st, float* o_s
 }
 
 // Merge the NW staged warp results in warp order and write the unit's result: bf16 `out` if the
-// sequence is not split, else fp32 partial O (normalised) and its natural-log LSE.
+// sequence is not split, else fp32 partial O (normalised) and its natural-log LSE, per column of the unit.
 // o_sm: [NW][o_stride floats], m_sm / l_sm: [NW][NT*8].
 template <int D, int NT, int NW>
 __device__ __forceinline__ void merge_and_write(const DecodeParams& p, const Unit& u, const float* o_sm, int o_stride,
                                                 const float* m_sm, const float* l_sm, int tid, int nthreads) {
-  const int G = p.group;
-  for (int idx = tid; idx < G * D; idx += nthreads) {
+  for (int idx = tid; idx < p.cols * D; idx += nthreads) {
     const int h = idx / D;
     const int dim = idx - h * D;
-    float m_all = -INFINITY;
+    float m_all = kNegBig;
 #pragma unroll
     for (int w = 0; w < NW; ++w) m_all = fmaxf(m_all, m_sm[w * NT * 8 + h]);
     float num = 0.f, den = 0.f;
 #pragma unroll
     for (int w = 0; w < NW; ++w) {
       const float mw = m_sm[w * NT * 8 + h];
-      const float f = (mw == -INFINITY) ? 0.f : ex2(mw - m_all);
+      const float f = ex2(mw - m_all);   // a warp that saw nothing has l = 0 and O = 0: its factor does not matter
       num += f * o_sm[w * o_stride + h * D + dim];
       den += f * l_sm[w * NT * 8 + h];
     }
-    const float o = num / den;
-    const int64_t head = int64_t(u.kvh) * G + h;
+    const float o = (den > 0.f) ? num / den : 0.f;   // a query token that sees nothing of this unit
+    const int64_t head = col_row(p, u.kvh, h);
     if (u.slot < 0) {
       p.out[(int64_t(u.b) * p.num_q_heads + head) * D + dim] = __float2bfloat16_rn(o);
     } else {
       p.partial_o[(int64_t(u.slot) * p.num_q_heads + head) * D + dim] = o;
-      if (dim == 0) p.partial_lse[int64_t(u.slot) * p.num_q_heads + head] = (m_all + lg2(den)) * 0.6931471805599453f;
+      if (dim == 0) {
+        p.partial_lse[int64_t(u.slot) * p.num_q_heads + head] =
+            (den > 0.f) ? (m_all + lg2(den)) * 0.6931471805599453f : -INFINITY;
+      }
     }
   }
 }
@@ -497,10 +521,21 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   };
   int32_t ids_cur = load_ids(0);
   int32_t ids_nxt = load_ids(1);
-  const int len_dev = (threadIdx.x == 0) ? __ldg(p.seq_lens + u.b) : 0;
+  const int len_dev = __ldg(p.seq_lens + u.b);
 
   uint32_t qf[NT][D / 16][2];
   load_q_frags<D, NT>(qf, p, u.b, kvh, lane);
+  // query token i stops seeing the cache q_len - 1 - i tokens before its end; this thread's columns:
+  int cut[NT][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int c = nt * 8 + 2 * (lane & 3) + e;
+      cut[nt][e] = (c < p.cols) ? p.q_len - 1 - c / p.group : 0;
+    }
+  }
+  const int common_end = min(u.kv_end, len_dev - (p.q_len - 1));   // tokens below this are seen by every column
 
   auto issue = [&](int j, int s) {
     if ((j & 31) == 0 && j > 0) {
@@ -575,7 +610,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
       __syncwarp();
     }
     process_page<D, NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes, u.kv_end - tok0,
-                        p.scale_log2, lane);
+                        p.scale_log2, lane, common_end - tok0, len_dev - tok0, cut);
     }
     __syncwarp();  // every lane has consumed the stage before lane 0 refills it
     if (it + STAGES < n_it) issue(it + STAGES, s);
@@ -607,7 +642,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 
   // ---- step C inside this kernel: the block that publishes the last partial of (b, kvh) merges them
   if (u.slot < 0 || !p.fused_combine) return;
-  const int G = p.group;
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -619,9 +653,10 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  // one warp per query head of this KV head, exactly as the combine kernel would do it
-  for (int h = warp; h < G; h += NW) {
-    combine_row<D>(p.partial_o, p.partial_lse, p.out, u.b, u.slot - u.chunk_j, u.n_chunks, p.num_q_heads, kvh * G + h, lane);
+  // one warp per column of this KV head, exactly as the combine kernel would do it
+  for (int c = warp; c < p.cols; c += NW) {
+    combine_row<D>(p.partial_o, p.partial_lse, p.out, u.b, u.slot - u.chunk_j, u.n_chunks, p.num_q_heads,
+                   col_row(p, kvh, c), lane);
   }
 }
 

@@ -63,10 +63,12 @@ const std::vector<Variant>& variants() {
   return v;
 }
 
-// Measurement build of the default block shape (copies only, no math); [D == 128]
+// Measurement build of the default block shape (copies only, no math); [D == 128][NT - 1]
 constexpr int kLoadsOnlyWarps = 8, kLoadsOnlyStages = 3;
-const DecodeKernelFn kLoadsOnlyFn[2] = {libra::decode_kernel<64, 1, kLoadsOnlyWarps, kLoadsOnlyStages, true>,
-                                        libra::decode_kernel<128, 1, kLoadsOnlyWarps, kLoadsOnlyStages, true>};
+const DecodeKernelFn kLoadsOnlyFn[2][2] = {{libra::decode_kernel<64, 1, kLoadsOnlyWarps, kLoadsOnlyStages, true>,
+                                            libra::decode_kernel<64, 2, kLoadsOnlyWarps, kLoadsOnlyStages, true>},
+                                           {libra::decode_kernel<128, 1, kLoadsOnlyWarps, kLoadsOnlyStages, true>,
+                                            libra::decode_kernel<128, 2, kLoadsOnlyWarps, kLoadsOnlyStages, true>}};
 const int kLoadsOnlySmem[2] = {libra::DecodeSmem<64, kLoadsOnlyWarps, kLoadsOnlyStages>::kDynamicBytes,
                                libra::DecodeSmem<128, kLoadsOnlyWarps, kLoadsOnlyStages>::kDynamicBytes};
 
@@ -101,6 +103,7 @@ struct libra_handle_s {
   int64_t pool_elems = 0;
   int last_cuda_error = 0;
   int variant = 0;
+  int max_q_len = 1;        // query tokens per sequence the workspace is laid out for
   EncodeTiledFn encode = nullptr;
 
   // workspace layout: control words | arrival counters | partial LSE | partial O | oversized plans
@@ -208,6 +211,25 @@ int encode_pool_map(libra_handle_t h, const void* base, CUtensorMap* map, int* p
     return LIBRA_CUDA_ERROR;
   }
   return LIBRA_OK;
+}
+
+// Workspace layout; the partial buffers hold max_q_len * num_q_heads rows per work item.
+void compute_layout(libra_handle_t h) {
+  const libra_config_t* cfg = &h->cfg;
+  const size_t rows = size_t(h->max_q_len) * cfg->num_q_heads;
+  h->max_items = libra::max_items(h->params, cfg->num_kv_heads, cfg->max_batch);
+  h->cnt_off = 256;  // the first 256 bytes hold the control words (the device error word)
+  h->cnt_bytes = align_up(size_t(cfg->max_batch) * cfg->num_kv_heads * 4, 256);
+  h->lse_off = h->cnt_off + h->cnt_bytes;
+  h->o_off = h->lse_off + align_up(size_t(h->max_items) * rows * 4, 256);
+  h->plan_off = h->o_off + align_up(size_t(h->max_items) * rows * cfg->head_dim * 4, 256);
+  // plan region: counts | per-sequence arrays (device planner) | entries (items + empties) | merges
+  h->dev_counts_off = h->plan_off;
+  h->dev_per_seq_off = h->dev_counts_off + 256;
+  h->dev_entries_off = h->dev_per_seq_off + align_up(size_t(4) * cfg->max_batch * sizeof(int32_t), 256);
+  h->dev_fixes_off = h->dev_entries_off + align_up((size_t(h->max_items) + size_t(cfg->max_batch)) * sizeof(int4), 256);
+  h->plan_bytes = h->dev_fixes_off + align_up(size_t(cfg->max_batch) * sizeof(int4), 256) - h->plan_off;
+  h->workspace_bytes = h->plan_off + h->plan_bytes;
 }
 
 // ---- built-in scratch for libra_decode_attn_static --------------------------------------------
@@ -380,9 +402,9 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
       }
     }
     if (status != LIBRA_OK) break;
-    for (int di = 0; di < 2; ++di) {
-      e = cudaFuncSetAttribute(reinterpret_cast<const void*>(kLoadsOnlyFn[di]), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               kLoadsOnlySmem[di]);
+    for (int di = 0; di < 4; ++di) {
+      e = cudaFuncSetAttribute(reinterpret_cast<const void*>(kLoadsOnlyFn[di >> 1][di & 1]),
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, kLoadsOnlySmem[di >> 1]);
       if (e != cudaSuccess) break;
     }
     if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
@@ -390,19 +412,7 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
                              int(libra::plan_kernel_smem_bytes()));
     if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
 
-    h->max_items = libra::max_items(h->params, cfg->num_kv_heads, cfg->max_batch);
-    h->cnt_off = 256;  // the first 256 bytes hold the control words (the device error word)
-    h->cnt_bytes = align_up(size_t(cfg->max_batch) * cfg->num_kv_heads * 4, 256);
-    h->lse_off = h->cnt_off + h->cnt_bytes;
-    h->o_off = h->lse_off + align_up(size_t(h->max_items) * cfg->num_q_heads * 4, 256);
-    h->plan_off = h->o_off + align_up(size_t(h->max_items) * cfg->num_q_heads * cfg->head_dim * 4, 256);
-    // plan region: counts | per-sequence arrays (device planner) | entries (items + empties) | merges
-    h->dev_counts_off = h->plan_off;
-    h->dev_per_seq_off = h->dev_counts_off + 256;
-    h->dev_entries_off = h->dev_per_seq_off + align_up(size_t(4) * cfg->max_batch * sizeof(int32_t), 256);
-    h->dev_fixes_off = h->dev_entries_off + align_up((size_t(h->max_items) + size_t(cfg->max_batch)) * sizeof(int4), 256);
-    h->plan_bytes = h->dev_fixes_off + align_up(size_t(cfg->max_batch) * sizeof(int4), 256) - h->plan_off;
-    h->workspace_bytes = h->plan_off + h->plan_bytes;
+    compute_layout(h);
 
     for (int i = 0; i < 2; ++i) {
       if ((e = cudaHostAlloc(reinterpret_cast<void**>(&h->staging[i]), h->plan_bytes, cudaHostAllocDefault)) != cudaSuccess ||
@@ -642,6 +652,17 @@ int libra_set_dependent_launch(libra_handle_t h, int32_t on) {
   return LIBRA_OK;
 }
 
+int libra_set_max_query_tokens(libra_handle_t h, int32_t max_q_len) {
+  if (!h || max_q_len < 1) return LIBRA_INVALID_ARGUMENT;
+  if (max_q_len * h->group > 16) return LIBRA_UNSUPPORTED_SHAPE;  // a unit's score tile has at most 16 columns
+  if (max_q_len == h->max_q_len) return LIBRA_OK;
+  h->max_q_len = max_q_len;
+  compute_layout(h);
+  h->planned = false;          // the workspace layout changed: plan again, into a workspace of the new size
+  h->clean_workspace = nullptr;
+  return LIBRA_OK;
+}
+
 int libra_set_variant(libra_handle_t h, int32_t warps, int32_t stages) {
   if (!h) return LIBRA_INVALID_ARGUMENT;
   const std::vector<Variant>& vs = variants();
@@ -663,7 +684,7 @@ namespace {
 // Steps D and C; k_new / v_new non-null = append the current token's K and V rows on the way.
 int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* v_new, const void* k_pages,
                 const void* v_pages, const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream,
-                bool loads_only = false) {
+                bool loads_only = false, int32_t q_len = 1) {
   if (!h || !q || !k_pages || !v_pages || !block_table || !seq_lens || !out) return LIBRA_INVALID_ARGUMENT;
   if ((k_new == nullptr) != (v_new == nullptr)) return LIBRA_INVALID_ARGUMENT;
   if (reinterpret_cast<uintptr_t>(k_new) % 16 || reinterpret_cast<uintptr_t>(v_new) % 16) return LIBRA_INVALID_ARGUMENT;
@@ -671,6 +692,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
       reinterpret_cast<uintptr_t>(q) % 4 || reinterpret_cast<uintptr_t>(out) % 4) {
     return LIBRA_INVALID_ARGUMENT;
   }
+  if (q_len < 1 || q_len > h->max_q_len || (q_len > 1 && k_new)) return LIBRA_INVALID_ARGUMENT;
   if (!h->planned) return LIBRA_NOT_PLANNED;
   DeviceGuard guard(h->cfg.device);
   if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
@@ -710,7 +732,8 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
 
   const Variant& v = variants()[h->variant];
   const int di = (h->cfg.head_dim == 128) ? 1 : 0;
-  const int ni = (h->group > 8) ? 1 : 0;
+  const int ni = (h->group * q_len > 8) ? 1 : 0;
+  const int32_t rows = q_len * h->cfg.num_q_heads;   // rows of q / out per sequence
   const bool fused = h->combine_mode == 1 || loads_only;
   // host plan: exact counts; device plan: upper bounds for the grids, the kernels read the counts themselves
   const int32_t n_empty = h->device_planned ? h->planned_batch : int32_t(h->plan.empty.size());
@@ -731,9 +754,12 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     p.error_word = err_dev;
     p.counters = reinterpret_cast<int32_t*>(ws + h->cnt_off);
     p.num_pages = h->cfg.num_pages;
-    p.num_q_heads = h->cfg.num_q_heads;
+    p.num_q_heads = rows;
     p.num_kv_heads = h->cfg.num_kv_heads;
     p.group = h->group;
+    p.q_len = q_len;
+    p.hq = h->cfg.num_q_heads;
+    p.cols = q_len * h->group;
     p.block_table_ld = h->cfg.block_table_ld;
     p.scale_log2 = h->scale_log2;
     p.pos_head = h->pos_head;
@@ -764,7 +790,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = h->pdl ? 1 : 0;
-    LIBRA_CUDA_TRY(h, cudaLaunchKernelEx(&lc, loads_only ? kLoadsOnlyFn[di] : v.fn[di][ni], pm->map_k, pm->map_v, p, h->pp));
+    LIBRA_CUDA_TRY(h, cudaLaunchKernelEx(&lc, loads_only ? kLoadsOnlyFn[di][ni] : v.fn[di][ni], pm->map_k, pm->map_v, p, h->pp));
     ++h->launches;
   }
   if (ev) LIBRA_CUDA_TRY(h, cudaEventRecord(ev[1], st));
@@ -779,11 +805,11 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     c.seq_lens = seq_lens;
     c.out = static_cast<__nv_bfloat16*>(out);
     c.error_word = err_dev;
-    c.num_q_heads = h->cfg.num_q_heads;
+    c.num_q_heads = rows;
     // a programmatic dependent of the decode kernel: it may be scheduled while that kernel drains and
     // waits inside (griddepcontrol.wait) for it to finish
     cudaLaunchConfig_t lc = {};
-    lc.gridDim = dim3(unsigned(n_combine), unsigned((h->cfg.num_q_heads + libra::kCombineWarps - 1) / libra::kCombineWarps));
+    lc.gridDim = dim3(unsigned(n_combine), unsigned((rows + libra::kCombineWarps - 1) / libra::kCombineWarps));
     lc.blockDim = dim3(libra::kCombineWarps * 32);
     lc.dynamicSmemBytes = 0;
     lc.stream = st;
@@ -998,6 +1024,11 @@ int libra_debug_wait_selftest(libra_handle_t h, void* stream) {
   LIBRA_CUDA_TRY(h, cudaGetLastError());
   h->last_stream = stream;
   return LIBRA_OK;
+}
+
+int libra_decode_attn_multi(libra_handle_t h, const void* q, int32_t q_len, const void* k_pages, const void* v_pages,
+                            const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream) {
+  return decode_impl(h, q, nullptr, nullptr, k_pages, v_pages, block_table, seq_lens, out, stream, false, q_len);
 }
 
 int libra_debug_gather_read(libra_handle_t h, const void* q, const void* k_pages, const void* v_pages,

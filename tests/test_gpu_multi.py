@@ -1,0 +1,181 @@
+"""GPU parity of libra_decode_attn_multi (several query tokens per sequence, causal over the newly appended
+tokens) against the float64 CPU oracle, through the C ABI, with the same two gates as single-token decode."""
+import numpy as np
+import pytest
+
+from oracle import attention_oracle as O
+from paper_2606_03077_b200 import workloads as W
+
+import gates
+import gpu_harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def check(got, ref, what=""):
+    assert np.all(np.isfinite(got)), f"{what}: non-finite output (unwritten row?)"
+    assert gates.stated_violations(got, ref) == 0, f"{what}: stated gate"
+    assert gates.tight_violations(got, ref) == 0, f"{what}: tight gate, ratio {gates.tight_ratio(got, ref):.2f}"
+
+
+def draw_q(seed, B, Tq, Hq, d):
+    rng = np.random.default_rng(seed)
+    return W.f32_to_bf16_bits(rng.standard_normal((B, Tq, Hq, d)).astype(np.float32))
+
+
+def run_multi(lib, q, k, v, bt, lens, layout="HND", plan=None, fused=None, max_q=None, page_size=16):
+    """q: uint16 [B, Tq, Hq, d] -> float32 [B, Tq, Hq, d]."""
+    import torch
+    dev = torch.device("cuda:0")
+    B, Tq, Hq, d = q.shape
+    Hkv = k.shape[1]
+    if layout == "NHD":
+        k = np.ascontiguousarray(k.transpose(0, 2, 1, 3))
+        v = np.ascontiguousarray(v.transpose(0, 2, 1, 3))
+    strides = (page_size * Hkv * d, d, Hkv * d) if layout == "NHD" else (0, 0, 0)
+    h = lib.Handle(Hq, Hkv, d, k.shape[0], max(B, 1), bt.shape[1], page_size=page_size, kv_strides=strides, plan=plan)
+    if fused is not None:
+        h.set_combine_mode(fused)
+    h.set_max_query_tokens(max_q or Tq)
+    ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=dev)
+    qd, kd, vd, btd = (H.to_dev(x, dev) for x in (q, k, v, bt))
+    lens_dev = torch.from_numpy(np.ascontiguousarray(lens, dtype=np.int32)).to(dev)
+    out = torch.full((B, Tq, Hq, d), H.CANARY, dtype=torch.int16, device=dev)
+    st = torch.cuda.current_stream().cuda_stream
+    h.plan(np.asarray(lens, dtype=np.int32), ws.data_ptr(), ws.numel(), st)
+    h.decode_attn_multi(qd.data_ptr(), Tq, kd.data_ptr(), vd.data_ptr(), btd.data_ptr(), lens_dev.data_ptr(),
+                        out.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert h.debug_error_word() == 0
+    res = H.bf16_dev_to_f32(out)
+    h.close()
+    return res
+
+
+def small_plan(lib):
+    return lib.PlanParams(4, 1, 2, 16, 16, 64)
+
+
+CASES = [
+    # (Hq, Hkv, d, Tq, lens)
+    (4, 1, 64, 4, [4, 5, 16, 17, 19, 33, 300]),         # G = 4, 16 columns
+    (8, 2, 128, 2, [255, 256, 257, 2, 700]),            # G = 4
+    (8, 8, 128, 16, [16, 100, 1000, 31]),               # G = 1, 16 query tokens: the limits span two tiles
+    (64, 8, 128, 2, [3000, 5, 1025]),                   # G = 8
+    (40, 8, 128, 3, [1200, 77, 2049]),                  # G = 5, 15 columns
+    (6, 2, 64, 5, [0, 40, 3, 300, 1, 5]),               # empty and shorter-than-Tq sequences
+    (4, 2, 128, 8, [513, 48, 520]),                     # G = 2
+]
+
+
+@pytest.mark.parametrize("layout", ["HND", "NHD"])
+@pytest.mark.parametrize("case", range(len(CASES)))
+def test_shapes_tails_and_causal_limits(lib, case, layout):
+    Hq, Hkv, d, Tq, lens = CASES[case]
+    lens_a, bt, _, k, v = W.random_case(400 + case, len(lens), Hq, Hkv, d, lens)
+    q = draw_q(500 + case, len(lens), Tq, Hq, d)
+    ref, _ = O.paged_multi_token_attention(q, k, v, bt, lens_a)
+    for plan in (None, small_plan(lib)):
+        got = run_multi(lib, q, k, v, bt, lens_a, layout=layout, plan=plan)
+        check(got, ref, f"case {case} {layout} plan={'default' if plan is None else 'small'}")
+    two = run_multi(lib, q, k, v, bt, lens_a, layout=layout, plan=small_plan(lib), fused=0)
+    assert np.array_equal(two, got)     # step C as its own kernel: same bits
+
+
+def test_one_query_token_equals_single_token_entry_point(lib):
+    lens = [2500, 300, 17, 4100, 0]
+    lens_a, bt, q, k, v = W.random_case(47, len(lens), 32, 8, 128, lens)
+    one = H.run_host_case(lib, q, k, v, bt, lens_a)
+    multi = run_multi(lib, q[:, None], k, v, bt, lens_a, max_q=2)
+    assert np.array_equal(multi[:, 0], one)
+
+
+def test_rows_match_single_token_steps_at_shorter_lengths(lib):
+    # row i of a q_len = 4 step against a single-token step on the sequence cut to L - 3 + i tokens: same
+    # inputs, same tolerance class; the two runs split differently, so compare through the oracle's gates
+    Tq = 4
+    lens = [1030, 2051, 600]
+    lens_a, bt, _, k, v = W.random_case(48, 3, 16, 4, 128, lens)
+    q = draw_q(49, 3, Tq, 16, 128)
+    got = run_multi(lib, q, k, v, bt, lens_a, plan=lib.PlanParams(8, 1, 2, 256, 256, 64))
+    for i in range(Tq):
+        ref, _ = O.paged_decode_attention(q[:, i], k, v, bt, lens_a - Tq + 1 + i)
+        check(got[:, i], ref, f"row {i}")
+
+
+def test_last_chunk_shorter_than_the_query_block(lib):
+    # chunks of 16 tokens: L = 16 j + 1 leaves a last chunk of ONE token, so the earlier query tokens see nothing
+    # of it (their partial result is empty) and are masked inside the second-to-last chunk too
+    Tq = 4
+    lens = [17, 33, 49, 18, 34]
+    lens_a, bt, _, k, v = W.random_case(50, len(lens), 4, 1, 64, lens)
+    q = draw_q(51, len(lens), Tq, 4, 64)
+    ref, _ = O.paged_multi_token_attention(q, k, v, bt, lens_a)
+    for fused in (0, 1):
+        got = run_multi(lib, q, k, v, bt, lens_a, plan=lib.PlanParams(64, 1, 8, 16, 16, 64), fused=fused)
+        check(got, ref, f"short last chunk, fused={fused}")
+
+
+def test_one_hot_keys_show_the_exact_causal_limit(lib):
+    # dominant keys at token 0 and at each new token: row i is the exact mean of the value rows of token 0 and new
+    # tokens 0..i (small integers, so the means of 2..5 rows round to bf16 the same way in any order)
+    import math
+    Tq, d, L = 4, 64, 70
+    c = math.sqrt(200.0 * math.sqrt(d))
+    lens_a, bt, _, k, v = W.random_case(52, 1, 2, 1, d, [L])
+    rng = np.random.default_rng(53)
+    vals = rng.integers(-8, 9, size=(L, d)).astype(np.float32)
+    new = list(range(L - Tq, L))
+    for t in range(L):
+        row = np.zeros(d, dtype=np.float32)
+        if t == 0 or t in new:
+            row[0] = c
+        k[bt[0, t // 16], 0, t % 16] = W.f32_to_bf16_bits(row)
+        v[bt[0, t // 16], 0, t % 16] = W.f32_to_bf16_bits(vals[t])
+    qrow = np.zeros(d, dtype=np.float32)
+    qrow[0] = c
+    q = np.broadcast_to(W.f32_to_bf16_bits(qrow), (1, Tq, 2, d)).copy()
+    for plan in (None, small_plan(lib)):
+        got = run_multi(lib, q, k, v, bt, lens_a, plan=plan)
+        for i in range(Tq):
+            seen = [0] + new[: i + 1]
+            want = O.round_to_bf16(vals[seen].astype(np.float64).mean(axis=0))
+            # P = 1 exactly for the dominant keys (equal scores), 0 for the rest; the division by the count is the
+            # only rounding before the bf16 store
+            assert np.max(np.abs(got[0, i, 0] - want)) <= 2.0 ** -7 * np.max(np.abs(want)), f"row {i}"
+            assert np.array_equal(got[0, i, 0], got[0, i, 1])
+
+
+def test_nan_garbage_and_larger_pages(lib):
+    # slots past the end of a sequence hold NaN (the generator's poison); page size 32
+    Tq = 3
+    lens = [1, 16, 17, 31, 32, 33, 700, 2]
+    lens_a, bt, _, k, v = W.random_case(54, len(lens), 8, 2, 128, lens, page_size=32)
+    q = draw_q(55, len(lens), Tq, 8, 128)
+    ref, _ = O.paged_multi_token_attention(q, k, v, bt, lens_a)
+    for layout in ("HND", "NHD"):
+        got = run_multi(lib, q, k, v, bt, lens_a, layout=layout, plan=lib.PlanParams(4, 1, 2, 32, 32, 64), page_size=32)
+        check(got, ref, f"page 32 {layout}")
+
+
+def test_misuse_is_rejected(lib):
+    import torch
+    h = lib.Handle(32, 8, 128, 64, 4, 8)
+    with pytest.raises(lib.LibraError):
+        h.set_max_query_tokens(0)
+    with pytest.raises(lib.LibraError):
+        h.set_max_query_tokens(5)          # 5 x G = 20 columns
+    size1 = h.workspace_size()
+    h.set_max_query_tokens(4)
+    assert h.workspace_size() > size1
+    ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device="cuda:0")
+    st = torch.cuda.current_stream().cuda_stream
+    x = torch.zeros(1 << 16, dtype=torch.int16, device="cuda:0")
+    with pytest.raises(lib.LibraError):    # the call above dropped the plan
+        h.decode_attn_multi(x.data_ptr(), 2, x.data_ptr(), x.data_ptr(), x.data_ptr(), x.data_ptr(), x.data_ptr(), st)
+    h.plan(np.array([5], dtype=np.int32), ws.data_ptr(), ws.numel(), st)
+    for bad in (0, 5, -1):
+        with pytest.raises(lib.LibraError):
+            h.decode_attn_multi(x.data_ptr(), bad, x.data_ptr(), x.data_ptr(), x.data_ptr(), x.data_ptr(), x.data_ptr(), st)
+    torch.cuda.synchronize()
+    h.close()
