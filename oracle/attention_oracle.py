@@ -33,7 +33,10 @@ loop-only brute force agrees on tiny inputs; chunked evaluation plus merge equal
 direct formula; an analytic two-token case.  The several-query-token form is pinned by
 its reduction to the single-token function row by row, by the loop-only brute force, by
 one-hot keys planted on either side of each query token's causal limit, and by the
-zero-query running mean in closed form.
+zero-query running mean in closed form.  The E4M3 decoder is pinned by the format's
+landmark values and by a library conversion of all 256 codes; the E4M3-cache form by its
+equality with the bf16 definition on the decoded values (every E4M3 value is a bf16 value)
+and by the scale identities.
 """
 from __future__ import annotations
 
@@ -145,6 +148,54 @@ def paged_multi_token_attention(q, k_pages, v_pages, block_table, seq_lens, layo
             z = e.sum(axis=2, keepdims=True)
             out[b, i] = np.matmul(e / z, V[:, :n]).reshape(Hq, d)
             lse[b, i] = (m + np.log(z)).reshape(Hq)
+    return out, lse
+
+
+def e4m3_to_f64(codes: np.ndarray) -> np.ndarray:
+    """8-bit floating point, 1 sign / 4 exponent / 3 mantissa bits, bias 7, no infinities ("E4M3", the
+    common KV-cache storage format) -> float64, exact.  Written from the format's definition:
+    exponent field 0 is subnormal (m / 8 * 2^-6), field e >= 1 is (1 + m / 8) * 2^(e - 7); the one
+    all-ones pattern per sign (e = 15, m = 7) is NaN; the largest finite value is 448."""
+    c = np.asarray(codes, dtype=np.uint8).astype(np.int64)
+    sign = np.where(c & 0x80, -1.0, 1.0)
+    e = (c >> 3) & 0xF
+    m = (c & 0x7).astype(np.float64)
+    mag = np.where(e == 0, m / 8.0 * 2.0 ** -6, (1.0 + m / 8.0) * np.exp2((e - 7).astype(np.float64)))
+    mag = np.where((e == 15) & (m == 7), np.nan, mag)
+    return sign * mag
+
+
+def paged_decode_attention_fp8(q, k_pages8, v_pages8, block_table, seq_lens, k_scale: float = 1.0,
+                               v_scale: float = 1.0, sm_scale: float | None = None):
+    """Single-token decode over a KV cache stored as E4M3 codes with one scale per tensor: the cached
+    key of token t is k_scale * e4m3(k code), the value v_scale * e4m3(v code); everything else is the
+    definition at the top of this file, in float64.  Pools: uint8 [num_pages, Hkv, page_size, d] (HND).
+    q: uint16 bf16 bits [B, Hq, d].  Returns (out float64[B, Hq, d], lse float64[B, Hq])."""
+    q = np.asarray(q)
+    B, Hq, d = q.shape
+    Hkv, page_size = k_pages8.shape[1], k_pages8.shape[2]
+    assert Hq % Hkv == 0
+    G = Hq // Hkv
+    scale = 1.0 / math.sqrt(d) if sm_scale is None else float(sm_scale)
+    out = np.zeros((B, Hq, d), dtype=np.float64)
+    lse = np.full((B, Hq), -np.inf, dtype=np.float64)
+    for b in range(B):
+        L = int(seq_lens[b])
+        if L == 0:
+            continue
+        n_pages = (L + page_size - 1) // page_size
+        ids = np.asarray(block_table[b, :n_pages], dtype=np.int64)
+        if np.any(ids < 0) or np.any(ids >= k_pages8.shape[0]):
+            raise IndexError("block table entry outside the pool")
+        K = e4m3_to_f64(k_pages8[ids].transpose(1, 0, 2, 3).reshape(Hkv, n_pages * page_size, d)[:, :L]) * float(k_scale)
+        V = e4m3_to_f64(v_pages8[ids].transpose(1, 0, 2, 3).reshape(Hkv, n_pages * page_size, d)[:, :L]) * float(v_scale)
+        qb = bf16_bits_to_f64(q[b]).reshape(Hkv, G, d)
+        s = np.matmul(qb, K.transpose(0, 2, 1)) * scale
+        m = s.max(axis=2, keepdims=True)
+        e = np.exp(s - m)
+        z = e.sum(axis=2, keepdims=True)
+        out[b] = np.matmul(e / z, V).reshape(Hq, d)
+        lse[b] = (m + np.log(z)).reshape(Hq)
     return out, lse
 
 

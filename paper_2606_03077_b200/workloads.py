@@ -259,6 +259,41 @@ def fill_device_pools(layout: Layout, device, seed: int | None = None, chunk_pag
     return q, k, v
 
 
+E4M3_NAN = 0x7F  # the poison of an 8-bit cache: slots past the end of a sequence hold NaN codes
+
+
+def random_case_e4m3(seed: int, batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int, seq_lens,
+                     spare_pages: int = 3, poison: bool = True, page_size: int = PAGE_SIZE, max_exp_field: int = 8):
+    """Ad-hoc case with an 8-bit KV cache: q as bf16 bits, K and V as E4M3 codes drawn as bit fields (sign,
+    exponent field 0..max_exp_field, mantissa: magnitudes below 2^(max_exp_field - 6), no NaN codes), so that
+    no float arithmetic is involved in making them.  Returns (lens, block_table, q, k_codes, v_codes)."""
+    rng = Generator(PCG64(seed))
+    lens = np.asarray(seq_lens, dtype=np.int32)
+    assert lens.shape == (batch,)
+    need = int(pages_needed(lens, page_size).sum())
+    bt, pool = draw_block_table(lens, need + spare_pages, rng, page_size)
+    q = _draw_bf16(rng, (batch, num_q_heads, head_dim), "normal")
+    shape = (pool, num_kv_heads, page_size, head_dim)
+
+    def codes():
+        sign = rng.integers(0, 2, size=shape, dtype=np.uint8)
+        expo = rng.integers(0, max_exp_field + 1, size=shape, dtype=np.uint8)
+        mant = rng.integers(0, 8, size=shape, dtype=np.uint8)
+        return (sign << 7) | (expo << 3) | mant
+
+    k, v = codes(), codes()
+    if poison:
+        keep = np.zeros((pool, page_size), dtype=bool)
+        for b in range(batch):
+            L = int(lens[b])
+            for t0 in range(0, L, page_size):
+                keep[bt[b, t0 // page_size], : min(page_size, L - t0)] = True
+        dead = ~keep
+        k[dead[:, None, :, None] & np.ones(shape, dtype=bool)] = E4M3_NAN
+        v[dead[:, None, :, None] & np.ones(shape, dtype=bool)] = E4M3_NAN | 0x80
+    return lens, bt, q, k, v
+
+
 def poison_tails(layout: Layout, k, v):
     """Overwrite the slots past the end of every sequence's last page (device HND pools) with the
     poison value.  Returns what was there, for ``restore_tails``: a multi-step workload reuses the
