@@ -361,6 +361,65 @@ def multi_token_measure(rep: Replica, q_len: int, steps: int = 200):
             "query_tokens_per_s": w.batch * q_len / (ms * 1e-3), "steps": steps}
 
 
+def fp8_cache_measure(rep: Replica, steps: int = 200, variant=None):
+    """The step over an E4M3 KV cache of the same geometry (same block tables and lengths, random finite codes):
+    half the bytes per cached token.  Also its page-gather read ceiling (same copies, no math)."""
+    torch, w = rep.torch, rep.w
+    if w.head_dim != 128:
+        return None
+    shape = rep.pools[0][0].shape
+    copies = len(rep.pools) * 2 if len(rep.pools) > 1 else 1     # half the bytes per copy: keep the live set the same
+
+    def codes():
+        r = torch.randint(0, 256, shape, dtype=torch.uint8, device=rep.dev)
+        r &= 0x87                                                 # sign and mantissa
+        r |= torch.randint(0, 9, shape, dtype=torch.uint8, device=rep.dev) << 3   # exponent field 0..8: |x| < 4
+        return r
+
+    pools = [(codes(), codes())]
+    pools += [(pools[0][0].clone(), pools[0][1].clone()) for _ in range(copies - 1)]
+    h = rep.binding.Handle(w.num_q_heads, w.num_kv_heads, w.head_dim, rep.layouts[0].pool_pages, w.batch, rep.ld,
+                           device=rep.dev.index or 0)
+    h.set_kv_dtype(rep.binding.KV_E4M3, 1.0, 1.0)
+    if variant is not None:
+        h.set_variant(*variant)
+    ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=rep.dev)
+    out = torch.zeros_like(rep.out)
+    st = torch.cuda.current_stream().cuda_stream
+
+    def run(fn, n):
+        for i in range(10):
+            fn(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        assert h.debug_error_word() == 0, "device error word set"
+        return e0.elapsed_time(e1) / n
+
+    def step(i, call=None):
+        s = i % len(rep.layouts)
+        k, v = pools[i % len(pools)]
+        h.plan(rep.layouts[s].seq_lens, ws.data_ptr(), ws.numel(), st)
+        (call or h.decode_attn)(rep.q.data_ptr(), k.data_ptr(), v.data_ptr(), rep.bts[s].data_ptr(),
+                                rep.lens_dev[s].data_ptr(), out.data_ptr(), st)
+
+    steps = max(len(rep.layouts), steps // len(rep.layouts) * len(rep.layouts))
+    ms = run(step, steps)
+    ms_read = run(lambda i: step(i, h.debug_gather_read), steps)
+    h.close()
+    del pools
+    torch.cuda.empty_cache()
+    bytes8 = rep.kv_bytes_per_step / 2
+    tokens = rep.kv_bytes_per_step / (4.0 * w.num_kv_heads * w.head_dim)
+    return {"ms_per_step": ms, "kv_gbs": bytes8 / (ms * 1e-3) / 1e9, "kv_bytes_per_step": bytes8,
+            "cached_tokens_per_s": tokens / (ms * 1e-3), "page_gather_read_gbs": bytes8 / (ms_read * 1e-3) / 1e9,
+            "pool_copies": copies, "steps": steps}
+
+
 def e2e_measure(rep: Replica, steps: int):
     """The step through libra_decode_attn_host with every input in pinned host memory."""
     torch = rep.torch
@@ -635,6 +694,7 @@ def run_libra(args):
             line["e2e_resident_kv"] = e2e_resident_kv_measure(rep, 200)
         line["ceilings"] = ceilings_measure(rep)
         line["multi_token"] = [m for m in (multi_token_measure(rep, t) for t in (2, 4)) if m]
+        line["fp8_cache"] = fp8_cache_measure(rep)
         if args.workload in ("longtail_mix_b256", "straggler_b8"):
             line["kv_migration"] = kv_migration_measure(rep)
         if not args.no_cpu:
@@ -672,6 +732,7 @@ def run_libra(args):
                             "kv_bytes_per_step": r.kv_bytes_per_step, "pool_copies": len(r.pools)}
             others[name]["ceilings"] = ceilings_measure(r, reps=10)
             others[name]["multi_token"] = [m for m in (multi_token_measure(r, t, 60) for t in (2, 3, 4)) if m]
+            others[name]["fp8_cache"] = fp8_cache_measure(r, 60)
             if name in ("longtail_mix_b256", "straggler_b8"):  # migrating the long sequences: gather to a dense buffer, scatter back
                 others[name]["kv_migration"] = kv_migration_measure(r)
             if name == "shift_b128":  # the re-planned-every-step workload: also with the device-side planner

@@ -148,6 +148,19 @@ int libra_get_plan_params(libra_handle_t handle, libra_plan_params_t* out);
  * 16 columns: max_q_len * (num_q_heads / num_kv_heads) <= 16, else UNSUPPORTED_SHAPE. */
 int libra_set_max_query_tokens(libra_handle_t handle, int32_t max_q_len);
 
+/* Storage type of the KV pools (default LIBRA_KV_BF16).  LIBRA_KV_E4M3: the pools hold 8-bit floating-point
+ * codes (1 sign, 4 exponent, 3 mantissa bits, bias 7, no infinities, one NaN per sign), one byte per element,
+ * with one scale per tensor: key = k_scale * value of the code, value = v_scale * value of the code; the
+ * attention is the same definition on those keys and values, q and out stay bf16.  The strides given at
+ * creation keep their meaning (elements, now bytes) and must be multiples of 16; head_dim must be 128
+ * (UNSUPPORTED_SHAPE otherwise); k_scale and v_scale must be positive and finite (ignored for BF16).
+ * Halving the bytes per cached token halves what the step has to read.  With E4M3 pools
+ * libra_decode_attn_append, libra_decode_attn_host, libra_kv_gather and libra_kv_scatter return
+ * UNSUPPORTED_SHAPE.  The plan and the workspace do not depend on the type. */
+#define LIBRA_KV_BF16 0
+#define LIBRA_KV_E4M3 1
+int libra_set_kv_dtype(libra_handle_t handle, int32_t dtype, float k_scale, float v_scale);
+
 /* Tuning knob: shape of the decode thread block: `warps` warps that each own `stages` shared-memory
  * stages of one K page plus one V page.  Only the compiled-in shapes are accepted (UNSUPPORTED_SHAPE
  * otherwise); the default is the tuned one.  Results do not depend on the stage count; the warp

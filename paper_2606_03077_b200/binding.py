@@ -20,6 +20,7 @@ LIB_PATH = _LIB_PATH
 
 STATIC_SCRATCH_BYTES = 8 << 20
 OK, INVALID_ARGUMENT, UNSUPPORTED_SHAPE, WORKSPACE_TOO_SMALL, NOT_PLANNED, CUDA_ERROR, DEVICE_FLAGGED = range(7)
+KV_BF16, KV_E4M3 = 0, 1
 ERR_WAIT_TIMEOUT, ERR_BAD_PAGE_ID, ERR_SEQ_LEN_MISMATCH, ERR_PLAN_OVERFLOW = 1, 2, 4, 8
 
 
@@ -59,6 +60,7 @@ SIGNATURES = {
     "libra_set_variant": (C.c_int, [_vp, C.c_int32, C.c_int32]),
     "libra_set_dependent_launch": (C.c_int, [_vp, C.c_int32]),
     "libra_set_max_query_tokens": (C.c_int, [_vp, C.c_int32]),
+    "libra_set_kv_dtype": (C.c_int, [_vp, C.c_int32, C.c_float, C.c_float]),
     "libra_decode_attn_multi": (C.c_int, [_vp, _vp, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_debug_stream_read": (C.c_int, [_vp, _vp, C.c_size_t, _vp]),
     "libra_debug_gather_read": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -280,6 +282,9 @@ class Handle:
                           out_ptr: int, stream: int) -> None:
         _check(lib.libra_debug_gather_read(self._h, q_ptr, k_ptr, v_ptr, block_table_ptr, seq_lens_ptr, out_ptr, stream),
                "libra_debug_gather_read")
+
+    def set_kv_dtype(self, dtype: int, k_scale: float = 1.0, v_scale: float = 1.0) -> None:
+        _check(lib.libra_set_kv_dtype(self._h, dtype, k_scale, v_scale), "libra_set_kv_dtype")
 
     def set_max_query_tokens(self, max_q_len: int) -> None:
         _check(lib.libra_set_max_query_tokens(self._h, max_q_len), "libra_set_max_query_tokens")

@@ -24,6 +24,7 @@
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -52,7 +53,8 @@ struct DecodeParams {
   int32_t hq;             // query heads of the model (num_q_heads = q_len * hq)
   int32_t cols;           // q_len * G: rows of q that share one KV head = columns of a unit's score tile
   int32_t block_table_ld;
-  float scale_log2;       // sm_scale * log2(e)
+  float scale_log2;       // sm_scale * log2(e) (times the key scale of an 8-bit cache)
+  float v_scale;          // value scale of an 8-bit cache; 1 for a bf16 cache
   int32_t pos_head;       // coordinate slot (1..3) of the head / page / token dimension in the tensor maps
   int32_t pos_page;
   int32_t pos_token;
@@ -143,6 +145,27 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// Same shape with fp16 operands (used with an 8-bit cache, whose codes convert to fp16 exactly).
+__device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// Four E4M3 codes -> two fp16 pairs: lo = codes 0, 1; hi = codes 2, 3 (exact: E4M3 is a subset of fp16).
+__device__ __forceinline__ void cvt_e4m3x4(uint32_t x, uint32_t& lo, uint32_t& hi) {
+  asm("{\n\t.reg .b16 a, b;\n\t"
+      "mov.b32 {a, b}, %2;\n\t"
+      "cvt.rn.f16x2.e4m3x2 %0, a;\n\t"
+      "cvt.rn.f16x2.e4m3x2 %1, b;\n\t}"
+      : "=r"(lo), "=r"(hi)
+      : "r"(x));
+}
+__device__ __forceinline__ uint32_t byte_perm_3120(uint32_t x) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, 0, 0x3120;" : "=r"(d) : "r"(x));
+  return d;
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -343,8 +366,160 @@ __device__ __forceinline__ void process_page(WarpAcc<D, NT>& st, const uint32_t 
   }
 }
 
+// ---- 8-bit (E4M3) cache, head_dim 128 -------------------------------------------------------------
+// A tile is 16 tokens x 128 bytes with the same 128-byte swizzle.  ldmatrix moves it as 16-bit units, i.e.
+// PAIRS of codes, so the fragments come out in an order of their own; sums over k and the assignment of
+// output rows do not care about order as long as both operands agree:
+//   scores : within a 16-dim chunk, mma k-slots (2t, 2t+1, 2t+8, 2t+9) carry dims (4t, 4t+1, 4t+2, 4t+3)
+//   output : within a 16-dim chunk, mma rows (g, g+8) carry dims (2g, 2g+1)
+// Codes are converted to fp16 (exact); q is converted bf16 -> fp16 (exact for |q| in [2^-14, 65504]) and P is
+// rounded to fp16.  (Converting the values with integer operations instead, to unload the pipe the conversion
+// instruction shares with the exponentials, measured 5-10 % slower.)
+
+// Q^T fragments in that k-order, fp16; columns >= cols are zero.
+template <int NT>
+__device__ __forceinline__ void load_q_frags_fp8(uint32_t (&qf)[NT][8][2], const DecodeParams& p, int b, int kvh, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    const int col = nt * 8 + g;
+    const bool live = col < p.cols;
+    const __nv_bfloat16* qrow = p.q + (int64_t(b) * p.num_q_heads + col_row(p, kvh, live ? col : 0)) * 128;
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {
+      const uint2 raw = __ldg(reinterpret_cast<const uint2*>(qrow + 16 * kk + 4 * t));   // dims 4t .. 4t+3 of chunk kk
+      const __nv_bfloat162 x01 = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+      const __nv_bfloat162 x23 = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+      const __half2 h01 = __floats2half2_rn(__low2float(x01), __high2float(x01));
+      const __half2 h23 = __floats2half2_rn(__low2float(x23), __high2float(x23));
+      qf[nt][kk][0] = live ? *reinterpret_cast<const uint32_t*>(&h01) : 0u;
+      qf[nt][kk][1] = live ? *reinterpret_cast<const uint32_t*>(&h23) : 0u;
+    }
+  }
+}
+
+// One page (16 tokens) of one KV head from an E4M3 cache; same contract as process_page.
+template <int NT>
+__device__ __forceinline__ void process_page_fp8(WarpAcc<128, NT>& st, const uint32_t (&qf)[NT][8][2], uint32_t kt,
+                                                 uint32_t vt, uint8_t* v_gen, int n_valid, float scale_log2, int lane,
+                                                 int n_common, int len_rel, const int (&cut)[NT][2]) {
+  const int g = lane >> 2;
+  // ldmatrix.x4: lanes 0-7 / 8-15 give the rows (tokens 0-7 / 8-15) of 16-byte chunk c, lanes 16-31 those of chunk c+1
+  const int row = (lane & 7) + ((lane >> 3) & 1) * 8;
+  const int csel = lane >> 4;
+  const uint32_t row_off = uint32_t(row) << 7;
+
+  if (n_valid < 16) {
+    // rows past the end may hold anything, NaN codes included: clear them in V so that 0 * garbage cannot leak
+    for (int i = lane; i < (16 - n_valid) * 8; i += 32) {
+      const int r = n_valid + (i >> 3);
+      *reinterpret_cast<uint4*>(v_gen + (r << 7) + ((i & 7) << 4)) = make_uint4(0, 0, 0, 0);
+    }
+    fence_proxy_async();  // these generic writes come before the next TMA write into this stage
+    __syncwarp();
+  }
+
+  // ---- S^T = K . Q^T
+  float sc[NT][4], sc2[NT][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+    sc2[nt][0] = sc2[nt][1] = sc2[nt][2] = sc2[nt][3] = 0.f;
+  }
+#pragma unroll
+  for (int c2 = 0; c2 < 4; ++c2) {
+    uint32_t r[4];   // (tokens 0-7, chunk 2 c2), (tokens 8-15, chunk 2 c2), (tokens 0-7, chunk 2 c2 + 1), (tokens 8-15, chunk 2 c2 + 1)
+    ldsm_x4(r, kt + row_off + (uint32_t((2 * c2 + csel) ^ (row & 7)) << 4));
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      uint32_t a[4];
+      cvt_e4m3x4(r[2 * half], a[0], a[2]);        // token g   : dims 4t, 4t+1 | 4t+2, 4t+3
+      cvt_e4m3x4(r[2 * half + 1], a[1], a[3]);    // token g+8
+      const int kk = 2 * c2 + half;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        if (half) mma_f16(sc2[nt], a, qf[nt][kk][0], qf[nt][kk][1]);
+        else mma_f16(sc[nt], a, qf[nt][kk][0], qf[nt][kk][1]);
+      }
+    }
+  }
+
+  // ---- online softmax; this thread holds tokens g, g+8 for columns 2t, 2t+1
+  uint32_t pb[NT][2];
+  bool grew = false;
+  float m_new[NT][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) sc[nt][e] = (sc[nt][e] + sc2[nt][e]) * scale_log2;
+    if (n_common < 16) {
+      const int nv0 = min(n_valid, len_rel - cut[nt][0]), nv1 = min(n_valid, len_rel - cut[nt][1]);
+      if (g >= nv0) sc[nt][0] = -INFINITY;
+      if (g >= nv1) sc[nt][1] = -INFINITY;
+      if (g + 8 >= nv0) sc[nt][2] = -INFINITY;
+      if (g + 8 >= nv1) sc[nt][3] = -INFINITY;
+    }
+    float mx0 = fmaxf(sc[nt][0], sc[nt][2]);
+    float mx1 = fmaxf(sc[nt][1], sc[nt][3]);
+#pragma unroll
+    for (int off = 4; off <= 16; off <<= 1) {
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+    }
+    m_new[nt][0] = fmaxf(st.m[nt][0], mx0);
+    m_new[nt][1] = fmaxf(st.m[nt][1], mx1);
+    grew = grew || (m_new[nt][0] > st.m[nt][0]) || (m_new[nt][1] > st.m[nt][1]);
+  }
+  if (__any_sync(0xffffffffu, grew)) {
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const float f0 = ex2(st.m[nt][0] - m_new[nt][0]);
+      const float f1 = ex2(st.m[nt][1] - m_new[nt][1]);
+      st.l[nt][0] *= f0;
+      st.l[nt][1] *= f1;
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt) {
+        st.acc[nt][mt][0] *= f0;
+        st.acc[nt][mt][1] *= f1;
+        st.acc[nt][mt][2] *= f0;
+        st.acc[nt][mt][3] *= f1;
+      }
+      st.m[nt][0] = m_new[nt][0];
+      st.m[nt][1] = m_new[nt][1];
+    }
+  }
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    const __half2 lo = __floats2half2_rn(ex2(sc[nt][0] - st.m[nt][0]), ex2(sc[nt][1] - st.m[nt][1]));  // token g
+    const __half2 hi = __floats2half2_rn(ex2(sc[nt][2] - st.m[nt][0]), ex2(sc[nt][3] - st.m[nt][1]));  // token g+8
+    // the denominator sums exactly the probabilities the tensor core will see
+    const float2 flo = __half22float2(lo), fhi = __half22float2(hi);
+    st.l[nt][0] += flo.x + fhi.x;
+    st.l[nt][1] += flo.y + fhi.y;
+    pb[nt][0] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&lo));  // column g : tokens 2t, 2t+1
+    pb[nt][1] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&hi));  // column g : tokens 2t+8, 2t+9
+  }
+
+  // ---- O^T += V^T . P^T
+#pragma unroll
+  for (int c2 = 0; c2 < 4; ++c2) {
+    uint32_t r[4];   // transposed: this thread gets, per matrix, {token 2t: dims 2g, 2g+1 | token 2t+1: dims 2g, 2g+1}
+    ldsm_x4_trans(r, vt + row_off + (uint32_t((2 * c2 + csel) ^ (row & 7)) << 4));
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      uint32_t a[4];
+      cvt_e4m3x4(byte_perm_3120(r[2 * half]), a[0], a[1]);      // dim 2g | dim 2g+1 : tokens 2t, 2t+1
+      cvt_e4m3x4(byte_perm_3120(r[2 * half + 1]), a[2], a[3]);  //                    tokens 2t+8, 2t+9
+      const int mt = 2 * c2 + half;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) mma_f16(st.acc[nt][mt], a, pb[nt][0], pb[nt][1]);
+    }
+  }
+}
+
 // A warp's unit result -> shared memory: stats m, l per head and O as [head][dim] fp32.
-template <int D, int NT>
+// kPairDims: accumulator rows (g, g+8) of a 16-dim chunk hold dims (2g, 2g+1) instead of (g, g+8).
+template <int D, int NT, bool kPairDims = false>
 __device__ __forceinline__ void stage_warp_result(WarpAcc<D, NT>& st, float* o_sm, float* m_sm, float* l_sm, int lane) {
   const int g = lane >> 2, t = lane & 3;
 #pragma unroll
@@ -363,11 +538,12 @@ __device__ __forceinline__ void stage_warp_result(WarpAcc<D, NT>& st, float* o_s
 #pragma unroll
     for (int mt = 0; mt < D / 16; ++mt) {
       const int h0 = nt * 8 + 2 * t;
-      const int d0 = mt * 16 + g;
+      const int d0 = mt * 16 + (kPairDims ? 2 * g : g);
+      constexpr int kStep = kPairDims ? 1 : 8;
       o_sm[h0 * D + d0] = st.acc[nt][mt][0];
       o_sm[(h0 + 1) * D + d0] = st.acc[nt][mt][1];
-      o_sm[h0 * D + d0 + 8] = st.acc[nt][mt][2];
-      o_sm[(h0 + 1) * D + d0 + 8] = st.acc[nt][mt][3];
+      o_sm[h0 * D + d0 + kStep] = st.acc[nt][mt][2];
+      o_sm[(h0 + 1) * D + d0 + kStep] = st.acc[nt][mt][3];
     }
   }
 }
@@ -392,7 +568,7 @@ __device__ __forceinline__ void merge_and_write(const DecodeParams& p, const Uni
       num += f * o_sm[w * o_stride + h * D + dim];
       den += f * l_sm[w * NT * 8 + h];
     }
-    const float o = (den > 0.f) ? num / den : 0.f;   // a query token that sees nothing of this unit
+    const float o = (den > 0.f) ? num / den * p.v_scale : 0.f;   // den = 0: a query token that sees nothing of this unit
     const int64_t head = col_row(p, u.kvh, h);
     if (u.slot < 0) {
       p.out[(int64_t(u.b) * p.num_q_heads + head) * D + dim] = __float2bfloat16_rn(o);
@@ -441,9 +617,9 @@ __global__ void wait_timeout_selftest_kernel(uint32_t* error_word, uint32_t trie
   if (!dev::mbar_wait(b, 0, tries) && threadIdx.x == 0) atomicOr(error_word, LIBRA_DEV_ERR_WAIT_TIMEOUT);
 }
 
-template <int D, int NW, int STAGES>
+template <int D, int NW, int STAGES, int EB = 2>   // EB: bytes per cache element
 struct DecodeSmem {
-  static constexpr int kTileBytes = 16 * D * 2;           // one page of one head: K or V
+  static constexpr int kTileBytes = 16 * D * EB;          // one page of one head: K or V
   static constexpr int kStageBytes = 2 * kTileBytes;      // K then V
   static constexpr int kWarpBytes = STAGES * kStageBytes;
   static constexpr int kRingBytes = NW * kWarpBytes;
@@ -455,13 +631,15 @@ struct DecodeSmem {
 // D: head_dim (64 | 128); NT: 8-wide head tiles (1: G <= 8, 2: G <= 16); NW warps; STAGES per warp.
 // kLoadsOnly: measurement build of the same kernel - same plan, page walk and copies, but each staged page
 // is only touched (one shared-memory word per lane) instead of computed on; `out` gets meaningless values.
-template <int D, int NT, int NW, int STAGES, bool kLoadsOnly = false>
+// kFp8: the pools hold E4M3 codes (head_dim 128 only); tiles are half as large, the page math is process_page_fp8.
+template <int D, int NT, int NW, int STAGES, bool kLoadsOnly = false, bool kFp8 = false>
 __global__ void __launch_bounds__(NW * 32)
 decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
               const __grid_constant__ DecodeParams p, const __grid_constant__ ParamPlan pp) {
   using namespace dev;
-  using SM = DecodeSmem<D, NW, STAGES>;
-  constexpr int NH = D / 64;   // 128-byte column blocks of a row
+  using SM = DecodeSmem<D, NW, STAGES, kFp8 ? 1 : 2>;
+  static_assert(!kFp8 || D == 128, "the 8-bit path is written for head_dim 128");
+  constexpr int NH = kFp8 ? 1 : D / 64;   // 128-byte column blocks of a row
   static_assert(NT * 8 * D * 4 <= SM::kWarpBytes, "epilogue staging must fit in the warp's ring");
 
   extern __shared__ uint8_t smem_raw[];
@@ -524,7 +702,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   const int len_dev = __ldg(p.seq_lens + u.b);
 
   uint32_t qf[NT][D / 16][2];
-  load_q_frags<D, NT>(qf, p, u.b, kvh, lane);
+  if constexpr (kFp8) load_q_frags_fp8<NT>(qf, p, u.b, kvh, lane);
+  else load_q_frags<D, NT>(qf, p, u.b, kvh, lane);
   // query token i stops seeing the cache q_len - 1 - i tokens before its end; this thread's columns:
   int cut[NT][2];
 #pragma unroll
@@ -585,6 +764,9 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
       const uint32_t* words = reinterpret_cast<const uint32_t*>(my_ring + s * SM::kStageBytes);
       st.l[0][0] += float((words[lane * 16] ^ words[SM::kTileBytes / 4 + lane * 16]) & 0xffu);
       st.m[0][0] = 0.f;
+    } else if constexpr (kFp8) {
+      process_page_fp8<NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes, u.kv_end - tok0,
+                           p.scale_log2, lane, common_end - tok0, len_dev - tok0, cut);
     } else {
     if (p.k_new != nullptr && u.chunk_j == u.n_chunks - 1 && u.kv_end - tok0 <= 16) {
       // this page holds the sequence's newest token: its K and V rows come from k_new / v_new.  The copy
@@ -635,7 +817,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 
   // ---- stage (m, l, O) of this warp in its own, now idle, ring; merge the warps; write
   __syncwarp();
-  stage_warp_result<D, NT>(st, reinterpret_cast<float*>(my_ring), stat_m[warp], stat_l[warp], lane);
+  stage_warp_result<D, NT, kFp8>(st, reinterpret_cast<float*>(my_ring), stat_m[warp], stat_l[warp], lane);
   __syncthreads();
   merge_and_write<D, NT, NW>(p, u, reinterpret_cast<const float*>(ring), SM::kWarpBytes / 4, &stat_m[0][0], &stat_l[0][0],
                              threadIdx.x, NW * 32);

@@ -72,6 +72,32 @@ const DecodeKernelFn kLoadsOnlyFn[2][2] = {{libra::decode_kernel<64, 1, kLoadsOn
 const int kLoadsOnlySmem[2] = {libra::DecodeSmem<64, kLoadsOnlyWarps, kLoadsOnlyStages>::kDynamicBytes,
                                libra::DecodeSmem<128, kLoadsOnlyWarps, kLoadsOnlyStages>::kDynamicBytes};
 
+// 8-bit (E4M3) cache, head_dim 128: block shapes compiled in.  Half the bytes per tile leave half the time per tile,
+// and two warps per scheduler cannot hide the conversion -> mma -> softmax chain in it: 16 warps x 3 stages of
+// 4 KB is the default where the registers allow it (one column tile), 8 x 6 otherwise.  fn[loads only][NT - 1]
+struct Fp8Variant {
+  int warps, stages;
+  DecodeKernelFn fn[2][2];
+  int smem;
+};
+template <int NW, int ST>
+Fp8Variant make_fp8_variant() {
+  Fp8Variant v;
+  v.warps = NW;
+  v.stages = ST;
+  v.fn[0][0] = libra::decode_kernel<128, 1, NW, ST, false, true>;
+  v.fn[0][1] = libra::decode_kernel<128, 2, NW, ST, false, true>;
+  v.fn[1][0] = libra::decode_kernel<128, 1, NW, ST, true, true>;
+  v.fn[1][1] = libra::decode_kernel<128, 2, NW, ST, true, true>;
+  v.smem = libra::DecodeSmem<128, NW, ST, 1>::kDynamicBytes;
+  return v;
+}
+const std::vector<Fp8Variant>& fp8_variants() {
+  static const std::vector<Fp8Variant> v = {make_fp8_variant<16, 3>(), make_fp8_variant<8, 6>(), make_fp8_variant<16, 2>(),
+                                            make_fp8_variant<8, 4>()};
+  return v;
+}
+
 constexpr int kMaxProfiledCalls = 4096;
 
 struct DeviceGuard {
@@ -104,6 +130,9 @@ struct libra_handle_s {
   int last_cuda_error = 0;
   int variant = 0;
   int max_q_len = 1;        // query tokens per sequence the workspace is laid out for
+  bool fp8 = false;         // the pools hold E4M3 codes; keys and values are code * k_scale / v_scale
+  float k_scale = 1.f, v_scale = 1.f;
+  int fp8_variant = -1;     // -1: chosen by the number of column tiles
   EncodeTiledFn encode = nullptr;
 
   // workspace layout: control words | arrival counters | partial LSE | partial O | oversized plans
@@ -191,19 +220,20 @@ int encode_pool_map(libra_handle_t h, const void* base, CUtensorMap* map, int* p
                  {h->stride_head, h->cfg.num_kv_heads, 1u, 1},
                  {h->stride_page, h->cfg.num_pages, 1u, 2}};
   std::stable_sort(dims, dims + 3, [](const Dim& a, const Dim& b) { return a.stride < b.stride; });
+  const int eb = h->fp8 ? 1 : 2;   // bytes per element; a box row is 128 bytes either way
   cuuint64_t gdim[4] = {cuuint64_t(h->cfg.head_dim), 0, 0, 0};
   cuuint64_t gstride[3];
-  cuuint32_t box[4] = {64, 0, 0, 0};
+  cuuint32_t box[4] = {cuuint32_t(128 / eb), 0, 0, 0};
   cuuint32_t estride[4] = {1, 1, 1, 1};
   for (int i = 0; i < 3; ++i) {
     gdim[i + 1] = cuuint64_t(dims[i].size);
-    gstride[i] = cuuint64_t(dims[i].stride) * 2;
+    gstride[i] = cuuint64_t(dims[i].stride) * eb;
     box[i + 1] = dims[i].box;
     if (dims[i].kind == 0) *pos_token = i + 1;
     if (dims[i].kind == 1) *pos_head = i + 1;
     if (dims[i].kind == 2) *pos_page = i + 1;
   }
-  CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gdim, gstride, box, estride,
+  CUresult r = h->encode(map, h->fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gdim, gstride, box, estride,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
@@ -406,6 +436,13 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
       e = cudaFuncSetAttribute(reinterpret_cast<const void*>(kLoadsOnlyFn[di >> 1][di & 1]),
                                cudaFuncAttributeMaxDynamicSharedMemorySize, kLoadsOnlySmem[di >> 1]);
       if (e != cudaSuccess) break;
+    }
+    if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
+    for (const Fp8Variant& fv : fp8_variants()) {
+      for (int di = 0; di < 4 && e == cudaSuccess; ++di) {
+        e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fv.fn[di >> 1][di & 1]),
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, fv.smem);
+      }
     }
     if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
     e = cudaFuncSetAttribute(reinterpret_cast<const void*>(libra::plan_kernel), cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -663,8 +700,34 @@ int libra_set_max_query_tokens(libra_handle_t h, int32_t max_q_len) {
   return LIBRA_OK;
 }
 
+int libra_set_kv_dtype(libra_handle_t h, int32_t dtype, float k_scale, float v_scale) {
+  if (!h || (dtype != LIBRA_KV_BF16 && dtype != LIBRA_KV_E4M3)) return LIBRA_INVALID_ARGUMENT;
+  if (dtype == LIBRA_KV_E4M3) {
+    if (!(k_scale > 0.f) || !(v_scale > 0.f) || !std::isfinite(k_scale) || !std::isfinite(v_scale)) return LIBRA_INVALID_ARGUMENT;
+    if (h->cfg.head_dim != 128) return LIBRA_UNSUPPORTED_SHAPE;
+    // strides are in elements = bytes here: the tiled copies need 16-byte multiples
+    if (h->stride_page % 16 || h->stride_head % 16 || h->stride_token % 16) return LIBRA_INVALID_ARGUMENT;
+  }
+  h->fp8 = (dtype == LIBRA_KV_E4M3);
+  h->fp8_variant = -1;
+  h->k_scale = h->fp8 ? k_scale : 1.f;
+  h->v_scale = h->fp8 ? v_scale : 1.f;
+  for (int i = 0; i < libra_handle_s::kMapCache; ++i) h->maps[i].k_ptr = h->maps[i].v_ptr = nullptr;  // maps depend on the type
+  return LIBRA_OK;
+}
+
 int libra_set_variant(libra_handle_t h, int32_t warps, int32_t stages) {
   if (!h) return LIBRA_INVALID_ARGUMENT;
+  if (h->fp8) {
+    const std::vector<Fp8Variant>& fv = fp8_variants();
+    for (size_t i = 0; i < fv.size(); ++i) {
+      if (fv[i].warps == warps && fv[i].stages == stages) {
+        h->fp8_variant = int(i);
+        return LIBRA_OK;
+      }
+    }
+    return LIBRA_UNSUPPORTED_SHAPE;
+  }
   const std::vector<Variant>& vs = variants();
   const int di = (h->cfg.head_dim == 128) ? 1 : 0;
   const int ni = (h->group > 8) ? 1 : 0;
@@ -693,6 +756,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     return LIBRA_INVALID_ARGUMENT;
   }
   if (q_len < 1 || q_len > h->max_q_len || (q_len > 1 && k_new)) return LIBRA_INVALID_ARGUMENT;
+  if (h->fp8 && k_new) return LIBRA_UNSUPPORTED_SHAPE;   // the fused append writes bf16 rows
   if (!h->planned) return LIBRA_NOT_PLANNED;
   DeviceGuard guard(h->cfg.device);
   if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
@@ -761,7 +825,8 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     p.hq = h->cfg.num_q_heads;
     p.cols = q_len * h->group;
     p.block_table_ld = h->cfg.block_table_ld;
-    p.scale_log2 = h->scale_log2;
+    p.scale_log2 = h->scale_log2 * h->k_scale;
+    p.v_scale = h->fp8 ? h->v_scale : 1.f;
     p.pos_head = h->pos_head;
     p.pos_page = h->pos_page;
     p.pos_token = h->pos_token;
@@ -782,15 +847,22 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     // resident while that kernel drains; inside, they wait for it to finish before reading any input
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(grid);
+    DecodeKernelFn fn = loads_only ? kLoadsOnlyFn[di][ni] : v.fn[di][ni];
     lc.blockDim = dim3(unsigned((loads_only ? kLoadsOnlyWarps : v.warps) * 32));
     lc.dynamicSmemBytes = size_t(loads_only ? kLoadsOnlySmem[di] : v.smem[di][ni]);
+    if (h->fp8) {
+      const Fp8Variant& fv = fp8_variants()[h->fp8_variant >= 0 ? h->fp8_variant : ni];   // [0] = 16 x 3, [1] = 8 x 6
+      fn = fv.fn[loads_only ? 1 : 0][ni];
+      lc.blockDim = dim3(unsigned(fv.warps * 32));
+      lc.dynamicSmemBytes = size_t(fv.smem);
+    }
     lc.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = h->pdl ? 1 : 0;
-    LIBRA_CUDA_TRY(h, cudaLaunchKernelEx(&lc, loads_only ? kLoadsOnlyFn[di][ni] : v.fn[di][ni], pm->map_k, pm->map_v, p, h->pp));
+    LIBRA_CUDA_TRY(h, cudaLaunchKernelEx(&lc, fn, pm->map_k, pm->map_v, p, h->pp));
     ++h->launches;
   }
   if (ev) LIBRA_CUDA_TRY(h, cudaEventRecord(ev[1], st));
@@ -864,6 +936,7 @@ int libra_decode_attn_host(libra_handle_t h, const void* q_host, const void* k_p
       !staging_dev || batch <= 0) {
     return LIBRA_INVALID_ARGUMENT;
   }
+  if (h->fp8) return LIBRA_UNSUPPORTED_SHAPE;   // the host-buffer path is sized for bf16 pools
   if (reinterpret_cast<uintptr_t>(staging_dev) % 256 != 0) return LIBRA_INVALID_ARGUMENT;
   size_t need = 0;
   int rc = libra_host_staging_size(h, batch, &need);
@@ -945,6 +1018,7 @@ namespace {
 int kv_move_impl(libra_handle_t h, bool gather, void* k_pages, void* v_pages, void* k_dense, void* v_dense,
                  const int32_t* block_table, const int32_t* seq_lens, const int64_t* token_offsets, int32_t batch,
                  int32_t max_seq_len, int32_t head_begin, int32_t head_count, void* error_word_dev, void* stream) {
+  if (h && h->fp8) return LIBRA_UNSUPPORTED_SHAPE;   // the move kernels are written for bf16 rows
   if (!h || !k_pages || !v_pages || !k_dense || !v_dense || !block_table || !seq_lens || !token_offsets ||
       !error_word_dev) {
     return LIBRA_INVALID_ARGUMENT;

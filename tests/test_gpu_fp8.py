@@ -1,0 +1,184 @@
+"""GPU parity of the decode step over an E4M3 KV cache (libra_set_kv_dtype) against the float64 CPU oracle,
+through the C ABI, with the same two gates as the bf16 cache."""
+import numpy as np
+import pytest
+
+from oracle import attention_oracle as O
+from paper_2606_03077_b200 import workloads as W
+
+import gates
+import gpu_harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def check(got, ref, what=""):
+    assert np.all(np.isfinite(got)), f"{what}: non-finite output (unwritten row?)"
+    assert gates.stated_violations(got, ref) == 0, f"{what}: stated gate"
+    assert gates.tight_violations(got, ref) == 0, f"{what}: tight gate, ratio {gates.tight_ratio(got, ref):.2f}"
+
+
+def run_fp8(lib, q, k8, v8, bt, lens, k_scale=1.0, v_scale=1.0, layout="HND", plan=None, fused=None, page_size=16):
+    """q: uint16 [B, Hq, d] or [B, Tq, Hq, d]; k8 / v8: uint8 HND pools.  Returns float32 like q."""
+    import torch
+    dev = torch.device("cuda:0")
+    multi = q.ndim == 4
+    B, Hq, d = q.shape[0], q.shape[-2], q.shape[-1]
+    Tq = q.shape[1] if multi else 1
+    Hkv = k8.shape[1]
+    strides = (0, 0, 0)
+    if layout == "NHD":
+        k8 = np.ascontiguousarray(k8.transpose(0, 2, 1, 3))
+        v8 = np.ascontiguousarray(v8.transpose(0, 2, 1, 3))
+        strides = (page_size * Hkv * d, d, Hkv * d)
+    h = lib.Handle(Hq, Hkv, d, k8.shape[0], max(B, 1), bt.shape[1], page_size=page_size, kv_strides=strides, plan=plan)
+    h.set_kv_dtype(lib.KV_E4M3, k_scale, v_scale)
+    if fused is not None:
+        h.set_combine_mode(fused)
+    if multi:
+        h.set_max_query_tokens(Tq)
+    ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=dev)
+    qd, btd = H.to_dev(q, dev), H.to_dev(bt, dev)
+    kd, vd = torch.from_numpy(k8).to(dev), torch.from_numpy(v8).to(dev)
+    lens_dev = torch.from_numpy(np.ascontiguousarray(lens, dtype=np.int32)).to(dev)
+    out = torch.full(q.shape, H.CANARY, dtype=torch.int16, device=dev)
+    st = torch.cuda.current_stream().cuda_stream
+    h.plan(np.asarray(lens, dtype=np.int32), ws.data_ptr(), ws.numel(), st)
+    if multi:
+        h.decode_attn_multi(qd.data_ptr(), Tq, kd.data_ptr(), vd.data_ptr(), btd.data_ptr(), lens_dev.data_ptr(),
+                            out.data_ptr(), st)
+    else:
+        h.decode_attn(qd.data_ptr(), kd.data_ptr(), vd.data_ptr(), btd.data_ptr(), lens_dev.data_ptr(), out.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert h.debug_error_word() == 0
+    res = H.bf16_dev_to_f32(out)
+    h.close()
+    return res
+
+
+def small_plan(lib):
+    return lib.PlanParams(4, 1, 2, 16, 16, 64)
+
+
+CASES = [
+    # (Hq, Hkv, lens)
+    (4, 1, [1, 2, 15, 16, 17, 31, 33]),        # G = 4
+    (8, 2, [255, 256, 257, 1, 700]),
+    (8, 8, [100, 1000]),                       # G = 1
+    (40, 8, [1200, 77, 2049]),                 # G = 5
+    (64, 8, [3000, 5]),                        # G = 8
+    (24, 2, [900, 130]),                       # G = 12: two column tiles
+    (32, 2, [777, 64]),                        # G = 16
+    (6, 2, [0, 40, 0, 300]),                   # empty sequences
+]
+
+
+@pytest.mark.parametrize("layout", ["HND", "NHD"])
+@pytest.mark.parametrize("case", range(len(CASES)))
+def test_shapes_and_tails(lib, case, layout):
+    Hq, Hkv, lens = CASES[case]
+    lens_a, bt, q, k8, v8 = W.random_case_e4m3(600 + case, len(lens), Hq, Hkv, 128, lens)
+    ks, vs = 0.75, 1.5
+    ref, _ = O.paged_decode_attention_fp8(q, k8, v8, bt, lens_a, ks, vs)
+    for plan in (None, small_plan(lib)):
+        got = run_fp8(lib, q, k8, v8, bt, lens_a, ks, vs, layout=layout, plan=plan)
+        check(got, ref, f"case {case} {layout} plan={'default' if plan is None else 'small'}")
+    two = run_fp8(lib, q, k8, v8, bt, lens_a, ks, vs, layout=layout, plan=small_plan(lib), fused=0)
+    assert np.array_equal(two, got)
+
+
+def test_length_one_is_the_scaled_value_row_exactly(lib):
+    lens_a, bt, q, k8, v8 = W.random_case_e4m3(620, 3, 8, 2, 128, [1, 1, 1])
+    got = run_fp8(lib, q, k8, v8, bt, lens_a, k_scale=3.0, v_scale=0.25)
+    for b in range(3):
+        for h in range(8):
+            want = 0.25 * O.e4m3_to_f64(v8[bt[b, 0], h // 4, 0])      # a power-of-two scale keeps it a bf16 value
+            assert np.array_equal(got[b, h].astype(np.float64), want)
+
+
+def test_every_code_and_every_dim_lands_where_it_should(lib):
+    # one-hot keys pick single tokens; their value rows hold the 254 finite codes spread over the 128 dims, so a
+    # fragment delivered to the wrong dim, or a code converted wrongly, shows up exactly
+    import math
+    L, d = 40, 128
+    lens_a, bt, _, k8, v8 = W.random_case_e4m3(621, 1, 2, 1, d, [L])
+    finite = np.array([c for c in range(256) if c not in (0x7F, 0xFF)], dtype=np.uint8)
+    for t in range(L):
+        v8[bt[0, t // 16], 0, t % 16] = finite[(np.arange(d) * 2 + 7 * t) % len(finite)]
+    # query c e_j against keys 8 e_j at one token: score 8 c k_scale / sqrt(128) >= 150 with c = 256
+    for tstar, j in ((0, 0), (15, 1), (16, 2), (17, 3), (31, 64), (39, 127), (22, 77)):
+        k8[bt[0], 0] = 0
+        k8[bt[0, tstar // 16], 0, tstar % 16, j] = 0x50          # code of 8.0
+        qrow = np.zeros(d, dtype=np.float32)
+        qrow[j] = 256.0
+        q = np.broadcast_to(W.f32_to_bf16_bits(qrow), (1, 2, d)).copy()
+        assert 8 * 256 / math.sqrt(d) > 150
+        for plan in (None, small_plan(lib)):
+            got = run_fp8(lib, q, k8, v8, bt, lens_a, plan=plan)
+            want = O.e4m3_to_f64(v8[bt[0, tstar // 16], 0, tstar % 16])
+            assert np.array_equal(got[0, 0].astype(np.float64), want), (tstar, j)
+            assert np.array_equal(got[0, 1], got[0, 0])
+
+
+def test_larger_pages(lib):
+    lens = [1, 16, 17, 31, 32, 33, 700, 2049, 0]
+    lens_a, bt, q, k8, v8 = W.random_case_e4m3(622, len(lens), 8, 2, 128, lens, page_size=32)
+    ref, _ = O.paged_decode_attention_fp8(q, k8, v8, bt, lens_a)
+    for layout in ("HND", "NHD"):
+        for plan in (None, lib.PlanParams(4, 1, 2, 32, 32, 64)):
+            got = run_fp8(lib, q, k8, v8, bt, lens_a, layout=layout, plan=plan, page_size=32)
+            check(got, ref, f"page 32 {layout}")
+
+
+def test_several_query_tokens_over_an_8bit_cache(lib):
+    # row i of the multi-token step = the single-token definition at length L - Tq + 1 + i
+    Tq = 3
+    lens = [3, 17, 300, 1030, 2]
+    lens_a, bt, _, k8, v8 = W.random_case_e4m3(623, len(lens), 8, 2, 128, lens)
+    rng = np.random.default_rng(624)
+    q = W.f32_to_bf16_bits(rng.standard_normal((len(lens), Tq, 8, 128)).astype(np.float32))
+    for plan in (None, small_plan(lib)):
+        got = run_fp8(lib, q, k8, v8, bt, lens_a, 0.5, 2.0, plan=plan)
+        for i in range(Tq):
+            ref, _ = O.paged_decode_attention_fp8(q[:, i], k8, v8, bt, np.maximum(lens_a - Tq + 1 + i, 0), 0.5, 2.0)
+            check(got[:, i], ref, f"row {i}")
+
+
+def test_split_and_unsplit_agree_and_runs_reproduce(lib):
+    lens_a, bt, q, k8, v8 = W.random_case_e4m3(625, 2, 32, 8, 128, [5000, 900])
+    ref, _ = O.paged_decode_attention_fp8(q, k8, v8, bt, lens_a)
+    one = run_fp8(lib, q, k8, v8, bt, lens_a, plan=lib.PlanParams(148, 1, 1, 256, 512, 1))
+    many = run_fp8(lib, q, k8, v8, bt, lens_a, plan=lib.PlanParams(148, 1, 1, 256, 512, 64))
+    check(one, ref, "unsplit")
+    check(many, ref, "split")
+    again = run_fp8(lib, q, k8, v8, bt, lens_a, plan=lib.PlanParams(148, 1, 1, 256, 512, 64))
+    assert np.array_equal(again, many)
+
+
+def test_what_is_not_supported_says_so(lib):
+    import torch
+    h64 = lib.Handle(4, 1, 64, 64, 4, 8)
+    with pytest.raises(lib.LibraError):
+        h64.set_kv_dtype(lib.KV_E4M3, 1.0, 1.0)           # head_dim 64
+    h64.close()
+    h = lib.Handle(8, 2, 128, 64, 4, 8)
+    for bad in ((0.0, 1.0), (1.0, -1.0), (float("inf"), 1.0), (float("nan"), 1.0)):
+        with pytest.raises(lib.LibraError):
+            h.set_kv_dtype(lib.KV_E4M3, *bad)
+    with pytest.raises(lib.LibraError):
+        h.set_kv_dtype(7, 1.0, 1.0)
+    h.set_kv_dtype(lib.KV_E4M3, 1.0, 1.0)
+    ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device="cuda:0")
+    st = torch.cuda.current_stream().cuda_stream
+    h.plan(np.array([5], dtype=np.int32), ws.data_ptr(), ws.numel(), st)
+    x = torch.zeros(1 << 16, dtype=torch.int16, device="cuda:0")
+    with pytest.raises(lib.LibraError):                   # the fused append writes bf16 rows
+        h.decode_attn_append(x.data_ptr(), x.data_ptr(), x.data_ptr(), x.data_ptr(), x.data_ptr(), x.data_ptr(),
+                             x.data_ptr(), x.data_ptr(), st)
+    h.set_kv_dtype(lib.KV_BF16)                           # and back
+    torch.cuda.synchronize()
+    h.close()
+    odd = lib.Handle(8, 2, 128, 64, 4, 8, kv_strides=(16 * 2 * 136, 16 * 136, 136))   # token stride 136: not a multiple of 16
+    with pytest.raises(lib.LibraError):
+        odd.set_kv_dtype(lib.KV_E4M3, 1.0, 1.0)
+    odd.close()
