@@ -45,7 +45,8 @@ FALLBACK_HBM_GBS = 6650.0
 L2_BYTES_ASSUMED = 126 * 1024 * 1024
 # DRAM bytes (read + write) of one decode-kernel launch on MAIN_WORKLOAD from an ncu capture, see
 # profiles/decode_kernel_lognormal_b64.md (370.62 MB read + 4.10 MB written).
-NCU_DECODE_TRAFFIC_BYTES = 374.7e6
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode launch, from the ncu captures summarised under profiles/
+NCU_DECODE_TRAFFIC_BYTES = {"lognormal_b64": 374.7e6, "straggler_b8": 1078.8e6}
 
 
 # ----------------------------------------------------------------------------- clocks
@@ -661,7 +662,7 @@ def run_libra(args):
     kernel_ms = (elapsed_ms / args.steps) if one_launch_per_step else dec_ms
     achieved = rep.kv_bytes_per_step / (kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_source": peak_src, "traffic": NCU_DECODE_TRAFFIC_BYTES,
+                "frac": achieved / peak, "peak_source": peak_src, "traffic": NCU_DECODE_TRAFFIC_BYTES.get(args.workload),
                 "algorithmic_bytes_per_launch": rep.kv_bytes_per_step, "kernel_us": kernel_ms * 1e3,
                 "timing": ("CUDA events around the timed region, one decode launch per step" if one_launch_per_step
                            else "CUDA event pair around every decode launch"),
@@ -692,10 +693,14 @@ def run_libra(args):
                            "note": "libra_decode_attn_host: q, both KV pools, block table, lengths copied from pinned "
                                    "host memory every step, output copied back"}
             line["e2e_resident_kv"] = e2e_resident_kv_measure(rep, 200)
-        line["ceilings"] = ceilings_measure(rep)
-        line["multi_token"] = [m for m in (multi_token_measure(rep, t) for t in (2, 4)) if m]
-        line["fp8_cache"] = fp8_cache_measure(rep)
-        if args.workload in ("longtail_mix_b256", "straggler_b8"):
+        extras = set(x for x in args.extras.split(",") if x)
+        if "ceilings" in extras:
+            line["ceilings"] = ceilings_measure(rep)
+        if "multi_token" in extras:
+            line["multi_token"] = [m for m in (multi_token_measure(rep, t) for t in (2, 4)) if m]
+        if "fp8_cache" in extras:
+            line["fp8_cache"] = fp8_cache_measure(rep, steps=min(200, max(10, args.steps)))
+        if "kv_migration" in extras and args.workload in ("longtail_mix_b256", "straggler_b8"):
             line["kv_migration"] = kv_migration_measure(rep)
         if not args.no_cpu:
             cb = oracle_baseline(args.workload, k0, v0, rep.q, budget_s=args.cpu_budget)
@@ -765,6 +770,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
+    ap.add_argument("--extras", default="ceilings,multi_token,fp8_cache,kv_migration",
+                    help="side measurements on the main workload at N=1 (comma list; empty = none)")
     ap.add_argument("--variant", default="", help="warps,stages of the decode block (default: the library's)")
     ap.add_argument("--ctas-per-sm", type=int, default=0, help="planner constant (0 = default)")
     ap.add_argument("--items-per-slot", type=int, default=0, help="planner constant (0 = default)")
