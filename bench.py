@@ -704,6 +704,15 @@ def run_libra(args):
         extras = set(x for x in args.extras.split(",") if x)
         if "ceilings" in extras:
             line["ceilings"] = ceilings_measure(rep)
+        if "early_prefetch" in extras:
+            # back-to-back steps with libra_set_early_prefetch: the kernel before each decode launch is the previous
+            # step's decode kernel, which writes only `out` and the workspace, so the promise holds
+            rep.h.set_early_prefetch(True)
+            n = min(args.steps, 1000)
+            ms_e, _ = rep.timed(n, max(3, args.warmup // 2))
+            rep.h.set_early_prefetch(False)
+            line["early_prefetch"] = {"ms_per_step": ms_e / n, "kv_gbs": rep.kv_bytes_per_step / (ms_e / n * 1e-3) / 1e9,
+                                      "steps": n, "note": "optional mode, off in the headline number"}
         if "multi_token" in extras:
             line["multi_token"] = [m for m in (multi_token_measure(rep, t) for t in (2, 4)) if m]
         if "fp8_cache" in extras:
@@ -778,7 +787,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
-    ap.add_argument("--extras", default="ceilings,multi_token,fp8_cache,kv_migration",
+    ap.add_argument("--extras", default="ceilings,early_prefetch,multi_token,fp8_cache,kv_migration",
                     help="side measurements on the main workload at N=1 (comma list; empty = none)")
     ap.add_argument("--variant", default="", help="warps,stages of the decode block (default: the library's)")
     ap.add_argument("--ctas-per-sm", type=int, default=0, help="planner constant (0 = default)")

@@ -174,6 +174,16 @@ int libra_set_variant(libra_handle_t handle, int32_t warps, int32_t stages);
  * and block start-up overlap the predecessor's tail.  on = 0 makes every launch an ordinary one. */
 int libra_set_dependent_launch(libra_handle_t handle, int32_t on);
 
+/* Early prefetch, off by default: a PROMISE by the caller about the kernel that precedes each decode call in the
+ * stream, namely that it writes none of: block_table, seq_lens (device), and the cached K/V rows of any token
+ * other than each sequence's newest q_len tokens (a projection / rotary / cache-write kernel qualifies; a kernel
+ * that moves or rewrites old pages does not).  With the promise, and dependent launch on, a decode block that
+ * becomes resident while that kernel drains walks its block-table row and starts the copies of its first tiles
+ * of old tokens before it waits for that kernel to finish; q, the newest rows, `out` and the workspace are
+ * still touched only afterwards.  Results are bit-identical to the default.  Applies to plans that travel in
+ * the kernel parameters (host plans of up to 768 entries); otherwise the setting has no effect. */
+int libra_set_early_prefetch(libra_handle_t handle, int32_t on);
+
 /* Where step C runs.  mode 1 (default): inside the decode kernel, by the block that publishes the last
  * partial result of a split sequence (one launch per step).  mode 0: as a separate combine kernel after
  * the decode kernel (two launches; the second is a programmatic dependent of the first).  The merge code

@@ -60,6 +60,7 @@ SIGNATURES = {
     "libra_set_variant": (C.c_int, [_vp, C.c_int32, C.c_int32]),
     "libra_set_dependent_launch": (C.c_int, [_vp, C.c_int32]),
     "libra_set_max_query_tokens": (C.c_int, [_vp, C.c_int32]),
+    "libra_set_early_prefetch": (C.c_int, [_vp, C.c_int32]),
     "libra_set_kv_dtype": (C.c_int, [_vp, C.c_int32, C.c_float, C.c_float]),
     "libra_decode_attn_multi": (C.c_int, [_vp, _vp, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_debug_stream_read": (C.c_int, [_vp, _vp, C.c_size_t, _vp]),
@@ -285,6 +286,9 @@ class Handle:
 
     def set_kv_dtype(self, dtype: int, k_scale: float = 1.0, v_scale: float = 1.0) -> None:
         _check(lib.libra_set_kv_dtype(self._h, dtype, k_scale, v_scale), "libra_set_kv_dtype")
+
+    def set_early_prefetch(self, on: bool) -> None:
+        _check(lib.libra_set_early_prefetch(self._h, 1 if on else 0), "libra_set_early_prefetch")
 
     def set_max_query_tokens(self, max_q_len: int) -> None:
         _check(lib.libra_set_max_query_tokens(self._h, max_q_len), "libra_set_max_query_tokens")

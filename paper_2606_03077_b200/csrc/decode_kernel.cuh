@@ -63,6 +63,7 @@ struct DecodeParams {
   int32_t num_units;      // work items x KV heads
   int32_t num_empty;      // empty sequences whose output row this launch zeroes
   int32_t fused_combine;  // 1: the last block of a split sequence merges its partials (step C) itself
+  int32_t early_prefetch; // 1: block-table walk and first copies of old tokens start before the grid dependency wait
   // KV append fused into the step (null k_new = off): the current token's K and V rows, bf16 [B, Hkv, D],
   // are written into slot (L_b - 1) % 16 of the sequence's last page, in the pools and in the staged tile
   const __nv_bfloat16* k_new;
@@ -666,7 +667,13 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   __syncwarp();
   // Up to here nothing was read that an earlier kernel in the stream could have written, so when this
   // launch overlaps the tail of its predecessor the block is resident and set up by the time that ends.
-  grid_dependency_wait();
+  // With early prefetch (a promise by the caller that the preceding kernel writes neither the block table, the
+  // lengths nor any cached row except those of each sequence's newest q_len tokens) the block goes further
+  // before it waits: it walks its block-table row and starts the copies of its first tiles of old tokens.
+  // Only a plan that travels in the kernel parameters allows it (a plan in device memory may itself have been
+  // written by the preceding kernel).
+  const bool early = p.early_prefetch != 0 && p.entries == nullptr && p.dev_counts == nullptr;
+  if (!early) grid_dependency_wait();
 
   // the plan lives in the kernel parameters unless it was too large for them (plain loads: the
   // pointer may address parameter space)
@@ -678,6 +685,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     num_units = num_items * p.num_kv_heads;
   }
   if (int(blockIdx.x) >= num_units) {
+    if (early) grid_dependency_wait();   // `out` may still be read by the kernel before this one
     if (int(blockIdx.x) - num_units < num_empty) {
       zero_empty_row<D>(p, entries, num_items, int(blockIdx.x) - num_units, threadIdx.x, NW * 32);
     }
@@ -701,9 +709,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   int32_t ids_nxt = load_ids(1);
   const int len_dev = __ldg(p.seq_lens + u.b);
 
-  uint32_t qf[NT][D / 16][2];
-  if constexpr (kFp8) load_q_frags_fp8<NT>(qf, p, u.b, kvh, lane);
-  else load_q_frags<D, NT>(qf, p, u.b, kvh, lane);
   // query token i stops seeing the cache q_len - 1 - i tokens before its end; this thread's columns:
   int cut[NT][2];
 #pragma unroll
@@ -743,10 +748,22 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   WarpAcc<D, NT> st;
   st.reset();
 
-  {
-    const int pre = n_it < STAGES ? n_it : STAGES;
-    for (int j = 0; j < pre; ++j) issue(j, j);
+  const int pre = n_it < STAGES ? n_it : STAGES;
+  int issued = 0;
+  if (early) {
+    // tokens [0, safe_end) were in the cache before the preceding kernel ran; with the fused append the pools are
+    // written by this kernel only, so every tile qualifies (the newest row is patched in after its tile lands)
+    const int safe_end = (p.k_new != nullptr) ? len_dev : len_dev - p.q_len;
+    while (issued < pre && u.kv_begin + ((warp + issued * NW) << 4) + 16 <= safe_end) {
+      issue(issued, issued);
+      ++issued;
+    }
+    grid_dependency_wait();
   }
+  uint32_t qf[NT][D / 16][2];
+  if constexpr (kFp8) load_q_frags_fp8<NT>(qf, p, u.b, kvh, lane);
+  else load_q_frags<D, NT>(qf, p, u.b, kvh, lane);
+  for (int j = issued; j < pre; ++j) issue(j, j);
   if (threadIdx.x == 0) check_planned_length(p, u, len_dev);
 
   bool timed_out = false;

@@ -141,6 +141,7 @@ struct libra_handle_s {
   void* clean_workspace = nullptr;  // workspace whose control words and counters are known to be zero
   int combine_mode = 1;     // 0: separate kernel, 1: inside the decode kernel
   bool pdl = true;          // programmatic dependent launches (decode after its predecessor, combine after decode)
+  bool early_prefetch = false;  // the caller's promise about the preceding kernel (libra_set_early_prefetch)
 
   // pinned staging for uploads of plans too large for the kernel parameters
   int32_t* staging[2] = {nullptr, nullptr};
@@ -716,6 +717,12 @@ int libra_set_kv_dtype(libra_handle_t h, int32_t dtype, float k_scale, float v_s
   return LIBRA_OK;
 }
 
+int libra_set_early_prefetch(libra_handle_t h, int32_t on) {
+  if (!h || (on != 0 && on != 1)) return LIBRA_INVALID_ARGUMENT;
+  h->early_prefetch = (on == 1);
+  return LIBRA_OK;
+}
+
 int libra_set_variant(libra_handle_t h, int32_t warps, int32_t stages) {
   if (!h) return LIBRA_INVALID_ARGUMENT;
   if (h->fp8) {
@@ -835,6 +842,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     p.num_units = n_units;
     p.num_empty = n_empty;
     p.fused_combine = fused ? 1 : 0;
+    p.early_prefetch = (h->early_prefetch && h->pdl) ? 1 : 0;
     p.k_new = static_cast<const __nv_bfloat16*>(k_new);
     p.v_new = static_cast<const __nv_bfloat16*>(v_new);
     p.k_pool = static_cast<__nv_bfloat16*>(const_cast<void*>(k_pages));

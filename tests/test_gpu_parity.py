@@ -345,3 +345,53 @@ def test_host_buffer_entry_point(lib):
     got = hout.view(torch.bfloat16).float().numpy()
     check(got, ref, "host entry point")
     h.close()
+
+
+def test_early_prefetch_is_bit_identical_behind_a_cache_write_kernel(lib):
+    """Steps issued back to back, each preceded by kernels that write q and the newest token's K/V rows (what the
+    promise of libra_set_early_prefetch allows the preceding kernel to do): same bits as the default."""
+    import torch
+    dev = torch.device("cuda:0")
+    lens = [2500, 300, 17, 4100, 1, 16, 33]
+    B, Hq, Hkv, d = len(lens), 32, 8, 128
+    lens_a, bt, q, k, v = W.random_case(71, B, Hq, Hkv, d, lens)
+    rng = np.random.default_rng(72)
+    steps = 4
+    new_k = [bits(rng.standard_normal((B, Hkv, d)).astype(np.float32)) for _ in range(steps)]
+    new_v = [bits(rng.standard_normal((B, Hkv, d)).astype(np.float32)) for _ in range(steps)]
+    new_q = [bits(rng.standard_normal((B, Hq, d)).astype(np.float32)) for _ in range(steps)]
+    pages = torch.tensor([bt[b, (lens_a[b] - 1) // 16] for b in range(B)], dtype=torch.long, device=dev)
+    slots = torch.tensor([(lens_a[b] - 1) % 16 for b in range(B)], dtype=torch.long, device=dev)
+    results = {}
+    for early in (False, True):
+        r = H.Runner(lib, Hq, Hkv, d, k.shape[0], B, bt.shape[1], plan=lib.PlanParams(148, 1, 1, 256, 512, 64))
+        r.h.set_early_prefetch(early)
+        kd, vd, btd = H.to_dev(k, dev), H.to_dev(v, dev), H.to_dev(bt, dev)
+        qd = torch.zeros((B, Hq, d), dtype=torch.int16, device=dev)
+        lens_dev = torch.from_numpy(lens_a).to(dev)
+        nk = [H.to_dev(x, dev) for x in new_k]
+        nv = [H.to_dev(x, dev) for x in new_v]
+        nq = [H.to_dev(x, dev) for x in new_q]
+        outs = [torch.zeros((B, Hq, d), dtype=torch.int16, device=dev) for _ in range(steps)]
+        st = torch.cuda.current_stream().cuda_stream
+        torch.cuda.synchronize()
+        for i in range(steps):            # no synchronisation inside: the kernels queue up behind each other
+            kd[pages, :, slots, :] = nk[i]        # index_put kernels: the newest token's rows
+            vd[pages, :, slots, :] = nv[i]
+            qd.copy_(nq[i])                       # a device-to-device copy kernel
+            r.h.plan(lens_a, r.ws.data_ptr(), r.ws.numel(), st)
+            r.h.decode_attn(qd.data_ptr(), kd.data_ptr(), vd.data_ptr(), btd.data_ptr(), lens_dev.data_ptr(),
+                            outs[i].data_ptr(), st)
+        torch.cuda.synchronize()
+        assert r.h.debug_error_word() == 0
+        results[early] = [H.bf16_dev_to_f32(o) for o in outs]
+        r.h.close()
+    for i in range(steps):
+        assert np.array_equal(results[True][i], results[False][i]), f"step {i}"
+    # and the last step against the oracle on the final pools
+    kk, vv = k.copy(), v.copy()
+    for b in range(B):
+        kk[bt[b, (lens_a[b] - 1) // 16], :, (lens_a[b] - 1) % 16] = new_k[-1][b]
+        vv[bt[b, (lens_a[b] - 1) // 16], :, (lens_a[b] - 1) % 16] = new_v[-1][b]
+    ref, _ = O.paged_decode_attention(new_q[-1], kk, vv, bt, lens_a)
+    check(results[True][-1], ref, "early prefetch, last step")
