@@ -154,8 +154,9 @@ int libra_set_max_query_tokens(libra_handle_t handle, int32_t max_q_len);
  * attention is the same definition on those keys and values, q and out stay bf16.  The strides given at
  * creation keep their meaning (elements, now bytes) and must be multiples of 16; head_dim must be 128
  * (UNSUPPORTED_SHAPE otherwise); k_scale and v_scale must be positive and finite (ignored for BF16).
- * Halving the bytes per cached token halves what the step has to read.  With E4M3 pools
- * libra_decode_attn_append, libra_decode_attn_host, libra_kv_gather and libra_kv_scatter return
+ * Halving the bytes per cached token halves what the step has to read.  With E4M3 pools the rows given to
+ * libra_decode_attn_append (k_new, v_new: [batch, num_kv_heads, head_dim]) and the dense buffers of
+ * libra_kv_gather / libra_kv_scatter hold codes too, one byte per element; libra_decode_attn_host returns
  * UNSUPPORTED_SHAPE.  The plan and the workspace do not depend on the type. */
 #define LIBRA_KV_BF16 0
 #define LIBRA_KV_E4M3 1

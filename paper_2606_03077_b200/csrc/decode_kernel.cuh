@@ -64,12 +64,12 @@ struct DecodeParams {
   int32_t num_empty;      // empty sequences whose output row this launch zeroes
   int32_t fused_combine;  // 1: the last block of a split sequence merges its partials (step C) itself
   int32_t early_prefetch; // 1: block-table walk and first copies of old tokens start before the grid dependency wait
-  // KV append fused into the step (null k_new = off): the current token's K and V rows, bf16 [B, Hkv, D],
-  // are written into slot (L_b - 1) % 16 of the sequence's last page, in the pools and in the staged tile
-  const __nv_bfloat16* k_new;
-  const __nv_bfloat16* v_new;
-  __nv_bfloat16* k_pool;
-  __nv_bfloat16* v_pool;
+  // KV append fused into the step (null k_new = off): the current token's K and V rows, [B, Hkv, D] in the cache's
+  // element type, are written into slot (L_b - 1) % 16 of the sequence's last page, in the pools and in the staged tile
+  const void* k_new;
+  const void* v_new;
+  void* k_pool;
+  void* v_pool;
   int64_t stride_page, stride_head, stride_token;  // pool strides in elements
 };
 
@@ -781,35 +781,40 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
       const uint32_t* words = reinterpret_cast<const uint32_t*>(my_ring + s * SM::kStageBytes);
       st.l[0][0] += float((words[lane * 16] ^ words[SM::kTileBytes / 4 + lane * 16]) & 0xffu);
       st.m[0][0] = 0.f;
-    } else if constexpr (kFp8) {
-      process_page_fp8<NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes, u.kv_end - tok0,
-                           p.scale_log2, lane, common_end - tok0, len_dev - tok0, cut);
     } else {
-    if (p.k_new != nullptr && u.chunk_j == u.n_chunks - 1 && u.kv_end - tok0 <= 16) {
-      // this page holds the sequence's newest token: its K and V rows come from k_new / v_new.  The copy
-      // that just landed predates them, so patch the staged tiles (swizzled row) and write the pools.
-      const int r = (u.kv_end - 1) & 15;
-      const int which = lane / (D / 8);   // 0: K, 1: V
-      const int c16 = lane % (D / 8);
-      if (which < 2) {
-        const int last = u.kv_end - 1;                       // the newest token
-        const int64_t page = __ldg(p.block_table + int64_t(u.b) * p.block_table_ld + (last >> (4 + p.tile_shift)));
-        const int slot = last & ((16 << p.tile_shift) - 1);  // its slot in that page
-        const __nv_bfloat16* src = (which ? p.v_new : p.k_new) + (int64_t(u.b) * p.num_kv_heads + kvh) * D + c16 * 8;
-        const uint4 row = __ldg(reinterpret_cast<const uint4*>(src));
-        uint8_t* tile = my_ring + s * SM::kStageBytes + which * SM::kTileBytes;
-        *reinterpret_cast<uint4*>(tile + tile_off(r, c16)) = row;
-        if (page >= 0 && page < p.num_pages) {
-          __nv_bfloat16* dst = (which ? p.v_pool : p.k_pool) + page * p.stride_page + int64_t(kvh) * p.stride_head +
-                               int64_t(slot) * p.stride_token + c16 * 8;
-          *reinterpret_cast<uint4*>(dst) = row;
+      if (p.k_new != nullptr && u.chunk_j == u.n_chunks - 1 && u.kv_end - tok0 <= 16) {
+        // this page holds the sequence's newest token: its K and V rows come from k_new / v_new.  The copy
+        // that just landed predates them, so patch the staged tiles (swizzled row) and write the pools.
+        constexpr int EB = kFp8 ? 1 : 2;           // bytes per cache element
+        constexpr int kRowChunks = D * EB / 16;    // 16-byte chunks of one row
+        const int r = (u.kv_end - 1) & 15;
+        const int which = lane / kRowChunks;       // 0: K, 1: V
+        const int c16 = lane % kRowChunks;
+        if (which < 2) {
+          const int last = u.kv_end - 1;                       // the newest token
+          const int64_t page = __ldg(p.block_table + int64_t(u.b) * p.block_table_ld + (last >> (4 + p.tile_shift)));
+          const int slot = last & ((16 << p.tile_shift) - 1);  // its slot in that page
+          const uint8_t* src = reinterpret_cast<const uint8_t*>(which ? p.v_new : p.k_new) +
+                               (int64_t(u.b) * p.num_kv_heads + kvh) * (D * EB) + c16 * 16;
+          const uint4 row = __ldg(reinterpret_cast<const uint4*>(src));
+          uint8_t* tile = my_ring + s * SM::kStageBytes + which * SM::kTileBytes;
+          *reinterpret_cast<uint4*>(tile + tile_off(r, c16)) = row;
+          if (page >= 0 && page < p.num_pages) {
+            uint8_t* dst = reinterpret_cast<uint8_t*>(which ? p.v_pool : p.k_pool) +
+                           (page * p.stride_page + int64_t(kvh) * p.stride_head + int64_t(slot) * p.stride_token) * EB + c16 * 16;
+            *reinterpret_cast<uint4*>(dst) = row;
+          }
         }
+        fence_proxy_async();  // these generic writes come before the next TMA write into this stage
+        __syncwarp();
       }
-      fence_proxy_async();  // these generic writes come before the next TMA write into this stage
-      __syncwarp();
-    }
-    process_page<D, NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes, u.kv_end - tok0,
-                        p.scale_log2, lane, common_end - tok0, len_dev - tok0, cut);
+      if constexpr (kFp8) {
+        process_page_fp8<NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes,
+                             u.kv_end - tok0, p.scale_log2, lane, common_end - tok0, len_dev - tok0, cut);
+      } else {
+        process_page<D, NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes,
+                            u.kv_end - tok0, p.scale_log2, lane, common_end - tok0, len_dev - tok0, cut);
+      }
     }
     __syncwarp();  // every lane has consumed the stage before lane 0 refills it
     if (it + STAGES < n_it) issue(it + STAGES, s);

@@ -763,7 +763,6 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     return LIBRA_INVALID_ARGUMENT;
   }
   if (q_len < 1 || q_len > h->max_q_len || (q_len > 1 && k_new)) return LIBRA_INVALID_ARGUMENT;
-  if (h->fp8 && k_new) return LIBRA_UNSUPPORTED_SHAPE;   // the fused append writes bf16 rows
   if (!h->planned) return LIBRA_NOT_PLANNED;
   DeviceGuard guard(h->cfg.device);
   if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
@@ -843,10 +842,10 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     p.num_empty = n_empty;
     p.fused_combine = fused ? 1 : 0;
     p.early_prefetch = (h->early_prefetch && h->pdl) ? 1 : 0;
-    p.k_new = static_cast<const __nv_bfloat16*>(k_new);
-    p.v_new = static_cast<const __nv_bfloat16*>(v_new);
-    p.k_pool = static_cast<__nv_bfloat16*>(const_cast<void*>(k_pages));
-    p.v_pool = static_cast<__nv_bfloat16*>(const_cast<void*>(v_pages));
+    p.k_new = k_new;
+    p.v_new = v_new;
+    p.k_pool = const_cast<void*>(k_pages);
+    p.v_pool = const_cast<void*>(v_pages);
     p.stride_page = h->stride_page;
     p.stride_head = h->stride_head;
     p.stride_token = h->stride_token;
@@ -1026,7 +1025,6 @@ namespace {
 int kv_move_impl(libra_handle_t h, bool gather, void* k_pages, void* v_pages, void* k_dense, void* v_dense,
                  const int32_t* block_table, const int32_t* seq_lens, const int64_t* token_offsets, int32_t batch,
                  int32_t max_seq_len, int32_t head_begin, int32_t head_count, void* error_word_dev, void* stream) {
-  if (h && h->fp8) return LIBRA_UNSUPPORTED_SHAPE;   // the move kernels are written for bf16 rows
   if (!h || !k_pages || !v_pages || !k_dense || !v_dense || !block_table || !seq_lens || !token_offsets ||
       !error_word_dev) {
     return LIBRA_INVALID_ARGUMENT;
@@ -1052,9 +1050,11 @@ int kv_move_impl(libra_handle_t h, bool gather, void* k_pages, void* v_pages, vo
   p.block_table = block_table;
   p.seq_lens = seq_lens;
   p.token_offsets = token_offsets;
-  p.stride_page = h->stride_page;
-  p.stride_head = h->stride_head;
-  p.stride_token = h->stride_token;
+  // an E4M3 row of 128 codes is moved as a row of 64 two-byte elements (strides are multiples of 16 bytes)
+  const int64_t unit = h->fp8 ? 2 : 1;
+  p.stride_page = h->stride_page / unit;
+  p.stride_head = h->stride_head / unit;
+  p.stride_token = h->stride_token / unit;
   p.num_pages = h->cfg.num_pages;
   p.block_table_ld = h->cfg.block_table_ld;
   p.head_begin = head_begin;
@@ -1064,7 +1064,7 @@ int kv_move_impl(libra_handle_t h, bool gather, void* k_pages, void* v_pages, vo
   const int pages = (max_seq_len + h->cfg.page_size - 1) / h->cfg.page_size;
   dim3 grid(unsigned((pages + libra::kMovePagesPerBlock - 1) / libra::kMovePagesPerBlock), unsigned(batch));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (h->cfg.head_dim == 128) {
+  if (h->cfg.head_dim == 128 && !h->fp8) {
     if (gather) libra::kv_move_kernel<128, true><<<grid, libra::kMoveThreads, 0, st>>>(p);
     else libra::kv_move_kernel<128, false><<<grid, libra::kMoveThreads, 0, st>>>(p);
   } else {

@@ -172,9 +172,10 @@ def test_what_is_not_supported_says_so(lib):
     st = torch.cuda.current_stream().cuda_stream
     h.plan(np.array([5], dtype=np.int32), ws.data_ptr(), ws.numel(), st)
     x = torch.zeros(1 << 16, dtype=torch.int16, device="cuda:0")
-    with pytest.raises(lib.LibraError):                   # the fused append writes bf16 rows
-        h.decode_attn_append(x.data_ptr(), x.data_ptr(), x.data_ptr(), x.data_ptr(), x.data_ptr(), x.data_ptr(),
-                             x.data_ptr(), x.data_ptr(), st)
+    hs = torch.zeros(1 << 16, dtype=torch.int16).pin_memory()
+    with pytest.raises(lib.LibraError):                   # the host-buffer entry point is sized for bf16 pools
+        h.decode_attn_host(hs.data_ptr(), hs.data_ptr(), hs.data_ptr(), hs.data_ptr(), hs.data_ptr(), 1, hs.data_ptr(),
+                           x.data_ptr(), x.numel() * 2, ws.data_ptr(), ws.numel(), st)
     h.set_kv_dtype(lib.KV_BF16)                           # and back
     torch.cuda.synchronize()
     h.close()
@@ -182,3 +183,93 @@ def test_what_is_not_supported_says_so(lib):
     with pytest.raises(lib.LibraError):
         odd.set_kv_dtype(lib.KV_E4M3, 1.0, 1.0)
     odd.close()
+
+
+@pytest.mark.parametrize("layout", ["HND", "NHD"])
+def test_fused_append_of_8bit_rows(lib, layout):
+    # the newest token's K and V rows arrive as E4M3 codes; afterwards the pools hold them and the output is the
+    # oracle's on the updated pools
+    import torch
+    dev = torch.device("cuda:0")
+    lens = [1, 16, 17, 300, 1025, 2048, 33]
+    B, Hq, Hkv, d = len(lens), 16, 4, 128
+    lens_a, bt, q, k8, v8 = W.random_case_e4m3(630, B, Hq, Hkv, d, lens)
+    _, _, _, kn, vn = W.random_case_e4m3(631, 1, Hq, Hkv, d, [B], poison=False)     # codes for the new rows
+    k_new = np.ascontiguousarray(kn[0, :, :B, :].transpose(1, 0, 2))                 # [B, Hkv, d]
+    v_new = np.ascontiguousarray(vn[0, :, :B, :].transpose(1, 0, 2))
+    k_ref, v_ref = k8.copy(), v8.copy()
+    for b, n in enumerate(lens_a):
+        k_ref[bt[b, (n - 1) // 16], :, (n - 1) % 16, :] = k_new[b]
+        v_ref[bt[b, (n - 1) // 16], :, (n - 1) % 16, :] = v_new[b]
+    ref, _ = O.paged_decode_attention_fp8(q, k_ref, v_ref, bt, lens_a, 0.5, 2.0)
+    strides = (0, 0, 0)
+    kd_h, vd_h = k8, v8
+    if layout == "NHD":
+        kd_h = np.ascontiguousarray(k8.transpose(0, 2, 1, 3))
+        vd_h = np.ascontiguousarray(v8.transpose(0, 2, 1, 3))
+        strides = (16 * Hkv * d, d, Hkv * d)
+    for plan in (None, small_plan(lib)):
+        h = lib.Handle(Hq, Hkv, d, k8.shape[0], B, bt.shape[1], kv_strides=strides, plan=plan)
+        h.set_kv_dtype(lib.KV_E4M3, 0.5, 2.0)
+        ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=dev)
+        qd, btd = H.to_dev(q, dev), H.to_dev(bt, dev)
+        kd, vd = torch.from_numpy(kd_h).to(dev), torch.from_numpy(vd_h).to(dev)
+        knd, vnd = torch.from_numpy(k_new).to(dev), torch.from_numpy(v_new).to(dev)
+        lens_dev = torch.from_numpy(lens_a).to(dev)
+        out = torch.full((B, Hq, d), H.CANARY, dtype=torch.int16, device=dev)
+        st = torch.cuda.current_stream().cuda_stream
+        h.plan(lens_a, ws.data_ptr(), ws.numel(), st)
+        h.decode_attn_append(qd.data_ptr(), knd.data_ptr(), vnd.data_ptr(), kd.data_ptr(), vd.data_ptr(), btd.data_ptr(),
+                             lens_dev.data_ptr(), out.data_ptr(), st)
+        torch.cuda.synchronize()
+        assert h.debug_error_word() == 0
+        check(H.bf16_dev_to_f32(out), ref, f"append {layout}")
+        got_k, got_v = kd.cpu().numpy(), vd.cpu().numpy()
+        if layout == "NHD":
+            got_k, got_v = got_k.transpose(0, 2, 1, 3), got_v.transpose(0, 2, 1, 3)
+        assert np.array_equal(got_k, k_ref) and np.array_equal(got_v, v_ref)
+        h.close()
+
+
+def test_gather_and_scatter_of_8bit_pools(lib):
+    # the migration copies on E4M3 pools: gather a head range to a dense buffer, scatter it under a new placement
+    import torch
+    from oracle import kv_move_oracle as M
+    dev = torch.device("cuda:0")
+    lens = [40, 1, 16, 333]
+    B, Hkv, d, h0, hn = len(lens), 8, 128, 2, 4
+    lens_a, bt, _, k8, v8 = W.random_case_e4m3(632, B, Hkv, Hkv, d, lens, poison=False)
+    h = lib.Handle(Hkv, Hkv, d, k8.shape[0], B, bt.shape[1])
+    h.set_kv_dtype(lib.KV_E4M3, 1.0, 1.0)
+    offs = np.concatenate([[0], np.cumsum(lens_a.astype(np.int64))])
+    total = int(offs[-1])
+    dk, dv, dbt = torch.from_numpy(k8).to(dev), torch.from_numpy(v8).to(dev), H.to_dev(bt, dev)
+    dl = torch.from_numpy(lens_a.copy()).to(dev)
+    doffs = torch.from_numpy(offs[:-1].copy()).to(dev)
+    err = torch.zeros(1, dtype=torch.int32, device=dev)
+    k_dense = torch.full((total, hn, d), 0x7F, dtype=torch.uint8, device=dev)
+    v_dense = torch.full((total, hn, d), 0x7F, dtype=torch.uint8, device=dev)
+    st = torch.cuda.current_stream().cuda_stream
+    h.kv_gather(dk.data_ptr(), dv.data_ptr(), dbt.data_ptr(), dl.data_ptr(), doffs.data_ptr(), B, int(lens_a.max()),
+                h0, hn, k_dense.data_ptr(), v_dense.data_ptr(), err.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    assert np.array_equal(k_dense.cpu().numpy(), M.gather(k8, bt, lens_a, h0, hn))
+    assert np.array_equal(v_dense.cpu().numpy(), M.gather(v8, bt, lens_a, h0, hn))
+    rng = np.random.default_rng(5)
+    bt2, pool2 = W.draw_block_table(lens_a, int(W.pages_needed(lens_a).sum()) + 5, rng, ld=bt.shape[1])
+    h2 = lib.Handle(hn, hn, d, pool2, B, bt.shape[1])
+    h2.set_kv_dtype(lib.KV_E4M3, 1.0, 1.0)
+    k2 = torch.full((pool2, hn, 16, d), 0xEE, dtype=torch.uint8, device=dev)
+    v2 = torch.full((pool2, hn, 16, d), 0xEE, dtype=torch.uint8, device=dev)
+    dbt2 = H.to_dev(bt2, dev)
+    h2.kv_scatter(k_dense.data_ptr(), v_dense.data_ptr(), dbt2.data_ptr(), dl.data_ptr(), doffs.data_ptr(),
+                  B, int(lens_a.max()), 0, hn, k2.data_ptr(), v2.data_ptr(), err.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    want_k = np.full((pool2, hn, 16, d), 0xEE, np.uint8)
+    want_v = np.full((pool2, hn, 16, d), 0xEE, np.uint8)
+    M.scatter(M.gather(k8, bt, lens_a, h0, hn), want_k, bt2, lens_a, 0)
+    M.scatter(M.gather(v8, bt, lens_a, h0, hn), want_v, bt2, lens_a, 0)
+    assert np.array_equal(k2.cpu().numpy(), want_k) and np.array_equal(v2.cpu().numpy(), want_v)
+    h.close(); h2.close()
