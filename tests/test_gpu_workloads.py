@@ -54,3 +54,85 @@ def test_workload_parity(lib, name, n_sample):
         r.h.set_combine_mode(1)
         W.restore_tails(saved, k, v)
     r.h.close()
+
+
+@pytest.mark.parametrize("name,n_sample", [("lognormal_b64", 24), ("longtail_mix_b256", 10), ("straggler_b8", 2)])
+def test_workload_parity_8bit_cache(lib, name, n_sample):
+    """The same full-size workloads over an E4M3 cache (device pools of random finite codes, default launch
+    configuration), sampled sequences against the oracle."""
+    import torch
+    dev = torch.device("cuda:0")
+    w = W.WORKLOADS[name]
+    lay, _ = W.make_layout(name, 0)
+    shape = (lay.pool_pages, w.num_kv_heads, w.page_size, w.head_dim)
+    gen = torch.Generator(device=dev).manual_seed(11)
+
+    def codes():   # sign and mantissa random, exponent field 0..8: finite, |x| < 4
+        r = torch.randint(0, 256, shape, dtype=torch.uint8, device=dev, generator=gen)
+        r &= 0x87
+        r |= torch.randint(0, 9, shape, dtype=torch.uint8, device=dev, generator=gen) << 3
+        return r
+
+    k8, v8 = codes(), codes()
+    q = torch.randn((w.batch, w.num_q_heads, w.head_dim), device=dev, generator=gen).to(torch.bfloat16)
+    h = lib.Handle(w.num_q_heads, w.num_kv_heads, w.head_dim, lay.pool_pages, w.batch, lay.block_table.shape[1])
+    h.set_kv_dtype(lib.KV_E4M3, 0.5, 1.25)
+    ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=dev)
+    btd = H.to_dev(lay.block_table, dev)
+    lens_dev = torch.from_numpy(lay.seq_lens.copy()).to(dev)
+    out = torch.full((w.batch, w.num_q_heads, w.head_dim), H.CANARY, dtype=torch.int16, device=dev)
+    st = torch.cuda.current_stream().cuda_stream
+    h.plan(lay.seq_lens, ws.data_ptr(), ws.numel(), st)
+    h.decode_attn(q.data_ptr(), k8.data_ptr(), v8.data_ptr(), btd.data_ptr(), lens_dev.data_ptr(), out.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert h.debug_error_word() == 0
+    got_all = H.bf16_dev_to_f32(out)
+    assert np.all(np.isfinite(got_all))
+    rows = sample_rows(lay.seq_lens, n_sample, 3)
+    ids, new_bt = [], np.full((len(rows), lay.block_table.shape[1]), -1, dtype=np.int32)
+    for i, b in enumerate(rows):
+        n = (int(lay.seq_lens[b]) + 15) // 16
+        new_bt[i, :n] = np.arange(len(ids), len(ids) + n)
+        ids.extend(int(x) for x in lay.block_table[b, :n])
+    idx = torch.tensor(ids, dtype=torch.long, device=dev)
+    kh, vh = k8[idx].cpu().numpy(), v8[idx].cpu().numpy()
+    qh = q.view(torch.int16)[torch.tensor(rows, device=dev)].cpu().numpy().view(np.uint16)
+    ref, _ = O.paged_decode_attention_fp8(qh, kh, vh, new_bt, lay.seq_lens[rows], 0.5, 1.25)
+    got = got_all[rows]
+    assert gates.stated_violations(got, ref) == 0
+    assert gates.tight_violations(got, ref) == 0, gates.tight_ratio(got, ref)
+    h.close()
+
+
+@pytest.mark.parametrize("name,q_len,n_sample", [("lognormal_b64", 4, 24), ("straggler_b8", 2, 2), ("shift_b128", 3, 8)])
+def test_workload_parity_several_query_tokens(lib, name, q_len, n_sample):
+    """The full-size workloads with q_len query tokens per sequence, sampled sequences against the oracle."""
+    import torch
+    dev = torch.device("cuda:0")
+    w = W.WORKLOADS[name]
+    lay, _ = W.make_layout(name, 0)
+    _, k, v = W.fill_device_pools(lay, dev, poison=True)
+    gen = torch.Generator(device=dev).manual_seed(12)
+    q = torch.randn((w.batch, q_len, w.num_q_heads, w.head_dim), device=dev, generator=gen).to(torch.bfloat16)
+    h = lib.Handle(w.num_q_heads, w.num_kv_heads, w.head_dim, lay.pool_pages, w.batch, lay.block_table.shape[1])
+    h.set_max_query_tokens(q_len)
+    ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=dev)
+    btd = H.to_dev(lay.block_table, dev)
+    lens_dev = torch.from_numpy(lay.seq_lens.copy()).to(dev)
+    out = torch.full(tuple(q.shape), H.CANARY, dtype=torch.int16, device=dev)
+    st = torch.cuda.current_stream().cuda_stream
+    h.plan(lay.seq_lens, ws.data_ptr(), ws.numel(), st)
+    h.decode_attn_multi(q.data_ptr(), q_len, k.data_ptr(), v.data_ptr(), btd.data_ptr(), lens_dev.data_ptr(),
+                        out.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert h.debug_error_word() == 0
+    got_all = H.bf16_dev_to_f32(out)
+    assert np.all(np.isfinite(got_all))
+    rows = sample_rows(lay.seq_lens, n_sample, 4)
+    kh, vh, bth, lh = H.gather_for_oracle(k, v, lay.block_table, lay.seq_lens, rows)
+    qh = q.view(torch.int16)[torch.tensor(rows, device=dev)].cpu().numpy().view(np.uint16)
+    ref, _ = O.paged_multi_token_attention(qh, kh, vh, bth, lh)
+    got = got_all[rows]
+    assert gates.stated_violations(got, ref) == 0
+    assert gates.tight_violations(got, ref) == 0, gates.tight_ratio(got, ref)
+    h.close()
