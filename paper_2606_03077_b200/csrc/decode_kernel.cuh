@@ -209,6 +209,7 @@ __device__ __forceinline__ Unit decode_unit(const int4 item, int kvh, int warp) 
 // Column c of a unit (KV head kvh) is query token c / G, head kvh * G + c % G of that token; q and out are
 // [B, q_len, hq, d], so the row within a sequence is:
 __device__ __forceinline__ int col_row(const DecodeParams& p, int kvh, int c) {
+  if (p.q_len == 1) return kvh * p.group + c;   // the usual case, without the division
   const int i = c / p.group;
   return i * p.hq + kvh * p.group + (c - i * p.group);
 }
@@ -716,7 +717,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
       const int c = nt * 8 + 2 * (lane & 3) + e;
-      cut[nt][e] = (c < p.cols) ? p.q_len - 1 - c / p.group : 0;
+      cut[nt][e] = (p.q_len > 1 && c < p.cols) ? p.q_len - 1 - c / p.group : 0;
     }
   }
   const int common_end = min(u.kv_end, len_dev - (p.q_len - 1));   // tokens below this are seen by every column
