@@ -322,7 +322,7 @@ def ceilings_measure(rep: Replica, reps: int = 20):
                     "tiled copies, no math); contiguous_read = libra_debug_stream_read over 4 GiB"}
 
 
-def multi_token_measure(rep: Replica, q_len: int, steps: int = 200):
+def multi_token_measure(rep: Replica, q_len: int, steps: int = 200, variant=None):
     """The step with q_len query tokens per sequence (libra_decode_attn_multi) on the same pools, block tables
     and lengths: one pass over K and V serves all q_len tokens."""
     torch, w = rep.torch, rep.w
@@ -331,6 +331,8 @@ def multi_token_measure(rep: Replica, q_len: int, steps: int = 200):
     h = rep.binding.Handle(w.num_q_heads, w.num_kv_heads, w.head_dim, rep.layouts[0].pool_pages, w.batch, rep.ld,
                            device=rep.dev.index or 0)
     h.set_max_query_tokens(q_len)
+    if variant is not None:
+        h.set_variant(*variant)
     ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=rep.dev)
     gen = torch.Generator(device=rep.dev).manual_seed(7)
     q = torch.randn((w.batch, q_len, w.num_q_heads, w.head_dim), generator=gen, device=rep.dev).to(torch.bfloat16)
