@@ -178,8 +178,9 @@ int libra_set_dependent_launch(libra_handle_t handle, int32_t on);
 
 /* Early prefetch, off by default: a PROMISE by the caller about the kernel that precedes each decode call in the
  * stream, namely that it writes none of: block_table, seq_lens (device), and the cached K/V rows of any token
- * other than each sequence's newest q_len tokens (a projection / rotary / cache-write kernel qualifies; a kernel
- * that moves or rewrites old pages does not).  With the promise, and dependent launch on, a decode block that
+ * other than each sequence's newest q_len + 1 tokens, counted by this call's seq_lens (a projection / rotary /
+ * cache-write kernel for this step's tokens qualifies, and so does the previous step's
+ * libra_decode_attn_append when the lengths grew by one; a kernel that moves or rewrites older pages does not).  With the promise, and dependent launch on, a decode block that
  * becomes resident while that kernel drains walks its block-table row and starts the copies of its first tiles
  * of old tokens before it waits for that kernel to finish; q, the newest rows, `out` and the workspace are
  * still touched only afterwards.  Results are bit-identical to the default.  Applies to plans that travel in

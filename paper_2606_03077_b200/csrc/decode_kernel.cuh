@@ -669,7 +669,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   // Up to here nothing was read that an earlier kernel in the stream could have written, so when this
   // launch overlaps the tail of its predecessor the block is resident and set up by the time that ends.
   // With early prefetch (a promise by the caller that the preceding kernel writes neither the block table, the
-  // lengths nor any cached row except those of each sequence's newest q_len tokens) the block goes further
+  // lengths nor any cached row except those of each sequence's newest q_len + 1 tokens) the block goes further
   // before it waits: it walks its block-table row and starts the copies of its first tiles of old tokens.
   // Only a plan that travels in the kernel parameters allows it (a plan in device memory may itself have been
   // written by the preceding kernel).
@@ -752,9 +752,9 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   const int pre = n_it < STAGES ? n_it : STAGES;
   int issued = 0;
   if (early) {
-    // tokens [0, safe_end) were in the cache before the preceding kernel ran; with the fused append the pools are
-    // written by this kernel only, so every tile qualifies (the newest row is patched in after its tile lands)
-    const int safe_end = (p.k_new != nullptr) ? len_dev : len_dev - p.q_len;
+    // tokens [0, safe_end) were in the cache before the preceding kernel ran: it may have written this step's
+    // newest q_len rows (a cache-write kernel) or the row before them (the fused append of the previous step)
+    const int safe_end = len_dev - p.q_len - 1;
     while (issued < pre && u.kv_begin + ((warp + issued * NW) << 4) + 16 <= safe_end) {
       issue(issued, issued);
       ++issued;

@@ -74,3 +74,49 @@ def test_append_matches_definition(lib, Hq, Hkv, d, lens, P, layout):
             k_after, v_after = k_after.transpose(0, 2, 1, 3), v_after.transpose(0, 2, 1, 3)
         assert np.array_equal(k_after, k_ref) and np.array_equal(v_after, v_ref)
         r.h.close()
+
+
+def test_chain_of_append_steps_with_early_prefetch(lib):
+    """Five decode steps with the fused append, lengths growing by one per step, queued without synchronising:
+    with early prefetch the step may start its copies while the previous step (which wrote the previous token's
+    rows) is still running; outputs and pools must equal the default's bit for bit, and the oracle's."""
+    import torch
+    dev = torch.device("cuda:0")
+    steps = 5
+    lens0 = np.array([1, 15, 16, 31, 300, 1024, 2047], dtype=np.int32)
+    B, Hq, Hkv, d = len(lens0), 16, 4, 128
+    lens_max, bt, q, k, v = W.random_case(81, B, Hq, Hkv, d, lens0 + steps, poison=False)
+    rng = np.random.default_rng(82)
+    new_k = W.f32_to_bf16_bits(rng.standard_normal((steps, B, Hkv, d)).astype(np.float32))
+    new_v = W.f32_to_bf16_bits(rng.standard_normal((steps, B, Hkv, d)).astype(np.float32))
+    new_q = W.f32_to_bf16_bits(rng.standard_normal((steps, B, Hq, d)).astype(np.float32))
+    res = {}
+    for early in (False, True):
+        r = H.Runner(lib, Hq, Hkv, d, k.shape[0], B, bt.shape[1], plan=lib.PlanParams(148, 1, 1, 256, 512, 64))
+        r.h.set_early_prefetch(early)
+        kd, vd, btd = H.to_dev(k, dev), H.to_dev(v, dev), H.to_dev(bt, dev)
+        nk, nv, nq = H.to_dev(new_k, dev), H.to_dev(new_v, dev), H.to_dev(new_q, dev)
+        lens_dev = [torch.from_numpy(lens0 + 1 + i).to(dev) for i in range(steps)]
+        outs = torch.zeros((steps, B, Hq, d), dtype=torch.int16, device=dev)
+        st = torch.cuda.current_stream().cuda_stream
+        torch.cuda.synchronize()
+        for i in range(steps):
+            r.h.plan(lens0 + 1 + i, r.ws.data_ptr(), r.ws.numel(), st)
+            r.h.decode_attn_append(nq[i].data_ptr(), nk[i].data_ptr(), nv[i].data_ptr(), kd.data_ptr(), vd.data_ptr(),
+                                   btd.data_ptr(), lens_dev[i].data_ptr(), outs[i].data_ptr(), st)
+        torch.cuda.synchronize()
+        assert r.h.debug_error_word() == 0
+        res[early] = (H.bf16_dev_to_f32(outs), kd.cpu().numpy().view(np.uint16), vd.cpu().numpy().view(np.uint16))
+        r.h.close()
+    assert np.array_equal(res[True][0], res[False][0])
+    assert np.array_equal(res[True][1], res[False][1]) and np.array_equal(res[True][2], res[False][2])
+    kk, vv = k.copy(), v.copy()
+    for i in range(steps):
+        for b in range(B):
+            t = int(lens0[b]) + i
+            kk[bt[b, t // 16], :, t % 16] = new_k[i, b]
+            vv[bt[b, t // 16], :, t % 16] = new_v[i, b]
+    assert np.array_equal(res[True][1], kk) and np.array_equal(res[True][2], vv)
+    ref, _ = O.paged_decode_attention(new_q[-1], kk, vv, bt, lens0 + steps)
+    got = res[True][0][-1]
+    assert gates.stated_violations(got, ref) == 0 and gates.tight_violations(got, ref) == 0
