@@ -53,3 +53,20 @@ def test_host_inputs_poisoned_outside():
     assert np.all(np.abs(kf[:, 0][owned]) <= 1.0)
     assert np.all(kf[:, 0][~owned] > 1e29)
     assert np.all(np.abs(W.bf16_bits_to_f32(q)) <= 1.0)
+
+
+def test_e4m3_case_generator():
+    # codes are made from bit fields: live slots are finite with exponent field <= 8, dead slots hold the NaN code
+    lens, bt, q, k8, v8 = W.random_case_e4m3(5, 3, 4, 2, 16, (3, 16, 21))
+    lens2, bt2, q2, k82, v82 = W.random_case_e4m3(5, 3, 4, 2, 16, (3, 16, 21))
+    assert np.array_equal(k8, k82) and np.array_equal(v8, v82) and np.array_equal(bt, bt2) and np.array_equal(q, q2)
+    assert k8.dtype == np.uint8 and k8.shape == v8.shape and k8.shape[1:] == (2, 16, 16)
+    live = np.zeros(k8.shape[0] * 16, dtype=bool).reshape(-1, 16)
+    for b, L in enumerate(lens):
+        for t in range(int(L)):
+            live[bt[b, t // 16], t % 16] = True
+    for pool, nan in ((k8, W.E4M3_NAN), (v8, W.E4M3_NAN | 0x80)):
+        lv = pool.transpose(0, 2, 1, 3)[live]
+        assert np.all(((lv >> 3) & 0xF) <= 8)
+        assert np.all(pool.transpose(0, 2, 1, 3)[~live] == nan)
+    assert len(np.unique(bt[bt >= 0])) == int(W.pages_needed(lens).sum())
