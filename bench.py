@@ -422,6 +422,40 @@ def fp8_cache_measure(rep: Replica, steps: int = 200, variant=None):
             "pool_copies": copies, "steps": steps}
 
 
+def ring_step_measure(rep: Replica, reps: int = 40):
+    """The ring all-reduce's data-plane step (libra_ring_step, flag already set) on 16 MB float32 chunks, the chunk
+    size the paper pipelines with: payload rate of a reduce step on 2 and on 4 thread blocks (= SMs)."""
+    torch = rep.torch
+    n = (16 << 20) // 4
+    sets = 10    # rotate over 480 MB of operands: larger than L2
+    own = torch.ones((sets, n), dtype=torch.float32, device=rep.dev)
+    recv = torch.ones((sets, n), dtype=torch.float32, device=rep.dev)
+    dst = torch.zeros((sets, n), dtype=torch.float32, device=rep.dev)
+    flag = torch.ones(1, dtype=torch.int32, device=rep.dev)
+    status = torch.zeros(1, dtype=torch.int32, device=rep.dev)
+    st = torch.cuda.current_stream().cuda_stream
+    out = {"chunk_bytes": n * 4}
+    for blocks in (2, 4):
+        def one(i):
+            k = i % sets
+            rep.binding.libra_ring_step(rep.dev.index or 0, dst[k].data_ptr(), own[k].data_ptr(), recv[k].data_ptr(), n * 4,
+                                        rep.binding.RING_F32, flag.data_ptr(), 1, 1000000, status.data_ptr(), blocks, st)
+        for i in range(5):
+            one(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(reps):
+            one(i)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        out[f"blocks_{blocks}"] = {"ms_per_step": ms, "payload_gbs": n * 4 / (ms * 1e-3) / 1e9,
+                                   "memory_gbs": 3 * n * 4 / (ms * 1e-3) / 1e9}
+    assert int(status.item()) == 0
+    return out
+
+
 def e2e_measure(rep: Replica, steps: int):
     """The step through libra_decode_attn_host with every input in pinned host memory."""
     torch = rep.torch
@@ -719,6 +753,8 @@ def run_libra(args):
             line["multi_token"] = [m for m in (multi_token_measure(rep, t) for t in (2, 4)) if m]
         if "fp8_cache" in extras:
             line["fp8_cache"] = fp8_cache_measure(rep, steps=min(200, max(10, args.steps)))
+        if "ring_step" in extras:
+            line["ring_step"] = ring_step_measure(rep)
         if "kv_migration" in extras and args.workload in ("longtail_mix_b256", "straggler_b8"):
             line["kv_migration"] = kv_migration_measure(rep)
         if not args.no_cpu:
@@ -789,7 +825,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
-    ap.add_argument("--extras", default="ceilings,early_prefetch,multi_token,fp8_cache,kv_migration",
+    ap.add_argument("--extras", default="ceilings,early_prefetch,multi_token,fp8_cache,kv_migration,ring_step",
                     help="side measurements on the main workload at N=1 (comma list; empty = none)")
     ap.add_argument("--variant", default="", help="warps,stages of the decode block (default: the library's)")
     ap.add_argument("--ctas-per-sm", type=int, default=0, help="planner constant (0 = default)")

@@ -413,6 +413,28 @@ int libra_trie_route(libra_trie_t trie, int64_t prompt_id, const int32_t* states
                      int32_t n_buckets, const double* decode_cost, const double* migration_cost,
                      int32_t* best_bucket, double* best_cost);
 
+/* ---- Data plane of the inter-replica ring all-reduce (Section 6, "Decoupled communication domains"; appendix
+ * "Decoupled Communication Domain") ----------------------------------------------------------------------------
+ * In the paper the CPU owns membership, transport and flow control of the gradient exchange between replicas; the
+ * GPU runs only the copy / reduce steps of a ring ReduceScatter + AllGather, polls a host-pinned arrival flag with a
+ * software timeout instead of blocking, and uses 2 SMs.  libra_ring_step enqueues ONE such step on `stream` of
+ * `device`:
+ *   wait until *ready_flag >= expected (ready_flag: host-pinned mapped memory or device memory, 4-byte aligned; the
+ *   producer writes the chunk first, then the flag), for at most timeout_us microseconds (1 .. 10,000,000);
+ *   then  own != NULL : dst[i] = own[i] + received[i]   (a ReduceScatter step; LIBRA_RING_F32: float32 addition;
+ *                        LIBRA_RING_BF16: bfloat16 values added in float32, rounded to nearest even)
+ *         own == NULL : dst[i] = received[i]            (an AllGather step)
+ * over `bytes` bytes (a multiple of 16; all buffers 16-byte aligned; dst may equal own).  num_blocks thread blocks of
+ * 512 threads do the work (0 = the default of 2; at most 64).  *status_dev (device memory) receives 0 when the step
+ * ran and 1 when the wait ran out, in which case nothing else was written and the context stays usable.  Everything
+ * around the step - who sends what to whom, chunking, membership - is the caller's.
+ * Errors: INVALID_ARGUMENT, CUDA_ERROR. */
+#define LIBRA_RING_F32 0
+#define LIBRA_RING_BF16 1
+int libra_ring_step(int32_t device, void* dst, const void* own, const void* received, size_t bytes, int32_t dtype,
+                    const uint32_t* ready_flag, uint32_t expected, uint32_t timeout_us, uint32_t* status_dev,
+                    int32_t num_blocks, void* stream);
+
 /* Self-test of the kernels' bounded waits: enqueues a one-warp kernel that waits, with a limit of a few
  * milliseconds, on a copy barrier that nothing completes.  It must return (no hang, no trap) and leave
  * LIBRA_ERR_WAIT_TIMEOUT in the device error word of the last planned workspace, which is how a real

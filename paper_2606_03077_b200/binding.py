@@ -21,6 +21,7 @@ LIB_PATH = _LIB_PATH
 STATIC_SCRATCH_BYTES = 8 << 20
 OK, INVALID_ARGUMENT, UNSUPPORTED_SHAPE, WORKSPACE_TOO_SMALL, NOT_PLANNED, CUDA_ERROR, DEVICE_FLAGGED = range(7)
 KV_BF16, KV_E4M3 = 0, 1
+RING_F32, RING_BF16 = 0, 1
 ERR_WAIT_TIMEOUT, ERR_BAD_PAGE_ID, ERR_SEQ_LEN_MISMATCH, ERR_PLAN_OVERFLOW = 1, 2, 4, 8
 
 
@@ -63,6 +64,8 @@ SIGNATURES = {
     "libra_set_early_prefetch": (C.c_int, [_vp, C.c_int32]),
     "libra_set_kv_dtype": (C.c_int, [_vp, C.c_int32, C.c_float, C.c_float]),
     "libra_decode_attn_multi": (C.c_int, [_vp, _vp, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "libra_ring_step": (C.c_int, [C.c_int32, _vp, _vp, _vp, C.c_size_t, C.c_int32, _vp, C.c_uint32, C.c_uint32, _vp, C.c_int32,
+                                  _vp]),
     "libra_debug_stream_read": (C.c_int, [_vp, _vp, C.c_size_t, _vp]),
     "libra_debug_gather_read": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_set_combine_mode": (C.c_int, [_vp, C.c_int32]),
@@ -147,6 +150,14 @@ def libra_plan_host(seq_lens, num_kv_heads: int, params: PlanParams, items_capac
             "item_offset": out["item_offset"][:B].copy(), "items": items[:n].copy(),
             "combine": out["combine"][:scal["num_combine"].value].copy(),
             "empty": out["empty"][:scal["num_empty"].value].copy()}
+
+
+def libra_ring_step(device: int, dst_ptr: int, own_ptr: int, received_ptr: int, nbytes: int, dtype: int,
+                    ready_flag_ptr: int, expected: int, timeout_us: int, status_ptr: int, num_blocks: int,
+                    stream: int) -> None:
+    """One copy / reduce step of the ring all-reduce's data plane (own_ptr = 0 for a copy step)."""
+    _check(lib.libra_ring_step(device, dst_ptr, own_ptr or None, received_ptr, nbytes, dtype, ready_flag_ptr, expected,
+                               timeout_us, status_ptr, num_blocks, stream), "libra_ring_step")
 
 
 def libra_rollout_dp(n_gpus: int, lengths, tp_set, cost_coef):

@@ -17,6 +17,7 @@
 #include "plan_layout.hpp"
 #include "planner.hpp"
 #include "read_kernel.cuh"
+#include "ring_kernel.cuh"
 
 static_assert(LIBRA_ERR_WAIT_TIMEOUT == LIBRA_DEV_ERR_WAIT_TIMEOUT, "error bits");
 static_assert(LIBRA_ERR_BAD_PAGE_ID == LIBRA_DEV_ERR_BAD_PAGE_ID, "error bits");
@@ -1132,6 +1133,37 @@ int libra_debug_stream_read(libra_handle_t h, const void* buf_dev, size_t bytes,
   LIBRA_CUDA_TRY(h, cudaGetLastError());
   ++h->launches;
   h->last_stream = stream;
+  return LIBRA_OK;
+}
+
+int libra_ring_step(int32_t device, void* dst, const void* own, const void* received, size_t bytes, int32_t dtype,
+                    const uint32_t* ready_flag, uint32_t expected, uint32_t timeout_us, uint32_t* status_dev,
+                    int32_t num_blocks, void* stream) {
+  if (device < 0 || !dst || !received || !ready_flag || !status_dev) return LIBRA_INVALID_ARGUMENT;
+  if (dtype != LIBRA_RING_F32 && dtype != LIBRA_RING_BF16) return LIBRA_INVALID_ARGUMENT;
+  if (bytes % 16 != 0 || num_blocks < 0 || num_blocks > 64 || timeout_us == 0 || timeout_us > 10000000u) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  if (reinterpret_cast<uintptr_t>(dst) % 16 || reinterpret_cast<uintptr_t>(own) % 16 ||
+      reinterpret_cast<uintptr_t>(received) % 16 || reinterpret_cast<uintptr_t>(ready_flag) % 4 ||
+      reinterpret_cast<uintptr_t>(status_dev) % 4) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  DeviceGuard guard(device);
+  if (guard.err != cudaSuccess) return fail_cuda(nullptr, guard.err);
+  libra::RingStepParams p;
+  p.dst = dst;
+  p.own = own;
+  p.received = received;
+  p.n16 = bytes / 16;
+  p.ready = ready_flag;
+  p.expected = expected;
+  p.timeout_us = timeout_us;
+  p.status = status_dev;
+  p.bf16 = (dtype == LIBRA_RING_BF16) ? 1 : 0;
+  libra::ring_step_kernel<<<unsigned(num_blocks == 0 ? 2 : num_blocks), libra::kRingThreads, 0,
+                            static_cast<cudaStream_t>(stream)>>>(p);
+  if (cudaGetLastError() != cudaSuccess) return LIBRA_CUDA_ERROR;
   return LIBRA_OK;
 }
 
