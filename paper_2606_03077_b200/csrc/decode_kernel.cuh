@@ -107,14 +107,23 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 
-// Tiled 4-D TMA load global -> shared (no multicast), completing on an mbarrier of this block.
+// L2 policy for data that is read once: pages of K and V are streamed, never reused, so they should be the first
+// to leave L2 and not push out what IS reused (q, block tables, the plan, partial results).
+// Measured: 57.7 -> 56.2 us per step on the headline workload, 0.5 - 1.5 % on the others.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+
+// Tiled 4-D TMA load global -> shared (no multicast) with an L2 cache policy, completing on an mbarrier of this block.
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
-                                            int c3) {
+                                            int c3, uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], "
-      "[%2];"
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
       :
-      : "r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy)
       : "memory");
 }
 
@@ -658,6 +667,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   const uint32_t my_ring_u32 = smem_u32(my_ring);
   const uint32_t my_bar0 = smem_u32(&bars[warp * STAGES]);
 
+  const uint64_t kv_policy = l2_evict_first_policy();
   if (lane == 0) {
     prefetch_tensormap(&map_k);
     prefetch_tensormap(&map_v);
@@ -740,9 +750,9 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
       fence_proxy_async();  // earlier generic-proxy accesses to this stage come before the async write
       mbar_expect_tx(bar, SM::kStageBytes);
 #pragma unroll
-      for (int h = 0; h < NH; ++h) tma_load_4d(kdst + h * 2048, &map_k, bar, h * 64, c1, c2, c3);
+      for (int h = 0; h < NH; ++h) tma_load_4d(kdst + h * 2048, &map_k, bar, h * 64, c1, c2, c3, kv_policy);
 #pragma unroll
-      for (int h = 0; h < NH; ++h) tma_load_4d(vdst + h * 2048, &map_v, bar, h * 64, c1, c2, c3);
+      for (int h = 0; h < NH; ++h) tma_load_4d(vdst + h * 2048, &map_v, bar, h * 64, c1, c2, c3, kv_policy);
     }
   };
 
