@@ -566,9 +566,31 @@ def kv_migration_measure(rep: Replica, reps: int = 10):
         ms = e0.elapsed_time(e1) / reps
         moved = 2 * 2 * total * w.num_kv_heads * w.head_dim * 2    # K and V, read and write
         res[what] = {"ms": ms, "copy_gbs": moved / (ms * 1e-3) / 1e9}
+    # the paper's offload / reload: the dense buffer in pinned host memory, written and read over the bus by the kernels
+    host = {}
+    if total * w.num_kv_heads * w.head_dim * 2 * 2 <= (6 << 30):
+        kh = torch.empty((total, w.num_kv_heads, w.head_dim), dtype=torch.bfloat16).pin_memory()
+        vh = torch.empty_like(kh).pin_memory()
+        for what in ("gather", "scatter"):
+            def one_h():
+                if what == "gather":
+                    rep.h.kv_gather(k.data_ptr(), v.data_ptr(), *args, kh.data_ptr(), vh.data_ptr(), err.data_ptr(), st)
+                else:
+                    rep.h.kv_scatter(kh.data_ptr(), vh.data_ptr(), *args, k.data_ptr(), v.data_ptr(), err.data_ptr(), st)
+            one_h()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(3):
+                one_h()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / 3
+            host[what] = {"ms": ms, "payload_gbs": 2 * total * w.num_kv_heads * w.head_dim * 2 / (ms * 1e-3) / 1e9}
+        del kh, vh
     assert int(err.item()) == 0
     peak, _ = measured_hbm_peak()
-    return {"sequences": int(len(rows)), "tokens": total, "kv_bytes": 2 * total * w.num_kv_heads * w.head_dim * 2,
+    return {"sequences": int(len(rows)), "tokens": total, "pinned_host": host, "kv_bytes": 2 * total * w.num_kv_heads * w.head_dim * 2,
             "gather": res["gather"], "scatter": res["scatter"],
             "gather_frac_of_measured_copy": res["gather"]["copy_gbs"] / peak,
             "scatter_frac_of_measured_copy": res["scatter"]["copy_gbs"] / peak,

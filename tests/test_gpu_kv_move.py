@@ -146,3 +146,46 @@ def test_decode_is_unchanged_by_a_head_reshard(lib):
     again = H.bf16_dev_to_f32(r8.run(H.to_dev(q, dev), back_k, back_v, dbt, lens_a))
     assert np.array_equal(again, base)
     r8.h.close(); src.close()
+
+
+def test_offload_to_pinned_host_memory_and_reload(lib):
+    """The dense buffer in pinned host memory (the paper's offload target): the gather kernel writes it over the bus,
+    the scatter kernel reads it back into a pool with a new page placement; both exact."""
+    import torch
+    dev = torch.device("cuda:0")
+    lens = [700, 33, 1, 2049]
+    B, Hkv, d = len(lens), 4, 128
+    lens_a, bt, q, k, v = W.random_case(95, B, Hkv, Hkv, d, lens, poison=False)
+    h = lib.Handle(Hkv, Hkv, d, k.shape[0], B, bt.shape[1])
+    offs = np.concatenate([[0], np.cumsum(lens_a.astype(np.int64))])
+    total = int(offs[-1])
+    dk, dv, dbt = (H.to_dev(x, dev) for x in (k, v, bt))
+    dl = torch.from_numpy(lens_a.copy()).to(dev)
+    doffs = dev_i64(offs[:-1], dev)
+    err = torch.zeros(1, dtype=torch.int32, device=dev)
+    k_host = torch.full((total, Hkv, d), 0x7FC0, dtype=torch.int16).pin_memory()
+    v_host = torch.full((total, Hkv, d), 0x7FC0, dtype=torch.int16).pin_memory()
+    st = torch.cuda.current_stream().cuda_stream
+    h.kv_gather(dk.data_ptr(), dv.data_ptr(), dbt.data_ptr(), dl.data_ptr(), doffs.data_ptr(), B, int(lens_a.max()),
+                0, Hkv, k_host.data_ptr(), v_host.data_ptr(), err.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    assert np.array_equal(k_host.numpy().view(np.uint16), M.gather(k, bt, lens_a, 0, Hkv))
+    assert np.array_equal(v_host.numpy().view(np.uint16), M.gather(v, bt, lens_a, 0, Hkv))
+    rng = np.random.default_rng(6)
+    bt2, pool2 = W.draw_block_table(lens_a, int(W.pages_needed(lens_a).sum()) + 3, rng, ld=bt.shape[1])
+    h2 = lib.Handle(Hkv, Hkv, d, pool2, B, bt.shape[1])
+    k2 = torch.full((pool2, Hkv, 16, d), -1, dtype=torch.int16, device=dev)
+    v2 = torch.full((pool2, Hkv, 16, d), -1, dtype=torch.int16, device=dev)
+    dbt2 = H.to_dev(bt2, dev)
+    h2.kv_scatter(k_host.data_ptr(), v_host.data_ptr(), dbt2.data_ptr(), dl.data_ptr(), doffs.data_ptr(), B,
+                  int(lens_a.max()), 0, Hkv, k2.data_ptr(), v2.data_ptr(), err.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    want_k = np.full((pool2, Hkv, 16, d), 0xFFFF, np.uint16)
+    want_v = np.full((pool2, Hkv, 16, d), 0xFFFF, np.uint16)
+    M.scatter(M.gather(k, bt, lens_a, 0, Hkv), want_k, bt2, lens_a, 0)
+    M.scatter(M.gather(v, bt, lens_a, 0, Hkv), want_v, bt2, lens_a, 0)
+    assert np.array_equal(k2.cpu().numpy().view(np.uint16), want_k)
+    assert np.array_equal(v2.cpu().numpy().view(np.uint16), want_v)
+    h.close(); h2.close()
