@@ -176,6 +176,15 @@ int libra_set_variant(libra_handle_t handle, int32_t warps, int32_t stages);
  * and block start-up overlap the predecessor's tail.  on = 0 makes every launch an ordinary one. */
 int libra_set_dependent_launch(libra_handle_t handle, int32_t on);
 
+/* Optional second output.  With a non-NULL lse_dev every later decode call (libra_decode_attn, _append, _multi,
+ * _static) also writes, for every row of q, the natural logarithm of the sum of its exponentiated scores,
+ * lse[b][row] = ln sum_t exp(s_t) with s_t = (q . k_t) * sm_scale, as float32 [batch, rows] (rows = q_len *
+ * num_q_heads); -inf for an empty sequence or a query token that sees nothing.  Together with `out` this is what
+ * merging the attention over several disjoint parts of one sequence needs (out = sum_i w_i out_i / sum_i w_i,
+ * w_i = exp(lse_i - max lse)).  The buffer is the caller's and must stay valid while calls use it; NULL switches
+ * the output off. */
+int libra_set_lse_output(libra_handle_t handle, float* lse_dev);
+
 /* Early prefetch, off by default: a PROMISE by the caller about the kernel that precedes each decode call in the
  * stream, namely that it writes none of: block_table, seq_lens (device), and the cached K/V rows of any token
  * other than each sequence's newest q_len + 1 tokens, counted by this call's seq_lens (a projection / rotary /

@@ -62,6 +62,7 @@ SIGNATURES = {
     "libra_set_dependent_launch": (C.c_int, [_vp, C.c_int32]),
     "libra_set_max_query_tokens": (C.c_int, [_vp, C.c_int32]),
     "libra_set_early_prefetch": (C.c_int, [_vp, C.c_int32]),
+    "libra_set_lse_output": (C.c_int, [_vp, _vp]),
     "libra_set_kv_dtype": (C.c_int, [_vp, C.c_int32, C.c_float, C.c_float]),
     "libra_decode_attn_multi": (C.c_int, [_vp, _vp, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_ring_step": (C.c_int, [C.c_int32, _vp, _vp, _vp, C.c_size_t, C.c_int32, _vp, C.c_uint32, C.c_uint32, _vp, C.c_int32,
@@ -297,6 +298,9 @@ class Handle:
 
     def set_kv_dtype(self, dtype: int, k_scale: float = 1.0, v_scale: float = 1.0) -> None:
         _check(lib.libra_set_kv_dtype(self._h, dtype, k_scale, v_scale), "libra_set_kv_dtype")
+
+    def set_lse_output(self, lse_ptr: int) -> None:
+        _check(lib.libra_set_lse_output(self._h, lse_ptr or None), "libra_set_lse_output")
 
     def set_early_prefetch(self, on: bool) -> None:
         _check(lib.libra_set_early_prefetch(self._h, 1 if on else 0), "libra_set_early_prefetch")

@@ -23,6 +23,7 @@ struct CombineParams {
   const float* partial_lse;  // [slot][Hq]
   const int32_t* seq_lens;
   __nv_bfloat16* out;        // [B][Hq][D]
+  float* lse_out;            // [B][Hq] natural-log sum of exponentials of each row, or null
   uint32_t* error_word;
   int32_t num_q_heads;
 };
@@ -32,9 +33,10 @@ constexpr int kCombineWarps = 4;
 // One warp merges the n (<= 64) partial results of one (sequence, head) row and writes the bf16 row.
 // Shared by the combine kernel and by the decode kernel's in-kernel merge, so both give the same bits.
 // Loads bypass L1 (the partials were written by other SMs, possibly during this very launch).
+// lse_out (nullable): the row's final LSE = M + ln(sum_i w_i) goes to lse_out[b * Hq + h].
 template <int D>
 __device__ __forceinline__ void combine_row(const float* partial_o, const float* partial_lse, __nv_bfloat16* out, int b,
-                                            int first, int n, int Hq, int h, int lane) {
+                                            int first, int n, int Hq, int h, int lane, float* lse_out = nullptr) {
   constexpr int V = D / 32;  // columns per lane: 4 (float4) or 2 (float2)
   const float* lse = partial_lse + int64_t(first) * Hq + h;
   const float l0 = (lane < n) ? __ldcg(lse + int64_t(lane) * Hq) : -INFINITY;
@@ -79,6 +81,7 @@ __device__ __forceinline__ void combine_row(const float* partial_o, const float*
     }
   }
   const float inv = (den > 0.f) ? 1.f / den : 0.f;
+  if (lse_out != nullptr && lane == 0) lse_out[int64_t(b) * Hq + h] = (den > 0.f) ? m + __logf(den) : -INFINITY;
   __nv_bfloat16* dst = out + (int64_t(b) * Hq + h) * D + lane * V;
 #pragma unroll
   for (int v = 0; v < V; v += 2) {
@@ -102,7 +105,7 @@ combine_kernel(const __grid_constant__ CombineParams p, const __grid_constant__ 
   if (lane == 0 && h == 0 && fix.w != __ldg(p.seq_lens + fix.x)) {
     atomicOr(p.error_word, LIBRA_DEV_ERR_SEQ_LEN_MISMATCH);
   }
-  combine_row<D>(p.partial_o, p.partial_lse, p.out, fix.x, fix.y, fix.z, Hq, h, lane);
+  combine_row<D>(p.partial_o, p.partial_lse, p.out, fix.x, fix.y, fix.z, Hq, h, lane, p.lse_out);
 }
 
 }  // namespace libra

@@ -39,6 +39,7 @@ struct DecodeParams {
   const int32_t* block_table;
   const int32_t* seq_lens;
   __nv_bfloat16* out;
+  float* lse_out;        // [B][rows] natural-log sum of exponentials of every row of q, or null
   const int4* entries;   // work items then empty-sequence entries in device memory, or null: in `pp`
   const int32_t* dev_counts;  // device-side plan: the counts below are read from here (null = host plan)
   float* partial_o;      // [slot][Hq][D]
@@ -583,6 +584,9 @@ __device__ __forceinline__ void merge_and_write(const DecodeParams& p, const Uni
     const int64_t head = col_row(p, u.kvh, h);
     if (u.slot < 0) {
       p.out[(int64_t(u.b) * p.num_q_heads + head) * D + dim] = __float2bfloat16_rn(o);
+      if (p.lse_out != nullptr && dim == 0) {
+        p.lse_out[int64_t(u.b) * p.num_q_heads + head] = (den > 0.f) ? (m_all + lg2(den)) * 0.6931471805599453f : -INFINITY;
+      }
     } else {
       p.partial_o[(int64_t(u.slot) * p.num_q_heads + head) * D + dim] = o;
       if (dim == 0) {
@@ -604,6 +608,9 @@ __device__ __forceinline__ void zero_empty_row(const DecodeParams& p, const int4
                                                int nthreads) {
   const int64_t row = int64_t(entries[num_items + e].x) * p.num_q_heads * D;
   for (int i = tid; i < p.num_q_heads * D; i += nthreads) p.out[row + i] = __float2bfloat16_rn(0.f);
+  if (p.lse_out != nullptr) {
+    for (int i = tid; i < p.num_q_heads; i += nthreads) p.lse_out[row / D + i] = -INFINITY;
+  }
 }
 
 // Programmatic dependent launch, both ends.  launch_dependents: kernels queued behind this one may have
@@ -871,7 +878,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   // one warp per column of this KV head, exactly as the combine kernel would do it
   for (int c = warp; c < p.cols; c += NW) {
     combine_row<D>(p.partial_o, p.partial_lse, p.out, u.b, u.slot - u.chunk_j, u.n_chunks, p.num_q_heads,
-                   col_row(p, kvh, c), lane);
+                   col_row(p, kvh, c), lane, p.lse_out);
   }
 }
 

@@ -145,6 +145,7 @@ struct libra_handle_s {
   void* clean_workspace = nullptr;  // workspace whose control words and counters are known to be zero
   int combine_mode = 1;     // 0: separate kernel, 1: inside the decode kernel
   bool pdl = true;          // programmatic dependent launches (decode after its predecessor, combine after decode)
+  float* lse_out = nullptr;     // optional second output of the step (libra_set_lse_output)
   bool early_prefetch = false;  // the caller's promise about the preceding kernel (libra_set_early_prefetch)
 
   // pinned staging for uploads of plans too large for the kernel parameters
@@ -721,6 +722,12 @@ int libra_set_kv_dtype(libra_handle_t h, int32_t dtype, float k_scale, float v_s
   return LIBRA_OK;
 }
 
+int libra_set_lse_output(libra_handle_t h, float* lse_dev) {
+  if (!h || reinterpret_cast<uintptr_t>(lse_dev) % 4 != 0) return LIBRA_INVALID_ARGUMENT;
+  h->lse_out = lse_dev;
+  return LIBRA_OK;
+}
+
 int libra_set_early_prefetch(libra_handle_t h, int32_t on) {
   if (!h || (on != 0 && on != 1)) return LIBRA_INVALID_ARGUMENT;
   h->early_prefetch = (on == 1);
@@ -821,6 +828,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     p.block_table = block_table;
     p.seq_lens = seq_lens;
     p.out = static_cast<__nv_bfloat16*>(out);
+    p.lse_out = loads_only ? nullptr : h->lse_out;
     p.entries = entries_dev;
     p.dev_counts = dev_counts;
     p.partial_o = reinterpret_cast<float*>(ws + h->o_off);
@@ -887,6 +895,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     c.partial_lse = reinterpret_cast<const float*>(ws + h->lse_off);
     c.seq_lens = seq_lens;
     c.out = static_cast<__nv_bfloat16*>(out);
+    c.lse_out = h->lse_out;
     c.error_word = err_dev;
     c.num_q_heads = rows;
     // a programmatic dependent of the decode kernel: it may be scheduled while that kernel drains and
