@@ -422,6 +422,48 @@ def fp8_cache_measure(rep: Replica, steps: int = 200, variant=None):
             "pool_copies": copies, "steps": steps}
 
 
+def nhd_layout_measure(rep: Replica, steps: int = 200):
+    """The same step with the pools laid out token-major inside a page (NHD: [page, token, head, d]); same values,
+    same block tables.  A (page, head) tile is then 16 rows of 256 bytes, 2 KB apart."""
+    torch, w = rep.torch, rep.w
+    if rep.pool_bytes * len(rep.pools) > (24 << 30):
+        return None
+    pools = [(k.permute(0, 2, 1, 3).contiguous(), v.permute(0, 2, 1, 3).contiguous()) for k, v in rep.pools]
+    P = w.page_size
+    strides = (P * w.num_kv_heads * w.head_dim, w.head_dim, w.num_kv_heads * w.head_dim)
+    h = rep.binding.Handle(w.num_q_heads, w.num_kv_heads, w.head_dim, rep.layouts[0].pool_pages, w.batch, rep.ld,
+                           device=rep.dev.index or 0, kv_strides=strides)
+    ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=rep.dev)
+    out = torch.zeros_like(rep.out)
+    st = torch.cuda.current_stream().cuda_stream
+
+    def step(i):
+        s = i % len(rep.layouts)
+        k, v = pools[i % len(pools)]
+        h.plan(rep.layouts[s].seq_lens, ws.data_ptr(), ws.numel(), st)
+        h.decode_attn(rep.q.data_ptr(), k.data_ptr(), v.data_ptr(), rep.bts[s].data_ptr(), rep.lens_dev[s].data_ptr(),
+                      out.data_ptr(), st)
+
+    steps = max(len(rep.layouts), steps // len(rep.layouts) * len(rep.layouts))
+    for i in range(10):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    assert h.debug_error_word() == 0, "device error word set"
+    same = bool(torch.equal(out, rep.out)) if len(rep.layouts) == 1 else None
+    h.close()
+    del pools
+    torch.cuda.empty_cache()
+    ms = e0.elapsed_time(e1) / steps
+    return {"ms_per_step": ms, "kv_gbs": rep.kv_bytes_per_step / (ms * 1e-3) / 1e9, "steps": steps,
+            "same_bits_as_hnd": same}
+
+
 def ring_step_measure(rep: Replica, reps: int = 40):
     """The ring all-reduce's data-plane step (libra_ring_step, flag already set) on 16 MB float32 chunks, the chunk
     size the paper pipelines with: payload rate of a reduce step on 2 and on 4 thread blocks (= SMs)."""
@@ -775,6 +817,8 @@ def run_libra(args):
             line["multi_token"] = [m for m in (multi_token_measure(rep, t) for t in (2, 4)) if m]
         if "fp8_cache" in extras:
             line["fp8_cache"] = fp8_cache_measure(rep, steps=min(200, max(10, args.steps)))
+        if "nhd_layout" in extras:
+            line["nhd_layout"] = nhd_layout_measure(rep)
         if "ring_step" in extras:
             line["ring_step"] = ring_step_measure(rep)
         if "kv_migration" in extras and args.workload in ("longtail_mix_b256", "straggler_b8"):
@@ -815,6 +859,7 @@ def run_libra(args):
             others[name]["ceilings"] = ceilings_measure(r, reps=10)
             others[name]["multi_token"] = [m for m in (multi_token_measure(r, t, 60) for t in (2, 3, 4)) if m]
             others[name]["fp8_cache"] = fp8_cache_measure(r, 60)
+            others[name]["nhd_layout"] = nhd_layout_measure(r, 60)
             if name in ("longtail_mix_b256", "straggler_b8"):  # migrating the long sequences: gather to a dense buffer, scatter back
                 others[name]["kv_migration"] = kv_migration_measure(r)
             if name == "shift_b128":  # the re-planned-every-step workload: also with the device-side planner
@@ -847,7 +892,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
-    ap.add_argument("--extras", default="ceilings,early_prefetch,multi_token,fp8_cache,kv_migration,ring_step",
+    ap.add_argument("--extras", default="ceilings,early_prefetch,multi_token,fp8_cache,nhd_layout,kv_migration,ring_step",
                     help="side measurements on the main workload at N=1 (comma list; empty = none)")
     ap.add_argument("--variant", default="", help="warps,stages of the decode block (default: the library's)")
     ap.add_argument("--ctas-per-sm", type=int, default=0, help="planner constant (0 = default)")
