@@ -427,7 +427,7 @@ int libra_trie_route(libra_trie_t trie, int64_t prompt_id, const int32_t* states
  * In the paper the CPU owns membership, transport and flow control of the gradient exchange between replicas; the
  * GPU runs only the copy / reduce steps of a ring ReduceScatter + AllGather, polls a host-pinned arrival flag with a
  * software timeout instead of blocking, and uses 2 SMs.  libra_ring_step enqueues ONE such step on `stream` of
- * `device`:
+ * `device` (a one-thread kernel that waits and writes the verdict, then the copy / reduce kernel, which acts on it):
  *   wait until *ready_flag >= expected (ready_flag: host-pinned mapped memory or device memory, 4-byte aligned; the
  *   producer writes the chunk first, then the flag), for at most timeout_us microseconds (1 .. 10,000,000);
  *   then  own != NULL : dst[i] = own[i] + received[i]   (a ReduceScatter step; LIBRA_RING_F32: float32 addition;

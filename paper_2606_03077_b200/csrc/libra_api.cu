@@ -1165,11 +1165,10 @@ int libra_ring_step(int32_t device, void* dst, const void* own, const void* rece
   p.own = own;
   p.received = received;
   p.n16 = bytes / 16;
-  p.ready = ready_flag;
-  p.expected = expected;
-  p.timeout_us = timeout_us;
   p.status = status_dev;
   p.bf16 = (dtype == LIBRA_RING_BF16) ? 1 : 0;
+  libra::ring_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ready_flag, expected, timeout_us, status_dev);
+  if (cudaGetLastError() != cudaSuccess) return LIBRA_CUDA_ERROR;
   libra::ring_step_kernel<<<unsigned(num_blocks == 0 ? 2 : num_blocks), libra::kRingThreads, 0,
                             static_cast<cudaStream_t>(stream)>>>(p);
   if (cudaGetLastError() != cudaSuccess) return LIBRA_CUDA_ERROR;

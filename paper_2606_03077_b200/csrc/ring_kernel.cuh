@@ -12,8 +12,8 @@
 //   COPY   : dst[i] = received[i]                     one AllGather step        and rounded to nearest even)
 //
 // A few blocks (2 by default) of 512 threads; every thread keeps kRingUnroll 16-byte loads of each operand in flight,
-// which is what lets so few SMs stream at a useful rate.  If the wait runs out the kernel writes nothing but the
-// status word and returns; the context stays usable.
+// which is what lets so few SMs stream at a useful rate.  If the wait runs out nothing but the status word is
+// written; the context stays usable.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -30,10 +30,7 @@ struct RingStepParams {
   const void* own;            // null for COPY
   const void* received;
   size_t n16;                 // 16-byte vectors (whole vectors only; the caller pads chunks to 16 bytes)
-  const uint32_t* ready;      // arrival flag (host-pinned, mapped, or device memory)
-  uint32_t expected;
-  uint32_t timeout_us;
-  uint32_t* status;           // device word: 0 = done, 1 = the wait ran out (nothing else was written)
+  const uint32_t* status;     // device word written by ring_wait_kernel: 0 = go, 1 = the wait ran out
   int32_t bf16;               // element type: 0 float32, 1 bfloat16
 };
 
@@ -77,29 +74,32 @@ __device__ __forceinline__ uint4 add16(uint4 a, uint4 b, bool bf16) {
 
 }  // namespace dev
 
-// grid = a few blocks (2 by default), block = kRingThreads
+// The wait is a kernel of its own, one thread: it polls the flag, bounded by the clock (timeout_us) and by an
+// iteration count, and writes the verdict to the status word.  The copy / reduce kernel behind it in the stream
+// reads the verdict, so all of its blocks agree on it (blocks polling on their own could disagree when the flag
+// arrives at the deadline), and no SM is held while waiting.
+__global__ void ring_wait_kernel(const uint32_t* ready, uint32_t expected, uint32_t timeout_us, uint32_t* status) {
+  using namespace dev;
+  if (threadIdx.x != 0) return;
+  const uint64_t t0 = global_timer_ns();
+  const uint64_t limit = uint64_t(timeout_us) * 1000ull;
+  uint32_t verdict = 1u;
+  for (uint32_t it = 0; it < (1u << 26); ++it) {
+    if (ld_flag(ready) >= expected) {
+      verdict = 0u;
+      break;
+    }
+    if (global_timer_ns() - t0 > limit) break;
+    __nanosleep(200);
+  }
+  __threadfence_system();   // the chunk was written before the flag: what follows in the stream reads it after the flag
+  *status = verdict;
+}
+
+// grid = a few blocks (2 by default), block = kRingThreads; runs behind ring_wait_kernel in the same stream
 __global__ void __launch_bounds__(kRingThreads) ring_step_kernel(const RingStepParams p) {
   using namespace dev;
-  __shared__ int s_go;
-  if (threadIdx.x == 0) {
-    // bounded wait: by the clock (timeout_us) and by an iteration count, whichever ends first
-    const uint64_t t0 = global_timer_ns();
-    const uint64_t limit = uint64_t(p.timeout_us) * 1000ull;
-    int go = 0;
-    for (uint32_t it = 0; it < (1u << 26); ++it) {
-      if (ld_flag(p.ready) >= p.expected) {
-        go = 1;
-        break;
-      }
-      if (global_timer_ns() - t0 > limit) break;
-      __nanosleep(200);
-    }
-    if (go) __threadfence_system();   // the chunk was written before the flag: order our reads after the flag
-    s_go = go;
-    if (blockIdx.x == 0) *p.status = go ? 0u : 1u;
-  }
-  __syncthreads();
-  if (!s_go) return;
+  if (*p.status != 0u) return;   // the wait ran out: write nothing
 
   const uint4* recv = static_cast<const uint4*>(p.received);
   const uint4* own = static_cast<const uint4*>(p.own);
