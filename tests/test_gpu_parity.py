@@ -395,3 +395,20 @@ def test_early_prefetch_is_bit_identical_behind_a_cache_write_kernel(lib):
         vv[bt[b, (lens_a[b] - 1) // 16], :, (lens_a[b] - 1) % 16] = new_v[-1][b]
     ref, _ = O.paged_decode_attention(new_q[-1], kk, vv, bt, lens_a)
     check(results[True][-1], ref, "early prefetch, last step")
+
+
+def test_block_shape_follows_the_longest_unit(lib):
+    """Left to itself the library runs a host plan whose units are all short on the small block shape (4 warps x 2
+    stages, three blocks per SM) and everything else on the default one: same bits as asking for that shape."""
+    short = [1, 100, 333, 1024, 16, 700, 0, 512]
+    mixed = short + [40000]          # the base chunk length grows with the total: units of over 2000 tokens
+    for lens, shape in ((short, (4, 2)), (mixed, (8, 3))):
+        lens_a, bt, q, k, v = W.random_case(111, len(lens), 32, 8, 128, lens)
+        ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
+        auto = H.run_host_case(lib, q, k, v, bt, lens_a)
+        check(auto, ref, f"auto shape, longest {max(lens)}")
+        for variant in ((4, 2), (8, 3)):
+            forced = H.run_host_case(lib, q, k, v, bt, lens_a, variant=variant)
+            check(forced, ref, f"variant {variant}")
+            if variant == shape:
+                assert np.array_equal(forced, auto)
