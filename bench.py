@@ -464,6 +464,59 @@ def nhd_layout_measure(rep: Replica, steps: int = 200):
             "same_bits_as_hnd": same}
 
 
+def short_batch_measure(rep: Replica, steps: int = 100):
+    """Batches of equally long, short sequences at a constant 262,144 cached tokens (1.07 GB of KV at 8 KV heads, d 128):
+    the block shape the library picks by itself against the default large shape forced."""
+    torch, W, w = rep.torch, rep.W, rep.w
+    if w.head_dim != 128 or w.num_kv_heads != 8:
+        return None
+    from numpy.random import Generator, PCG64
+    res = []
+    total = 262144
+    npg = total // 16
+    copies = 4
+    pool = npg * copies
+    k = torch.randn((pool, 8, 16, 128), device=rep.dev, dtype=torch.bfloat16)
+    v = torch.randn((pool, 8, 16, 128), device=rep.dev, dtype=torch.bfloat16)
+    perm = Generator(PCG64(1)).permutation(pool)
+    st = torch.cuda.current_stream().cuda_stream
+    for L in (128, 256, 512, 1024):
+        Bn = total // L
+        lens = np.full(Bn, L, dtype=np.int32)
+        bts = [torch.from_numpy(perm[c * npg:(c + 1) * npg].reshape(Bn, -1).astype(np.int32)).to(rep.dev) for c in range(copies)]
+        lens_dev = torch.from_numpy(lens).to(rep.dev)
+        q = torch.randn((Bn, w.num_q_heads, 128), device=rep.dev, dtype=torch.bfloat16)
+        out = torch.zeros_like(q)
+        row = {"tokens_per_sequence": L, "batch": Bn}
+        for label, variant in (("auto_shape", None), ("default_shape_forced", (8, 3))):
+            h = rep.binding.Handle(w.num_q_heads, 8, 128, pool, Bn, bts[0].shape[1], device=rep.dev.index or 0)
+            if variant:
+                h.set_variant(*variant)
+            ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=rep.dev)
+
+            def step(i):
+                h.plan(lens, ws.data_ptr(), ws.numel(), st)
+                h.decode_attn(q.data_ptr(), k.data_ptr(), v.data_ptr(), bts[i % copies].data_ptr(), lens_dev.data_ptr(),
+                              out.data_ptr(), st)
+            for i in range(8):
+                step(i)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(steps):
+                step(i)
+            e1.record()
+            torch.cuda.synchronize()
+            assert h.debug_error_word() == 0, "device error word set"
+            h.close()
+            ms = e0.elapsed_time(e1) / steps
+            row[label] = {"ms_per_step": ms, "kv_gbs": total * 8 * 128 * 4 / (ms * 1e-3) / 1e9}
+        res.append(row)
+    del k, v
+    torch.cuda.empty_cache()
+    return res
+
+
 def ring_step_measure(rep: Replica, reps: int = 40):
     """The ring all-reduce's data-plane step (libra_ring_step, flag already set) on 16 MB float32 chunks, the chunk
     size the paper pipelines with: payload rate of a reduce step on 2 and on 4 thread blocks (= SMs)."""
@@ -831,6 +884,8 @@ def run_libra(args):
             line["fp8_cache"] = fp8_cache_measure(rep, steps=min(200, max(10, args.steps)))
         if "nhd_layout" in extras:
             line["nhd_layout"] = nhd_layout_measure(rep)
+        if "short_batch" in extras:
+            line["short_batch"] = short_batch_measure(rep)
         if "ring_step" in extras:
             line["ring_step"] = ring_step_measure(rep)
         if "kv_migration" in extras and args.workload in ("longtail_mix_b256", "straggler_b8"):
@@ -904,7 +959,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
-    ap.add_argument("--extras", default="ceilings,early_prefetch,multi_token,fp8_cache,nhd_layout,kv_migration,ring_step",
+    ap.add_argument("--extras", default="ceilings,early_prefetch,multi_token,fp8_cache,nhd_layout,short_batch,kv_migration,ring_step",
                     help="side measurements on the main workload at N=1 (comma list; empty = none)")
     ap.add_argument("--variant", default="", help="warps,stages of the decode block (default: the library's)")
     ap.add_argument("--ctas-per-sm", type=int, default=0, help="planner constant (0 = default)")
