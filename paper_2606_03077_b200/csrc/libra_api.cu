@@ -58,17 +58,20 @@ Variant make_variant() {
 // Block shapes that are compiled in.  Defaults: index 0 (8 warps x 3 stages) for one column tile, index 1
 // (12 x 2) for two: twice the tensor-core and softmax work per tile wants a third warp per scheduler to hide
 // its latency (measured 2.5 - 4 % faster there, 0.5 - 1 % slower with one tile).
-constexpr int kVariantOneTile = 0, kVariantTwoTiles = 1, kVariantShortUnits = 4;
+constexpr int kVariantOneTile = 0, kVariantTwoTiles = 1, kVariantShortUnits = 4, kVariantTinyUnits = 9;
 // A block costs ~4 us of start-up and epilogue whatever its size and the default block is alone on its SM, so a batch
 // of short sequences leaves the SMs waiting most of the time.  When no unit of a host plan is longer than this many
 // tokens, 4 warps x 2 stages (64 KB: three blocks per SM, three units in flight) is used instead: the same bytes in
-// flight per SM, measured 2.2x / 1.6x / 1.16x / 1.05x faster at 128 / 256 / 512 / 1024 tokens per sequence.  A long unit
-// on such a block would stream at a third of the SM's rate, hence only when there is none.
+// flight per SM, measured 1.6x / 1.16x / 1.05x faster at 256 / 512 / 1024 tokens per sequence; and when none is longer
+// than kTinyUnitTokens, 2 warps x 2 stages (32 KB, seven blocks per SM): 2.6x at 128 tokens.  A long unit on such a
+// block would stream at a fraction of the SM's rate, hence only when there is none.
 constexpr int kShortUnitTokens = 1024;
+constexpr int kTinyUnitTokens = 256;
 const std::vector<Variant>& variants() {
   static const std::vector<Variant> v = {
       make_variant<8, 3>(), make_variant<12, 2>(), make_variant<8, 2>(), make_variant<4, 3>(), make_variant<4, 2>(),
       make_variant<4, 4>(), make_variant<4, 6>(), make_variant<2, 6>(), make_variant<2, 4>(),
+      make_variant<2, 2>(),
   };
   return v;
 }
@@ -820,9 +823,10 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
   const int di = (h->cfg.head_dim == 128) ? 1 : 0;
   const int ni = (h->group * q_len > 8) ? 1 : 0;
   int auto_variant = ni ? kVariantTwoTiles : kVariantOneTile;
-  if (!ni && !h->device_planned && !h->plan.items.empty() &&
-      h->plan.items.front().kv_end - h->plan.items.front().kv_begin <= kShortUnitTokens) {
-    auto_variant = kVariantShortUnits;   // items are sorted longest first
+  if (!ni && !h->device_planned && !h->plan.items.empty()) {
+    const int longest = h->plan.items.front().kv_end - h->plan.items.front().kv_begin;   // items are sorted longest first
+    if (longest <= kTinyUnitTokens) auto_variant = kVariantTinyUnits;
+    else if (longest <= kShortUnitTokens) auto_variant = kVariantShortUnits;
   }
   const Variant& v = variants()[h->variant >= 0 ? h->variant : auto_variant];
   const int32_t rows = q_len * h->cfg.num_q_heads;   // rows of q / out per sequence

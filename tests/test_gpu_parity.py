@@ -87,7 +87,7 @@ def test_every_block_shape_agrees(lib):
     lens = [2500, 300, 17, 4100]
     lens_a, bt, q, k, v = W.random_case(7, 4, 32, 8, 128, lens)
     ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
-    for variant in [(4, 3), (4, 2), (4, 4), (4, 6), (8, 2), (8, 3), (2, 6), (2, 4), (12, 2)]:
+    for variant in [(4, 3), (4, 2), (4, 4), (4, 6), (8, 2), (8, 3), (2, 6), (2, 4), (12, 2), (2, 2)]:
         got = H.run_host_case(lib, q, k, v, bt, lens_a, plan=lib.PlanParams(8, 1, 2, 256, 256, 64), variant=variant)
         check(got, ref, f"variant {variant}")
 
@@ -398,16 +398,18 @@ def test_early_prefetch_is_bit_identical_behind_a_cache_write_kernel(lib):
 
 
 def test_block_shape_follows_the_longest_unit(lib):
-    """Left to itself the library runs a host plan whose units are all short on the small block shape (4 warps x 2
-    stages, three blocks per SM) and everything else on the default one: same bits as asking for that shape."""
+    """Left to itself the library runs a host plan whose units are all short on a small block shape (4 warps x 2
+    stages, three blocks per SM; 2 x 2, seven per SM, when none exceeds 256 tokens) and everything else on the default
+    one: same bits as asking for that shape."""
+    tiny = [1, 100, 256, 16, 0, 33]
     short = [1, 100, 333, 1024, 16, 700, 0, 512]
     mixed = short + [40000]          # the base chunk length grows with the total: units of over 2000 tokens
-    for lens, shape in ((short, (4, 2)), (mixed, (8, 3))):
+    for lens, shape in ((tiny, (2, 2)), (short, (4, 2)), (mixed, (8, 3))):
         lens_a, bt, q, k, v = W.random_case(111, len(lens), 32, 8, 128, lens)
         ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
         auto = H.run_host_case(lib, q, k, v, bt, lens_a)
         check(auto, ref, f"auto shape, longest {max(lens)}")
-        for variant in ((4, 2), (8, 3)):
+        for variant in ((2, 2), (4, 2), (8, 3)):
             forced = H.run_host_case(lib, q, k, v, bt, lens_a, variant=variant)
             check(forced, ref, f"variant {variant}")
             if variant == shape:
