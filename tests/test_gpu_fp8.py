@@ -273,3 +273,29 @@ def test_gather_and_scatter_of_8bit_pools(lib):
     M.scatter(M.gather(v8, bt, lens_a, h0, hn), want_v, bt2, lens_a, 0)
     assert np.array_equal(k2.cpu().numpy(), want_k) and np.array_equal(v2.cpu().numpy(), want_v)
     h.close(); h2.close()
+
+
+def test_block_shape_follows_the_longest_unit(lib):
+    # batches of short units run on small blocks (several per SM): same bits as asking for that shape, right answers
+    import torch
+    for lens, shape in (([1, 100, 256, 16, 0, 33], (2, 4)), ([1, 100, 333, 1024, 16, 700, 0, 512], (4, 2))):
+        lens_a, bt, q, k8, v8 = W.random_case_e4m3(640, len(lens), 32, 8, 128, lens)
+        ref, _ = O.paged_decode_attention_fp8(q, k8, v8, bt, lens_a, 0.5, 2.0)
+        auto = run_fp8(lib, q, k8, v8, bt, lens_a, 0.5, 2.0)
+        check(auto, ref, f"auto shape, longest {max(lens)}")
+        dev = torch.device("cuda:0")
+        h = lib.Handle(32, 8, 128, k8.shape[0], len(lens), bt.shape[1])
+        h.set_kv_dtype(lib.KV_E4M3, 0.5, 2.0)
+        h.set_variant(*shape)
+        ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=dev)
+        qd, btd = H.to_dev(q, dev), H.to_dev(bt, dev)
+        kd, vd = torch.from_numpy(k8).to(dev), torch.from_numpy(v8).to(dev)
+        lens_dev = torch.from_numpy(lens_a).to(dev)
+        out = torch.full(q.shape, H.CANARY, dtype=torch.int16, device=dev)
+        st = torch.cuda.current_stream().cuda_stream
+        h.plan(lens_a, ws.data_ptr(), ws.numel(), st)
+        h.decode_attn(qd.data_ptr(), kd.data_ptr(), vd.data_ptr(), btd.data_ptr(), lens_dev.data_ptr(), out.data_ptr(), st)
+        torch.cuda.synchronize()
+        assert h.debug_error_word() == 0
+        assert np.array_equal(H.bf16_dev_to_f32(out), auto)
+        h.close()
