@@ -165,8 +165,8 @@ int libra_set_kv_dtype(libra_handle_t handle, int32_t dtype, float k_scale, floa
 /* Tuning knob: shape of the decode thread block: `warps` warps that each own `stages` shared-memory
  * stages of one K page plus one V page.  Only the compiled-in shapes are accepted (UNSUPPORTED_SHAPE
  * otherwise); the default is the tuned one (8 x 3; 4 x 2, three blocks per SM, when no unit of a host plan exceeds
- * 1024 tokens, and 2 x 2, seven per SM, when none exceeds 256; 12 x 2 when a KV head serves more than 8 rows of q; with an E4M3 cache, whose tiles are half the size, 16 x 3, 8 x 6
- * for two column tiles, and 4 x 2 / 2 x 4 for short units).  Results do not depend on the stage count; the warp
+ * 1024 tokens, and 2 x 2, seven per SM, when none exceeds 256; 12 x 2 when a KV head serves more than 8 rows of q; with an E4M3 cache, whose tiles are half the size, 16 x 3, 8 x 6 for
+ * two column tiles, and 4 x 2 / 2 x 4 for short units).  Results do not depend on the stage count; the warp
  * count changes the order of the per-unit merge and hence the last bits of the result. */
 int libra_set_variant(libra_handle_t handle, int32_t warps, int32_t stages);
 

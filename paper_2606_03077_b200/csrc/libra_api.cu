@@ -86,10 +86,13 @@ const int kLoadsOnlySmem[2] = {libra::DecodeSmem<64, kLoadsOnlyWarps, kLoadsOnly
                                libra::DecodeSmem<128, kLoadsOnlyWarps, kLoadsOnlyStages>::kDynamicBytes};
 
 // 8-bit (E4M3) cache, head_dim 128: block shapes compiled in.  Half the bytes per tile leave half the time per tile,
-// and two warps per scheduler cannot hide the conversion -> mma -> softmax chain in it: 16 warps x 3 stages of
-// 4 KB is the default where the registers allow it (one column tile), 8 x 6 otherwise; batches of short units get
-// 4 x 2 (index 4) or, up to kTinyUnitTokens, 2 x 4 (index 5): 32 KB, seven blocks per SM, measured 1.4x / 1.9x / 2.6x /
-// 3.5x faster than 16 x 3 at 1024 / 512 / 256 / 128 tokens per sequence.  fn[loads only][NT - 1]
+// and two warps per scheduler cannot hide the conversion -> mma -> softmax chain in it, so 16 warps per SM are wanted:
+// one block of 16 warps x 3 stages of 4 KB where the registers allow it (one column tile), 8 x 6 otherwise.  (Two blocks
+// of 8 x 3 per SM instead: 5 % faster on the long mix and 3 % on the headline workload, 2 % slower on 8 equal long
+// sequences and 5 % on the drifting workload: no clear winner, available through libra_set_variant.)  Batches of short
+// units get 4 x 2 or, up to kTinyUnitTokens, 2 x 4 (32 KB, seven blocks per SM: 1.4x / 1.9x / 2.6x / 3.5x faster than
+// 16 x 3 at 1024 / 512 / 256 / 128 tokens per sequence).  fn[loads only][NT - 1]
+constexpr int kFp8OneTile = 2, kFp8TwoTiles = 1, kFp8ShortUnits = 5, kFp8TinyUnits = 6;
 struct Fp8Variant {
   int warps, stages;
   DecodeKernelFn fn[2][2];
@@ -108,8 +111,9 @@ Fp8Variant make_fp8_variant() {
   return v;
 }
 const std::vector<Fp8Variant>& fp8_variants() {
-  static const std::vector<Fp8Variant> v = {make_fp8_variant<16, 3>(), make_fp8_variant<8, 6>(), make_fp8_variant<16, 2>(),
-                                            make_fp8_variant<8, 4>(), make_fp8_variant<4, 2>(), make_fp8_variant<2, 4>()};
+  static const std::vector<Fp8Variant> v = {make_fp8_variant<8, 3>(), make_fp8_variant<8, 6>(), make_fp8_variant<16, 3>(),
+                                            make_fp8_variant<16, 2>(), make_fp8_variant<8, 4>(), make_fp8_variant<4, 2>(),
+                                            make_fp8_variant<2, 4>()};
   return v;
 }
 
@@ -887,9 +891,9 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     lc.blockDim = dim3(unsigned((loads_only ? kLoadsOnlyWarps : v.warps) * 32));
     lc.dynamicSmemBytes = size_t(loads_only ? kLoadsOnlySmem[di] : v.smem[di][ni]);
     if (h->fp8) {
-      int fp8_auto = ni;   // [0] = 16 x 3, [1] = 8 x 6
-      if (!ni && !loads_only && auto_variant == kVariantShortUnits) fp8_auto = 4;
-      if (!ni && !loads_only && auto_variant == kVariantTinyUnits) fp8_auto = 5;
+      int fp8_auto = ni ? kFp8TwoTiles : kFp8OneTile;
+      if (!ni && !loads_only && auto_variant == kVariantShortUnits) fp8_auto = kFp8ShortUnits;
+      if (!ni && !loads_only && auto_variant == kVariantTinyUnits) fp8_auto = kFp8TinyUnits;
       const Fp8Variant& fv = fp8_variants()[h->fp8_variant >= 0 ? h->fp8_variant : fp8_auto];
       fn = fv.fn[loads_only ? 1 : 0][ni];
       lc.blockDim = dim3(unsigned(fv.warps * 32));
