@@ -117,7 +117,7 @@ __device__ __forceinline__ uint64_t l2_evict_first_policy() {
   return pol;
 }
 
-// Tiled 4-D TMA load global -> shared (no multicast) with an L2 cache policy, completing on an mbarrier of this block.
+// Tiled 4-D TMA load global -> shared (one destination block only) with an L2 cache policy, completing on an mbarrier of this block.
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
                                             int c3, uint64_t policy) {
   asm volatile(
