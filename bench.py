@@ -803,12 +803,21 @@ def run_libra(args):
     import torch
 
     rank, local_rank, world = dist_env()
+    # one rank per GPU over NCCL; LIBRA_BENCH_BACKEND=gloo lets the N > 1 path be exercised where there are fewer
+    # GPUs than ranks (the replicas are independent: no kernel of one rank ever waits for another's)
+    backend = os.environ.get("LIBRA_BENCH_BACKEND", "nccl")
+    if backend != "nccl":
+        local_rank %= max(1, torch.cuda.device_count())
     if world > 1:
         import torch.distributed as dist
 
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        else:
+            dist.init_process_group(backend)
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
+    agg_dev = dev if backend == "nccl" else None
     barrier = (lambda: torch.distributed.barrier()) if world > 1 else None
 
     from paper_2606_03077_b200 import binding as _b
@@ -823,7 +832,7 @@ def run_libra(args):
     clocks = sampler.stop()
 
     units = rep.kv_bytes_per_step * args.steps
-    t_max, units_all = aggregate_over_ranks(elapsed_ms, units, world, dev)
+    t_max, units_all = aggregate_over_ranks(elapsed_ms, units, world, agg_dev)
     ms_per_step = t_max / args.steps
     value = units_all / (t_max * 1e-3) / 1e9
 
@@ -897,7 +906,7 @@ def run_libra(args):
         # end-to-end at N GPUs: every rank copies its own replica's inputs from its own pinned memory
         if not args.no_e2e:
             ms, h2d, d2h, same = e2e_measure(rep, args.e2e_steps)
-            t_e2e, u_e2e = aggregate_over_ranks(ms, rep.layouts[0].kv_bytes, world, dev)
+            t_e2e, u_e2e = aggregate_over_ranks(ms, rep.layouts[0].kv_bytes, world, agg_dev)
             line["e2e"] = {"value": u_e2e / (t_e2e * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": t_e2e,
                            "h2d_bytes_per_step": h2d * world, "d2h_bytes_per_step": d2h * world,
                            "steps": args.e2e_steps}
