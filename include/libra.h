@@ -290,6 +290,15 @@ int libra_decode_attn_append(libra_handle_t handle, const void* q, const void* k
                              void* k_pages, void* v_pages, const int32_t* block_table, const int32_t* seq_lens,
                              void* out, void* stream);
 
+/* Several query tokens with the append fused in: k_new and v_new hold the rows of the newest q_len tokens of every
+ * sequence, [batch, q_len, num_kv_heads, head_dim] in the cache's element type (token i of the block is token
+ * L_b - q_len + i of the sequence); they are written into their slots (which may lie in two pages) and the result
+ * is libra_decode_attn_multi's on the updated pools.  Sequences shorter than q_len take only their last L_b rows
+ * (the rows of block positions q_len - L_b .. q_len - 1).  Errors: as libra_decode_attn_multi. */
+int libra_decode_attn_multi_append(libra_handle_t handle, const void* q, int32_t q_len, const void* k_new,
+                                   const void* v_new, void* k_pages, void* v_pages, const int32_t* block_table,
+                                   const int32_t* seq_lens, void* out, void* stream);
+
 /* The same step for callers whose data lives in host memory: copies q, both pools, the block
  * table and the lengths to `staging_dev` (a caller-owned device region of at least
  * libra_host_staging_size bytes, 256-byte aligned), plans, runs D and C and copies `out` back

@@ -65,6 +65,7 @@ SIGNATURES = {
     "libra_set_lse_output": (C.c_int, [_vp, _vp]),
     "libra_set_kv_dtype": (C.c_int, [_vp, C.c_int32, C.c_float, C.c_float]),
     "libra_decode_attn_multi": (C.c_int, [_vp, _vp, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "libra_decode_attn_multi_append": (C.c_int, [_vp, _vp, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_ring_step": (C.c_int, [C.c_int32, _vp, _vp, _vp, C.c_size_t, C.c_int32, _vp, C.c_uint32, C.c_uint32, _vp, C.c_int32,
                                   _vp]),
     "libra_debug_stream_read": (C.c_int, [_vp, _vp, C.c_size_t, _vp]),
@@ -312,6 +313,12 @@ class Handle:
                           seq_lens_ptr: int, out_ptr: int, stream: int) -> None:
         _check(lib.libra_decode_attn_multi(self._h, q_ptr, q_len, k_ptr, v_ptr, block_table_ptr, seq_lens_ptr,
                                            out_ptr, stream), "libra_decode_attn_multi")
+
+    def decode_attn_multi_append(self, q_ptr: int, q_len: int, k_new_ptr: int, v_new_ptr: int, k_ptr: int, v_ptr: int,
+                                 block_table_ptr: int, seq_lens_ptr: int, out_ptr: int, stream: int) -> None:
+        _check(lib.libra_decode_attn_multi_append(self._h, q_ptr, q_len, k_new_ptr, v_new_ptr, k_ptr, v_ptr,
+                                                  block_table_ptr, seq_lens_ptr, out_ptr, stream),
+               "libra_decode_attn_multi_append")
 
     def decode_attn_append(self, q_ptr: int, k_new_ptr: int, v_new_ptr: int, k_ptr: int, v_ptr: int,
                            block_table_ptr: int, seq_lens_ptr: int, out_ptr: int, stream: int) -> None:

@@ -65,8 +65,9 @@ struct DecodeParams {
   int32_t num_empty;      // empty sequences whose output row this launch zeroes
   int32_t fused_combine;  // 1: the last block of a split sequence merges its partials (step C) itself
   int32_t early_prefetch; // 1: block-table walk and first copies of old tokens start before the grid dependency wait
-  // KV append fused into the step (null k_new = off): the current token's K and V rows, [B, Hkv, D] in the cache's
-  // element type, are written into slot (L_b - 1) % 16 of the sequence's last page, in the pools and in the staged tile
+  // KV append fused into the step (null k_new = off): the K and V rows of the newest q_len tokens, [B, q_len, Hkv, D]
+  // in the cache's element type, are written into their slots of the sequence's last page(s), in the pools and in the
+  // staged tiles
   const void* k_new;
   const void* v_new;
   void* k_pool;
@@ -800,27 +801,30 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
       st.l[0][0] += float((words[lane * 16] ^ words[SM::kTileBytes / 4 + lane * 16]) & 0xffu);
       st.m[0][0] = 0.f;
     } else {
-      if (p.k_new != nullptr && u.chunk_j == u.n_chunks - 1 && u.kv_end - tok0 <= 16) {
-        // this page holds the sequence's newest token: its K and V rows come from k_new / v_new.  The copy
-        // that just landed predates them, so patch the staged tiles (swizzled row) and write the pools.
+      if (p.k_new != nullptr && tok0 + 16 > len_dev - p.q_len && tok0 < len_dev) {
+        // this tile holds some of the sequence's newest q_len tokens: their K and V rows come from k_new / v_new
+        // ([batch, q_len, Hkv, D]).  The copy that just landed predates them, so patch the staged tiles (swizzled
+        // rows) and write the pools.
         constexpr int EB = kFp8 ? 1 : 2;           // bytes per cache element
         constexpr int kRowChunks = D * EB / 16;    // 16-byte chunks of one row
-        const int r = (u.kv_end - 1) & 15;
         const int which = lane / kRowChunks;       // 0: K, 1: V
         const int c16 = lane % kRowChunks;
-        if (which < 2) {
-          const int last = u.kv_end - 1;                       // the newest token
-          const int64_t page = __ldg(p.block_table + int64_t(u.b) * p.block_table_ld + (last >> (4 + p.tile_shift)));
-          const int slot = last & ((16 << p.tile_shift) - 1);  // its slot in that page
-          const uint8_t* src = reinterpret_cast<const uint8_t*>(which ? p.v_new : p.k_new) +
-                               (int64_t(u.b) * p.num_kv_heads + kvh) * (D * EB) + c16 * 16;
-          const uint4 row = __ldg(reinterpret_cast<const uint4*>(src));
-          uint8_t* tile = my_ring + s * SM::kStageBytes + which * SM::kTileBytes;
-          *reinterpret_cast<uint4*>(tile + tile_off(r, c16)) = row;
-          if (page >= 0 && page < p.num_pages) {
-            uint8_t* dst = reinterpret_cast<uint8_t*>(which ? p.v_pool : p.k_pool) +
-                           (page * p.stride_page + int64_t(kvh) * p.stride_head + int64_t(slot) * p.stride_token) * EB + c16 * 16;
-            *reinterpret_cast<uint4*>(dst) = row;
+        const int t_lo = max(tok0, len_dev - p.q_len), t_hi = min(min(tok0 + 16, len_dev), u.kv_end);
+        for (int t = t_lo; t < t_hi; ++t) {
+          if (which < 2) {
+            const int i = t - (len_dev - p.q_len);               // which of the new tokens
+            const int64_t page = __ldg(p.block_table + int64_t(u.b) * p.block_table_ld + (t >> (4 + p.tile_shift)));
+            const int slot = t & ((16 << p.tile_shift) - 1);     // its slot in that page
+            const uint8_t* src = reinterpret_cast<const uint8_t*>(which ? p.v_new : p.k_new) +
+                                 ((int64_t(u.b) * p.q_len + i) * p.num_kv_heads + kvh) * (D * EB) + c16 * 16;
+            const uint4 row = __ldg(reinterpret_cast<const uint4*>(src));
+            uint8_t* tile = my_ring + s * SM::kStageBytes + which * SM::kTileBytes;
+            *reinterpret_cast<uint4*>(tile + tile_off(t - tok0, c16)) = row;
+            if (page >= 0 && page < p.num_pages) {
+              uint8_t* dst = reinterpret_cast<uint8_t*>(which ? p.v_pool : p.k_pool) +
+                             (page * p.stride_page + int64_t(kvh) * p.stride_head + int64_t(slot) * p.stride_token) * EB + c16 * 16;
+              *reinterpret_cast<uint4*>(dst) = row;
+            }
           }
         }
         fence_proxy_async();  // these generic writes come before the next TMA write into this stage

@@ -788,7 +788,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
       reinterpret_cast<uintptr_t>(q) % 4 || reinterpret_cast<uintptr_t>(out) % 4) {
     return LIBRA_INVALID_ARGUMENT;
   }
-  if (q_len < 1 || q_len > h->max_q_len || (q_len > 1 && k_new)) return LIBRA_INVALID_ARGUMENT;
+  if (q_len < 1 || q_len > h->max_q_len) return LIBRA_INVALID_ARGUMENT;
   if (!h->planned) return LIBRA_NOT_PLANNED;
   DeviceGuard guard(h->cfg.device);
   if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
@@ -1148,6 +1148,13 @@ int libra_debug_wait_selftest(libra_handle_t h, void* stream) {
 int libra_decode_attn_multi(libra_handle_t h, const void* q, int32_t q_len, const void* k_pages, const void* v_pages,
                             const int32_t* block_table, const int32_t* seq_lens, void* out, void* stream) {
   return decode_impl(h, q, nullptr, nullptr, k_pages, v_pages, block_table, seq_lens, out, stream, false, q_len);
+}
+
+int libra_decode_attn_multi_append(libra_handle_t h, const void* q, int32_t q_len, const void* k_new, const void* v_new,
+                                   void* k_pages, void* v_pages, const int32_t* block_table, const int32_t* seq_lens,
+                                   void* out, void* stream) {
+  if (!k_new || !v_new) return LIBRA_INVALID_ARGUMENT;
+  return decode_impl(h, q, k_new, v_new, k_pages, v_pages, block_table, seq_lens, out, stream, false, q_len);
 }
 
 int libra_debug_gather_read(libra_handle_t h, const void* q, const void* k_pages, const void* v_pages,

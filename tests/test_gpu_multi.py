@@ -179,3 +179,55 @@ def test_misuse_is_rejected(lib):
             h.decode_attn_multi(x.data_ptr(), bad, x.data_ptr(), x.data_ptr(), x.data_ptr(), x.data_ptr(), x.data_ptr(), st)
     torch.cuda.synchronize()
     h.close()
+
+
+@pytest.mark.parametrize("layout", ["HND", "NHD"])
+def test_append_of_the_new_tokens_fused_in(lib, layout):
+    """libra_decode_attn_multi_append: the rows of the newest q_len tokens arrive with the call, land in their slots
+    (across a tile and page boundary where the block straddles one) and the output is the oracle's on the updated
+    pools; pools afterwards equal the definition bit for bit."""
+    import torch
+    dev = torch.device("cuda:0")
+    Tq = 4
+    lens = [4, 5, 16, 17, 18, 19, 20, 33, 300, 1027, 2, 0, 2050]
+    B, Hq, Hkv, d = len(lens), 8, 2, 128
+    lens_a, bt, _, k, v = W.random_case(120, B, Hq, Hkv, d, lens, poison=False)
+    q = draw_q(121, B, Tq, Hq, d)
+    rng = np.random.default_rng(122)
+    k_new = W.f32_to_bf16_bits(rng.standard_normal((B, Tq, Hkv, d)).astype(np.float32))
+    v_new = W.f32_to_bf16_bits(rng.standard_normal((B, Tq, Hkv, d)).astype(np.float32))
+    k_ref, v_ref = k.copy(), v.copy()
+    for b, L in enumerate(lens_a):
+        for i in range(Tq):
+            t = int(L) - Tq + i
+            if t >= 0:
+                k_ref[bt[b, t // 16], :, t % 16, :] = k_new[b, i]
+                v_ref[bt[b, t // 16], :, t % 16, :] = v_new[b, i]
+    ref, _ = O.paged_multi_token_attention(q, k_ref, v_ref, bt, lens_a)
+    kh, vh, strides = k, v, (0, 0, 0)
+    if layout == "NHD":
+        kh = np.ascontiguousarray(k.transpose(0, 2, 1, 3))
+        vh = np.ascontiguousarray(v.transpose(0, 2, 1, 3))
+        strides = (16 * Hkv * d, d, Hkv * d)
+    for plan in (None, small_plan(lib)):
+        for early in (False, True):
+            h = lib.Handle(Hq, Hkv, d, k.shape[0], B, bt.shape[1], kv_strides=strides, plan=plan)
+            h.set_max_query_tokens(Tq)
+            h.set_early_prefetch(early)
+            ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=dev)
+            qd, kd, vd, btd = (H.to_dev(x, dev) for x in (q, kh, vh, bt))
+            knd, vnd = H.to_dev(k_new, dev), H.to_dev(v_new, dev)
+            lens_dev = torch.from_numpy(lens_a).to(dev)
+            out = torch.full((B, Tq, Hq, d), H.CANARY, dtype=torch.int16, device=dev)
+            st = torch.cuda.current_stream().cuda_stream
+            h.plan(lens_a, ws.data_ptr(), ws.numel(), st)
+            h.decode_attn_multi_append(qd.data_ptr(), Tq, knd.data_ptr(), vnd.data_ptr(), kd.data_ptr(), vd.data_ptr(),
+                                       btd.data_ptr(), lens_dev.data_ptr(), out.data_ptr(), st)
+            torch.cuda.synchronize()
+            assert h.debug_error_word() == 0
+            check(H.bf16_dev_to_f32(out), ref, f"multi append {layout} early={early}")
+            got_k, got_v = kd.cpu().numpy().view(np.uint16), vd.cpu().numpy().view(np.uint16)
+            if layout == "NHD":
+                got_k, got_v = got_k.transpose(0, 2, 1, 3), got_v.transpose(0, 2, 1, 3)
+            assert np.array_equal(got_k, k_ref) and np.array_equal(got_v, v_ref)
+            h.close()
