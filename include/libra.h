@@ -402,6 +402,14 @@ int libra_rollout_dp(int32_t n_gpus, const int32_t* lengths, int32_t n_requests,
                      const double* cost_coef, double* makespan, int32_t* inst_tp, int32_t* inst_first,
                      int32_t* inst_count, int32_t inst_capacity, int32_t* n_instances);
 
+/* libra_rollout_dp evaluates the minimum over x by bisection when no cost coefficient is negative (the first term of
+ * the max cannot grow with x and the second cannot shrink, so the minimum sits where they cross); otherwise, and
+ * always in libra_rollout_dp_scan, every x is tried as the recurrence is written.  Same arguments, same results bit
+ * for bit (ties go to the smaller x and the earlier degree in both); the scan is kept as the reference. */
+int libra_rollout_dp_scan(int32_t n_gpus, const int32_t* lengths, int32_t n_requests, const int32_t* tp_set,
+                          int32_t n_tp, const double* cost_coef, double* makespan, int32_t* inst_tp,
+                          int32_t* inst_first, int32_t* inst_count, int32_t inst_capacity, int32_t* n_instances);
+
 /* Causality-aware prefix tree (Section 5): a node is (prompt id, sequence of tool-return states); every
  * node keeps a histogram of the remaining trajectory length seen from that point, with bins aligned to
  * the buckets' length thresholds: bin k holds lengths <= bin_upper[k] (increasing), the last bin

@@ -90,6 +90,8 @@ SIGNATURES = {
                                    _vp, _vp]),
     "libra_rollout_dp": (C.c_int, [C.c_int32, _i32p, C.c_int32, _i32p, C.c_int32, C.POINTER(C.c_double),
                                    C.POINTER(C.c_double), _i32p, _i32p, _i32p, C.c_int32, _i32p]),
+    "libra_rollout_dp_scan": (C.c_int, [C.c_int32, _i32p, C.c_int32, _i32p, C.c_int32, C.POINTER(C.c_double),
+                                        C.POINTER(C.c_double), _i32p, _i32p, _i32p, C.c_int32, _i32p]),
     "libra_trie_create": (C.c_int, [C.POINTER(_vp), _i32p, C.c_int32]),
     "libra_trie_destroy": (C.c_int, [_vp]),
     "libra_trie_insert": (C.c_int, [_vp, C.c_int64, _i32p, C.c_int32, _i32p]),
@@ -162,8 +164,8 @@ def libra_ring_step(device: int, dst_ptr: int, own_ptr: int, received_ptr: int, 
                                timeout_us, status_ptr, num_blocks, stream), "libra_ring_step")
 
 
-def libra_rollout_dp(n_gpus: int, lengths, tp_set, cost_coef):
-    """RolloutDP: returns (makespan, [(tp, first_sorted_index, count), ...])."""
+def libra_rollout_dp(n_gpus: int, lengths, tp_set, cost_coef, scan: bool = False):
+    """RolloutDP: returns (makespan, [(tp, first_sorted_index, count), ...]).  scan = the term-by-term reference."""
     lens = _as_i32(lengths)
     tps = _as_i32(tp_set)
     coef = np.ascontiguousarray(cost_coef, dtype=np.float64).reshape(len(tps), 4)
@@ -171,8 +173,9 @@ def libra_rollout_dp(n_gpus: int, lengths, tp_set, cost_coef):
     itp, ifirst, icount = (np.zeros(cap, np.int32) for _ in range(3))
     mk, n = C.c_double(0), C.c_int32(0)
     p = lambda a: a.ctypes.data_as(_i32p)
-    st = lib.libra_rollout_dp(n_gpus, p(lens), len(lens), p(tps), len(tps), coef.ctypes.data_as(C.POINTER(C.c_double)),
-                              C.byref(mk), p(itp), p(ifirst), p(icount), cap, C.byref(n))
+    fn = lib.libra_rollout_dp_scan if scan else lib.libra_rollout_dp
+    st = fn(n_gpus, p(lens), len(lens), p(tps), len(tps), coef.ctypes.data_as(C.POINTER(C.c_double)),
+            C.byref(mk), p(itp), p(ifirst), p(icount), cap, C.byref(n))
     _check(st, "libra_rollout_dp")
     return mk.value, [(int(itp[k]), int(ifirst[k]), int(icount[k])) for k in range(n.value)]
 

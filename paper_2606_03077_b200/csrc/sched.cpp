@@ -50,11 +50,17 @@ struct libra_trie_s {
   }
 };
 
-extern "C" {
+namespace {
 
-int libra_rollout_dp(int32_t n_gpus, const int32_t* lengths, int32_t n_requests, const int32_t* tp_set, int32_t n_tp,
-                     const double* cost_coef, double* makespan, int32_t* inst_tp, int32_t* inst_first,
-                     int32_t* inst_count, int32_t inst_capacity, int32_t* n_instances) {
+// The recurrence as printed, and a faster evaluation of the same minimum.
+//   dp[g][i] = min over tp <= g, 0 <= x <= i of max(dp[g - tp][i - x], Cost(tp, i - x + 1, i))
+// Plain: every x is tried.  Fast (valid when no cost coefficient is negative): as x grows the first term cannot
+// grow (fewer requests left for the other instances) and the second cannot shrink (more requests on this one), so
+// the minimum of their maximum sits where they cross; a binary search finds the crossing and a second one the
+// leftmost x of the same value, which is the x the plain scan would have kept.  Same dp, same arg-mins, bit for bit.
+int rollout_dp_impl(bool allow_fast, int32_t n_gpus, const int32_t* lengths, int32_t n_requests, const int32_t* tp_set,
+                    int32_t n_tp, const double* cost_coef, double* makespan, int32_t* inst_tp, int32_t* inst_first,
+                    int32_t* inst_count, int32_t inst_capacity, int32_t* n_instances) {
   if (n_gpus < 0 || n_requests < 0 || n_tp <= 0 || !tp_set || !cost_coef || !makespan || !n_instances) {
     return LIBRA_INVALID_ARGUMENT;
   }
@@ -64,6 +70,9 @@ int libra_rollout_dp(int32_t n_gpus, const int32_t* lengths, int32_t n_requests,
   const int G = n_gpus, L = n_requests;
   std::vector<int32_t> sorted(lengths, lengths + L);
   std::sort(sorted.begin(), sorted.end());  // non-decreasing: every instance gets a contiguous segment
+  bool fast = allow_fast;
+  for (int t = 0; t < 4 * n_tp; ++t) fast = fast && cost_coef[t] >= 0.0;
+  for (int i = 0; i < L; ++i) fast = fast && sorted[size_t(i)] >= 0;
   SegmentCost cost;
   cost.coef = cost_coef;
   cost.s1.assign(L + 1, 0.0);
@@ -77,7 +86,6 @@ int libra_rollout_dp(int32_t n_gpus, const int32_t* lengths, int32_t n_requests,
   std::vector<double> dp((size_t(G) + 1) * W, inf);
   std::vector<int32_t> arg_tp((size_t(G) + 1) * W, -1), arg_x((size_t(G) + 1) * W, -1);
   dp[0] = 0.0;  // dp[0][0]
-  // dp[g][i] = min over tp <= g, 0 <= x <= i of max(dp[g - tp][i - x], Cost(tp, i - x + 1, i))
   for (int g = 1; g <= G; ++g) {
     for (int i = 0; i <= L; ++i) {
       double best = inf;
@@ -86,16 +94,46 @@ int libra_rollout_dp(int32_t n_gpus, const int32_t* lengths, int32_t n_requests,
         const int tp = tp_set[t];
         if (tp > g) continue;
         const double* prev = &dp[size_t(g - tp) * W];
-        for (int x = 0; x <= i; ++x) {
-          const double p = prev[i - x];
-          if (!(p < best)) continue;  // max(p, cost) >= p: cannot improve
-          const double cand = std::max(p, cost(t, i - x + 1, i));
-          if (cand < best) {
-            best = cand;
-            btp = t;
-            bx = x;
+        if (!fast) {
+          for (int x = 0; x <= i; ++x) {
+            const double p = prev[i - x];
+            if (!(p < best)) continue;  // max(p, cost) >= p: cannot improve
+            const double cand = std::max(p, cost(t, i - x + 1, i));
+            if (cand < best) {
+              best = cand;
+              btp = t;
+              bx = x;
+            }
+          }
+          continue;
+        }
+        // first x at which this instance's cost reaches what the others need (x = i + 1 if it never does)
+        int lo = 0, hi = i + 1;
+        while (lo < hi) {
+          const int mid = (lo + hi) / 2;
+          if (cost(t, i - mid + 1, i) >= prev[i - mid]) hi = mid;
+          else lo = mid + 1;
+        }
+        double cand = inf;
+        int cx = -1;
+        for (int x = std::max(0, lo - 1); x <= std::min(i, lo); ++x) {   // the two sides of the crossing
+          const double v = std::max(prev[i - x], cost(t, i - x + 1, i));
+          if (v < cand) {
+            cand = v;
+            cx = x;
           }
         }
+        if (cx < 0 || !(cand < best)) continue;
+        // the leftmost x with the same value: left of the crossing the maximum is prev[i - x], which does not grow
+        int l2 = 0, h2 = cx;
+        while (l2 < h2) {
+          const int mid = (l2 + h2) / 2;
+          if (prev[i - mid] <= cand) h2 = mid;
+          else l2 = mid + 1;
+        }
+        best = cand;
+        btp = t;
+        bx = l2;
       }
       dp[size_t(g) * W + i] = best;
       arg_tp[size_t(g) * W + i] = btp;
@@ -126,6 +164,24 @@ int libra_rollout_dp(int32_t n_gpus, const int32_t* lengths, int32_t n_requests,
     inst_count[k] = counts[size_t(count - 1 - k)];
   }
   return LIBRA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int libra_rollout_dp(int32_t n_gpus, const int32_t* lengths, int32_t n_requests, const int32_t* tp_set, int32_t n_tp,
+                     const double* cost_coef, double* makespan, int32_t* inst_tp, int32_t* inst_first,
+                     int32_t* inst_count, int32_t inst_capacity, int32_t* n_instances) {
+  return rollout_dp_impl(true, n_gpus, lengths, n_requests, tp_set, n_tp, cost_coef, makespan, inst_tp, inst_first,
+                         inst_count, inst_capacity, n_instances);
+}
+
+int libra_rollout_dp_scan(int32_t n_gpus, const int32_t* lengths, int32_t n_requests, const int32_t* tp_set, int32_t n_tp,
+                          const double* cost_coef, double* makespan, int32_t* inst_tp, int32_t* inst_first,
+                          int32_t* inst_count, int32_t inst_capacity, int32_t* n_instances) {
+  return rollout_dp_impl(false, n_gpus, lengths, n_requests, tp_set, n_tp, cost_coef, makespan, inst_tp, inst_first,
+                         inst_count, inst_capacity, n_instances);
 }
 
 int libra_trie_create(libra_trie_t* trie, const int32_t* bin_upper, int32_t n_thresholds) {

@@ -112,3 +112,39 @@ def test_prefix_tree_small_example(lib):
     assert t.route(7, [1, 2], cost, [0.0, 1.0])[0] == 0
     assert t.route(7, [1, 3], cost, [0.0, 1.0])[0] == 1
     t.close()
+
+
+def test_bisection_gives_the_scan_bit_for_bit(lib):
+    """libra_rollout_dp (bisection on x where the coefficients allow it) against libra_rollout_dp_scan (every x):
+    same makespan, same partition, ties included; and with a negative coefficient the two are the same code path."""
+    import time
+    rng = np.random.default_rng(7)
+    for trial in range(60):
+        n = int(rng.integers(0, 220))
+        g = int(rng.integers(1, 33))
+        kind = trial % 4
+        if kind == 0:
+            lens = rng.integers(1, 40000, size=n)
+        elif kind == 1:
+            lens = rng.integers(1, 6, size=n)                    # many equal lengths: ties everywhere
+        elif kind == 2:
+            lens = np.full(n, 1000)
+        else:
+            lens = np.floor(1024 * np.exp(rng.standard_normal(n))).astype(np.int64) + 1
+        tp_set = sorted(set(int(x) for x in rng.choice([1, 2, 4, 8], size=int(rng.integers(1, 5)))))
+        coef = [[float(rng.integers(0, 4)) / (1 + t), float(rng.integers(0, 3)) * 1e-4 / (1 + t), float(rng.integers(0, 3)),
+                 float(rng.integers(0, 5))] for t in range(len(tp_set))]
+        fast = lib.libra_rollout_dp(g, lens, tp_set, coef)
+        scan = lib.libra_rollout_dp(g, lens, tp_set, coef, scan=True)
+        assert fast == scan or (math.isinf(fast[0]) and math.isinf(scan[0])), (trial, fast, scan)
+    coef = [[1.0, 0.0, -0.5, 0.0], [0.5, 0.0, 0.0, 1.0]]        # a negative coefficient: no bisection
+    lens = rng.integers(1, 100, size=50)
+    assert lib.libra_rollout_dp(8, lens, [1, 2], coef) == lib.libra_rollout_dp(8, lens, [1, 2], coef, scan=True)
+    # and it is what makes the planner cheap: 128 GPUs x 4096 requests
+    lens = np.floor(2048 * np.exp(rng.standard_normal(4096))).astype(np.int64) + 1
+    coef = [[1.0 / tp, 2e-5 / tp, 5.0, 100.0 * tp] for tp in (1, 2, 4, 8)]
+    t0 = time.perf_counter()
+    mk, inst = lib.libra_rollout_dp(128, lens, [1, 2, 4, 8], coef)
+    dt = time.perf_counter() - t0
+    assert math.isfinite(mk) and sum(c for _, _, c in inst) == 4096 and sum(tp for tp, _, _ in inst) == 128
+    assert dt < 5.0
