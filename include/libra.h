@@ -152,8 +152,8 @@ int libra_set_max_query_tokens(libra_handle_t handle, int32_t max_q_len);
  * codes (1 sign, 4 exponent, 3 mantissa bits, bias 7, no infinities, one NaN per sign), one byte per element,
  * with one scale per tensor: key = k_scale * value of the code, value = v_scale * value of the code; the
  * attention is the same definition on those keys and values, q and out stay bf16.  The strides given at
- * creation keep their meaning (elements, now bytes) and must be multiples of 16; head_dim must be 128
- * (UNSUPPORTED_SHAPE otherwise); k_scale and v_scale must be positive and finite (ignored for BF16).
+ * creation keep their meaning (elements, now bytes) and must be multiples of 16; k_scale and v_scale must be
+ * positive and finite (ignored for BF16).
  * Halving the bytes per cached token halves what the step has to read.  With E4M3 pools the rows given to
  * libra_decode_attn_append (k_new, v_new: [batch, num_kv_heads, head_dim]) and the dense buffers of
  * libra_kv_gather / libra_kv_scatter hold codes too, one byte per element; libra_decode_attn_host returns

@@ -379,8 +379,9 @@ __device__ __forceinline__ void process_page(WarpAcc<D, NT>& st, const uint32_t 
   }
 }
 
-// ---- 8-bit (E4M3) cache, head_dim 128 -------------------------------------------------------------
-// A tile is 16 tokens x 128 bytes with the same 128-byte swizzle.  ldmatrix moves it as 16-bit units, i.e.
+// ---- 8-bit (E4M3) cache ---------------------------------------------------------------------------
+// A tile is 16 tokens x D bytes: rows of 128 bytes with the 128-byte swizzle (head_dim 128) or rows of 64 bytes
+// with the 64-byte swizzle (head_dim 64).  ldmatrix moves it as 16-bit units, i.e.
 // PAIRS of codes, so the fragments come out in an order of their own; sums over k and the assignment of
 // output rows do not care about order as long as both operands agree:
 //   scores : within a 16-dim chunk, mma k-slots (2t, 2t+1, 2t+8, 2t+9) carry dims (4t, 4t+1, 4t+2, 4t+3)
@@ -389,17 +390,26 @@ __device__ __forceinline__ void process_page(WarpAcc<D, NT>& st, const uint32_t 
 // rounded to fp16.  (Converting the values with integer operations instead, to unload the pipe the conversion
 // instruction shares with the exponentials, measured 5-10 % slower.)
 
+// Byte offset of 16-byte chunk c of row r in such a tile (the copy engine's swizzle: the chunk index is XORed with
+// address bits 7 and up - 3 of them for 128-byte rows, 2 for 64-byte rows).
+template <int D>
+__device__ __forceinline__ uint32_t tile_off_fp8(int r, int c) {
+  if constexpr (D == 128) return uint32_t((r << 7) + ((c ^ (r & 7)) << 4));
+  else return uint32_t((r << 6) + ((c ^ ((r >> 1) & 3)) << 4));
+}
+
 // Q^T fragments in that k-order, fp16; columns >= cols are zero.
-template <int NT>
-__device__ __forceinline__ void load_q_frags_fp8(uint32_t (&qf)[NT][8][2], const DecodeParams& p, int b, int kvh, int lane) {
+template <int D, int NT>
+__device__ __forceinline__ void load_q_frags_fp8(uint32_t (&qf)[NT][D / 16][2], const DecodeParams& p, int b, int kvh,
+                                                 int lane) {
   const int g = lane >> 2, t = lane & 3;
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
     const int col = nt * 8 + g;
     const bool live = col < p.cols;
-    const __nv_bfloat16* qrow = p.q + (int64_t(b) * p.num_q_heads + col_row(p, kvh, live ? col : 0)) * 128;
+    const __nv_bfloat16* qrow = p.q + (int64_t(b) * p.num_q_heads + col_row(p, kvh, live ? col : 0)) * D;
 #pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
+    for (int kk = 0; kk < D / 16; ++kk) {
       const uint2 raw = __ldg(reinterpret_cast<const uint2*>(qrow + 16 * kk + 4 * t));   // dims 4t .. 4t+3 of chunk kk
       const __nv_bfloat162 x01 = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
       const __nv_bfloat162 x23 = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
@@ -412,21 +422,20 @@ __device__ __forceinline__ void load_q_frags_fp8(uint32_t (&qf)[NT][8][2], const
 }
 
 // One page (16 tokens) of one KV head from an E4M3 cache; same contract as process_page.
-template <int NT>
-__device__ __forceinline__ void process_page_fp8(WarpAcc<128, NT>& st, const uint32_t (&qf)[NT][8][2], uint32_t kt,
+template <int D, int NT>
+__device__ __forceinline__ void process_page_fp8(WarpAcc<D, NT>& st, const uint32_t (&qf)[NT][D / 16][2], uint32_t kt,
                                                  uint32_t vt, uint8_t* v_gen, int n_valid, float scale_log2, int lane,
                                                  int n_common, int len_rel, const int (&cut)[NT][2]) {
   const int g = lane >> 2;
   // ldmatrix.x4: lanes 0-7 / 8-15 give the rows (tokens 0-7 / 8-15) of 16-byte chunk c, lanes 16-31 those of chunk c+1
   const int row = (lane & 7) + ((lane >> 3) & 1) * 8;
   const int csel = lane >> 4;
-  const uint32_t row_off = uint32_t(row) << 7;
 
   if (n_valid < 16) {
     // rows past the end may hold anything, NaN codes included: clear them in V so that 0 * garbage cannot leak
-    for (int i = lane; i < (16 - n_valid) * 8; i += 32) {
-      const int r = n_valid + (i >> 3);
-      *reinterpret_cast<uint4*>(v_gen + (r << 7) + ((i & 7) << 4)) = make_uint4(0, 0, 0, 0);
+    for (int i = lane; i < (16 - n_valid) * (D / 16); i += 32) {
+      const int r = n_valid + i / (D / 16);
+      *reinterpret_cast<uint4*>(v_gen + r * D + ((i % (D / 16)) << 4)) = make_uint4(0, 0, 0, 0);
     }
     fence_proxy_async();  // these generic writes come before the next TMA write into this stage
     __syncwarp();
@@ -440,9 +449,9 @@ __device__ __forceinline__ void process_page_fp8(WarpAcc<128, NT>& st, const uin
     sc2[nt][0] = sc2[nt][1] = sc2[nt][2] = sc2[nt][3] = 0.f;
   }
 #pragma unroll
-  for (int c2 = 0; c2 < 4; ++c2) {
+  for (int c2 = 0; c2 < D / 32; ++c2) {
     uint32_t r[4];   // (tokens 0-7, chunk 2 c2), (tokens 8-15, chunk 2 c2), (tokens 0-7, chunk 2 c2 + 1), (tokens 8-15, chunk 2 c2 + 1)
-    ldsm_x4(r, kt + row_off + (uint32_t((2 * c2 + csel) ^ (row & 7)) << 4));
+    ldsm_x4(r, kt + tile_off_fp8<D>(row, 2 * c2 + csel));
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       uint32_t a[4];
@@ -491,7 +500,7 @@ __device__ __forceinline__ void process_page_fp8(WarpAcc<128, NT>& st, const uin
       st.l[nt][0] *= f0;
       st.l[nt][1] *= f1;
 #pragma unroll
-      for (int mt = 0; mt < 8; ++mt) {
+      for (int mt = 0; mt < D / 16; ++mt) {
         st.acc[nt][mt][0] *= f0;
         st.acc[nt][mt][1] *= f1;
         st.acc[nt][mt][2] *= f0;
@@ -515,9 +524,9 @@ __device__ __forceinline__ void process_page_fp8(WarpAcc<128, NT>& st, const uin
 
   // ---- O^T += V^T . P^T
 #pragma unroll
-  for (int c2 = 0; c2 < 4; ++c2) {
+  for (int c2 = 0; c2 < D / 32; ++c2) {
     uint32_t r[4];   // transposed: this thread gets, per matrix, {token 2t: dims 2g, 2g+1 | token 2t+1: dims 2g, 2g+1}
-    ldsm_x4_trans(r, vt + row_off + (uint32_t((2 * c2 + csel) ^ (row & 7)) << 4));
+    ldsm_x4_trans(r, vt + tile_off_fp8<D>(row, 2 * c2 + csel));
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       uint32_t a[4];
@@ -650,14 +659,13 @@ struct DecodeSmem {
 // D: head_dim (64 | 128); NT: 8-wide head tiles (1: G <= 8, 2: G <= 16); NW warps; STAGES per warp.
 // kLoadsOnly: measurement build of the same kernel - same plan, page walk and copies, but each staged page
 // is only touched (one shared-memory word per lane) instead of computed on; `out` gets meaningless values.
-// kFp8: the pools hold E4M3 codes (head_dim 128 only); tiles are half as large, the page math is process_page_fp8.
+// kFp8: the pools hold E4M3 codes; tiles are half as large, the page math is process_page_fp8.
 template <int D, int NT, int NW, int STAGES, bool kLoadsOnly = false, bool kFp8 = false>
 __global__ void __launch_bounds__(NW * 32)
 decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
               const __grid_constant__ DecodeParams p, const __grid_constant__ ParamPlan pp) {
   using namespace dev;
   using SM = DecodeSmem<D, NW, STAGES, kFp8 ? 1 : 2>;
-  static_assert(!kFp8 || D == 128, "the 8-bit path is written for head_dim 128");
   constexpr int NH = kFp8 ? 1 : D / 64;   // 128-byte column blocks of a row
   static_assert(NT * 8 * D * 4 <= SM::kWarpBytes, "epilogue staging must fit in the warp's ring");
 
@@ -780,7 +788,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     grid_dependency_wait();
   }
   uint32_t qf[NT][D / 16][2];
-  if constexpr (kFp8) load_q_frags_fp8<NT>(qf, p, u.b, kvh, lane);
+  if constexpr (kFp8) load_q_frags_fp8<D, NT>(qf, p, u.b, kvh, lane);
   else load_q_frags<D, NT>(qf, p, u.b, kvh, lane);
   for (int j = issued; j < pre; ++j) issue(j, j);
   if (threadIdx.x == 0) check_planned_length(p, u, len_dev);
@@ -819,7 +827,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
                                  ((int64_t(u.b) * p.q_len + i) * p.num_kv_heads + kvh) * (D * EB) + c16 * 16;
             const uint4 row = __ldg(reinterpret_cast<const uint4*>(src));
             uint8_t* tile = my_ring + s * SM::kStageBytes + which * SM::kTileBytes;
-            *reinterpret_cast<uint4*>(tile + tile_off(t - tok0, c16)) = row;
+            const uint32_t off = kFp8 ? tile_off_fp8<D>(t - tok0, c16) : tile_off(t - tok0, c16);
+            *reinterpret_cast<uint4*>(tile + off) = row;
             if (page >= 0 && page < p.num_pages) {
               uint8_t* dst = reinterpret_cast<uint8_t*>(which ? p.v_pool : p.k_pool) +
                              (page * p.stride_page + int64_t(kvh) * p.stride_head + int64_t(slot) * p.stride_token) * EB + c16 * 16;
@@ -831,7 +840,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
         __syncwarp();
       }
       if constexpr (kFp8) {
-        process_page_fp8<NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes,
+        process_page_fp8<D, NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes,
                              u.kv_end - tok0, p.scale_log2, lane, common_end - tok0, len_dev - tok0, cut);
       } else {
         process_page<D, NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes,

@@ -95,19 +95,24 @@ const int kLoadsOnlySmem[2] = {libra::DecodeSmem<64, kLoadsOnlyWarps, kLoadsOnly
 constexpr int kFp8OneTile = 2, kFp8TwoTiles = 1, kFp8ShortUnits = 5, kFp8TinyUnits = 6;
 struct Fp8Variant {
   int warps, stages;
-  DecodeKernelFn fn[2][2];
-  int smem;
+  DecodeKernelFn fn[2][2][2];   // [D == 128][loads only][NT - 1]
+  int smem[2];                  // [D == 128]
 };
 template <int NW, int ST>
 Fp8Variant make_fp8_variant() {
   Fp8Variant v;
   v.warps = NW;
   v.stages = ST;
-  v.fn[0][0] = libra::decode_kernel<128, 1, NW, ST, false, true>;
-  v.fn[0][1] = libra::decode_kernel<128, 2, NW, ST, false, true>;
-  v.fn[1][0] = libra::decode_kernel<128, 1, NW, ST, true, true>;
-  v.fn[1][1] = libra::decode_kernel<128, 2, NW, ST, true, true>;
-  v.smem = libra::DecodeSmem<128, NW, ST, 1>::kDynamicBytes;
+  v.fn[0][0][0] = libra::decode_kernel<64, 1, NW, ST, false, true>;
+  v.fn[0][0][1] = libra::decode_kernel<64, 2, NW, ST, false, true>;
+  v.fn[0][1][0] = libra::decode_kernel<64, 1, NW, ST, true, true>;
+  v.fn[0][1][1] = libra::decode_kernel<64, 2, NW, ST, true, true>;
+  v.fn[1][0][0] = libra::decode_kernel<128, 1, NW, ST, false, true>;
+  v.fn[1][0][1] = libra::decode_kernel<128, 2, NW, ST, false, true>;
+  v.fn[1][1][0] = libra::decode_kernel<128, 1, NW, ST, true, true>;
+  v.fn[1][1][1] = libra::decode_kernel<128, 2, NW, ST, true, true>;
+  v.smem[0] = libra::DecodeSmem<64, NW, ST, 1>::kDynamicBytes;
+  v.smem[1] = libra::DecodeSmem<128, NW, ST, 1>::kDynamicBytes;
   return v;
 }
 const std::vector<Fp8Variant>& fp8_variants() {
@@ -241,10 +246,11 @@ int encode_pool_map(libra_handle_t h, const void* base, CUtensorMap* map, int* p
                  {h->stride_head, h->cfg.num_kv_heads, 1u, 1},
                  {h->stride_page, h->cfg.num_pages, 1u, 2}};
   std::stable_sort(dims, dims + 3, [](const Dim& a, const Dim& b) { return a.stride < b.stride; });
-  const int eb = h->fp8 ? 1 : 2;   // bytes per element; a box row is 128 bytes either way
+  const int eb = h->fp8 ? 1 : 2;   // bytes per element; a box row is 128 bytes, or the whole 64-byte row of an 8-bit cache at head_dim 64
+  const int row_bytes = std::min(128, h->cfg.head_dim * eb);
   cuuint64_t gdim[4] = {cuuint64_t(h->cfg.head_dim), 0, 0, 0};
   cuuint64_t gstride[3];
-  cuuint32_t box[4] = {cuuint32_t(128 / eb), 0, 0, 0};
+  cuuint32_t box[4] = {cuuint32_t(row_bytes / eb), 0, 0, 0};
   cuuint32_t estride[4] = {1, 1, 1, 1};
   for (int i = 0; i < 3; ++i) {
     gdim[i + 1] = cuuint64_t(dims[i].size);
@@ -255,7 +261,8 @@ int encode_pool_map(libra_handle_t h, const void* base, CUtensorMap* map, int* p
     if (dims[i].kind == 2) *pos_page = i + 1;
   }
   CUresult r = h->encode(map, h->fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gdim, gstride, box, estride,
-                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     h->last_cuda_error = int(cudaErrorInvalidValue);
@@ -460,9 +467,9 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
     }
     if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
     for (const Fp8Variant& fv : fp8_variants()) {
-      for (int di = 0; di < 4 && e == cudaSuccess; ++di) {
-        e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fv.fn[di >> 1][di & 1]),
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, fv.smem);
+      for (int i = 0; i < 8 && e == cudaSuccess; ++i) {
+        e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fv.fn[i >> 2][(i >> 1) & 1][i & 1]),
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, fv.smem[i >> 2]);
       }
     }
     if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
@@ -725,7 +732,6 @@ int libra_set_kv_dtype(libra_handle_t h, int32_t dtype, float k_scale, float v_s
   if (!h || (dtype != LIBRA_KV_BF16 && dtype != LIBRA_KV_E4M3)) return LIBRA_INVALID_ARGUMENT;
   if (dtype == LIBRA_KV_E4M3) {
     if (!(k_scale > 0.f) || !(v_scale > 0.f) || !std::isfinite(k_scale) || !std::isfinite(v_scale)) return LIBRA_INVALID_ARGUMENT;
-    if (h->cfg.head_dim != 128) return LIBRA_UNSUPPORTED_SHAPE;
     // strides are in elements = bytes here: the tiled copies need 16-byte multiples
     if (h->stride_page % 16 || h->stride_head % 16 || h->stride_token % 16) return LIBRA_INVALID_ARGUMENT;
   }
@@ -895,9 +901,9 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
       if (!ni && !loads_only && auto_variant == kVariantShortUnits) fp8_auto = kFp8ShortUnits;
       if (!ni && !loads_only && auto_variant == kVariantTinyUnits) fp8_auto = kFp8TinyUnits;
       const Fp8Variant& fv = fp8_variants()[h->fp8_variant >= 0 ? h->fp8_variant : fp8_auto];
-      fn = fv.fn[loads_only ? 1 : 0][ni];
+      fn = fv.fn[di][loads_only ? 1 : 0][ni];
       lc.blockDim = dim3(unsigned(fv.warps * 32));
-      lc.dynamicSmemBytes = size_t(fv.smem);
+      lc.dynamicSmemBytes = size_t(fv.smem[di]);
     }
     lc.stream = st;
     cudaLaunchAttribute attr[1];
@@ -1101,12 +1107,16 @@ int kv_move_impl(libra_handle_t h, bool gather, void* k_pages, void* v_pages, vo
   const int pages = (max_seq_len + h->cfg.page_size - 1) / h->cfg.page_size;
   dim3 grid(unsigned((pages + libra::kMovePagesPerBlock - 1) / libra::kMovePagesPerBlock), unsigned(batch));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (h->cfg.head_dim == 128 && !h->fp8) {
+  const int row_units = h->cfg.head_dim / int(unit);   // two-byte elements per row: 128, 64, or 32 (8-bit, head_dim 64)
+  if (row_units == 128) {
     if (gather) libra::kv_move_kernel<128, true><<<grid, libra::kMoveThreads, 0, st>>>(p);
     else libra::kv_move_kernel<128, false><<<grid, libra::kMoveThreads, 0, st>>>(p);
-  } else {
+  } else if (row_units == 64) {
     if (gather) libra::kv_move_kernel<64, true><<<grid, libra::kMoveThreads, 0, st>>>(p);
     else libra::kv_move_kernel<64, false><<<grid, libra::kMoveThreads, 0, st>>>(p);
+  } else {
+    if (gather) libra::kv_move_kernel<32, true><<<grid, libra::kMoveThreads, 0, st>>>(p);
+    else libra::kv_move_kernel<32, false><<<grid, libra::kMoveThreads, 0, st>>>(p);
   }
   LIBRA_CUDA_TRY(h, cudaGetLastError());
   ++h->launches;

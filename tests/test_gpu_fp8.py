@@ -157,10 +157,6 @@ def test_split_and_unsplit_agree_and_runs_reproduce(lib):
 
 def test_what_is_not_supported_says_so(lib):
     import torch
-    h64 = lib.Handle(4, 1, 64, 64, 4, 8)
-    with pytest.raises(lib.LibraError):
-        h64.set_kv_dtype(lib.KV_E4M3, 1.0, 1.0)           # head_dim 64
-    h64.close()
     h = lib.Handle(8, 2, 128, 64, 4, 8)
     for bad in ((0.0, 1.0), (1.0, -1.0), (float("inf"), 1.0), (float("nan"), 1.0)):
         with pytest.raises(lib.LibraError):
@@ -299,3 +295,90 @@ def test_block_shape_follows_the_longest_unit(lib):
         assert h.debug_error_word() == 0
         assert np.array_equal(H.bf16_dev_to_f32(out), auto)
         h.close()
+
+
+CASES_D64 = [
+    (4, 1, [1, 7, 64, 300]),                   # the tiny workload's shape
+    (8, 2, [255, 256, 257, 1, 700, 0]),
+    (24, 2, [900, 130, 17]),                   # G = 12: two column tiles
+    (8, 8, [100, 1000, 33]),                   # G = 1
+]
+
+
+@pytest.mark.parametrize("layout", ["HND", "NHD"])
+@pytest.mark.parametrize("case", range(len(CASES_D64)))
+def test_head_dim_64(lib, case, layout):
+    # rows of 64 bytes: tiles of 1 KB under the 64-byte swizzle
+    Hq, Hkv, lens = CASES_D64[case]
+    lens_a, bt, q, k8, v8 = W.random_case_e4m3(650 + case, len(lens), Hq, Hkv, 64, lens)
+    ref, _ = O.paged_decode_attention_fp8(q, k8, v8, bt, lens_a, 0.75, 1.5)
+    for plan in (None, small_plan(lib)):
+        got = run_fp8(lib, q, k8, v8, bt, lens_a, 0.75, 1.5, layout=layout, plan=plan)
+        check(got, ref, f"d64 case {case} {layout} plan={'default' if plan is None else 'small'}")
+
+
+def test_head_dim_64_every_code_and_dim_lands_where_it_should(lib):
+    import math
+    L, d = 40, 64
+    lens_a, bt, _, k8, v8 = W.random_case_e4m3(660, 1, 2, 1, d, [L])
+    finite = np.array([c for c in range(256) if c not in (0x7F, 0xFF)], dtype=np.uint8)
+    for t in range(L):
+        v8[bt[0, t // 16], 0, t % 16] = finite[(np.arange(d) * 3 + 11 * t) % len(finite)]
+    for tstar, j in ((0, 0), (15, 1), (16, 2), (17, 31), (31, 32), (39, 63), (22, 47)):
+        k8[bt[0], 0] = 0
+        k8[bt[0, tstar // 16], 0, tstar % 16, j] = 0x50          # code of 8.0
+        qrow = np.zeros(d, dtype=np.float32)
+        qrow[j] = 256.0
+        q = np.broadcast_to(W.f32_to_bf16_bits(qrow), (1, 2, d)).copy()
+        assert 8 * 256 / math.sqrt(d) > 150
+        for plan in (None, small_plan(lib)):
+            got = run_fp8(lib, q, k8, v8, bt, lens_a, plan=plan)
+            want = O.e4m3_to_f64(v8[bt[0, tstar // 16], 0, tstar % 16])
+            assert np.array_equal(got[0, 0].astype(np.float64), want), (tstar, j)
+
+
+def test_head_dim_64_append_and_move(lib):
+    import torch
+    from oracle import kv_move_oracle as M
+    dev = torch.device("cuda:0")
+    lens = [1, 16, 17, 300, 33]
+    B, Hq, Hkv, d = len(lens), 8, 4, 64
+    lens_a, bt, q, k8, v8 = W.random_case_e4m3(670, B, Hq, Hkv, d, lens, poison=False)
+    rng = np.random.default_rng(671)
+    k_new = rng.integers(0, 0x78, size=(B, Hkv, d)).astype(np.uint8)
+    v_new = rng.integers(0, 0x78, size=(B, Hkv, d)).astype(np.uint8)
+    k_ref, v_ref = k8.copy(), v8.copy()
+    for b, n in enumerate(lens_a):
+        k_ref[bt[b, (n - 1) // 16], :, (n - 1) % 16, :] = k_new[b]
+        v_ref[bt[b, (n - 1) // 16], :, (n - 1) % 16, :] = v_new[b]
+    ref, _ = O.paged_decode_attention_fp8(q, k_ref, v_ref, bt, lens_a)
+    h = lib.Handle(Hq, Hkv, d, k8.shape[0], B, bt.shape[1], plan=small_plan(lib))
+    h.set_kv_dtype(lib.KV_E4M3, 1.0, 1.0)
+    ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=dev)
+    qd, btd = H.to_dev(q, dev), H.to_dev(bt, dev)
+    kd, vd = torch.from_numpy(k8).to(dev), torch.from_numpy(v8).to(dev)
+    knd, vnd = torch.from_numpy(k_new).to(dev), torch.from_numpy(v_new).to(dev)
+    lens_dev = torch.from_numpy(lens_a).to(dev)
+    out = torch.full((B, Hq, d), H.CANARY, dtype=torch.int16, device=dev)
+    st = torch.cuda.current_stream().cuda_stream
+    h.plan(lens_a, ws.data_ptr(), ws.numel(), st)
+    h.decode_attn_append(qd.data_ptr(), knd.data_ptr(), vnd.data_ptr(), kd.data_ptr(), vd.data_ptr(), btd.data_ptr(),
+                         lens_dev.data_ptr(), out.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert h.debug_error_word() == 0
+    check(H.bf16_dev_to_f32(out), ref, "d64 append")
+    assert np.array_equal(kd.cpu().numpy(), k_ref) and np.array_equal(vd.cpu().numpy(), v_ref)
+    # gather heads 1..2 of the updated pools
+    offs = np.concatenate([[0], np.cumsum(lens_a.astype(np.int64))])
+    doffs = torch.from_numpy(offs[:-1].copy()).to(dev)
+    err = torch.zeros(1, dtype=torch.int32, device=dev)
+    total = int(offs[-1])
+    k_dense = torch.full((total, 2, d), 0x7F, dtype=torch.uint8, device=dev)
+    v_dense = torch.full((total, 2, d), 0x7F, dtype=torch.uint8, device=dev)
+    h.kv_gather(kd.data_ptr(), vd.data_ptr(), btd.data_ptr(), lens_dev.data_ptr(), doffs.data_ptr(), B, int(lens_a.max()),
+                1, 2, k_dense.data_ptr(), v_dense.data_ptr(), err.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    assert np.array_equal(k_dense.cpu().numpy(), M.gather(k_ref, bt, lens_a, 1, 2))
+    assert np.array_equal(v_dense.cpu().numpy(), M.gather(v_ref, bt, lens_a, 1, 2))
+    h.close()
