@@ -36,8 +36,9 @@ typedef void (*DecodeKernelFn)(const CUtensorMap, const CUtensorMap, const Decod
 
 struct Variant {
   int warps, stages;
-  DecodeKernelFn fn[2][2];  // [D == 128][NT - 1]
-  int smem[2][2];           // dynamic bytes
+  DecodeKernelFn fn[2][2];         // [D == 128][NT - 1]
+  DecodeKernelFn fn_append[2][2];  // the same with the KV append compiled in
+  int smem[2][2];                  // dynamic bytes
 };
 
 
@@ -50,6 +51,10 @@ Variant make_variant() {
   v.fn[0][1] = libra::decode_kernel<64, 2, NW, ST>;
   v.fn[1][0] = libra::decode_kernel<128, 1, NW, ST>;
   v.fn[1][1] = libra::decode_kernel<128, 2, NW, ST>;
+  v.fn_append[0][0] = libra::decode_kernel<64, 1, NW, ST, false, false, true>;
+  v.fn_append[0][1] = libra::decode_kernel<64, 2, NW, ST, false, false, true>;
+  v.fn_append[1][0] = libra::decode_kernel<128, 1, NW, ST, false, false, true>;
+  v.fn_append[1][1] = libra::decode_kernel<128, 2, NW, ST, false, false, true>;
   v.smem[0][0] = v.smem[0][1] = libra::DecodeSmem<64, NW, ST>::kDynamicBytes;
   v.smem[1][0] = v.smem[1][1] = libra::DecodeSmem<128, NW, ST>::kDynamicBytes;
   return v;
@@ -95,8 +100,9 @@ const int kLoadsOnlySmem[2] = {libra::DecodeSmem<64, kLoadsOnlyWarps, kLoadsOnly
 constexpr int kFp8OneTile = 2, kFp8TwoTiles = 1, kFp8ShortUnits = 5, kFp8TinyUnits = 6;
 struct Fp8Variant {
   int warps, stages;
-  DecodeKernelFn fn[2][2][2];   // [D == 128][loads only][NT - 1]
-  int smem[2];                  // [D == 128]
+  DecodeKernelFn fn[2][2][2];      // [D == 128][loads only][NT - 1]
+  DecodeKernelFn fn_append[2][2];  // [D == 128][NT - 1], with the KV append compiled in
+  int smem[2];                     // [D == 128]
 };
 template <int NW, int ST>
 Fp8Variant make_fp8_variant() {
@@ -111,6 +117,10 @@ Fp8Variant make_fp8_variant() {
   v.fn[1][0][1] = libra::decode_kernel<128, 2, NW, ST, false, true>;
   v.fn[1][1][0] = libra::decode_kernel<128, 1, NW, ST, true, true>;
   v.fn[1][1][1] = libra::decode_kernel<128, 2, NW, ST, true, true>;
+  v.fn_append[0][0] = libra::decode_kernel<64, 1, NW, ST, false, true, true>;
+  v.fn_append[0][1] = libra::decode_kernel<64, 2, NW, ST, false, true, true>;
+  v.fn_append[1][0] = libra::decode_kernel<128, 1, NW, ST, false, true, true>;
+  v.fn_append[1][1] = libra::decode_kernel<128, 2, NW, ST, false, true, true>;
   v.smem[0] = libra::DecodeSmem<64, NW, ST, 1>::kDynamicBytes;
   v.smem[1] = libra::DecodeSmem<128, NW, ST, 1>::kDynamicBytes;
   return v;
@@ -455,6 +465,10 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
           if (!v.fn[di][ni]) continue;
           e = cudaFuncSetAttribute(reinterpret_cast<const void*>(v.fn[di][ni]),
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem[di][ni]);
+          if (e == cudaSuccess) {
+            e = cudaFuncSetAttribute(reinterpret_cast<const void*>(v.fn_append[di][ni]),
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem[di][ni]);
+          }
           if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
         }
       }
@@ -470,6 +484,10 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
       for (int i = 0; i < 8 && e == cudaSuccess; ++i) {
         e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fv.fn[i >> 2][(i >> 1) & 1][i & 1]),
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, fv.smem[i >> 2]);
+      }
+      for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
+        e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fv.fn_append[i >> 1][i & 1]),
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, fv.smem[i >> 1]);
       }
     }
     if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
@@ -893,7 +911,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     // resident while that kernel drains; inside, they wait for it to finish before reading any input
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(grid);
-    DecodeKernelFn fn = loads_only ? kLoadsOnlyFn[di][ni] : v.fn[di][ni];
+    DecodeKernelFn fn = loads_only ? kLoadsOnlyFn[di][ni] : (k_new ? v.fn_append[di][ni] : v.fn[di][ni]);
     lc.blockDim = dim3(unsigned((loads_only ? kLoadsOnlyWarps : v.warps) * 32));
     lc.dynamicSmemBytes = size_t(loads_only ? kLoadsOnlySmem[di] : v.smem[di][ni]);
     if (h->fp8) {
@@ -901,7 +919,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
       if (!ni && !loads_only && auto_variant == kVariantShortUnits) fp8_auto = kFp8ShortUnits;
       if (!ni && !loads_only && auto_variant == kVariantTinyUnits) fp8_auto = kFp8TinyUnits;
       const Fp8Variant& fv = fp8_variants()[h->fp8_variant >= 0 ? h->fp8_variant : fp8_auto];
-      fn = fv.fn[di][loads_only ? 1 : 0][ni];
+      fn = (k_new && !loads_only) ? fv.fn_append[di][ni] : fv.fn[di][loads_only ? 1 : 0][ni];
       lc.blockDim = dim3(unsigned(fv.warps * 32));
       lc.dynamicSmemBytes = size_t(fv.smem[di]);
     }
