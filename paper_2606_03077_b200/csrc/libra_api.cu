@@ -911,7 +911,8 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     // resident while that kernel drains; inside, they wait for it to finish before reading any input
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(grid);
-    DecodeKernelFn fn = loads_only ? kLoadsOnlyFn[di][ni] : (k_new ? v.fn_append[di][ni] : v.fn[di][ni]);
+    const bool full = k_new != nullptr || q_len > 1;   // the build with the append and several query tokens in it
+    DecodeKernelFn fn = loads_only ? kLoadsOnlyFn[di][ni] : (full ? v.fn_append[di][ni] : v.fn[di][ni]);
     lc.blockDim = dim3(unsigned((loads_only ? kLoadsOnlyWarps : v.warps) * 32));
     lc.dynamicSmemBytes = size_t(loads_only ? kLoadsOnlySmem[di] : v.smem[di][ni]);
     if (h->fp8) {
@@ -919,7 +920,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
       if (!ni && !loads_only && auto_variant == kVariantShortUnits) fp8_auto = kFp8ShortUnits;
       if (!ni && !loads_only && auto_variant == kVariantTinyUnits) fp8_auto = kFp8TinyUnits;
       const Fp8Variant& fv = fp8_variants()[h->fp8_variant >= 0 ? h->fp8_variant : fp8_auto];
-      fn = (k_new && !loads_only) ? fv.fn_append[di][ni] : fv.fn[di][loads_only ? 1 : 0][ni];
+      fn = (full && !loads_only) ? fv.fn_append[di][ni] : fv.fn[di][loads_only ? 1 : 0][ni];
       lc.blockDim = dim3(unsigned(fv.warps * 32));
       lc.dynamicSmemBytes = size_t(fv.smem[di]);
     }
