@@ -585,28 +585,22 @@ def e2e_measure(rep: Replica, steps: int):
 
 
 def e2e_resident_kv_measure(rep: Replica, steps: int):
-    """One decode step as a serving engine issues it: the KV cache stays in HBM; the step's own inputs (q,
-    block table, lengths) start in pinned host memory and the output ends there; every step is
-    synchronised (latency, not pipelined throughput)."""
+    """One decode step as a serving engine issues it, through libra_decode_attn_host_io: the KV cache stays in
+    HBM; the step's own inputs (q, block table, lengths) start in pinned host memory and the output ends there;
+    the call returns after synchronising its stream (latency, not pipelined throughput)."""
     torch = rep.torch
     k, v = rep.pools[0]
     hq = rep.q.cpu().pin_memory()
     hbt = rep.bts[0].cpu().pin_memory()
     hl = rep.lens_dev[0].cpu().pin_memory()
     hout = torch.zeros(rep.out.shape, dtype=torch.bfloat16).pin_memory()
-    dq, dbt, dl = torch.empty_like(rep.q), torch.empty_like(rep.bts[0]), torch.empty_like(rep.lens_dev[0])
-    lens_host = rep.layouts[0].seq_lens
-    stream = torch.cuda.current_stream()
-    st = stream.cuda_stream
+    stg = torch.empty(rep.h.host_io_staging_size(rep.w.batch), dtype=torch.uint8, device=rep.dev)
+    st = torch.cuda.current_stream().cuda_stream
 
     def one():
-        dq.copy_(hq, non_blocking=True)
-        dbt.copy_(hbt, non_blocking=True)
-        dl.copy_(hl, non_blocking=True)
-        rep.h.plan(lens_host, rep.ws.data_ptr(), rep.ws.numel(), st)
-        rep.h.decode_attn(dq.data_ptr(), k.data_ptr(), v.data_ptr(), dbt.data_ptr(), dl.data_ptr(), rep.out.data_ptr(), st)
-        hout.copy_(rep.out, non_blocking=True)
-        stream.synchronize()
+        rep.h.decode_attn_host_io(hq.data_ptr(), k.data_ptr(), v.data_ptr(), hbt.data_ptr(), hl.data_ptr(),
+                                  rep.w.batch, hout.data_ptr(), stg.data_ptr(), stg.numel(), rep.ws.data_ptr(),
+                                  rep.ws.numel(), st)
 
     for _ in range(5):
         one()
@@ -614,11 +608,15 @@ def e2e_resident_kv_measure(rep: Replica, steps: int):
     for _ in range(steps):
         one()
     ms = (time.perf_counter() - t0) / steps * 1e3
+    rep.step(st)
+    torch.cuda.synchronize()
+    same = bool(torch.equal(hout.to(rep.dev), rep.out)) if len(rep.layouts) == 1 else None   # pool copies hold the same data
     return {"value": rep.layouts[0].kv_bytes / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms, "steps": steps,
             "h2d_bytes_per_step": int(hq.numel() * 2 + hbt.numel() * 4 + hl.numel() * 4),
-            "d2h_bytes_per_step": int(hout.numel() * 2),
-            "note": "KV pools resident in HBM (as in any serving engine); q, block table and lengths copied from pinned "
-                    "host memory and the output copied back every step; host-synchronised per step, wall clock"}
+            "d2h_bytes_per_step": int(hout.numel() * 2 + 4), "matches_resident_run": same,
+            "note": "libra_decode_attn_host_io: KV pools resident in HBM (as in any serving engine); q, block table and "
+                    "lengths copied from pinned host memory and the output copied back every step; the call "
+                    "synchronises its stream, wall clock"}
 
 
 def kv_migration_measure(rep: Replica, reps: int = 10):

@@ -314,6 +314,17 @@ int libra_decode_attn_host(libra_handle_t handle, const void* q_host, const void
 /* Bytes of device staging libra_decode_attn_host needs for `batch` sequences. */
 int libra_host_staging_size(libra_handle_t handle, int32_t batch, size_t* bytes);
 
+/* The step as a serving loop sees it: the cache stays on the device (k_pages, v_pages: device pointers, bf16 or
+ * E4M3 as set on the handle) and only what changes every step crosses the bus: q, the block table and the lengths
+ * come from host memory, `out` goes back to it.  Copies them to `staging_dev` (at least libra_host_io_staging_size
+ * bytes, 256-byte aligned), plans, runs D and C, copies the result to out_host, all on `stream`, and returns after
+ * synchronising it.  Errors: as libra_decode_attn_host. */
+int libra_decode_attn_host_io(libra_handle_t handle, const void* q_host, const void* k_pages, const void* v_pages,
+                              const int32_t* block_table_host, const int32_t* seq_lens_host, int32_t batch,
+                              void* out_host, void* staging_dev, size_t staging_bytes, void* workspace_dev,
+                              size_t workspace_bytes, void* stream);
+int libra_host_io_staging_size(libra_handle_t handle, int32_t batch, size_t* bytes);
+
 /* Size of the scratch region built into the library for libra_decode_attn_static: 8 MiB of device
  * memory that every GPU holds from the moment it loads the library until the process exits. */
 #define LIBRA_STATIC_SCRATCH_BYTES (8u << 20)

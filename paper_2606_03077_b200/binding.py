@@ -82,6 +82,9 @@ SIGNATURES = {
                                          C.c_size_t, _vp]),
     "libra_decode_attn_static": (C.c_int, [_vp, _i32p, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_host_staging_size": (C.c_int, [_vp, C.c_int32, C.POINTER(C.c_size_t)]),
+    "libra_decode_attn_host_io": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, C.c_int32, _vp, _vp, C.c_size_t, _vp,
+                                            C.c_size_t, _vp]),
+    "libra_host_io_staging_size": (C.c_int, [_vp, C.c_int32, C.POINTER(C.c_size_t)]),
     "libra_last_cuda_error": (C.c_int, [_vp]),
     "libra_debug_error_word": (C.c_int, [_vp, C.POINTER(C.c_uint32)]),
     "libra_kv_gather": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _vp, _vp,
@@ -348,6 +351,18 @@ class Handle:
         _check(lib.libra_decode_attn_host(self._h, q_host_ptr, k_host_ptr, v_host_ptr, block_table_host_ptr,
                                           seq_lens_host_ptr, batch, out_host_ptr, staging_ptr, staging_bytes,
                                           workspace_ptr, workspace_bytes, stream), "libra_decode_attn_host")
+
+    def host_io_staging_size(self, batch: int) -> int:
+        n = C.c_size_t(0)
+        _check(lib.libra_host_io_staging_size(self._h, batch, C.byref(n)), "libra_host_io_staging_size")
+        return n.value
+
+    def decode_attn_host_io(self, q_host_ptr: int, k_ptr: int, v_ptr: int, block_table_host_ptr: int,
+                            seq_lens_host_ptr: int, batch: int, out_host_ptr: int, staging_ptr: int,
+                            staging_bytes: int, workspace_ptr: int, workspace_bytes: int, stream: int) -> None:
+        _check(lib.libra_decode_attn_host_io(self._h, q_host_ptr, k_ptr, v_ptr, block_table_host_ptr,
+                                             seq_lens_host_ptr, batch, out_host_ptr, staging_ptr, staging_bytes,
+                                             workspace_ptr, workspace_bytes, stream), "libra_decode_attn_host_io")
 
     def last_cuda_error(self) -> int:
         return lib.libra_last_cuda_error(self._h)

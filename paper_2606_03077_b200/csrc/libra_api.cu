@@ -1046,6 +1046,56 @@ int libra_decode_attn_host(libra_handle_t h, const void* q_host, const void* k_p
   return word ? LIBRA_DEVICE_FLAGGED : LIBRA_OK;
 }
 
+int libra_host_io_staging_size(libra_handle_t h, int32_t batch, size_t* bytes) {
+  if (!h || !bytes || batch < 0 || batch > h->cfg.max_batch) return LIBRA_INVALID_ARGUMENT;
+  const size_t qo = align_up(size_t(batch) * h->cfg.num_q_heads * h->cfg.head_dim * 2, 256);
+  const size_t bt = align_up(size_t(batch) * h->cfg.block_table_ld * 4, 256);
+  const size_t sl = align_up(size_t(batch) * 4, 256);
+  *bytes = 2 * qo + bt + sl;
+  return LIBRA_OK;
+}
+
+int libra_decode_attn_host_io(libra_handle_t h, const void* q_host, const void* k_pages, const void* v_pages,
+                              const int32_t* block_table_host, const int32_t* seq_lens_host, int32_t batch,
+                              void* out_host, void* staging_dev, size_t staging_bytes, void* workspace_dev,
+                              size_t workspace_bytes, void* stream) {
+  if (!h || !q_host || !k_pages || !v_pages || !block_table_host || !seq_lens_host || !out_host || !staging_dev ||
+      batch <= 0) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  if (reinterpret_cast<uintptr_t>(staging_dev) % 256 != 0) return LIBRA_INVALID_ARGUMENT;
+  size_t need = 0;
+  int rc = libra_host_io_staging_size(h, batch, &need);
+  if (rc != LIBRA_OK) return rc;
+  if (staging_bytes < need) return LIBRA_WORKSPACE_TOO_SMALL;
+  DeviceGuard guard(h->cfg.device);
+  if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  const size_t q_bytes = size_t(batch) * h->cfg.num_q_heads * h->cfg.head_dim * 2;
+  const size_t bt_bytes = size_t(batch) * h->cfg.block_table_ld * 4;
+  const size_t sl_bytes = size_t(batch) * 4;
+  uint8_t* d_q = static_cast<uint8_t*>(staging_dev);
+  uint8_t* d_out = d_q + align_up(q_bytes, 256);
+  uint8_t* d_bt = d_out + align_up(q_bytes, 256);
+  uint8_t* d_sl = d_bt + align_up(bt_bytes, 256);
+
+  rc = libra_plan(h, seq_lens_host, batch, workspace_dev, workspace_bytes, stream);
+  if (rc != LIBRA_OK) return rc;
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(d_q, q_host, q_bytes, cudaMemcpyHostToDevice, st));
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(d_bt, block_table_host, bt_bytes, cudaMemcpyHostToDevice, st));
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(d_sl, seq_lens_host, sl_bytes, cudaMemcpyHostToDevice, st));
+  rc = libra_decode_attn(h, d_q, k_pages, v_pages, reinterpret_cast<const int32_t*>(d_bt),
+                         reinterpret_cast<const int32_t*>(d_sl), d_out, stream);
+  if (rc != LIBRA_OK) return rc;
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(out_host, d_out, q_bytes, cudaMemcpyDeviceToHost, st));
+  uint32_t word = 0;
+  LIBRA_CUDA_TRY(h, cudaMemcpyAsync(&word, workspace_dev, 4, cudaMemcpyDeviceToHost, st));
+  LIBRA_CUDA_TRY(h, cudaStreamSynchronize(st));
+  if (word) LIBRA_CUDA_TRY(h, cudaMemsetAsync(workspace_dev, 0, 4, st));
+  return word ? LIBRA_DEVICE_FLAGGED : LIBRA_OK;
+}
+
 int libra_decode_attn_static(libra_handle_t h, const int32_t* seq_lens_host, int32_t batch, const void* q,
                              const void* k_pages, const void* v_pages, const int32_t* block_table,
                              const int32_t* seq_lens, void* out, void* stream) {

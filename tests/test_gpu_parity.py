@@ -347,6 +347,39 @@ def test_host_buffer_entry_point(lib):
     h.close()
 
 
+def test_host_io_entry_point_with_resident_cache(lib):
+    """q, block table and lengths from pinned host memory, the cache on the device: the bits of the all-device call."""
+    import torch
+    dev = torch.device("cuda:0")
+    lens = [700, 1, 0, 33, 20000]
+    lens_a, bt, q, k, v = W.random_case(55, 5, 32, 8, 128, lens)
+    base = H.run_host_case(lib, q, k, v, bt, lens_a)
+    h = lib.Handle(32, 8, 128, k.shape[0], 8, bt.shape[1])
+    ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=dev)
+    stg = torch.empty(h.host_io_staging_size(5), dtype=torch.uint8, device=dev)
+    dk, dv = H.to_dev(k, dev), H.to_dev(v, dev)
+    hq = torch.from_numpy(q.view(np.int16)).pin_memory()
+    hbt, hl = torch.from_numpy(bt.copy()).pin_memory(), torch.from_numpy(lens_a.copy()).pin_memory()
+    hout = torch.full((5, 32, 128), H.CANARY, dtype=torch.int16).pin_memory()
+    st = torch.cuda.current_stream().cuda_stream
+    h.decode_attn_host_io(hq.data_ptr(), dk.data_ptr(), dv.data_ptr(), hbt.data_ptr(), hl.data_ptr(), 5, hout.data_ptr(),
+                          stg.data_ptr(), stg.numel(), ws.data_ptr(), ws.numel(), st)
+    assert np.array_equal(hout.view(torch.bfloat16).float().numpy(), base)
+    with pytest.raises(lib.LibraError):     # staging too small
+        h.decode_attn_host_io(hq.data_ptr(), dk.data_ptr(), dv.data_ptr(), hbt.data_ptr(), hl.data_ptr(), 5,
+                              hout.data_ptr(), stg.data_ptr(), 256, ws.data_ptr(), ws.numel(), st)
+    bad = bt.copy(); bad[4, 3] = k.shape[0] + 9     # a page id outside the pool: reported by the call itself
+    hbad = torch.from_numpy(bad).pin_memory()
+    with pytest.raises(lib.LibraError) as ei:
+        h.decode_attn_host_io(hq.data_ptr(), dk.data_ptr(), dv.data_ptr(), hbad.data_ptr(), hl.data_ptr(), 5,
+                              hout.data_ptr(), stg.data_ptr(), stg.numel(), ws.data_ptr(), ws.numel(), st)
+    assert ei.value.status == lib.DEVICE_FLAGGED
+    h.decode_attn_host_io(hq.data_ptr(), dk.data_ptr(), dv.data_ptr(), hbt.data_ptr(), hl.data_ptr(), 5, hout.data_ptr(),
+                          stg.data_ptr(), stg.numel(), ws.data_ptr(), ws.numel(), st)     # and the handle works on
+    assert np.array_equal(hout.view(torch.bfloat16).float().numpy(), base)
+    h.close()
+
+
 def test_early_prefetch_is_bit_identical_behind_a_cache_write_kernel(lib):
     """Steps issued back to back, each preceded by kernels that write q and the newest token's K/V rows (what the
     promise of libra_set_early_prefetch allows the preceding kernel to do): same bits as the default."""
