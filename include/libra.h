@@ -473,6 +473,21 @@ int libra_ring_step(int32_t device, void* dst, const void* own, const void* rece
                     const uint32_t* ready_flag, uint32_t expected, uint32_t timeout_us, uint32_t* status_dev,
                     int32_t num_blocks, void* stream);
 
+/* Merge of attention results over disjoint parts of the same sequences: the one exchange step of cutting a
+ * sequence's TOKENS across GPUs (the paper's tensor parallelism cuts the cache by attention head, Section 5.3, and
+ * needs none; this is the remaining way to shard the step).  Each holder of a part runs the decode call with
+ * libra_set_lse_output; once the (out, lse) pairs are gathered,
+ *     M = max_i lse_i,  w_i = exp(lse_i - M),  out = sum_i w_i out_i / sum_i w_i,  lse = M + ln sum_i w_i
+ * gives the attention over the whole sequence (the rule of step C).  parts_out: bf16 [n_parts][rows][head_dim],
+ * parts_lse: float32 [n_parts][rows] (-inf = that part holds no token for the row; its out row is ignored), out:
+ * bf16 [rows][head_dim], lse_out: float32 [rows] or NULL; device pointers on `device`, 16-byte aligned, out not
+ * overlapping the inputs; rows = batch * q_len * num_q_heads in any order common to all parts; head_dim 64 or 128;
+ * 1 <= n_parts <= 64.  A row whose parts are all empty gets zeros and lse = -inf.  Parts are added in index order
+ * in float32: bit-reproducible.  Asynchronous on `stream`.
+ * Errors: INVALID_ARGUMENT, UNSUPPORTED_SHAPE (head_dim), CUDA_ERROR. */
+int libra_merge_parts(int32_t device, const void* parts_out, const float* parts_lse, int32_t n_parts, int64_t rows,
+                      int32_t head_dim, void* out, float* lse_out, void* stream);
+
 /* Self-test of the kernels' bounded waits: enqueues a one-warp kernel that waits, with a limit of a few
  * milliseconds, on a copy barrier that nothing completes.  It must return (no hang, no trap) and leave
  * LIBRA_ERR_WAIT_TIMEOUT in the device error word of the last planned workspace, which is how a real

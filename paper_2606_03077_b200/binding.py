@@ -68,6 +68,7 @@ SIGNATURES = {
     "libra_decode_attn_multi_append": (C.c_int, [_vp, _vp, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_ring_step": (C.c_int, [C.c_int32, _vp, _vp, _vp, C.c_size_t, C.c_int32, _vp, C.c_uint32, C.c_uint32, _vp, C.c_int32,
                                   _vp]),
+    "libra_merge_parts": (C.c_int, [C.c_int32, _vp, _vp, C.c_int32, C.c_int64, C.c_int32, _vp, _vp, _vp]),
     "libra_debug_stream_read": (C.c_int, [_vp, _vp, C.c_size_t, _vp]),
     "libra_debug_gather_read": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_set_combine_mode": (C.c_int, [_vp, C.c_int32]),
@@ -165,6 +166,13 @@ def libra_ring_step(device: int, dst_ptr: int, own_ptr: int, received_ptr: int, 
     """One copy / reduce step of the ring all-reduce's data plane (own_ptr = 0 for a copy step)."""
     _check(lib.libra_ring_step(device, dst_ptr, own_ptr or None, received_ptr, nbytes, dtype, ready_flag_ptr, expected,
                                timeout_us, status_ptr, num_blocks, stream), "libra_ring_step")
+
+
+def libra_merge_parts(device: int, parts_out_ptr: int, parts_lse_ptr: int, n_parts: int, rows: int, head_dim: int,
+                      out_ptr: int, lse_out_ptr: int, stream: int) -> None:
+    """Log-sum-exp merge of (out, lse) pairs computed over disjoint parts of the same sequences."""
+    _check(lib.libra_merge_parts(device, parts_out_ptr, parts_lse_ptr, n_parts, rows, head_dim, out_ptr,
+                                 lse_out_ptr or None, stream), "libra_merge_parts")
 
 
 def libra_rollout_dp(n_gpus: int, lengths, tp_set, cost_coef, scan: bool = False):

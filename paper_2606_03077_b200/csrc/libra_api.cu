@@ -13,6 +13,7 @@
 #include "decode_kernel.cuh"
 #include "kv_move_kernel.cuh"
 #include "libra.h"
+#include "merge_kernel.cuh"
 #include "plan_kernel.cuh"
 #include "plan_layout.hpp"
 #include "planner.hpp"
@@ -1252,6 +1253,35 @@ int libra_debug_stream_read(libra_handle_t h, const void* buf_dev, size_t bytes,
   LIBRA_CUDA_TRY(h, cudaGetLastError());
   ++h->launches;
   h->last_stream = stream;
+  return LIBRA_OK;
+}
+
+int libra_merge_parts(int32_t device, const void* parts_out, const float* parts_lse, int32_t n_parts, int64_t rows,
+                      int32_t head_dim, void* out, float* lse_out, void* stream) {
+  if (device < 0 || !parts_out || !parts_lse || !out || n_parts < 1 || n_parts > 64 || rows < 0) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  if (head_dim != 64 && head_dim != 128) return LIBRA_UNSUPPORTED_SHAPE;
+  if (reinterpret_cast<uintptr_t>(parts_out) % 16 || reinterpret_cast<uintptr_t>(parts_lse) % 16 ||
+      reinterpret_cast<uintptr_t>(out) % 16 || reinterpret_cast<uintptr_t>(lse_out) % 4) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  if (rows > (int64_t(1) << 31) * libra::kMergeWarps - 1) return LIBRA_INVALID_ARGUMENT;   // grid limit
+  if (rows == 0) return LIBRA_OK;
+  DeviceGuard guard(device);
+  if (guard.err != cudaSuccess) return fail_cuda(nullptr, guard.err);
+  libra::MergeParams p;
+  p.parts_out = static_cast<const __nv_bfloat16*>(parts_out);
+  p.parts_lse = parts_lse;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.lse_out = lse_out;
+  p.rows = rows;
+  p.n_parts = n_parts;
+  const unsigned grid = unsigned((rows + libra::kMergeWarps - 1) / libra::kMergeWarps);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (head_dim == 128) libra::merge_parts_kernel<128><<<grid, libra::kMergeWarps * 32, 0, st>>>(p);
+  else libra::merge_parts_kernel<64><<<grid, libra::kMergeWarps * 32, 0, st>>>(p);
+  LIBRA_CUDA_TRY(nullptr, cudaGetLastError());
   return LIBRA_OK;
 }
 

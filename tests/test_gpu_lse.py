@@ -114,3 +114,105 @@ def test_two_parts_of_a_sequence_merge_to_the_whole(lib):
     assert gates.stated_violations(merged, ref) == 0
     assert gates.tight_violations(merged, ref) == 0, gates.tight_ratio(merged, ref)   # each part was rounded to bf16 once
     assert np.max(np.abs(merged_lse - ref_lse)) <= 2 * LSE_TOL
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("n_parts", [1, 2, 5, 33, 64])
+def test_device_merge_against_the_oracle_merge(lib, n_parts, d):
+    """libra_merge_parts on random (out, lse) pairs, some parts empty (lse = -inf, NaN in their out rows), one row
+    empty in every part, against the float64 merge of the same bf16 / float32 inputs."""
+    import torch
+    dev = torch.device("cuda:0")
+    rows = 37
+    rng = np.random.default_rng(1000 * n_parts + d)
+    outs = W.f32_to_bf16_bits(rng.standard_normal((n_parts, rows, d), dtype=np.float32))
+    lses = (rng.standard_normal((n_parts, rows)) * 6.0).astype(np.float32)
+    empty = rng.random((n_parts, rows)) < 0.2
+    empty[:, 5] = True
+    if n_parts > 1:
+        empty[0, 7] = False
+        empty[1:, 7] = True          # exactly one part holds tokens: its row comes back unchanged
+    lses[empty] = -np.inf
+    outs[empty] = 0x7FC0             # NaN where a part holds nothing
+    d_outs, d_lses = H.to_dev(outs, dev), torch.from_numpy(lses).to(dev)
+    got = torch.full((rows, d), H.CANARY, dtype=torch.int16, device=dev)
+    got_lse = torch.full((rows,), float("nan"), dtype=torch.float32, device=dev)
+    st = torch.cuda.current_stream().cuda_stream
+    lib.libra_merge_parts(0, d_outs.data_ptr(), d_lses.data_ptr(), n_parts, rows, d, got.data_ptr(), got_lse.data_ptr(), st)
+    torch.cuda.synchronize()
+    got, got_lse = H.bf16_dev_to_f32(got).astype(np.float64), got_lse.cpu().numpy().astype(np.float64)
+    vals = np.where(empty[:, :, None], 0.0, W.bf16_bits_to_f32(outs).astype(np.float64))
+    for r in range(rows):
+        want, want_lse = O.merge_partials(vals[:, r], lses[:, r].astype(np.float64))
+        if np.isneginf(want_lse):
+            assert np.isneginf(got_lse[r]) and np.all(got[r] == 0.0)
+            continue
+        assert np.all(np.abs(got[r] - want) <= 2.0 ** -8 * np.abs(want) + 3e-5), (r, np.max(np.abs(got[r] - want)))
+        assert abs(got_lse[r] - want_lse) <= 1e-5 * (1.0 + abs(want_lse)), (r, got_lse[r], want_lse)
+    if n_parts > 1:
+        assert np.array_equal(got[7], W.bf16_bits_to_f32(outs[0, 7]).astype(np.float64))
+    # the second output is optional
+    got2 = torch.full((rows, d), H.CANARY, dtype=torch.int16, device=dev)
+    lib.libra_merge_parts(0, d_outs.data_ptr(), d_lses.data_ptr(), n_parts, rows, d, got2.data_ptr(), 0, st)
+    torch.cuda.synchronize()
+    assert np.array_equal(H.bf16_dev_to_f32(got2).astype(np.float64), got)
+
+
+def test_merge_misuse_is_rejected(lib):
+    import torch
+    dev = torch.device("cuda:0")
+    a = torch.zeros((2, 4, 128), dtype=torch.int16, device=dev)
+    l = torch.zeros((2, 4), dtype=torch.float32, device=dev)
+    o = torch.zeros((4, 128), dtype=torch.int16, device=dev)
+    for args in ((0, a.data_ptr(), l.data_ptr(), 0, 4, 128, o.data_ptr(), 0, 0),
+                 (0, a.data_ptr(), l.data_ptr(), 65, 4, 128, o.data_ptr(), 0, 0),
+                 (0, a.data_ptr(), l.data_ptr(), 2, 4, 96, o.data_ptr(), 0, 0),
+                 (0, a.data_ptr() + 2, l.data_ptr(), 2, 4, 128, o.data_ptr(), 0, 0),
+                 (0, 0, l.data_ptr(), 2, 4, 128, o.data_ptr(), 0, 0),
+                 (0, a.data_ptr(), l.data_ptr(), 2, -1, 128, o.data_ptr(), 0, 0)):
+        with pytest.raises(lib.LibraError):
+            lib.libra_merge_parts(*args)
+    lib.libra_merge_parts(0, a.data_ptr(), l.data_ptr(), 2, 0, 128, o.data_ptr(), 0, 0)   # no rows: nothing to do
+
+
+@pytest.mark.parametrize("n_parts", [2, 3, 8])
+def test_token_sharded_sequences_merge_on_the_device(lib, n_parts):
+    """Every sequence cut at page boundaries into n_parts runs of pages (some empty), the parts decoded as rows of one
+    batch laid out part-major - which is the [n_parts][rows][d] layout the merge takes - and merged on the device:
+    the attention over the whole sequence."""
+    import torch
+    dev = torch.device("cuda:0")
+    lens = [700, 33, 2049, 4000, 1, 0]
+    B, Hq, Hkv, d = len(lens), 8, 2, 128
+    lens_a, bt, q, k, v = W.random_case(106, B, Hq, Hkv, d, lens)
+    ref, ref_lse = O.paged_decode_attention(q, k, v, bt, lens_a)
+    ld = bt.shape[1]
+    bt2 = np.full((n_parts * B, ld), -1, dtype=np.int32)
+    lens2 = np.zeros(n_parts * B, dtype=np.int32)
+    rng = np.random.default_rng(n_parts)
+    for b in range(B):
+        n_pages = (int(lens_a[b]) + 15) // 16
+        cuts = np.sort(rng.integers(0, n_pages + 1, size=n_parts - 1))
+        edges = [0] + [int(c) for c in cuts] + [n_pages]
+        for i in range(n_parts):
+            p0, p1 = edges[i], edges[i + 1]
+            bt2[i * B + b, :p1 - p0] = bt[b, p0:p1]
+            lens2[i * B + b] = max(0, min(int(lens_a[b]), p1 * 16) - p0 * 16)
+        assert lens2[b::B].sum() == lens_a[b]
+    q2 = np.tile(q, (n_parts, 1, 1))
+    out, lse = run_with_lse(lib, q2, k, v, bt2, lens2)
+    parts_out = H.to_dev(W.f32_to_bf16_bits(out.astype(np.float32)), dev)      # exact: out holds bf16 values
+    parts_lse = torch.from_numpy(lse).to(dev)
+    got = torch.full((B, Hq, d), H.CANARY, dtype=torch.int16, device=dev)
+    got_lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device=dev)
+    lib.libra_merge_parts(0, parts_out.data_ptr(), parts_lse.data_ptr(), n_parts, B * Hq, d, got.data_ptr(),
+                          got_lse.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    merged = H.bf16_dev_to_f32(got)
+    assert np.all(np.isfinite(merged))
+    assert gates.stated_violations(merged, ref) == 0
+    assert gates.tight_violations(merged, ref) == 0, gates.tight_ratio(merged, ref)
+    got_lse = got_lse.cpu().numpy()
+    inf = np.isneginf(ref_lse)
+    assert np.array_equal(np.isneginf(got_lse), inf)
+    assert np.max(np.abs(got_lse[~inf] - ref_lse[~inf])) <= 2 * LSE_TOL
