@@ -464,6 +464,61 @@ def nhd_layout_measure(rep: Replica, steps: int = 200):
             "same_bits_as_hnd": same}
 
 
+def head_shard_measure(rep: Replica, steps: int = 200):
+    """One rank's share of the step under the paper's tensor-parallel sharding of the cache (by attention head,
+    Section 5.3; larger degrees for the long-tail buckets, Section 2.3): KV heads [0, Hkv / tp) of every page and their
+    query heads, read in place from the full pool through the handle's strides.  No collective is part of the step."""
+    torch, w = rep.torch, rep.w
+    P, Hkv, d = w.page_size, w.num_kv_heads, w.head_dim
+    st = torch.cuda.current_stream().cuda_stream
+    res = []
+    base_ms = None
+    for tp in (1, 2, 4, 8):
+        if Hkv % tp:
+            continue
+        hk, hq = Hkv // tp, w.num_q_heads // tp
+        h = rep.binding.Handle(hq, hk, d, rep.layouts[0].pool_pages, w.batch, rep.ld, device=rep.dev.index or 0,
+                               kv_strides=(Hkv * P * d, P * d, d))
+        ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=rep.dev)
+        q = rep.q[:, :hq].contiguous()
+        out = torch.zeros_like(q)
+
+        slice_bytes = hk * P * d * 2   # rank r's heads start this many bytes into every page
+
+        def step(i, h=h, ws=ws, q=q, out=out, tp=tp, slice_bytes=slice_bytes):
+            # successive steps take successive ranks' head slices and pool copies, so that a step never finds the
+            # bytes of an earlier one in L2 (a rank's share of a small workload would fit there)
+            s = i % len(rep.layouts)
+            r = (i // len(rep.layouts)) % tp
+            k, v = rep.pools[(i // (len(rep.layouts) * tp)) % len(rep.pools)]
+            h.plan(rep.layouts[s].seq_lens, ws.data_ptr(), ws.numel(), st)
+            h.decode_attn(q.data_ptr(), k.data_ptr() + r * slice_bytes, v.data_ptr() + r * slice_bytes,
+                          rep.bts[s].data_ptr(), rep.lens_dev[s].data_ptr(), out.data_ptr(), st)
+
+        n = max(len(rep.layouts), steps // len(rep.layouts) * len(rep.layouts))
+        for i in range(10):
+            step(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n):
+            step(i)
+        e1.record()
+        torch.cuda.synchronize()
+        assert h.debug_error_word() == 0, "device error word set"
+        step(0)                      # rank 0's slice again: its rows of the full result
+        torch.cuda.synchronize()
+        same = (bool(torch.allclose(out.float(), rep.out[:, :hq].float(), atol=2e-3, rtol=2e-2))
+                if len(rep.layouts) == 1 else None)   # other chunking, hence other last bits, than the full step
+        h.close()
+        ms = e0.elapsed_time(e1) / n
+        base_ms = ms if tp == 1 else base_ms
+        res.append({"tp": tp, "kv_heads_per_rank": hk, "ms_per_step": ms,
+                    "rank_kv_gbs": rep.kv_bytes_per_step / tp / (ms * 1e-3) / 1e9,
+                    "speedup_vs_tp1": base_ms / ms, "matches_full_step": same})
+    return res
+
+
 def short_batch_measure(rep: Replica, steps: int = 100):
     """Batches of equally long, short sequences at a constant 262,144 cached tokens (1.07 GB of KV at 8 KV heads, d 128):
     the block shape the library picks by itself against the default large shape forced."""
@@ -891,6 +946,8 @@ def run_libra(args):
             line["fp8_cache"] = fp8_cache_measure(rep, steps=min(200, max(10, args.steps)))
         if "nhd_layout" in extras:
             line["nhd_layout"] = nhd_layout_measure(rep)
+        if "head_shard" in extras:
+            line["head_shard"] = head_shard_measure(rep)
         if "short_batch" in extras:
             line["short_batch"] = short_batch_measure(rep)
         if "ring_step" in extras:
@@ -934,6 +991,7 @@ def run_libra(args):
             others[name]["multi_token"] = [m for m in (multi_token_measure(r, t, 60) for t in (2, 3, 4)) if m]
             others[name]["fp8_cache"] = fp8_cache_measure(r, 60)
             others[name]["nhd_layout"] = nhd_layout_measure(r, 60)
+            others[name]["head_shard"] = head_shard_measure(r, 60)
             if name in ("longtail_mix_b256", "straggler_b8"):  # migrating the long sequences: gather to a dense buffer, scatter back
                 others[name]["kv_migration"] = kv_migration_measure(r)
             if name == "shift_b128":  # the re-planned-every-step workload: also with the device-side planner
@@ -966,7 +1024,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
-    ap.add_argument("--extras", default="ceilings,early_prefetch,multi_token,fp8_cache,nhd_layout,short_batch,kv_migration,ring_step",
+    ap.add_argument("--extras", default="ceilings,early_prefetch,multi_token,fp8_cache,nhd_layout,head_shard,short_batch,kv_migration,ring_step",
                     help="side measurements on the main workload at N=1 (comma list; empty = none)")
     ap.add_argument("--variant", default="", help="warps,stages of the decode block (default: the library's)")
     ap.add_argument("--ctas-per-sm", type=int, default=0, help="planner constant (0 = default)")

@@ -207,7 +207,10 @@ int libra_set_combine_mode(libra_handle_t handle, int32_t mode);
  * and 5 of the paper give the bucket properties it mirrors).  With W = n_sm * ctas_per_sm,
  * T = sum of lengths, cd = ceiling division, au(a,b) = cd(a,b)*b, p2 = next power of two:
  *   C       = max(min_chunk, au(cd(num_kv_heads * T, W * items_per_slot), chunk_align))
- *   s_b     = min(p2(cd(L_b, C)), max_splits)           bucket_b = log2 s_b
+ *   s_b     = p2(cd(L_b, C)); if C < 4096 and s_b > 1 and 128 * L_b < 181 * (s_b / 2) * C: s_b = s_b / 2
+ *             (short base chunks: the power of two nearer to L_b / C in ratio, 181 / 128 ~ sqrt 2; a work item
+ *             costs ~4 us whatever its length, so fewer and longer items win there)
+ *   s_b     = min(s_b, max_splits)                       bucket_b = log2 s_b
  *   chunk_b = au(cd(L_b, s_b), chunk_align)              n_b = cd(L_b, chunk_b)
  *   items   = (b, j, j*chunk_b, min(L_b, (j+1)*chunk_b)) sorted by (length desc, b asc, j asc)
  * params->n_sm must be > 0 here.  All outputs are caller-allocated host arrays: the per-sequence

@@ -15,6 +15,10 @@ share its KV range, so:
 
   * bucket k holds the sequences whose length lies in (C * 2^(k-1), C * 2^k]; bucket 0
     is (0, C]; the degree of bucket k is 2^k, capped at S_max;
+  * when C is short (C < 4096 tokens, where the fixed cost of a work item shows), the
+    bucket limits move up to the geometric means of those limits: a sequence of bucket
+    k >= 1 with L * 128 < 2^(k-1) * C * 181 (181 / 128 ~ sqrt 2) takes degree 2^(k-1),
+    the power of two nearer to L / C in ratio;
   * C, the base length, is recomputed for every batch from the total work so that the
     launch has about `items_per_slot` work items per resident block;
   * items are issued longest first (the classic greedy rule for the min-max objective).
@@ -37,6 +41,7 @@ class PlanParams:
     chunk_align: int = 256      # A: chunk lengths are multiples of this many tokens
     min_chunk: int = 512        # C_min
     max_splits: int = 64        # S_max
+    small_base: int = 4096      # base lengths below this take the nearer power of two (0 = never: the plain rule)
 
 
 def cd(a: int, b: int) -> int:
@@ -79,7 +84,10 @@ def plan(seq_lens, num_kv_heads: int, params: PlanParams = PlanParams()) -> Plan
         if L == 0:
             bucket.append(-1); nsplit.append(0); chunk.append(0)
             continue
-        s = min(p2(cd(L, C)), params.max_splits)
+        s = p2(cd(L, C))
+        if C < params.small_base and s > 1 and L * 128 < (s // 2) * C * 181:
+            s //= 2
+        s = min(s, params.max_splits)
         c = au(cd(L, s), A)
         bucket.append(s.bit_length() - 1)
         chunk.append(c)

@@ -152,6 +152,10 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
       long long deg = 1;
       const long long want = (len + base - 1) / base;
       while (deg < want) deg <<= 1;
+      if (base < plan_layout::kSmallBaseTokens && deg > 1 &&
+          len * plan_layout::kGeoMeanDen < (deg / 2) * base * plan_layout::kGeoMeanNum) {
+        deg >>= 1;   // short chunks: the nearer power of two
+      }
       if (deg > p.max_splits) deg = p.max_splits;
       const long long ch = ((len + deg - 1) / deg + A - 1) / A * A;
       n = int((len + ch - 1) / ch);

@@ -23,6 +23,14 @@ constexpr int kCountShift = 24;
 constexpr int kMaxBatch = 1 << kChunkShift;
 constexpr int kParamEntries = 768;  // 12 KB of the 32 KB kernel-parameter space
 constexpr int kParamFixEntries = 256;
+// Split degree of a sequence (both planners): the least power of two >= ceil(len / base) - except that, when the base
+// chunk is shorter than kSmallBaseTokens, the power of two below it is taken if len / base is nearer to it in ratio
+// (below the geometric mean of the two: len * 128 < (degree / 2) * base * 181, 181 / 128 ~ sqrt 2).  A unit costs
+// ~4 us of start-up and epilogue whatever its length; on chunks that short, fewer and longer units win (measured
+// 8 - 18 % on batches cut by KV head over 4 - 8 ranks, nothing lost elsewhere; with longer chunks the finer cut is
+// the better one).
+constexpr int kSmallBaseTokens = 4096;
+constexpr int kGeoMeanNum = 181, kGeoMeanDen = 128;
 // counts written by the device-side planner (int32 words at the start of the workspace's plan region)
 constexpr int kCountInts = 8;
 constexpr int kCntItems = 0;

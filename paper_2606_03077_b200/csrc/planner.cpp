@@ -1,5 +1,7 @@
 #include "planner.hpp"
 
+#include "plan_layout.hpp"
+
 #include <algorithm>
 
 namespace libra {
@@ -60,7 +62,12 @@ bool make_plan(const PlanParams& p, int32_t num_kv_heads, const int32_t* seq_len
       pl.empty.push_back(b);
       continue;
     }
-    const int64_t degree = std::min<int64_t>(next_pow2(ceil_div(len, base)), p.max_splits);
+    int64_t degree = next_pow2(ceil_div(len, base));
+    if (base < plan_layout::kSmallBaseTokens && degree > 1 &&
+        len * plan_layout::kGeoMeanDen < (degree / 2) * base * plan_layout::kGeoMeanNum) {
+      degree /= 2;   // short chunks: the nearer power of two, see plan_layout.hpp
+    }
+    degree = std::min<int64_t>(degree, p.max_splits);
     const int64_t chunk = round_up(ceil_div(len, degree), p.chunk_align);
     const int64_t pieces = ceil_div(len, chunk);
     pl.bucket[b] = log2_exact(degree);

@@ -93,16 +93,16 @@ def test_every_block_shape_agrees(lib):
 
 
 def test_plan_too_large_for_kernel_parameters(lib):
-    # 20 sequences x 64 chunks = 1280 work items: more than travel with a launch, so the plan is uploaded
-    lens = [2048] * 20
-    lens_a, bt, q, k, v = W.random_case(9, 20, 4, 1, 64, lens)
+    # 40 sequences x 32 chunks = 1280 work items: more than travel with a launch, so the plan is uploaded
+    lens = [2048] * 40
+    lens_a, bt, q, k, v = W.random_case(9, 40, 4, 1, 64, lens)
     ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
     prm = lib.PlanParams(148, 2, 4, 16, 16, 64)
     for variant in [(4, 3), (8, 3)]:
         got = H.run_host_case(lib, q, k, v, bt, lens_a, plan=prm, variant=variant)
         check(got, ref, f"uploaded plan, variant {variant}")
     import torch
-    h = lib.Handle(4, 1, 64, k.shape[0], 20, bt.shape[1], plan=prm)
+    h = lib.Handle(4, 1, 64, k.shape[0], 40, bt.shape[1], plan=prm)
     ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device="cuda:0")
     h.plan(lens_a, ws.data_ptr(), ws.numel(), torch.cuda.current_stream().cuda_stream)
     assert len(h.plan_export()["items"]) == 1280

@@ -25,12 +25,19 @@ def check_plan(lens, hkv, params):
         s = 1 << pl.bucket[b]
         assert 1 <= pl.num_splits[b] <= s <= params.max_splits
         assert pl.chunk_len[b] % A == 0 and pl.chunk_len[b] % 16 == 0
-        # bucket bins: (C 2^(k-1), C 2^k], except that the top bucket is open-ended
+        # bucket bins: (C 2^(k-1), C 2^k], except that the top bucket is open-ended; with a short base chunk the
+        # limits sit at the geometric means instead: [C 2^(k-1) * 181/128, C 2^k * 181/128)
         C = pl.chunk_target
-        if s < params.max_splits:
-            assert L <= C * s
-        if s > 1:
-            assert L > C * (s // 2)
+        if C >= params.small_base:
+            if s < params.max_splits:
+                assert L <= C * s
+            if s > 1:
+                assert L > C * (s // 2)
+        else:
+            if s < params.max_splits:
+                assert 128 * L < 181 * C * s
+            if s > 1:
+                assert 128 * L >= 181 * C * (s // 2)
         # chunks tile [0, L) exactly
         mine = sorted((it for it in pl.items if it[0] == b), key=lambda it: it[1])
         assert [it[1] for it in mine] == list(range(pl.num_splits[b]))
@@ -66,14 +73,19 @@ def test_exhaustive_small_vectors():
 def test_hand_worked_example():
     # n_sm 2, 1 block each, 2 items per slot, A = 16, C_min = 16, S_max = 4, one KV head
     # T = 100 + 16 + 40 = 156; C = max(16, au(cd(156, 4), 16)) = au(39, 16) = 48
-    # L=100: cd(100,48)=3 -> p2 = 4 splits; chunk = au(25,16) = 32; n = cd(100,32) = 4
+    # L=100: cd(100,48)=3 -> p2 = 4; C is short and 100 * 128 = 12800 < 2 * 48 * 181 = 17376, so 2 splits (100 / 48 = 2.08
+    #        is nearer to 2 than to 4); chunk = au(50,16) = 64; n = cd(100,64) = 2
     # L=16 : 1 split, chunk 16; L=40: 1 split, chunk au(40,16)=48, n = 1
     prm = P.PlanParams(n_sm=2, ctas_per_sm=1, items_per_slot=2, chunk_align=16, min_chunk=16, max_splits=4)
     pl = P.plan([100, 16, 40], 1, prm)
     assert pl.chunk_target == 48
-    assert pl.bucket == [2, 0, 0] and pl.num_splits == [4, 1, 1] and pl.chunk_len == [32, 16, 48]
-    assert pl.item_offset == [0, 4, 5]
-    assert pl.items == [(2, 0, 0, 40), (0, 0, 0, 32), (0, 1, 32, 64), (0, 2, 64, 96), (1, 0, 0, 16), (0, 3, 96, 100)]
+    assert pl.bucket == [1, 0, 0] and pl.num_splits == [2, 1, 1] and pl.chunk_len == [64, 16, 48]
+    assert pl.item_offset == [0, 2, 3]
+    assert pl.items == [(0, 0, 0, 64), (2, 0, 0, 40), (0, 1, 64, 100), (1, 0, 0, 16)]
+    # L=140 (T = 156 again): cd(140,48)=3 -> p2 = 4 and 140 * 128 = 17920 >= 17376: degree 4 stays; chunk au(35,16)=48, n = 3
+    pl = P.plan([140, 16, 0], 1, prm)
+    assert pl.chunk_target == 48 and pl.bucket == [2, 0, -1] and pl.num_splits == [3, 1, 0] and pl.chunk_len == [48, 16, 0]
+    pl = P.plan([100, 16, 40], 1, prm)
     assert pl.combine == [0] and pl.empty == []
 
 
@@ -85,18 +97,30 @@ def test_random_vectors_default_params():
         check_plan(list(lens), int(rng.choice([1, 2, 8])), P.PlanParams())
 
 
-@pytest.mark.parametrize("name,step,C,n_items", [
-    ("tiny", 0, 512, 4), ("lognormal_b64", 0, 768, 158), ("longtail_mix_b256", 0, 8192, 334),
-    ("straggler_b8", 0, 1792, 256), ("shift_b128", 0, 1536, 226), ("shift_b128", 1, 2560, 222),
-    ("shift_b128", 2, 5632, 239)])
-def test_workload_plans(name, step, C, n_items):
+@pytest.mark.parametrize("name,step,C,n_plain,n_items", [
+    ("tiny", 0, 512, 4, 4), ("lognormal_b64", 0, 768, 158, 122), ("longtail_mix_b256", 0, 8192, 334, 334),
+    ("straggler_b8", 0, 1792, 256, 128), ("shift_b128", 0, 1536, 226, 182), ("shift_b128", 1, 2560, 222, 186),
+    ("shift_b128", 2, 5632, 239, 239)])
+def test_workload_plans(name, step, C, n_plain, n_items):
+    """With 2 x 148 slots and 4 items per slot: the item counts of the plain rule (least power of two above L / C for
+    every base length) and of the rule as it stands (the nearer power of two where the base is short)."""
     lay, _ = W.make_layout(name, step)
-    pl = check_plan([int(x) for x in lay.seq_lens], lay.workload.num_kv_heads, P.PlanParams(ctas_per_sm=2, items_per_slot=4))
+    lens = [int(x) for x in lay.seq_lens]
+    plain = P.plan(lens, lay.workload.num_kv_heads, P.PlanParams(ctas_per_sm=2, items_per_slot=4, small_base=0))
+    assert plain.chunk_target == C and len(plain.items) == n_plain
+    for b, L in enumerate(lens):
+        s = 1 << plain.bucket[b]
+        assert C * (s // 2) < L and (L <= C * s or s == 64)
+    pl = check_plan(lens, lay.workload.num_kv_heads, P.PlanParams(ctas_per_sm=2, items_per_slot=4))
     assert pl.chunk_target == C and len(pl.items) == n_items
-    check_plan([int(x) for x in lay.seq_lens], lay.workload.num_kv_heads, P.PlanParams())
+    check_plan(lens, lay.workload.num_kv_heads, P.PlanParams())
 
 
-def test_straggler_is_split_32_ways():
+def test_straggler_split_follows_the_base_chunk():
     lay, _ = W.make_layout("straggler_b8")
+    # 8 x 148 slots: base 1792 tokens, 32768 / 1792 = 18.3 is nearer to 16 than to 32 and the base is short: 16 ways
     pl = P.plan(lay.seq_lens, 8, P.PlanParams(ctas_per_sm=2, items_per_slot=4))
-    assert set(pl.bucket) == {5} and set(pl.chunk_len) == {1024} and set(pl.num_splits) == {32}
+    assert pl.chunk_target == 1792 and set(pl.bucket) == {4} and set(pl.chunk_len) == {2048} and set(pl.num_splits) == {16}
+    # 148 slots: base 14336 tokens, long chunks keep the least power of two above 32768 / 14336 = 2.3: 4 ways
+    pl = P.plan(lay.seq_lens, 8, P.PlanParams())
+    assert pl.chunk_target == 14336 and set(pl.bucket) == {2} and set(pl.chunk_len) == {8192} and set(pl.num_splits) == {4}
