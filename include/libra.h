@@ -28,7 +28,7 @@
  *   - one handle serves one stream at a time (no internal locking).
  *
  * Data layout
- *   q, out        bf16 [batch, num_q_heads, head_dim], row-major, contiguous
+ *   q, out        bf16 [batch, num_q_heads, head_dim], row-major, contiguous; q 4-byte, out 8-byte aligned
  *   k_pages,
  *   v_pages       bf16, two separate pools indexed by the same page ids; element (page, head,
  *                 token, c) lives at  page*kv_stride_page + head*kv_stride_head +

@@ -79,6 +79,15 @@ namespace dev {
 
 constexpr uint32_t kWaitLimit = 1u << 20;  // tries of a bounded wait on a copy barrier (each suspends <= ~2 us)
 constexpr uint32_t kWaitHintNs = 2000;
+// The running maximum of a column is raised only when a tile's maximum exceeds it by more than this many powers of
+// two (and then every column of the warp is brought up to date): between raises the probabilities may reach
+// 2^kMaxSlack instead of 1, which bf16 / fp16 and the fp32 sums hold with the same relative precision, and the
+// accumulators are not rescaled tile after tile (a warp sees every NW-th tile of a unit, so its maximum keeps
+// growing for most of a short unit).
+#ifndef LIBRA_MAX_SLACK
+#define LIBRA_MAX_SLACK 8.0f
+#endif
+constexpr float kMaxSlack = LIBRA_MAX_SLACK;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
@@ -332,7 +341,7 @@ __device__ __forceinline__ void process_page(WarpAcc<D, NT>& st, const uint32_t 
     }
     m_new[nt][0] = fmaxf(st.m[nt][0], mx0);
     m_new[nt][1] = fmaxf(st.m[nt][1], mx1);
-    grew = grew || (m_new[nt][0] > st.m[nt][0]) || (m_new[nt][1] > st.m[nt][1]);
+    grew = grew || (mx0 > st.m[nt][0] + kMaxSlack) || (mx1 > st.m[nt][1] + kMaxSlack);
   }
   if (__any_sync(0xffffffffu, grew)) {
 #pragma unroll
@@ -490,7 +499,7 @@ __device__ __forceinline__ void process_page_fp8(WarpAcc<D, NT>& st, const uint3
     }
     m_new[nt][0] = fmaxf(st.m[nt][0], mx0);
     m_new[nt][1] = fmaxf(st.m[nt][1], mx1);
-    grew = grew || (m_new[nt][0] > st.m[nt][0]) || (m_new[nt][1] > st.m[nt][1]);
+    grew = grew || (mx0 > st.m[nt][0] + kMaxSlack) || (mx1 > st.m[nt][1] + kMaxSlack);
   }
   if (__any_sync(0xffffffffu, grew)) {
 #pragma unroll
@@ -562,47 +571,64 @@ __device__ __forceinline__ void stage_warp_result(WarpAcc<D, NT>& st, float* o_s
       const int h0 = nt * 8 + 2 * t;
       const int d0 = mt * 16 + (kPairDims ? 2 * g : g);
       constexpr int kStep = kPairDims ? 1 : 8;
-      o_sm[h0 * D + d0] = st.acc[nt][mt][0];
-      o_sm[(h0 + 1) * D + d0] = st.acc[nt][mt][1];
-      o_sm[h0 * D + d0 + kStep] = st.acc[nt][mt][2];
-      o_sm[(h0 + 1) * D + d0 + kStep] = st.acc[nt][mt][3];
+      // rows are D floats apart, a multiple of the 32 banks, so the four lanes that share g would hit one bank:
+      // the dim index is XORed with 8 t = stage_swizzle(row), which spreads a warp's store over all 32 banks and
+      // keeps every group of four dims together for the merge's 16-byte loads
+      const int sw = t << 3;
+      o_sm[h0 * D + (d0 ^ sw)] = st.acc[nt][mt][0];
+      o_sm[(h0 + 1) * D + (d0 ^ sw)] = st.acc[nt][mt][1];
+      o_sm[h0 * D + ((d0 + kStep) ^ sw)] = st.acc[nt][mt][2];
+      o_sm[(h0 + 1) * D + ((d0 + kStep) ^ sw)] = st.acc[nt][mt][3];
     }
   }
 }
 
+// Dim-index swizzle of a staged row (see stage_warp_result): rows 2t and 2t+1 of every column tile use 8 t.
+__device__ __forceinline__ int stage_swizzle(int row) { return ((row >> 1) & 3) << 3; }
+
 // Merge the NW staged warp results in warp order and write the unit's result: bf16 `out` if the
 // sequence is not split, else fp32 partial O (normalised) and its natural-log LSE, per column of the unit.
-// o_sm: [NW][o_stride floats], m_sm / l_sm: [NW][NT*8].
+// o_sm: [NW][o_stride floats], m_sm / l_sm: [NW][NT*8].  `out` is written 8 bytes at a time.
 template <int D, int NT, int NW>
 __device__ __forceinline__ void merge_and_write(const DecodeParams& p, const Unit& u, const float* o_sm, int o_stride,
                                                 const float* m_sm, const float* l_sm, int tid, int nthreads) {
-  for (int idx = tid; idx < p.cols * D; idx += nthreads) {
-    const int h = idx / D;
-    const int dim = idx - h * D;
+  constexpr int V4 = D / 4;   // a thread merges four consecutive dims of one column: one 16-byte load per warp result
+  for (int idx = tid; idx < p.cols * V4; idx += nthreads) {
+    const int h = idx / V4;
+    const int dim = (idx - h * V4) * 4;
     float m_all = kNegBig;
 #pragma unroll
     for (int w = 0; w < NW; ++w) m_all = fmaxf(m_all, m_sm[w * NT * 8 + h]);
-    float num = 0.f, den = 0.f;
+    float num[4] = {0.f, 0.f, 0.f, 0.f};
+    float den = 0.f;
+    const float* src = o_sm + h * D + (dim ^ stage_swizzle(h));
 #pragma unroll
     for (int w = 0; w < NW; ++w) {
       const float mw = m_sm[w * NT * 8 + h];
       const float f = ex2(mw - m_all);   // a warp that saw nothing has l = 0 and O = 0: its factor does not matter
-      num += f * o_sm[w * o_stride + h * D + dim];
+      const float4 o4 = *reinterpret_cast<const float4*>(src + w * o_stride);
+      num[0] += f * o4.x;
+      num[1] += f * o4.y;
+      num[2] += f * o4.z;
+      num[3] += f * o4.w;
       den += f * l_sm[w * NT * 8 + h];
     }
-    const float o = (den > 0.f) ? num / den * p.v_scale : 0.f;   // den = 0: a query token that sees nothing of this unit
+    float o[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) o[k] = (den > 0.f) ? num[k] / den * p.v_scale : 0.f;   // den = 0: a query token that sees nothing of this unit
     const int64_t head = col_row(p, u.kvh, h);
+    const float lse = (den > 0.f) ? (m_all + lg2(den)) * 0.6931471805599453f : -INFINITY;
     if (u.slot < 0) {
-      p.out[(int64_t(u.b) * p.num_q_heads + head) * D + dim] = __float2bfloat16_rn(o);
-      if (p.lse_out != nullptr && dim == 0) {
-        p.lse_out[int64_t(u.b) * p.num_q_heads + head] = (den > 0.f) ? (m_all + lg2(den)) * 0.6931471805599453f : -INFINITY;
-      }
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(o[0], o[1]), hi = __floats2bfloat162_rn(o[2], o[3]);
+      uint2 packed;
+      packed.x = *reinterpret_cast<const uint32_t*>(&lo);
+      packed.y = *reinterpret_cast<const uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>(p.out + (int64_t(u.b) * p.num_q_heads + head) * D + dim) = packed;
+      if (p.lse_out != nullptr && dim == 0) p.lse_out[int64_t(u.b) * p.num_q_heads + head] = lse;
     } else {
-      p.partial_o[(int64_t(u.slot) * p.num_q_heads + head) * D + dim] = o;
-      if (dim == 0) {
-        p.partial_lse[int64_t(u.slot) * p.num_q_heads + head] =
-            (den > 0.f) ? (m_all + lg2(den)) * 0.6931471805599453f : -INFINITY;
-      }
+      *reinterpret_cast<float4*>(p.partial_o + (int64_t(u.slot) * p.num_q_heads + head) * D + dim) =
+          make_float4(o[0], o[1], o[2], o[3]);
+      if (dim == 0) p.partial_lse[int64_t(u.slot) * p.num_q_heads + head] = lse;
     }
   }
 }

@@ -810,7 +810,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
   if ((k_new == nullptr) != (v_new == nullptr)) return LIBRA_INVALID_ARGUMENT;
   if (reinterpret_cast<uintptr_t>(k_new) % 16 || reinterpret_cast<uintptr_t>(v_new) % 16) return LIBRA_INVALID_ARGUMENT;
   if (reinterpret_cast<uintptr_t>(k_pages) % 16 || reinterpret_cast<uintptr_t>(v_pages) % 16 ||
-      reinterpret_cast<uintptr_t>(q) % 4 || reinterpret_cast<uintptr_t>(out) % 4) {
+      reinterpret_cast<uintptr_t>(q) % 4 || reinterpret_cast<uintptr_t>(out) % 8) {
     return LIBRA_INVALID_ARGUMENT;
   }
   if (q_len < 1 || q_len > h->max_q_len) return LIBRA_INVALID_ARGUMENT;
