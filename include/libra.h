@@ -136,8 +136,16 @@ int libra_destroy(libra_handle_t handle);
 
 /* Bytes of device workspace that libra_plan / libra_decode_attn need for any batch <= max_batch.
  * The workspace holds the device error word, arrival counters, the fp32 partial results of split
- * sequences and room for a plan too large for the kernel parameters.  It must be 256-byte aligned. */
+ * sequences and room for a plan too large for the kernel parameters.  It must be 256-byte aligned.
+ * The handle remembers the address of the workspace it cleared last and does not clear it again on later
+ * plans (the kernels leave the counters at zero).  If that memory was meanwhile used for anything else - freed and
+ * handed out again by an allocator at the same address, say - call libra_workspace_invalidate before the next plan.
+ * A handle is not thread-safe: one host thread at a time per handle; different handles are independent. */
 int libra_workspace_size(libra_handle_t handle, size_t* bytes);
+
+/* Forget which workspace was cleared last: the next libra_plan / libra_plan_device clears the control words and
+ * arrival counters of its workspace again, on its stream.  The current plan is dropped.  Errors: INVALID_ARGUMENT. */
+int libra_workspace_invalidate(libra_handle_t handle);
 
 /* The planner constants the handle uses, defaults resolved (n_sm = the device's SM count). */
 int libra_get_plan_params(libra_handle_t handle, libra_plan_params_t* out);

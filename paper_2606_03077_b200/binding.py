@@ -74,6 +74,7 @@ SIGNATURES = {
     "libra_set_combine_mode": (C.c_int, [_vp, C.c_int32]),
     "libra_plan_host": (C.c_int, [C.POINTER(PlanParams), C.c_int32, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p,
                                   _i32p, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p]),
+    "libra_workspace_invalidate": (C.c_int, [_vp]),
     "libra_plan": (C.c_int, [_vp, _i32p, C.c_int32, _vp, C.c_size_t, _vp]),
     "libra_plan_device": (C.c_int, [_vp, _vp, C.c_int32, _vp, C.c_size_t, _vp]),
     "libra_plan_export": (C.c_int, [_vp, C.POINTER(PlanView)]),
@@ -347,6 +348,9 @@ class Handle:
         _check(lib.libra_decode_attn_static(self._h, lens.ctypes.data_as(_i32p), int(lens.shape[0]), q_ptr, k_ptr,
                                             v_ptr, block_table_ptr, seq_lens_ptr, out_ptr, stream),
                "libra_decode_attn_static")
+
+    def workspace_invalidate(self) -> None:
+        _check(lib.libra_workspace_invalidate(self._h), "libra_workspace_invalidate")
 
     def host_staging_size(self, batch: int) -> int:
         n = C.c_size_t(0)

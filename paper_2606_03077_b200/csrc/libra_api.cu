@@ -536,6 +536,13 @@ int libra_workspace_size(libra_handle_t h, size_t* bytes) {
   return LIBRA_OK;
 }
 
+int libra_workspace_invalidate(libra_handle_t h) {
+  if (!h) return LIBRA_INVALID_ARGUMENT;
+  h->clean_workspace = nullptr;
+  h->planned = false;
+  return LIBRA_OK;
+}
+
 int libra_get_plan_params(libra_handle_t h, libra_plan_params_t* out) {
   if (!h || !out) return LIBRA_INVALID_ARGUMENT;
   out->n_sm = h->params.n_sm;

@@ -347,6 +347,28 @@ def test_host_buffer_entry_point(lib):
     h.close()
 
 
+def test_workspace_reused_by_someone_else_needs_invalidate(lib):
+    """A workspace that was overwritten between two plans (an allocator handed the address to someone else): after
+    libra_workspace_invalidate the next plan clears it again and the split sequences merge correctly."""
+    import torch
+    dev = torch.device("cuda:0")
+    lens = [9000, 40, 5000]
+    lens_a, bt, q, k, v = W.random_case(56, 3, 8, 2, 128, lens)
+    ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
+    r = H.Runner(lib, 8, 2, 128, k.shape[0], 3, bt.shape[1], plan=lib.PlanParams(8, 1, 2, 256, 256, 64))
+    dq, dk, dv, dbt = (H.to_dev(x, dev) for x in (q, k, v, bt))
+    first = H.bf16_dev_to_f32(r.run(dq, dk, dv, dbt, lens_a))
+    check(first, ref, "first run")
+    r.ws.fill_(0x5A)                      # arrival counters and control words now hold garbage
+    torch.cuda.synchronize()
+    with pytest.raises(lib.LibraError):   # the plan is dropped with the invalidation
+        r.h.workspace_invalidate()
+        r.h.decode_attn(dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dbt.data_ptr(), dbt.data_ptr(), dq.data_ptr(), 0)
+    again = H.bf16_dev_to_f32(r.run(dq, dk, dv, dbt, lens_a))   # plans (clearing the workspace) and decodes
+    assert np.array_equal(again, first)
+    r.h.close()
+
+
 def test_host_io_entry_point_with_resident_cache(lib):
     """q, block table and lengths from pinned host memory, the cache on the device: the bits of the all-device call."""
     import torch
