@@ -160,3 +160,41 @@ def test_offsets_beyond_32_bits_8bit_cache(lib):
         h.close()
     assert np.array_equal(outs[0], outs[1])
     assert gates.stated_violations(outs[1], ref) == 0 and gates.tight_violations(outs[1], ref) == 0
+
+
+def test_largest_batch(lib):
+    """The largest batch a handle takes (2^18 sequences, the width of the plan's sequence field): short ragged
+    sequences incl. empty ones, a plan far too large for the kernel parameters, half a million thread blocks;
+    sampled rows against the oracle, every row written, empty rows zero."""
+    import torch
+    dev = torch.device("cuda:0")
+    B, Hq, Hkv, d = 1 << 18, 4, 2, 64
+    rng = np.random.default_rng(77)
+    lens = rng.integers(0, 33, size=B).astype(np.int32)          # 0 .. 32 tokens: one or two pages
+    lens[:5] = [0, 1, 16, 17, 32]
+    n_pages = (lens.astype(np.int64) + 15) // 16
+    first = np.concatenate([[0], np.cumsum(n_pages)[:-1]])
+    total_pages = int(n_pages.sum())
+    perm = rng.permutation(total_pages).astype(np.int32)
+    bt = np.full((B, 2), -1, dtype=np.int32)
+    for j in range(2):
+        has = n_pages > j
+        bt[has, j] = perm[first[has] + j]
+    gen = torch.Generator(device=dev).manual_seed(5)
+    k = torch.randn((total_pages, Hkv, 16, d), device=dev, generator=gen).to(torch.bfloat16)
+    v = torch.randn((total_pages, Hkv, 16, d), device=dev, generator=gen).to(torch.bfloat16)
+    q = torch.randn((B, Hq, d), device=dev, generator=gen).to(torch.bfloat16)
+    with pytest.raises(lib.LibraError):
+        lib.Handle(Hq, Hkv, d, total_pages, B + 1, 2)             # one more than the plan format holds
+    r = H.Runner(lib, Hq, Hkv, d, total_pages, B, 2)
+    out = H.bf16_dev_to_f32(r.run(q, k, v, H.to_dev(bt, dev), lens))
+    assert np.all(np.isfinite(out))                               # every row written (the canary is a NaN)
+    assert np.all(out[lens == 0] == 0.0)
+    assert len(r.h.plan_export()["items"]) == int((lens > 0).sum())
+    rows = [0, 1, 2, 3, 4, B - 1] + [int(x) for x in rng.choice(B, size=300, replace=False)]
+    kh, vh, bth, lh = H.gather_for_oracle(k, v, bt, lens, rows)
+    qh = q.view(torch.int16)[torch.tensor(rows, device=dev)].cpu().numpy().view(np.uint16)
+    ref, _ = O.paged_decode_attention(qh, kh, vh, bth, lh)
+    got = out[rows]
+    assert gates.stated_violations(got, ref) == 0 and gates.tight_violations(got, ref) == 0
+    r.h.close()
