@@ -89,7 +89,7 @@ typedef struct {
   int32_t head_dim;            /* 64 or 128                                                      */
   int32_t page_size;           /* 16, 32 or 64 tokens per page                                   */
   int64_t num_pages;           /* pages in each pool                                             */
-  int32_t max_batch;           /* upper bound of `batch` in libra_plan                           */
+  int32_t max_batch;           /* upper bound of `batch` in libra_plan; at most 262144 (2^18)    */
   int32_t block_table_ld;      /* row pitch of block_table in entries                            */
   int64_t kv_stride_page;      /* in elements; all three 0 = HND                                 */
   int64_t kv_stride_head;
