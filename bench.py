@@ -519,6 +519,46 @@ def head_shard_measure(rep: Replica, steps: int = 200):
     return res
 
 
+def wide_group_measure(rep: Replica, steps: int = 200):
+    """The same cache, block tables and lengths read with 8 and 16 query heads per KV head (one and two column tiles
+    of the score matrix; the paper's model family includes such ratios): q and out grow, the KV bytes do not."""
+    torch, w = rep.torch, rep.w
+    st = torch.cuda.current_stream().cuda_stream
+    res = []
+    for group in (8, 16):
+        hq = w.num_kv_heads * group
+        h = rep.binding.Handle(hq, w.num_kv_heads, w.head_dim, rep.layouts[0].pool_pages, w.batch, rep.ld,
+                               device=rep.dev.index or 0)
+        ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=rep.dev)
+        gen = torch.Generator(device=rep.dev).manual_seed(9)
+        q = torch.randn((w.batch, hq, w.head_dim), generator=gen, device=rep.dev).to(torch.bfloat16)
+        out = torch.zeros_like(q)
+
+        def step(i, h=h, ws=ws, q=q, out=out):
+            s = i % len(rep.layouts)
+            k, v = rep.pools[i % len(rep.pools)]
+            h.plan(rep.layouts[s].seq_lens, ws.data_ptr(), ws.numel(), st)
+            h.decode_attn(q.data_ptr(), k.data_ptr(), v.data_ptr(), rep.bts[s].data_ptr(), rep.lens_dev[s].data_ptr(),
+                          out.data_ptr(), st)
+
+        n = max(len(rep.layouts), steps // len(rep.layouts) * len(rep.layouts))
+        for i in range(10):
+            step(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n):
+            step(i)
+        e1.record()
+        torch.cuda.synchronize()
+        assert h.debug_error_word() == 0, "device error word set"
+        h.close()
+        ms = e0.elapsed_time(e1) / n
+        res.append({"q_heads_per_kv_head": group, "ms_per_step": ms, "kv_gbs": rep.kv_bytes_per_step / (ms * 1e-3) / 1e9,
+                    "steps": n})
+    return res
+
+
 def short_batch_measure(rep: Replica, steps: int = 100):
     """Batches of equally long, short sequences at a constant 262,144 cached tokens (1.07 GB of KV at 8 KV heads, d 128):
     the block shape the library picks by itself against the default large shape forced."""
@@ -948,6 +988,8 @@ def run_libra(args):
             line["nhd_layout"] = nhd_layout_measure(rep)
         if "head_shard" in extras:
             line["head_shard"] = head_shard_measure(rep)
+        if "wide_group" in extras:
+            line["wide_group"] = wide_group_measure(rep)
         if "short_batch" in extras:
             line["short_batch"] = short_batch_measure(rep)
         if "ring_step" in extras:
@@ -1024,7 +1066,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
-    ap.add_argument("--extras", default="ceilings,early_prefetch,multi_token,fp8_cache,nhd_layout,head_shard,short_batch,kv_migration,ring_step",
+    ap.add_argument("--extras", default="ceilings,early_prefetch,multi_token,fp8_cache,nhd_layout,head_shard,wide_group,short_batch,kv_migration,ring_step",
                     help="side measurements on the main workload at N=1 (comma list; empty = none)")
     ap.add_argument("--variant", default="", help="warps,stages of the decode block (default: the library's)")
     ap.add_argument("--ctas-per-sm", type=int, default=0, help="planner constant (0 = default)")
