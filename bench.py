@@ -45,7 +45,7 @@ FALLBACK_HBM_GBS = 6650.0
 L2_BYTES_ASSUMED = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode launch, from the ncu captures summarised under
 # profiles/ (lognormal_b64: 370.63 MB read + 3.4 MB written)
-NCU_DECODE_TRAFFIC_BYTES = {"lognormal_b64": 374.2e6, "straggler_b8": 1078.1e6}
+NCU_DECODE_TRAFFIC_BYTES = {"lognormal_b64": 374.9e6, "straggler_b8": 1078.1e6}
 
 
 # ----------------------------------------------------------------------------- clocks

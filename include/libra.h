@@ -185,6 +185,16 @@ int libra_set_variant(libra_handle_t handle, int32_t warps, int32_t stages);
  * and block start-up overlap the predecessor's tail.  on = 0 makes every launch an ordinary one. */
 int libra_set_dependent_launch(libra_handle_t handle, int32_t on);
 
+/* L2 warm-up at the start of a step, on by default (and only with dependent launches on).  The blocks of a step's
+ * first wave become resident while the kernel before them in the stream drains, when DRAM is all but idle.  Before they
+ * wait for that kernel they look up the page ids of their first tiles and ask for those tiles to be brought into L2
+ * (a prefetch without destination); after the wait they read ids and tiles again, for real, so the results do not
+ * depend on it: an id that the preceding kernel had not yet written only warms the wrong lines, and a line written
+ * after it was warmed is updated in L2, where the copies read.  It needs no promise from the caller (unlike
+ * libra_set_early_prefetch) but it does read block_table - as a hint - while the preceding kernel may still be writing
+ * it, which a memory checker reports; on = 0 switches it off.  Worth 2 % on a 55 us step, nothing on long ones. */
+int libra_set_cache_warmup(libra_handle_t handle, int32_t on);
+
 /* Optional second output.  With a non-NULL lse_dev every later decode call (libra_decode_attn, _append, _multi,
  * _static) also writes, for every row of q, the natural logarithm of the sum of its exponentiated scores,
  * lse[b][row] = ln sum_t exp(s_t) with s_t = (q . k_t) * sm_scale, as float32 [batch, rows] (rows = q_len *

@@ -62,6 +62,7 @@ SIGNATURES = {
     "libra_set_dependent_launch": (C.c_int, [_vp, C.c_int32]),
     "libra_set_max_query_tokens": (C.c_int, [_vp, C.c_int32]),
     "libra_set_early_prefetch": (C.c_int, [_vp, C.c_int32]),
+    "libra_set_cache_warmup": (C.c_int, [_vp, C.c_int32]),
     "libra_set_lse_output": (C.c_int, [_vp, _vp]),
     "libra_set_kv_dtype": (C.c_int, [_vp, C.c_int32, C.c_float, C.c_float]),
     "libra_decode_attn_multi": (C.c_int, [_vp, _vp, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -317,6 +318,9 @@ class Handle:
 
     def set_lse_output(self, lse_ptr: int) -> None:
         _check(lib.libra_set_lse_output(self._h, lse_ptr or None), "libra_set_lse_output")
+
+    def set_cache_warmup(self, on: bool) -> None:
+        _check(lib.libra_set_cache_warmup(self._h, 1 if on else 0), "libra_set_cache_warmup")
 
     def set_early_prefetch(self, on: bool) -> None:
         _check(lib.libra_set_early_prefetch(self._h, 1 if on else 0), "libra_set_early_prefetch")

@@ -65,6 +65,7 @@ struct DecodeParams {
   int32_t num_empty;      // empty sequences whose output row this launch zeroes
   int32_t fused_combine;  // 1: the last block of a split sequence merges its partials (step C) itself
   int32_t early_prefetch; // 1: block-table walk and first copies of old tokens start before the grid dependency wait
+  int32_t l2_warmup;      // 1: first-wave blocks ask for their first tiles to be brought into L2 before that wait
   // KV append fused into the step (null k_new = off): the K and V rows of the newest q_len tokens, [B, q_len, Hkv, D]
   // in the cache's element type, are written into their slots of the sequence's last page(s), in the pools and in the
   // staged tiles
@@ -136,6 +137,27 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       :
       : "r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy)
       : "memory");
+}
+
+// Ask for one box of a tiled tensor to be brought into L2 (no destination, nothing to wait for).
+__device__ __forceinline__ void tma_prefetch_l2_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3, uint64_t policy) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile.L2::cache_hint [%0, {%1, %2, %3, %4}], %5;"
+               :
+               : "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy)
+               : "memory");
+}
+
+// A 32-bit load that goes to L2, not through this SM's L1 (for memory another kernel may still be writing).
+__device__ __forceinline__ int32_t ld_cg_s32(const int32_t* ptr) {
+  int32_t v;
+  asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+  return v;
+}
+
+__device__ __forceinline__ uint32_t sm_count() {
+  uint32_t n;
+  asm volatile("mov.u32 %0, %%nsmid;" : "=r"(n));
+  return n;
 }
 
 // Pull a tensor map (a kernel parameter) into the descriptor cache ahead of its first use.
@@ -736,7 +758,34 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   // Only a plan that travels in the kernel parameters allows it (a plan in device memory may itself have been
   // written by the preceding kernel).
   const bool early = p.early_prefetch != 0 && p.entries == nullptr && p.dev_counts == nullptr;
-  if (!early) grid_dependency_wait();
+  if (!early) {
+    // Without that promise nothing this block needs may be READ for use before the wait - but it may be asked for.
+    // A block of the first wave (resident while the kernel before it drains, DRAM all but idle) looks up the pages
+    // of its first tiles and has them brought into L2; ids and data are fetched again, for real, after the wait.  A
+    // stale id only warms the wrong lines, a line written later is updated in L2, which is where the copies read.
+    if (p.l2_warmup != 0 && p.entries == nullptr && p.dev_counts == nullptr && blockIdx.x < sm_count() &&
+        int(blockIdx.x) < p.num_units) {
+      const int w_item = blockIdx.x / p.num_kv_heads;
+      const int w_kvh = blockIdx.x - w_item * p.num_kv_heads;
+      const Unit w = decode_unit<NW>(pp.e[w_item], w_kvh, warp);
+      if (lane < STAGES && lane < w.n_it) {   // more tiles per warp helped long units and cost the short ones more
+        const int tile = w.first_page + warp + lane * NW;
+        const int32_t pid = ld_cg_s32(p.block_table + int64_t(w.b) * p.block_table_ld + (tile >> p.tile_shift));
+        if (pid >= 0 && int64_t(pid) < p.num_pages) {
+          const int tok = (tile & ((1 << p.tile_shift) - 1)) << 4;
+          const int c1 = (p.pos_head == 1) ? w_kvh : ((p.pos_page == 1) ? pid : tok);
+          const int c2 = (p.pos_head == 2) ? w_kvh : ((p.pos_page == 2) ? pid : tok);
+          const int c3 = (p.pos_head == 3) ? w_kvh : ((p.pos_page == 3) ? pid : tok);
+#pragma unroll
+          for (int h = 0; h < NH; ++h) {
+            tma_prefetch_l2_4d(&map_k, h * 64, c1, c2, c3, kv_policy);
+            tma_prefetch_l2_4d(&map_v, h * 64, c1, c2, c3, kv_policy);
+          }
+        }
+      }
+    }
+    grid_dependency_wait();
+  }
 
   // the plan lives in the kernel parameters unless it was too large for them (plain loads: the
   // pointer may address parameter space)

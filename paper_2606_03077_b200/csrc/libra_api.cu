@@ -178,6 +178,7 @@ struct libra_handle_s {
   bool pdl = true;          // programmatic dependent launches (decode after its predecessor, combine after decode)
   float* lse_out = nullptr;     // optional second output of the step (libra_set_lse_output)
   bool early_prefetch = false;  // the caller's promise about the preceding kernel (libra_set_early_prefetch)
+  bool l2_warmup = true;        // libra_set_cache_warmup
 
   // pinned staging for uploads of plans too large for the kernel parameters
   int32_t* staging[2] = {nullptr, nullptr};
@@ -781,6 +782,12 @@ int libra_set_early_prefetch(libra_handle_t h, int32_t on) {
   return LIBRA_OK;
 }
 
+int libra_set_cache_warmup(libra_handle_t h, int32_t on) {
+  if (!h || (on != 0 && on != 1)) return LIBRA_INVALID_ARGUMENT;
+  h->l2_warmup = (on == 1);
+  return LIBRA_OK;
+}
+
 int libra_set_variant(libra_handle_t h, int32_t warps, int32_t stages) {
   if (!h) return LIBRA_INVALID_ARGUMENT;
   if (h->fp8) {
@@ -907,6 +914,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     p.num_empty = n_empty;
     p.fused_combine = fused ? 1 : 0;
     p.early_prefetch = (h->early_prefetch && h->pdl) ? 1 : 0;
+    p.l2_warmup = (h->l2_warmup && h->pdl) ? 1 : 0;
     p.k_new = k_new;
     p.v_new = v_new;
     p.k_pool = const_cast<void*>(k_pages);

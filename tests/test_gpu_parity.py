@@ -402,6 +402,55 @@ def test_host_io_entry_point_with_resident_cache(lib):
     h.close()
 
 
+def test_cache_warmup_never_changes_a_result(lib):
+    """The L2 warm-up reads the block table, as a hint, while the kernel before the step may still be writing it.
+    Steps queued back to back, each behind kernels that rewrite the WHOLE block table (a new page placement every
+    step), the lengths' device copy, q and the pools' contents: the same bits with the warm-up on and off, and the
+    oracle's values for the last step."""
+    import torch
+    dev = torch.device("cuda:0")
+    lens = [2500, 300, 17, 4100, 1, 16, 33, 900]
+    B, Hq, Hkv, d = len(lens), 32, 8, 128
+    lens_a, bt, q, k, v = W.random_case(81, B, Hq, Hkv, d, lens, spare_pages=40)
+    rng = np.random.default_rng(82)
+    steps = 5
+    n_pages = k.shape[0]
+    perms = [rng.permutation(n_pages) for _ in range(steps)]            # step i: page p of the case lives at perms[i][p]
+    bts = [np.where(bt >= 0, perms[i][np.maximum(bt, 0)], -1).astype(np.int32) for i in range(steps)]
+    results = {}
+    for warm in (True, False):
+        r = H.Runner(lib, Hq, Hkv, d, n_pages, B, bt.shape[1])
+        r.h.set_cache_warmup(warm)
+        k0, v0 = H.to_dev(k, dev), H.to_dev(v, dev)
+        kd, vd = torch.zeros_like(k0), torch.zeros_like(v0)
+        btd = torch.full(bt.shape, -1, dtype=torch.int32, device=dev)
+        dl = torch.zeros(B, dtype=torch.int32, device=dev)
+        qd = torch.zeros((B, Hq, d), dtype=torch.int16, device=dev)
+        src_bt = [H.to_dev(x, dev) for x in bts]
+        src_perm = [torch.from_numpy(x).to(dev) for x in perms]
+        src_l, src_q = torch.from_numpy(lens_a.copy()).to(dev), H.to_dev(q, dev)
+        outs = [torch.full((B, Hq, d), H.CANARY, dtype=torch.int16, device=dev) for _ in range(steps)]
+        st = torch.cuda.current_stream().cuda_stream
+        torch.cuda.synchronize()
+        for i in range(steps):      # nothing synchronises inside this loop: the step overlaps the tail of the writers
+            kd.index_copy_(0, src_perm[i], k0)
+            vd.index_copy_(0, src_perm[i], v0)
+            qd.copy_(src_q)
+            torch.add(src_l, 0, out=dl)
+            torch.add(src_bt[i], 0, out=btd)    # an elementwise KERNEL right before the step writes the block table
+            r.h.plan(lens_a, r.ws.data_ptr(), r.ws.numel(), st)
+            r.h.decode_attn(qd.data_ptr(), kd.data_ptr(), vd.data_ptr(), btd.data_ptr(), dl.data_ptr(), outs[i].data_ptr(), st)
+        torch.cuda.synchronize()
+        assert r.h.debug_error_word() == 0
+        results[warm] = [H.bf16_dev_to_f32(o) for o in outs]
+        r.h.close()
+    ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
+    for i in range(steps):
+        assert np.array_equal(results[True][i], results[False][i]), i
+        assert np.array_equal(results[True][i], results[True][0]), i      # the placement never changes a result
+    check(results[True][-1], ref, "behind writers of the block table")
+
+
 def test_early_prefetch_is_bit_identical_behind_a_cache_write_kernel(lib):
     """Steps issued back to back, each preceded by kernels that write q and the newest token's K/V rows (what the
     promise of libra_set_early_prefetch allows the preceding kernel to do): same bits as the default."""
