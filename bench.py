@@ -3,18 +3,25 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl libra|reference]
 
-One "step" is one pass of the whole path over one batch: libra_plan (host planner + plan upload)
-followed by libra_decode_attn (decode kernel + combine kernel).  The headline workload is
-`lognormal_b64` (batch 64, 32 query / 8 KV heads, head_dim 128, lognormal lengths); the other
-workloads are reported under "workloads" on the same line.
+One "step" is one pass of the whole path over one batch: libra_plan (host planner) followed by
+libra_decode_attn (decode kernel with the combine step inside it).  The headline workload is
+`longtail_mix_b256`, the largest of the configurations and a long-tailed one (batch 256, 32 query / 8 KV
+heads, head_dim 128, 90 % of the lengths in [512, 4096] and 10 % in [16384, 32768]); the other three
+large workloads are measured in the same run and summarised in `roofline.per_workload` (and in full
+under "workloads").
 
 metric  = achieved KV bandwidth: algorithmic bytes (K and V of every cached token, bf16, exact
           token count) / time of one step; "steps_per_s" is reported beside it.
-value   = inputs resident in HBM; timed with CUDA events around exactly K steps.
+value   = inputs resident in HBM.  A region of exactly K back-to-back steps is timed with CUDA events
+          (barrier + synchronize on both sides, max over ranks); the region is repeated REGIONS times and
+          ms_per_step is the median region / K (best and spread are reported too).
+roofline= frac is the decode kernel's own duration (a CUDA event pair around every launch) against the
+          measured copy rate; frac_chained is the same bytes over the step spacing of the chained region,
+          where consecutive launches overlap (programmatic dependent launch).
 e2e     = the same step through libra_decode_attn_host: q, both KV pools, block table and lengths
           start in pinned host memory and the output ends there, copies inside the timed region.
-L2      = steps rotate over several copies of the KV pools so that a pool is long evicted from
-          the 126 MB L2 when it is read again (see config.l2).
+L2      = every workload moves at least 8 x the 126 MB L2 per step, or rotates over several copies of
+          its KV pools (see config.l2).
 
 With N > 1 (torchrun) every rank runs its own replica of the workload on its own GPU: the path
 shards by sequence and has no collective; value is the sum over ranks / the slowest rank's time.
@@ -39,13 +46,16 @@ if ROOT not in sys.path:
 
 METRIC = "paged decode-attn achieved HBM GB/s (KV bytes / step time)"
 UNIT = "GB/s"
-MAIN_WORKLOAD = "lognormal_b64"
+MAIN_WORKLOAD = "longtail_mix_b256"
+REGIONS = 25   # timed regions of K steps each; the figures are medians over them
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES_ASSUMED = 126 * 1024 * 1024
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode launch, from the ncu captures summarised under
-# profiles/ (lognormal_b64: 370.63 MB read + 3.4 MB written)
-NCU_DECODE_TRAFFIC_BYTES = {"lognormal_b64": 374.9e6, "straggler_b8": 1078.1e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode launch divided by its algorithmic bytes, from the ncu
+# captures summarised under profiles/ (a constant of those captures, not something this run measures):
+# lognormal_b64 374.9 MB / 368.1 MB, straggler_b8 1078.1 MB / 1073.7 MB.  The large mix is too big to capture under
+# the profiler; its traffic is scaled from these (traffic grows with the pages read).
+NCU_TRAFFIC_OVER_ALGORITHMIC = {"lognormal_b64": 374.9e6 / 368.128e6, "straggler_b8": 1078.1e6 / 1073.741824e6}
 
 
 # ----------------------------------------------------------------------------- clocks
@@ -153,9 +163,7 @@ class Replica:
         self.q = q
         pool_bytes = 2 * k.numel() * 2
         if copies is None:  # enough copies that 4 x L2 of other data passes before a pool is read again
-            copies = 1 if self.w.steps > 1 else max(1, min(8, -(-4 * L2_BYTES_ASSUMED // max(1, lay0.kv_bytes)) + 1))
-            if lay0.kv_bytes >= 6 * L2_BYTES_ASSUMED:
-                copies = 1
+            copies = pool_copies_for(self.w.steps, lay0.kv_bytes)
         self.pools = [(k, v)] + [(k.clone(), v.clone()) for _ in range(copies - 1)]
         self.pool_bytes = pool_bytes
         self.bts, self.lens_dev = [], []
@@ -193,9 +201,59 @@ class Replica:
         self.h.decode_attn(self.q.data_ptr(), k.data_ptr(), v.data_ptr(), self.bts[s].data_ptr(),
                            self.lens_dev[s].data_ptr(), self.out.data_ptr(), stream)
 
-    def timed_device_plan(self, steps: int, warmup: int, graph: bool):
-        """ms per step with the device-side planner, issued eagerly or replayed from one CUDA graph that
-        holds one step per layout x pool copy."""
+    def bytes_of_steps(self, i0: int, n: int) -> int:
+        """KV bytes of steps i0 .. i0 + n - 1 (a workload with several layouts cycles through them, and their
+        sizes differ: the bytes of a region are those of the layouts it actually ran)."""
+        L = len(self.layouts)
+        full, rem = divmod(n, L)
+        b = full * sum(l.kv_bytes for l in self.layouts)
+        for j in range(rem):
+            b += self.layouts[(i0 + j) % L].kv_bytes
+        return int(b)
+
+    def step_decode_only(self, stream: int) -> None:
+        """decode + combine on the plan already in the workspace (one layout only)."""
+        k, v = self.pools[self.i % len(self.pools)]
+        self.i += 1
+        self.h.decode_attn(self.q.data_ptr(), k.data_ptr(), v.data_ptr(), self.bts[0].data_ptr(),
+                           self.lens_dev[0].data_ptr(), self.out.data_ptr(), stream)
+
+    def timed_regions(self, fn, steps: int, warmup: int, regions: int, barrier=None, world: int = 1, agg_dev=None,
+                      stream=None):
+        """`regions` timed regions of exactly `steps` back-to-back calls of fn(stream) each, CUDA events on the
+        launching stream, barrier + synchronize on both sides of every region; with several ranks a region's time
+        is the slowest rank's and its bytes the sum.  Returns (list of (ms, kv bytes), launches of this rank)."""
+        torch = self.torch
+        ts = stream if stream is not None else torch.cuda.current_stream()
+        st = ts.cuda_stream
+        with torch.cuda.stream(ts):
+            for _ in range(warmup):
+                fn(st)
+        torch.cuda.synchronize()
+        out = []
+        n0 = self.h.launch_count()
+        for _ in range(regions):
+            if barrier:
+                barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            i0 = self.i
+            torch.cuda.synchronize()
+            with torch.cuda.stream(ts):
+                e0.record()
+                for _ in range(steps):
+                    fn(st)
+                e1.record()
+            torch.cuda.synchronize()
+            if barrier:
+                barrier()
+            ms, b = aggregate_over_ranks(e0.elapsed_time(e1), float(self.bytes_of_steps(i0, steps)), world, agg_dev)
+            out.append((ms, b))
+        assert self.h.debug_error_word() == 0, "device error word set"
+        return out, self.h.launch_count() - n0
+
+    def device_plan_regions(self, steps: int, warmup: int, regions: int, graph: bool):
+        """The step with the device-side planner (libra_plan_device + decode), issued eagerly or replayed from a CUDA
+        graph that holds one step per layout x pool copy; same regime as timed_regions.  Returns ms per step (median)."""
         torch = self.torch
         side = torch.cuda.Stream()
         per_replay = len(self.layouts) * len(self.pools)
@@ -203,50 +261,32 @@ class Replica:
             for _ in range(max(warmup, per_replay)):
                 self.step_device(side.cuda_stream)
         torch.cuda.synchronize()
-        g = None
-        if graph:
-            self.i = 0
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=side):
-                for _ in range(per_replay):
-                    self.step_device(side.cuda_stream)
-            g.replay()
-            torch.cuda.synchronize()
+        if not graph:
+            res, _ = self.timed_regions(self.step_device, steps, 0, regions, stream=side)
+            return float(np.median([ms / steps for ms, _ in res])), float(np.median([b / (ms * 1e-3) / 1e9 for ms, b in res]))
+        self.i = 0
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(per_replay):
+                self.step_device(side.cuda_stream)
+        g.replay()
+        torch.cuda.synchronize()
         reps = max(1, steps // per_replay)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        with torch.cuda.stream(side):
-            e0.record()
-            for _ in range(reps):
-                if graph:
+        per, gbs = [], []
+        for _ in range(regions):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            with torch.cuda.stream(side):
+                e0.record()
+                for _ in range(reps):
                     g.replay()
-                else:
-                    for _ in range(per_replay):
-                        self.step_device(side.cuda_stream)
-            e1.record()
-        torch.cuda.synchronize()
+                e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            per.append(ms / (reps * per_replay))
+            gbs.append(self.bytes_of_steps(0, reps * per_replay) / (ms * 1e-3) / 1e9)
         assert self.h.debug_error_word() == 0, "device error word set"
-        return e0.elapsed_time(e1) / (reps * per_replay)
-
-    def timed(self, steps: int, warmup: int, barrier=None):
-        torch = self.torch
-        st = torch.cuda.current_stream().cuda_stream
-        for _ in range(warmup):
-            self.step(st)
-        torch.cuda.synchronize()
-        if barrier:
-            barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n0 = self.h.launch_count()
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(steps):
-            self.step(st)
-        e1.record()
-        torch.cuda.synchronize()
-        if barrier:
-            barrier()
-        assert self.h.debug_error_word() == 0, "device error word set"
-        return e0.elapsed_time(e1), self.h.launch_count() - n0
+        return float(np.median(per)), float(np.median(gbs))
 
     def step_gather_read(self, stream: int) -> None:
         """The step with the attention math removed: same plan, page walk and copies (a read ceiling)."""
@@ -262,64 +302,113 @@ class Replica:
             self._scratch_out = self.torch.zeros_like(self.out)
         return self._scratch_out
 
-    def repeats(self, fn, reps: int, calls_each: int):
-        """(median, best) ms per call over `reps` event-timed batches of `calls_each` back-to-back calls."""
-        torch = self.torch
-        st = torch.cuda.current_stream().cuda_stream
-        times = []
-        for r in range(reps + 3):  # three untimed batches first
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
-            e0.record()
-            for _ in range(calls_each):
-                fn(st)
-            e1.record()
-            torch.cuda.synchronize()
-            if r >= 3:
-                times.append(e0.elapsed_time(e1) / calls_each)
-        return float(np.median(times)), float(min(times))
-
     def kernel_times(self, steps: int):
-        """Same steps with CUDA events around each kernel (recorded by the library on its stream)."""
+        """The same steps with a CUDA event pair around every kernel (recorded by the library on its stream): the
+        decode kernel's own duration, launch by launch, without the overlap of consecutive launches.
+        Returns (decode ms per launch, ms after decode per launch, launches, KV bytes of those launches)."""
         torch = self.torch
         st = torch.cuda.current_stream().cuda_stream
         steps = min(steps, 4096)
+        i0 = self.i
         self.h.profile_begin()
         for _ in range(steps):
             self.step(st)
         torch.cuda.synchronize()
         d, c, n = self.h.profile_end()
-        return d / n, c / n, n
+        return d / n, c / n, n, self.bytes_of_steps(i0, n)
 
     def close(self):
         self.h.close()
 
 
-def ceilings_measure(rep: Replica, reps: int = 20):
-    """What the step's read rate is set against: the step itself, the same step with the attention math removed
-    (same plan, page walk and tiled copies), and a plain streaming read of a contiguous 4 GiB buffer; each as
-    (median, best) over `reps` batches."""
+def median_gbs(res):
+    return float(np.median([b / (ms * 1e-3) / 1e9 for ms, b in res]))
+
+
+def ceilings_measure(rep: Replica, steps: int, regions: int, step_gbs: float):
+    """What the step's read rate is set against, timed in the SAME regime as the step (regions of `steps` chained
+    calls, median): the step with the attention math removed (same plan, page walk and tiled copies), and a plain
+    streaming read of a contiguous 4 GiB buffer (as many calls per region as take about as long as the step's)."""
     torch = rep.torch
-    ms_guess = rep.kv_bytes_per_step / 6.4e12 * 1e3   # batches of ~1.5 ms, whole cycles of a multi-step workload
-    per_batch = len(rep.layouts) * max(1, int(round(1.5 / (ms_guess * len(rep.layouts)))))
-    step_med, step_best = rep.repeats(rep.step, reps, per_batch)
-    gat_med, gat_best = rep.repeats(rep.step_gather_read, reps, per_batch)
-    assert rep.h.debug_error_word() == 0, "device error word set"
+    gat, _ = rep.timed_regions(rep.step_gather_read, steps, 3, regions)
+    gat_gbs = median_gbs(gat)
     nbytes = 4 << 30
     buf = torch.zeros(nbytes, dtype=torch.uint8, device=rep.dev)
-    rd_med, rd_best = rep.repeats(lambda st: rep.h.debug_stream_read(buf.data_ptr(), nbytes, st), reps, 2)
+    region_ms = float(np.median([ms for ms, _ in gat]))
+    calls = max(2, int(round(region_ms / (nbytes / 7.2e12 * 1e3))))
+    rd = []
+    st = torch.cuda.current_stream().cuda_stream
+    for r in range(regions + 2):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(calls):
+            rep.h.debug_stream_read(buf.data_ptr(), nbytes, st)
+        e1.record()
+        torch.cuda.synchronize()
+        if r >= 2:
+            rd.append((e0.elapsed_time(e1), float(nbytes) * calls))
     del buf
-    gbs = lambda b, ms: b / (ms * 1e-3) / 1e9
-    kv = rep.kv_bytes_per_step
-    return {"reps": reps, "calls_per_rep": per_batch,
-            "step_us_median": step_med * 1e3, "step_us_best": step_best * 1e3,
-            "step_gbs_median": gbs(kv, step_med), "step_gbs_best": gbs(kv, step_best),
-            "page_gather_read_gbs_median": gbs(kv, gat_med), "page_gather_read_gbs_best": gbs(kv, gat_best),
-            "contiguous_read_gbs_median": gbs(nbytes, rd_med), "contiguous_read_gbs_best": gbs(nbytes, rd_best),
-            "step_frac_of_page_gather_read": gat_med / step_med,
-            "step_frac_of_contiguous_read": gbs(kv, step_med) / gbs(nbytes, rd_med),
+    rd_gbs = median_gbs(rd)
+    return {"regions": regions, "steps_per_region": steps, "read_calls_per_region": calls,
+            "page_gather_read_gbs": gat_gbs, "contiguous_read_gbs": rd_gbs,
+            "step_frac_of_page_gather_read": step_gbs / gat_gbs, "step_frac_of_contiguous_read": step_gbs / rd_gbs,
             "note": "page_gather_read = libra_debug_gather_read (the decode kernel's plan, grid, block-table walk and "
-                    "tiled copies, no math); contiguous_read = libra_debug_stream_read over 4 GiB"}
+                    "tiled copies, no math); contiguous_read = libra_debug_stream_read over 4 GiB; both in regions of "
+                    "chained calls like the step"}
+
+
+def measure_workload(rep: Replica, steps: int, warmup: int, regions: int, peak: float, barrier=None, world: int = 1,
+                     agg_dev=None, with_ceilings: bool = True, with_device_plan: bool = True):
+    """Everything the summary of one workload needs, from one replica: the chained regions, the per-launch kernel
+    duration, the read ceilings and the device-planned step."""
+    res, launches = rep.timed_regions(rep.step, steps, warmup, regions, barrier, world, agg_dev)
+    per_step = np.array([ms / steps for ms, _ in res])
+    gbs = np.array([b / (ms * 1e-3) / 1e9 for ms, b in res])
+    kv_per_step = float(np.mean([b / steps for _, b in res])) / world
+    dec_ms, after_ms, n_prof, prof_bytes = rep.kernel_times(max(steps, 3 * len(rep.layouts)) if steps < 200 else 200)
+    kernel_gbs = prof_bytes / n_prof / (dec_ms * 1e-3) / 1e9
+    m = {"kv_bytes_per_step": kv_per_step, "ms_per_step": float(np.median(per_step)),
+         "ms_per_step_best": float(per_step.min()), "ms_per_step_worst": float(per_step.max()),
+         "spread_pct": float((per_step.max() - per_step.min()) / np.median(per_step) * 100.0),
+         "regions": regions, "steps_per_region": steps,
+         "kv_gbs": float(np.median(gbs)), "kv_gbs_best": float(gbs.max()),
+         "frac_chained_of_measured": float(np.median(gbs)) / world / peak,
+         "frac_chained_of_8TBs": float(np.median(gbs)) / world / NOMINAL_HBM_GBS,
+         "kernel_us_event_pairs": dec_ms * 1e3, "after_decode_us_event_pairs": after_ms * 1e3,
+         "kernel_gbs": kernel_gbs, "frac_kernel_of_measured": kernel_gbs / peak,
+         "frac_kernel_of_8TBs": kernel_gbs / NOMINAL_HBM_GBS, "kernel_launches_timed": n_prof,
+         "launches": int(launches), "pool_copies": len(rep.pools)}
+    if world == 1:
+        if len(rep.layouts) == 1:   # the plan reused: decode + combine only (a caller whose lengths did not change)
+            st = rep.torch.cuda.current_stream().cuda_stream
+            rep.h.plan(rep.layouts[0].seq_lens, rep.ws.data_ptr(), rep.ws.numel(), st)
+            r2, _ = rep.timed_regions(rep.step_decode_only, steps, 3, regions)
+            m["ms_per_step_plan_reused"] = float(np.median([ms / steps for ms, _ in r2]))
+        if with_ceilings:
+            m["ceilings"] = ceilings_measure(rep, steps, max(5, regions // 2), m["kv_gbs"])
+        if with_device_plan:
+            e_ms, e_gbs = rep.device_plan_regions(steps, 6, max(5, regions // 2), graph=False)
+            g_ms, g_gbs = rep.device_plan_regions(steps, 6, max(5, regions // 2), graph=True)
+            m["device_plan"] = {"ms_per_step_eager": e_ms, "kv_gbs_eager": e_gbs, "ms_per_step_cuda_graph": g_ms,
+                                "kv_gbs_cuda_graph": g_gbs, "over_host_plan_us": (g_ms - m["ms_per_step"]) * 1e3,
+                                "note": "libra_plan_device + decode; the graph holds one step per layout x pool copy"}
+    return m
+
+
+def compact(m: dict) -> dict:
+    """The per-workload figures that must survive in the top-level line."""
+    c = {"kv_gbs": round(m["kv_gbs"], 1), "ms_per_step": round(m["ms_per_step"], 5),
+         "frac_of_measured": round(m["frac_chained_of_measured"], 4), "frac_of_8TBs": round(m["frac_chained_of_8TBs"], 4),
+         "kernel_us_event_pairs": round(m["kernel_us_event_pairs"], 2),
+         "frac_kernel_of_measured": round(m["frac_kernel_of_measured"], 4),
+         "frac_kernel_of_8TBs": round(m["frac_kernel_of_8TBs"], 4), "spread_pct": round(m["spread_pct"], 2)}
+    if "ceilings" in m:
+        c["frac_of_contiguous_read"] = round(m["ceilings"]["step_frac_of_contiguous_read"], 4)
+        c["frac_of_page_gather_read"] = round(m["ceilings"]["step_frac_of_page_gather_read"], 4)
+    if "device_plan" in m:
+        c["device_plan_graph_ms"] = round(m["device_plan"]["ms_per_step_cuda_graph"], 5)
+    return c
 
 
 def multi_token_measure(rep: Replica, q_len: int, steps: int = 200, variant=None):
@@ -857,6 +946,29 @@ def oracle_baseline(name: str, k_dev=None, v_dev=None, q_dev=None, budget_s: flo
 
 
 # ----------------------------------------------------------------------------- arms
+def make_config(name: str, world: int) -> dict:
+    """The `config` of the JSON line: what the workload is, the same for both arms."""
+    from paper_2606_03077_b200 import workloads as W
+
+    w = W.WORKLOADS[name]
+    kv = [W.make_layout(name, s)[0].kv_bytes for s in range(w.steps)]
+    copies = pool_copies_for(w.steps, kv[0])
+    l2 = (f"every step reads {min(kv) / 1e9:.2f} GB or more of KV, at least {min(kv) / L2_BYTES_ASSUMED:.0f} x the 126 MB L2"
+          if copies == 1 else
+          f"steps rotate over {copies} copies of the KV pools ({copies * kv[0] / 1e9:.2f} GB live KV vs 126 MB L2)")
+    return {"workload": name, "batch": w.batch, "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads,
+            "head_dim": w.head_dim, "page_size": w.page_size, "kv_bytes_per_step": float(np.mean(kv)),
+            "parallelism": f"replicas x{world}", "l2": l2,
+            "step": "libra_plan + decode kernel (the combine step runs inside it)"}
+
+
+def pool_copies_for(steps_in_workload: int, kv_bytes: int) -> int:
+    """Copies of the KV pools a replica rotates over, so that 4 x L2 of other data passes before a pool is read again."""
+    if steps_in_workload > 1 or kv_bytes >= 6 * L2_BYTES_ASSUMED:
+        return 1
+    return max(1, min(8, -(-4 * L2_BYTES_ASSUMED // max(1, kv_bytes)) + 1))
+
+
 def run_reference(args):
     rank, _, world = dist_env()
     if rank != 0:
@@ -880,14 +992,12 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
             "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "batch": lay.workload.batch, "q_heads": lay.workload.num_q_heads,
-                       "kv_heads": lay.workload.num_kv_heads, "head_dim": lay.workload.head_dim, "page_size": 16,
-                       "kv_bytes_per_step": lay.kv_bytes,
-                       "note": "each step times the CPU oracle on a bounded sample of the workload's sequences; "
-                               "ms_per_step extrapolates to the whole batch"},
+            "config": make_config(args.workload, max(1, args.gpus)),
             "cpu_baseline": {k: t_all[-1][k] for k in ("value", "unit", "cores", "kind", "sample")},
             "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-            "steps_per_s": 1e3 / ms, "gpu_launches": 0}
+            "steps_per_s": 1e3 / ms, "gpu_launches": 0,
+            "note": "each step times the CPU oracle on a bounded sample of the workload's sequences; ms_per_step "
+                    "extrapolates to the whole batch"}
     line["cpu_baseline"]["value"] = gbs
     print(json.dumps(line), flush=True)
 
@@ -914,51 +1024,56 @@ def run_libra(args):
     barrier = (lambda: torch.distributed.barrier()) if world > 1 else None
 
     from paper_2606_03077_b200 import binding as _b
+    from paper_2606_03077_b200 import workloads as W
 
     variant = tuple(int(x) for x in args.variant.split(",")) if args.variant else None
     plan = _b.PlanParams(0, args.ctas_per_sm, args.items_per_slot, 0, 0, 0) if (args.ctas_per_sm or args.items_per_slot) else None
+    peak, peak_src = measured_hbm_peak()
+    regions = max(1, args.regions)
+    solo = rank == 0 and world == 1
+
     rep = Replica(args.workload, dev, plan=plan, variant=variant)
     sampler = ClockSampler(local_rank)
     sampler.start()
-    elapsed_ms, launches = rep.timed(args.steps, args.warmup, barrier)
-    dec_ms, cmb_ms, n_prof = rep.kernel_times(min(args.steps, 2000))
+    m = measure_workload(rep, args.steps, args.warmup, regions, peak, barrier, world, agg_dev,
+                         with_ceilings=solo and not args.only_main, with_device_plan=solo and not args.only_main)
     clocks = sampler.stop()
 
-    units = rep.kv_bytes_per_step * args.steps
-    t_max, units_all = aggregate_over_ranks(elapsed_ms, units, world, agg_dev)
-    ms_per_step = t_max / args.steps
-    value = units_all / (t_max * 1e-3) / 1e9
+    ratio = NCU_TRAFFIC_OVER_ALGORITHMIC.get(args.workload)
+    roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": m["kernel_gbs"], "peak": peak, "unit": "GB/s",
+                "frac": m["frac_kernel_of_measured"], "frac_kernel": m["frac_kernel_of_measured"],
+                "frac_chained": m["frac_chained_of_measured"],
+                "frac_kernel_of_8TBs": m["frac_kernel_of_8TBs"], "frac_chained_of_8TBs": m["frac_chained_of_8TBs"],
+                "peak_source": peak_src,
+                "traffic": (m["kv_bytes_per_step"] * (ratio if ratio else float(np.mean(list(NCU_TRAFFIC_OVER_ALGORITHMIC.values()))))),
+                "traffic_source": ("ncu capture of this workload, profiles/" if ratio else
+                                   "scaled from the ncu captures of lognormal_b64 and straggler_b8 (1.004 - 1.018 x the "
+                                   "algorithmic bytes): this workload is too large to capture under the profiler"),
+                "algorithmic_bytes_per_launch": m["kv_bytes_per_step"], "kernel_us": m["kernel_us_event_pairs"],
+                "chained_step_us": m["ms_per_step"] * 1e3,
+                "timing": "frac / frac_kernel: a CUDA event pair around every decode launch (the kernel's own duration); "
+                          "frac_chained: step spacing of the timed region, where consecutive launches overlap",
+                "launches_timed": m["kernel_launches_timed"],
+                "per_workload": {args.workload: compact(m)}}
 
-    peak, peak_src = measured_hbm_peak()
-    # average launch duration of the decode kernel: when a step is that one launch, the timed region itself
-    # (events around K back-to-back launches) gives it; otherwise the per-kernel event pairs do, each of
-    # which adds ~3 us to what it brackets
-    one_launch_per_step = launches == args.steps
-    kernel_ms = (elapsed_ms / args.steps) if one_launch_per_step else dec_ms
-    achieved = rep.kv_bytes_per_step / (kernel_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_source": peak_src, "traffic": NCU_DECODE_TRAFFIC_BYTES.get(args.workload),
-                "algorithmic_bytes_per_launch": rep.kv_bytes_per_step, "kernel_us": kernel_ms * 1e3,
-                "timing": ("CUDA events around the timed region, one decode launch per step" if one_launch_per_step
-                           else "CUDA event pair around every decode launch"),
-                "decode_kernel_us_with_event_pairs": dec_ms * 1e3, "after_decode_us_with_event_pairs": cmb_ms * 1e3,
-                "launches_timed": n_prof, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
-
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+    line = {"metric": METRIC, "value": m["kv_gbs"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": m["ms_per_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": args.workload, "batch": rep.w.batch, "q_heads": rep.w.num_q_heads,
-                       "kv_heads": rep.w.num_kv_heads, "head_dim": rep.w.head_dim, "page_size": 16,
-                       "kv_bytes_per_step": rep.kv_bytes_per_step, "parallelism": f"replicas x{world}",
-                       "l2": f"rotating {len(rep.pools)} copies of the KV pools "
-                             f"({len(rep.pools) * rep.layouts[0].kv_bytes / 1e9:.2f} GB live KV vs 126 MB L2)",
-                       "step": "libra_plan + decode kernel (step C runs inside it)"},
-            "steps_per_s": 1e3 / ms_per_step * world,
-            "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
-            "frac_of_measured_copy": value / world / peak,
-            "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline}
+            "config": make_config(args.workload, world),
+            "steps_per_s": 1e3 / m["ms_per_step"] * world,
+            "regions": {"count": regions, "steps_each": args.steps, "ms_per_step_median": m["ms_per_step"],
+                        "ms_per_step_best": m["ms_per_step_best"], "ms_per_step_worst": m["ms_per_step_worst"],
+                        "spread_pct": m["spread_pct"]},
+            "frac_of_nominal_8TBs": m["frac_chained_of_8TBs"],
+            "frac_of_measured_copy": m["frac_chained_of_measured"],
+            "gpu_launches": int(m["launches"]), "clocks": clocks, "roofline": roofline}
+    if "ms_per_step_plan_reused" in m:
+        line["steps_per_s_plan_reused"] = 1e3 / m["ms_per_step_plan_reused"]
+    for key in ("ceilings", "device_plan"):
+        if key in m:
+            line[key] = m[key]
 
-    if rank == 0 and world == 1:
+    if solo:
         k0, v0 = rep.pools[0]
         if not args.no_e2e:
             ms, h2d, d2h, same = e2e_measure(rep, args.e2e_steps)
@@ -967,29 +1082,27 @@ def run_libra(args):
                            "matches_resident_run": same,
                            "note": "libra_decode_attn_host: q, both KV pools, block table, lengths copied from pinned "
                                    "host memory every step, output copied back"}
-            line["e2e_resident_kv"] = e2e_resident_kv_measure(rep, 200)
+            line["e2e_resident_kv"] = e2e_resident_kv_measure(rep, 100)
         extras = set(x for x in args.extras.split(",") if x)
-        if "ceilings" in extras:
-            line["ceilings"] = ceilings_measure(rep)
         if "early_prefetch" in extras:
             # back-to-back steps with libra_set_early_prefetch: the kernel before each decode launch is the previous
             # step's decode kernel, which writes only `out` and the workspace, so the promise holds
             rep.h.set_early_prefetch(True)
-            n = min(args.steps, 1000)
-            ms_e, _ = rep.timed(n, max(3, args.warmup // 2))
+            r_e, _ = rep.timed_regions(rep.step, args.steps, 3, max(5, regions // 2))
             rep.h.set_early_prefetch(False)
-            line["early_prefetch"] = {"ms_per_step": ms_e / n, "kv_gbs": rep.kv_bytes_per_step / (ms_e / n * 1e-3) / 1e9,
-                                      "steps": n, "note": "optional mode, off in the headline number"}
+            line["early_prefetch"] = {"ms_per_step": float(np.median([ms / args.steps for ms, _ in r_e])),
+                                      "kv_gbs": median_gbs(r_e), "note": "optional mode, off in the headline number"}
+        n_x = min(200, max(20, args.steps))
         if "multi_token" in extras:
-            line["multi_token"] = [m for m in (multi_token_measure(rep, t) for t in (2, 4)) if m]
+            line["multi_token"] = [x for x in (multi_token_measure(rep, t, n_x) for t in (2, 4)) if x]
         if "fp8_cache" in extras:
-            line["fp8_cache"] = fp8_cache_measure(rep, steps=min(200, max(10, args.steps)))
+            line["fp8_cache"] = fp8_cache_measure(rep, steps=n_x)
         if "nhd_layout" in extras:
-            line["nhd_layout"] = nhd_layout_measure(rep)
+            line["nhd_layout"] = nhd_layout_measure(rep, n_x)
         if "head_shard" in extras:
-            line["head_shard"] = head_shard_measure(rep)
+            line["head_shard"] = head_shard_measure(rep, n_x)
         if "wide_group" in extras:
-            line["wide_group"] = wide_group_measure(rep)
+            line["wide_group"] = wide_group_measure(rep, n_x)
         if "short_batch" in extras:
             line["short_batch"] = short_batch_measure(rep)
         if "ring_step" in extras:
@@ -1012,37 +1125,22 @@ def run_libra(args):
     torch.cuda.empty_cache()
 
     if not args.only_main and world == 1:
-        from paper_2606_03077_b200 import workloads as W
-
         others = {}
         for name in W.WORKLOAD_ORDER[1:]:
             if name == args.workload:
                 continue
             r = Replica(name, dev)
-            n = max(20, min(args.steps, 400))
-            ms, _ = r.timed(n, max(3, args.warmup // 4))
-            d, c, _ = r.kernel_times(min(n, 200))
-            per = ms / n
-            others[name] = {"kv_gbs": r.kv_bytes_per_step / (per * 1e-3) / 1e9, "ms_per_step": per, "steps": n,
-                            "decode_kernel_us": d * 1e3, "combine_kernel_us": c * 1e3,
-                            "decode_kernel_gbs": r.kv_bytes_per_step / (d * 1e-3) / 1e9,
-                            "frac_of_nominal_8TBs": r.kv_bytes_per_step / (per * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-                            "frac_of_measured_copy": r.kv_bytes_per_step / (per * 1e-3) / 1e9 / peak,
-                            "kv_bytes_per_step": r.kv_bytes_per_step, "pool_copies": len(r.pools)}
-            others[name]["ceilings"] = ceilings_measure(r, reps=10)
-            others[name]["multi_token"] = [m for m in (multi_token_measure(r, t, 60) for t in (2, 3, 4)) if m]
-            others[name]["fp8_cache"] = fp8_cache_measure(r, 60)
-            others[name]["nhd_layout"] = nhd_layout_measure(r, 60)
-            others[name]["head_shard"] = head_shard_measure(r, 60)
-            if name in ("longtail_mix_b256", "straggler_b8"):  # migrating the long sequences: gather to a dense buffer, scatter back
-                others[name]["kv_migration"] = kv_migration_measure(r)
-            if name == "shift_b128":  # the re-planned-every-step workload: also with the device-side planner
-                eager = r.timed_device_plan(n, 6, graph=False)
-                graph = r.timed_device_plan(n, 6, graph=True)
-                others[name]["device_plan"] = {
-                    "ms_per_step_eager": eager, "ms_per_step_cuda_graph": graph,
-                    "kv_gbs_cuda_graph": r.kv_bytes_per_step / (graph * 1e-3) / 1e9,
-                    "note": "libra_plan_device + decode + combine; the graph holds one step per layout and is replayed"}
+            mo = measure_workload(r, args.steps, max(3, args.warmup), regions, peak)
+            roofline["per_workload"][name] = compact(mo)
+            if args.full:
+                n_x = min(60, max(20, args.steps))
+                mo["multi_token"] = [x for x in (multi_token_measure(r, t, n_x) for t in (2, 3, 4)) if x]
+                mo["fp8_cache"] = fp8_cache_measure(r, n_x)
+                mo["nhd_layout"] = nhd_layout_measure(r, n_x)
+                mo["head_shard"] = head_shard_measure(r, n_x)
+                if name in ("longtail_mix_b256", "straggler_b8"):
+                    mo["kv_migration"] = kv_migration_measure(r)
+            others[name] = mo
             r.close()
             del r
             torch.cuda.empty_cache()
@@ -1057,16 +1155,18 @@ def run_libra(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--regions", type=int, default=REGIONS, help="timed regions of --steps steps each (median reported)")
     ap.add_argument("--impl", default="libra", choices=["libra", "reference"])
     ap.add_argument("--workload", default=MAIN_WORKLOAD)
-    ap.add_argument("--only-main", action="store_true", help="skip the other workloads")
+    ap.add_argument("--only-main", action="store_true", help="skip the other workloads, the ceilings and the device plan")
+    ap.add_argument("--full", action="store_true", help="the side measurements on every workload, not only the headline")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
-    ap.add_argument("--extras", default="ceilings,early_prefetch,multi_token,fp8_cache,nhd_layout,head_shard,wide_group,short_batch,kv_migration,ring_step",
+    ap.add_argument("--extras", default="early_prefetch,multi_token,fp8_cache,nhd_layout,head_shard,wide_group,short_batch,kv_migration,ring_step",
                     help="side measurements on the main workload at N=1 (comma list; empty = none)")
     ap.add_argument("--variant", default="", help="warps,stages of the decode block (default: the library's)")
     ap.add_argument("--ctas-per-sm", type=int, default=0, help="planner constant (0 = default)")

@@ -93,15 +93,17 @@ __device__ __forceinline__ void combine_row(const float* partial_o, const float*
 template <int D>
 __global__ void __launch_bounds__(kCombineWarps * 32)
 combine_kernel(const __grid_constant__ CombineParams p, const __grid_constant__ ParamFix pf) {
+  // Launched as a programmatic dependent of the decode kernel: wait until that grid has finished and its
+  // partial results (and a device-side plan's counts) are visible.  EVERY thread waits, also those that have
+  // nothing to do: a grid that completes without waiting would let whatever follows it in the stream start
+  // while the decode kernel is still running.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int lane = threadIdx.x & 31;
   const int h = blockIdx.y * kCombineWarps + (threadIdx.x >> 5);
   const int Hq = p.num_q_heads;
   if (h >= Hq) return;
   if (p.dev_counts && int(blockIdx.x) >= p.dev_counts[plan_layout::kCntCombine]) return;  // grid is an upper bound
   const int4 fix = (p.entries ? p.entries : pf.e)[blockIdx.x];  // plain load: may address parameter space
-  // launched as a programmatic dependent of the decode kernel: wait until that grid has finished
-  // and its partial results are visible
-  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (lane == 0 && h == 0 && fix.w != __ldg(p.seq_lens + fix.x)) {
     atomicOr(p.error_word, LIBRA_DEV_ERR_SEQ_LEN_MISMATCH);
   }

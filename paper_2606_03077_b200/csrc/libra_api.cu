@@ -1117,6 +1117,20 @@ int libra_decode_attn_static(libra_handle_t h, const int32_t* seq_lens_host, int
                              const int32_t* seq_lens, void* out, void* stream) {
   if (!h) return LIBRA_INVALID_ARGUMENT;
   if (h->workspace_bytes > size_t(LIBRA_STATIC_SCRATCH_BYTES)) return LIBRA_WORKSPACE_TOO_SMALL;
+  // everything libra_decode_attn would refuse is refused here, before the shared region or the handle's
+  // plan is touched: a rejected call must not clear another call's error word or re-plan the handle
+  if (!q || !k_pages || !v_pages || !block_table || !seq_lens || !out) return LIBRA_INVALID_ARGUMENT;
+  if (reinterpret_cast<uintptr_t>(k_pages) % 16 || reinterpret_cast<uintptr_t>(v_pages) % 16 ||
+      reinterpret_cast<uintptr_t>(q) % 4 || reinterpret_cast<uintptr_t>(out) % 8) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  if (batch < 0 || batch > h->cfg.max_batch || (batch > 0 && !seq_lens_host)) return LIBRA_INVALID_ARGUMENT;
+  {
+    const int64_t max_len = int64_t(h->cfg.block_table_ld) * h->cfg.page_size;
+    for (int32_t b = 0; b < batch; ++b) {
+      if (seq_lens_host[b] < 0 || seq_lens_host[b] > max_len) return LIBRA_INVALID_ARGUMENT;
+    }
+  }
   void* scratch = nullptr;
   {
     DeviceGuard guard(h->cfg.device);  // the symbol's address is per device: look it up with that device current

@@ -46,11 +46,14 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
+// A streaming 16-byte load on the coherent path (not `.nc`): `dst` may be `own` (in-place ReduceScatter), and the
+// read-only path is defined only for memory that nothing writes while the kernel runs.
 __device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
   uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+  asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
+               : "l"(p)
+               : "memory");
   return v;
 }
 __device__ __forceinline__ uint32_t add_bf16x2(uint32_t a, uint32_t b) {

@@ -76,7 +76,7 @@ def run_host_case(binding, q, k, v, bt, lens, layout="HND", plan=None, sm_scale=
 
 def gather_for_oracle(k_dev, v_dev, block_table, seq_lens, rows):
     """Copy the pages of sequences `rows` back to the host as a compact pool and a remapped block
-    table, so that the CPU oracle can evaluate a sample of a workload whose pools live on the GPU."""
+    table, so that the CPU oracle can evaluate sequences of a workload whose pools live on the GPU."""
     import torch
     ids = []
     new_bt = np.full((len(rows), block_table.shape[1]), -1, dtype=np.int32)
@@ -85,6 +85,44 @@ def gather_for_oracle(k_dev, v_dev, block_table, seq_lens, rows):
         new_bt[i, :n] = np.arange(len(ids), len(ids) + n)
         ids.extend(int(x) for x in block_table[b, :n])
     idx = torch.tensor(ids, dtype=torch.long, device=k_dev.device)
-    k = k_dev.view(torch.int16)[idx].cpu().numpy().view(np.uint16)
-    v = v_dev.view(torch.int16)[idx].cpu().numpy().view(np.uint16)
+    if k_dev.dtype == torch.uint8:   # an 8-bit cache: the codes as they are
+        k, v = k_dev[idx].cpu().numpy(), v_dev[idx].cpu().numpy()
+    else:
+        k = k_dev.view(torch.int16)[idx].cpu().numpy().view(np.uint16)
+        v = v_dev.view(torch.int16)[idx].cpu().numpy().view(np.uint16)
     return k, v, new_bt, np.asarray([seq_lens[b] for b in rows], dtype=np.int32)
+
+
+def row_groups(seq_lens, max_tokens=65536):
+    """Every sequence of a batch, in batch order, cut into groups of at most `max_tokens` cached tokens (a
+    sequence longer than that is a group of its own): bounds the host memory of one oracle call."""
+    groups, cur, tok = [], [], 0
+    for b, L in enumerate(int(x) for x in seq_lens):
+        if cur and tok + L > max_tokens:
+            groups.append(cur)
+            cur, tok = [], 0
+        cur.append(b)
+        tok += L
+    if cur:
+        groups.append(cur)
+    return groups
+
+
+def compare_every_sequence(got, q_dev, k_dev, v_dev, block_table, seq_lens, oracle_fn, gates, max_tokens=65536):
+    """Compares `got` (float array, first axis = sequence) with the oracle on EVERY sequence of the batch: the pages
+    of one group of sequences at a time are copied back from the device pools and `oracle_fn(q, k, v, bt, lens)`
+    is evaluated on them.  Asserts both gates element-wise; returns (max abs err, worst tight-gate ratio)."""
+    import torch
+    worst_abs, worst_ratio, checked = 0.0, 0.0, 0
+    for rows in row_groups(seq_lens, max_tokens):
+        kh, vh, bth, lh = gather_for_oracle(k_dev, v_dev, block_table, seq_lens, rows)
+        qh = q_dev.view(torch.int16)[rows[0]:rows[-1] + 1].cpu().numpy().view(np.uint16)
+        ref = oracle_fn(qh, kh, vh, bth, lh)
+        g = got[rows[0]:rows[-1] + 1]
+        assert gates.stated_violations(g, ref) == 0, (rows[0], rows[-1])
+        assert gates.tight_violations(g, ref) == 0, (rows[0], rows[-1], gates.tight_ratio(g, ref))
+        worst_abs = max(worst_abs, float(np.max(np.abs(g - ref))) if g.size else 0.0)
+        worst_ratio = max(worst_ratio, gates.tight_ratio(g, ref))
+        checked += len(rows)
+    assert checked == len(seq_lens)
+    return worst_abs, worst_ratio

@@ -173,3 +173,33 @@ def test_recorded_step_replays_over_changing_lengths(lib):
         assert gates.tight_violations(got, ref) == 0 and gates.stated_violations(got, ref) == 0, lens
     assert h.debug_error_word() == 0
     h.close()
+
+
+def test_separate_combine_with_nothing_to_merge_keeps_the_chain_ordered(lib):
+    """Device-side plan, step C as its own kernel, and a batch in which no sequence is split: every block of the
+    combine grid has nothing to do.  It must still wait for the decode kernel before it ends, or the next step in
+    the stream (a programmatic dependent of the combine grid) could overtake a decode kernel that is still writing.
+    A chain of such steps that feed each other (each step's q is the previous step's output) gives the bits of the
+    chain run with step C inside the decode kernel."""
+    import torch
+    dev = torch.device("cuda:0")
+    lens = [700, 40, 1, 333, 512, 16, 0, 90]
+    Hq, Hkv, d = 32, 8, 128
+    lens_a, bt, q, k, v = W.random_case(77, len(lens), Hq, Hkv, d, lens)
+    dq, dk, dv, dbt = (H.to_dev(x, dev) for x in (q, k, v, bt))
+    dl = torch.from_numpy(lens_a.copy()).to(dev)
+    results = []
+    for mode in (1, 0):
+        r = H.Runner(lib, Hq, Hkv, d, k.shape[0], len(lens), bt.shape[1], variant=(8, 3), fused=mode)
+        st = torch.cuda.current_stream().cuda_stream
+        bufs = [dq.clone(), torch.zeros_like(dq)]
+        r.h.plan_device(dl.data_ptr(), len(lens), r.ws.data_ptr(), r.ws.numel(), st)
+        for i in range(24):   # back to back, no host synchronisation in between
+            r.h.decode_attn(bufs[i & 1].data_ptr(), dk.data_ptr(), dv.data_ptr(), dbt.data_ptr(), dl.data_ptr(),
+                            bufs[(i + 1) & 1].data_ptr(), st)
+        torch.cuda.synchronize()
+        assert r.h.debug_error_word() == 0
+        assert len(r.h.plan_export()["combine"]) == 0
+        results.append(bufs[0].cpu().numpy().copy())
+        r.h.close()
+    assert np.array_equal(results[0], results[1])

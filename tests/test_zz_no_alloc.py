@@ -8,6 +8,7 @@ here cannot hide another test's result in a stop-at-first-failure run."""
 import numpy as np
 import pytest
 
+from oracle import attention_oracle as O
 from paper_2606_03077_b200 import workloads as W
 
 import gates
@@ -29,21 +30,85 @@ def test_static_scratch_entry_point_matches_workspace_path(lib):
     want = H.bf16_dev_to_f32(r.run(dq, dk, dv, dbt, lens_a))
     assert len(r.h.plan_export()["combine"]) >= 2
 
+    ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)   # the definition itself, not only the other entry point
+
     dl = torch.from_numpy(lens_a.copy()).to(dev)
     st = torch.cuda.current_stream().cuda_stream
     launches = r.h.launch_count()
+    outs = [torch.full((len(lens), Hq, d), H.CANARY, dtype=torch.int16, device=dev) for _ in range(2)]
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info(dev)[0]
     for call in range(2):   # the second call runs on whatever the first left in the region
-        out = torch.full((len(lens), Hq, d), H.CANARY, dtype=torch.int16, device=dev)
         r.h.decode_attn_static(lens_a, dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dbt.data_ptr(), dl.data_ptr(),
-                               out.data_ptr(), st)
+                               outs[call].data_ptr(), st)
         torch.cuda.synchronize()
         assert r.h.debug_error_word() == 0
-        got = H.bf16_dev_to_f32(out)
+    # what the entry point is for: the device's free memory is what it was before the two calls
+    assert torch.cuda.mem_get_info(dev)[0] == free_before
+    for call in range(2):
+        got = H.bf16_dev_to_f32(outs[call])
         assert np.all(np.isfinite(got)), f"call {call}"
+        assert gates.stated_violations(got, ref) == 0, f"call {call}"
+        assert gates.tight_violations(got, ref) == 0, f"call {call}"
         assert gates.stated_violations(got, want) == 0, f"call {call}"
         assert gates.tight_violations(got, want) == 0, f"call {call}"
         assert np.array_equal(got, want), f"call {call}: same kernels, same order -> same bits"
     assert r.h.launch_count() == launches + 4   # decode + combine, twice: the GPU did the work
+    r.h.close()
+
+
+def test_two_handles_take_turns_on_the_shared_region(lib):
+    """Two handles of different shapes alternate on one stream: each call finds the region as the OTHER handle left it
+    (other counters, other partial results) and must still give its own workspace-path bits."""
+    import torch
+    dev = torch.device("cuda:0")
+    st = torch.cuda.current_stream().cuda_stream
+    cases = []
+    for seed, (Hq, Hkv, d, lens) in enumerate([(32, 8, 128, [5000, 1300, 0, 37, 2049]), (8, 2, 64, [3000, 16, 900, 4100])]):
+        lens_a, bt, q, k, v = W.random_case(60 + seed, len(lens), Hq, Hkv, d, lens)
+        r = H.Runner(lib, Hq, Hkv, d, k.shape[0], len(lens), bt.shape[1], plan=lib.PlanParams(0, 2, 4, 256, 512, 64))
+        dq, dk, dv, dbt = (H.to_dev(x, dev) for x in (q, k, v, bt))
+        want = H.bf16_dev_to_f32(r.run(dq, dk, dv, dbt, lens_a))
+        assert len(r.h.plan_export()["combine"]) >= 1
+        dl = torch.from_numpy(lens_a.copy()).to(dev)
+        cases.append((r, lens_a, dq, dk, dv, dbt, dl, want, (len(lens), Hq, d)))
+    outs = []
+    for turn in range(6):   # no synchronisation between the calls: one stream orders them
+        r, lens_a, dq, dk, dv, dbt, dl, want, shape = cases[turn & 1]
+        out = torch.full(shape, H.CANARY, dtype=torch.int16, device=dev)
+        r.h.decode_attn_static(lens_a, dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dbt.data_ptr(), dl.data_ptr(),
+                               out.data_ptr(), st)
+        outs.append(out)
+    torch.cuda.synchronize()
+    for turn, out in enumerate(outs):
+        assert np.array_equal(H.bf16_dev_to_f32(out), cases[turn & 1][7]), turn
+    for c in cases:
+        assert c[0].h.debug_error_word() == 0
+        c[0].h.close()
+
+
+def test_a_rejected_call_leaves_the_region_and_the_plan_alone(lib):
+    """A call that is refused for a bad argument must not clear the shared region (which may hold another call's error
+    word) nor re-plan the handle."""
+    import torch
+    dev = torch.device("cuda:0")
+    lens = [600, 3000]
+    lens_a, bt, q, k, v = W.random_case(63, len(lens), 8, 2, 128, lens)
+    r = H.Runner(lib, 8, 2, 128, k.shape[0], len(lens), bt.shape[1])
+    dq, dk, dv, dbt = (H.to_dev(x, dev) for x in (q, k, v, bt))
+    want = H.bf16_dev_to_f32(r.run(dq, dk, dv, dbt, lens_a))
+    n_items = len(r.h.plan_export()["items"])
+    dl = torch.from_numpy(lens_a.copy()).to(dev)
+    st = torch.cuda.current_stream().cuda_stream
+    out = torch.zeros((len(lens), 8, 128), dtype=torch.int16, device=dev)
+    with pytest.raises(lib.LibraError) as e:   # a null output pointer
+        r.h.decode_attn_static(np.array([5, 5], np.int32), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dbt.data_ptr(),
+                               dl.data_ptr(), 0, st)
+    assert e.value.status == lib.INVALID_ARGUMENT
+    assert len(r.h.plan_export()["items"]) == n_items          # the handle still holds the plan of `lens`
+    r.h.decode_attn(dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dbt.data_ptr(), dl.data_ptr(), out.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert np.array_equal(H.bf16_dev_to_f32(out), want)
     r.h.close()
 
 
