@@ -21,7 +21,15 @@ share its KV range, so:
     the power of two nearer to L / C in ratio;
   * C, the base length, is recomputed for every batch from the total work so that the
     launch has about `items_per_slot` work items per resident block;
-  * items are issued longest first (the classic greedy rule for the min-max objective).
+  * items are issued longest first (the classic greedy rule for the min-max objective);
+  * wave fill: when the whole launch is at most `wave_fill` waves of the W resident blocks (k = cd(U, W) waves of
+    U = Hkv * sum n_b blocks), the free block slots of the last wave are handed out as extra chunks: the
+    floor((k * W - U) / Hkv) sequences with the longest chunks (ties: lower index first) are cut into one chunk
+    more.  A batch of a few equally long sequences - the tail end of a rollout, when only the stragglers are still
+    decoding (Section 2.2) - otherwise runs a full first wave and a part-empty second one of equally long blocks.
+    The paper takes its degrees from {1, 2, 4, 8} because they are tensor-parallel degrees of GPU groups
+    (Section 4.3); chunks inside one GPU have no such constraint, so a topped-up sequence has a chunk count that
+    is not a power of two.  Its bucket (its length class) is unchanged.
 
 The paper states no single-GPU rule; this is the reading this library takes.
 
@@ -42,6 +50,7 @@ class PlanParams:
     min_chunk: int = 512        # C_min
     max_splits: int = 64        # S_max
     small_base: int = 4096      # base lengths below this take the nearer power of two (0 = never: the plain rule)
+    wave_fill: int = 2          # launches of at most this many waves get their last wave filled (0 = never)
 
 
 def cd(a: int, b: int) -> int:
@@ -92,6 +101,17 @@ def plan(seq_lens, num_kv_heads: int, params: PlanParams = PlanParams()) -> Plan
         bucket.append(s.bit_length() - 1)
         chunk.append(c)
         nsplit.append(cd(L, c))
+    # wave fill: free slots of the last wave become extra chunks of the sequences with the longest chunks
+    U = num_kv_heads * sum(nsplit)
+    k = cd(U, W)
+    if 1 <= k <= params.wave_fill:
+        spare = (k * W - U) // num_kv_heads
+        order = sorted((b for b, L in enumerate(lens) if L > 0), key=lambda b: (-chunk[b], b))
+        for b in order[:spare]:
+            c = au(cd(lens[b], nsplit[b] + 1), A)
+            if c >= params.min_chunk and nsplit[b] + 1 <= params.max_splits:
+                chunk[b] = c
+                nsplit[b] = cd(lens[b], c)
     offs, run = [], 0
     for n in nsplit:
         offs.append(run)

@@ -89,6 +89,10 @@ constexpr uint32_t kWaitHintNs = 2000;
 #define LIBRA_MAX_SLACK 8.0f
 #endif
 constexpr float kMaxSlack = LIBRA_MAX_SLACK;
+// 1: the probabilities of a bf16 cache go to the tensor core as two bf16 terms (see process_page)
+#ifndef LIBRA_SPLIT_P
+#define LIBRA_SPLIT_P 1
+#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
@@ -383,6 +387,9 @@ __device__ __forceinline__ void process_page(WarpAcc<D, NT>& st, const uint32_t 
       st.m[nt][1] = m_new[nt][1];
     }
   }
+#if LIBRA_SPLIT_P
+  uint32_t pr[NT][2];   // what rounding P to bf16 lost, as a second bf16 operand
+#endif
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
     const float p0 = ex2(sc[nt][0] - st.m[nt][0]);
@@ -393,9 +400,23 @@ __device__ __forceinline__ void process_page(WarpAcc<D, NT>& st, const uint32_t 
     const __nv_bfloat162 hi = __floats2bfloat162_rn(p2, p3);  // token g+8
     const uint32_t ulo = *reinterpret_cast<const uint32_t*>(&lo);
     const uint32_t uhi = *reinterpret_cast<const uint32_t*>(&hi);
+    const float r0 = __uint_as_float(ulo << 16), r1 = __uint_as_float(ulo & 0xffff0000u);
+    const float r2 = __uint_as_float(uhi << 16), r3 = __uint_as_float(uhi & 0xffff0000u);
+#if LIBRA_SPLIT_P
+    // P = head + tail, both bf16: the tail carries the 8 bits that the head's rounding dropped, so the weights the
+    // tensor core applies are P to 2^-17 instead of 2^-9 (the tensor pipe is all but idle in this kernel; without the
+    // tail the rounding of P is the largest error of the whole step, ~0.2 % of a row's rms)
+    const __nv_bfloat162 lo2 = __floats2bfloat162_rn(p0 - r0, p1 - r1);
+    const __nv_bfloat162 hi2 = __floats2bfloat162_rn(p2 - r2, p3 - r3);
+    pr[nt][0] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&lo2));
+    pr[nt][1] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&hi2));
+    st.l[nt][0] += p0 + p2;
+    st.l[nt][1] += p1 + p3;
+#else
     // the denominator sums exactly the probabilities the tensor core will see
-    st.l[nt][0] += __uint_as_float(ulo << 16) + __uint_as_float(uhi << 16);
-    st.l[nt][1] += __uint_as_float(ulo & 0xffff0000u) + __uint_as_float(uhi & 0xffff0000u);
+    st.l[nt][0] += r0 + r2;
+    st.l[nt][1] += r1 + r3;
+#endif
     pb[nt][0] = movmatrix_trans(ulo);  // head g : tokens 2t, 2t+1
     pb[nt][1] = movmatrix_trans(uhi);  // head g : tokens 2t+8, 2t+9
   }
@@ -406,7 +427,12 @@ __device__ __forceinline__ void process_page(WarpAcc<D, NT>& st, const uint32_t 
     uint32_t a[4];
     ldsm_x4_trans(a, vt + tile_off(v_row, 2 * mt + v_sel));
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) mma_bf16(st.acc[nt][mt], a, pb[nt][0], pb[nt][1]);
+    for (int nt = 0; nt < NT; ++nt) {
+      mma_bf16(st.acc[nt][mt], a, pb[nt][0], pb[nt][1]);
+#if LIBRA_SPLIT_P
+      mma_bf16(st.acc[nt][mt], a, pr[nt][0], pr[nt][1]);
+#endif
+    }
   }
 }
 

@@ -7,6 +7,8 @@
 //   C       = max(min_chunk, au(cd(heads * T, slots), chunk_align))          T = sum of lengths
 //   s_b     = min(p2(cd(L_b, C)), max_splits)      chunk_b = au(cd(L_b, s_b), chunk_align)
 //   n_b     = cd(L_b, chunk_b)                     items sorted by (length desc, b asc, j asc)
+//   wave fill: a launch of at most wave_fill waves of `wave_slots` blocks hands the free slots of its last wave
+//   to the sequences with the longest chunks, one extra chunk each (see planner.cpp)
 //
 // Integer arithmetic only; the result must equal the host planner's bit for bit.  Limits: batch and
 // work items <= kDevPlanMax each (one block, four elements per thread); beyond that, or when a length
@@ -31,6 +33,8 @@ struct PlanKernelParams {
   int32_t heads;             // work units per item (KV heads)
   int64_t slots;             // n_sm * ctas_per_sm * items_per_slot
   int32_t chunk_align, min_chunk, max_splits;
+  int64_t wave_slots;        // n_sm * ctas_per_sm: thread blocks of one wave
+  int32_t wave_fill;         // launches of at most this many waves get their last wave filled (0 = never)
   int32_t max_items;         // capacity of `entries` for work items
   int32_t max_len;           // longest sequence the block table can describe
   int32_t* counts;           // [plan_layout::kCountInts]: num_items, num_combine, num_empty, chunk_target, overflow
@@ -167,12 +171,53 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
     chunk[b] = c;
     offs[b] = n;
     p.per_seq[b] = bucket;
-    p.per_seq[B + b] = n;
-    p.per_seq[2 * B + b] = c;
   }
   __syncthreads();
-  const int n_items = dev::block_exclusive_scan(offs, B, warp_tot);
-  for (int b = tid; b < B; b += kDevPlanThreads) p.per_seq[3 * B + b] = offs[b];
+  int n_items = dev::block_exclusive_scan(offs, B, warp_tot);
+
+  // ---- wave fill: the free slots of the last wave become extra chunks of the sequences with the longest chunks
+  {
+    const long long blocks = (long long)p.heads * n_items;
+    const long long waves = (blocks + p.wave_slots - 1) / p.wave_slots;
+    const long long spare = (waves >= 1 && waves <= p.wave_fill) ? (waves * p.wave_slots - blocks) / p.heads : 0;
+    if (spare > 0) {   // the same for every thread
+      int* new_n = it_len;   // not in use yet
+      int* new_c = it_b;
+      for (int b = tid; b < B; b += kDevPlanThreads) {
+        int n = nsplit[b], c = chunk[b];
+        if (n > 0) {
+          long long rank = 0;   // sequences before this one in (chunk desc, index asc) order
+          for (int k = 0; k < B; ++k) {
+            const int ck = chunk[k];
+            rank += (nsplit[k] > 0 && (ck > c || (ck == c && k < b))) ? 1 : 0;
+          }
+          if (rank < spare) {
+            const long long len = p.seq_lens[b];
+            const long long ch = ((len + n) / (n + 1) + A - 1) / A * A;
+            if (ch >= p.min_chunk && n + 1 <= p.max_splits) {
+              c = int(ch);
+              n = int((len + ch - 1) / ch);
+            }
+          }
+        }
+        new_n[b] = n;
+        new_c[b] = c;
+      }
+      __syncthreads();
+      for (int b = tid; b < B; b += kDevPlanThreads) {
+        nsplit[b] = new_n[b];
+        chunk[b] = new_c[b];
+        offs[b] = new_n[b];
+      }
+      __syncthreads();
+      n_items = dev::block_exclusive_scan(offs, B, warp_tot);
+    }
+  }
+  for (int b = tid; b < B; b += kDevPlanThreads) {
+    p.per_seq[B + b] = nsplit[b];
+    p.per_seq[2 * B + b] = chunk[b];
+    p.per_seq[3 * B + b] = offs[b];
+  }
 
   overflow = n_items > kDevPlanMax || n_items > p.max_items;
   if (overflow) {

@@ -25,6 +25,7 @@ bool valid_params(const PlanParams& p) {
   if (p.chunk_align <= 0 || p.chunk_align % 16 != 0) return false;
   if (p.min_chunk <= 0) return false;
   if (p.max_splits <= 0 || p.max_splits > 64 || (p.max_splits & (p.max_splits - 1)) != 0) return false;
+  if (p.wave_fill < 0 || p.wave_fill > 2) return false;   // max_items() covers two waves
   return true;
 }
 
@@ -54,14 +55,9 @@ bool make_plan(const PlanParams& p, int32_t num_kv_heads, const int32_t* seq_len
   pl.combine.clear();
   pl.empty.clear();
 
-  int32_t running = 0;
   for (int32_t b = 0; b < batch; ++b) {
     const int64_t len = seq_lens[b];
-    pl.item_offset[b] = running;
-    if (len == 0) {
-      pl.empty.push_back(b);
-      continue;
-    }
+    if (len == 0) continue;
     int64_t degree = next_pow2(ceil_div(len, base));
     if (base < plan_layout::kSmallBaseTokens && degree > 1 &&
         len * plan_layout::kGeoMeanDen < (degree / 2) * base * plan_layout::kGeoMeanNum) {
@@ -73,6 +69,45 @@ bool make_plan(const PlanParams& p, int32_t num_kv_heads, const int32_t* seq_len
     pl.bucket[b] = log2_exact(degree);
     pl.chunk_len[b] = int32_t(chunk);
     pl.num_splits[b] = int32_t(pieces);
+  }
+
+  // Wave fill.  The launch is `blocks` thread blocks on `wave` resident ones.  When that is at most wave_fill waves,
+  // the slots the last wave leaves free are handed out as extra chunks, one each to the sequences with the longest
+  // chunks (ties: lower index first): a few equally long sequences otherwise run one full wave and one part-empty
+  // wave of equally long blocks.  The bucket of a sequence (its length class) stays.
+  const int64_t wave = int64_t(p.n_sm) * p.ctas_per_sm;
+  int64_t blocks = 0;
+  for (int32_t b = 0; b < batch; ++b) blocks += int64_t(num_kv_heads) * pl.num_splits[b];
+  const int64_t waves = ceil_div(blocks, wave);
+  if (waves >= 1 && waves <= p.wave_fill) {
+    const int64_t spare = (waves * wave - blocks) / num_kv_heads;
+    std::vector<int32_t> order;
+    for (int32_t b = 0; b < batch; ++b)
+      if (seq_lens[b] > 0) order.push_back(b);
+    const size_t take = size_t(std::min<int64_t>(spare, int64_t(order.size())));
+    std::partial_sort(order.begin(), order.begin() + take, order.end(), [&](int32_t x, int32_t y) {
+      return pl.chunk_len[x] != pl.chunk_len[y] ? pl.chunk_len[x] > pl.chunk_len[y] : x < y;
+    });
+    for (size_t i = 0; i < take; ++i) {
+      const int32_t b = order[i];
+      const int64_t len = seq_lens[b];
+      const int64_t chunk = round_up(ceil_div(len, int64_t(pl.num_splits[b]) + 1), p.chunk_align);
+      if (chunk < p.min_chunk || pl.num_splits[b] + 1 > p.max_splits) continue;
+      pl.chunk_len[b] = int32_t(chunk);
+      pl.num_splits[b] = int32_t(ceil_div(len, chunk));
+    }
+  }
+
+  int32_t running = 0;
+  for (int32_t b = 0; b < batch; ++b) {
+    const int64_t len = seq_lens[b];
+    pl.item_offset[b] = running;
+    if (len == 0) {
+      pl.empty.push_back(b);
+      continue;
+    }
+    const int64_t chunk = pl.chunk_len[b];
+    const int64_t pieces = pl.num_splits[b];
     for (int64_t j = 0; j < pieces; ++j) {
       pl.items.push_back(WorkItem{b, int32_t(j), int32_t(j * chunk), int32_t(std::min(len, (j + 1) * chunk))});
     }

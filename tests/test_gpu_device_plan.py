@@ -16,7 +16,8 @@ pytestmark = pytest.mark.gpu
 
 def ref_params(h):
     p = h.plan_params()
-    return P.PlanParams(p.n_sm, p.ctas_per_sm, p.items_per_slot, p.chunk_align, p.min_chunk, p.max_splits)
+    return P.PlanParams(p.n_sm, p.ctas_per_sm, p.items_per_slot, p.chunk_align, p.min_chunk, p.max_splits,
+                        wave_fill=max(p.wave_fill, 0))
 
 
 def assert_same_plan(got, ref):
@@ -75,6 +76,33 @@ def test_random_and_edge_vectors_bit_exact(lib):
             assert_same_plan(h.plan_export(), ref)
             assert h.debug_error_word() == 0
         h.close()
+
+
+def test_few_waves_bit_exact(lib):
+    """Small batches of long sequences: launches of one or two waves, where the planner hands the free slots of the
+    last wave out as extra chunks (and ties between equal chunks go to the lower index)."""
+    rng = np.random.default_rng(12)
+    filled = 0
+    for i in range(60):
+        B = int(rng.integers(1, 40))
+        base = int(rng.choice([600, 3000, 12000, 30000]))
+        lens = (np.full(B, base) if i % 3 == 0 else
+                np.clip(np.floor(base * np.exp(rng.normal(size=B) * rng.uniform(0.05, 0.8))), 0, 40960)).astype(np.int32)
+        if i % 5 == 0:
+            lens[rng.integers(0, B)] = 0
+        hkv = int(rng.choice([1, 2, 4, 8]))
+        plan = lib.PlanParams(int(rng.choice([16, 74, 148])), int(rng.integers(1, 3)), int(rng.integers(1, 3)),
+                              int(rng.choice([16, 256])), int(rng.choice([16, 512])), int(rng.choice([2, 8, 64])),
+                              int(rng.choice([0, 1, 2, -1])))
+        h, ws, dl = device_plan(lib, lens, hkv, plan)
+        prm = ref_params(h)
+        ref = P.plan(lens, hkv, prm)
+        assert_same_plan(h.plan_export(), ref)
+        assert h.debug_error_word() == 0
+        import dataclasses
+        filled += ref.num_splits != P.plan(lens, hkv, dataclasses.replace(prm, wave_fill=0)).num_splits
+        h.close()
+    assert filled > 10
 
 
 def test_overflow_is_flagged_and_nothing_runs(lib):
