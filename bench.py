@@ -1027,8 +1027,8 @@ def run_libra(args):
     from paper_2606_03077_b200 import workloads as W
 
     variant = tuple(int(x) for x in args.variant.split(",")) if args.variant else None
-    plan = (_b.PlanParams(0, args.ctas_per_sm, args.items_per_slot, 0, 0, 0, args.wave_fill)
-            if (args.ctas_per_sm or args.items_per_slot or args.wave_fill) else None)
+    plan = (_b.PlanParams(0, args.ctas_per_sm, args.items_per_slot, 0, 0, 0, args.refine)
+            if (args.ctas_per_sm or args.items_per_slot or args.refine) else None)
     peak, peak_src = measured_hbm_peak()
     regions = max(1, args.regions)
     solo = rank == 0 and world == 1
@@ -1172,7 +1172,7 @@ def main():
     ap.add_argument("--variant", default="", help="warps,stages of the decode block (default: the library's)")
     ap.add_argument("--ctas-per-sm", type=int, default=0, help="planner constant (0 = default)")
     ap.add_argument("--items-per-slot", type=int, default=0, help="planner constant (0 = default)")
-    ap.add_argument("--wave-fill", type=int, default=0, help="planner constant (0 = default, -1 = never)")
+    ap.add_argument("--refine", type=int, default=0, help="planner constant (0 = default, -1 = never)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":

@@ -81,9 +81,9 @@ typedef struct {
                              multiple of 16); default 256                                       */
   int32_t min_chunk;      /* C_min: lower bound of the base chunk length; default 512           */
   int32_t max_splits;     /* S_max: cap of the split degree (power of two <= 64); default 64     */
-  int32_t wave_fill;      /* launches of at most this many waves of n_sm * ctas_per_sm blocks get the
-                             free slots of their last wave filled with extra chunks of the sequences
-                             with the longest chunks; default 2; -1 = never                      */
+  int32_t refine;         /* 0 or 1 (default): a plan of fewer than one and a half waves of
+                             n_sm * ctas_per_sm blocks whose base chunk is 4096 tokens or longer is
+                             made again for twice as many slots; -1 = never                      */
 } libra_plan_params_t;
 
 typedef struct {

@@ -28,7 +28,7 @@ ERR_WAIT_TIMEOUT, ERR_BAD_PAGE_ID, ERR_SEQ_LEN_MISMATCH, ERR_PLAN_OVERFLOW = 1, 
 class PlanParams(C.Structure):
     _fields_ = [("n_sm", C.c_int32), ("ctas_per_sm", C.c_int32), ("items_per_slot", C.c_int32),
                 ("chunk_align", C.c_int32), ("min_chunk", C.c_int32), ("max_splits", C.c_int32),
-                ("wave_fill", C.c_int32)]
+                ("refine", C.c_int32)]
 
 
 class Config(C.Structure):

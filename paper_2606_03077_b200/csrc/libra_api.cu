@@ -242,8 +242,7 @@ libra::PlanParams resolve_params(const libra_plan_params_t& in, int n_sm_device)
   if (in.chunk_align > 0) p.chunk_align = in.chunk_align;
   if (in.min_chunk > 0) p.min_chunk = in.min_chunk;
   if (in.max_splits > 0) p.max_splits = in.max_splits;
-  if (in.wave_fill > 0) p.wave_fill = in.wave_fill;
-  else if (in.wave_fill < 0) p.wave_fill = 0;   // -1 = never
+  if (in.refine < 0) p.refine = 0;   // -1 = never
   return p;
 }
 
@@ -414,7 +413,7 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
   }
   libra_plan_params_t pin = cfg->plan;
   if (pin.n_sm < 0 || pin.ctas_per_sm < 0 || pin.items_per_slot < 0 || pin.chunk_align < 0 || pin.min_chunk < 0 ||
-      pin.max_splits < 0 || pin.wave_fill < -1) {
+      pin.max_splits < 0 || pin.refine < -1 || pin.refine > 1) {
     return LIBRA_INVALID_ARGUMENT;
   }
 
@@ -554,7 +553,7 @@ int libra_get_plan_params(libra_handle_t h, libra_plan_params_t* out) {
   out->chunk_align = h->params.chunk_align;
   out->min_chunk = h->params.min_chunk;
   out->max_splits = h->params.max_splits;
-  out->wave_fill = h->params.wave_fill > 0 ? h->params.wave_fill : -1;
+  out->refine = h->params.refine ? 1 : -1;
   return LIBRA_OK;
 }
 
@@ -655,7 +654,7 @@ int libra_plan_device(libra_handle_t h, const int32_t* seq_lens_dev, int32_t bat
   p.min_chunk = h->params.min_chunk;
   p.max_splits = h->params.max_splits;
   p.wave_slots = int64_t(h->params.n_sm) * h->params.ctas_per_sm;
-  p.wave_fill = h->params.wave_fill;
+  p.refine = h->params.refine;
   p.max_items = int32_t(std::min<int64_t>(h->max_items, libra::kDevPlanMax));
   p.max_len = int32_t(std::min<int64_t>(int64_t(h->cfg.block_table_ld) * h->cfg.page_size, 0x7fffffff));
   p.counts = reinterpret_cast<int32_t*>(ws + h->dev_counts_off);

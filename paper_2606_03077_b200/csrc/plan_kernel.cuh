@@ -7,8 +7,7 @@
 //   C       = max(min_chunk, au(cd(heads * T, slots), chunk_align))          T = sum of lengths
 //   s_b     = min(p2(cd(L_b, C)), max_splits)      chunk_b = au(cd(L_b, s_b), chunk_align)
 //   n_b     = cd(L_b, chunk_b)                     items sorted by (length desc, b asc, j asc)
-//   wave fill: a launch of at most wave_fill waves of `wave_slots` blocks hands the free slots of its last wave
-//   to the sequences with the longest chunks, one extra chunk each (see planner.cpp)
+//   a plan of fewer than one and a half waves of long blocks is made again for twice as many slots (plan_layout.hpp)
 //
 // Integer arithmetic only; the result must equal the host planner's bit for bit.  Limits: batch and
 // work items <= kDevPlanMax each (one block, four elements per thread); beyond that, or when a length
@@ -34,7 +33,7 @@ struct PlanKernelParams {
   int64_t slots;             // n_sm * ctas_per_sm * items_per_slot
   int32_t chunk_align, min_chunk, max_splits;
   int64_t wave_slots;        // n_sm * ctas_per_sm: thread blocks of one wave
-  int32_t wave_fill;         // launches of at most this many waves get their last wave filled (0 = never)
+  int32_t refine;            // 1: a coarse plan of long blocks is made again for twice as many slots
   int32_t max_items;         // capacity of `entries` for work items
   int32_t max_len;           // longest sequence the block table can describe
   int32_t* counts;           // [plan_layout::kCountInts]: num_items, num_combine, num_empty, chunk_target, overflow
@@ -148,70 +147,42 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
   base = (base + A - 1) / A * A;
   if (base < p.min_chunk) base = p.min_chunk;
 
-  // ---- per sequence: degree, chunk length, chunk count
-  for (int b = tid; b < B; b += kDevPlanThreads) {
-    const long long len = max(p.seq_lens[b], 0);
-    int bucket = -1, n = 0, c = 0;
-    if (len > 0) {
-      long long deg = 1;
-      const long long want = (len + base - 1) / base;
-      while (deg < want) deg <<= 1;
-      if (base < plan_layout::kSmallBaseTokens && deg > 1 &&
-          len * plan_layout::kGeoMeanDen < (deg / 2) * base * plan_layout::kGeoMeanNum) {
-        deg >>= 1;   // short chunks: the nearer power of two
-      }
-      if (deg > p.max_splits) deg = p.max_splits;
-      const long long ch = ((len + deg - 1) / deg + A - 1) / A * A;
-      n = int((len + ch - 1) / ch);
-      c = int(ch);
-      bucket = 0;
-      while ((1ll << bucket) < deg) ++bucket;
-    }
-    nsplit[b] = n;
-    chunk[b] = c;
-    offs[b] = n;
-    p.per_seq[b] = bucket;
-  }
-  __syncthreads();
-  int n_items = dev::block_exclusive_scan(offs, B, warp_tot);
-
-  // ---- wave fill: the free slots of the last wave become extra chunks of the sequences with the longest chunks
-  {
-    const long long blocks = (long long)p.heads * n_items;
-    const long long waves = (blocks + p.wave_slots - 1) / p.wave_slots;
-    const long long spare = (waves >= 1 && waves <= p.wave_fill) ? (waves * p.wave_slots - blocks) / p.heads : 0;
-    if (spare > 0) {   // the same for every thread
-      int* new_n = it_len;   // not in use yet
-      int* new_c = it_b;
-      for (int b = tid; b < B; b += kDevPlanThreads) {
-        int n = nsplit[b], c = chunk[b];
-        if (n > 0) {
-          long long rank = 0;   // sequences before this one in (chunk desc, index asc) order
-          for (int k = 0; k < B; ++k) {
-            const int ck = chunk[k];
-            rank += (nsplit[k] > 0 && (ck > c || (ck == c && k < b))) ? 1 : 0;
-          }
-          if (rank < spare) {
-            const long long len = p.seq_lens[b];
-            const long long ch = ((len + n) / (n + 1) + A - 1) / A * A;
-            if (ch >= p.min_chunk && n + 1 <= p.max_splits) {
-              c = int(ch);
-              n = int((len + ch - 1) / ch);
-            }
-          }
+  // ---- per sequence: degree, chunk length, chunk count; twice if the first plan is coarse
+  int n_items = 0;
+  for (int pass = 0; pass < 2; ++pass) {
+    for (int b = tid; b < B; b += kDevPlanThreads) {
+      const long long len = max(p.seq_lens[b], 0);
+      int bucket = -1, n = 0, c = 0;
+      if (len > 0) {
+        long long deg = 1;
+        const long long want = (len + base - 1) / base;
+        while (deg < want) deg <<= 1;
+        if (base < plan_layout::kSmallBaseTokens && deg > 1 &&
+            len * plan_layout::kGeoMeanDen < (deg / 2) * base * plan_layout::kGeoMeanNum) {
+          deg >>= 1;   // short chunks: the nearer power of two
         }
-        new_n[b] = n;
-        new_c[b] = c;
+        if (deg > p.max_splits) deg = p.max_splits;
+        const long long ch = ((len + deg - 1) / deg + A - 1) / A * A;
+        n = int((len + ch - 1) / ch);
+        c = int(ch);
+        bucket = 0;
+        while ((1ll << bucket) < deg) ++bucket;
       }
-      __syncthreads();
-      for (int b = tid; b < B; b += kDevPlanThreads) {
-        nsplit[b] = new_n[b];
-        chunk[b] = new_c[b];
-        offs[b] = new_n[b];
-      }
-      __syncthreads();
-      n_items = dev::block_exclusive_scan(offs, B, warp_tot);
+      nsplit[b] = n;
+      chunk[b] = c;
+      offs[b] = n;
+      p.per_seq[b] = bucket;
     }
+    __syncthreads();
+    n_items = dev::block_exclusive_scan(offs, B, warp_tot);
+    // fewer than one and a half waves of long blocks: once more, for twice as many slots (the same for every thread)
+    if (pass == 1 || !p.refine || base < plan_layout::kRefineMinBaseTokens ||
+        (long long)plan_layout::kRefineWavesDen * p.heads * n_items >= plan_layout::kRefineWavesNum * p.wave_slots) {
+      break;
+    }
+    base = (p.heads * T + 2 * p.slots - 1) / (2 * p.slots);
+    base = (base + A - 1) / A * A;
+    if (base < p.min_chunk) base = p.min_chunk;
   }
   for (int b = tid; b < B; b += kDevPlanThreads) {
     p.per_seq[B + b] = nsplit[b];

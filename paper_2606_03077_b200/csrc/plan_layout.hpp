@@ -31,6 +31,13 @@ constexpr int kParamFixEntries = 256;
 // the better one).
 constexpr int kSmallBaseTokens = 4096;
 constexpr int kGeoMeanNum = 181, kGeoMeanDen = 128;
+// A plan with fewer than kRefineWavesNum / kRefineWavesDen waves of blocks whose base chunk is at least
+// kRefineMinBaseTokens long is made again for twice as many slots (both planners).  Few long blocks leave most SMs idle
+// through the last wave, and the blocks that do run cannot pull the memory bandwidth alone: 12 sequences of 20,000
+// tokens 169 -> 147 us, 26 sequences of 16K - 32K tokens 420 -> 389 us, 3 of 40,000 89 -> 79 us; batches of 1.5 waves
+// and more lose 1 - 3 % when cut finer, and on short bases the fixed cost of a block dominates.
+constexpr int kRefineWavesNum = 3, kRefineWavesDen = 2;
+constexpr int kRefineMinBaseTokens = 4096;
 // counts written by the device-side planner (int32 words at the start of the workspace's plan region)
 constexpr int kCountInts = 8;
 constexpr int kCntItems = 0;

@@ -25,12 +25,12 @@ bool valid_params(const PlanParams& p) {
   if (p.chunk_align <= 0 || p.chunk_align % 16 != 0) return false;
   if (p.min_chunk <= 0) return false;
   if (p.max_splits <= 0 || p.max_splits > 64 || (p.max_splits & (p.max_splits - 1)) != 0) return false;
-  if (p.wave_fill < 0 || p.wave_fill > 2) return false;   // max_items() covers two waves
+  if (p.refine != 0 && p.refine != 1) return false;
   return true;
 }
 
 int64_t max_items(const PlanParams& p, int32_t num_kv_heads, int32_t max_batch) {
-  const int64_t slots = int64_t(p.n_sm) * p.ctas_per_sm * p.items_per_slot;
+  const int64_t slots = int64_t(p.n_sm) * p.ctas_per_sm * p.items_per_slot * (p.refine ? 2 : 1);
   return 2 * ceil_div(slots, num_kv_heads) + max_batch;
 }
 
@@ -42,11 +42,10 @@ bool make_plan(const PlanParams& p, int32_t num_kv_heads, const int32_t* seq_len
     total += seq_lens[b];
   }
   const int64_t slots = int64_t(p.n_sm) * p.ctas_per_sm * p.items_per_slot;
-  const int64_t base = std::max<int64_t>(p.min_chunk, round_up(ceil_div(int64_t(num_kv_heads) * total, slots), p.chunk_align));
+  int64_t base = std::max<int64_t>(p.min_chunk, round_up(ceil_div(int64_t(num_kv_heads) * total, slots), p.chunk_align));
 
   HostPlan& pl = *out;
   pl.batch = batch;
-  pl.chunk_target = int32_t(base);
   pl.bucket.assign(batch, -1);
   pl.num_splits.assign(batch, 0);
   pl.chunk_len.assign(batch, 0);
@@ -55,48 +54,38 @@ bool make_plan(const PlanParams& p, int32_t num_kv_heads, const int32_t* seq_len
   pl.combine.clear();
   pl.empty.clear();
 
-  for (int32_t b = 0; b < batch; ++b) {
-    const int64_t len = seq_lens[b];
-    if (len == 0) continue;
-    int64_t degree = next_pow2(ceil_div(len, base));
-    if (base < plan_layout::kSmallBaseTokens && degree > 1 &&
-        len * plan_layout::kGeoMeanDen < (degree / 2) * base * plan_layout::kGeoMeanNum) {
-      degree /= 2;   // short chunks: the nearer power of two, see plan_layout.hpp
-    }
-    degree = std::min<int64_t>(degree, p.max_splits);
-    const int64_t chunk = round_up(ceil_div(len, degree), p.chunk_align);
-    const int64_t pieces = ceil_div(len, chunk);
-    pl.bucket[b] = log2_exact(degree);
-    pl.chunk_len[b] = int32_t(chunk);
-    pl.num_splits[b] = int32_t(pieces);
-  }
-
-  // Wave fill.  The launch is `blocks` thread blocks on `wave` resident ones.  When that is at most wave_fill waves,
-  // the slots the last wave leaves free are handed out as extra chunks, one each to the sequences with the longest
-  // chunks (ties: lower index first): a few equally long sequences otherwise run one full wave and one part-empty
-  // wave of equally long blocks.  The bucket of a sequence (its length class) stays.
-  const int64_t wave = int64_t(p.n_sm) * p.ctas_per_sm;
-  int64_t blocks = 0;
-  for (int32_t b = 0; b < batch; ++b) blocks += int64_t(num_kv_heads) * pl.num_splits[b];
-  const int64_t waves = ceil_div(blocks, wave);
-  if (waves >= 1 && waves <= p.wave_fill) {
-    const int64_t spare = (waves * wave - blocks) / num_kv_heads;
-    std::vector<int32_t> order;
-    for (int32_t b = 0; b < batch; ++b)
-      if (seq_lens[b] > 0) order.push_back(b);
-    const size_t take = size_t(std::min<int64_t>(spare, int64_t(order.size())));
-    std::partial_sort(order.begin(), order.begin() + take, order.end(), [&](int32_t x, int32_t y) {
-      return pl.chunk_len[x] != pl.chunk_len[y] ? pl.chunk_len[x] > pl.chunk_len[y] : x < y;
-    });
-    for (size_t i = 0; i < take; ++i) {
-      const int32_t b = order[i];
+  // buckets for a base length; returns the number of work items
+  auto bucket_all = [&](int64_t base_len) -> int64_t {
+    int64_t n_items = 0;
+    for (int32_t b = 0; b < batch; ++b) {
       const int64_t len = seq_lens[b];
-      const int64_t chunk = round_up(ceil_div(len, int64_t(pl.num_splits[b]) + 1), p.chunk_align);
-      if (chunk < p.min_chunk || pl.num_splits[b] + 1 > p.max_splits) continue;
+      if (len == 0) continue;
+      int64_t degree = next_pow2(ceil_div(len, base_len));
+      if (base_len < plan_layout::kSmallBaseTokens && degree > 1 &&
+          len * plan_layout::kGeoMeanDen < (degree / 2) * base_len * plan_layout::kGeoMeanNum) {
+        degree /= 2;   // short chunks: the nearer power of two, see plan_layout.hpp
+      }
+      degree = std::min<int64_t>(degree, p.max_splits);
+      const int64_t chunk = round_up(ceil_div(len, degree), p.chunk_align);
+      const int64_t pieces = ceil_div(len, chunk);
+      pl.bucket[b] = log2_exact(degree);
       pl.chunk_len[b] = int32_t(chunk);
-      pl.num_splits[b] = int32_t(ceil_div(len, chunk));
+      pl.num_splits[b] = int32_t(pieces);
+      n_items += pieces;
     }
+    return n_items;
+  };
+  const int64_t n_items = bucket_all(base);
+  // A coarse plan of long blocks - fewer than one and a half waves of the resident blocks - is made again for twice
+  // as many slots: with so few blocks most SMs idle through the second wave and the rest cannot pull the memory
+  // bandwidth alone (plan_layout.hpp).
+  const int64_t wave = int64_t(p.n_sm) * p.ctas_per_sm;
+  if (p.refine && base >= plan_layout::kRefineMinBaseTokens &&
+      plan_layout::kRefineWavesDen * num_kv_heads * n_items < plan_layout::kRefineWavesNum * wave) {
+    base = std::max<int64_t>(p.min_chunk, round_up(ceil_div(int64_t(num_kv_heads) * total, 2 * slots), p.chunk_align));
+    bucket_all(base);
   }
+  pl.chunk_target = int32_t(base);
 
   int32_t running = 0;
   for (int32_t b = 0; b < batch; ++b) {

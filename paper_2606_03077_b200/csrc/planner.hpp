@@ -18,7 +18,7 @@ struct PlanParams {
   int32_t chunk_align = 256;
   int32_t min_chunk = 512;
   int32_t max_splits = 64;
-  int32_t wave_fill = 2;   // launches of at most this many waves get their last wave filled (0 = never)
+  int32_t refine = 1;      // 1: a plan of fewer than 1.5 waves of long blocks is made again twice as fine (0 = never)
 };
 
 struct WorkItem {  // one (sequence, chunk) unit; the decode grid is items x KV heads
@@ -38,9 +38,8 @@ bool valid_params(const PlanParams& p);
 bool make_plan(const PlanParams& p, int32_t num_kv_heads, const int32_t* seq_lens, int32_t batch, HostPlan* out);
 
 // Upper bound of the number of work items for any batch <= max_batch:
-// n_b <= 2*cd(L_b, C) - 1 and C >= num_kv_heads*T/(W*items_per_slot) give sum n_b <= 2*cd(W*ips, Hkv) + B.
-// The wave fill only adds items while the launch stays within wave_fill * W blocks, i.e. within
-// wave_fill * W / Hkv items, which the bound covers for wave_fill <= 2.
+// n_b <= 2*cd(L_b, C) - 1 and C >= num_kv_heads*T/(W*items_per_slot) give sum n_b <= 2*cd(W*ips, Hkv) + B;
+// a refined plan is a plan for twice as many slots, so with `refine` the bound is taken for 2*W*ips.
 int64_t max_items(const PlanParams& p, int32_t num_kv_heads, int32_t max_batch);
 
 }  // namespace libra

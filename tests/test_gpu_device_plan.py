@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 def ref_params(h):
     p = h.plan_params()
     return P.PlanParams(p.n_sm, p.ctas_per_sm, p.items_per_slot, p.chunk_align, p.min_chunk, p.max_splits,
-                        wave_fill=max(p.wave_fill, 0))
+                        refine=1 if p.refine > 0 else 0)
 
 
 def assert_same_plan(got, ref):
@@ -78,14 +78,15 @@ def test_random_and_edge_vectors_bit_exact(lib):
         h.close()
 
 
-def test_few_waves_bit_exact(lib):
-    """Small batches of long sequences: launches of one or two waves, where the planner hands the free slots of the
-    last wave out as extra chunks (and ties between equal chunks go to the lower index)."""
+def test_few_long_sequences_bit_exact(lib):
+    """Small batches of long sequences: plans of fewer than one and a half waves of long blocks, which the planner
+    makes again for twice as many slots."""
+    import dataclasses
     rng = np.random.default_rng(12)
-    filled = 0
-    for i in range(60):
+    refined = 0
+    for i in range(120):
         B = int(rng.integers(1, 40))
-        base = int(rng.choice([600, 3000, 12000, 30000]))
+        base = int(rng.choice([3000, 12000, 20000, 30000]))
         lens = (np.full(B, base) if i % 3 == 0 else
                 np.clip(np.floor(base * np.exp(rng.normal(size=B) * rng.uniform(0.05, 0.8))), 0, 40960)).astype(np.int32)
         if i % 5 == 0:
@@ -93,16 +94,15 @@ def test_few_waves_bit_exact(lib):
         hkv = int(rng.choice([1, 2, 4, 8]))
         plan = lib.PlanParams(int(rng.choice([16, 74, 148])), int(rng.integers(1, 3)), int(rng.integers(1, 3)),
                               int(rng.choice([16, 256])), int(rng.choice([16, 512])), int(rng.choice([2, 8, 64])),
-                              int(rng.choice([0, 1, 2, -1])))
-        h, ws, dl = device_plan(lib, lens, hkv, plan)
+                              int(rng.choice([0, 1, -1])))
+        h, ws, dl = device_plan(lib, lens, hkv, plan, ld=40960 // 16)
         prm = ref_params(h)
         ref = P.plan(lens, hkv, prm)
         assert_same_plan(h.plan_export(), ref)
         assert h.debug_error_word() == 0
-        import dataclasses
-        filled += ref.num_splits != P.plan(lens, hkv, dataclasses.replace(prm, wave_fill=0)).num_splits
+        refined += ref != P.plan(lens, hkv, dataclasses.replace(prm, refine=0))
         h.close()
-    assert filled > 10
+    assert refined > 3
 
 
 def test_overflow_is_flagged_and_nothing_runs(lib):
@@ -218,7 +218,8 @@ def test_separate_combine_with_nothing_to_merge_keeps_the_chain_ordered(lib):
     dl = torch.from_numpy(lens_a.copy()).to(dev)
     results = []
     for mode in (1, 0):
-        r = H.Runner(lib, Hq, Hkv, d, k.shape[0], len(lens), bt.shape[1], variant=(8, 3), fused=mode)
+        r = H.Runner(lib, Hq, Hkv, d, k.shape[0], len(lens), bt.shape[1], variant=(8, 3), fused=mode,
+                     plan=lib.PlanParams(0, 0, 0, 0, 0, 0, -1))   # the plain plan: every sequence stays in one piece
         st = torch.cuda.current_stream().cuda_stream
         bufs = [dq.clone(), torch.zeros_like(dq)]
         r.h.plan_device(dl.data_ptr(), len(lens), r.ws.data_ptr(), r.ws.numel(), st)

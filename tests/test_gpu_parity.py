@@ -321,7 +321,7 @@ def test_plan_export_matches_reference(lib):
     h.plan(lay.seq_lens, ws.data_ptr(), ws.numel(), torch.cuda.current_stream().cuda_stream)
     got = h.plan_export()
     ref = P.plan(lay.seq_lens, 8, P.PlanParams(prm.n_sm, prm.ctas_per_sm, prm.items_per_slot, prm.chunk_align,
-                                               prm.min_chunk, prm.max_splits, wave_fill=max(prm.wave_fill, 0)))
+                                               prm.min_chunk, prm.max_splits, refine=1 if prm.refine > 0 else 0))
     assert got["chunk_target"] == ref.chunk_target and [tuple(r) for r in got["items"]] == ref.items
     assert list(got["num_splits"]) == ref.num_splits and list(got["item_offset"]) == ref.item_offset
     assert list(got["combine"]) == ref.combine

@@ -11,7 +11,7 @@ def both(lib, lens, hkv, prm: P.PlanParams):
     ref = P.plan(lens, hkv, prm)
     got = lib.libra_plan_host(lens, hkv, lib.PlanParams(prm.n_sm, prm.ctas_per_sm, prm.items_per_slot,
                                                         prm.chunk_align, prm.min_chunk, prm.max_splits,
-                                                        prm.wave_fill if prm.wave_fill > 0 else -1))
+                                                        1 if prm.refine else -1))
     assert got["chunk_target"] == ref.chunk_target
     assert list(got["bucket"]) == ref.bucket
     assert list(got["num_splits"]) == ref.num_splits
@@ -43,26 +43,27 @@ def test_random_vectors_bit_exact(lib):
         both(lib, lens, int(rng.choice([1, 2, 4, 8])), prm)
 
 
-def test_few_waves_bit_exact(lib):
-    """Small batches on many slots: launches of one or two waves, where the wave fill hands out extra chunks."""
+def test_few_long_sequences_bit_exact(lib):
+    """Small batches of long sequences on many slots: plans of fewer than one and a half waves, which are made again
+    for twice as many slots."""
+    import dataclasses
     rng = np.random.default_rng(6)
-    filled = 0
+    refined = 0
     for i in range(400):
         B = int(rng.integers(1, 40))
-        base = int(rng.choice([600, 3000, 12000, 30000]))
+        base = int(rng.choice([3000, 12000, 20000, 30000]))
         if i % 3 == 0:
-            lens = np.full(B, base, dtype=np.int32)                    # equal lengths: ties broken by index
+            lens = np.full(B, base, dtype=np.int32)
         else:
             lens = np.clip(np.floor(base * np.exp(rng.normal(size=B) * rng.uniform(0.05, 0.8))), 0, 40960).astype(np.int32)
         hkv = int(rng.choice([1, 2, 4, 8]))
-        for wf in (2, 1, 0):
+        for rf in (1, 0):
             prm = P.PlanParams(n_sm=int(rng.choice([16, 74, 148, 296])), ctas_per_sm=int(rng.integers(1, 3)),
                                items_per_slot=int(rng.integers(1, 3)), chunk_align=int(rng.choice([16, 256])),
-                               min_chunk=int(rng.choice([16, 512])), max_splits=int(rng.choice([2, 8, 64])), wave_fill=wf)
+                               min_chunk=int(rng.choice([16, 512])), max_splits=int(rng.choice([2, 8, 64])), refine=rf)
             ref = both(lib, lens, hkv, prm)
-            import dataclasses
-            filled += ref.num_splits != P.plan(lens, hkv, dataclasses.replace(prm, wave_fill=0)).num_splits
-    assert filled > 100   # the cases did exercise the rule
+            refined += ref != P.plan(lens, hkv, dataclasses.replace(prm, refine=0))
+    assert refined > 30   # the cases did exercise the rule
 
 
 def test_edge_cases(lib):

@@ -23,7 +23,7 @@ def check_plan(lens, hkv, params):
             assert pl.num_splits[b] == 0 and pl.bucket[b] == -1 and pl.chunk_len[b] == 0
             continue
         s = 1 << pl.bucket[b]
-        assert s <= params.max_splits and 1 <= pl.num_splits[b] <= min(s + 1, params.max_splits)   # + 1: wave fill
+        assert 1 <= pl.num_splits[b] <= s <= params.max_splits
         assert pl.chunk_len[b] % A == 0 and pl.chunk_len[b] % 16 == 0
         # bucket bins: (C 2^(k-1), C 2^k], except that the top bucket is open-ended; with a short base chunk the
         # limits sit at the geometric means instead: [C 2^(k-1) * 181/128, C 2^k * 181/128)
@@ -57,33 +57,22 @@ def check_plan(lens, hkv, params):
     order = np.argsort(lens, kind="stable")
     bk = [pl.bucket[i] for i in order]
     assert bk == sorted(bk)
-    check_wave_fill(lens, hkv, params, pl)
+    check_refine(lens, hkv, params, pl)
     return pl
 
 
-def check_wave_fill(lens, hkv, params, pl):
-    """What the wave fill may and may not do, against the same rule without it."""
+def check_refine(lens, hkv, params, pl):
+    """The second pass: made exactly when the first plan is coarse (fewer than 1.5 waves) on a long base, and then it is
+    the plain plan for twice as many slots."""
     import dataclasses
-    pl0 = P.plan(lens, hkv, dataclasses.replace(params, wave_fill=0))
+    pl0 = P.plan(lens, hkv, dataclasses.replace(params, refine=0))
     W_ = params.n_sm * params.ctas_per_sm
-    U0 = hkv * sum(pl0.num_splits)
-    k = P.cd(U0, W_)
-    assert pl.chunk_target == pl0.chunk_target and pl.bucket == pl0.bucket
-    if not (1 <= k <= params.wave_fill):
+    coarse = pl0.chunk_target >= 4096 and 2 * hkv * len(pl0.items) < 3 * W_
+    if not (params.refine and coarse):
         assert pl == pl0
         return
-    spare = (k * W_ - U0) // hkv
-    assert hkv * sum(pl.num_splits) <= k * W_             # the launch does not grow into another wave
-    changed = [b for b in range(len(lens)) if (pl.num_splits[b], pl.chunk_len[b]) != (pl0.num_splits[b], pl0.chunk_len[b])]
-    first = sorted((b for b in range(len(lens)) if lens[b] > 0), key=lambda b: (-pl0.chunk_len[b], b))[:spare]
-    assert set(changed) <= set(first)                     # only the sequences with the longest chunks
-    for b in first:
-        c = P.au(P.cd(lens[b], pl0.num_splits[b] + 1), params.chunk_align)
-        if b in changed:
-            assert c >= params.min_chunk and c < pl0.chunk_len[b] and pl0.num_splits[b] < params.max_splits
-            assert pl.chunk_len[b] == c and pl.num_splits[b] == P.cd(lens[b], c)
-        else:   # left alone: the shorter chunk is not allowed, or rounding made it the same chunk
-            assert c < params.min_chunk or pl0.num_splits[b] >= params.max_splits or c == pl0.chunk_len[b]
+    twice = P.plan(lens, hkv, dataclasses.replace(params, refine=0, items_per_slot=2 * params.items_per_slot))
+    assert pl == twice and pl.chunk_target <= pl0.chunk_target and len(pl.items) >= len(pl0.items)
 
 
 def test_exhaustive_small_vectors():
@@ -147,42 +136,42 @@ def test_straggler_split_follows_the_base_chunk():
     # 8 x 148 slots: base 1792 tokens, 32768 / 1792 = 18.3 is nearer to 16 than to 32 and the base is short: 16 ways
     pl = P.plan(lay.seq_lens, 8, P.PlanParams(ctas_per_sm=2, items_per_slot=4))
     assert pl.chunk_target == 1792 and set(pl.bucket) == {4} and set(pl.chunk_len) == {2048} and set(pl.num_splits) == {16}
-    # 148 slots: base 14336 tokens, long chunks keep the least power of two above 32768 / 14336 = 2.3: 4 ways
-    pl = P.plan(lay.seq_lens, 8, P.PlanParams(wave_fill=0))
-    assert pl.chunk_target == 14336 and set(pl.bucket) == {2} and set(pl.chunk_len) == {8192} and set(pl.num_splits) == {4}
-    # that is 8 * 4 * 8 = 256 blocks on 148 slots: 1.73 waves.  The 40 free slots of the second wave are 5 work items:
-    # the first five sequences are cut 5 ways, chunk au(cd(32768, 5), 256) = 6656 -> 37 items = 296 blocks = 2 full waves
+    # 148 slots: base 14336 tokens, long chunks keep the least power of two above 32768 / 14336 = 2.3: 4 ways;
+    # 8 * 4 * 8 = 256 blocks are 1.73 waves, not fewer than 1.5: the plan stands
     pl = P.plan(lay.seq_lens, 8, P.PlanParams())
-    assert pl.chunk_target == 14336 and set(pl.bucket) == {2}
-    assert pl.num_splits == [5] * 5 + [4] * 3 and pl.chunk_len == [6656] * 5 + [8192] * 3
-    assert len(pl.items) * 8 == 2 * 148
-    assert [it[3] - it[2] for it in pl.items] == [8192] * 12 + [6656] * 20 + [6144] * 5
+    assert pl.chunk_target == 14336 and set(pl.bucket) == {2} and set(pl.chunk_len) == {8192} and set(pl.num_splits) == {4}
 
 
-def test_wave_fill_hand_worked():
-    # one wave: 4 slots, one KV head, A = 16, C_min = 16.  T = 288, C = au(cd(288, 4), 16) = 80; every 96 is one chunk
-    # (cd(96, 80) = 2 -> p2 = 2, but C is short and 96 * 128 = 12288 < 1 * 80 * 181 = 14480: 1).  3 blocks on 4 slots:
-    # 1 free slot -> the first sequence (equal chunks: lowest index) is cut in two, chunk au(cd(96, 2), 16) = 48
-    prm = P.PlanParams(n_sm=4, ctas_per_sm=1, items_per_slot=1, chunk_align=16, min_chunk=16, max_splits=8)
-    pl = P.plan([96, 96, 96], 1, prm)
-    assert pl.chunk_target == 80 and pl.bucket == [0, 0, 0]
-    assert pl.num_splits == [2, 1, 1] and pl.chunk_len == [48, 96, 96] and pl.item_offset == [0, 2, 3]
-    assert pl.items == [(1, 0, 0, 96), (2, 0, 0, 96), (0, 0, 0, 48), (0, 1, 48, 96)] and pl.combine == [0]
-    # two waves: 3 slots, four sequences of 64.  T = 256, C = au(cd(256, 3), 16) = 96, one chunk each: 4 blocks = 2 waves
-    # with 2 free slots -> sequences 0 and 1 are cut in two (chunk 32)
-    prm = P.PlanParams(n_sm=3, ctas_per_sm=1, items_per_slot=1, chunk_align=16, min_chunk=16, max_splits=8)
-    pl = P.plan([64, 64, 64, 64], 1, prm)
-    assert pl.chunk_target == 96 and pl.num_splits == [2, 2, 1, 1] and pl.chunk_len == [32, 32, 64, 64]
-    assert pl.items == [(2, 0, 0, 64), (3, 0, 0, 64), (0, 0, 0, 32), (0, 1, 32, 64), (1, 0, 0, 32), (1, 1, 32, 64)]
-    # two KV heads: every work item is two blocks.  [64] * 4 on 5 slots: T = 256, C = au(cd(512, 5), 16) = 112; 8 blocks
-    # = 2 waves of 5 with 2 free slots = 1 item -> only sequence 0 is cut
-    prm = P.PlanParams(n_sm=5, ctas_per_sm=1, items_per_slot=1, chunk_align=16, min_chunk=16, max_splits=8)
-    pl = P.plan([64, 64, 64, 64], 2, prm)
-    assert pl.chunk_target == 112 and pl.num_splits == [2, 1, 1, 1] and pl.chunk_len == [32, 64, 64, 64]
-    # three waves and more: left alone (wave_fill = 2)
-    prm = P.PlanParams(n_sm=2, ctas_per_sm=1, items_per_slot=1, chunk_align=16, min_chunk=16, max_splits=8)
-    pl = P.plan([64, 64, 64, 64, 64], 1, prm)
-    assert pl.num_splits == [1] * 5
-    # a chunk below C_min is not made: 1 wave of 4 slots, lengths 16: nothing to cut
-    prm = P.PlanParams(n_sm=4, ctas_per_sm=1, items_per_slot=1, chunk_align=16, min_chunk=16, max_splits=8)
-    assert P.plan([16, 16], 1, prm).num_splits == [1, 1]
+def test_coarse_plans_are_cut_finer_hand_worked():
+    # 12 sequences of 20,000 tokens, 8 KV heads, 148 slots.  T = 240,000; C = au(cd(1,920,000, 148), 256) = au(12973, 256)
+    # = 13056; cd(20000, 13056) = 2 -> 2 chunks of au(10000, 256) = 10240: 24 items = 192 blocks, and 2 * 192 = 384 < 3 * 148
+    # = 444: fewer than one and a half waves, on a base >= 4096 -> again for 296 slots: C = au(cd(1,920,000, 296), 256) =
+    # au(6487, 256) = 6656; cd(20000, 6656) = 4 -> 4 chunks of au(5000, 256) = 5120: 48 items = 384 blocks
+    pl = P.plan([20000] * 12, 8, P.PlanParams())
+    assert pl.chunk_target == 6656 and pl.bucket == [2] * 12 and pl.num_splits == [4] * 12 and pl.chunk_len == [5120] * 12
+    assert [it[3] - it[2] for it in pl.items] == [5120] * 36 + [4640] * 12
+    plain = P.plan([20000] * 12, 8, P.PlanParams(refine=0))
+    assert plain.chunk_target == 13056 and plain.num_splits == [2] * 12 and plain.chunk_len == [10240] * 12
+    # 3 sequences of 40,000: C = au(cd(960,000, 148), 256) = 6656, 8 chunks of 5120 each: 24 items = 192 blocks -> again:
+    # C = au(cd(960,000, 296), 256) = au(3244, 256) = 3328, now a short base: cd(40000, 3328) = 13 -> 16, and 40000 * 128 =
+    # 5,120,000 >= 8 * 3328 * 181 = 4,818,944 keeps 16: chunks of au(2500, 256) = 2560, 16 each
+    pl = P.plan([40000] * 3, 8, P.PlanParams())
+    assert pl.chunk_target == 3328 and pl.num_splits == [16] * 3 and pl.chunk_len == [2560] * 3
+    # a short base is never cut finer: 2 sequences of 3000 on 148 slots (C = 512, 8 heads): 2 * 8 * 2 * ... stays
+    pl = P.plan([3000, 3000], 8, P.PlanParams())
+    assert pl.chunk_target == 512 and pl == P.plan([3000, 3000], 8, P.PlanParams(refine=0))
+    # one and a half waves or more stand: 28 x 20000 -> C = au(cd(4,480,000, 148), 256) = 30464, one chunk each:
+    # 28 * 8 = 224 blocks, 448 >= 444
+    pl = P.plan([20000] * 28, 8, P.PlanParams())
+    assert pl.chunk_target == 30464 and pl.num_splits == [1] * 28
+    # 27 x 20000 -> 216 blocks, 432 < 444: cut
+    pl = P.plan([20000] * 27, 8, P.PlanParams())
+    assert pl.chunk_target == au_ref(cd_ref(27 * 20000 * 8, 296), 256) and pl.num_splits == [2] * 27
+
+
+def cd_ref(a, b):
+    return (a + b - 1) // b
+
+
+def au_ref(a, b):
+    return cd_ref(a, b) * b

@@ -23,7 +23,7 @@ def test_static_scratch_entry_point_matches_workspace_path(lib):
     lens = [5000, 1300, 0, 37, 2049]
     Hq, Hkv, d = 32, 8, 128
     lens_a, bt, q, k, v = W.random_case(41, len(lens), Hq, Hkv, d, lens)
-    plan = lib.PlanParams(0, 2, 4, 256, 512, 64)     # several split sequences: partial results go through the scratch
+    plan = lib.PlanParams(0, 1, 4, 256, 512, 64)     # several split sequences: partial results go through the scratch
     r = H.Runner(lib, Hq, Hkv, d, k.shape[0], len(lens), bt.shape[1], plan=plan, fused=0)   # decode + combine kernels
     assert r.h.workspace_size() <= lib.STATIC_SCRATCH_BYTES
     dq, dk, dv, dbt = (H.to_dev(x, dev) for x in (q, k, v, bt))
@@ -66,7 +66,7 @@ def test_two_handles_take_turns_on_the_shared_region(lib):
     cases = []
     for seed, (Hq, Hkv, d, lens) in enumerate([(32, 8, 128, [5000, 1300, 0, 37, 2049]), (8, 2, 64, [3000, 16, 900, 4100])]):
         lens_a, bt, q, k, v = W.random_case(60 + seed, len(lens), Hq, Hkv, d, lens)
-        r = H.Runner(lib, Hq, Hkv, d, k.shape[0], len(lens), bt.shape[1], plan=lib.PlanParams(0, 2, 4, 256, 512, 64))
+        r = H.Runner(lib, Hq, Hkv, d, k.shape[0], len(lens), bt.shape[1], plan=lib.PlanParams(0, 1, 4, 256, 512, 64))
         dq, dk, dv, dbt = (H.to_dev(x, dev) for x in (q, k, v, bt))
         want = H.bf16_dev_to_f32(r.run(dq, dk, dv, dbt, lens_a))
         assert len(r.h.plan_export()["combine"]) >= 1
