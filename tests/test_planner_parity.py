@@ -94,12 +94,13 @@ def test_bad_arguments(lib):
 
 
 def test_item_bound_holds(lib):
-    # sum n_b <= 2*ceil(W*ips / Hkv) + B, the bound the workspace is sized by
+    # sum n_b <= 2*ceil(W*ips / Hkv) + B, the bound the workspace is sized by; a refined plan is a plan for twice the slots
     rng = np.random.default_rng(6)
-    for _ in range(200):
-        B = int(rng.integers(1, 257)); hkv = int(rng.choice([1, 2, 8]))
+    for i in range(300):
+        B = int(rng.integers(1, 257 if i % 2 else 12)); hkv = int(rng.choice([1, 2, 8]))
         lens = rng.integers(0, 40961, B).astype(np.int32)
-        prm = P.PlanParams(n_sm=int(rng.choice([4, 148])), items_per_slot=int(rng.integers(1, 6)))
-        pl = P.plan(lens, hkv, prm)
-        W_ = prm.n_sm * prm.ctas_per_sm * prm.items_per_slot
-        assert len(pl.items) <= 2 * (-(-W_ // hkv)) + B
+        for refine in (0, 1):
+            prm = P.PlanParams(n_sm=int(rng.choice([4, 148])), items_per_slot=int(rng.integers(1, 6)), refine=refine)
+            pl = P.plan(lens, hkv, prm)
+            W_ = prm.n_sm * prm.ctas_per_sm * prm.items_per_slot * (2 if refine else 1)
+            assert len(pl.items) <= 2 * (-(-W_ // hkv)) + B
