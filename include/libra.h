@@ -497,6 +497,60 @@ int libra_ring_step(int32_t device, void* dst, const void* own, const void* rece
                     const uint32_t* ready_flag, uint32_t expected, uint32_t timeout_us, uint32_t* status_dev,
                     int32_t num_blocks, void* stream);
 
+/* ---- The ring's host side: membership descriptor and schedule (same passages of the paper) ---------------------
+ * libra_ring_t is the metadata the CPU control plane owns: the live replicas in ring order (members[i] sends to
+ * members[(i + 1) % n_members]).  A replica that died or leaves is taken out with libra_ring_remove - the order of
+ * the others stays, its neighbours become each other's neighbours - and one that joins is put in at any position
+ * with libra_ring_insert; both are plain edits of this struct (no GPU state, no allocation) and bump `epoch`, so a
+ * data plane can tell that its peer list is stale.  Ids are the caller's (any distinct int32 values).
+ * Errors: INVALID_ARGUMENT (null, duplicate or unknown id, position out of range, more than 64 members). */
+#define LIBRA_RING_MAX_MEMBERS 64
+typedef struct {
+  int32_t n_members;
+  int32_t members[LIBRA_RING_MAX_MEMBERS];   /* unused entries are -1 */
+  uint32_t epoch;                            /* number of edits since libra_ring_init */
+} libra_ring_t;
+int libra_ring_init(libra_ring_t* ring, const int32_t* ids, int32_t n);
+int libra_ring_remove(libra_ring_t* ring, int32_t id);
+int libra_ring_insert(libra_ring_t* ring, int32_t id, int32_t position);
+int libra_ring_neighbors(const libra_ring_t* ring, int32_t id, int32_t* predecessor, int32_t* successor);
+
+/* What member `id` does in one all-reduce of a vector of `bytes` bytes (a multiple of 16) over the ring as it stands:
+ * the ReduceScatter steps 0 .. n-2 followed by the AllGather steps 0 .. n-2, every step cut into pipeline pieces of
+ * at most piece_bytes (a multiple of 16; the paper pipelines 16 MB pieces).  The vector is cut into n segments of
+ * whole 16-byte units, equal parts with the first (bytes / 16) % n one unit longer; the member at ring position p
+ *   ReduceScatter step s : sends segment (p - s) mod n to its successor, adds what its predecessor sends into its
+ *                          own segment (p - 1 - s) mod n       (so segment c is summed starting at position c)
+ *   AllGather step s     : sends segment (p + 1 - s) mod n, overwrites its segment (p - s) mod n with what arrives.
+ * ops[] receives, in the order they are to be issued, one record per piece: kind, phase (0 ReduceScatter, 1
+ * AllGather), step, segment, piece index, the peer's id and the byte range [offset, offset + bytes) of the vector.
+ * A receive record is one libra_ring_step (dst = own = vector + offset for RECV_REDUCE, own = NULL for RECV_COPY).
+ * *n_ops = records needed; WORKSPACE_TOO_SMALL if capacity is less (the first `capacity` are written).  A ring of
+ * one member has no steps.  Errors: INVALID_ARGUMENT. */
+#define LIBRA_RING_OP_SEND 0
+#define LIBRA_RING_OP_RECV_REDUCE 1
+#define LIBRA_RING_OP_RECV_COPY 2
+typedef struct {
+  int32_t kind, phase, step, segment, piece, peer;
+  int64_t offset, bytes;
+} libra_ring_op_t;
+int libra_ring_schedule(const libra_ring_t* ring, int32_t id, int64_t bytes, int64_t piece_bytes, libra_ring_op_t* ops,
+                        int32_t capacity, int32_t* n_ops);
+
+/* The whole ReduceScatter + AllGather over n_members vectors that live on ONE device (bufs[i] = the vector of the
+ * member at ring position i, `bytes` each, 16-byte aligned), every receive record of every member's schedule enqueued
+ * on `stream` as one libra_ring_step, step by step: within a step no member reads a range that another member's
+ * record of the same step writes, so the launches of a step may run in any order.  This is the data plane of several
+ * replicas hosted on one GPU, and the way the schedule is exercised where there is one GPU; between real GPUs the
+ * same records are issued by each rank for itself, with the transport delivering `received` and setting the flag.
+ * ready_flag / expected / timeout_us / status_dev / num_blocks as for libra_ring_step (the same flag guards every
+ * step here; *status_dev holds the verdict of the last step).  Results are bit-identical to the ring's definition:
+ * segment c is summed in the order position c, c + 1, ..., in the element type.
+ * Errors: INVALID_ARGUMENT (also: n_members < 1 or > 64), CUDA_ERROR. */
+int libra_ring_all_reduce_local(int32_t device, void* const* bufs, int32_t n_members, size_t bytes, int32_t dtype,
+                                size_t piece_bytes, const uint32_t* ready_flag, uint32_t expected, uint32_t timeout_us,
+                                uint32_t* status_dev, int32_t num_blocks, void* stream);
+
 /* Merge of attention results over disjoint parts of the same sequences: the one exchange step of cutting a
  * sequence's TOKENS across GPUs (the paper's tensor parallelism cuts the cache by attention head, Section 5.3, and
  * needs none; this is the remaining way to shard the step).  Each holder of a part runs the decode call with

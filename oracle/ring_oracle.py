@@ -22,12 +22,16 @@ from __future__ import annotations
 import numpy as np
 
 
-def chunk_bounds(n: int, ranks: int) -> list[int]:
-    """Chunk c covers [bounds[c], bounds[c+1]): equal parts, the first n % ranks one element longer."""
-    base, extra = divmod(n, ranks)
+def chunk_bounds(n: int, ranks: int, granule: int = 1) -> list[int]:
+    """Chunk c covers [bounds[c], bounds[c+1]): equal parts, the first ones one unit longer.  The unit is `granule`
+    elements (1 by default; a transport that moves whole 16-byte vectors cuts at multiples of 16 bytes: granule 4
+    for float32, 8 for bfloat16); n must be a multiple of it.  The paper does not say where a vector is cut."""
+    if n % granule:
+        raise ValueError("vector length is not a multiple of the granule")
+    base, extra = divmod(n // granule, ranks)
     bounds = [0]
     for c in range(ranks):
-        bounds.append(bounds[-1] + base + (1 if c < extra else 0))
+        bounds.append(bounds[-1] + (base + (1 if c < extra else 0)) * granule)
     return bounds
 
 
@@ -47,11 +51,11 @@ def add_step(own: np.ndarray, received: np.ndarray, dtype: str) -> np.ndarray:
     raise ValueError(dtype)
 
 
-def ring_all_reduce(xs, dtype: str = "f32"):
+def ring_all_reduce(xs, dtype: str = "f32", granule: int = 1):
     """xs: list of R equal-length float32 arrays (for "bf16": exact bf16 values).  Returns the R result vectors."""
     R = len(xs)
     n = len(xs[0])
-    bounds = chunk_bounds(n, R)
+    bounds = chunk_bounds(n, R, granule)
     bufs = [np.array(x, dtype=np.float32, copy=True) for x in xs]
     sl = lambda c: slice(bounds[c % R], bounds[c % R + 1])
     for s in range(R - 1):                       # ReduceScatter

@@ -48,6 +48,20 @@ class PlanView(C.Structure):
                 ("empty", C.POINTER(C.c_int32))]
 
 
+RING_MAX_MEMBERS = 64
+RING_OP_SEND, RING_OP_RECV_REDUCE, RING_OP_RECV_COPY = 0, 1, 2
+
+
+class Ring(C.Structure):
+    """libra_ring_t: the live replicas in ring order (host metadata)."""
+    _fields_ = [("n_members", C.c_int32), ("members", C.c_int32 * RING_MAX_MEMBERS), ("epoch", C.c_uint32)]
+
+
+class RingOp(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("phase", C.c_int32), ("step", C.c_int32), ("segment", C.c_int32),
+                ("piece", C.c_int32), ("peer", C.c_int32), ("offset", C.c_int64), ("bytes", C.c_int64)]
+
+
 _i32p = C.POINTER(C.c_int32)
 _vp = C.c_void_p
 
@@ -70,6 +84,14 @@ SIGNATURES = {
     "libra_decode_attn_multi_append": (C.c_int, [_vp, _vp, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_ring_step": (C.c_int, [C.c_int32, _vp, _vp, _vp, C.c_size_t, C.c_int32, _vp, C.c_uint32, C.c_uint32, _vp, C.c_int32,
                                   _vp]),
+    "libra_ring_init": (C.c_int, [C.POINTER(Ring), _i32p, C.c_int32]),
+    "libra_ring_remove": (C.c_int, [C.POINTER(Ring), C.c_int32]),
+    "libra_ring_insert": (C.c_int, [C.POINTER(Ring), C.c_int32, C.c_int32]),
+    "libra_ring_neighbors": (C.c_int, [C.POINTER(Ring), C.c_int32, _i32p, _i32p]),
+    "libra_ring_schedule": (C.c_int, [C.POINTER(Ring), C.c_int32, C.c_int64, C.c_int64, C.POINTER(RingOp), C.c_int32,
+                                      _i32p]),
+    "libra_ring_all_reduce_local": (C.c_int, [C.c_int32, C.POINTER(_vp), C.c_int32, C.c_size_t, C.c_int32, C.c_size_t,
+                                              _vp, C.c_uint32, C.c_uint32, _vp, C.c_int32, _vp]),
     "libra_merge_parts": (C.c_int, [C.c_int32, _vp, _vp, C.c_int32, C.c_int64, C.c_int32, _vp, _vp, _vp]),
     "libra_debug_stream_read": (C.c_int, [_vp, _vp, C.c_size_t, _vp]),
     "libra_debug_gather_read": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -169,6 +191,48 @@ def libra_ring_step(device: int, dst_ptr: int, own_ptr: int, received_ptr: int, 
     """One copy / reduce step of the ring all-reduce's data plane (own_ptr = 0 for a copy step)."""
     _check(lib.libra_ring_step(device, dst_ptr, own_ptr or None, received_ptr, nbytes, dtype, ready_flag_ptr, expected,
                                timeout_us, status_ptr, num_blocks, stream), "libra_ring_step")
+
+
+def libra_ring_init(ids) -> Ring:
+    ring = Ring()
+    a = _as_i32(ids)
+    _check(lib.libra_ring_init(C.byref(ring), a.ctypes.data_as(_i32p), len(a)), "libra_ring_init")
+    return ring
+
+
+def libra_ring_remove(ring: Ring, member_id: int) -> None:
+    _check(lib.libra_ring_remove(C.byref(ring), member_id), "libra_ring_remove")
+
+
+def libra_ring_insert(ring: Ring, member_id: int, position: int) -> None:
+    _check(lib.libra_ring_insert(C.byref(ring), member_id, position), "libra_ring_insert")
+
+
+def libra_ring_neighbors(ring: Ring, member_id: int):
+    pred, succ = C.c_int32(0), C.c_int32(0)
+    _check(lib.libra_ring_neighbors(C.byref(ring), member_id, C.byref(pred), C.byref(succ)), "libra_ring_neighbors")
+    return pred.value, succ.value
+
+
+def libra_ring_schedule(ring: Ring, member_id: int, nbytes: int, piece_bytes: int):
+    """The member's records, in issue order, as dicts."""
+    n = C.c_int32(0)
+    st = lib.libra_ring_schedule(C.byref(ring), member_id, nbytes, piece_bytes, None, 0, C.byref(n))
+    if st not in (OK, WORKSPACE_TOO_SMALL):
+        _check(st, "libra_ring_schedule")
+    ops = (RingOp * max(1, n.value))()
+    _check(lib.libra_ring_schedule(C.byref(ring), member_id, nbytes, piece_bytes, ops, n.value, C.byref(n)),
+           "libra_ring_schedule")
+    return [{f: getattr(ops[i], f) for f, _ in RingOp._fields_} for i in range(n.value)]
+
+
+def libra_ring_all_reduce_local(device: int, buf_ptrs, nbytes: int, dtype: int, piece_bytes: int, ready_flag_ptr: int,
+                                expected: int, timeout_us: int, status_ptr: int, num_blocks: int, stream: int) -> None:
+    """ReduceScatter + AllGather over vectors on one device (buf_ptrs[i] = the member at ring position i)."""
+    arr = (_vp * len(buf_ptrs))(*buf_ptrs)
+    _check(lib.libra_ring_all_reduce_local(device, arr, len(buf_ptrs), nbytes, dtype, piece_bytes, ready_flag_ptr,
+                                           expected, timeout_us, status_ptr, num_blocks, stream),
+           "libra_ring_all_reduce_local")
 
 
 def libra_merge_parts(device: int, parts_out_ptr: int, parts_lse_ptr: int, n_parts: int, rows: int, head_dim: int,

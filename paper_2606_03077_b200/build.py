@@ -18,7 +18,7 @@ INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(HERE, "liblibra.so")
 STAMP_PATH = os.path.join(HERE, "liblibra.so.stamp")
 
-SOURCES = ["libra_api.cu", "planner.cpp", "sched.cpp"]
+SOURCES = ["libra_api.cu", "planner.cpp", "sched.cpp", "ring_sched.cpp"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--use_fast_math", "-Xcompiler", "-fPIC", "-shared", "-cudart", "static",

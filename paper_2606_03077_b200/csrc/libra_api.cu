@@ -1348,6 +1348,54 @@ int libra_ring_step(int32_t device, void* dst, const void* own, const void* rece
   return LIBRA_OK;
 }
 
+int libra_ring_all_reduce_local(int32_t device, void* const* bufs, int32_t n_members, size_t bytes, int32_t dtype,
+                                size_t piece_bytes, const uint32_t* ready_flag, uint32_t expected, uint32_t timeout_us,
+                                uint32_t* status_dev, int32_t num_blocks, void* stream) {
+  if (!bufs || n_members < 1 || n_members > LIBRA_RING_MAX_MEMBERS || bytes % 16 != 0 || piece_bytes < 16 ||
+      piece_bytes % 16 != 0) {
+    return LIBRA_INVALID_ARGUMENT;
+  }
+  for (int32_t i = 0; i < n_members; ++i) {
+    if (!bufs[i] || reinterpret_cast<uintptr_t>(bufs[i]) % 16 != 0) return LIBRA_INVALID_ARGUMENT;
+  }
+  libra_ring_t ring;
+  int32_t ids[LIBRA_RING_MAX_MEMBERS];
+  for (int32_t i = 0; i < n_members; ++i) ids[i] = i;
+  int rc = libra_ring_init(&ring, ids, n_members);
+  if (rc != LIBRA_OK) return rc;
+  // every member's schedule; the receive records of one (phase, step) of all members form one round of launches
+  std::vector<std::vector<libra_ring_op_t>> sched;
+  sched.resize(size_t(n_members));
+  for (int32_t i = 0; i < n_members; ++i) {
+    int32_t need = 0;
+    rc = libra_ring_schedule(&ring, i, int64_t(bytes), int64_t(piece_bytes), nullptr, 0, &need);
+    if (rc != LIBRA_OK && rc != LIBRA_WORKSPACE_TOO_SMALL) return rc;
+    sched[size_t(i)].resize(size_t(need));
+    rc = libra_ring_schedule(&ring, i, int64_t(bytes), int64_t(piece_bytes), sched[size_t(i)].data(), need, &need);
+    if (rc != LIBRA_OK) return rc;
+  }
+  std::vector<size_t> cursor;
+  cursor.assign(size_t(n_members), 0);
+  for (int32_t phase = 0; phase < 2; ++phase) {
+    for (int32_t step = 0; step + 1 < n_members; ++step) {
+      for (int32_t i = 0; i < n_members; ++i) {
+        const std::vector<libra_ring_op_t>& ops = sched[size_t(i)];
+        size_t& c = cursor[size_t(i)];
+        for (; c < ops.size() && ops[c].phase == phase && ops[c].step == step; ++c) {
+          const libra_ring_op_t& op = ops[c];
+          if (op.kind == LIBRA_RING_OP_SEND) continue;   // on one device the receiver reads the sender's buffer in place
+          uint8_t* mine = static_cast<uint8_t*>(bufs[i]) + op.offset;
+          const uint8_t* theirs = static_cast<const uint8_t*>(bufs[op.peer]) + op.offset;
+          rc = libra_ring_step(device, mine, op.kind == LIBRA_RING_OP_RECV_REDUCE ? mine : nullptr, theirs,
+                               size_t(op.bytes), dtype, ready_flag, expected, timeout_us, status_dev, num_blocks, stream);
+          if (rc != LIBRA_OK) return rc;
+        }
+      }
+    }
+  }
+  return LIBRA_OK;
+}
+
 int libra_profile_begin(libra_handle_t h) {
   if (!h) return LIBRA_INVALID_ARGUMENT;
   h->profiling = true;

@@ -67,6 +67,43 @@ def test_emulated_ring_is_bit_exact(lib, ranks, chunk):
         assert np.array_equal(gotb[r], wantb[r]), f"bf16 rank {r}"
 
 
+@pytest.mark.parametrize("ranks", [1, 2, 3, 4, 5, 6, 7, 8])
+def test_library_schedule_over_local_buffers_is_bit_exact(lib, ranks):
+    """libra_ring_all_reduce_local: the whole ReduceScatter + AllGather enqueued by the library from its own schedule
+    records (pipeline pieces of a few KB here, so that every segment is several pieces), against the oracle."""
+    import torch
+    dev = torch.device("cuda:0")
+    rng = np.random.default_rng(40 + ranks)
+    flag = torch.ones(1, dtype=torch.int32, device=dev)
+    status = torch.full((1,), 7, dtype=torch.int32, device=dev)
+    st = torch.cuda.current_stream().cuda_stream
+    for n_units, piece in ((ranks * 700 + 3, 4096), (max(1, ranks - 1), 16), (1 << 16, 16 << 20)):
+        # float32: 4 elements per 16-byte unit
+        n = n_units * 4
+        xs = [rng.standard_normal(n).astype(np.float32) * np.float32(10.0 ** rng.integers(-3, 4)) for _ in range(ranks)]
+        want = R.ring_all_reduce(xs, "f32", granule=4)
+        bufs = [torch.from_numpy(x).to(dev) for x in xs]
+        lib.libra_ring_all_reduce_local(0, [b.data_ptr() for b in bufs], n * 4, lib.RING_F32, piece, flag.data_ptr(), 1,
+                                        1000000, status.data_ptr(), 0, st)
+        torch.cuda.synchronize()
+        assert ranks == 1 or int(status.item()) == 0
+        for r in range(ranks):
+            assert np.array_equal(bufs[r].cpu().numpy().view(np.uint32), want[r].view(np.uint32)), (n_units, piece, r)
+        # bfloat16: 8 elements per unit
+        n = n_units * 8
+        xb = [torch.from_numpy(rng.standard_normal(n).astype(np.float32)).to(torch.bfloat16) for _ in range(ranks)]
+        wantb = R.ring_all_reduce([x.to(torch.float32).numpy() for x in xb], "bf16", granule=8)
+        bufs = [x.to(dev) for x in xb]
+        lib.libra_ring_all_reduce_local(0, [b.data_ptr() for b in bufs], n * 2, lib.RING_BF16, piece, flag.data_ptr(), 1,
+                                        1000000, status.data_ptr(), 3, st)
+        torch.cuda.synchronize()
+        for r in range(ranks):
+            assert np.array_equal(bufs[r].to(torch.float32).cpu().numpy(), wantb[r]), (n_units, piece, r)
+    with pytest.raises(lib.LibraError):
+        lib.libra_ring_all_reduce_local(0, [bufs[0].data_ptr() + 4], 64, lib.RING_F32, 16, flag.data_ptr(), 1, 1000,
+                                        status.data_ptr(), 0, st)
+
+
 def test_flag_set_by_the_host_while_the_kernel_polls(lib):
     import torch
     dev = torch.device("cuda:0")

@@ -1,8 +1,9 @@
-"""The exchange step of sharding a sequence's TOKENS over ranks, on CPU with two gloo ranks: each rank evaluates the
-attention over its own run of pages with the oracle, the (out, lse) pairs are all-gathered into the part-major
-[n_parts][rows][d] layout that libra_merge_parts takes, and the log-sum-exp merge of the gathered pairs is the attention
-over the whole sequence.  (On GPUs the per-rank step is the decode call with libra_set_lse_output and the merge is
-libra_merge_parts; tests/test_gpu_lse.py covers those on one device.)"""
+"""The exchange step of sharding a sequence's TOKENS over ranks, on CPU with two gloo ranks.  What this file checks is
+the ORACLE's merge identity and the layout of the exchange only: each rank evaluates the attention over its own run of
+pages with the oracle, the (out, lse) pairs are all-gathered into the part-major [n_parts][rows][d] layout that
+libra_merge_parts takes, and the oracle's log-sum-exp merge of the gathered pairs is the attention over the whole
+sequence.  The library's own step (decode with libra_set_lse_output per rank, libra_merge_parts on the gathered
+pairs) runs with two ranks in tests/test_gpu_token_shard_ranks.py and on one process in tests/test_gpu_lse.py."""
 import json
 import os
 import socket
