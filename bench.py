@@ -251,18 +251,20 @@ class Replica:
         assert self.h.debug_error_word() == 0, "device error word set"
         return out, self.h.launch_count() - n0
 
-    def device_plan_regions(self, steps: int, warmup: int, regions: int, graph: bool):
+    def device_plan_regions(self, steps: int, warmup: int, regions: int, graph: bool, overlap: bool = False):
         """The step with the device-side planner (libra_plan_device + decode), issued eagerly or replayed from a CUDA
         graph that holds one step per layout x pool copy; same regime as timed_regions.  Returns ms per step (median)."""
         torch = self.torch
         side = torch.cuda.Stream()
         per_replay = len(self.layouts) * len(self.pools)
+        self.h.set_plan_overlap(overlap)   # the lengths are not written by the kernel before the plan call here
         with torch.cuda.stream(side):
             for _ in range(max(warmup, per_replay)):
                 self.step_device(side.cuda_stream)
         torch.cuda.synchronize()
         if not graph:
             res, _ = self.timed_regions(self.step_device, steps, 0, regions, stream=side)
+            self.h.set_plan_overlap(False)
             return float(np.median([ms / steps for ms, _ in res])), float(np.median([b / (ms * 1e-3) / 1e9 for ms, b in res]))
         self.i = 0
         g = torch.cuda.CUDAGraph()
@@ -286,6 +288,7 @@ class Replica:
             per.append(ms / (reps * per_replay))
             gbs.append(self.bytes_of_steps(0, reps * per_replay) / (ms * 1e-3) / 1e9)
         assert self.h.debug_error_word() == 0, "device error word set"
+        self.h.set_plan_overlap(False)
         return float(np.median(per)), float(np.median(gbs))
 
     def step_gather_read(self, stream: int) -> None:
@@ -390,9 +393,14 @@ def measure_workload(rep: Replica, steps: int, warmup: int, regions: int, peak: 
         if with_device_plan:
             e_ms, e_gbs = rep.device_plan_regions(steps, 6, max(5, regions // 2), graph=False)
             g_ms, g_gbs = rep.device_plan_regions(steps, 6, max(5, regions // 2), graph=True)
+            o_ms, o_gbs = rep.device_plan_regions(steps, 6, max(5, regions // 2), graph=True, overlap=True)
             m["device_plan"] = {"ms_per_step_eager": e_ms, "kv_gbs_eager": e_gbs, "ms_per_step_cuda_graph": g_ms,
                                 "kv_gbs_cuda_graph": g_gbs, "over_host_plan_us": (g_ms - m["ms_per_step"]) * 1e3,
-                                "note": "libra_plan_device + decode; the graph holds one step per layout x pool copy"}
+                                "ms_per_step_cuda_graph_overlapped": o_ms, "kv_gbs_cuda_graph_overlapped": o_gbs,
+                                "overlapped_over_host_plan_us": (o_ms - m["ms_per_step"]) * 1e3,
+                                "note": "libra_plan_device + decode; the graph holds one step per layout x pool copy; "
+                                        "overlapped = libra_set_plan_overlap (the plan is made while the previous "
+                                        "step drains; the lengths here are not written by the kernel before it)"}
     return m
 
 
@@ -408,6 +416,7 @@ def compact(m: dict) -> dict:
         c["frac_of_page_gather_read"] = round(m["ceilings"]["step_frac_of_page_gather_read"], 4)
     if "device_plan" in m:
         c["device_plan_graph_ms"] = round(m["device_plan"]["ms_per_step_cuda_graph"], 5)
+        c["device_plan_overlapped_graph_ms"] = round(m["device_plan"]["ms_per_step_cuda_graph_overlapped"], 5)
     return c
 
 
@@ -1125,7 +1134,7 @@ def run_libra(args):
     del rep
     torch.cuda.empty_cache()
 
-    if not args.only_main and world == 1:
+    if not args.only_main and not args.no_others and world == 1:
         others = {}
         for name in W.WORKLOAD_ORDER[1:]:
             if name == args.workload:
@@ -1162,6 +1171,7 @@ def main():
     ap.add_argument("--impl", default="libra", choices=["libra", "reference"])
     ap.add_argument("--workload", default=MAIN_WORKLOAD)
     ap.add_argument("--only-main", action="store_true", help="skip the other workloads, the ceilings and the device plan")
+    ap.add_argument("--no-others", action="store_true", help="measure the chosen workload only (with its ceilings and device plan)")
     ap.add_argument("--full", action="store_true", help="the side measurements on every workload, not only the headline")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

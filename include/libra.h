@@ -198,6 +198,17 @@ int libra_set_dependent_launch(libra_handle_t handle, int32_t on);
  * it, which a memory checker reports; on = 0 switches it off.  Worth 2 % on a 55 us step, nothing on long ones. */
 int libra_set_cache_warmup(libra_handle_t handle, int32_t on);
 
+/* Device-side planning overlapped with the previous step (default off).  libra_plan_device's kernel is launched as a
+ * programmatic dependent of whatever precedes it and normally waits for that kernel to finish before it reads the
+ * lengths.  With this switch the caller PROMISES that the kernel directly before the libra_plan_device call in the
+ * stream does not write the lengths (true of back-to-back decode steps whose lengths were updated earlier, e.g. by the
+ * sampling kernel of the previous token): the plan is then made while that kernel drains and the planning kernel waits
+ * for it only before it exits, so the decode kernel behind it starts as early as it would after a host-side plan.
+ * Nothing else is relaxed: the plan region of the workspace is free by then (every block of a preceding decode kernel
+ * has read its entries before the planning kernel can start), and the decode kernel still waits for the planning
+ * kernel, which has waited for everything before it.  Ignored when dependent launches are off. */
+int libra_set_plan_overlap(libra_handle_t handle, int32_t on);
+
 /* Optional second output.  With a non-NULL lse_dev every later decode call (libra_decode_attn, _append, _multi,
  * _static) also writes, for every row of q, the natural logarithm of the sum of its exponentiated scores,
  * lse[b][row] = ln sum_t exp(s_t) with s_t = (q . k_t) * sm_scale, as float32 [batch, rows] (rows = q_len *
@@ -432,18 +443,13 @@ int libra_kv_scatter(libra_handle_t handle, const void* k_dense, const void* v_d
  * Outputs: *makespan (+inf if no partition uses exactly n_gpus GPUs) and the optimal partition recovered
  * by backtracking, instances in sorted-request order: degree, index of the first request in the sorted
  * list, number of requests.  Errors: INVALID_ARGUMENT, WORKSPACE_TOO_SMALL (inst_capacity too small;
- * *n_instances holds the number needed). */
+ * *n_instances holds the number needed).  Ties go to the earlier degree of tp_set, then to the smaller x.
+ * When no cost coefficient is negative the minimum over x is found by bisection (the first term of the max cannot
+ * grow with x and the second cannot shrink, so the minimum sits where they cross); otherwise the states are relaxed
+ * one by one.  Either way the result is the recurrence's, bit for bit. */
 int libra_rollout_dp(int32_t n_gpus, const int32_t* lengths, int32_t n_requests, const int32_t* tp_set, int32_t n_tp,
                      const double* cost_coef, double* makespan, int32_t* inst_tp, int32_t* inst_first,
                      int32_t* inst_count, int32_t inst_capacity, int32_t* n_instances);
-
-/* libra_rollout_dp evaluates the minimum over x by bisection when no cost coefficient is negative (the first term of
- * the max cannot grow with x and the second cannot shrink, so the minimum sits where they cross); otherwise, and
- * always in libra_rollout_dp_scan, every x is tried as the recurrence is written.  Same arguments, same results bit
- * for bit (ties go to the smaller x and the earlier degree in both); the scan is kept as the reference. */
-int libra_rollout_dp_scan(int32_t n_gpus, const int32_t* lengths, int32_t n_requests, const int32_t* tp_set,
-                          int32_t n_tp, const double* cost_coef, double* makespan, int32_t* inst_tp,
-                          int32_t* inst_first, int32_t* inst_count, int32_t inst_capacity, int32_t* n_instances);
 
 /* Causality-aware prefix tree (Section 5): a node is (prompt id, sequence of tool-return states); every
  * node keeps a histogram of the remaining trajectory length seen from that point, with bins aligned to

@@ -96,6 +96,7 @@ SIGNATURES = {
     "libra_debug_stream_read": (C.c_int, [_vp, _vp, C.c_size_t, _vp]),
     "libra_debug_gather_read": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_set_combine_mode": (C.c_int, [_vp, C.c_int32]),
+    "libra_set_plan_overlap": (C.c_int, [_vp, C.c_int32]),
     "libra_plan_host": (C.c_int, [C.POINTER(PlanParams), C.c_int32, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p,
                                   _i32p, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p]),
     "libra_workspace_invalidate": (C.c_int, [_vp]),
@@ -119,8 +120,6 @@ SIGNATURES = {
                                    _vp, _vp]),
     "libra_rollout_dp": (C.c_int, [C.c_int32, _i32p, C.c_int32, _i32p, C.c_int32, C.POINTER(C.c_double),
                                    C.POINTER(C.c_double), _i32p, _i32p, _i32p, C.c_int32, _i32p]),
-    "libra_rollout_dp_scan": (C.c_int, [C.c_int32, _i32p, C.c_int32, _i32p, C.c_int32, C.POINTER(C.c_double),
-                                        C.POINTER(C.c_double), _i32p, _i32p, _i32p, C.c_int32, _i32p]),
     "libra_trie_create": (C.c_int, [C.POINTER(_vp), _i32p, C.c_int32]),
     "libra_trie_destroy": (C.c_int, [_vp]),
     "libra_trie_insert": (C.c_int, [_vp, C.c_int64, _i32p, C.c_int32, _i32p]),
@@ -242,8 +241,8 @@ def libra_merge_parts(device: int, parts_out_ptr: int, parts_lse_ptr: int, n_par
                                  lse_out_ptr or None, stream), "libra_merge_parts")
 
 
-def libra_rollout_dp(n_gpus: int, lengths, tp_set, cost_coef, scan: bool = False):
-    """RolloutDP: returns (makespan, [(tp, first_sorted_index, count), ...]).  scan = the term-by-term reference."""
+def libra_rollout_dp(n_gpus: int, lengths, tp_set, cost_coef):
+    """RolloutDP: returns (makespan, [(tp, first_sorted_index, count), ...])."""
     lens = _as_i32(lengths)
     tps = _as_i32(tp_set)
     coef = np.ascontiguousarray(cost_coef, dtype=np.float64).reshape(len(tps), 4)
@@ -251,8 +250,7 @@ def libra_rollout_dp(n_gpus: int, lengths, tp_set, cost_coef, scan: bool = False
     itp, ifirst, icount = (np.zeros(cap, np.int32) for _ in range(3))
     mk, n = C.c_double(0), C.c_int32(0)
     p = lambda a: a.ctypes.data_as(_i32p)
-    fn = lib.libra_rollout_dp_scan if scan else lib.libra_rollout_dp
-    st = fn(n_gpus, p(lens), len(lens), p(tps), len(tps), coef.ctypes.data_as(C.POINTER(C.c_double)),
+    st = lib.libra_rollout_dp(n_gpus, p(lens), len(lens), p(tps), len(tps), coef.ctypes.data_as(C.POINTER(C.c_double)),
             C.byref(mk), p(itp), p(ifirst), p(icount), cap, C.byref(n))
     _check(st, "libra_rollout_dp")
     return mk.value, [(int(itp[k]), int(ifirst[k]), int(icount[k])) for k in range(n.value)]
@@ -386,6 +384,9 @@ class Handle:
 
     def set_cache_warmup(self, on: bool) -> None:
         _check(lib.libra_set_cache_warmup(self._h, 1 if on else 0), "libra_set_cache_warmup")
+
+    def set_plan_overlap(self, on: bool) -> None:
+        _check(lib.libra_set_plan_overlap(self._h, 1 if on else 0), "libra_set_plan_overlap")
 
     def set_early_prefetch(self, on: bool) -> None:
         _check(lib.libra_set_early_prefetch(self._h, 1 if on else 0), "libra_set_early_prefetch")

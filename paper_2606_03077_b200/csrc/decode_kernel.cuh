@@ -767,6 +767,21 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   const uint32_t my_ring_u32 = smem_u32(my_ring);
   const uint32_t my_bar0 = smem_u32(&bars[warp * STAGES]);
 
+  // A device-side plan comes with a grid sized for the worst case: most blocks past the first wave have nothing to
+  // do.  They find that out first (the counts are only valid once the planning kernel has finished) and leave
+  // without setting anything up.
+  if (p.dev_counts != nullptr && blockIdx.x >= sm_count()) {
+    grid_dependency_wait();
+    const int n_items = p.dev_counts[plan_layout::kCntItems];
+    const int n_units = n_items * p.num_kv_heads;
+    if (int(blockIdx.x) >= n_units) {
+      if (int(blockIdx.x) - n_units < p.dev_counts[plan_layout::kCntEmpty]) {
+        zero_empty_row<D>(p, p.entries, n_items, int(blockIdx.x) - n_units, threadIdx.x, NW * 32);
+      }
+      return;
+    }
+  }
+
   const uint64_t kv_policy = l2_evict_first_policy();
   if (lane == 0) {
     prefetch_tensormap(&map_k);

@@ -179,6 +179,7 @@ struct libra_handle_s {
   float* lse_out = nullptr;     // optional second output of the step (libra_set_lse_output)
   bool early_prefetch = false;  // the caller's promise about the preceding kernel (libra_set_early_prefetch)
   bool l2_warmup = true;        // libra_set_cache_warmup
+  bool plan_overlap = false;    // libra_set_plan_overlap: the caller's promise about the kernel before libra_plan_device
 
   // pinned staging for uploads of plans too large for the kernel parameters
   int32_t* staging[2] = {nullptr, nullptr};
@@ -655,6 +656,7 @@ int libra_plan_device(libra_handle_t h, const int32_t* seq_lens_dev, int32_t bat
   p.max_splits = h->params.max_splits;
   p.wave_slots = int64_t(h->params.n_sm) * h->params.ctas_per_sm;
   p.refine = h->params.refine;
+  p.overlap = (h->plan_overlap && h->pdl) ? 1 : 0;
   p.max_items = int32_t(std::min<int64_t>(h->max_items, libra::kDevPlanMax));
   p.max_len = int32_t(std::min<int64_t>(int64_t(h->cfg.block_table_ld) * h->cfg.page_size, 0x7fffffff));
   p.counts = reinterpret_cast<int32_t*>(ws + h->dev_counts_off);
@@ -662,8 +664,19 @@ int libra_plan_device(libra_handle_t h, const int32_t* seq_lens_dev, int32_t bat
   p.entries = reinterpret_cast<int4*>(ws + h->dev_entries_off);
   p.fixes = reinterpret_cast<int4*>(ws + h->dev_fixes_off);
   p.error_word = reinterpret_cast<uint32_t*>(ws);
-  libra::plan_kernel<<<1, libra::kDevPlanThreads, libra::plan_kernel_smem_bytes(), st>>>(p);
-  LIBRA_CUDA_TRY(h, cudaGetLastError());
+  {
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(1);
+    lc.blockDim = dim3(libra::kDevPlanThreads);
+    lc.dynamicSmemBytes = libra::plan_kernel_smem_bytes();
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = h->pdl ? 1 : 0;   // a dependent of its predecessor: it waits inside before it reads or writes anything
+    LIBRA_CUDA_TRY(h, cudaLaunchKernelEx(&lc, libra::plan_kernel, p));
+  }
   ++h->launches;
   h->workspace = workspace_dev;
   h->last_stream = stream;
@@ -783,6 +796,12 @@ int libra_set_lse_output(libra_handle_t h, float* lse_dev) {
 int libra_set_early_prefetch(libra_handle_t h, int32_t on) {
   if (!h || (on != 0 && on != 1)) return LIBRA_INVALID_ARGUMENT;
   h->early_prefetch = (on == 1);
+  return LIBRA_OK;
+}
+
+int libra_set_plan_overlap(libra_handle_t h, int32_t on) {
+  if (!h || (on != 0 && on != 1)) return LIBRA_INVALID_ARGUMENT;
+  h->plan_overlap = (on == 1);
   return LIBRA_OK;
 }
 

@@ -52,13 +52,16 @@ struct libra_trie_s {
 
 namespace {
 
-// The recurrence as printed, and a faster evaluation of the same minimum.
+// dp[g][i] = best makespan of "exactly g GPUs serve the first i sorted requests" (Section 4.3):
 //   dp[g][i] = min over tp <= g, 0 <= x <= i of max(dp[g - tp][i - x], Cost(tp, i - x + 1, i))
-// Plain: every x is tried.  Fast (valid when no cost coefficient is negative): as x grows the first term cannot
-// grow (fewer requests left for the other instances) and the second cannot shrink (more requests on this one), so
-// the minimum of their maximum sits where they cross; a binary search finds the crossing and a second one the
-// leftmost x of the same value, which is the x the plain scan would have kept.  Same dp, same arg-mins, bit for bit.
-int rollout_dp_impl(bool allow_fast, int32_t n_gpus, const int32_t* lengths, int32_t n_requests, const int32_t* tp_set,
+// Ties go to the earlier degree, then to the smaller x.
+// When no cost coefficient is negative, the minimum over x is found without trying every x: as x grows the first
+// term cannot grow (fewer requests left for the other instances) and the second cannot shrink (more requests on this
+// one), so the minimum of their maximum sits where they cross; one bisection finds the crossing and a second one the
+// leftmost x of the same value.  With a negative coefficient nothing is monotone and the states are relaxed forwards
+// instead (every state offers max(its value, cost of the next segment) to its successors; the smallest
+// (value, degree, x) wins).
+int rollout_dp_impl(int32_t n_gpus, const int32_t* lengths, int32_t n_requests, const int32_t* tp_set,
                     int32_t n_tp, const double* cost_coef, double* makespan, int32_t* inst_tp, int32_t* inst_first,
                     int32_t* inst_count, int32_t inst_capacity, int32_t* n_instances) {
   if (n_gpus < 0 || n_requests < 0 || n_tp <= 0 || !tp_set || !cost_coef || !makespan || !n_instances) {
@@ -70,9 +73,9 @@ int rollout_dp_impl(bool allow_fast, int32_t n_gpus, const int32_t* lengths, int
   const int G = n_gpus, L = n_requests;
   std::vector<int32_t> sorted(lengths, lengths + L);
   std::sort(sorted.begin(), sorted.end());  // non-decreasing: every instance gets a contiguous segment
-  bool fast = allow_fast;
-  for (int t = 0; t < 4 * n_tp; ++t) fast = fast && cost_coef[t] >= 0.0;
-  for (int i = 0; i < L; ++i) fast = fast && sorted[size_t(i)] >= 0;
+  bool monotone = true;
+  for (int t = 0; t < 4 * n_tp; ++t) monotone = monotone && cost_coef[t] >= 0.0;
+  for (int i = 0; i < L; ++i) monotone = monotone && sorted[size_t(i)] >= 0;
   SegmentCost cost;
   cost.coef = cost_coef;
   cost.s1.assign(L + 1, 0.0);
@@ -86,7 +89,30 @@ int rollout_dp_impl(bool allow_fast, int32_t n_gpus, const int32_t* lengths, int
   std::vector<double> dp((size_t(G) + 1) * W, inf);
   std::vector<int32_t> arg_tp((size_t(G) + 1) * W, -1), arg_x((size_t(G) + 1) * W, -1);
   dp[0] = 0.0;  // dp[0][0]
-  for (int g = 1; g <= G; ++g) {
+  if (!monotone) {
+    // forward relaxation; dp[g'][.] is final once every g < g' has been expanded, because degrees are positive
+    for (int g = 0; g < G; ++g) {
+      for (int i = 0; i <= L; ++i) {
+        const double here = dp[size_t(g) * W + i];
+        if (here == inf) continue;
+        for (int t = 0; t < n_tp; ++t) {
+          const int g2 = g + tp_set[t];
+          if (g2 > G) continue;
+          for (int x = 0; i + x <= L; ++x) {
+            const double v = std::max(here, cost(t, i + 1, i + x));
+            const size_t at = size_t(g2) * W + size_t(i + x);
+            const bool better = v < dp[at] || (v == dp[at] && (t < arg_tp[at] || (t == arg_tp[at] && x < arg_x[at])));
+            if (better) {
+              dp[at] = v;
+              arg_tp[at] = t;
+              arg_x[at] = x;
+            }
+          }
+        }
+      }
+    }
+  }
+  for (int g = 1; monotone && g <= G; ++g) {
     for (int i = 0; i <= L; ++i) {
       double best = inf;
       int btp = -1, bx = -1;
@@ -94,19 +120,6 @@ int rollout_dp_impl(bool allow_fast, int32_t n_gpus, const int32_t* lengths, int
         const int tp = tp_set[t];
         if (tp > g) continue;
         const double* prev = &dp[size_t(g - tp) * W];
-        if (!fast) {
-          for (int x = 0; x <= i; ++x) {
-            const double p = prev[i - x];
-            if (!(p < best)) continue;  // max(p, cost) >= p: cannot improve
-            const double cand = std::max(p, cost(t, i - x + 1, i));
-            if (cand < best) {
-              best = cand;
-              btp = t;
-              bx = x;
-            }
-          }
-          continue;
-        }
         // first x at which this instance's cost reaches what the others need (x = i + 1 if it never does)
         int lo = 0, hi = i + 1;
         while (lo < hi) {
@@ -173,15 +186,8 @@ extern "C" {
 int libra_rollout_dp(int32_t n_gpus, const int32_t* lengths, int32_t n_requests, const int32_t* tp_set, int32_t n_tp,
                      const double* cost_coef, double* makespan, int32_t* inst_tp, int32_t* inst_first,
                      int32_t* inst_count, int32_t inst_capacity, int32_t* n_instances) {
-  return rollout_dp_impl(true, n_gpus, lengths, n_requests, tp_set, n_tp, cost_coef, makespan, inst_tp, inst_first,
-                         inst_count, inst_capacity, n_instances);
-}
-
-int libra_rollout_dp_scan(int32_t n_gpus, const int32_t* lengths, int32_t n_requests, const int32_t* tp_set, int32_t n_tp,
-                          const double* cost_coef, double* makespan, int32_t* inst_tp, int32_t* inst_first,
-                          int32_t* inst_count, int32_t inst_capacity, int32_t* n_instances) {
-  return rollout_dp_impl(false, n_gpus, lengths, n_requests, tp_set, n_tp, cost_coef, makespan, inst_tp, inst_first,
-                         inst_count, inst_capacity, n_instances);
+  return rollout_dp_impl(n_gpus, lengths, n_requests, tp_set, n_tp, cost_coef, makespan, inst_tp, inst_first, inst_count,
+                         inst_capacity, n_instances);
 }
 
 int libra_trie_create(libra_trie_t* trie, const int32_t* bin_upper, int32_t n_thresholds) {

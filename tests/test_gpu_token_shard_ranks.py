@@ -59,11 +59,11 @@ torch.cuda.synchronize()
 assert h.debug_error_word() == 0
 n_split = int(len(h.plan_export()["combine"]))
 # the exchange: every rank ends up with all parts, part-major
-outs = [torch.zeros((B * Hq, d), dtype=torch.int16) for _ in range(world)]
+outs = [torch.zeros((B * Hq, d // 2), dtype=torch.int32) for _ in range(world)]   # bf16 pairs as int32 words on the wire
 lses = [torch.zeros((B * Hq,), dtype=torch.float32) for _ in range(world)]
-dist.all_gather(outs, out.cpu())
+dist.all_gather(outs, out.cpu().view(torch.int32))
 dist.all_gather(lses, lse.cpu())
-parts_out = torch.stack(outs).to(dev)      # [n_parts][rows][d] bf16 bits
+parts_out = torch.stack(outs).view(torch.int16).to(dev)      # [n_parts][rows][d] bf16 bits
 parts_lse = torch.stack(lses).to(dev)      # [n_parts][rows]
 merged = torch.full((B * Hq, d), 0x7FC0, dtype=torch.int16, device=dev)
 merged_lse = torch.full((B * Hq,), float("nan"), dtype=torch.float32, device=dev)

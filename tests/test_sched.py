@@ -114,14 +114,30 @@ def test_prefix_tree_small_example(lib):
     t.close()
 
 
-def test_bisection_gives_the_scan_bit_for_bit(lib):
-    """libra_rollout_dp (bisection on x where the coefficients allow it) against libra_rollout_dp_scan (every x):
-    same makespan, same partition, ties included; and with a negative coefficient the two are the same code path."""
+def test_scan_reference_finds_the_exhaustive_optimum():
+    """The term-by-term evaluation of the recurrence (the reference below) against exhaustive search."""
+    rng = np.random.default_rng(17)
+    for trial in range(40):
+        n = int(rng.integers(0, 7)); g = int(rng.integers(1, 7))
+        lens = rng.integers(1, 50, size=n)
+        tp_set = sorted(set(int(x) for x in rng.choice([1, 2, 4], size=int(rng.integers(1, 4)))))
+        coef = [[float(rng.integers(0, 4)), float(rng.integers(0, 3)) * 1e-2, float(rng.integers(0, 3)), float(rng.integers(0, 5))]
+                for _ in tp_set]
+        mk, inst = R.rollout_dp_scan(g, lens, tp_set, coef)
+        want = R.rollout_partition_brute_force(g, lens, tp_set, coef)
+        assert (math.isinf(mk) and math.isinf(want)) or abs(mk - want) <= 1e-9 * max(1.0, abs(want))
+        if not math.isinf(mk):
+            assert sum(tp for tp, _, _ in inst) == g and sum(c for _, _, c in inst) == n
+
+
+def test_library_gives_the_recurrence_bit_for_bit(lib):
+    """libra_rollout_dp (bisection on x where no coefficient is negative, forward relaxation otherwise) against the
+    term-by-term evaluation of the recurrence: same makespan, same partition, ties included."""
     import time
     rng = np.random.default_rng(7)
-    for trial in range(60):
-        n = int(rng.integers(0, 220))
-        g = int(rng.integers(1, 33))
+    for trial in range(48):
+        n = int(rng.integers(0, 90))
+        g = int(rng.integers(1, 20))
         kind = trial % 4
         if kind == 0:
             lens = rng.integers(1, 40000, size=n)
@@ -134,12 +150,12 @@ def test_bisection_gives_the_scan_bit_for_bit(lib):
         tp_set = sorted(set(int(x) for x in rng.choice([1, 2, 4, 8], size=int(rng.integers(1, 5)))))
         coef = [[float(rng.integers(0, 4)) / (1 + t), float(rng.integers(0, 3)) * 1e-4 / (1 + t), float(rng.integers(0, 3)),
                  float(rng.integers(0, 5))] for t in range(len(tp_set))]
-        fast = lib.libra_rollout_dp(g, lens, tp_set, coef)
-        scan = lib.libra_rollout_dp(g, lens, tp_set, coef, scan=True)
-        assert fast == scan or (math.isinf(fast[0]) and math.isinf(scan[0])), (trial, fast, scan)
-    coef = [[1.0, 0.0, -0.5, 0.0], [0.5, 0.0, 0.0, 1.0]]        # a negative coefficient: no bisection
-    lens = rng.integers(1, 100, size=50)
-    assert lib.libra_rollout_dp(8, lens, [1, 2], coef) == lib.libra_rollout_dp(8, lens, [1, 2], coef, scan=True)
+        if trial % 6 == 5:
+            coef[0][2] = -0.5                                    # a negative coefficient: no bisection
+        got = lib.libra_rollout_dp(g, lens, tp_set, coef)
+        want = R.rollout_dp_scan(g, lens, tp_set, coef)
+        assert got == want or (math.isinf(got[0]) and math.isinf(want[0])), (trial, got, want)
+    rng = np.random.default_rng(8)
     # and it is what makes the planner cheap: 128 GPUs x 4096 requests
     lens = np.floor(2048 * np.exp(rng.standard_normal(4096))).astype(np.int64) + 1
     coef = [[1.0 / tp, 2e-5 / tp, 5.0, 100.0 * tp] for tp in (1, 2, 4, 8)]
