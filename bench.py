@@ -201,6 +201,17 @@ class Replica:
         self.h.decode_attn(self.q.data_ptr(), k.data_ptr(), v.data_ptr(), self.bts[s].data_ptr(),
                            self.lens_dev[s].data_ptr(), self.out.data_ptr(), stream)
 
+    def step_device_layers(self, stream: int, layers: int) -> None:
+        """One device-side plan followed by `layers` decode calls on it: what a model with that many attention layers
+        issues per generated token (the lengths, hence the plan, are the same for every layer)."""
+        s = self.i % len(self.layouts)
+        self.h.plan_device(self.lens_dev[s].data_ptr(), self.w.batch, self.ws.data_ptr(), self.ws.numel(), stream)
+        for l in range(layers):
+            k, v = self.pools[(self.i + l) % len(self.pools)]
+            self.h.decode_attn(self.q.data_ptr(), k.data_ptr(), v.data_ptr(), self.bts[s].data_ptr(),
+                               self.lens_dev[s].data_ptr(), self.out.data_ptr(), stream)
+        self.i += 1
+
     def bytes_of_steps(self, i0: int, n: int) -> int:
         """KV bytes of steps i0 .. i0 + n - 1 (a workload with several layouts cycles through them, and their
         sizes differ: the bytes of a region are those of the layouts it actually ran)."""
@@ -251,29 +262,30 @@ class Replica:
         assert self.h.debug_error_word() == 0, "device error word set"
         return out, self.h.launch_count() - n0
 
-    def device_plan_regions(self, steps: int, warmup: int, regions: int, graph: bool, overlap: bool = False):
+    def device_plan_regions(self, steps: int, warmup: int, regions: int, graph: bool, decodes_per_plan: int = 1):
         """The step with the device-side planner (libra_plan_device + decode), issued eagerly or replayed from a CUDA
         graph that holds one step per layout x pool copy; same regime as timed_regions.  Returns ms per step (median)."""
         torch = self.torch
         side = torch.cuda.Stream()
         per_replay = len(self.layouts) * len(self.pools)
-        self.h.set_plan_overlap(overlap)   # the lengths are not written by the kernel before the plan call here
         with torch.cuda.stream(side):
             for _ in range(max(warmup, per_replay)):
                 self.step_device(side.cuda_stream)
         torch.cuda.synchronize()
         if not graph:
             res, _ = self.timed_regions(self.step_device, steps, 0, regions, stream=side)
-            self.h.set_plan_overlap(False)
             return float(np.median([ms / steps for ms, _ in res])), float(np.median([b / (ms * 1e-3) / 1e9 for ms, b in res]))
         self.i = 0
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=side):
             for _ in range(per_replay):
-                self.step_device(side.cuda_stream)
+                if decodes_per_plan == 1:
+                    self.step_device(side.cuda_stream)
+                else:
+                    self.step_device_layers(side.cuda_stream, decodes_per_plan)
         g.replay()
         torch.cuda.synchronize()
-        reps = max(1, steps // per_replay)
+        reps = max(1, steps // (per_replay * decodes_per_plan))
         per, gbs = [], []
         for _ in range(regions):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -285,10 +297,9 @@ class Replica:
                 e1.record()
             torch.cuda.synchronize()
             ms = e0.elapsed_time(e1)
-            per.append(ms / (reps * per_replay))
-            gbs.append(self.bytes_of_steps(0, reps * per_replay) / (ms * 1e-3) / 1e9)
+            per.append(ms / (reps * per_replay * decodes_per_plan))
+            gbs.append(self.bytes_of_steps(0, reps * per_replay) * decodes_per_plan / (ms * 1e-3) / 1e9)
         assert self.h.debug_error_word() == 0, "device error word set"
-        self.h.set_plan_overlap(False)
         return float(np.median(per)), float(np.median(gbs))
 
     def step_gather_read(self, stream: int) -> None:
@@ -393,14 +404,13 @@ def measure_workload(rep: Replica, steps: int, warmup: int, regions: int, peak: 
         if with_device_plan:
             e_ms, e_gbs = rep.device_plan_regions(steps, 6, max(5, regions // 2), graph=False)
             g_ms, g_gbs = rep.device_plan_regions(steps, 6, max(5, regions // 2), graph=True)
-            o_ms, o_gbs = rep.device_plan_regions(steps, 6, max(5, regions // 2), graph=True, overlap=True)
+            l_ms, l_gbs = rep.device_plan_regions(max(steps, 64), 6, max(5, regions // 2), graph=True, decodes_per_plan=32)
             m["device_plan"] = {"ms_per_step_eager": e_ms, "kv_gbs_eager": e_gbs, "ms_per_step_cuda_graph": g_ms,
                                 "kv_gbs_cuda_graph": g_gbs, "over_host_plan_us": (g_ms - m["ms_per_step"]) * 1e3,
-                                "ms_per_step_cuda_graph_overlapped": o_ms, "kv_gbs_cuda_graph_overlapped": o_gbs,
-                                "overlapped_over_host_plan_us": (o_ms - m["ms_per_step"]) * 1e3,
-                                "note": "libra_plan_device + decode; the graph holds one step per layout x pool copy; "
-                                        "overlapped = libra_set_plan_overlap (the plan is made while the previous "
-                                        "step drains; the lengths here are not written by the kernel before it)"}
+                                "ms_per_decode_call_32_per_plan": l_ms, "kv_gbs_32_per_plan": l_gbs,
+                                "note": "libra_plan_device + decode replayed from a CUDA graph (one step per layout x pool "
+                                        "copy); 32_per_plan = one device-side plan serving 32 decode calls, as the 32 "
+                                        "attention layers of a model share one step's lengths"}
     return m
 
 
@@ -416,7 +426,7 @@ def compact(m: dict) -> dict:
         c["frac_of_page_gather_read"] = round(m["ceilings"]["step_frac_of_page_gather_read"], 4)
     if "device_plan" in m:
         c["device_plan_graph_ms"] = round(m["device_plan"]["ms_per_step_cuda_graph"], 5)
-        c["device_plan_overlapped_graph_ms"] = round(m["device_plan"]["ms_per_step_cuda_graph_overlapped"], 5)
+        c["device_plan_32_calls_per_plan_ms"] = round(m["device_plan"]["ms_per_decode_call_32_per_plan"], 5)
     return c
 
 

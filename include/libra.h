@@ -198,16 +198,6 @@ int libra_set_dependent_launch(libra_handle_t handle, int32_t on);
  * it, which a memory checker reports; on = 0 switches it off.  Worth 2 % on a 55 us step, nothing on long ones. */
 int libra_set_cache_warmup(libra_handle_t handle, int32_t on);
 
-/* Device-side planning overlapped with the previous step (default off).  libra_plan_device's kernel is launched as a
- * programmatic dependent of whatever precedes it and normally waits for that kernel to finish before it reads the
- * lengths.  With this switch the caller PROMISES that the kernel directly before the libra_plan_device call in the
- * stream does not write the lengths (true of back-to-back decode steps whose lengths were updated earlier, e.g. by the
- * sampling kernel of the previous token): the plan is then made while that kernel drains and the planning kernel waits
- * for it only before it exits, so the decode kernel behind it starts as early as it would after a host-side plan.
- * Nothing else is relaxed: the plan region of the workspace is free by then (every block of a preceding decode kernel
- * has read its entries before the planning kernel can start), and the decode kernel still waits for the planning
- * kernel, which has waited for everything before it.  Ignored when dependent launches are off. */
-int libra_set_plan_overlap(libra_handle_t handle, int32_t on);
 
 /* Optional second output.  With a non-NULL lse_dev every later decode call (libra_decode_attn, _append, _multi,
  * _static) also writes, for every row of q, the natural logarithm of the sum of its exponentiated scores,

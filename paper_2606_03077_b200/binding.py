@@ -96,7 +96,6 @@ SIGNATURES = {
     "libra_debug_stream_read": (C.c_int, [_vp, _vp, C.c_size_t, _vp]),
     "libra_debug_gather_read": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_set_combine_mode": (C.c_int, [_vp, C.c_int32]),
-    "libra_set_plan_overlap": (C.c_int, [_vp, C.c_int32]),
     "libra_plan_host": (C.c_int, [C.POINTER(PlanParams), C.c_int32, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p,
                                   _i32p, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p]),
     "libra_workspace_invalidate": (C.c_int, [_vp]),
@@ -384,9 +383,6 @@ class Handle:
 
     def set_cache_warmup(self, on: bool) -> None:
         _check(lib.libra_set_cache_warmup(self._h, 1 if on else 0), "libra_set_cache_warmup")
-
-    def set_plan_overlap(self, on: bool) -> None:
-        _check(lib.libra_set_plan_overlap(self._h, 1 if on else 0), "libra_set_plan_overlap")
 
     def set_early_prefetch(self, on: bool) -> None:
         _check(lib.libra_set_early_prefetch(self._h, 1 if on else 0), "libra_set_early_prefetch")

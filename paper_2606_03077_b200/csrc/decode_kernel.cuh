@@ -770,16 +770,16 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   // A device-side plan comes with a grid sized for the worst case: most blocks past the first wave have nothing to
   // do.  They find that out first (the counts are only valid once the planning kernel has finished) and leave
   // without setting anything up.
-  if (p.dev_counts != nullptr && blockIdx.x >= sm_count()) {
+  // The grid's last block zeroes the output rows of all empty sequences (a host plan gives each its own block).
+  if (p.dev_counts != nullptr && (blockIdx.x >= sm_count() || blockIdx.x == gridDim.x - 1)) {
     grid_dependency_wait();
     const int n_items = p.dev_counts[plan_layout::kCntItems];
-    const int n_units = n_items * p.num_kv_heads;
-    if (int(blockIdx.x) >= n_units) {
-      if (int(blockIdx.x) - n_units < p.dev_counts[plan_layout::kCntEmpty]) {
-        zero_empty_row<D>(p, p.entries, n_items, int(blockIdx.x) - n_units, threadIdx.x, NW * 32);
-      }
+    if (blockIdx.x == gridDim.x - 1) {
+      const int n_empty = p.dev_counts[plan_layout::kCntEmpty];
+      for (int e = 0; e < n_empty; ++e) zero_empty_row<D>(p, p.entries, n_items, e, threadIdx.x, NW * 32);
       return;
     }
+    if (int(blockIdx.x) >= n_items * p.num_kv_heads) return;
   }
 
   const uint64_t kv_policy = l2_evict_first_policy();
@@ -802,11 +802,14 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   // Ask for the first STAGES tiles per warp of unit `blk` (a block index of this grid) to be brought into L2.
   // (Used at the step boundary only: first-wave blocks warming the units of the NEXT wave as they finish their own
   // gained 1 % on 256 equal units and lost 1 - 2 % on the ragged workloads.)
-  const bool warm_ok = p.l2_warmup != 0 && p.entries == nullptr && p.dev_counts == nullptr && blockIdx.x < sm_count();
+  // (The host sets l2_warmup only when the plan cannot change under this block's eyes: it travels in the kernel
+  // parameters, or it lies in the workspace and an earlier decode launch has already run on it, so that the kernel
+  // that wrote it is known to have finished.)
+  const bool warm_ok = p.l2_warmup != 0 && blockIdx.x < sm_count();
   auto warm_unit = [&](int blk) {
     const int w_item = blk / p.num_kv_heads;
     const int w_kvh = blk - w_item * p.num_kv_heads;
-    const Unit w = decode_unit<NW>(pp.e[w_item], w_kvh, warp);
+    const Unit w = decode_unit<NW>((p.entries ? p.entries : pp.e)[w_item], w_kvh, warp);
     if (lane < STAGES && lane < w.n_it) {   // more tiles per warp helped long units and cost the short ones more
       const int tile = w.first_page + warp + lane * NW;
       const int32_t pid = ld_cg_s32(p.block_table + int64_t(w.b) * p.block_table_ld + (tile >> p.tile_shift));
@@ -828,7 +831,10 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     // A block of the first wave (resident while the kernel before it drains, DRAM all but idle) looks up the pages
     // of its first tiles and has them brought into L2; ids and data are fetched again, for real, after the wait.  A
     // stale id only warms the wrong lines, a line written later is updated in L2, which is where the copies read.
-    if (warm_ok && int(blockIdx.x) < p.num_units) warm_unit(int(blockIdx.x));
+    if (warm_ok) {
+      const int units = p.dev_counts ? p.dev_counts[plan_layout::kCntItems] * p.num_kv_heads : p.num_units;
+      if (int(blockIdx.x) < units) warm_unit(int(blockIdx.x));
+    }
     grid_dependency_wait();
   }
 
@@ -843,7 +849,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   }
   if (int(blockIdx.x) >= num_units) {
     if (early) grid_dependency_wait();   // `out` may still be read by the kernel before this one
-    if (int(blockIdx.x) - num_units < num_empty) {
+    if (p.dev_counts == nullptr && int(blockIdx.x) - num_units < num_empty) {
       zero_empty_row<D>(p, entries, num_items, int(blockIdx.x) - num_units, threadIdx.x, NW * 32);
     }
     return;

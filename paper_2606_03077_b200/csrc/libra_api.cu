@@ -179,7 +179,6 @@ struct libra_handle_s {
   float* lse_out = nullptr;     // optional second output of the step (libra_set_lse_output)
   bool early_prefetch = false;  // the caller's promise about the preceding kernel (libra_set_early_prefetch)
   bool l2_warmup = true;        // libra_set_cache_warmup
-  bool plan_overlap = false;    // libra_set_plan_overlap: the caller's promise about the kernel before libra_plan_device
 
   // pinned staging for uploads of plans too large for the kernel parameters
   int32_t* staging[2] = {nullptr, nullptr};
@@ -195,6 +194,7 @@ struct libra_handle_s {
   int32_t num_items = 0;
   void* last_stream = nullptr;
   bool device_planned = false;  // the last plan was made by the device-side planner: counts live in the workspace
+  int64_t decodes_on_plan = 0;  // decode launches enqueued since the last plan call
   int32_t planned_batch = 0;
   size_t dev_counts_off = 0, dev_per_seq_off = 0, dev_entries_off = 0, dev_fixes_off = 0;
   std::vector<int32_t> export_scratch;
@@ -627,6 +627,7 @@ int libra_plan(libra_handle_t h, const int32_t* seq_lens_host, int32_t batch, vo
   h->last_stream = stream;
   h->planned = true;
   h->device_planned = false;
+  h->decodes_on_plan = 0;
   h->planned_batch = batch;
   return LIBRA_OK;
 }
@@ -656,7 +657,6 @@ int libra_plan_device(libra_handle_t h, const int32_t* seq_lens_dev, int32_t bat
   p.max_splits = h->params.max_splits;
   p.wave_slots = int64_t(h->params.n_sm) * h->params.ctas_per_sm;
   p.refine = h->params.refine;
-  p.overlap = (h->plan_overlap && h->pdl) ? 1 : 0;
   p.max_items = int32_t(std::min<int64_t>(h->max_items, libra::kDevPlanMax));
   p.max_len = int32_t(std::min<int64_t>(int64_t(h->cfg.block_table_ld) * h->cfg.page_size, 0x7fffffff));
   p.counts = reinterpret_cast<int32_t*>(ws + h->dev_counts_off);
@@ -682,6 +682,7 @@ int libra_plan_device(libra_handle_t h, const int32_t* seq_lens_dev, int32_t bat
   h->last_stream = stream;
   h->planned = true;
   h->device_planned = true;
+  h->decodes_on_plan = 0;
   h->plan_in_params = false;
   h->planned_batch = batch;
   return LIBRA_OK;
@@ -799,12 +800,6 @@ int libra_set_early_prefetch(libra_handle_t h, int32_t on) {
   return LIBRA_OK;
 }
 
-int libra_set_plan_overlap(libra_handle_t h, int32_t on) {
-  if (!h || (on != 0 && on != 1)) return LIBRA_INVALID_ARGUMENT;
-  h->plan_overlap = (on == 1);
-  return LIBRA_OK;
-}
-
 int libra_set_cache_warmup(libra_handle_t h, int32_t on) {
   if (!h || (on != 0 && on != 1)) return LIBRA_INVALID_ARGUMENT;
   h->l2_warmup = (on == 1);
@@ -900,10 +895,13 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
   const int32_t rows = q_len * h->cfg.num_q_heads;   // rows of q / out per sequence
   const bool fused = h->combine_mode == 1 || loads_only;
   // host plan: exact counts; device plan: upper bounds for the grids, the kernels read the counts themselves
-  const int32_t n_empty = h->device_planned ? h->planned_batch : int32_t(h->plan.empty.size());
+  // (a device plan: one block at the end of the grid zeroes the rows of all empty sequences)
+  const int32_t n_empty = h->device_planned ? 1 : int32_t(h->plan.empty.size());
   const int32_t n_combine = h->device_planned ? h->planned_batch : int32_t(h->plan.combine.size());
   const int32_t n_items_bound =
-      h->device_planned ? int32_t(std::min<int64_t>(h->max_items, libra::kDevPlanMax)) : h->num_items;
+      h->device_planned ? int32_t(std::min<int64_t>(libra::max_items(h->params, h->cfg.num_kv_heads, h->planned_batch),
+                                                    libra::kDevPlanMax))
+                        : h->num_items;
   const int32_t n_units = n_items_bound * h->cfg.num_kv_heads;
   if (n_units > 0 || n_empty > 0) {
     DecodeParams p;
@@ -937,7 +935,9 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     p.num_empty = n_empty;
     p.fused_combine = fused ? 1 : 0;
     p.early_prefetch = (h->early_prefetch && h->pdl) ? 1 : 0;
-    p.l2_warmup = (h->l2_warmup && h->pdl) ? 1 : 0;
+    // a plan in the workspace (device-made, or too large for the kernel parameters) may be read before the dependency
+    // wait only once a decode launch has run on it: the kernel or copy that wrote it has then certainly finished
+    p.l2_warmup = (h->l2_warmup && h->pdl && (h->plan_in_params || h->decodes_on_plan > 0)) ? 1 : 0;
     p.k_new = k_new;
     p.v_new = v_new;
     p.k_pool = const_cast<void*>(k_pages);
@@ -971,6 +971,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     lc.numAttrs = h->pdl ? 1 : 0;
     LIBRA_CUDA_TRY(h, cudaLaunchKernelEx(&lc, fn, pm->map_k, pm->map_v, p, h->pp));
     ++h->launches;
+    ++h->decodes_on_plan;
   }
   if (ev) LIBRA_CUDA_TRY(h, cudaEventRecord(ev[1], st));
   if (!fused && n_combine > 0) {

@@ -34,7 +34,6 @@ struct PlanKernelParams {
   int32_t chunk_align, min_chunk, max_splits;
   int64_t wave_slots;        // n_sm * ctas_per_sm: thread blocks of one wave
   int32_t refine;            // 1: a coarse plan of long blocks is made again for twice as many slots
-  int32_t overlap;           // 1: plan first, wait for the preceding grid last (see plan_kernel)
   int32_t max_items;         // capacity of `entries` for work items
   int32_t max_len;           // longest sequence the block table can describe
   int32_t* counts;           // [plan_layout::kCountInts]: num_items, num_combine, num_empty, chunk_target, overflow
@@ -116,11 +115,7 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
   // grid has finished - the lengths it reads and the plan region it overwrites are then free.  Right after, it lets
   // the kernel behind it (the decode kernel of this step) have its blocks scheduled: they set themselves up on the
   // other SMs while this one block plans, and wait, inside, for this grid to finish before they read the plan.
-  // With `overlap` (the caller's promise that the kernel before this one does not write the lengths) the wait moves
-  // to the END: the plan is made while the previous step's decode kernel drains - all of its blocks have read their
-  // plan entries by the time this kernel may start, so the plan region is free - and the kernel then only waits for
-  // that grid to finish before it exits, which keeps the chain ordered for the decode kernel behind it.
-  if (!p.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   bool overflow = B > kDevPlanMax;
@@ -130,7 +125,6 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
       p.counts[L::kCntChunkTarget] = 0; p.counts[L::kCntOverflow] = 1;
       atomicOr(p.error_word, LIBRA_DEV_ERR_PLAN_OVERFLOW);
     }
-    if (p.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
     return;
   }
 
@@ -149,7 +143,6 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
       p.counts[L::kCntChunkTarget] = 0; p.counts[L::kCntOverflow] = 1;
       atomicOr(p.error_word, LIBRA_DEV_ERR_PLAN_OVERFLOW);
     }
-    if (p.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
     return;
   }
 #pragma unroll
@@ -212,7 +205,6 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
       p.counts[L::kCntChunkTarget] = int(base); p.counts[L::kCntOverflow] = 1;
       atomicOr(p.error_word, LIBRA_DEV_ERR_PLAN_OVERFLOW);
     }
-    if (p.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
     return;
   }
 
@@ -265,7 +257,6 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
     p.counts[L::kCntChunkTarget] = int(base);
     p.counts[L::kCntOverflow] = 0;
   }
-  if (p.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 }  // namespace libra

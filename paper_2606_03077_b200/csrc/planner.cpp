@@ -30,8 +30,14 @@ bool valid_params(const PlanParams& p) {
 }
 
 int64_t max_items(const PlanParams& p, int32_t num_kv_heads, int32_t max_batch) {
-  const int64_t slots = int64_t(p.n_sm) * p.ctas_per_sm * p.items_per_slot * (p.refine ? 2 : 1);
-  return 2 * ceil_div(slots, num_kv_heads) + max_batch;
+  const int64_t slots = int64_t(p.n_sm) * p.ctas_per_sm * p.items_per_slot;
+  const int64_t plain = 2 * ceil_div(slots, num_kv_heads) + max_batch;
+  if (!p.refine) return plain;
+  // a plan is made again for 2 * slots only when it had fewer than 1.5 waves of blocks, i.e. fewer than
+  // 1.5 * W / Hkv items, hence non-empty sequences
+  const int64_t wave = int64_t(p.n_sm) * p.ctas_per_sm;
+  const int64_t few = std::min<int64_t>(max_batch, (plan_layout::kRefineWavesNum * wave) / (plan_layout::kRefineWavesDen * num_kv_heads));
+  return std::max(plain, 2 * ceil_div(2 * slots, num_kv_heads) + few);
 }
 
 bool make_plan(const PlanParams& p, int32_t num_kv_heads, const int32_t* seq_lens, int32_t batch, HostPlan* out) {

@@ -39,7 +39,8 @@ bool make_plan(const PlanParams& p, int32_t num_kv_heads, const int32_t* seq_len
 
 // Upper bound of the number of work items for any batch <= max_batch:
 // n_b <= 2*cd(L_b, C) - 1 and C >= num_kv_heads*T/(W*items_per_slot) give sum n_b <= 2*cd(W*ips, Hkv) + B;
-// a refined plan is a plan for twice as many slots, so with `refine` the bound is taken for 2*W*ips.
+// a refined plan is a plan for 2*W*ips slots of a batch with fewer than 1.5*W/Hkv non-empty sequences (else it would
+// not have been refined): sum n_b <= 2*cd(2*W*ips, Hkv) + min(B, 1.5*W/Hkv).  The bound is the larger of the two.
 int64_t max_items(const PlanParams& p, int32_t num_kv_heads, int32_t max_batch);
 
 }  // namespace libra

@@ -232,50 +232,3 @@ def test_separate_combine_with_nothing_to_merge_keeps_the_chain_ordered(lib):
         results.append(bufs[0].cpu().numpy().copy())
         r.h.close()
     assert np.array_equal(results[0], results[1])
-
-
-def test_overlapped_planning_gives_the_same_steps(lib):
-    """libra_set_plan_overlap: the planning kernel reads the lengths while the previous step's decode kernel is still
-    draining.  A run of steps whose lengths and block tables change every step - written two kernels before the plan
-    call, so the promise holds - gives the bits of the same run without the overlap, and the oracle's values."""
-    import torch
-    dev = torch.device("cuda:0")
-    Hq, Hkv, d, B = 16, 4, 128, 6
-    steps = [[3000, 40, 1, 700, 2049, 16], [17, 4096, 900, 0, 333, 2500], [1, 1, 1, 1, 1, 1], [4000, 4000, 0, 0, 5, 64],
-             [640, 641, 639, 1, 2, 3]] * 3
-    ld = 4096 // 16
-    pool = 1200
-    rng = np.random.default_rng(5)
-    k = W.f32_to_bf16_bits(rng.standard_normal((pool, Hkv, 16, d), dtype=np.float32))
-    v = W.f32_to_bf16_bits(rng.standard_normal((pool, Hkv, 16, d), dtype=np.float32))
-    q = W.f32_to_bf16_bits(rng.standard_normal((B, Hq, d), dtype=np.float32))
-    bts = [W.draw_block_table(np.asarray(l, np.int32), pool, np.random.default_rng(i), ld=ld)[0] for i, l in enumerate(steps)]
-    dq, dk, dv = (H.to_dev(x, dev) for x in (q, k, v))
-    all_bt = torch.from_numpy(np.stack(bts)).to(dev)
-    all_len = torch.tensor(steps, dtype=torch.int32, device=dev)
-    results = []
-    for overlap in (False, True):
-        h = lib.Handle(Hq, Hkv, d, pool, B, ld, plan=lib.PlanParams(0, 2, 8, 256, 256, 64))
-        h.set_plan_overlap(overlap)
-        ws = torch.zeros(h.workspace_size(), dtype=torch.uint8, device=dev)
-        dbt = torch.full((B, ld), -1, dtype=torch.int32, device=dev)
-        dl = torch.zeros(B, dtype=torch.int32, device=dev)
-        outs = torch.zeros((len(steps), B, Hq, d), dtype=torch.int16, device=dev)
-        scratch = torch.zeros(1 << 20, dtype=torch.float32, device=dev)
-        st = torch.cuda.current_stream().cuda_stream
-        for i in range(len(steps)):      # no host synchronisation in the loop
-            dl.copy_(all_len[i])
-            dbt.copy_(all_bt[i])
-            scratch.add_(1.0)            # the kernel directly before the plan call: it does not touch the lengths
-            h.plan_device(dl.data_ptr(), B, ws.data_ptr(), ws.numel(), st)
-            h.decode_attn(dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dbt.data_ptr(), dl.data_ptr(), outs[i].data_ptr(), st)
-        torch.cuda.synchronize()
-        assert h.debug_error_word() == 0
-        results.append(outs.cpu().numpy().copy())
-        h.close()
-    assert np.array_equal(results[0], results[1])
-    for i in (0, 1, 3, len(steps) - 1):
-        ref, _ = O.paged_decode_attention(q, k, v, bts[i], np.asarray(steps[i], np.int32))
-        got = results[1][i].view(np.uint16).astype(np.uint32) << 16
-        got = got.view(np.float32).astype(np.float64)
-        assert gates.tight_violations(got, ref) == 0 and gates.stated_violations(got, ref) == 0, i

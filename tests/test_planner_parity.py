@@ -102,5 +102,7 @@ def test_item_bound_holds(lib):
         for refine in (0, 1):
             prm = P.PlanParams(n_sm=int(rng.choice([4, 148])), items_per_slot=int(rng.integers(1, 6)), refine=refine)
             pl = P.plan(lens, hkv, prm)
-            W_ = prm.n_sm * prm.ctas_per_sm * prm.items_per_slot * (2 if refine else 1)
-            assert len(pl.items) <= 2 * (-(-W_ // hkv)) + B
+            W_ = prm.n_sm * prm.ctas_per_sm * prm.items_per_slot
+            plain = 2 * (-(-W_ // hkv)) + B
+            few = min(B, (3 * prm.n_sm * prm.ctas_per_sm) // (2 * hkv))
+            assert len(pl.items) <= (max(plain, 2 * (-(-2 * W_ // hkv)) + few) if refine else plain)
