@@ -53,9 +53,9 @@ FALLBACK_HBM_GBS = 6650.0
 L2_BYTES_ASSUMED = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode launch divided by its algorithmic bytes, from the ncu
 # captures summarised under profiles/ (a constant of those captures, not something this run measures):
-# lognormal_b64 374.9 MB / 368.1 MB, straggler_b8 1078.1 MB / 1073.7 MB.  The large mix is too big to capture under
+# lognormal_b64 374.4 MB / 368.1 MB, straggler_b8 1078.0 MB / 1073.7 MB.  The large mix is too big to capture under
 # the profiler; its traffic is scaled from these (traffic grows with the pages read).
-NCU_TRAFFIC_OVER_ALGORITHMIC = {"lognormal_b64": 374.9e6 / 368.128e6, "straggler_b8": 1078.1e6 / 1073.741824e6}
+NCU_TRAFFIC_OVER_ALGORITHMIC = {"lognormal_b64": 374.4e6 / 368.128e6, "straggler_b8": 1078.0e6 / 1073.741824e6}
 
 
 # ----------------------------------------------------------------------------- clocks
