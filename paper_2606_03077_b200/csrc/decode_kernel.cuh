@@ -93,10 +93,6 @@ constexpr float kMaxSlack = LIBRA_MAX_SLACK;
 #ifndef LIBRA_SPLIT_P
 #define LIBRA_SPLIT_P 1
 #endif
-// > 0: first-wave blocks prefetch the look-ups of this many later blocks of their slot into L2 (see decode_kernel)
-#ifndef LIBRA_PREFETCH_NEXT
-#define LIBRA_PREFETCH_NEXT 0
-#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
@@ -153,11 +149,6 @@ __device__ __forceinline__ void tma_prefetch_l2_4d(const CUtensorMap* map, int c
                :
                : "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy)
                : "memory");
-}
-
-// Ask for one line of global memory to be brought into L2 (no destination, nothing to wait for).
-__device__ __forceinline__ void prefetch_l2(const void* ptr) {
-  asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr) : "memory");
 }
 
 // A 32-bit load that goes to L2, not through this SM's L1 (for memory another kernel may still be writing).
@@ -937,33 +928,6 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   else load_q_frags<D, NT>(qf, p, u.b, kvh, lane);
   for (int j = issued; j < pre; ++j) issue(j, j);
   if (threadIdx.x == 0) check_planned_length(p, u, len_dev);
-#if LIBRA_PREFETCH_NEXT
-  // A block of the first wave, once its own copies are on their way, asks for what the blocks that will follow on
-  // this SM's slot look up first - their block-table rows, their rows of q, their lengths - to be brought into L2:
-  // a few hundred bytes per unit, so that a later block's first look-ups are L2 hits instead of DRAM round trips
-  // (unlike prefetching K/V tiles, which competes with the copies that are needed now, this costs next to nothing).
-  if (blockIdx.x < sm_count()) {
-    const int n_sm = int(sm_count());
-    for (int j = 1; j <= LIBRA_PREFETCH_NEXT; ++j) {
-      const int blk = int(blockIdx.x) + j * n_sm;
-      if (blk >= num_units) break;
-      const int n_item = blk / p.num_kv_heads;
-      const int n_kvh = blk - n_item * p.num_kv_heads;
-      const Unit nu = decode_unit<NW>(entries[n_item], n_kvh, 0);
-      const int n_pages = (nu.kv_end - nu.kv_begin + 15) >> 4;
-      const char* row = reinterpret_cast<const char*>(p.block_table + int64_t(nu.b) * p.block_table_ld +
-                                                      (nu.first_page >> p.tile_shift));
-      const int row_bytes = ((n_pages >> p.tile_shift) + 1) * 4;
-      for (int off = int(threadIdx.x) * 128; off < row_bytes; off += NW * 32 * 128) prefetch_l2(row + off);
-      if (threadIdx.x < 2 * p.cols) {   // the unit's rows of q: cols rows of D * 2 bytes = 2 lines each at D = 128
-        const int c = threadIdx.x >> 1;
-        prefetch_l2(reinterpret_cast<const char*>(p.q + (int64_t(nu.b) * p.num_q_heads + col_row(p, n_kvh, c)) * D) +
-                    (threadIdx.x & 1) * 128);
-      }
-      if (threadIdx.x == 64) prefetch_l2(p.seq_lens + nu.b);
-    }
-  }
-#endif
 
   bool timed_out = false;
   int s = 0;
