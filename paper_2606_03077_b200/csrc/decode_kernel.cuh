@@ -93,6 +93,10 @@ constexpr float kMaxSlack = LIBRA_MAX_SLACK;
 #ifndef LIBRA_SPLIT_P
 #define LIBRA_SPLIT_P 1
 #endif
+// 1: with 9 - 16 score columns per KV head (bf16 cache) the columns are the M side of the tiles (process_page_rows)
+#ifndef LIBRA_ROWS_LAYOUT
+#define LIBRA_ROWS_LAYOUT 1
+#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
@@ -436,6 +440,179 @@ __device__ __forceinline__ void process_page(WarpAcc<D, NT>& st, const uint32_t 
   }
 }
 
+// ---- 9 to 16 score columns per KV head: the columns on the M side --------------------------------------
+// With more than 8 rows of q per KV head (a wide head group, or several query tokens) the tile shapes turn round: the
+// 16 rows of q are the M side of every mma, so
+//   S[16 cols x 16 tokens]  = Q . K_page^T      A = Q fragments (registers), B = K rows as ldmatrix delivers them
+//   O[16 cols x d]         += P . V_page        A = P, which is S's accumulator layout as it stands (no register
+//                                               transposes), B = V by ldmatrix.trans
+// A thread holds rows g and g + 8 of S: one running maximum and sum per row (two per thread instead of four), and a
+// row's maximum is two shuffles away (over the four lanes of a quad) instead of three.  The state lives in the same
+// WarpAcc<D, 2>: m[0][0] / m[0][1] (and l) are rows g / g + 8, acc[n / (D/16)][n % (D/16)] is the 8-dim slice n of O with
+// c0, c1 = row g, dims 8n + 2t, + 1 and c2, c3 = row g + 8.
+
+// Q fragments as the A operand, kept in qf[NT = 2][D / 16][2]: {qf[0][kk][0], qf[0][kk][1], qf[1][kk][0], qf[1][kk][1]}
+// = {row g dims 16kk + 2t.., row g + 8 same dims, row g dims 16kk + 8 + 2t.., row g + 8}; rows >= cols are zero.
+template <int D>
+__device__ __forceinline__ void load_q_frags_rows(uint32_t (&qf)[2][D / 16][2], const DecodeParams& p, int b, int kvh,
+                                                  int lane) {
+  const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+  for (int hi = 0; hi < 2; ++hi) {
+    const int row = g + 8 * hi;
+    const bool live = row < p.cols;
+    const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+        p.q + (int64_t(b) * p.num_q_heads + col_row(p, kvh, live ? row : 0)) * D);
+#pragma unroll
+    for (int kk = 0; kk < D / 16; ++kk) {
+      qf[0][kk][hi] = live ? __ldg(qrow + 8 * kk + t) : 0u;
+      qf[1][kk][hi] = live ? __ldg(qrow + 8 * kk + t + 4) : 0u;
+    }
+  }
+}
+
+// One page (16 tokens) of one KV head in that layout; same contract as process_page, `cut` per row: cut[0][0] for row
+// g, cut[0][1] for row g + 8.
+template <int D>
+__device__ __forceinline__ void process_page_rows(WarpAcc<D, 2>& st, const uint32_t (&qf)[2][D / 16][2], uint32_t kt,
+                                                  uint32_t vt, uint8_t* v_gen, int n_valid, float scale_log2, int lane,
+                                                  int n_common, int len_rel, const int (&cut)[2][2]) {
+  constexpr int KS = D / 16;
+  const int t = lane & 3;
+  const int k_row = lane & 15, k_sel = lane >> 4;
+  const int v_row = (lane & 7) + ((lane >> 4) << 3), v_sel = (lane >> 3) & 1;
+
+  if (n_valid < 16) {
+    // rows past the end may hold anything, NaN included: clear them in V so that 0 * garbage cannot leak
+    for (int i = lane; i < (16 - n_valid) * (D / 8); i += 32) {
+      const int r = n_valid + i / (D / 8);
+      const int c16 = i % (D / 8);
+      *reinterpret_cast<uint4*>(v_gen + ((c16 >> 3) << 11) + (r << 7) + ((c16 & 7) << 4)) = make_uint4(0, 0, 0, 0);
+    }
+    fence_proxy_async();  // these generic writes come before the next TMA write into this stage
+    __syncwarp();
+  }
+
+  // ---- S = Q . K^T: n-tile 0 = tokens 0 - 7, n-tile 1 = tokens 8 - 15; even and odd k-steps in separate accumulators
+  float sc[2][4], sc2[2][4];
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+    sc2[nt][0] = sc2[nt][1] = sc2[nt][2] = sc2[nt][3] = 0.f;
+  }
+#pragma unroll
+  for (int kk = 0; kk < KS; ++kk) {
+    uint32_t r[4];   // {tokens 0-7 dims lo, tokens 8-15 dims lo, tokens 0-7 dims hi, tokens 8-15 dims hi} of k-step kk
+    ldsm_x4(r, kt + tile_off(k_row, 2 * kk + k_sel));
+    const uint32_t a[4] = {qf[0][kk][0], qf[0][kk][1], qf[1][kk][0], qf[1][kk][1]};
+    if (kk & 1) {
+      mma_bf16(sc2[0], a, r[0], r[2]);
+      mma_bf16(sc2[1], a, r[1], r[3]);
+    } else {
+      mma_bf16(sc[0], a, r[0], r[2]);
+      mma_bf16(sc[1], a, r[1], r[3]);
+    }
+  }
+
+  // ---- online softmax; this thread holds rows g (e = 0, 1) and g + 8 (e = 2, 3) at tokens 8 nt + 2t, + 1
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) sc[nt][e] = (sc[nt][e] + sc2[nt][e]) * scale_log2;
+  }
+  if (n_common < 16) {
+    const int nv0 = min(n_valid, len_rel - cut[0][0]), nv1 = min(n_valid, len_rel - cut[0][1]);
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+      const int tok = 8 * nt + 2 * t;
+      if (tok >= nv0) sc[nt][0] = -INFINITY;
+      if (tok + 1 >= nv0) sc[nt][1] = -INFINITY;
+      if (tok >= nv1) sc[nt][2] = -INFINITY;
+      if (tok + 1 >= nv1) sc[nt][3] = -INFINITY;
+    }
+  }
+  float mx0 = fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1]));
+  float mx1 = fmaxf(fmaxf(sc[0][2], sc[0][3]), fmaxf(sc[1][2], sc[1][3]));
+#pragma unroll
+  for (int off = 1; off <= 2; off <<= 1) {
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+  }
+  const bool grew = (mx0 > st.m[0][0] + kMaxSlack) || (mx1 > st.m[0][1] + kMaxSlack);
+  if (__any_sync(0xffffffffu, grew)) {
+    const float m0 = fmaxf(st.m[0][0], mx0), m1 = fmaxf(st.m[0][1], mx1);
+    const float f0 = ex2(st.m[0][0] - m0), f1 = ex2(st.m[0][1] - m1);
+    st.l[0][0] *= f0;
+    st.l[0][1] *= f1;
+#pragma unroll
+    for (int n = 0; n < D / 8; ++n) {
+      st.acc[n / KS][n % KS][0] *= f0;
+      st.acc[n / KS][n % KS][1] *= f0;
+      st.acc[n / KS][n % KS][2] *= f1;
+      st.acc[n / KS][n % KS][3] *= f1;
+    }
+    st.m[0][0] = m0;
+    st.m[0][1] = m1;
+  }
+  // P as the A operand of the second product: {row g tokens 2t.., row g + 8 tokens 2t.., row g tokens 8 + 2t.., row g + 8}
+  uint32_t pa[4], pr[4];
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    const float p0 = ex2(sc[nt][0] - st.m[0][0]), p1 = ex2(sc[nt][1] - st.m[0][0]);
+    const float p2 = ex2(sc[nt][2] - st.m[0][1]), p3 = ex2(sc[nt][3] - st.m[0][1]);
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(p0, p1), hi = __floats2bfloat162_rn(p2, p3);
+    const uint32_t ulo = *reinterpret_cast<const uint32_t*>(&lo), uhi = *reinterpret_cast<const uint32_t*>(&hi);
+    pa[2 * nt] = ulo;
+    pa[2 * nt + 1] = uhi;
+    // the residue of the rounding as a second bf16 term (see process_page)
+    const __nv_bfloat162 lo2 = __floats2bfloat162_rn(p0 - __uint_as_float(ulo << 16), p1 - __uint_as_float(ulo & 0xffff0000u));
+    const __nv_bfloat162 hi2 = __floats2bfloat162_rn(p2 - __uint_as_float(uhi << 16), p3 - __uint_as_float(uhi & 0xffff0000u));
+    pr[2 * nt] = *reinterpret_cast<const uint32_t*>(&lo2);
+    pr[2 * nt + 1] = *reinterpret_cast<const uint32_t*>(&hi2);
+    st.l[0][0] += p0 + p1;
+    st.l[0][1] += p2 + p3;
+  }
+
+  // ---- O += P . V: one ldmatrix.trans feeds two 8-dim slices
+#pragma unroll
+  for (int mt = 0; mt < KS; ++mt) {
+    uint32_t r[4];   // {tokens 0-7 dims 16mt.., tokens 0-7 dims 16mt + 8.., tokens 8-15 dims 16mt.., tokens 8-15 dims 16mt + 8..}
+    ldsm_x4_trans(r, vt + tile_off(v_row, 2 * mt + v_sel));
+    float (&o0)[4] = st.acc[(2 * mt) / KS][(2 * mt) % KS];
+    float (&o1)[4] = st.acc[(2 * mt + 1) / KS][(2 * mt + 1) % KS];
+    mma_bf16(o0, pa, r[0], r[2]);
+    mma_bf16(o1, pa, r[1], r[3]);
+    mma_bf16(o0, pr, r[0], r[2]);
+    mma_bf16(o1, pr, r[1], r[3]);
+  }
+}
+
+// That layout's result -> shared memory, in the form merge_and_write reads: stats per row, O as [row][dim] fp32 with
+// the dim index XORed with stage_swizzle(row).
+template <int D>
+__device__ __forceinline__ void stage_warp_result_rows(WarpAcc<D, 2>& st, float* o_sm, float* m_sm, float* l_sm, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+  for (int off = 1; off <= 2; off <<= 1) {   // l is spread over the four lanes of a quad
+    st.l[0][0] += __shfl_xor_sync(0xffffffffu, st.l[0][0], off);
+    st.l[0][1] += __shfl_xor_sync(0xffffffffu, st.l[0][1], off);
+  }
+  if (t == 0) {
+    m_sm[g] = st.m[0][0];
+    m_sm[g + 8] = st.m[0][1];
+    l_sm[g] = st.l[0][0];
+    l_sm[g + 8] = st.l[0][1];
+  }
+  const int sw0 = ((g >> 1) & 3) << 3;   // = stage_swizzle(g) = stage_swizzle(g + 8)
+#pragma unroll
+  for (int n = 0; n < D / 8; ++n) {
+    const float (&o)[4] = st.acc[n / (D / 16)][n % (D / 16)];
+    const int d0 = (8 * n + 2 * t) ^ sw0;   // the XOR moves whole groups of 8 dims: the pair stays together
+    *reinterpret_cast<float2*>(o_sm + g * D + d0) = make_float2(o[0], o[1]);
+    *reinterpret_cast<float2*>(o_sm + (g + 8) * D + d0) = make_float2(o[2], o[3]);
+  }
+}
+
 // ---- 8-bit (E4M3) cache ---------------------------------------------------------------------------
 // A tile is 16 tokens x D bytes: rows of 128 bytes with the 128-byte swizzle (head_dim 128) or rows of 64 bytes
 // with the 64-byte swizzle (head_dim 64).  ldmatrix moves it as 16-bit units, i.e.
@@ -750,6 +927,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
     p.v_new = nullptr;
   }
   using SM = DecodeSmem<D, NW, STAGES, kFp8 ? 1 : 2>;
+  constexpr bool kRows = LIBRA_ROWS_LAYOUT && NT == 2 && !kFp8 && !kLoadsOnly;   // two column tiles of a bf16 cache: columns on the M side
   constexpr int NH = kFp8 ? 1 : D / 64;   // 128-byte column blocks of a row
   static_assert(NT * 8 * D * 4 <= SM::kWarpBytes, "epilogue staging must fit in the warp's ring");
 
@@ -878,7 +1056,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
-      const int c = nt * 8 + 2 * (lane & 3) + e;
+      // (two column tiles of a bf16 cache: the columns are rows g and g + 8 of the score tile, kept in cut[0][.])
+      const int c = kRows ? (lane >> 2) + 8 * e : nt * 8 + 2 * (lane & 3) + e;
       cut[nt][e] = (p.q_len > 1 && c < p.cols) ? p.q_len - 1 - c / p.group : 0;
     }
   }
@@ -925,6 +1104,7 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
   }
   uint32_t qf[NT][D / 16][2];
   if constexpr (kFp8) load_q_frags_fp8<D, NT>(qf, p, u.b, kvh, lane);
+  else if constexpr (kRows) load_q_frags_rows<D>(qf, p, u.b, kvh, lane);
   else load_q_frags<D, NT>(qf, p, u.b, kvh, lane);
   for (int j = issued; j < pre; ++j) issue(j, j);
   if (threadIdx.x == 0) check_planned_length(p, u, len_dev);
@@ -978,6 +1158,9 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
       if constexpr (kFp8) {
         process_page_fp8<D, NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes,
                              u.kv_end - tok0, p.scale_log2, lane, common_end - tok0, len_dev - tok0, cut);
+      } else if constexpr (kRows) {
+        process_page_rows<D>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes,
+                             u.kv_end - tok0, p.scale_log2, lane, common_end - tok0, len_dev - tok0, cut);
       } else {
         process_page<D, NT>(st, qf, kt, kt + SM::kTileBytes, my_ring + s * SM::kStageBytes + SM::kTileBytes,
                             u.kv_end - tok0, p.scale_log2, lane, common_end - tok0, len_dev - tok0, cut);
@@ -1006,7 +1189,8 @@ decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__
 
   // ---- stage (m, l, O) of this warp in its own, now idle, ring; merge the warps; write
   __syncwarp();
-  stage_warp_result<D, NT, kFp8>(st, reinterpret_cast<float*>(my_ring), stat_m[warp], stat_l[warp], lane);
+  if constexpr (kRows) stage_warp_result_rows<D>(st, reinterpret_cast<float*>(my_ring), stat_m[warp], stat_l[warp], lane);
+  else stage_warp_result<D, NT, kFp8>(st, reinterpret_cast<float*>(my_ring), stat_m[warp], stat_l[warp], lane);
   __syncthreads();
   merge_and_write<D, NT, NW>(p, u, reinterpret_cast<const float*>(ring), SM::kWarpBytes / 4, &stat_m[0][0], &stat_l[0][0],
                              threadIdx.x, NW * 32);
