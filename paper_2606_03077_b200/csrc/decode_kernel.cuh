@@ -9,11 +9,13 @@
 //            complete on the stage's mbarrier; up to STAGES pages per warp are in flight
 //   warp   : S^T[16 tokens x 8 heads]  = K_page . Q^T       mma.sync m16n8k16 bf16 -> fp32
 //            online softmax in fp32 (running max m and sum l per head, base-2 exponent)
-//            O^T[d x 8 heads]         += V_page^T . P^T     P rounded to bf16, l sums the rounded P
+//            O^T[d x 8 heads]         += V_page^T . P^T     P as two bf16 terms (head + rounding residue)
 //
 // Tokens are the M side of the tiles, the (padded) head group the N side, so a group of up to
-// 8 heads costs one 8-wide tile and nothing is wasted on padding rows.  The kernel is bound by
-// the HBM read of K and V: 2 * head_dim * 2 bytes per token per KV head, 4 * G * head_dim flop.
+// 8 heads costs one 8-wide tile and nothing is wasted on padding rows; with 9 to 16 rows of q per KV
+// head (a wider group, or several query tokens) the rows of q take the M side instead (process_page_rows).
+// The kernel is bound by the HBM read of K and V: 2 * head_dim * 2 bytes per token per KV head,
+// 4 * G * head_dim flop.
 //
 // The warps never synchronise with each other while they stream pages; they merge their (m, l, O)
 // in shared memory once per unit, in warp order, so results are bit-reproducible.
