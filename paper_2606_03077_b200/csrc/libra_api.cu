@@ -195,6 +195,7 @@ struct libra_handle_s {
   void* last_stream = nullptr;
   bool device_planned = false;  // the last plan was made by the device-side planner: counts live in the workspace
   int64_t decodes_on_plan = 0;  // decode launches enqueued since the last plan call
+  int32_t dev_item_bound = 0;   // device-side plan: the most work items the planned batch can have (sizes the grids)
   int32_t planned_batch = 0;
   size_t dev_counts_off = 0, dev_per_seq_off = 0, dev_entries_off = 0, dev_fixes_off = 0;
   std::vector<int32_t> export_scratch;
@@ -496,7 +497,7 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
     }
     if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
     e = cudaFuncSetAttribute(reinterpret_cast<const void*>(libra::plan_kernel), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             int(libra::plan_kernel_smem_bytes()));
+                             int(libra::plan_kernel_smem_bytes(libra::kDevPlanThreads)));
     if (e != cudaSuccess) { status = fail_cuda(h, e); break; }
 
     compute_layout(h);
@@ -657,7 +658,10 @@ int libra_plan_device(libra_handle_t h, const int32_t* seq_lens_dev, int32_t bat
   p.max_splits = h->params.max_splits;
   p.wave_slots = int64_t(h->params.n_sm) * h->params.ctas_per_sm;
   p.refine = h->params.refine;
-  p.max_items = int32_t(std::min<int64_t>(h->max_items, libra::kDevPlanMax));
+  const int64_t item_bound = std::min<int64_t>(libra::max_items(h->params, h->cfg.num_kv_heads, batch), h->max_items);
+  p.max_items = int32_t(std::min<int64_t>(item_bound, libra::kDevPlanMax));
+  const int threads = libra::plan_kernel_threads(batch, p.max_items);
+  h->dev_item_bound = p.max_items;
   p.max_len = int32_t(std::min<int64_t>(int64_t(h->cfg.block_table_ld) * h->cfg.page_size, 0x7fffffff));
   p.counts = reinterpret_cast<int32_t*>(ws + h->dev_counts_off);
   p.per_seq = reinterpret_cast<int32_t*>(ws + h->dev_per_seq_off);
@@ -667,8 +671,8 @@ int libra_plan_device(libra_handle_t h, const int32_t* seq_lens_dev, int32_t bat
   {
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(1);
-    lc.blockDim = dim3(libra::kDevPlanThreads);
-    lc.dynamicSmemBytes = libra::plan_kernel_smem_bytes();
+    lc.blockDim = dim3(unsigned(threads));
+    lc.dynamicSmemBytes = libra::plan_kernel_smem_bytes(threads);
     lc.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -898,10 +902,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
   // (a device plan: one block at the end of the grid zeroes the rows of all empty sequences)
   const int32_t n_empty = h->device_planned ? 1 : int32_t(h->plan.empty.size());
   const int32_t n_combine = h->device_planned ? h->planned_batch : int32_t(h->plan.combine.size());
-  const int32_t n_items_bound =
-      h->device_planned ? int32_t(std::min<int64_t>(libra::max_items(h->params, h->cfg.num_kv_heads, h->planned_batch),
-                                                    libra::kDevPlanMax))
-                        : h->num_items;
+  const int32_t n_items_bound = h->device_planned ? h->dev_item_bound : h->num_items;
   const int32_t n_units = n_items_bound * h->cfg.num_kv_heads;
   if (n_units > 0 || n_empty > 0) {
     DecodeParams p;

@@ -10,21 +10,24 @@
 //   a plan of fewer than one and a half waves of long blocks is made again for twice as many slots (plan_layout.hpp)
 //
 // Integer arithmetic only; the result must equal the host planner's bit for bit.  Limits: batch and
-// work items <= kDevPlanMax each (one block, four elements per thread); beyond that, or when a length
+// work items <= kDevPlanMax each (one block of up to 1024 threads, four elements per thread; the block is sized to the
+// batch, because its barriers and scans are what its time is made of); beyond that, or when a length
 // exceeds what a block-table row can describe, the kernel writes an empty plan and sets
 // LIBRA_DEV_ERR_PLAN_OVERFLOW.  Negative lengths count as empty sequences.
 #pragma once
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdint>
 
 #include "plan_layout.hpp"
 
 namespace libra {
 
-constexpr int kDevPlanThreads = 1024;
+constexpr int kDevPlanThreads = 1024;   // the most threads one planning block has
 constexpr int kDevPlanPerThread = 4;
 constexpr int kDevPlanMax = kDevPlanThreads * kDevPlanPerThread;
+constexpr int kDevPlanArrays = 8;       // shared-memory arrays of kDevPlanPerThread * blockDim.x ints each
 
 struct PlanKernelParams {
   const int32_t* seq_lens;   // device, [batch]
@@ -43,12 +46,24 @@ struct PlanKernelParams {
   uint32_t* error_word;
 };
 
+// Threads of the planning block for a batch and an item bound: every thread owns up to kDevPlanPerThread elements
+// of each array; a small batch gets a small block (its barriers and scans are what the kernel's time is made of).
+inline int plan_kernel_threads(int64_t batch, int64_t item_bound) {
+  // one element per thread where that fits in a block (the ranking step is quadratic in the items), never fewer
+  // threads than the arrays need
+  const int64_t n = std::max<int64_t>(std::max(batch, item_bound), 1);
+  return int(std::min<int64_t>(kDevPlanThreads, std::max<int64_t>(128, (n + 31) / 32 * 32)));
+}
+inline size_t plan_kernel_smem_bytes(int threads) {
+  return size_t(kDevPlanArrays) * kDevPlanPerThread * threads * sizeof(int);
+}
+
 namespace dev {
 
-// Exclusive scan of `n` ints in shared memory (n <= kDevPlanMax), in place; returns the total.
-// `warp_tot` is scratch for 32 ints.  All threads of the block call it.
+// Exclusive scan of `n` ints in shared memory (n <= kDevPlanPerThread * blockDim.x), in place; returns the total.
+// `warp_tot` is scratch for 33 ints.  All threads of the block call it.
 __device__ __forceinline__ int block_exclusive_scan(int* data, int n, int* warp_tot) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_warps = blockDim.x >> 5;
   int v[kDevPlanPerThread];
   int sum = 0;
 #pragma unroll
@@ -66,7 +81,7 @@ __device__ __forceinline__ int block_exclusive_scan(int* data, int n, int* warp_
   if (lane == 31) warp_tot[warp] = incl;
   __syncthreads();
   if (warp == 0) {
-    int w = warp_tot[lane];
+    int w = (lane < n_warps) ? warp_tot[lane] : 0;
     int wi = w;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -89,24 +104,31 @@ __device__ __forceinline__ int block_exclusive_scan(int* data, int n, int* warp_
   return total;
 }
 
+// ceil(a / b) for 0 <= a < 2^31 and b >= 1 (b may exceed 32 bits: then the quotient is 0 or 1)
+__device__ __forceinline__ int ceil_div_len(int a, long long b) {
+  if (b > 0x7fffffffll) return a > 0 ? 1 : 0;
+  const unsigned ub = unsigned(b);
+  return int((unsigned(a) + ub - 1u) / ub);
+}
+
 }  // namespace dev
 
-// grid = 1 block of kDevPlanThreads threads; dynamic shared memory = plan_kernel_smem_bytes()
-constexpr size_t plan_kernel_smem_bytes() { return size_t(7) * kDevPlanMax * sizeof(int); }
-
+// grid = 1 block of plan_kernel_threads(batch, item bound) threads; dynamic shared memory = plan_kernel_smem_bytes(threads)
 __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelParams p) {
   extern __shared__ int sm[];
-  int* nsplit = sm;                      // [batch]
-  int* chunk = sm + kDevPlanMax;         // [batch]
-  int* offs = sm + 2 * kDevPlanMax;      // [batch] exclusive scan of nsplit
-  int* aux = sm + 3 * kDevPlanMax;       // [batch] flags / their scans
-  int* it_len = sm + 4 * kDevPlanMax;    // [items]
-  int* it_b = sm + 5 * kDevPlanMax;      // [items]
-  int* it_j = sm + 6 * kDevPlanMax;      // [items]
+  const int cap = kDevPlanPerThread * int(blockDim.x);
+  int* len_s = sm;                // [batch] lengths (negative ones taken as 0)
+  int* nsplit = sm + cap;         // [batch]
+  int* chunk = sm + 2 * cap;      // [batch]
+  int* offs = sm + 3 * cap;       // [batch] exclusive scan of nsplit
+  int* aux = sm + 4 * cap;        // [batch] flags / their scans
+  int* it_len = sm + 5 * cap;     // [items]
+  int* it_b = sm + 6 * cap;       // [items]
+  int* it_j = sm + 7 * cap;       // [items]
   __shared__ int warp_tot[33];
-  __shared__ long long s_total;
+  __shared__ long long warp_sum[32];
 
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, nthr = blockDim.x;
   const int B = p.batch;
   namespace L = plan_layout;
 
@@ -118,38 +140,36 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-  bool overflow = B > kDevPlanMax;
-  if (overflow) {
+  auto refuse = [&](int base_out) {
     if (tid == 0) {
       p.counts[L::kCntItems] = 0; p.counts[L::kCntCombine] = 0; p.counts[L::kCntEmpty] = 0;
-      p.counts[L::kCntChunkTarget] = 0; p.counts[L::kCntOverflow] = 1;
+      p.counts[L::kCntChunkTarget] = base_out; p.counts[L::kCntOverflow] = 1;
       atomicOr(p.error_word, LIBRA_DEV_ERR_PLAN_OVERFLOW);
     }
+  };
+  if (B > cap) {   // more sequences than this block was sized for
+    refuse(0);
     return;
   }
 
-  // ---- T = sum of lengths
-  if (tid == 0) s_total = 0;
-  __syncthreads();
+  // ---- the lengths, once, into shared memory; T = their sum
   long long part = 0;
   int too_long = 0;
-  for (int b = tid; b < B; b += kDevPlanThreads) {
-    part += max(p.seq_lens[b], 0);
-    too_long |= (p.seq_lens[b] > p.max_len) ? 1 : 0;
-  }
-  if (__syncthreads_or(too_long)) {  // a length the block table cannot hold: refuse the whole batch
-    if (tid == 0) {
-      p.counts[L::kCntItems] = 0; p.counts[L::kCntCombine] = 0; p.counts[L::kCntEmpty] = 0;
-      p.counts[L::kCntChunkTarget] = 0; p.counts[L::kCntOverflow] = 1;
-      atomicOr(p.error_word, LIBRA_DEV_ERR_PLAN_OVERFLOW);
-    }
-    return;
+  for (int b = tid; b < B; b += nthr) {
+    const int len = p.seq_lens[b];
+    too_long |= (len > p.max_len) ? 1 : 0;
+    len_s[b] = max(len, 0);
+    part += max(len, 0);
   }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
-  if ((tid & 31) == 0 && part) atomicAdd(reinterpret_cast<unsigned long long*>(&s_total), (unsigned long long)part);
-  __syncthreads();
-  const long long T = s_total;
+  if ((tid & 31) == 0) warp_sum[tid >> 5] = part;
+  if (__syncthreads_or(too_long)) {  // a length the block table cannot hold: refuse the whole batch
+    refuse(0);
+    return;
+  }
+  long long T = 0;
+  for (int w = 0; w < (nthr >> 5); ++w) T += warp_sum[w];
   const long long A = p.chunk_align;
   long long base = (p.heads * T + p.slots - 1) / p.slots;
   base = (base + A - 1) / A * A;
@@ -158,23 +178,30 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
   // ---- per sequence: degree, chunk length, chunk count; twice if the first plan is coarse
   int n_items = 0;
   for (int pass = 0; pass < 2; ++pass) {
-    for (int b = tid; b < B; b += kDevPlanThreads) {
-      const long long len = max(p.seq_lens[b], 0);
+    for (int b = tid; b < B; b += nthr) {
+      const int len = len_s[b];
       int bucket = -1, n = 0, c = 0;
       if (len > 0) {
-        long long deg = 1;
-        const long long want = (len + base - 1) / base;
-        while (deg < want) deg <<= 1;
-        if (base < plan_layout::kSmallBaseTokens && deg > 1 &&
-            len * plan_layout::kGeoMeanDen < (deg / 2) * base * plan_layout::kGeoMeanNum) {
-          deg >>= 1;   // short chunks: the nearer power of two
-        }
-        if (deg > p.max_splits) deg = p.max_splits;
-        const long long ch = ((len + deg - 1) / deg + A - 1) / A * A;
-        n = int((len + ch - 1) / ch);
-        c = int(ch);
+        const int want = dev::ceil_div_len(len, base);
+        int deg = 1;
         bucket = 0;
-        while ((1ll << bucket) < deg) ++bucket;
+        while (deg < want) {
+          deg <<= 1;
+          ++bucket;
+        }
+        if (base < plan_layout::kSmallBaseTokens && deg > 1 &&
+            (long long)len * plan_layout::kGeoMeanDen < (long long)(deg / 2) * base * plan_layout::kGeoMeanNum) {
+          deg >>= 1;   // short chunks: the nearer power of two
+          --bucket;
+        }
+        while (deg > p.max_splits) {
+          deg >>= 1;
+          --bucket;
+        }
+        const unsigned a = unsigned(A);
+        const unsigned per = (unsigned(len) + unsigned(deg) - 1u) >> bucket;   // ceil(len / deg), deg = 2^bucket
+        c = int((per + a - 1u) / a * a);
+        n = int((unsigned(len) + unsigned(c) - 1u) / unsigned(c));
       }
       nsplit[b] = n;
       chunk[b] = c;
@@ -192,40 +219,31 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
     base = (base + A - 1) / A * A;
     if (base < p.min_chunk) base = p.min_chunk;
   }
-  for (int b = tid; b < B; b += kDevPlanThreads) {
+  for (int b = tid; b < B; b += nthr) {
     p.per_seq[B + b] = nsplit[b];
     p.per_seq[2 * B + b] = chunk[b];
     p.per_seq[3 * B + b] = offs[b];
   }
 
-  overflow = n_items > kDevPlanMax || n_items > p.max_items;
-  if (overflow) {
-    if (tid == 0) {
-      p.counts[L::kCntItems] = 0; p.counts[L::kCntCombine] = 0; p.counts[L::kCntEmpty] = 0;
-      p.counts[L::kCntChunkTarget] = int(base); p.counts[L::kCntOverflow] = 1;
-      atomicOr(p.error_word, LIBRA_DEV_ERR_PLAN_OVERFLOW);
-    }
+  if (n_items > cap || n_items > p.max_items) {
+    refuse(int(base));
     return;
   }
 
-  // ---- merges (n_b > 1) and empty sequences, each in batch order
-  for (int b = tid; b < B; b += kDevPlanThreads) aux[b] = nsplit[b] > 1 ? 1 : 0;
+  // ---- merges (n_b > 1) and empty sequences, each in batch order: one scan counts both (16 bits each)
+  for (int b = tid; b < B; b += nthr) aux[b] = (nsplit[b] > 1 ? 1 : 0) | (nsplit[b] == 0 ? (1 << 16) : 0);
   __syncthreads();
-  const int n_combine = dev::block_exclusive_scan(aux, B, warp_tot);
-  for (int b = tid; b < B; b += kDevPlanThreads) {
-    if (nsplit[b] > 1) p.fixes[aux[b]] = make_int4(b, offs[b], nsplit[b], p.seq_lens[b]);
-  }
-  __syncthreads();
-  for (int b = tid; b < B; b += kDevPlanThreads) aux[b] = (nsplit[b] == 0) ? 1 : 0;
-  __syncthreads();
-  const int n_empty = dev::block_exclusive_scan(aux, B, warp_tot);
-  for (int b = tid; b < B; b += kDevPlanThreads) {
-    if (nsplit[b] == 0) p.entries[n_items + aux[b]] = make_int4(b, 0, 0, 0);
+  const int both = dev::block_exclusive_scan(aux, B, warp_tot);
+  const int n_combine = both & 0xffff, n_empty = both >> 16;
+  for (int b = tid; b < B; b += nthr) {
+    if (nsplit[b] > 1) p.fixes[aux[b] & 0xffff] = make_int4(b, offs[b], nsplit[b], len_s[b]);
+    if (nsplit[b] == 0) p.entries[n_items + (aux[b] >> 16)] = make_int4(b, 0, 0, 0);
   }
 
-  // ---- items in (b, j) order
-  for (int b = tid; b < B; b += kDevPlanThreads) {
-    const int len = p.seq_lens[b];
+  // ---- items in (b, j) order (the list is padded to a multiple of four with lengths that rank after everything)
+  if (tid < 4 && (n_items & ~3) + tid >= n_items && (n_items & ~3) + tid < cap) it_len[(n_items & ~3) + tid] = -1;
+  for (int b = tid; b < B; b += nthr) {
+    const int len = len_s[b];
     for (int j = 0; j < nsplit[b]; ++j) {
       const int i = offs[b] + j;
       const int lo = j * chunk[b];
@@ -238,12 +256,19 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
   __syncthreads();
 
   // ---- longest first, ties in (b, j) order: the rank of item i is the number of items before it
-  for (int i = tid; i < n_items; i += kDevPlanThreads) {
+  const int4* len4 = reinterpret_cast<const int4*>(it_len);
+  const int n_quads = (n_items + 3) >> 2;
+  for (int i = tid; i < n_items; i += nthr) {
     const int len = it_len[i];
     int rank = 0;
-    for (int k = 0; k < n_items; ++k) {
-      const int lk = it_len[k];
-      rank += (lk > len || (lk == len && k < i)) ? 1 : 0;
+#pragma unroll 4
+    for (int k4 = 0; k4 < n_quads; ++k4) {   // four lengths per load, independent of each other: the loop is not a chain of loads
+      const int4 x = len4[k4];
+      const int k = 4 * k4;
+      rank += (x.x > len || (x.x == len && k < i)) ? 1 : 0;
+      rank += (x.y > len || (x.y == len && k + 1 < i)) ? 1 : 0;
+      rank += (x.z > len || (x.z == len && k + 2 < i)) ? 1 : 0;
+      rank += (x.w > len || (x.w == len && k + 3 < i)) ? 1 : 0;
     }
     const int b = it_b[i], j = it_j[i];
     const int lo = j * chunk[b];
