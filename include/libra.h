@@ -195,9 +195,10 @@ int libra_set_dependent_launch(libra_handle_t handle, int32_t on);
  * depend on it: an id that the preceding kernel had not yet written only warms the wrong lines, and a line written
  * after it was warmed is updated in L2, where the copies read.  It needs no promise from the caller (unlike
  * libra_set_early_prefetch) but it does read block_table - as a hint - while the preceding kernel may still be writing
- * it, which a memory checker reports; on = 0 switches it off.  Worth 2 % on a 55 us step, nothing on long ones. */
+ * it, which a memory checker reports; on = 0 switches it off.  Worth 2 % on a 55 us step, nothing on long ones.
+ * A plan that lies in the workspace (made by libra_plan_device, or too large for the kernel parameters) is warmed
+ * from the second decode call on it onwards: the kernel or copy that wrote it is then known to have finished. */
 int libra_set_cache_warmup(libra_handle_t handle, int32_t on);
-
 
 /* Optional second output.  With a non-NULL lse_dev every later decode call (libra_decode_attn, _append, _multi,
  * _static) also writes, for every row of q, the natural logarithm of the sum of its exponentiated scores,
@@ -234,8 +235,14 @@ int libra_set_combine_mode(libra_handle_t handle, int32_t mode);
  *             costs ~4 us whatever its length, so fewer and longer items win there)
  *   s_b     = min(s_b, max_splits)                       bucket_b = log2 s_b
  *   chunk_b = au(cd(L_b, s_b), chunk_align)              n_b = cd(L_b, chunk_b)
+ *   if refine and C >= 4096 and 2 * num_kv_heads * sum n_b < 3 * W   (fewer than one and a half waves of long blocks:
+ *             the tail end of a rollout, a few long stragglers; so few blocks cannot pull the memory bandwidth):
+ *             C = max(min_chunk, au(cd(num_kv_heads * T, 2 * W * items_per_slot), chunk_align)) and s_b, chunk_b, n_b
+ *             are computed again with it
  *   items   = (b, j, j*chunk_b, min(L_b, (j+1)*chunk_b)) sorted by (length desc, b asc, j asc)
- * params->n_sm must be > 0 here.  All outputs are caller-allocated host arrays: the per-sequence
+ * The number of items never exceeds max(2 * cd(W * items_per_slot, num_kv_heads) + batch,
+ * 2 * cd(2 * W * items_per_slot, num_kv_heads) + min(batch, 3 * W / (2 * num_kv_heads))) (the second term only with
+ * refine), which is what the workspace is sized for.  params->n_sm must be > 0 here.  All outputs are caller-allocated host arrays: the per-sequence
  * arrays hold `batch` entries, `items` holds items_capacity*4 entries.  Errors: INVALID_ARGUMENT
  * (null, negative length, bad params), WORKSPACE_TOO_SMALL (items_capacity too small; *num_items
  * then holds the number needed). */
@@ -265,7 +272,9 @@ int libra_plan(libra_handle_t handle, const int32_t* seq_lens_host, int32_t batc
  * Limits: batch <= 4096 (UNSUPPORTED_SHAPE otherwise); at most 4096 work items and no length beyond
  * block_table_ld * page_size, else the plan is empty and LIBRA_ERR_PLAN_OVERFLOW is set in the device error
  * word (checked on the device, since the host does not see the lengths).  The result equals
- * libra_plan's bit for bit (libra_plan_export reads it back).
+ * libra_plan's bit for bit (libra_plan_export reads it back).  The planning kernel is one more kernel on the stream's
+ * critical path (about 6 us for 64 sequences, 8.5 us for 256); one plan serves any number of decode calls on the same
+ * lengths - the attention layers of one generated token - so per call the cost is a fraction of that.
  * Errors: INVALID_ARGUMENT, WORKSPACE_TOO_SMALL, UNSUPPORTED_SHAPE, CUDA_ERROR. */
 int libra_plan_device(libra_handle_t handle, const int32_t* seq_lens_dev, int32_t batch, void* workspace_dev,
                       size_t workspace_bytes, void* stream);
