@@ -720,6 +720,77 @@ def short_batch_measure(rep: Replica, steps: int = 100):
     return res
 
 
+def few_long_measure(rep: Replica, steps: int = 40, regions: int = 5):
+    """The tail end of a rollout: a few long stragglers are all that is still decoding.  Batches of 3 to 26 sequences
+    of 12K - 40K tokens, planned with and without the planner's second pass (a plan of fewer than one and a half waves
+    of long blocks is made again for twice as many slots), on pools of their own (1.2 M tokens, block tables rotated
+    over as many placements as fit)."""
+    torch, w = rep.torch, rep.w
+    if w.head_dim != 128 or w.num_kv_heads != 8:
+        return None
+    from numpy.random import Generator, PCG64
+    rng = Generator(PCG64(0))
+    pool_pages = 75000
+    k = torch.randn((pool_pages, 8, 16, 128), device=rep.dev, dtype=torch.bfloat16)
+    v = torch.randn((pool_pages, 8, 16, 128), device=rep.dev, dtype=torch.bfloat16)
+    st = torch.cuda.current_stream().cuda_stream
+    batches = {"12 x 20000": np.full(12, 20000), "20 x 12000": np.full(20, 12000), "6 x 30000": np.full(6, 30000),
+               "3 x 40000": np.full(3, 40000), "8 x U[16K,32K]": rng.integers(16384, 32769, 8),
+               "26 x U[16K,32K]": rng.integers(16384, 32769, 26), "8 x 32768": np.full(8, 32768),
+               "32 x 8192": np.full(32, 8192)}
+    res = []
+    for name, lens in batches.items():
+        lens = lens.astype(np.int32)
+        Bn = len(lens)
+        npg = (lens.astype(np.int64) + 15) // 16
+        need = int(npg.sum())
+        copies = max(1, min(8, pool_pages // need))
+        ld = int(npg.max())
+        perm = rng.permutation(pool_pages)
+        bts = []
+        for c in range(copies):
+            bt = np.full((Bn, ld), -1, np.int32)
+            pos = c * need
+            for b in range(Bn):
+                bt[b, :npg[b]] = perm[pos:pos + npg[b]]
+                pos += npg[b]
+            bts.append(torch.from_numpy(bt).to(rep.dev))
+        dl = torch.from_numpy(lens).to(rep.dev)
+        q = torch.randn((Bn, w.num_q_heads, 128), device=rep.dev, dtype=torch.bfloat16)
+        out = torch.zeros_like(q)
+        row = {"batch": name, "kv_bytes": int(lens.astype(np.int64).sum()) * 8 * 128 * 4}
+        for label, refine in (("plain", -1), ("refined", 0)):
+            h = rep.binding.Handle(w.num_q_heads, 8, 128, pool_pages, Bn, ld, device=rep.dev.index or 0,
+                                   plan=rep.binding.PlanParams(0, 0, 0, 0, 0, 0, refine))
+            ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=rep.dev)
+
+            def step(i):
+                h.plan(lens, ws.data_ptr(), ws.numel(), st)
+                h.decode_attn(q.data_ptr(), k.data_ptr(), v.data_ptr(), bts[i % copies].data_ptr(), dl.data_ptr(),
+                              out.data_ptr(), st)
+            for i in range(8):
+                step(i)
+            torch.cuda.synchronize()
+            ts = []
+            for _ in range(regions):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for i in range(steps):
+                    step(i)
+                e1.record()
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1) / steps)
+            assert h.debug_error_word() == 0, "device error word set"
+            ms = float(np.median(ts))
+            row[label] = {"ms_per_step": ms, "kv_gbs": row["kv_bytes"] / (ms * 1e-3) / 1e9,
+                          "blocks": int(len(h.plan_export()["items"])) * 8}
+            h.close()
+        res.append(row)
+    del k, v
+    torch.cuda.empty_cache()
+    return res
+
+
 def ring_step_measure(rep: Replica, reps: int = 40):
     """The ring all-reduce's data-plane step (libra_ring_step, flag already set) on 16 MB float32 chunks, the chunk
     size the paper pipelines with: payload rate of a reduce step on 2 and on 4 thread blocks (= SMs)."""
@@ -1127,6 +1198,8 @@ def run_libra(args):
             line["short_batch"] = short_batch_measure(rep)
         if "ring_step" in extras:
             line["ring_step"] = ring_step_measure(rep)
+        if "few_long" in extras:
+            line["few_long"] = few_long_measure(rep)
         if "kv_migration" in extras and args.workload in ("longtail_mix_b256", "straggler_b8"):
             line["kv_migration"] = kv_migration_measure(rep)
         if not args.no_cpu:
@@ -1187,7 +1260,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle work for cpu_baseline")
-    ap.add_argument("--extras", default="early_prefetch,multi_token,fp8_cache,nhd_layout,head_shard,wide_group,short_batch,kv_migration,ring_step",
+    ap.add_argument("--extras", default="early_prefetch,multi_token,fp8_cache,nhd_layout,head_shard,wide_group,short_batch,kv_migration,ring_step,few_long",
                     help="side measurements on the main workload at N=1 (comma list; empty = none)")
     ap.add_argument("--variant", default="", help="warps,stages of the decode block (default: the library's)")
     ap.add_argument("--ctas-per-sm", type=int, default=0, help="planner constant (0 = default)")
