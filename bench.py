@@ -669,7 +669,8 @@ def wide_group_measure(rep: Replica, steps: int = 200):
 
 def short_batch_measure(rep: Replica, steps: int = 100):
     """Batches of equally long, short sequences at a constant 262,144 cached tokens (1.07 GB of KV at 8 KV heads, d 128):
-    the block shape the library picks by itself against the default large shape forced."""
+    the block shape the library picks by itself against the default large shape forced, on host plans; and the plan
+    made on the device, without and with the caller's bound on the lengths (libra_set_length_hint)."""
     torch, W, w = rep.torch, rep.W, rep.w
     if w.head_dim != 128 or w.num_kv_heads != 8:
         return None
@@ -691,14 +692,20 @@ def short_batch_measure(rep: Replica, steps: int = 100):
         q = torch.randn((Bn, w.num_q_heads, 128), device=rep.dev, dtype=torch.bfloat16)
         out = torch.zeros_like(q)
         row = {"tokens_per_sequence": L, "batch": Bn}
-        for label, variant in (("auto_shape", None), ("default_shape_forced", (8, 3))):
+        for label, variant, hint in (("auto_shape", None, None), ("default_shape_forced", (8, 3), None),
+                                     ("device_plan", None, 0), ("device_plan_length_hint", None, L)):
             h = rep.binding.Handle(w.num_q_heads, 8, 128, pool, Bn, bts[0].shape[1], device=rep.dev.index or 0)
             if variant:
                 h.set_variant(*variant)
+            if hint is not None:
+                h.set_length_hint(hint)
             ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=rep.dev)
 
             def step(i):
-                h.plan(lens, ws.data_ptr(), ws.numel(), st)
+                if hint is None:
+                    h.plan(lens, ws.data_ptr(), ws.numel(), st)
+                else:
+                    h.plan_device(lens_dev.data_ptr(), Bn, ws.data_ptr(), ws.numel(), st)
                 h.decode_attn(q.data_ptr(), k.data_ptr(), v.data_ptr(), bts[i % copies].data_ptr(), lens_dev.data_ptr(),
                               out.data_ptr(), st)
             for i in range(8):

@@ -273,11 +273,20 @@ int libra_plan(libra_handle_t handle, const int32_t* seq_lens_host, int32_t batc
  * block_table_ld * page_size, else the plan is empty and LIBRA_ERR_PLAN_OVERFLOW is set in the device error
  * word (checked on the device, since the host does not see the lengths).  The result equals
  * libra_plan's bit for bit (libra_plan_export reads it back).  The planning kernel is one more kernel on the stream's
- * critical path (about 6 us for 64 sequences, 8.5 us for 256); one plan serves any number of decode calls on the same
- * lengths - the attention layers of one generated token - so per call the cost is a fraction of that.
+ * critical path (about 6 us for 64 sequences, 8.5 us for 256, 19 us for 1024 and 54 us for 4096 work items); one plan
+ * serves any number of decode calls on the same lengths - the attention layers of one generated token - so per call
+ * the cost is a fraction of that.
  * Errors: INVALID_ARGUMENT, WORKSPACE_TOO_SMALL, UNSUPPORTED_SHAPE, CUDA_ERROR. */
 int libra_plan_device(libra_handle_t handle, const int32_t* seq_lens_dev, int32_t batch, void* workspace_dev,
                       size_t workspace_bytes, void* stream);
+
+/* A bound on the lengths of device-planned batches (0 = none, the default).  For a host plan the library sees the
+ * longest work unit and picks the decode block's shape by it (small blocks, several per SM, when every unit is short:
+ * up to 2.6 x faster on batches of short sequences); after libra_plan_device it cannot, and uses the large block.  A
+ * caller who knows that no sequence of the coming batches is longer than max_seq_len tokens says so here, and the
+ * same choice is made from that bound.  It is a hint: a longer sequence is still computed correctly, only on a block
+ * shape that is slow for it.  Errors: INVALID_ARGUMENT (negative). */
+int libra_set_length_hint(libra_handle_t handle, int32_t max_seq_len);
 
 /* Host view of the last plan (see libra_plan_view_t); after libra_plan_device this copies the plan
  * back from the workspace and synchronises that call's stream.  Errors: NOT_PLANNED, CUDA_ERROR. */

@@ -96,6 +96,7 @@ SIGNATURES = {
     "libra_debug_stream_read": (C.c_int, [_vp, _vp, C.c_size_t, _vp]),
     "libra_debug_gather_read": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "libra_set_combine_mode": (C.c_int, [_vp, C.c_int32]),
+    "libra_set_length_hint": (C.c_int, [_vp, C.c_int32]),
     "libra_plan_host": (C.c_int, [C.POINTER(PlanParams), C.c_int32, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p,
                                   _i32p, _i32p, C.c_int32, _i32p, _i32p, _i32p, _i32p, _i32p]),
     "libra_workspace_invalidate": (C.c_int, [_vp]),
@@ -383,6 +384,10 @@ class Handle:
 
     def set_cache_warmup(self, on: bool) -> None:
         _check(lib.libra_set_cache_warmup(self._h, 1 if on else 0), "libra_set_cache_warmup")
+
+    def set_length_hint(self, max_seq_len: int) -> None:
+        """The caller's bound on the lengths of device-planned batches (0 = none): picks the block shape."""
+        _check(lib.libra_set_length_hint(self._h, int(max_seq_len)), "libra_set_length_hint")
 
     def set_early_prefetch(self, on: bool) -> None:
         _check(lib.libra_set_early_prefetch(self._h, 1 if on else 0), "libra_set_early_prefetch")

@@ -195,6 +195,7 @@ struct libra_handle_s {
   void* last_stream = nullptr;
   bool device_planned = false;  // the last plan was made by the device-side planner: counts live in the workspace
   int64_t decodes_on_plan = 0;  // decode launches enqueued since the last plan call
+  int32_t length_hint = 0;      // libra_set_length_hint: the caller's bound on the lengths of device-planned batches (0 = none)
   int32_t dev_item_bound = 0;   // device-side plan: the most work items the planned batch can have (sizes the grids)
   int32_t planned_batch = 0;
   size_t dev_counts_off = 0, dev_per_seq_off = 0, dev_entries_off = 0, dev_fixes_off = 0;
@@ -804,6 +805,12 @@ int libra_set_early_prefetch(libra_handle_t h, int32_t on) {
   return LIBRA_OK;
 }
 
+int libra_set_length_hint(libra_handle_t h, int32_t max_seq_len) {
+  if (!h || max_seq_len < 0) return LIBRA_INVALID_ARGUMENT;
+  h->length_hint = max_seq_len;
+  return LIBRA_OK;
+}
+
 int libra_set_cache_warmup(libra_handle_t h, int32_t on) {
   if (!h || (on != 0 && on != 1)) return LIBRA_INVALID_ARGUMENT;
   h->l2_warmup = (on == 1);
@@ -890,6 +897,11 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
   const int di = (h->cfg.head_dim == 128) ? 1 : 0;
   const int ni = (h->group * q_len > 8) ? 1 : 0;
   int auto_variant = ni ? kVariantTwoTiles : kVariantOneTile;
+  if (!ni && h->device_planned && h->length_hint > 0) {
+    // the host has not seen the lengths; the caller's bound on them stands in for the longest unit
+    if (h->length_hint <= kTinyUnitTokens) auto_variant = kVariantTinyUnits;
+    else if (h->length_hint <= kShortUnitTokens) auto_variant = kVariantShortUnits;
+  }
   if (!ni && !h->device_planned && !h->plan.items.empty()) {
     const int longest = h->plan.items.front().kv_end - h->plan.items.front().kv_begin;   // items are sorted longest first
     if (longest <= kTinyUnitTokens) auto_variant = kVariantTinyUnits;

@@ -78,6 +78,34 @@ def test_random_and_edge_vectors_bit_exact(lib):
         h.close()
 
 
+def test_large_batches_bit_exact(lib):
+    """More items than the planning kernel ranks with its quadratic loop: the sort in shared memory.  Equal lengths
+    (every comparison a tie), a few distinct lengths, long-tailed ones; item counts up to the kernel's capacity."""
+    rng = np.random.default_rng(13)
+    seen = []
+    for B in (257, 300, 511, 512, 1000, 2048, 3000, 4096):
+        for kind in ("equal", "few", "tail"):
+            if kind == "equal":
+                lens = np.full(B, int(rng.integers(1, 600)))
+            elif kind == "few":
+                lens = rng.choice([0, 16, 128, 129, 1024], size=B)
+            else:
+                lens = np.clip(np.floor(200 * np.exp(rng.normal(size=B) * 1.2)), 0, 40960)
+            lens = lens.astype(np.int32)
+            hkv = int(rng.choice([1, 8]))
+            plan = lib.PlanParams(148, int(rng.choice([1, 7])), int(rng.choice([1, 4])), 16, int(rng.choice([16, 512])), 64)
+            h, ws, dl = device_plan(lib, lens, hkv, plan)
+            ref = P.plan(lens, hkv, ref_params(h))
+            if len(ref.items) > 4096:
+                assert h.debug_error_word() & lib.ERR_PLAN_OVERFLOW
+            else:
+                assert_same_plan(h.plan_export(), ref)
+                assert h.debug_error_word() == 0
+                seen.append(len(ref.items))
+            h.close()
+    assert max(seen) > 3000 and sum(n > 256 for n in seen) >= 15
+
+
 def test_few_long_sequences_bit_exact(lib):
     """Small batches of long sequences: plans of fewer than one and a half waves of long blocks, which the planner
     makes again for twice as many slots."""
@@ -232,3 +260,32 @@ def test_separate_combine_with_nothing_to_merge_keeps_the_chain_ordered(lib):
         results.append(bufs[0].cpu().numpy().copy())
         r.h.close()
     assert np.array_equal(results[0], results[1])
+
+
+@pytest.mark.parametrize("L,hint", [(200, 256), (900, 1024), (900, 0), (900, 256)])
+def test_length_hint_picks_the_block_shape_of_a_host_plan(lib, L, hint):
+    """A device-planned batch of short sequences with the caller's bound on the lengths runs on the block shape a host
+    plan would have picked: the same bits as the host-planned step.  Without the hint (or with one that turns out too
+    small) the result is as correct, on another shape."""
+    import torch
+    dev = torch.device("cuda:0")
+    B, Hq, Hkv, d = 40, 32, 8, 128
+    lens = [L - (i % 7) * 3 for i in range(B)]
+    lens_a, bt, q, k, v = W.random_case(130 + L, B, Hq, Hkv, d, lens)
+    ref, _ = O.paged_decode_attention(q, k, v, bt, lens_a)
+    r = H.Runner(lib, Hq, Hkv, d, k.shape[0], B, bt.shape[1])
+    dq, dk, dv, dbt = (H.to_dev(x, dev) for x in (q, k, v, bt))
+    host = H.bf16_dev_to_f32(r.run(dq, dk, dv, dbt, lens_a))          # host plan: the library sees the longest unit
+    dl = torch.from_numpy(lens_a.copy()).to(dev)
+    out = torch.full((B, Hq, d), H.CANARY, dtype=torch.int16, device=dev)
+    st = torch.cuda.current_stream().cuda_stream
+    r.h.set_length_hint(hint)
+    r.h.plan_device(dl.data_ptr(), B, r.ws.data_ptr(), r.ws.numel(), st)
+    r.h.decode_attn(dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dbt.data_ptr(), dl.data_ptr(), out.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert r.h.debug_error_word() == 0
+    got = H.bf16_dev_to_f32(out)
+    assert gates.tight_violations(got, ref) == 0 and gates.stated_violations(got, ref) == 0
+    if hint >= L:
+        assert np.array_equal(got, host)
+    r.h.close()
