@@ -273,7 +273,7 @@ int libra_plan(libra_handle_t handle, const int32_t* seq_lens_host, int32_t batc
  * block_table_ld * page_size, else the plan is empty and LIBRA_ERR_PLAN_OVERFLOW is set in the device error
  * word (checked on the device, since the host does not see the lengths).  The result equals
  * libra_plan's bit for bit (libra_plan_export reads it back).  The planning kernel is one more kernel on the stream's
- * critical path (about 6 us for 64 sequences, 8.5 us for 256, 19 us for 1024 and 54 us for 4096 work items); one plan
+ * critical path (about 6 us for 64 sequences, 8.5 us for 256, 12 us for 1024 and 21 us for 4096 work items); one plan
  * serves any number of decode calls on the same lengths - the attention layers of one generated token - so per call
  * the cost is a fraction of that.
  * Errors: INVALID_ARGUMENT, WORKSPACE_TOO_SMALL, UNSUPPORTED_SHAPE, CUDA_ERROR. */

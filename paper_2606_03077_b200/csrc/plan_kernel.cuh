@@ -27,12 +27,14 @@ namespace libra {
 constexpr int kDevPlanThreads = 1024;   // the most threads one planning block has
 constexpr int kDevPlanPerThread = 4;
 constexpr int kDevPlanMax = kDevPlanThreads * kDevPlanPerThread;
-// Items up to which the quadratic ranking loop beats the bitonic sort.  Measured on a B200, time of one planning
-// kernel in a chain of them: 64 items 4.3 us, 256 items 6.9, 384 items 10.0 (loop) against 11.4 (sort), 512 items 14.5
-// against 11.9; the sort alone above that: 1024 items 18.6 us, 2048 items 30.4, 4096 items 54.4 (the loop: 44.5 us at
-// 1024 items; a decode step over 2048 items became 122 us shorter when the sort replaced it).
-constexpr int kDevPlanRankLoopMax = 400;
-constexpr int kDevPlanArrays = 8;       // shared-memory arrays of kDevPlanPerThread * blockDim.x ints each
+// Items up to which the quadratic ranking loop is used; above, a radix sort in shared memory (a bitonic sort if a
+// work unit has 2^16 tokens or more).  Measured on a B200, one planning kernel in a chain of them, of which the
+// ordering step: 64 items 4.3 us (0.3), 256 items 6.7 (2.4), 384 items 9.8 (5.1) with the loop, which takes 44 us at 1024
+// items and about 150 us at 2048; with the radix sort 512 items 8.5 us (3.4), 1024 items 11.7 (4.9), 2048 items 14.9
+// (6.3), 4096 items 21.3 (9.7); the bitonic sort takes 6.8 / 11.7 / 21.8 / 42.9 us at those four sizes.
+constexpr int kDevPlanRankLoopMax = 256;
+constexpr int kDevPlanArrays = 10;      // shared-memory arrays of kDevPlanPerThread * blockDim.x ints each
+constexpr int kDevPlanRadixMaxLen = 1 << 16;   // the radix sort packs (length, index) into one word: lengths below this
 
 struct PlanKernelParams {
   const int32_t* seq_lens;   // device, [batch]
@@ -130,6 +132,8 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
   int* it_len = sm + 5 * cap;     // [items]
   int* it_b = sm + 6 * cap;       // [items]
   int* it_j = sm + 7 * cap;       // [items]
+  int* hist = sm + 8 * cap;       // [warps][256] digit counts of the radix sort (two arrays: 8 ints per thread)
+  __shared__ int digit_tot[256];
   __shared__ int warp_tot[33];
   __shared__ long long warp_sum[32];
 
@@ -247,8 +251,10 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
 
   // ---- items in (b, j) order (the list is padded to a multiple of four with lengths that rank after everything)
   if (tid < 4 && (n_items & ~3) + tid >= n_items && (n_items & ~3) + tid < cap) it_len[(n_items & ~3) + tid] = -1;
+  int wide = 0;
   for (int b = tid; b < B; b += nthr) {
     const int len = len_s[b];
+    wide |= (chunk[b] >= kDevPlanRadixMaxLen) ? 1 : 0;
     for (int j = 0; j < nsplit[b]; ++j) {
       const int i = offs[b] + j;
       const int lo = j * chunk[b];
@@ -258,7 +264,7 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
       it_j[i] = j;
     }
   }
-  __syncthreads();
+  wide = __syncthreads_or(wide);
 
   auto emit = [&](int rank, int i) {
     const int b = it_b[i], j = it_j[i];
@@ -268,8 +274,92 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
                                 (nsplit[b] > 1) ? offs[b] + j : -1);
   };
 
+  auto finish = [&]() {
+    if (tid == 0) {
+      p.counts[L::kCntItems] = n_items;
+      p.counts[L::kCntCombine] = n_combine;
+      p.counts[L::kCntEmpty] = n_empty;
+      p.counts[L::kCntChunkTarget] = int(base);
+      p.counts[L::kCntOverflow] = 0;
+    }
+  };
+
+  if (n_items > kDevPlanRankLoopMax && !wide) {
+    // ---- many items, lengths below 2^16: a stable radix sort, two passes of 8 bits, of the words
+    // (0xffff - length) << 16 | index.  Ascending and stable, so longest first with ties in index order, which is
+    // the (b, j) order.  Warp w owns the items [w * per, (w + 1) * per), 32 at a time: within a warp the items of one
+    // digit are ranked by warp votes and a per-warp counter, across warps by a scan of the counters.
+    const int lane = tid & 31, warp = tid >> 5, n_warps = nthr >> 5;
+    const int per = ((n_items + n_warps - 1) / n_warps + 31) & ~31;      // <= 128: n_items <= cap = 128 * n_warps
+    unsigned* src = reinterpret_cast<unsigned*>(it_len);
+    unsigned* dst = reinterpret_cast<unsigned*>(aux);                     // the flags in aux were last read before the barrier above
+    for (int i = tid; i < n_items; i += nthr) src[i] = (unsigned(0xffff - it_len[i]) << 16) | unsigned(i);
+    for (int shift = 16; shift < 32; shift += 8) {
+      for (int i = tid; i < n_warps * 64; i += nthr) reinterpret_cast<int4*>(hist)[i] = make_int4(0, 0, 0, 0);
+      __syncthreads();
+      int loc[4], dig[4];
+      unsigned word[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        dig[e] = 256;
+        if (e * 32 >= per) continue;                                       // the same for the whole warp
+        const int i = warp * per + e * 32 + lane;
+        const bool live = i < n_items;
+        word[e] = live ? src[i] : 0u;
+        const unsigned d = (word[e] >> shift) & 255u;
+        // the lanes that hold the same digit: eight votes, one per bit (the hardware's match instruction takes a
+        // round per distinct value, up to 32 of them here)
+        unsigned grp = __ballot_sync(0xffffffffu, live);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const unsigned vote = __ballot_sync(0xffffffffu, (d >> k) & 1u);
+          grp &= ((d >> k) & 1u) ? vote : ~vote;
+        }
+        int first = 0;
+        if (live) {
+          dig[e] = int(d);
+          const int leader = __ffs(grp) - 1;
+          if (lane == leader) {
+            first = hist[warp * 256 + d];
+            hist[warp * 256 + d] = first + __popc(grp);
+          }
+          // every lane of a group reads its leader's value; groups are disjoint, so one shuffle serves them all
+        }
+        const int src_lane = live ? __ffs(grp) - 1 : lane;
+        loc[e] = __shfl_sync(0xffffffffu, first, src_lane) + __popc(grp & ((1u << lane) - 1u));
+        __syncwarp();                                                      // the counter's new value, before the next 32 items
+      }
+      __syncthreads();
+      for (int d = tid; d < 256; d += nthr) {   // per digit: the warps' counts become their exclusive prefix, the total goes to digit_tot
+        int run = 0;
+        for (int w0 = 0; w0 < n_warps; w0 += 8) {      // eight loads in flight, then their prefixes
+          int t[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) t[k] = (w0 + k < n_warps) ? hist[(w0 + k) * 256 + d] : 0;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            if (w0 + k < n_warps) hist[(w0 + k) * 256 + d] = run;
+            run += t[k];
+          }
+        }
+        digit_tot[d] = run;
+      }
+      __syncthreads();
+      dev::block_exclusive_scan(digit_tot, 256, warp_tot);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if (dig[e] < 256) dst[digit_tot[dig[e]] + hist[warp * 256 + dig[e]] + loc[e]] = word[e];
+      }
+      __syncthreads();
+      unsigned* t = src; src = dst; dst = t;
+    }
+    for (int r = tid; r < n_items; r += nthr) emit(r, int(src[r] & 0xffffu));
+    finish();
+    return;
+  }
+
   if (n_items > kDevPlanRankLoopMax) {
-    // ---- many items: a bitonic sort of (length, index) pairs in shared memory, longest first, ties by index (which
+    // ---- many items, some of 2^16 tokens or more: a bitonic sort of (length, index) pairs in shared memory, longest first, ties by index (which
     // is the (b, j) order).  n log^2 n compare-exchanges against the n^2 comparisons of the ranking loop below.
     int n2 = 1;
     while (n2 < n_items) n2 <<= 1;                       // <= cap: cap is four times the thread count
@@ -297,13 +387,7 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
       }
     }
     for (int r = tid; r < n_items; r += nthr) emit(r, idx[r]);
-    if (tid == 0) {
-      p.counts[L::kCntItems] = n_items;
-      p.counts[L::kCntCombine] = n_combine;
-      p.counts[L::kCntEmpty] = n_empty;
-      p.counts[L::kCntChunkTarget] = int(base);
-      p.counts[L::kCntOverflow] = 0;
-    }
+    finish();
     return;
   }
 
@@ -324,13 +408,7 @@ __global__ void __launch_bounds__(kDevPlanThreads) plan_kernel(const PlanKernelP
     }
     emit(rank, i);
   }
-  if (tid == 0) {
-    p.counts[L::kCntItems] = n_items;
-    p.counts[L::kCntCombine] = n_combine;
-    p.counts[L::kCntEmpty] = n_empty;
-    p.counts[L::kCntChunkTarget] = int(base);
-    p.counts[L::kCntOverflow] = 0;
-  }
+  finish();
 }
 
 }  // namespace libra

@@ -103,7 +103,17 @@ def test_large_batches_bit_exact(lib):
                 assert h.debug_error_word() == 0
                 seen.append(len(ref.items))
             h.close()
-    assert max(seen) > 3000 and sum(n > 256 for n in seen) >= 15
+    assert max(seen) > 3000 and sum(n > 400 for n in seen) >= 12
+    # a work unit of 2^16 tokens or more among many: the kernel's other sort (its radix sort packs 16-bit lengths)
+    for B, long_len, max_splits in ((450, 70000, 1), (1500, 2 ** 20, 8), (4000, 65536, 1)):
+        lens = rng.integers(0, 300, B).astype(np.int32)
+        lens[rng.integers(0, B)] = long_len
+        h, ws, dl = device_plan(lib, lens, 8, lib.PlanParams(148, 1, 1, 16, 16, max_splits))
+        ref = P.plan(lens, 8, ref_params(h))
+        assert max(e - b for _, _, b, e in ref.items) >= 65536 and 400 < len(ref.items) <= 4096
+        assert_same_plan(h.plan_export(), ref)
+        assert h.debug_error_word() == 0
+        h.close()
 
 
 def test_few_long_sequences_bit_exact(lib):
