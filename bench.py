@@ -53,9 +53,11 @@ FALLBACK_HBM_GBS = 6650.0
 L2_BYTES_ASSUMED = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode launch divided by its algorithmic bytes, from the ncu
 # captures summarised under profiles/ (a constant of those captures, not something this run measures):
-# lognormal_b64 374.4 MB / 368.1 MB, straggler_b8 1078.0 MB / 1073.7 MB.  The large mix is too big to capture under
-# the profiler; its traffic is scaled from these (traffic grows with the pages read).
-NCU_TRAFFIC_OVER_ALGORITHMIC = {"lognormal_b64": 374.4e6 / 368.128e6, "straggler_b8": 1078.0e6 / 1073.741824e6}
+# lognormal_b64 374.4 MB / 368.1 MB, straggler_b8 1078.0 MB / 1073.7 MB (full captures); longtail_mix_b256 4834.1 MB /
+# 4821.6 MB and shift_b128 5774.0 MB / 5754.9 MB over its cycle of three layouts (one-pass captures of the two byte
+# counters at full size).
+NCU_TRAFFIC_OVER_ALGORITHMIC = {"lognormal_b64": 374.4e6 / 368.128e6, "straggler_b8": 1078.0e6 / 1073.741824e6,
+                                "longtail_mix_b256": 4834.1e6 / 4821.590016e6, "shift_b128": 5774.01e6 / 5754.925056e6}
 
 
 # ----------------------------------------------------------------------------- clocks
@@ -1145,8 +1147,8 @@ def run_libra(args):
                 "peak_source": peak_src,
                 "traffic": (m["kv_bytes_per_step"] * (ratio if ratio else float(np.mean(list(NCU_TRAFFIC_OVER_ALGORITHMIC.values()))))),
                 "traffic_source": ("ncu capture of this workload, profiles/" if ratio else
-                                   "scaled from the ncu captures of lognormal_b64 and straggler_b8 (1.004 - 1.018 x the "
-                                   "algorithmic bytes): this workload is too large to capture under the profiler"),
+                                   "scaled from the ncu captures of the four large workloads (1.003 - 1.017 x the "
+                                   "algorithmic bytes)"),
                 "algorithmic_bytes_per_launch": m["kv_bytes_per_step"], "kernel_us": m["kernel_us_event_pairs"],
                 "chained_step_us": m["ms_per_step"] * 1e3,
                 "timing": "frac / frac_kernel: a CUDA event pair around every decode launch (the kernel's own duration); "
