@@ -64,7 +64,16 @@ Variant make_variant() {
 // Block shapes that are compiled in.  Defaults: index 0 (8 warps x 3 stages) for one column tile, index 1
 // (12 x 2) for two: twice the tensor-core and softmax work per tile wants a third warp per scheduler to hide
 // its latency (measured 2.5 - 4 % faster there, 0.5 - 1 % slower with one tile).
-constexpr int kVariantOneTile = 0, kVariantTwoTiles = 1, kVariantShortUnits = 4, kVariantTinyUnits = 9;
+constexpr int kVariantOneTile = 0, kVariantTwoTiles = 1, kVariantShortUnits = 4, kVariantTinyUnits = 9, kVariantPair = 10;
+// Two column tiles (9 - 16 score columns per KV head: more than 8 query heads per KV head, or several query tokens)
+// double the work per tile and the per-unit merge; there two blocks of 6 warps x 2 stages per SM (96 KB and 168
+// registers each, the kernel's launch bounds see to the registers), planned as two slots per SM, beat one block of
+// 12 x 2: one block's start-up and merge overlap the other's streaming.  Same-run A/B, us per step, 12 x 2 -> 2 x (6 x 2):
+// 16 query heads per KV head 64.3 -> 61.3 (lognormal_b64), 303 -> 286 (shift_b128), the two long workloads unchanged;
+// two query tokens 57.6 -> 56.8, 180.6 -> 175.8 (straggler_b8), 306 -> 290, 681 -> 676 (longtail_mix_b256); four query
+// tokens 68.1 -> 63.4, 746 -> 749.  With one column tile the two shapes are a wash; over an E4M3 cache the two-slot plan
+// is 1 - 8 % slower (its block shapes are one per SM), so it keeps one slot.
+constexpr int kTwoSlotCtas = 2;
 // A block costs ~4 us of start-up and epilogue whatever its size and the default block is alone on its SM, so a batch
 // of short sequences leaves the SMs waiting most of the time.  When no unit of a host plan is longer than this many
 // tokens, 4 warps x 2 stages (64 KB: three blocks per SM, three units in flight) is used instead: the same bytes in
@@ -77,7 +86,7 @@ const std::vector<Variant>& variants() {
   static const std::vector<Variant> v = {
       make_variant<8, 3>(), make_variant<12, 2>(), make_variant<8, 2>(), make_variant<4, 3>(), make_variant<4, 2>(),
       make_variant<4, 4>(), make_variant<4, 6>(), make_variant<2, 6>(), make_variant<2, 4>(),
-      make_variant<2, 2>(),
+      make_variant<2, 2>(), make_variant<6, 2>(),
   };
   return v;
 }
@@ -157,7 +166,10 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct libra_handle_s {
   libra_config_t cfg;
-  libra::PlanParams params;
+  libra::PlanParams params;          // the planner's parameters in force (defaults resolved)
+  libra_plan_params_t params_in{};   // as given at creation (0 = default)
+  int n_sm_dev = 0;
+  bool two_slot_auto = false;        // the default of two slots per SM is in force (see kVariantPair)
   int group = 0;
   float scale_log2 = 0.f;
   int64_t stride_page = 0, stride_head = 0, stride_token = 0;
@@ -236,8 +248,9 @@ int fail_cuda(libra_handle_t h, cudaError_t e) {
     if (e__ != cudaSuccess) return fail_cuda(h, e__); \
   } while (0)
 
-libra::PlanParams resolve_params(const libra_plan_params_t& in, int n_sm_device) {
+libra::PlanParams resolve_params(const libra_plan_params_t& in, int n_sm_device, bool two_slots = false) {
   libra::PlanParams p;
+  if (two_slots) p.ctas_per_sm = kTwoSlotCtas;   // the default where two blocks per SM are resident (see kVariantPair)
   if (in.n_sm > 0) p.n_sm = in.n_sm;
   else if (n_sm_device > 0) p.n_sm = n_sm_device;
   if (in.ctas_per_sm > 0) p.ctas_per_sm = in.ctas_per_sm;
@@ -287,11 +300,28 @@ int encode_pool_map(libra_handle_t h, const void* base, CUtensorMap* map, int* p
   return LIBRA_OK;
 }
 
-// Workspace layout; the partial buffers hold max_q_len * num_q_heads rows per work item.
+// Two slots per SM are the planner's default where a step has two column tiles and the pools are bf16.
+bool wants_two_slots(const libra_handle_s* h, bool whatever_the_pools) {
+  return h->params_in.ctas_per_sm == 0 && h->group * h->max_q_len > 8 && (whatever_the_pools || !h->fp8);
+}
+
+// The parameters in force for the handle's present state; true if they changed (a plan made before is then void).
+bool refresh_params(libra_handle_t h) {
+  const bool two = wants_two_slots(h, false);
+  const libra::PlanParams now = resolve_params(h->params_in, h->n_sm_dev, two);
+  const bool changed = now.ctas_per_sm != h->params.ctas_per_sm;
+  h->params = now;
+  h->two_slot_auto = two;
+  return changed;
+}
+
+// Workspace layout; the partial buffers hold max_q_len * num_q_heads rows per work item.  Sized for the larger of the
+// two defaults, so that switching the pools' type never asks for a larger workspace.
 void compute_layout(libra_handle_t h) {
   const libra_config_t* cfg = &h->cfg;
   const size_t rows = size_t(h->max_q_len) * cfg->num_q_heads;
-  h->max_items = libra::max_items(h->params, cfg->num_kv_heads, cfg->max_batch);
+  h->max_items = libra::max_items(resolve_params(h->params_in, h->n_sm_dev, wants_two_slots(h, true)), cfg->num_kv_heads,
+                                  cfg->max_batch);
   h->cnt_off = 256;  // the first 256 bytes hold the control words (the device error word)
   h->cnt_bytes = align_up(size_t(cfg->max_batch) * cfg->num_kv_heads * 4, 256);
   h->lse_off = h->cnt_off + h->cnt_bytes;
@@ -450,7 +480,9 @@ int libra_create(libra_handle_t* handle, const libra_config_t* cfg) {
       status = fail_cuda(h, cudaErrorNoKernelImageForDevice);
       break;
     }
-    h->params = resolve_params(pin, n_sm);
+    h->params_in = pin;
+    h->n_sm_dev = n_sm;
+    refresh_params(h);
     if (!libra::valid_params(h->params) || h->params.chunk_align % cfg->page_size != 0) {
       status = LIBRA_INVALID_ARGUMENT;  // chunks must start on page boundaries
       break;
@@ -772,6 +804,7 @@ int libra_set_max_query_tokens(libra_handle_t h, int32_t max_q_len) {
   if (max_q_len * h->group > 16) return LIBRA_UNSUPPORTED_SHAPE;  // a unit's score tile has at most 16 columns
   if (max_q_len == h->max_q_len) return LIBRA_OK;
   h->max_q_len = max_q_len;
+  refresh_params(h);
   compute_layout(h);
   h->planned = false;          // the workspace layout changed: plan again, into a workspace of the new size
   h->clean_workspace = nullptr;
@@ -786,6 +819,7 @@ int libra_set_kv_dtype(libra_handle_t h, int32_t dtype, float k_scale, float v_s
     if (h->stride_page % 16 || h->stride_head % 16 || h->stride_token % 16) return LIBRA_INVALID_ARGUMENT;
   }
   h->fp8 = (dtype == LIBRA_KV_E4M3);
+  if (refresh_params(h)) h->planned = false;   // the planner's default slot count follows the pools' type: plan again
   h->fp8_variant = -1;
   h->k_scale = h->fp8 ? k_scale : 1.f;
   h->v_scale = h->fp8 ? v_scale : 1.f;
@@ -896,7 +930,10 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
 
   const int di = (h->cfg.head_dim == 128) ? 1 : 0;
   const int ni = (h->group * q_len > 8) ? 1 : 0;
-  int auto_variant = ni ? kVariantTwoTiles : kVariantOneTile;
+  // two column tiles: two blocks per SM where the plan was made for two slots; one column tile on such a plan
+  // (a handle laid out for several query tokens that is given one): the same shape, so that the plan fits
+  int auto_variant = ni ? (h->params.ctas_per_sm >= kTwoSlotCtas ? kVariantPair : kVariantTwoTiles)
+                        : (h->two_slot_auto ? kVariantPair : kVariantOneTile);
   if (!ni && h->device_planned && h->length_hint > 0) {
     // the host has not seen the lengths; the caller's bound on them stands in for the longest unit
     if (h->length_hint <= kTinyUnitTokens) auto_variant = kVariantTinyUnits;

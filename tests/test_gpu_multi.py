@@ -231,3 +231,54 @@ def test_append_of_the_new_tokens_fused_in(lib, layout):
                 got_k, got_v = got_k.transpose(0, 2, 1, 3), got_v.transpose(0, 2, 1, 3)
             assert np.array_equal(got_k, k_ref) and np.array_equal(got_v, v_ref)
             h.close()
+
+
+def test_two_column_tiles_plan_for_two_slots_per_sm_by_default(lib):
+    """More than 8 rows of q per KV head (16 query heads per KV head, or several query tokens): the planner's default
+    is two slots per SM over bf16 pools and the step runs two 6-warp blocks per SM; over an E4M3 cache it is one slot,
+    and switching the type voids the plan.  Outputs against the oracle under the default and under a forced one-slot
+    plan (the 12-warp block), on the same handle state a caller would have."""
+    import torch
+    dev = torch.device("cuda:0")
+    lens = [5000, 1300, 257, 16, 1, 0, 2048, 90]
+    B, Hkv, d = len(lens), 2, 128
+    st = torch.cuda.current_stream().cuda_stream
+    for Hq, Tq in ((32, 1), (8, 3), (16, 2)):
+        lens_a, bt, _, k, v = W.random_case(900 + Hq + Tq, B, Hq, Hkv, d, lens)
+        q = draw_q(901 + Hq, B, Tq, Hq, d)
+        ref, _ = O.paged_multi_token_attention(q, k, v, bt, lens_a)
+        for plan, want in ((None, 2), (lib.PlanParams(0, 1, 0, 0, 0, 0), 1)):
+            h = lib.Handle(Hq, Hkv, d, k.shape[0], B, bt.shape[1], plan=plan)
+            assert h.plan_params().ctas_per_sm == (want if Hq // Hkv > 8 else 1)
+            h.set_max_query_tokens(Tq)
+            assert h.plan_params().ctas_per_sm == want
+            ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=dev)
+            qd, kd, vd, btd = (H.to_dev(x, dev) for x in (q, k, v, bt))
+            dl = torch.from_numpy(lens_a.copy()).to(dev)
+            out = torch.full((B, Tq, Hq, d), H.CANARY, dtype=torch.int16, device=dev)
+            h.plan(lens_a, ws.data_ptr(), ws.numel(), st)
+            h.decode_attn_multi(qd.data_ptr(), Tq, kd.data_ptr(), vd.data_ptr(), btd.data_ptr(), dl.data_ptr(), out.data_ptr(), st)
+            torch.cuda.synchronize()
+            assert h.debug_error_word() == 0
+            check(H.bf16_dev_to_f32(out), ref, f"Hq {Hq} Tq {Tq} slots {want}")
+            if Tq > 1:   # one query token on the handle laid out for several: the same plan, one column tile
+                q1 = np.ascontiguousarray(q[:, :1])
+                ref1, _ = O.paged_multi_token_attention(q1, k, v, bt, lens_a)
+                out1 = torch.full((B, 1, Hq, d), H.CANARY, dtype=torch.int16, device=dev)
+                h.decode_attn(H.to_dev(q1, dev).data_ptr(), kd.data_ptr(), vd.data_ptr(), btd.data_ptr(), dl.data_ptr(),
+                              out1.data_ptr(), st)
+                torch.cuda.synchronize()
+                assert h.debug_error_word() == 0
+                check(H.bf16_dev_to_f32(out1), ref1, f"Hq {Hq} Tq 1 of {Tq} slots {want}")
+            # the 8-bit cache keeps one slot per SM: the default follows the type and the old plan is void
+            h.set_kv_dtype(lib.KV_E4M3, 1.0, 1.0)
+            assert h.plan_params().ctas_per_sm == 1
+            if want == 2:
+                with pytest.raises(lib.LibraError) as e:
+                    h.decode_attn_multi(qd.data_ptr(), Tq, kd.data_ptr(), vd.data_ptr(), btd.data_ptr(), dl.data_ptr(),
+                                        out.data_ptr(), st)
+                assert e.value.status == lib.NOT_PLANNED
+            assert h.workspace_size() <= ws.numel()
+            h.set_kv_dtype(lib.KV_BF16)
+            assert h.plan_params().ctas_per_sm == want
+            h.close()
