@@ -71,8 +71,7 @@ constexpr int kVariantOneTile = 0, kVariantTwoTiles = 1, kVariantShortUnits = 4,
 // 12 x 2: one block's start-up and merge overlap the other's streaming.  Same-run A/B, us per step, 12 x 2 -> 2 x (6 x 2):
 // 16 query heads per KV head 64.3 -> 61.3 (lognormal_b64), 303 -> 286 (shift_b128), the two long workloads unchanged;
 // two query tokens 57.6 -> 56.8, 180.6 -> 175.8 (straggler_b8), 306 -> 290, 681 -> 676 (longtail_mix_b256); four query
-// tokens 68.1 -> 63.4, 746 -> 749.  With one column tile the two shapes are a wash; over an E4M3 cache the two-slot plan
-// is 1 - 8 % slower (its block shapes are one per SM), so it keeps one slot.
+// tokens 68.1 -> 63.4, 746 -> 749.  With one column tile the two shapes are a wash.  Over an E4M3 cache: kFp8Pair.
 constexpr int kTwoSlotCtas = 2;
 // A block costs ~4 us of start-up and epilogue whatever its size and the default block is alone on its SM, so a batch
 // of short sequences leaves the SMs waiting most of the time.  When no unit of a host plan is longer than this many
@@ -107,7 +106,12 @@ const int kLoadsOnlySmem[2] = {libra::DecodeSmem<64, kLoadsOnlyWarps, kLoadsOnly
 // sequences and 5 % on the drifting workload: no clear winner, available through libra_set_variant.)  Batches of short
 // units get 4 x 2 or, up to kTinyUnitTokens, 2 x 4 (32 KB, seven blocks per SM: 1.4x / 1.9x / 2.6x / 3.5x faster than
 // 16 x 3 at 1024 / 512 / 256 / 128 tokens per sequence).  fn[loads only][NT - 1]
-constexpr int kFp8OneTile = 2, kFp8TwoTiles = 1, kFp8ShortUnits = 5, kFp8TinyUnits = 6;
+// Two column tiles on a two-slot plan: two blocks of 6 x 4 per SM, as over bf16 pools (kVariantPair).  Same-run A/B
+// against 8 x 6 on a one-slot plan, 16 query heads per KV head: 50.2 -> 44.7 us (lognormal_b64), 124.7 -> 114.0
+// (straggler_b8), 225 -> 196 (shift_b128), 530 -> 512 (longtail_mix_b256); with two query tokens (8 query heads per KV
+// head) 39.7 -> 36.7, 133.3 -> 122.0, 239 -> 209, but 391 -> 452 on longtail_mix_b256, where 8 x 6 is already near the
+// gather ceiling: two slots are the default only for more than 8 query heads per KV head.
+constexpr int kFp8OneTile = 2, kFp8TwoTiles = 1, kFp8ShortUnits = 5, kFp8TinyUnits = 6, kFp8Pair = 7;
 struct Fp8Variant {
   int warps, stages;
   DecodeKernelFn fn[2][2][2];      // [D == 128][loads only][NT - 1]
@@ -138,7 +142,7 @@ Fp8Variant make_fp8_variant() {
 const std::vector<Fp8Variant>& fp8_variants() {
   static const std::vector<Fp8Variant> v = {make_fp8_variant<8, 3>(), make_fp8_variant<8, 6>(), make_fp8_variant<16, 3>(),
                                             make_fp8_variant<16, 2>(), make_fp8_variant<8, 4>(), make_fp8_variant<4, 2>(),
-                                            make_fp8_variant<2, 4>()};
+                                            make_fp8_variant<2, 4>(), make_fp8_variant<6, 4>()};
   return v;
 }
 
@@ -300,9 +304,10 @@ int encode_pool_map(libra_handle_t h, const void* base, CUtensorMap* map, int* p
   return LIBRA_OK;
 }
 
-// Two slots per SM are the planner's default where a step has two column tiles and the pools are bf16.
+// Two slots per SM are the planner's default where a step has two column tiles and the pools are bf16, or E4M3 with
+// more than 8 query heads per KV head (kVariantPair, kFp8Pair).
 bool wants_two_slots(const libra_handle_s* h, bool whatever_the_pools) {
-  return h->params_in.ctas_per_sm == 0 && h->group * h->max_q_len > 8 && (whatever_the_pools || !h->fp8);
+  return h->params_in.ctas_per_sm == 0 && h->group * h->max_q_len > 8 && (whatever_the_pools || !h->fp8 || h->group > 8);
 }
 
 // The parameters in force for the handle's present state; true if they changed (a plan made before is then void).
@@ -1005,7 +1010,7 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     lc.blockDim = dim3(unsigned((loads_only ? kLoadsOnlyWarps : v.warps) * 32));
     lc.dynamicSmemBytes = size_t(loads_only ? kLoadsOnlySmem[di] : v.smem[di][ni]);
     if (h->fp8) {
-      int fp8_auto = ni ? kFp8TwoTiles : kFp8OneTile;
+      int fp8_auto = ni ? (h->params.ctas_per_sm >= kTwoSlotCtas ? kFp8Pair : kFp8TwoTiles) : kFp8OneTile;
       if (!ni && !loads_only && auto_variant == kVariantShortUnits) fp8_auto = kFp8ShortUnits;
       if (!ni && !loads_only && auto_variant == kVariantTinyUnits) fp8_auto = kFp8TinyUnits;
       const Fp8Variant& fv = fp8_variants()[h->fp8_variant >= 0 ? h->fp8_variant : fp8_auto];
