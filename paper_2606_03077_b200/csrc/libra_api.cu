@@ -61,9 +61,10 @@ Variant make_variant() {
   return v;
 }
 
-// Block shapes that are compiled in.  Defaults: index 0 (8 warps x 3 stages) for one column tile, index 1
-// (12 x 2) for two: twice the tensor-core and softmax work per tile wants a third warp per scheduler to hide
-// its latency (measured 2.5 - 4 % faster there, 0.5 - 1 % slower with one tile).
+// Block shapes that are compiled in.  Defaults: index 0 (8 warps x 3 stages) for one column tile; for two, on a plan
+// with one slot per SM, index 1 (12 x 2): twice the tensor-core and softmax work per tile wants a third warp per
+// scheduler to hide its latency (measured 2.5 - 4 % faster there than 8 x 3, 0.5 - 1 % slower with one tile); on a plan
+// with two slots per SM (the default for two tiles) index 10, see below.
 constexpr int kVariantOneTile = 0, kVariantTwoTiles = 1, kVariantShortUnits = 4, kVariantTinyUnits = 9, kVariantPair = 10;
 // Two column tiles (9 - 16 score columns per KV head: more than 8 query heads per KV head, or several query tokens)
 // double the work per tile and the per-unit merge; there two blocks of 6 warps x 2 stages per SM (96 KB and 168
