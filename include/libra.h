@@ -77,8 +77,7 @@ typedef struct {
   int32_t n_sm;           /* SMs to plan for; 0 = the device's count (148 on B200)               */
   int32_t ctas_per_sm;    /* resident decode blocks per SM the plan assumes; default 1, and 2 where
                              a KV head serves more than 8 rows of q (query heads per KV head x
-                             libra_set_max_query_tokens) over bf16 pools, or has more than 8
-                             query heads over E4M3 pools: those steps run two blocks per SM       */
+                             libra_set_max_query_tokens): those steps run two blocks per SM      */
   int32_t items_per_slot; /* target work units per resident block; default 1                    */
   int32_t chunk_align;    /* A: chunk lengths are multiples of this many tokens (itself a
                              multiple of 16); default 256                                       */
@@ -171,8 +170,7 @@ int libra_set_max_query_tokens(libra_handle_t handle, int32_t max_q_len);
  * Halving the bytes per cached token halves what the step has to read.  With E4M3 pools the rows given to
  * libra_decode_attn_append (k_new, v_new: [batch, num_kv_heads, head_dim]) and the dense buffers of
  * libra_kv_gather / libra_kv_scatter hold codes too, one byte per element; libra_decode_attn_host returns
- * UNSUPPORTED_SHAPE.  The workspace does not depend on the type; the plan does where the default of ctas_per_sm does
- * (see libra_plan_params_t): there the call voids the plan (NOT_PLANNED until the next plan call). */
+ * UNSUPPORTED_SHAPE.  The plan and the workspace do not depend on the type. */
 #define LIBRA_KV_BF16 0
 #define LIBRA_KV_E4M3 1
 int libra_set_kv_dtype(libra_handle_t handle, int32_t dtype, float k_scale, float v_scale);

@@ -71,8 +71,9 @@ constexpr int kVariantOneTile = 0, kVariantTwoTiles = 1, kVariantShortUnits = 4,
 // registers each, the kernel's launch bounds see to the registers), planned as two slots per SM, beat one block of
 // 12 x 2: one block's start-up and merge overlap the other's streaming.  Same-run A/B, us per step, 12 x 2 -> 2 x (6 x 2):
 // 16 query heads per KV head 64.3 -> 61.3 (lognormal_b64), 303 -> 286 (shift_b128), the two long workloads unchanged;
-// two query tokens 57.6 -> 56.8, 180.6 -> 175.8 (straggler_b8), 306 -> 290, 681 -> 676 (longtail_mix_b256); four query
-// tokens 68.1 -> 63.4, 746 -> 749.  With one column tile the two shapes are a wash.  Over an E4M3 cache: kFp8Pair.
+// 9 - 16 columns from several query tokens 68.1 -> 63.4 (lognormal_b64), 180.6 -> 175.8 (straggler_b8), 306 -> 290
+// (shift_b128), 746 -> 749 (longtail_mix_b256).  With one column tile the two shapes are a wash.  Over an E4M3 cache:
+// kFp8Pair.
 constexpr int kTwoSlotCtas = 2;
 // A block costs ~4 us of start-up and epilogue whatever its size and the default block is alone on its SM, so a batch
 // of short sequences leaves the SMs waiting most of the time.  When no unit of a host plan is longer than this many
@@ -107,11 +108,10 @@ const int kLoadsOnlySmem[2] = {libra::DecodeSmem<64, kLoadsOnlyWarps, kLoadsOnly
 // sequences and 5 % on the drifting workload: no clear winner, available through libra_set_variant.)  Batches of short
 // units get 4 x 2 or, up to kTinyUnitTokens, 2 x 4 (32 KB, seven blocks per SM: 1.4x / 1.9x / 2.6x / 3.5x faster than
 // 16 x 3 at 1024 / 512 / 256 / 128 tokens per sequence).  fn[loads only][NT - 1]
-// Two column tiles on a two-slot plan: two blocks of 6 x 4 per SM, as over bf16 pools (kVariantPair).  Same-run A/B
-// against 8 x 6 on a one-slot plan, 16 query heads per KV head: 50.2 -> 44.7 us (lognormal_b64), 124.7 -> 114.0
-// (straggler_b8), 225 -> 196 (shift_b128), 530 -> 512 (longtail_mix_b256); with two query tokens (8 query heads per KV
-// head) 39.7 -> 36.7, 133.3 -> 122.0, 239 -> 209, but 391 -> 452 on longtail_mix_b256, where 8 x 6 is already near the
-// gather ceiling: two slots are the default only for more than 8 query heads per KV head.
+// Two column tiles on a two-slot plan (the default for two tiles): two blocks of 6 x 4 per SM, as over bf16 pools
+// (kVariantPair).  Same-run A/B against 8 x 6 on a one-slot plan, us per step: 16 query heads per KV head 50.2 -> 44.7
+// (lognormal_b64), 124.7 -> 114.0 (straggler_b8), 225 -> 196 (shift_b128), 530 -> 512 (longtail_mix_b256); 16 columns
+// from several query tokens 56.4 -> 48.6, 132.2 -> 121.0, 220.7 -> 195.9, 542 -> 530.
 constexpr int kFp8OneTile = 2, kFp8TwoTiles = 1, kFp8ShortUnits = 5, kFp8TinyUnits = 6, kFp8Pair = 7;
 struct Fp8Variant {
   int warps, stages;
@@ -305,15 +305,14 @@ int encode_pool_map(libra_handle_t h, const void* base, CUtensorMap* map, int* p
   return LIBRA_OK;
 }
 
-// Two slots per SM are the planner's default where a step has two column tiles and the pools are bf16, or E4M3 with
-// more than 8 query heads per KV head (kVariantPair, kFp8Pair).
-bool wants_two_slots(const libra_handle_s* h, bool whatever_the_pools) {
-  return h->params_in.ctas_per_sm == 0 && h->group * h->max_q_len > 8 && (whatever_the_pools || !h->fp8 || h->group > 8);
+// Two slots per SM are the planner's default where a step has two column tiles (kVariantPair, kFp8Pair).
+bool wants_two_slots(const libra_handle_s* h) {
+  return h->params_in.ctas_per_sm == 0 && h->group * h->max_q_len > 8;
 }
 
 // The parameters in force for the handle's present state; true if they changed (a plan made before is then void).
 bool refresh_params(libra_handle_t h) {
-  const bool two = wants_two_slots(h, false);
+  const bool two = wants_two_slots(h);
   const libra::PlanParams now = resolve_params(h->params_in, h->n_sm_dev, two);
   const bool changed = now.ctas_per_sm != h->params.ctas_per_sm;
   h->params = now;
@@ -321,13 +320,11 @@ bool refresh_params(libra_handle_t h) {
   return changed;
 }
 
-// Workspace layout; the partial buffers hold max_q_len * num_q_heads rows per work item.  Sized for the larger of the
-// two defaults, so that switching the pools' type never asks for a larger workspace.
+// Workspace layout; the partial buffers hold max_q_len * num_q_heads rows per work item.
 void compute_layout(libra_handle_t h) {
   const libra_config_t* cfg = &h->cfg;
   const size_t rows = size_t(h->max_q_len) * cfg->num_q_heads;
-  h->max_items = libra::max_items(resolve_params(h->params_in, h->n_sm_dev, wants_two_slots(h, true)), cfg->num_kv_heads,
-                                  cfg->max_batch);
+  h->max_items = libra::max_items(h->params, cfg->num_kv_heads, cfg->max_batch);
   h->cnt_off = 256;  // the first 256 bytes hold the control words (the device error word)
   h->cnt_bytes = align_up(size_t(cfg->max_batch) * cfg->num_kv_heads * 4, 256);
   h->lse_off = h->cnt_off + h->cnt_bytes;
@@ -825,7 +822,6 @@ int libra_set_kv_dtype(libra_handle_t h, int32_t dtype, float k_scale, float v_s
     if (h->stride_page % 16 || h->stride_head % 16 || h->stride_token % 16) return LIBRA_INVALID_ARGUMENT;
   }
   h->fp8 = (dtype == LIBRA_KV_E4M3);
-  if (refresh_params(h)) h->planned = false;   // the planner's default slot count follows the pools' type: plan again
   h->fp8_variant = -1;
   h->k_scale = h->fp8 ? k_scale : 1.f;
   h->v_scale = h->fp8 ? v_scale : 1.f;

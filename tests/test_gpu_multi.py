@@ -235,8 +235,7 @@ def test_append_of_the_new_tokens_fused_in(lib, layout):
 
 def test_two_column_tiles_plan_for_two_slots_per_sm_by_default(lib):
     """More than 8 rows of q per KV head (16 query heads per KV head, or several query tokens): the planner's default
-    is two slots per SM over bf16 pools and the step runs two 6-warp blocks per SM; over an E4M3 cache only with more
-    than 8 query heads per KV head, and switching the type voids a plan made under the other default.  Outputs against the oracle under the default and under a forced one-slot
+    is two slots per SM and the step runs two 6-warp blocks per SM (bf16 and E4M3 pools alike).  Outputs against the oracle under the default and under a forced one-slot
     plan (the 12-warp block), on the same handle state a caller would have."""
     import torch
     dev = torch.device("cuda:0")
@@ -270,17 +269,8 @@ def test_two_column_tiles_plan_for_two_slots_per_sm_by_default(lib):
                 torch.cuda.synchronize()
                 assert h.debug_error_word() == 0
                 check(H.bf16_dev_to_f32(out1), ref1, f"Hq {Hq} Tq 1 of {Tq} slots {want}")
-            # over an 8-bit cache two slots are the default only for more than 8 query heads per KV head: the default
-            # follows the type, and a plan made under the other default is void
+            # the default does not depend on the pools' type, so the plan stays and the workspace fits
             h.set_kv_dtype(lib.KV_E4M3, 1.0, 1.0)
-            want8 = want if Hq // Hkv > 8 else 1
-            assert h.plan_params().ctas_per_sm == want8
-            if want8 != want:
-                with pytest.raises(lib.LibraError) as e:
-                    h.decode_attn_multi(qd.data_ptr(), Tq, kd.data_ptr(), vd.data_ptr(), btd.data_ptr(), dl.data_ptr(),
-                                        out.data_ptr(), st)
-                assert e.value.status == lib.NOT_PLANNED
-            assert h.workspace_size() <= ws.numel()
+            assert h.plan_params().ctas_per_sm == want and h.workspace_size() <= ws.numel()
             h.set_kv_dtype(lib.KV_BF16)
-            assert h.plan_params().ctas_per_sm == want
             h.close()
