@@ -77,7 +77,8 @@ typedef struct {
   int32_t n_sm;           /* SMs to plan for; 0 = the device's count (148 on B200)               */
   int32_t ctas_per_sm;    /* resident decode blocks per SM the plan assumes; default 1, and 2 where
                              a KV head serves more than 8 rows of q (query heads per KV head x
-                             libra_set_max_query_tokens): those steps run two blocks per SM      */
+                             libra_set_max_query_tokens) or the pools are E4M3: those steps run
+                             two blocks per SM                                                   */
   int32_t items_per_slot; /* target work units per resident block; default 1                    */
   int32_t chunk_align;    /* A: chunk lengths are multiples of this many tokens (itself a
                              multiple of 16); default 256                                       */
@@ -170,7 +171,8 @@ int libra_set_max_query_tokens(libra_handle_t handle, int32_t max_q_len);
  * Halving the bytes per cached token halves what the step has to read.  With E4M3 pools the rows given to
  * libra_decode_attn_append (k_new, v_new: [batch, num_kv_heads, head_dim]) and the dense buffers of
  * libra_kv_gather / libra_kv_scatter hold codes too, one byte per element; libra_decode_attn_host returns
- * UNSUPPORTED_SHAPE.  The plan and the workspace do not depend on the type. */
+ * UNSUPPORTED_SHAPE.  The workspace does not depend on the type; the plan does where the default of ctas_per_sm does
+ * (see libra_plan_params_t): there the call voids the plan (NOT_PLANNED until the next plan call). */
 #define LIBRA_KV_BF16 0
 #define LIBRA_KV_E4M3 1
 int libra_set_kv_dtype(libra_handle_t handle, int32_t dtype, float k_scale, float v_scale);
@@ -180,8 +182,8 @@ int libra_set_kv_dtype(libra_handle_t handle, int32_t dtype, float k_scale, floa
  * otherwise); the default is the tuned one (8 x 3; 4 x 2, three blocks per SM, when no unit of a host plan exceeds
  * 1024 tokens, and 2 x 2, seven per SM, when none exceeds 256; 6 x 2, two blocks per SM, when a KV head serves more than
  * 8 rows of q and the plan has two slots per SM (the default then), 12 x 2 on a one-slot plan; with an E4M3 cache,
- * whose tiles are half the size, 16 x 3, 8 x 6 for two column tiles (6 x 4, two per SM, on a two-slot plan), 4 x 2 / 2 x 4
- * for short units).  Results do not depend on the stage count; the warp
+ * whose tiles are half the size, 8 x 3 / 6 x 4 for one / two column tiles, two blocks per SM, on a two-slot plan (the
+ * default), 16 x 3 / 8 x 6 on a one-slot plan, 4 x 2 / 2 x 4 for short units).  Results do not depend on the stage count; the warp
  * count changes the order of the per-unit merge and hence the last bits of the result. */
 int libra_set_variant(libra_handle_t handle, int32_t warps, int32_t stages);
 

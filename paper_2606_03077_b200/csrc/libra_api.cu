@@ -103,16 +103,19 @@ const int kLoadsOnlySmem[2] = {libra::DecodeSmem<64, kLoadsOnlyWarps, kLoadsOnly
 
 // 8-bit (E4M3) cache, head_dim 128: block shapes compiled in.  Half the bytes per tile leave half the time per tile,
 // and two warps per scheduler cannot hide the conversion -> mma -> softmax chain in it, so 16 warps per SM are wanted:
-// one block of 16 warps x 3 stages of 4 KB where the registers allow it (one column tile), 8 x 6 otherwise.  (Two blocks
-// of 8 x 3 per SM instead: 5 % faster on the long mix and 3 % on the headline workload, 2 % slower on 8 equal long
-// sequences and 5 % on the drifting workload: no clear winner, available through libra_set_variant.)  Batches of short
+// on a one-slot plan one block of 16 warps x 3 stages of 4 KB where the registers allow it (one column tile), 8 x 6
+// otherwise; on a two-slot plan, the default, two blocks per SM (kFp8OnePair, kFp8Pair below).  Batches of short
 // units get 4 x 2 or, up to kTinyUnitTokens, 2 x 4 (32 KB, seven blocks per SM: 1.4x / 1.9x / 2.6x / 3.5x faster than
 // 16 x 3 at 1024 / 512 / 256 / 128 tokens per sequence).  fn[loads only][NT - 1]
 // Two column tiles on a two-slot plan (the default for two tiles): two blocks of 6 x 4 per SM, as over bf16 pools
 // (kVariantPair).  Same-run A/B against 8 x 6 on a one-slot plan, us per step: 16 query heads per KV head 50.2 -> 44.7
 // (lognormal_b64), 124.7 -> 114.0 (straggler_b8), 225 -> 196 (shift_b128), 530 -> 512 (longtail_mix_b256); 16 columns
 // from several query tokens 56.4 -> 48.6, 132.2 -> 121.0, 220.7 -> 195.9, 542 -> 530.
-constexpr int kFp8OneTile = 2, kFp8TwoTiles = 1, kFp8ShortUnits = 5, kFp8TinyUnits = 6, kFp8Pair = 7;
+// One column tile on a two-slot plan (the default over E4M3 pools): two blocks of 8 x 3 per SM (the kernel's launch
+// bounds hold them at 128 registers; at 130 only one was resident and the arrangement lost 5 - 20 %) against one block
+// of 16 x 3 on a one-slot plan: 36.2 -> 31.5 us (lognormal_b64), 91.1 -> 91.1 (straggler_b8), 158.9 -> 142.0
+// (shift_b128), 393 -> 351 (longtail_mix_b256; best regions 346.9 -> 334.7).
+constexpr int kFp8OneTile = 2, kFp8TwoTiles = 1, kFp8ShortUnits = 5, kFp8TinyUnits = 6, kFp8Pair = 7, kFp8OnePair = 0;
 struct Fp8Variant {
   int warps, stages;
   DecodeKernelFn fn[2][2][2];      // [D == 128][loads only][NT - 1]
@@ -305,14 +308,15 @@ int encode_pool_map(libra_handle_t h, const void* base, CUtensorMap* map, int* p
   return LIBRA_OK;
 }
 
-// Two slots per SM are the planner's default where a step has two column tiles (kVariantPair, kFp8Pair).
-bool wants_two_slots(const libra_handle_s* h) {
-  return h->params_in.ctas_per_sm == 0 && h->group * h->max_q_len > 8;
+// Two slots per SM are the planner's default where a step has two column tiles (kVariantPair, kFp8Pair) and for every
+// step over E4M3 pools (kFp8OnePair).
+bool wants_two_slots(const libra_handle_s* h, bool whatever_the_pools) {
+  return h->params_in.ctas_per_sm == 0 && (h->group * h->max_q_len > 8 || h->fp8 || whatever_the_pools);
 }
 
 // The parameters in force for the handle's present state; true if they changed (a plan made before is then void).
 bool refresh_params(libra_handle_t h) {
-  const bool two = wants_two_slots(h);
+  const bool two = wants_two_slots(h, false);
   const libra::PlanParams now = resolve_params(h->params_in, h->n_sm_dev, two);
   const bool changed = now.ctas_per_sm != h->params.ctas_per_sm;
   h->params = now;
@@ -320,11 +324,13 @@ bool refresh_params(libra_handle_t h) {
   return changed;
 }
 
-// Workspace layout; the partial buffers hold max_q_len * num_q_heads rows per work item.
+// Workspace layout; the partial buffers hold max_q_len * num_q_heads rows per work item.  Sized for the larger of the
+// planner's two defaults, so that switching the pools' type never asks for a larger workspace.
 void compute_layout(libra_handle_t h) {
   const libra_config_t* cfg = &h->cfg;
   const size_t rows = size_t(h->max_q_len) * cfg->num_q_heads;
-  h->max_items = libra::max_items(h->params, cfg->num_kv_heads, cfg->max_batch);
+  h->max_items = libra::max_items(resolve_params(h->params_in, h->n_sm_dev, wants_two_slots(h, true)), cfg->num_kv_heads,
+                                  cfg->max_batch);
   h->cnt_off = 256;  // the first 256 bytes hold the control words (the device error word)
   h->cnt_bytes = align_up(size_t(cfg->max_batch) * cfg->num_kv_heads * 4, 256);
   h->lse_off = h->cnt_off + h->cnt_bytes;
@@ -822,6 +828,7 @@ int libra_set_kv_dtype(libra_handle_t h, int32_t dtype, float k_scale, float v_s
     if (h->stride_page % 16 || h->stride_head % 16 || h->stride_token % 16) return LIBRA_INVALID_ARGUMENT;
   }
   h->fp8 = (dtype == LIBRA_KV_E4M3);
+  if (refresh_params(h)) h->planned = false;   // the planner's default slot count follows the pools' type: plan again
   h->fp8_variant = -1;
   h->k_scale = h->fp8 ? k_scale : 1.f;
   h->v_scale = h->fp8 ? v_scale : 1.f;
@@ -1007,7 +1014,8 @@ int decode_impl(libra_handle_t h, const void* q, const void* k_new, const void* 
     lc.blockDim = dim3(unsigned((loads_only ? kLoadsOnlyWarps : v.warps) * 32));
     lc.dynamicSmemBytes = size_t(loads_only ? kLoadsOnlySmem[di] : v.smem[di][ni]);
     if (h->fp8) {
-      int fp8_auto = ni ? (h->params.ctas_per_sm >= kTwoSlotCtas ? kFp8Pair : kFp8TwoTiles) : kFp8OneTile;
+      const bool two_slots = h->params.ctas_per_sm >= kTwoSlotCtas;
+      int fp8_auto = ni ? (two_slots ? kFp8Pair : kFp8TwoTiles) : (two_slots ? kFp8OnePair : kFp8OneTile);
       if (!ni && !loads_only && auto_variant == kVariantShortUnits) fp8_auto = kFp8ShortUnits;
       if (!ni && !loads_only && auto_variant == kVariantTinyUnits) fp8_auto = kFp8TinyUnits;
       const Fp8Variant& fv = fp8_variants()[h->fp8_variant >= 0 ? h->fp8_variant : fp8_auto];

@@ -382,3 +382,37 @@ def test_head_dim_64_append_and_move(lib):
     assert np.array_equal(k_dense.cpu().numpy(), M.gather(k_ref, bt, lens_a, 1, 2))
     assert np.array_equal(v_dense.cpu().numpy(), M.gather(v_ref, bt, lens_a, 1, 2))
     h.close()
+
+
+def test_default_plan_has_two_slots_per_sm_and_switching_the_type_voids_the_plan(lib):
+    """Over E4M3 pools the planner's default is two slots per SM (the step runs two blocks per SM), over bf16 pools with
+    one column tile it is one: switching the type on a planned handle voids the plan, the workspace still fits, and the
+    step planned again is right under either default and under an explicit one-slot plan."""
+    import torch
+    dev = torch.device("cuda:0")
+    lens = [5000, 1300, 257, 16, 1, 0, 2048, 90]
+    lens_a, bt, q, k8, v8 = W.random_case_e4m3(660, len(lens), 32, 8, 128, lens)
+    ref, _ = O.paged_decode_attention_fp8(q, k8, v8, bt, lens_a, 0.5, 2.0)
+    st = torch.cuda.current_stream().cuda_stream
+    for plan, want8 in ((None, 2), (lib.PlanParams(0, 1, 0, 0, 0, 0), 1)):
+        h = lib.Handle(32, 8, 128, k8.shape[0], len(lens), bt.shape[1], plan=plan)
+        assert h.plan_params().ctas_per_sm == 1
+        ws = torch.empty(h.workspace_size(), dtype=torch.uint8, device=dev)
+        h.plan(lens_a, ws.data_ptr(), ws.numel(), st)
+        h.set_kv_dtype(lib.KV_E4M3, 0.5, 2.0)
+        assert h.plan_params().ctas_per_sm == want8 and h.workspace_size() <= ws.numel()
+        qd, btd = H.to_dev(q, dev), H.to_dev(bt, dev)
+        kd, vd = torch.from_numpy(k8).to(dev), torch.from_numpy(v8).to(dev)
+        dl = torch.from_numpy(lens_a.copy()).to(dev)
+        out = torch.full(q.shape, H.CANARY, dtype=torch.int16, device=dev)
+        args = (qd.data_ptr(), kd.data_ptr(), vd.data_ptr(), btd.data_ptr(), dl.data_ptr(), out.data_ptr(), st)
+        if want8 == 2:
+            with pytest.raises(lib.LibraError) as e:
+                h.decode_attn(*args)
+            assert e.value.status == lib.NOT_PLANNED
+            h.plan(lens_a, ws.data_ptr(), ws.numel(), st)
+        h.decode_attn(*args)
+        torch.cuda.synchronize()
+        assert h.debug_error_word() == 0
+        check(H.bf16_dev_to_f32(out), ref, f"E4M3, {want8} slot(s) per SM")
+        h.close()
