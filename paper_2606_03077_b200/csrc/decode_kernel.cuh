@@ -916,7 +916,9 @@ struct DecodeSmem {
 // kAppend: the full build - several query tokens per sequence and the fused append of the newest tokens' rows
 // (k_new / v_new).  The plain build knows q_len = 1 and has no append code, which makes its loop leaner.
 template <int D, int NT, int NW, int STAGES, bool kLoadsOnly = false, bool kFp8 = false, bool kAppend = false>
-__global__ void __launch_bounds__(NW * 32, (NW == 6 || (kFp8 && NW == 8 && STAGES == 3 && NT == 1)) ? 2 : 1)   // the 6-warp shape is meant to run two blocks per SM
+// Two shapes are meant to run two blocks per SM and are held to the registers that allows: 6 warps (two column tiles)
+// and, over an E4M3 cache, 8 warps x 3 stages with one column tile.
+__global__ void __launch_bounds__(NW * 32, (NW == 6 || (kFp8 && NW == 8 && STAGES == 3 && NT == 1)) ? 2 : 1)
 decode_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
               const __grid_constant__ DecodeParams p_in, const __grid_constant__ ParamPlan pp) {
   using namespace dev;
