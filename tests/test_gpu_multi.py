@@ -260,6 +260,13 @@ def test_two_column_tiles_plan_for_two_slots_per_sm_by_default(lib):
             torch.cuda.synchronize()
             assert h.debug_error_word() == 0
             check(H.bf16_dev_to_f32(out), ref, f"Hq {Hq} Tq {Tq} slots {want}")
+            # the same plan made on the device: the same bits
+            out_d = torch.full((B, Tq, Hq, d), H.CANARY, dtype=torch.int16, device=dev)
+            h.plan_device(dl.data_ptr(), B, ws.data_ptr(), ws.numel(), st)
+            h.decode_attn_multi(qd.data_ptr(), Tq, kd.data_ptr(), vd.data_ptr(), btd.data_ptr(), dl.data_ptr(), out_d.data_ptr(), st)
+            torch.cuda.synchronize()
+            assert h.debug_error_word() == 0 and torch.equal(out_d, out)
+            h.plan(lens_a, ws.data_ptr(), ws.numel(), st)
             if Tq > 1:   # one query token on the handle laid out for several: the same plan, one column tile
                 q1 = np.ascontiguousarray(q[:, :1])
                 ref1, _ = O.paged_multi_token_attention(q1, k, v, bt, lens_a)
