@@ -159,7 +159,8 @@ int libra_get_plan_params(libra_handle_t handle, libra_plan_params_t* out);
 /* Several query tokens per sequence (default 1).  Lays the workspace out for up to `max_q_len` query tokens
  * per sequence in libra_decode_attn_multi: the partial buffers grow by that factor, so ask
  * libra_workspace_size again afterwards; the current plan is dropped.  A KV head's score tile has at most
- * 16 columns: max_q_len * (num_q_heads / num_kv_heads) <= 16, else UNSUPPORTED_SHAPE. */
+ * 16 columns: max_q_len * (num_q_heads / num_kv_heads) <= 16, else UNSUPPORTED_SHAPE.  Past 8 columns the default of
+ * ctas_per_sm becomes 2 (see libra_plan_params_t; libra_get_plan_params shows what is in force). */
 int libra_set_max_query_tokens(libra_handle_t handle, int32_t max_q_len);
 
 /* Storage type of the KV pools (default LIBRA_KV_BF16).  LIBRA_KV_E4M3: the pools hold 8-bit floating-point
